@@ -1,0 +1,171 @@
+"""Python face of the CPU oracle (``nk_oracle.c``).
+
+TEST INFRASTRUCTURE ONLY.  Tests, the smoke check and the benchmark's CPU
+baseline leg may import this package; the product package never does, and this
+package never imports the product.  It compiles ``nk_oracle.c`` with gcc on
+first use and calls it through ctypes; the arithmetic lives in the C file.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+import subprocess
+
+import numpy as np
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+_SRC = os.path.join(_HERE, "nk_oracle.c")
+_LIB = os.path.join(_HERE, "libnk_oracle.so")
+
+F32, BF16 = 0, 1
+ROW, BLOCKED32 = 0, 1
+EPI_NONE, EPI_BIAS_RELU = 0, 1
+ACC_F64, ACC_F32_SEQ = 0, 1
+
+
+class Desc(ctypes.Structure):
+    _fields_ = [("M", ctypes.c_int64), ("N", ctypes.c_int64), ("K", ctypes.c_int64),
+                ("in_dtype", ctypes.c_int32), ("layout_a", ctypes.c_int32),
+                ("layout_b", ctypes.c_int32), ("epilogue", ctypes.c_int32),
+                ("acc_mode", ctypes.c_int32)]
+
+
+def build(force: bool = False) -> str:
+    """Compile the oracle's C file (plain gcc, -O2, no fast-math)."""
+    if force or not os.path.exists(_LIB) or os.path.getmtime(_LIB) < os.path.getmtime(_SRC):
+        tmp = _LIB + f".{os.getpid()}.tmp"
+        subprocess.check_call(["gcc", "-O2", "-std=c11", "-fPIC", "-shared", "-pthread",
+                               "-o", tmp, _SRC, "-lm"])
+        os.replace(tmp, _LIB)
+    return _LIB
+
+
+_lib = None
+
+
+def lib():
+    global _lib
+    if _lib is None:
+        L = ctypes.CDLL(build())
+        L.nko_bf16_to_f32.restype = ctypes.c_float
+        L.nko_bf16_to_f32.argtypes = [ctypes.c_uint16]
+        L.nko_f32_to_bf16_rne.restype = ctypes.c_uint16
+        L.nko_f32_to_bf16_rne.argtypes = [ctypes.c_float]
+        for f in (L.nko_pack_vnni2, L.nko_unpack_vnni2):
+            f.restype = None
+            f.argtypes = [ctypes.c_void_p, ctypes.c_int64, ctypes.c_int64, ctypes.c_void_p]
+        for f in (L.nko_a_index, L.nko_b_index):
+            f.restype = ctypes.c_int64
+            f.argtypes = [ctypes.POINTER(Desc), ctypes.c_int64, ctypes.c_int64]
+        L.nko_gemm.restype = ctypes.c_int
+        L.nko_gemm.argtypes = [ctypes.POINTER(Desc), ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p,
+                               ctypes.c_void_p, ctypes.c_int64, ctypes.c_void_p, ctypes.c_int64,
+                               ctypes.c_void_p, ctypes.c_void_p, ctypes.c_int]
+        _lib = L
+    return _lib
+
+
+def bf16_to_f32(bits: np.ndarray) -> np.ndarray:
+    """Decode uint16 BF16 patterns element by element through the C routine."""
+    L = lib()
+    flat = np.ascontiguousarray(bits, dtype=np.uint16).ravel()
+    out = np.fromiter((L.nko_bf16_to_f32(int(h)) for h in flat), dtype=np.float32, count=flat.size)
+    return out.reshape(np.shape(bits))
+
+
+def f32_to_bf16_rne(x: np.ndarray) -> np.ndarray:
+    L = lib()
+    flat = np.ascontiguousarray(x, dtype=np.float32).ravel()
+    out = np.fromiter((L.nko_f32_to_bf16_rne(float(v)) for v in flat), dtype=np.uint16, count=flat.size)
+    return out.reshape(np.shape(x))
+
+
+def pack_vnni2(flat: np.ndarray) -> np.ndarray:
+    """[K][N] uint16 -> [K/2][N][2] (Figure 1)."""
+    flat = np.ascontiguousarray(flat, dtype=np.uint16)
+    K, N = flat.shape
+    assert K % 2 == 0
+    out = np.empty((K // 2, N, 2), dtype=np.uint16)
+    lib().nko_pack_vnni2(flat.ctypes.data, K, N, out.ctypes.data)
+    return out
+
+
+def unpack_vnni2(packed: np.ndarray) -> np.ndarray:
+    packed = np.ascontiguousarray(packed, dtype=np.uint16)
+    K2, N, two = packed.shape
+    assert two == 2
+    out = np.empty((K2 * 2, N), dtype=np.uint16)
+    lib().nko_unpack_vnni2(packed.ctypes.data, K2 * 2, N, out.ctypes.data)
+    return out
+
+
+def _np_dtype(in_dtype):
+    return np.float32 if in_dtype == F32 else np.uint16
+
+
+def to_blocked(flat_a: np.ndarray, flat_b: np.ndarray, in_dtype: int):
+    """Scatter row-major A[M][K], B[K][N] into the blocked storage order using the
+    oracle's own index functions (slow Python loop over rows; test sizes only)."""
+    M, K = flat_a.shape
+    K2, N = flat_b.shape
+    assert K == K2
+    d = Desc(M, N, K, in_dtype, BLOCKED32, BLOCKED32, EPI_NONE, ACC_F64)
+    L = lib()
+    A = np.empty(M * K, dtype=flat_a.dtype)
+    B = np.empty(K * N, dtype=flat_b.dtype)
+    for i in range(M):
+        for k in range(K):
+            A[L.nko_a_index(ctypes.byref(d), i, k)] = flat_a[i, k]
+    for k in range(K):
+        for j in range(N):
+            B[L.nko_b_index(ctypes.byref(d), k, j)] = flat_b[k, j]
+    return A, B
+
+
+def gemm(M, N, K, A, B, bias=None, *, in_dtype=F32, layout_a=ROW, layout_b=ROW,
+         epilogue=EPI_NONE, rows=None, cols=None, acc_mode=ACC_F64, nthreads=None,
+         want_scale=True):
+    """Run the oracle.  A, B, bias are 1-D (or any-shape, C-contiguous) storage
+    buffers: float32, or uint16 BF16 bit patterns.  Returns (Y, S) as float64
+    arrays of shape [len(rows) or M][len(cols) or N]; S is None when
+    ``want_scale`` is False."""
+    dt = _np_dtype(in_dtype)
+    A = np.ascontiguousarray(A, dtype=dt)
+    B = np.ascontiguousarray(B, dtype=dt)
+    assert A.size == M * K and B.size == K * N, "operand size mismatch"
+    bp = None
+    if bias is not None:
+        bias = np.ascontiguousarray(bias, dtype=dt)
+        assert bias.size == N
+        bp = bias.ctypes.data
+    rp, nrows = None, M
+    if rows is not None:
+        rows = np.ascontiguousarray(rows, dtype=np.int64)
+        assert rows.min() >= 0 and rows.max() < M
+        rp, nrows = rows.ctypes.data, rows.size
+    cp, ncols = None, N
+    if cols is not None:
+        cols = np.ascontiguousarray(cols, dtype=np.int64)
+        assert cols.min() >= 0 and cols.max() < N
+        cp, ncols = cols.ctypes.data, cols.size
+    Y = np.empty((nrows, ncols), dtype=np.float64)
+    S = np.empty((nrows, ncols), dtype=np.float64) if want_scale else None
+    d = Desc(M, N, K, in_dtype, layout_a, layout_b, epilogue, acc_mode)
+    if nthreads is None:
+        nthreads = os.cpu_count() or 1
+    rc = lib().nko_gemm(ctypes.byref(d), A.ctypes.data, B.ctypes.data, bp, rp, nrows, cp, ncols,
+                        Y.ctypes.data, S.ctypes.data if S is not None else None, int(nthreads))
+    if rc != 0:
+        raise ValueError("oracle rejected the arguments")
+    return Y, S
+
+
+def gemm_workload(w, A, B, bias, rows=None, cols=None, **kw):
+    """Oracle on an ``nk_inputs.Workload``-shaped object (duck-typed: M, N, K,
+    in_dtype, layout, epilogue attributes)."""
+    lay = BLOCKED32 if w.layout == "blocked32" else ROW
+    return gemm(w.M, w.N, w.K, A, B, bias,
+                in_dtype=F32 if w.in_dtype == "f32" else BF16,
+                layout_a=lay, layout_b=lay,
+                epilogue=EPI_BIAS_RELU if w.epilogue == "bias_relu" else EPI_NONE,
+                rows=rows, cols=cols, **kw)

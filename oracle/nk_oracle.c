@@ -1,0 +1,175 @@
+/*
+ * CPU oracle for the dense GEMM path.  TEST INFRASTRUCTURE ONLY: nothing on the
+ * product path may call, link or import this file; it shares no code, header,
+ * table or constant with the CUDA library.
+ *
+ * What it computes is the plain definition the method reaches up to summation
+ * order (Algorithm 1: C = beta*C + sum_i A_i x B_i, taken with beta = 0):
+ *
+ *     C[i][j] = sum_{k=0}^{K-1} a(i,k) * b(k,j)       accumulated in FP64, k ascending
+ *     y[i][j] = C[i][j]                               (no epilogue)
+ *     y[i][j] = max(C[i][j] + bias[j], 0)             (bias + ReLU fused before the store,
+ *                                                      Section 6 "MLP")
+ *     S[i][j] = sum_k |a(i,k) * b(k,j)| (+ |bias[j]|) (scale of the error bound)
+ *
+ * a, b are the stored operand values: FP32, or BF16 widened exactly to FP32 (the
+ * appendix kernels' scalar body: extf, extf, mulf, addf).  y is returned
+ * unrounded, as double; a BF16-storing implementation rounds once afterwards.
+ *
+ * Layouts: row-major A[M][K], B[K][N]; or 32x32-blocked with the VNNI-2
+ * interleave of Figure 1 inside each B block:
+ *     A_blk[M/32][K/32][32][32]         (m-block, k-block, m-in-block, k-in-block)
+ *     B_blk[N/32][K/32][16][32][2]      (n-block, k-block, k-pair, n-in-block, k-parity)
+ *
+ * Pins (tests/test_oracle_*.py): Figure 1's printed packing, identity /
+ * permutation / diagonal / rank-1 / all-ones closed forms, brute force in a
+ * different loop order, numpy float64 matmul on small shapes, blocked-vs-flat
+ * bit equality, epilogue closed forms, exhaustive BF16 codec round trip.
+ */
+#include <math.h>
+#include <pthread.h>
+#include <stdint.h>
+#include <stdlib.h>
+#include <string.h>
+
+enum { NKO_F32 = 0, NKO_BF16 = 1 };
+enum { NKO_ROW = 0, NKO_BLOCKED32 = 1 };
+enum { NKO_EPI_NONE = 0, NKO_EPI_BIAS_RELU = 1 };
+enum { NKO_ACC_F64 = 0, NKO_ACC_F32_SEQ = 1 };
+
+typedef struct {
+    int64_t M, N, K;
+    int32_t in_dtype;   /* NKO_F32 | NKO_BF16: element type of A, B and bias */
+    int32_t layout_a;   /* NKO_ROW | NKO_BLOCKED32 */
+    int32_t layout_b;
+    int32_t epilogue;
+    int32_t acc_mode;   /* NKO_ACC_F64 (the oracle) | NKO_ACC_F32_SEQ (tolerance sanity only) */
+} nko_desc_t;
+
+/* BF16 -> FP32 is a 16-bit left shift of the bit pattern (Algorithm 2, fallback branch). */
+float nko_bf16_to_f32(uint16_t h) {
+    uint32_t u = (uint32_t)h << 16;
+    float f;
+    memcpy(&f, &u, 4);
+    return f;
+}
+
+/* FP32 -> BF16, round to nearest, ties to even (finite inputs). */
+uint16_t nko_f32_to_bf16_rne(float f) {
+    uint32_t u;
+    memcpy(&u, &f, 4);
+    uint32_t keep = u >> 16, rest = u & 0xFFFFu;
+    if (rest > 0x8000u || (rest == 0x8000u && (keep & 1u))) keep += 1;
+    return (uint16_t)keep;
+}
+
+/* Figure 1: packed[k/2][n][k%2] = flat[k][n]; K even. */
+void nko_pack_vnni2(const uint16_t* flat, int64_t K, int64_t N, uint16_t* packed) {
+    for (int64_t k = 0; k < K; ++k)
+        for (int64_t n = 0; n < N; ++n)
+            packed[((k / 2) * N + n) * 2 + (k % 2)] = flat[k * N + n];
+}
+
+void nko_unpack_vnni2(const uint16_t* packed, int64_t K, int64_t N, uint16_t* flat) {
+    for (int64_t k = 0; k < K; ++k)
+        for (int64_t n = 0; n < N; ++n)
+            flat[k * N + n] = packed[((k / 2) * N + n) * 2 + (k % 2)];
+}
+
+static int64_t a_index(const nko_desc_t* d, int64_t i, int64_t k) {
+    if (d->layout_a == NKO_ROW) return i * d->K + k;
+    return (((i / 32) * (d->K / 32) + k / 32) * 32 + i % 32) * 32 + k % 32;
+}
+
+static int64_t b_index(const nko_desc_t* d, int64_t k, int64_t j) {
+    if (d->layout_b == NKO_ROW) return k * d->N + j;
+    return ((((j / 32) * (d->K / 32) + k / 32) * 16 + (k % 32) / 2) * 32 + j % 32) * 2 + k % 2;
+}
+
+/* Storage index of logical element (i,k) of A / (k,j) of B: exported so tests can pack. */
+int64_t nko_a_index(const nko_desc_t* d, int64_t i, int64_t k) { return a_index(d, i, k); }
+int64_t nko_b_index(const nko_desc_t* d, int64_t k, int64_t j) { return b_index(d, k, j); }
+
+static double load(const void* p, int32_t dtype, int64_t idx) {
+    if (dtype == NKO_F32) return (double)((const float*)p)[idx];
+    return (double)nko_bf16_to_f32(((const uint16_t*)p)[idx]);
+}
+
+typedef struct {
+    const nko_desc_t* d;
+    const void *A, *B, *bias;
+    const int64_t *rows, *cols;
+    int64_t r0, r1, ncols;
+    double *Y, *S;
+} job_t;
+
+static void* worker(void* arg) {
+    job_t* w = (job_t*)arg;
+    const nko_desc_t* d = w->d;
+    int64_t nc = w->ncols;
+    float* accf = NULL;
+    if (d->acc_mode == NKO_ACC_F32_SEQ) accf = (float*)malloc(sizeof(float) * (size_t)nc);
+    for (int64_t r = w->r0; r < w->r1; ++r) {
+        int64_t i = w->rows ? w->rows[r] : r;
+        double* y = w->Y + r * nc;
+        double* s = w->S ? w->S + r * nc : NULL;
+        for (int64_t c = 0; c < nc; ++c) y[c] = 0.0;
+        if (s) for (int64_t c = 0; c < nc; ++c) s[c] = 0.0;
+        if (accf) for (int64_t c = 0; c < nc; ++c) accf[c] = 0.0f;
+        /* k outermost of the two inner loops: every y[c] still receives its
+           products in ascending k, exactly as the definition's sum is written. */
+        for (int64_t k = 0; k < d->K; ++k) {
+            double a = load(w->A, d->in_dtype, a_index(d, i, k));
+            for (int64_t c = 0; c < nc; ++c) {
+                int64_t j = w->cols ? w->cols[c] : c;
+                double p = a * load(w->B, d->in_dtype, b_index(d, k, j));
+                if (accf) accf[c] = accf[c] + (float)p; else y[c] += p;
+                if (s) s[c] += fabs(p);
+            }
+        }
+        if (accf) for (int64_t c = 0; c < nc; ++c) y[c] = (double)accf[c];
+        if (d->epilogue == NKO_EPI_BIAS_RELU) {
+            for (int64_t c = 0; c < nc; ++c) {
+                int64_t j = w->cols ? w->cols[c] : c;
+                double b = load(w->bias, d->in_dtype, j);
+                double v = y[c] + b;
+                y[c] = v > 0.0 ? v : 0.0;
+                if (s) s[c] += fabs(b);
+            }
+        }
+    }
+    free(accf);
+    return NULL;
+}
+
+/*
+ * rows: list of nrows row indices, or NULL for rows 0..nrows-1.
+ * cols: list of ncols column indices, or NULL for columns 0..ncols-1.
+ * Y, S: [nrows][ncols] doubles (S may be NULL).  Threads split the row list
+ * statically; the result does not depend on nthreads.  Returns 0, or -1 on
+ * invalid arguments.
+ */
+int nko_gemm(const nko_desc_t* d, const void* A, const void* B, const void* bias,
+             const int64_t* rows, int64_t nrows, const int64_t* cols, int64_t ncols,
+             double* Y, double* S, int nthreads) {
+    if (!d || !A || !B || !Y || d->M <= 0 || d->N <= 0 || d->K <= 0) return -1;
+    if (d->epilogue == NKO_EPI_BIAS_RELU && !bias) return -1;
+    if (d->layout_a == NKO_BLOCKED32 && (d->M % 32 || d->K % 32)) return -1;
+    if (d->layout_b == NKO_BLOCKED32 && (d->N % 32 || d->K % 32)) return -1;
+    if (nrows <= 0 || ncols <= 0) return -1;
+    if (nthreads < 1) nthreads = 1;
+    if (nthreads > nrows) nthreads = (int)nrows;
+    pthread_t* th = (pthread_t*)malloc(sizeof(pthread_t) * (size_t)nthreads);
+    job_t* jobs = (job_t*)malloc(sizeof(job_t) * (size_t)nthreads);
+    for (int t = 0; t < nthreads; ++t) {
+        job_t j = { d, A, B, bias, rows, cols, nrows * t / nthreads, nrows * (t + 1) / nthreads,
+                    ncols, Y, S };
+        jobs[t] = j;
+        if (t > 0) pthread_create(&th[t], NULL, worker, &jobs[t]);
+    }
+    worker(&jobs[0]);
+    for (int t = 1; t < nthreads; ++t) pthread_join(th[t], NULL);
+    free(th);
+    free(jobs);
+    return 0;
+}

@@ -1,0 +1,334 @@
+"""Pins for the CPU oracle: values the paper prints, closed forms, invariants,
+brute force in a different loop order, and a library routine on small shapes.
+Each is chosen so that a plausible slip in the oracle (dropped term, wrong
+index, transposed operand, wrong pair order, missing bias) fails at least one.
+"""
+import os
+
+import numpy as np
+import pytest
+
+import oracle
+from oracle import F32, BF16, ROW, BLOCKED32, EPI_NONE, EPI_BIAS_RELU
+import nk_inputs
+
+GOLD = os.path.join(os.path.dirname(__file__), "golden")
+
+
+def _bits(x):
+    """float array (values exactly representable in BF16) -> uint16 patterns."""
+    u = np.ascontiguousarray(x, dtype=np.float32).view(np.uint32)
+    assert np.all((u & 0xFFFF) == 0), "test value is not a BF16 number"
+    return (u >> 16).astype(np.uint16)
+
+
+# ---------------------------------------------------------------- layouts
+def test_fig1_vnni2_printed_values():
+    flat, packed = [], []
+    for line in open(os.path.join(GOLD, "fig1_vnni2.txt")):
+        t = line.split()
+        if t and t[0] == "flat":
+            flat.append([int(v) for v in t[1:]])
+        elif t and t[0] == "packed":
+            packed.append([int(v) for v in t[1:]])
+    flat = np.array(flat, dtype=np.uint16)
+    want = np.array(packed, dtype=np.uint16).reshape(2, 4, 2)
+    got = oracle.pack_vnni2(flat)
+    assert got.shape == (2, 4, 2)
+    assert np.array_equal(got, want)
+    assert np.array_equal(oracle.unpack_vnni2(got), flat)
+
+
+def test_vnni2_round_trip_random():
+    rng = np.random.default_rng(1)
+    x = rng.integers(0, 65536, size=(34, 19), dtype=np.uint16)
+    assert np.array_equal(oracle.unpack_vnni2(oracle.pack_vnni2(x)), x)
+
+
+def test_blocked_b_block_is_fig1_packing_of_the_flat_block():
+    """Inside one 32x32 block the blocked-B storage is exactly Figure 1's
+    packing of that block; blocks are ordered (n-block, k-block)."""
+    K, N = 64, 96
+    flat_b = np.arange(K * N, dtype=np.float32).reshape(K, N)
+    flat_a = np.zeros((32, K), dtype=np.float32)
+    _, Bblk = oracle.to_blocked(flat_a, flat_b, F32)
+    Bblk = Bblk.reshape(N // 32, K // 32, 16, 32, 2)
+    for nb in range(N // 32):
+        for kb in range(K // 32):
+            blk = flat_b[kb * 32:(kb + 1) * 32, nb * 32:(nb + 1) * 32]
+            want = oracle.pack_vnni2(blk.astype(np.uint16))          # values < 65536
+            assert np.array_equal(Bblk[nb, kb].astype(np.uint16), want)
+
+
+def test_blocked_a_is_block_row_major():
+    M, K = 64, 96
+    flat_a = np.arange(M * K, dtype=np.float32).reshape(M, K)
+    Ablk, _ = oracle.to_blocked(flat_a, np.zeros((K, 32), np.float32), F32)
+    Ablk = Ablk.reshape(M // 32, K // 32, 32, 32)
+    for mb in range(M // 32):
+        for kb in range(K // 32):
+            assert np.array_equal(Ablk[mb, kb], flat_a[mb * 32:(mb + 1) * 32, kb * 32:(kb + 1) * 32])
+
+
+# ---------------------------------------------------------------- bf16 codec
+def test_bf16_decode_encode_exhaustive():
+    bits = np.arange(65536, dtype=np.uint16)
+    exp = (bits >> 7) & 0xFF
+    finite = bits[exp != 0xFF]
+    f = oracle.bf16_to_f32(finite)
+    # decode agrees with the IEEE reading: sign, 8-bit exponent, 7-bit mantissa
+    sign = np.where(finite >> 15, -1.0, 1.0)
+    e = ((finite >> 7) & 0xFF).astype(np.int64)
+    m = (finite & 0x7F).astype(np.float64)
+    want = np.where(e == 0, sign * m * 2.0 ** -133, sign * (1 + m / 128) * 2.0 ** (e - 127))
+    assert np.array_equal(f.astype(np.float64), want)
+    assert np.array_equal(oracle.f32_to_bf16_rne(f), finite)
+
+
+def test_bf16_rne_ties():
+    one = np.float32(1.0)
+    cases = [
+        (1 + 2.0 ** -8, 1.0),                    # tie, even mantissa -> down
+        (1 + 3 * 2.0 ** -8, 1 + 2.0 ** -6),      # tie, odd mantissa -> up
+        (1 + 2.0 ** -8 + 2.0 ** -20, 1 + 2.0 ** -7),   # above tie -> up
+        (1 + 2.0 ** -8 - 2.0 ** -20, 1.0),       # below tie -> down
+        (-(1 + 3 * 2.0 ** -8), -(1 + 2.0 ** -6)),
+        (0.0, 0.0),
+    ]
+    x = np.array([c[0] for c in cases], dtype=np.float32)
+    got = oracle.bf16_to_f32(oracle.f32_to_bf16_rne(x))
+    assert np.array_equal(got, np.array([c[1] for c in cases], dtype=np.float32))
+    assert one == 1.0
+
+
+def test_input_generator_rounding_matches_oracle_codec():
+    v = nk_inputs.fill(3, 0, 5000, "uniform", dtype="f32")
+    assert np.array_equal(nk_inputs.f32_to_bf16_bits(v), oracle.f32_to_bf16_rne(v))
+
+
+# ---------------------------------------------------------------- GEMM core
+def _rand_int(shape, seed):
+    return np.random.default_rng(seed).integers(-4, 5, size=shape).astype(np.float32)
+
+
+def test_identity_permutation_diagonal():
+    M = K = N = 37
+    A = _rand_int((M, K), 2) + np.float32(0.5)
+    Y, _ = oracle.gemm(M, N, K, A, np.eye(K, dtype=np.float32))
+    assert np.array_equal(Y, A.astype(np.float64))
+    perm = np.random.default_rng(3).permutation(K)
+    P = np.zeros((K, N), dtype=np.float32)
+    P[perm, np.arange(N)] = 1.0                       # (A.P)[:, j] = A[:, perm[j]]
+    Y, _ = oracle.gemm(M, N, K, A, P)
+    assert np.array_equal(Y, A[:, perm].astype(np.float64))
+    Y, _ = oracle.gemm(M, N, K, P, A)                  # (P.A)[i, :] = A[inv[i], :]
+    inv = np.argsort(perm)
+    assert np.array_equal(Y, A[inv, :].astype(np.float64))
+    dvec = (2.0 ** np.random.default_rng(4).integers(-3, 4, size=K)).astype(np.float32)
+    Y, _ = oracle.gemm(M, N, K, A, np.diag(dvec))
+    assert np.array_equal(Y, (A * dvec[None, :]).astype(np.float64))
+
+
+def test_rank1_and_all_ones_closed_forms():
+    M, N, K = 9, 13, 50
+    u = np.arange(-4, 5, dtype=np.float32)
+    v = np.arange(-6, 7, dtype=np.float32)
+    # K = 1: C = u v^T
+    Y, S = oracle.gemm(M, N, 1, u.reshape(M, 1), v.reshape(1, N))
+    assert np.array_equal(Y, np.outer(u, v).astype(np.float64))
+    assert np.array_equal(S, np.abs(np.outer(u, v)).astype(np.float64))
+    # A[i][k] = u_i, B[k][j] = v_j for every k: C = K u v^T
+    A = np.repeat(u.reshape(M, 1), K, axis=1)
+    B = np.repeat(v.reshape(1, N), K, axis=0)
+    Y, S = oracle.gemm(M, N, K, A, B)
+    assert np.array_equal(Y, K * np.outer(u, v).astype(np.float64))
+    assert np.array_equal(S, K * np.abs(np.outer(u, v)).astype(np.float64))
+    Y, _ = oracle.gemm(5, 7, K, np.ones((5, K), np.float32), np.ones((K, 7), np.float32))
+    assert np.all(Y == K)
+
+
+def test_non_square_operand_roles():
+    """A is M x K and B is K x N: a transposed or swapped operand changes this result."""
+    M, N, K = 3, 5, 7
+    A = _rand_int((M, K), 10)
+    B = _rand_int((K, N), 11)
+    Y, _ = oracle.gemm(M, N, K, A, B)
+    want = np.zeros((M, N))
+    for j in range(N):                 # j-k-i order: different from the oracle's
+        for k in range(K):
+            for i in range(M):
+                want[i, j] += float(A[i, k]) * float(B[k, j])
+    assert np.array_equal(Y, want)
+
+
+def _shapes():
+    for line in open(os.path.join(GOLD, "shapes.txt")):
+        if line.startswith("#") or not line.strip():
+            continue
+        name, batch, M, N, K, dt, lay = line.split()
+        yield name, int(batch), int(M), int(N), int(K), dt, lay
+
+
+@pytest.mark.parametrize("case", list(_shapes()), ids=lambda c: c[0])
+def test_paper_example_shapes_brute_force(case):
+    """Batch-reduce over the paper's example shapes: sum_i A_i.B_i equals one GEMM
+    whose K axis is the concatenation of the batch (Algorithm 1's output line)."""
+    name, batch, M, N, K, dt, lay = case
+    As = [_rand_int((M, K), 100 + i) for i in range(batch)]
+    Bs = [_rand_int((K, N), 200 + i) for i in range(batch)]
+    want = np.zeros((M, N))
+    for i in range(batch):
+        for m in range(M):
+            for n in range(N):
+                want[m, n] += float(np.dot(As[i][m, :].astype(np.float64), Bs[i][:, n].astype(np.float64)))
+    Acat = np.concatenate(As, axis=1)
+    Bcat = np.concatenate(Bs, axis=0)
+    if dt == "bf16":
+        Y, _ = oracle.gemm(M, N, batch * K, _bits(Acat), _bits(Bcat), in_dtype=BF16)
+    else:
+        Y, _ = oracle.gemm(M, N, batch * K, Acat, Bcat)
+    assert np.array_equal(Y, want)
+    if lay == "vnni" and M % 32 == 0 and N % 32 == 0:
+        Ab, Bb = oracle.to_blocked(_bits(Acat), _bits(Bcat), BF16)
+        Yb, _ = oracle.gemm(M, N, batch * K, Ab, Bb, in_dtype=BF16, layout_a=BLOCKED32, layout_b=BLOCKED32)
+        assert np.array_equal(Yb, want)
+
+
+def test_numpy_float64_matmul_small():
+    M, N, K = 96, 80, 128
+    w = nk_inputs.Workload("t", M, N, K, "f32", "f32", seed=5)
+    A, B, _ = w.make()
+    Y, S = oracle.gemm_workload(w, A, B, None)
+    ref = A.reshape(M, K).astype(np.float64) @ B.reshape(K, N).astype(np.float64)
+    sref = np.abs(A.reshape(M, K)).astype(np.float64) @ np.abs(B.reshape(K, N)).astype(np.float64)
+    assert np.max(np.abs(Y - ref)) <= 1e-13 * sref.max()
+    assert np.max(np.abs(S - sref)) <= 1e-13 * sref.max()
+
+
+def test_bf16_inputs_decoded_exactly():
+    M, N, K = 33, 40, 64
+    w = nk_inputs.Workload("t", M, N, K, "bf16", "f32", seed=6)
+    A, B, _ = w.make()
+    Y, _ = oracle.gemm_workload(w, A, B, None)
+    Af = (A.astype(np.uint32) << 16).view(np.float32).reshape(M, K).astype(np.float64)
+    Bf = (B.astype(np.uint32) << 16).view(np.float32).reshape(K, N).astype(np.float64)
+    assert np.max(np.abs(Y - Af @ Bf)) <= 1e-13 * (np.abs(Af) @ np.abs(Bf)).max()
+
+
+def test_blocked_equals_flat_bit_for_bit():
+    M, N, K = 64, 96, 128
+    w = nk_inputs.Workload("t", M, N, K, "bf16", "f32", seed=7)
+    A, B, _ = w.make()
+    Yf, Sf = oracle.gemm(M, N, K, A, B, in_dtype=BF16)
+    Ab, Bb = oracle.to_blocked(A.reshape(M, K), B.reshape(K, N), BF16)
+    Yb, Sb = oracle.gemm(M, N, K, Ab, Bb, in_dtype=BF16, layout_a=BLOCKED32, layout_b=BLOCKED32)
+    assert np.array_equal(Yf, Yb) and np.array_equal(Sf, Sb)
+    # mixed: only B blocked
+    Ym, _ = oracle.gemm(M, N, K, A, Bb, in_dtype=BF16, layout_a=ROW, layout_b=BLOCKED32)
+    assert np.array_equal(Yf, Ym)
+
+
+def test_transpose_invariant():
+    M, N, K = 17, 23, 31
+    A = nk_inputs.fill(8, 0, M * K).reshape(M, K)
+    B = nk_inputs.fill(8, 1, K * N).reshape(K, N)
+    Y, _ = oracle.gemm(M, N, K, A, B)
+    Yt, _ = oracle.gemm(N, M, K, np.ascontiguousarray(B.T), np.ascontiguousarray(A.T))
+    assert np.array_equal(Y, Yt.T)     # same products, same k order
+
+
+def test_row_and_column_subsets_and_thread_independence():
+    M, N, K = 50, 60, 70
+    A = nk_inputs.fill(9, 0, M * K)
+    B = nk_inputs.fill(9, 1, K * N)
+    Y, S = oracle.gemm(M, N, K, A, B, nthreads=1)
+    Y8, S8 = oracle.gemm(M, N, K, A, B, nthreads=7)
+    assert np.array_equal(Y, Y8) and np.array_equal(S, S8)
+    rows = np.array([49, 0, 17], dtype=np.int64)
+    cols = np.array([3, 59, 4, 30], dtype=np.int64)
+    Ys, Ss = oracle.gemm(M, N, K, A, B, rows=rows, cols=cols)
+    assert np.array_equal(Ys, Y[np.ix_(rows, cols)])
+    assert np.array_equal(Ss, S[np.ix_(rows, cols)])
+
+
+# ---------------------------------------------------------------- epilogue
+def test_epilogue_closed_forms():
+    M, N, K = 12, 20, 16
+    A = _rand_int((M, K), 20)
+    B = _rand_int((K, N), 21)
+    C = A.astype(np.float64) @ B.astype(np.float64)
+    big = np.full(N, 1024.0, dtype=np.float32)
+    Y, S = oracle.gemm(M, N, K, A, B, big, epilogue=EPI_BIAS_RELU)
+    assert np.array_equal(Y, C + 1024.0)              # ReLU inactive: GEMM + bias
+    _, S0 = oracle.gemm(M, N, K, A, B)
+    assert np.array_equal(S, S0 + 1024.0)             # |bias| enters the scale
+    Y, _ = oracle.gemm(M, N, K, A, B, -big, epilogue=EPI_BIAS_RELU)
+    assert np.all(Y == 0.0)                           # everything clipped
+    # per-column bias: column j shifted by j - 8, clipped at zero
+    bias = (np.arange(N) - 8).astype(np.float32)
+    Y, _ = oracle.gemm(M, N, K, A, B, bias, epilogue=EPI_BIAS_RELU)
+    assert np.array_equal(Y, np.maximum(C + bias[None, :].astype(np.float64), 0.0))
+    # bias = -(row of A.B) on a one-row problem: exactly zero
+    Y, _ = oracle.gemm(1, N, K, A[:1], B, (-C[0]).astype(np.float32), epilogue=EPI_BIAS_RELU)
+    assert np.all(Y == 0.0)
+    with pytest.raises(ValueError):
+        oracle.gemm(M, N, K, A, B, None, epilogue=EPI_BIAS_RELU)
+
+
+def test_bf16_bias_decoded():
+    M, N, K = 4, 8, 8
+    A = _bits(_rand_int((M, K), 30))
+    B = _bits(_rand_int((K, N), 31))
+    bias = _bits(np.full(N, 0.5, dtype=np.float32))
+    Y, _ = oracle.gemm(M, N, K, A, B, bias, in_dtype=BF16, epilogue=EPI_BIAS_RELU)
+    Y0, _ = oracle.gemm(M, N, K, A, B, in_dtype=BF16)
+    assert np.array_equal(Y, np.maximum(Y0 + 0.5, 0.0))
+
+
+# ---------------------------------------------------------------- tolerance sanity
+def test_fp32_sequential_accumulation_meets_the_bar():
+    """The acceptance bar (1e-5 x max sum|a.b|) is reachable by FP32 accumulation:
+    the oracle's own FP32-sequential mode passes it at K = 16384."""
+    M, N, K = 4, 64, 16384
+    w = nk_inputs.Workload("t", M, N, K, "bf16", "f32", seed=11)
+    A, B, _ = w.make()
+    Y, S = oracle.gemm_workload(w, A, B, None)
+    Y32, _ = oracle.gemm_workload(w, A, B, None, acc_mode=oracle.ACC_F32_SEQ)
+    err = np.max(np.abs(Y - Y32)) / S.max()
+    assert 0 < err <= 1e-5
+
+
+def test_planted_mistakes_are_caught():
+    """A wrong VNNI pair order or a dropped k term changes results the pins fix."""
+    flat = np.arange(16, dtype=np.uint16).reshape(4, 4)
+    good = oracle.pack_vnni2(flat)
+    swapped = good[:, :, ::-1]
+    assert not np.array_equal(swapped, good)
+    M, N, K = 4, 4, 8
+    A = _rand_int((M, K), 40) + 1
+    B = _rand_int((K, N), 41) + 1
+    Y, _ = oracle.gemm(M, N, K, A, B)
+    Ydrop, _ = oracle.gemm(M, N, K - 1, np.ascontiguousarray(A[:, :-1]), np.ascontiguousarray(B[:-1]))
+    assert not np.array_equal(Y, Ydrop)
+
+
+# ---------------------------------------------------------------- generator
+def test_generator_golden_and_ranges():
+    """SplitMix64's published test vector (seed 1234567: first outputs) pins mix64;
+    ranges and grid of the uniform draw; normal moments."""
+    # SplitMix64 state s -> output mix64(s + GOLDEN); known vector for seed 1234567
+    s = np.array([1234567], dtype=np.uint64)
+    with np.errstate(over="ignore"):
+        o1 = nk_inputs.mix64(s + nk_inputs.GOLDEN)[0]
+        o2 = nk_inputs.mix64(s + nk_inputs.GOLDEN * np.uint64(2))[0]
+    assert int(o1) == 6457827717110365317 and int(o2) == 3203168211198807973
+    u = nk_inputs.fill(1, 0, 200000)
+    assert u.min() >= -1.0 and u.max() < 1.0
+    assert np.all(u * 2.0 ** 23 == np.round(u * 2.0 ** 23))
+    assert abs(u.mean()) < 0.01 and abs(u.var() - 1 / 3) < 0.01
+    z = nk_inputs.fill(1, 1, 200000, "normal", 0.02)
+    assert abs(z.mean()) < 3e-4 and abs(z.std() - 0.02) < 3e-4
+    # stateless: any slice equals the same indices of a longer buffer
+    assert np.array_equal(nk_inputs.fill(1, 0, 100), u[:100])
+    rows = nk_inputs.stratified_rows(4017, 8192, 64)
+    assert len(rows) == 64 and np.array_equal(rows // 128, np.arange(64))
