@@ -1,0 +1,150 @@
+/*
+ * nk_gemm — dense GEMM for NVIDIA B200 (sm_100a) behind a plain C ABI.
+ *
+ * The operation is the batch-reduce GEMM of the paper's Algorithm 1
+ * ("BRGEMM - nanokernels()", C = beta*C + sum_i A_i x B_i) taken with beta = 0
+ * and the batch folded into K:
+ *
+ *     C[M][N] = A[M][K] . B[K][N]                     FP32 accumulation
+ *     C[M][N] = ReLU(A.B + bias[N])                   optional fused epilogue
+ *                                                     (Section 6, "MLP": bias and ReLU are
+ *                                                     applied before the single store of C)
+ *
+ * Element types (Section 2.3): FP32 operands, or BF16 operands widened exactly to
+ * FP32 with the products accumulated in FP32.  C is FP32, or BF16 (BF16 operands
+ * only) rounded to nearest-even once, after the epilogue.
+ *
+ * Operand layouts (Section 2.3, Figure 1 and Listing 1):
+ *   NK_ROW_MAJOR   A[M][K], B[K][N]                      ("flat")
+ *   NK_BLOCKED32   A[M/32][K/32][32][32]                 (m-block, k-block, m, k)
+ *                  B[N/32][K/32][16][32][2]              (n-block, k-block, k/2, n, k%2):
+ *                  every 32x32 block of B is VNNI-2 packed as in Figure 1,
+ *                  packed[k/2][n][k%2] = flat[k][n]; BF16 only.
+ * C is row-major [M][N] in every case; bias is [N] in the operand type.
+ *
+ * All data pointers are DEVICE pointers on the plan's device unless a function
+ * says otherwise.  The library never allocates or frees device memory, never
+ * synchronises inside nk_gemm_run, and reports every failure as a status code
+ * (nothing is printed, nothing is thrown).  No CPU fallback exists: without a
+ * usable sm_100 device every call that needs one returns NK_ERR_DEVICE.
+ */
+#ifndef NK_GEMM_H
+#define NK_GEMM_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct nk_gemm_s* nk_gemm_t; /* opaque plan; host memory only */
+
+typedef enum {
+    NK_OK = 0,
+    NK_ERR_INVALID_ARG = 1, /* null pointer, non-positive size, bad enum                */
+    NK_ERR_UNSUPPORTED = 2, /* legal request this build has no kernel for               */
+    NK_ERR_MISALIGNED = 3,  /* pointer not 16-byte aligned / size not a required multiple */
+    NK_ERR_WORKSPACE = 4,   /* workspace null or smaller than nk_gemm_workspace_bytes   */
+    NK_ERR_DEVICE = 5,      /* no CUDA device, wrong device, or not compute capability 10.x */
+    NK_ERR_CUDA = 6,        /* a CUDA runtime/driver call failed                        */
+    NK_ERR_TIMEOUT = 7      /* a bounded device-side wait ran out (see nk_gemm_check)    */
+} nk_status_t;
+
+typedef enum { NK_F32 = 0, NK_BF16 = 1 } nk_dtype_t;
+typedef enum { NK_ROW_MAJOR = 0, NK_BLOCKED32 = 1 } nk_layout_t;
+typedef enum { NK_EPI_NONE = 0, NK_EPI_BIAS_RELU = 1 } nk_epilogue_t;
+
+/* desc.flags: 0 lets the plan choose.  The rest are tuning/debug overrides. */
+#define NK_FLAG_KERNEL_MASK 0x0000000Fu
+#define NK_FLAG_KERNEL_AUTO 0x0u
+#define NK_FLAG_KERNEL_NAIVE 0x1u /* one thread per output element; debug cross-check only   */
+#define NK_FLAG_KERNEL_SIMT 0x2u  /* register-blocked FFMA kernel (FP32 operands)             */
+#define NK_FLAG_KERNEL_UMMA 0x3u  /* TMA + tcgen05.mma + TMEM pipeline (BF16 operands)        */
+#define NK_FLAG_REPACK_B 0x10u    /* blocked B: unpack to row-major in the workspace first,
+                                     instead of re-laying it out inside the GEMM kernel      */
+#define NK_FLAG_SPLITK_SHIFT 8    /* bits 8..15: force this many K splits (0 = auto)          */
+#define NK_FLAG_TILE_N_SHIFT 16   /* bits 16..19: force tile N: 1=32 2=64 3=128 4=256 (0 = auto) */
+
+typedef struct {
+    int64_t M, N, K;
+    int32_t in_dtype;  /* nk_dtype_t of A, B and bias                        */
+    int32_t out_dtype; /* nk_dtype_t of C: NK_F32, or NK_BF16 with BF16 inputs */
+    int32_t layout_a;  /* nk_layout_t                                         */
+    int32_t layout_b;  /* nk_layout_t                                         */
+    int32_t epilogue;  /* nk_epilogue_t                                       */
+    int32_t device;    /* CUDA device ordinal                                 */
+    uint32_t flags;    /* NK_FLAG_*                                           */
+} nk_gemm_desc_t;
+
+/*
+ * Build a plan (Section 3.1, register tiling; Section 5(a), tile-size selection:
+ * here the choice of kernel, output tile and K split is made once, from the
+ * shape).  Validates the descriptor, queries the device, and keeps only host
+ * state.  Requirements: M, N, K > 0; blocked layouts need BF16 and the blocked
+ * operand's two dimensions to be multiples of 32; row-major BF16 needs N and K
+ * to be multiples of 8, row-major FP32 needs N and K to be multiples of 4
+ * (16-byte rows); BF16 output needs BF16 inputs.  On failure *out is NULL.
+ */
+nk_status_t nk_gemm_create(const nk_gemm_desc_t* desc, nk_gemm_t* out);
+
+/*
+ * Bytes of device scratch nk_gemm_run needs for this plan: 0 unless the plan
+ * splits K (FP32 partial tiles, reduced in a fixed order: deterministic) or
+ * unpacks a blocked operand first.  The caller allocates it; contents need not
+ * be initialised and are undefined afterwards.
+ */
+size_t nk_gemm_workspace_bytes(nk_gemm_t plan);
+
+/*
+ * Enqueue C = A.B (+ epilogue) on `cuda_stream` (a cudaStream_t; NULL is the
+ * default stream) and return without synchronising (Algorithm 1: tile loop,
+ * accumulator resident over the whole K loop, epilogue, one store of C).
+ * C's previous contents are never read.  A, B, C (and bias, workspace when
+ * used) must be 16-byte aligned device pointers on the plan's device, must not
+ * overlap, and must stay valid until the stream reaches the end of the work.
+ * bias may be NULL only when the plan has no epilogue.  Nothing is launched
+ * when an error is returned.  A plan must not be run from two host threads at
+ * once; distinct plans may be.
+ */
+nk_status_t nk_gemm_run(nk_gemm_t plan, const void* A, const void* B, const void* bias, void* C,
+                        void* workspace, size_t workspace_bytes, void* cuda_stream);
+
+/*
+ * The same operation for callers holding HOST buffers (pageable or pinned):
+ * copies hA, hB (and hbias) into the caller-provided device staging buffers
+ * dA, dB, dbias, runs the plan, copies dC back into hC, and waits for the
+ * stream.  Sizes are those implied by the plan's descriptor.  Returns after the
+ * result is in hC.
+ */
+nk_status_t nk_gemm_run_host(nk_gemm_t plan, const void* hA, const void* hB, const void* hbias,
+                             void* hC, void* dA, void* dB, void* dbias, void* dC, void* workspace,
+                             size_t workspace_bytes, void* cuda_stream);
+
+/*
+ * Synchronise the plan's device and read the library's device status word.
+ * Every wait inside the kernels (on a TMA or MMA completion barrier) is
+ * bounded; a wait that runs out records itself in that word, the kernel drains
+ * and exits, and this call returns NK_ERR_TIMEOUT once (the word is cleared;
+ * results of the affected run are undefined).  NK_OK otherwise.  The word is a
+ * small static device variable of the library, one per device, shared by all
+ * plans on that device.
+ */
+nk_status_t nk_gemm_check(nk_gemm_t plan);
+
+/* Free the plan's host state.  NULL is accepted. */
+nk_status_t nk_gemm_destroy(nk_gemm_t plan);
+
+/* Static strings; never NULL. */
+const char* nk_status_str(nk_status_t s);
+/* Name of the kernel variant the plan selected, e.g. "umma_bf16_128x256x64_s4". */
+const char* nk_gemm_kernel_name(nk_gemm_t plan);
+/* Number of kernel launches one nk_gemm_run of this plan enqueues. */
+int nk_gemm_launches_per_run(nk_gemm_t plan);
+/* Message of the last CUDA error a call on this plan captured ("" if none). */
+const char* nk_gemm_last_cuda_error(nk_gemm_t plan);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* NK_GEMM_H */

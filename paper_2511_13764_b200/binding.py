@@ -1,0 +1,171 @@
+"""ctypes binding of include/nk_gemm.h.  Same names, argument marshalling only.
+
+The binding loads the in-tree ``libnk_gemm.so`` and fails loudly when it is
+missing or cannot be loaded: there is no Python or CPU fallback.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+
+from . import _build
+
+F32, BF16 = 0, 1
+ROW_MAJOR, BLOCKED32 = 0, 1
+EPI_NONE, EPI_BIAS_RELU = 0, 1
+FLAG_KERNEL_NAIVE, FLAG_KERNEL_SIMT, FLAG_KERNEL_UMMA = 0x1, 0x2, 0x3
+FLAG_REPACK_B = 0x10
+
+EXPORTS = ["nk_gemm_create", "nk_gemm_workspace_bytes", "nk_gemm_run", "nk_gemm_run_host",
+           "nk_gemm_check", "nk_gemm_destroy", "nk_status_str", "nk_gemm_kernel_name",
+           "nk_gemm_launches_per_run", "nk_gemm_last_cuda_error"]
+
+
+def flag_splitk(n: int) -> int:
+    return (n & 0xFF) << 8
+
+
+def flag_tile_n(code: int) -> int:
+    """1=32, 2=64, 3=128, 4=256."""
+    return (code & 0xF) << 16
+
+
+class NkError(RuntimeError):
+    def __init__(self, status: int, msg: str):
+        super().__init__(f"nk_gemm status {status}: {msg}")
+        self.status = status
+
+
+class Desc(ctypes.Structure):
+    _fields_ = [("M", ctypes.c_int64), ("N", ctypes.c_int64), ("K", ctypes.c_int64),
+                ("in_dtype", ctypes.c_int32), ("out_dtype", ctypes.c_int32),
+                ("layout_a", ctypes.c_int32), ("layout_b", ctypes.c_int32),
+                ("epilogue", ctypes.c_int32), ("device", ctypes.c_int32),
+                ("flags", ctypes.c_uint32)]
+
+
+_lib = None
+
+
+def lib_path() -> str:
+    return _build.LIB
+
+
+def lib():
+    """Load libnk_gemm.so (building it first when the sources are newer)."""
+    global _lib
+    if _lib is None:
+        path = _build.LIB
+        if not os.path.exists(path) or os.environ.get("NK_GEMM_REBUILD"):
+            path = _build.build()
+        L = ctypes.CDLL(path)          # raises OSError when unusable: no fallback
+        vp, sz = ctypes.c_void_p, ctypes.c_size_t
+        L.nk_gemm_create.restype = ctypes.c_int
+        L.nk_gemm_create.argtypes = [ctypes.POINTER(Desc), ctypes.POINTER(vp)]
+        L.nk_gemm_workspace_bytes.restype = sz
+        L.nk_gemm_workspace_bytes.argtypes = [vp]
+        L.nk_gemm_run.restype = ctypes.c_int
+        L.nk_gemm_run.argtypes = [vp, vp, vp, vp, vp, vp, sz, vp]
+        L.nk_gemm_run_host.restype = ctypes.c_int
+        L.nk_gemm_run_host.argtypes = [vp, vp, vp, vp, vp, vp, vp, vp, vp, vp, sz, vp]
+        L.nk_gemm_check.restype = ctypes.c_int
+        L.nk_gemm_check.argtypes = [vp]
+        L.nk_gemm_destroy.restype = ctypes.c_int
+        L.nk_gemm_destroy.argtypes = [vp]
+        L.nk_status_str.restype = ctypes.c_char_p
+        L.nk_status_str.argtypes = [ctypes.c_int]
+        L.nk_gemm_kernel_name.restype = ctypes.c_char_p
+        L.nk_gemm_kernel_name.argtypes = [vp]
+        L.nk_gemm_launches_per_run.restype = ctypes.c_int
+        L.nk_gemm_launches_per_run.argtypes = [vp]
+        L.nk_gemm_last_cuda_error.restype = ctypes.c_char_p
+        L.nk_gemm_last_cuda_error.argtypes = [vp]
+        _lib = L
+    return _lib
+
+
+def exported_symbols():
+    L = lib()
+    return [s for s in EXPORTS if hasattr(L, s)]
+
+
+def _check(status: int, plan=None):
+    if status != 0:
+        msg = lib().nk_status_str(status).decode()
+        if plan is not None:
+            extra = lib().nk_gemm_last_cuda_error(plan).decode()
+            if extra:
+                msg += f" ({extra})"
+        raise NkError(status, msg)
+
+
+def _ptr(x):
+    """Device/host pointer of a torch tensor, an int, or None."""
+    if x is None:
+        return None
+    if isinstance(x, int):
+        return x
+    return x.data_ptr()
+
+
+class Plan:
+    """nk_gemm_create / run / destroy.  Tensors are torch tensors used only for
+    their pointers; the caller owns every buffer."""
+
+    def __init__(self, M, N, K, in_dtype=BF16, out_dtype=F32, layout_a=ROW_MAJOR,
+                 layout_b=ROW_MAJOR, epilogue=EPI_NONE, device=0, flags=0):
+        self.desc = Desc(M, N, K, in_dtype, out_dtype, layout_a, layout_b, epilogue, device, flags)
+        self._h = ctypes.c_void_p()
+        _check(lib().nk_gemm_create(ctypes.byref(self.desc), ctypes.byref(self._h)))
+
+    @property
+    def workspace_bytes(self) -> int:
+        return lib().nk_gemm_workspace_bytes(self._h)
+
+    @property
+    def kernel_name(self) -> str:
+        return lib().nk_gemm_kernel_name(self._h).decode()
+
+    @property
+    def launches_per_run(self) -> int:
+        return lib().nk_gemm_launches_per_run(self._h)
+
+    def run(self, A, B, C, bias=None, workspace=None, workspace_bytes=None, stream=None):
+        if workspace_bytes is None:
+            workspace_bytes = 0 if workspace is None else workspace.numel() * workspace.element_size()
+        _check(lib().nk_gemm_run(self._h, _ptr(A), _ptr(B), _ptr(bias), _ptr(C), _ptr(workspace),
+                                 workspace_bytes, stream), self._h)
+
+    def run_host(self, hA, hB, hC, dA, dB, dC, hbias=None, dbias=None, workspace=None,
+                 workspace_bytes=None, stream=None):
+        if workspace_bytes is None:
+            workspace_bytes = 0 if workspace is None else workspace.numel() * workspace.element_size()
+        _check(lib().nk_gemm_run_host(self._h, _ptr(hA), _ptr(hB), _ptr(hbias), _ptr(hC), _ptr(dA),
+                                      _ptr(dB), _ptr(dbias), _ptr(dC), _ptr(workspace),
+                                      workspace_bytes, stream), self._h)
+
+    def check(self):
+        _check(lib().nk_gemm_check(self._h), self._h)
+
+    def destroy(self):
+        if self._h:
+            lib().nk_gemm_destroy(self._h)
+            self._h = ctypes.c_void_p()
+
+    def __del__(self):
+        try:
+            self.destroy()
+        except Exception:
+            pass
+
+
+def plan_for(w, device=0, flags=0) -> Plan:
+    """Plan for a workload record with M, N, K, in_dtype ("f32"/"bf16"), out_dtype,
+    layout ("row"/"blocked32") and epilogue ("none"/"bias_relu") attributes."""
+    lay = BLOCKED32 if w.layout == "blocked32" else ROW_MAJOR
+    return Plan(w.M, w.N, w.K,
+                in_dtype=F32 if w.in_dtype == "f32" else BF16,
+                out_dtype=F32 if w.out_dtype == "f32" else BF16,
+                layout_a=lay, layout_b=lay,
+                epilogue=EPI_BIAS_RELU if w.epilogue == "bias_relu" else EPI_NONE,
+                device=device, flags=flags)

@@ -1,0 +1,110 @@
+// Small kernels around the two GEMM mainloops: the one-thread-per-output debug
+// kernel, the deterministic split-K reduction with the fused epilogue, and the
+// unpacking of a VNNI-blocked B operand into row-major scratch.
+#pragma once
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+namespace nk {
+
+struct NaiveParams {
+    int M, N, K;
+    int in_bf16, out_bf16, a_blocked, b_blocked, epilogue;
+    const void *A, *B, *bias;
+    void* C;
+};
+
+__device__ __forceinline__ float ld_elem(const void* p, int bf16, size_t i) {
+    return bf16 ? __uint_as_float(static_cast<uint32_t>(static_cast<const uint16_t*>(p)[i]) << 16)
+                : static_cast<const float*>(p)[i];
+}
+
+// Debug cross-check only: one thread per C element, FP32 accumulation in k order,
+// operands addressed through the layout index functions (Figure 1 for blocked B).
+__global__ void naive_gemm_kernel(const NaiveParams p) {
+    const int j = blockIdx.x * blockDim.x + threadIdx.x;
+    const int i = blockIdx.y;
+    if (j >= p.N || i >= p.M) return;
+    const size_t kb32 = p.K / 32;
+    float acc = 0.f;
+    for (int k = 0; k < p.K; ++k) {
+        const size_t ia = p.a_blocked
+            ? (((static_cast<size_t>(i / 32) * kb32 + k / 32) * 32 + i % 32) * 32 + k % 32)
+            : static_cast<size_t>(i) * p.K + k;
+        const size_t ib = p.b_blocked
+            ? (((((static_cast<size_t>(j / 32) * kb32 + k / 32) * 16 + (k % 32) / 2) * 32 + j % 32) * 2) + k % 2)
+            : static_cast<size_t>(k) * p.N + j;
+        acc = fmaf(ld_elem(p.A, p.in_bf16, ia), ld_elem(p.B, p.in_bf16, ib), acc);
+    }
+    if (p.epilogue) acc = fmaxf(acc + ld_elem(p.bias, p.in_bf16, j), 0.f);
+    const size_t o = static_cast<size_t>(i) * p.N + j;
+    if (p.out_bf16)
+        static_cast<__nv_bfloat16*>(p.C)[o] = __float2bfloat16_rn(acc);
+    else
+        static_cast<float*>(p.C)[o] = acc;
+}
+
+struct ReduceParams {
+    size_t MN;          // elements of C
+    int N;
+    int splits;
+    int epilogue, bias_bf16, out_bf16;
+    const float* partial;  // [splits][M][N]
+    const void* bias;
+    void* C;
+};
+
+// C = epilogue(sum over splits, in split order): fixed order, so the result does
+// not depend on how CTAs were scheduled.  Four consecutive columns per thread.
+__global__ void splitk_reduce_kernel(const ReduceParams p) {
+    const size_t q = static_cast<size_t>(blockIdx.x) * blockDim.x + threadIdx.x;
+    const size_t e = q * 4;
+    if (e >= p.MN) return;
+    float4 s = __ldcs(reinterpret_cast<const float4*>(p.partial + e));
+    for (int sp = 1; sp < p.splits; ++sp) {
+        const float4 v = __ldcs(reinterpret_cast<const float4*>(p.partial + sp * p.MN + e));
+        s.x += v.x; s.y += v.y; s.z += v.z; s.w += v.w;
+    }
+    if (p.epilogue) {
+        const int n = static_cast<int>(e % p.N);
+        float b0, b1, b2, b3;
+        if (p.bias_bf16) {
+            const uint2 w = __ldg(reinterpret_cast<const uint2*>(static_cast<const uint16_t*>(p.bias) + n));
+            b0 = __uint_as_float(w.x << 16); b1 = __uint_as_float(w.x & 0xFFFF0000u);
+            b2 = __uint_as_float(w.y << 16); b3 = __uint_as_float(w.y & 0xFFFF0000u);
+        } else {
+            const float4 w = __ldg(reinterpret_cast<const float4*>(static_cast<const float*>(p.bias) + n));
+            b0 = w.x; b1 = w.y; b2 = w.z; b3 = w.w;
+        }
+        s.x = fmaxf(s.x + b0, 0.f); s.y = fmaxf(s.y + b1, 0.f);
+        s.z = fmaxf(s.z + b2, 0.f); s.w = fmaxf(s.w + b3, 0.f);
+    }
+    if (p.out_bf16) {
+        __nv_bfloat162 lo = __floats2bfloat162_rn(s.x, s.y), hi = __floats2bfloat162_rn(s.z, s.w);
+        uint2 o;
+        o.x = *reinterpret_cast<uint32_t*>(&lo);
+        o.y = *reinterpret_cast<uint32_t*>(&hi);
+        *reinterpret_cast<uint2*>(static_cast<uint16_t*>(p.C) + e) = o;
+    } else {
+        *reinterpret_cast<float4*>(static_cast<float*>(p.C) + e) = s;
+    }
+}
+
+// VNNI-blocked B[N/32][K/32][16][32][2] -> row-major B[K][N] (BF16).  One CTA per
+// 32 x 32 block; thread (r, lane) reads word (k2 = r.., n = lane) and writes the two
+// k rows.  Reads are 128-byte rows; writes are 64-byte row segments.
+__global__ void unpack_vnni_b_kernel(const uint32_t* __restrict__ Bblk, uint16_t* __restrict__ Brow,
+                                     int N, int K) {
+    const int kb = blockIdx.x, nb = blockIdx.y;
+    const int lane = threadIdx.x & 31, r = threadIdx.x >> 5;  // 8 warps
+    const size_t blk = (static_cast<size_t>(nb) * (K / 32) + kb) * 512;
+    for (int k2 = r; k2 < 16; k2 += 8) {
+        const uint32_t w = Bblk[blk + k2 * 32 + lane];
+        const size_t row0 = static_cast<size_t>(kb * 32 + 2 * k2) * N + nb * 32 + lane;
+        Brow[row0] = static_cast<uint16_t>(w & 0xFFFFu);       // even k: low half
+        Brow[row0 + N] = static_cast<uint16_t>(w >> 16);       // odd k: high half
+    }
+}
+
+}  // namespace nk

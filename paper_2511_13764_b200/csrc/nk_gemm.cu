@@ -1,0 +1,515 @@
+// Host side of the nk_gemm C ABI: descriptor validation, the plan-time choice of
+// kernel / tile / K split, TMA tensor-map encoding, and the launches.  All the
+// arithmetic of the GEMM runs in the kernels included below.
+#include "../../include/nk_gemm.h"
+
+#include <cuda.h>
+#include <cuda_runtime.h>
+
+#include <cstdio>
+#include <cstdlib>
+#include <cstring>
+#include <new>
+
+#include "aux_kernels.cuh"
+#include "simt_f32.cuh"
+#include "umma_bf16.cuh"
+
+namespace nk {
+
+// One status word per device (the module is instantiated on every device that
+// loads the library).  Kernels receive its device address as a parameter.
+__device__ unsigned int g_status_word[4];
+
+enum Variant { V_NAIVE = 0, V_SIMT = 1, V_UMMA = 2 };
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*,
+                                  const cuuint64_t*, const cuuint64_t*, const cuuint32_t*,
+                                  const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
+                                  CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+}  // namespace nk
+
+struct nk_gemm_s {
+    nk_gemm_desc_t d;
+    int variant;
+    int sm_count;
+    // UMMA
+    int bn, stages, splits, group_m;
+    bool b_vnni_inkernel;  // blocked B re-laid inside the GEMM kernel
+    bool b_repack;         // blocked B unpacked to row-major scratch first
+    // SIMT
+    int simt_tile;  // 128, 64 or 32
+    int kt_per_split;
+    // workspace layout
+    size_t ws_repack_bytes, ws_partial_bytes;
+    // device status word
+    unsigned int* status_dev;
+    // cached tensor maps
+    CUtensorMap tmap_a, tmap_b;
+    const void *cached_a, *cached_b;
+    nk::EncodeTiledFn encode;
+    char name[96];
+    char cuda_err[256];
+    int launches;
+};
+
+namespace nk {
+
+static void set_err(nk_gemm_s* p, const char* what, cudaError_t e) {
+    snprintf(p->cuda_err, sizeof(p->cuda_err), "%s: %s", what, cudaGetErrorString(e));
+}
+
+struct DeviceGuard {
+    int prev = -1;
+    bool changed = false;
+    cudaError_t err = cudaSuccess;
+    explicit DeviceGuard(int dev) {
+        err = cudaGetDevice(&prev);
+        if (err == cudaSuccess && prev != dev) {
+            err = cudaSetDevice(dev);
+            changed = (err == cudaSuccess);
+        }
+    }
+    ~DeviceGuard() {
+        if (changed) cudaSetDevice(prev);
+    }
+};
+
+static inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
+static inline int ceil_div(int64_t a, int64_t b) { return static_cast<int>((a + b - 1) / b); }
+
+// tcgen05 instruction descriptor, kind::f16: D format FP32 (bit 4), A and B format
+// BF16 (bits 7, 10), B major-ness (bit 16: 0 = K-major, 1 = N-major), N/8 at bit 17,
+// M/16 at bit 24.  A is always K-major.
+static uint32_t make_idesc(int m, int n, bool b_n_major) {
+    uint32_t d = 0;
+    d |= 1u << 4;
+    d |= 1u << 7;
+    d |= 1u << 10;
+    d |= (b_n_major ? 1u : 0u) << 16;
+    d |= static_cast<uint32_t>(n >> 3) << 17;
+    d |= static_cast<uint32_t>(m >> 4) << 24;
+    return d;
+}
+
+template <typename K>
+static cudaError_t allow_smem(K kernel, int bytes) {
+    return cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes);
+}
+
+static int umma_stages_for(int bn) { return bn == 256 ? 4 : bn == 128 ? 6 : 8; }
+
+static void choose_umma(nk_gemm_s* p) {
+    const nk_gemm_desc_t& d = p->d;
+    const int sms = p->sm_count;
+    const int tiles_m = ceil_div(d.M, UMMA_BM);
+    const int kb_total = ceil_div(d.K, UMMA_BK);
+    int bn = 64;
+    const int forced = (d.flags >> NK_FLAG_TILE_N_SHIFT) & 0xF;
+    if (forced >= 2 && forced <= 4) {
+        bn = 32 << (forced - 1);
+    } else {
+        const int cands[3] = {256, 128, 64};
+        for (int c : cands) {
+            if (static_cast<int64_t>(tiles_m) * ceil_div(d.N, c) >= sms) { bn = c; break; }
+        }
+    }
+    p->bn = bn;
+    p->stages = umma_stages_for(bn);
+    const int tiles = tiles_m * ceil_div(d.N, bn);
+    int splits = 1;
+    const int forced_s = (d.flags >> NK_FLAG_SPLITK_SHIFT) & 0xFF;
+    if (forced_s > 0) {
+        splits = forced_s;
+    } else if (tiles * 2 <= sms) {
+        splits = sms / tiles;
+        const int max_by_k = kb_total / 4 > 0 ? kb_total / 4 : 1;  // >= 4 k-blocks per split
+        if (splits > max_by_k) splits = max_by_k;
+        if (splits > 32) splits = 32;
+    }
+    if (splits > kb_total) splits = kb_total;
+    if (splits < 1) splits = 1;
+    // no empty split: shrink until the last one starts inside the K range
+    int per = ceil_div(kb_total, splits);
+    splits = ceil_div(kb_total, per);
+    p->splits = splits;
+    p->group_m = 8;
+}
+
+static void choose_simt(nk_gemm_s* p) {
+    const nk_gemm_desc_t& d = p->d;
+    const int sms = p->sm_count;
+    const int ktiles = ceil_div(d.K, SIMT_BK);
+    const int64_t t128 = static_cast<int64_t>(ceil_div(d.M, 128)) * ceil_div(d.N, 128);
+    const int64_t t64 = static_cast<int64_t>(ceil_div(d.M, 64)) * ceil_div(d.N, 64);
+    const int64_t t32 = static_cast<int64_t>(ceil_div(d.M, 32)) * ceil_div(d.N, 32);
+    int tile;
+    int64_t tiles;
+    int resident;  // CTAs of this variant one SM holds
+    if (t128 >= 2 * sms && d.M >= 96) { tile = 128; tiles = t128; resident = 2; }
+    else if (t64 >= sms && d.M >= 48) { tile = 64; tiles = t64; resident = 6; }
+    else { tile = 32; tiles = t32; resident = 16; }
+    const int forced = (d.flags >> NK_FLAG_TILE_N_SHIFT) & 0xF;
+    if (forced == 1) { tile = 32; tiles = t32; resident = 16; }
+    if (forced == 2) { tile = 64; tiles = t64; resident = 6; }
+    if (forced == 3) { tile = 128; tiles = t128; resident = 2; }
+    p->simt_tile = tile;
+    int splits = 1;
+    const int forced_s = (d.flags >> NK_FLAG_SPLITK_SHIFT) & 0xFF;
+    if (forced_s > 0) {
+        splits = forced_s;
+    } else if (tiles < static_cast<int64_t>(sms) * resident / 2) {
+        splits = static_cast<int>(static_cast<int64_t>(sms) * resident / tiles);
+        const int max_by_k = ktiles / 8 > 0 ? ktiles / 8 : 1;  // >= 8 k-tiles (128 k) per split
+        if (splits > max_by_k) splits = max_by_k;
+        if (splits > 64) splits = 64;
+    }
+    if (splits > ktiles) splits = ktiles;
+    if (splits < 1) splits = 1;
+    int per = ceil_div(ktiles, splits);
+    splits = ceil_div(ktiles, per);
+    p->splits = splits;
+    p->kt_per_split = per;
+}
+
+static nk_status_t encode_maps(nk_gemm_s* p, const void* A, const void* B) {
+    if (p->cached_a == A && p->cached_b == B) return NK_OK;
+    const nk_gemm_desc_t& d = p->d;
+    CUresult r;
+    if (d.layout_a == NK_BLOCKED32) {
+        // [M/32][K/32][32][32] viewed with dims (k, k-block, m, m-block): a box of
+        // 32 x 2 x 32 x 4 lands in shared memory as 128 rows of 64 consecutive k.
+        cuuint64_t dims[4] = {32, static_cast<cuuint64_t>(d.K / 32), 32, static_cast<cuuint64_t>(d.M / 32)};
+        cuuint64_t strides[3] = {1024 * 2, 32 * 2, static_cast<cuuint64_t>(d.K / 32) * 1024 * 2};
+        cuuint32_t box[4] = {32, 2, 32, 4};
+        cuuint32_t es[4] = {1, 1, 1, 1};
+        r = p->encode(&p->tmap_a, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void*>(A), dims, strides,
+                      box, es, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+                      CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    } else {
+        cuuint64_t dims[2] = {static_cast<cuuint64_t>(d.K), static_cast<cuuint64_t>(d.M)};
+        cuuint64_t strides[1] = {static_cast<cuuint64_t>(d.K) * 2};
+        cuuint32_t box[2] = {UMMA_BK, UMMA_BM};
+        cuuint32_t es[2] = {1, 1};
+        r = p->encode(&p->tmap_a, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(A), dims, strides,
+                      box, es, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+                      CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    }
+    if (r != CUDA_SUCCESS) {
+        snprintf(p->cuda_err, sizeof(p->cuda_err), "cuTensorMapEncodeTiled(A) failed: %d", (int)r);
+        return NK_ERR_CUDA;
+    }
+    if (!p->b_vnni_inkernel) {
+        // B row-major [K][N]: 64 (n) x 64 (k) boxes, N contiguous.
+        cuuint64_t dims[2] = {static_cast<cuuint64_t>(d.N), static_cast<cuuint64_t>(d.K)};
+        cuuint64_t strides[1] = {static_cast<cuuint64_t>(d.N) * 2};
+        cuuint32_t box[2] = {64, UMMA_BK};
+        cuuint32_t es[2] = {1, 1};
+        r = p->encode(&p->tmap_b, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(B), dims, strides,
+                      box, es, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+                      CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+        if (r != CUDA_SUCCESS) {
+            snprintf(p->cuda_err, sizeof(p->cuda_err), "cuTensorMapEncodeTiled(B) failed: %d", (int)r);
+            return NK_ERR_CUDA;
+        }
+    } else {
+        memset(&p->tmap_b, 0, sizeof(p->tmap_b));
+    }
+    p->cached_a = A;
+    p->cached_b = B;
+    return NK_OK;
+}
+
+template <int BN, int STAGES, bool VNNI>
+static cudaError_t launch_umma_t(nk_gemm_s* p, const UmmaParams& up, int grid, cudaStream_t st) {
+    auto k = umma_bf16_kernel<BN, STAGES, VNNI>;
+    umma_bf16_kernel<BN, STAGES, VNNI><<<grid, VNNI ? 320 : 192, umma_smem_bytes(BN, STAGES), st>>>(
+        p->tmap_a, p->tmap_b, up);
+    (void)k;
+    return cudaGetLastError();
+}
+
+static cudaError_t launch_umma(nk_gemm_s* p, const UmmaParams& up, int grid, cudaStream_t st) {
+    const bool v = p->b_vnni_inkernel;
+    switch (p->bn) {
+        case 256: return v ? launch_umma_t<256, 4, true>(p, up, grid, st) : launch_umma_t<256, 4, false>(p, up, grid, st);
+        case 128: return v ? launch_umma_t<128, 6, true>(p, up, grid, st) : launch_umma_t<128, 6, false>(p, up, grid, st);
+        default:  return v ? launch_umma_t<64, 8, true>(p, up, grid, st) : launch_umma_t<64, 8, false>(p, up, grid, st);
+    }
+}
+
+static cudaError_t prepare_umma_attrs() {
+    cudaError_t e;
+    if ((e = allow_smem(umma_bf16_kernel<256, 4, false>, umma_smem_bytes(256, 4))) != cudaSuccess) return e;
+    if ((e = allow_smem(umma_bf16_kernel<128, 6, false>, umma_smem_bytes(128, 6))) != cudaSuccess) return e;
+    if ((e = allow_smem(umma_bf16_kernel<64, 8, false>, umma_smem_bytes(64, 8))) != cudaSuccess) return e;
+    if ((e = allow_smem(umma_bf16_kernel<256, 4, true>, umma_smem_bytes(256, 4))) != cudaSuccess) return e;
+    if ((e = allow_smem(umma_bf16_kernel<128, 6, true>, umma_smem_bytes(128, 6))) != cudaSuccess) return e;
+    if ((e = allow_smem(umma_bf16_kernel<64, 8, true>, umma_smem_bytes(64, 8))) != cudaSuccess) return e;
+    return cudaSuccess;
+}
+
+static cudaError_t launch_simt(nk_gemm_s* p, const SimtParams& sp, cudaStream_t st) {
+    const int t = p->simt_tile;
+    dim3 grid(ceil_div(sp.N, t), ceil_div(sp.M, t), sp.splits);
+    if (t == 128) simt_f32_kernel<128, 128, 8, 8><<<grid, 256, 0, st>>>(sp);
+    else if (t == 64) simt_f32_kernel<64, 64, 4, 4><<<grid, 256, 0, st>>>(sp);
+    else simt_f32_kernel<32, 32, 4, 4><<<grid, 64, 0, st>>>(sp);
+    return cudaGetLastError();
+}
+
+}  // namespace nk
+
+using namespace nk;
+
+extern "C" {
+
+const char* nk_status_str(nk_status_t s) {
+    switch (s) {
+        case NK_OK: return "ok";
+        case NK_ERR_INVALID_ARG: return "invalid argument";
+        case NK_ERR_UNSUPPORTED: return "unsupported configuration";
+        case NK_ERR_MISALIGNED: return "misaligned pointer or size";
+        case NK_ERR_WORKSPACE: return "workspace missing or too small";
+        case NK_ERR_DEVICE: return "no usable sm_100 CUDA device";
+        case NK_ERR_CUDA: return "CUDA call failed";
+        case NK_ERR_TIMEOUT: return "device-side wait timed out";
+    }
+    return "unknown status";
+}
+
+nk_status_t nk_gemm_create(const nk_gemm_desc_t* desc, nk_gemm_t* out) {
+    if (out) *out = nullptr;
+    if (!desc || !out) return NK_ERR_INVALID_ARG;
+    const nk_gemm_desc_t& d = *desc;
+    if (d.M <= 0 || d.N <= 0 || d.K <= 0) return NK_ERR_INVALID_ARG;
+    if (d.M > (1 << 24) || d.N > (1 << 24) || d.K > (1 << 24)) return NK_ERR_UNSUPPORTED;
+    if (d.M * d.N >= (1ll << 31) || d.M * d.K >= (1ll << 33) || d.K * d.N >= (1ll << 33)) return NK_ERR_UNSUPPORTED;
+    if (d.in_dtype != NK_F32 && d.in_dtype != NK_BF16) return NK_ERR_INVALID_ARG;
+    if (d.out_dtype != NK_F32 && d.out_dtype != NK_BF16) return NK_ERR_INVALID_ARG;
+    if (d.layout_a != NK_ROW_MAJOR && d.layout_a != NK_BLOCKED32) return NK_ERR_INVALID_ARG;
+    if (d.layout_b != NK_ROW_MAJOR && d.layout_b != NK_BLOCKED32) return NK_ERR_INVALID_ARG;
+    if (d.epilogue != NK_EPI_NONE && d.epilogue != NK_EPI_BIAS_RELU) return NK_ERR_INVALID_ARG;
+    if (d.out_dtype == NK_BF16 && d.in_dtype != NK_BF16) return NK_ERR_INVALID_ARG;
+    const bool blocked = d.layout_a == NK_BLOCKED32 || d.layout_b == NK_BLOCKED32;
+    if (blocked && d.in_dtype != NK_BF16) return NK_ERR_UNSUPPORTED;
+    if (d.layout_a == NK_BLOCKED32 && (d.M % 32 || d.K % 32)) return NK_ERR_MISALIGNED;
+    if (d.layout_b == NK_BLOCKED32 && (d.N % 32 || d.K % 32)) return NK_ERR_MISALIGNED;
+    const uint32_t force = d.flags & NK_FLAG_KERNEL_MASK;
+    if (force > NK_FLAG_KERNEL_UMMA) return NK_ERR_INVALID_ARG;
+    if (force != NK_FLAG_KERNEL_NAIVE) {
+        if (d.in_dtype == NK_BF16 && (d.N % 8 || d.K % 8)) return NK_ERR_MISALIGNED;
+        if (d.in_dtype == NK_F32 && (d.N % 4 || d.K % 4)) return NK_ERR_MISALIGNED;
+        if (force == NK_FLAG_KERNEL_SIMT && d.in_dtype != NK_F32) return NK_ERR_UNSUPPORTED;
+        if (force == NK_FLAG_KERNEL_UMMA && d.in_dtype != NK_BF16) return NK_ERR_UNSUPPORTED;
+    }
+
+    int ndev = 0;
+    if (cudaGetDeviceCount(&ndev) != cudaSuccess || ndev <= 0) {
+        cudaGetLastError();
+        return NK_ERR_DEVICE;
+    }
+    if (d.device < 0 || d.device >= ndev) return NK_ERR_DEVICE;
+    cudaDeviceProp prop;
+    if (cudaGetDeviceProperties(&prop, d.device) != cudaSuccess) return NK_ERR_DEVICE;
+    if (prop.major != 10) return NK_ERR_DEVICE;
+
+    nk_gemm_s* p = new (std::nothrow) nk_gemm_s();
+    if (!p) return NK_ERR_INVALID_ARG;
+    memset(p, 0, sizeof(*p));
+    p->d = d;
+    p->sm_count = prop.multiProcessorCount;
+
+    DeviceGuard guard(d.device);
+    if (guard.err != cudaSuccess) { delete p; return NK_ERR_DEVICE; }
+    void* sym = nullptr;
+    if (cudaGetSymbolAddress(&sym, g_status_word) != cudaSuccess) { delete p; return NK_ERR_CUDA; }
+    p->status_dev = static_cast<unsigned int*>(sym);
+
+    if (force == NK_FLAG_KERNEL_NAIVE) {
+        p->variant = V_NAIVE;
+        p->launches = 1;
+        snprintf(p->name, sizeof(p->name), "naive");
+    } else if (d.in_dtype == NK_F32) {
+        p->variant = V_SIMT;
+        choose_simt(p);
+        p->ws_partial_bytes = p->splits > 1 ? static_cast<size_t>(p->splits) * d.M * d.N * 4 : 0;
+        p->launches = p->splits > 1 ? 2 : 1;
+        snprintf(p->name, sizeof(p->name), "simt_f32_%dx%dx16_splitk%d", p->simt_tile, p->simt_tile, p->splits);
+    } else {
+        p->variant = V_UMMA;
+        void* fn = nullptr;
+        cudaDriverEntryPointQueryResult q;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &q) != cudaSuccess ||
+            q != cudaDriverEntryPointSuccess || !fn) {
+            delete p;
+            return NK_ERR_CUDA;
+        }
+        p->encode = reinterpret_cast<EncodeTiledFn>(fn);
+        if (prepare_umma_attrs() != cudaSuccess) { cudaGetLastError(); delete p; return NK_ERR_CUDA; }
+        choose_umma(p);
+        if (d.layout_b == NK_BLOCKED32) {
+            p->b_repack = (d.flags & NK_FLAG_REPACK_B) != 0;
+            p->b_vnni_inkernel = !p->b_repack;
+        }
+        p->ws_repack_bytes = p->b_repack ? align_up(static_cast<size_t>(d.K) * d.N * 2, 256) : 0;
+        p->ws_partial_bytes = p->splits > 1 ? static_cast<size_t>(p->splits) * d.M * d.N * 4 : 0;
+        p->launches = 1 + (p->splits > 1 ? 1 : 0) + (p->b_repack ? 1 : 0);
+        snprintf(p->name, sizeof(p->name), "umma_bf16_128x%dx64_s%d_splitk%d%s%s", p->bn, p->stages,
+                 p->splits, d.layout_a == NK_BLOCKED32 ? "_ablk" : "",
+                 p->b_vnni_inkernel ? "_bvnni" : (p->b_repack ? "_brepack" : ""));
+    }
+    *out = p;
+    return NK_OK;
+}
+
+size_t nk_gemm_workspace_bytes(nk_gemm_t p) { return p ? p->ws_repack_bytes + p->ws_partial_bytes : 0; }
+
+int nk_gemm_launches_per_run(nk_gemm_t p) { return p ? p->launches : 0; }
+
+const char* nk_gemm_kernel_name(nk_gemm_t p) { return p ? p->name : ""; }
+
+const char* nk_gemm_last_cuda_error(nk_gemm_t p) { return p ? p->cuda_err : ""; }
+
+nk_status_t nk_gemm_run(nk_gemm_t p, const void* A, const void* B, const void* bias, void* C,
+                        void* workspace, size_t workspace_bytes, void* cuda_stream) {
+    if (!p || !A || !B || !C) return NK_ERR_INVALID_ARG;
+    const nk_gemm_desc_t& d = p->d;
+    if (d.epilogue != NK_EPI_NONE && !bias) return NK_ERR_INVALID_ARG;
+    auto mis = [](const void* q) { return (reinterpret_cast<uintptr_t>(q) & 15u) != 0; };
+    if (mis(A) || mis(B) || mis(C) || (bias && mis(bias)) || (workspace && mis(workspace)))
+        return NK_ERR_MISALIGNED;
+    const size_t need = p->ws_repack_bytes + p->ws_partial_bytes;
+    if (need > 0 && (!workspace || workspace_bytes < need)) return NK_ERR_WORKSPACE;
+    cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+    DeviceGuard guard(d.device);
+    if (guard.err != cudaSuccess) { set_err(p, "cudaSetDevice", guard.err); return NK_ERR_DEVICE; }
+    cudaError_t e = cudaSuccess;
+
+    if (p->variant == V_NAIVE) {
+        NaiveParams np = {static_cast<int>(d.M), static_cast<int>(d.N), static_cast<int>(d.K),
+                          d.in_dtype == NK_BF16, d.out_dtype == NK_BF16, d.layout_a == NK_BLOCKED32,
+                          d.layout_b == NK_BLOCKED32, d.epilogue, A, B, bias, C};
+        dim3 grid(ceil_div(d.N, 128), static_cast<unsigned>(d.M));
+        if (d.M > 65535) return NK_ERR_UNSUPPORTED;
+        naive_gemm_kernel<<<grid, 128, 0, st>>>(np);
+        e = cudaGetLastError();
+        if (e != cudaSuccess) { set_err(p, "naive launch", e); return NK_ERR_CUDA; }
+        return NK_OK;
+    }
+
+    uint8_t* ws = static_cast<uint8_t*>(workspace);
+    float* partial = p->ws_partial_bytes ? reinterpret_cast<float*>(ws + p->ws_repack_bytes) : nullptr;
+
+    if (p->variant == V_SIMT) {
+        SimtParams sp = {static_cast<int>(d.M), static_cast<int>(d.N), static_cast<int>(d.K), p->splits,
+                         p->kt_per_split, d.epilogue, static_cast<const float*>(A),
+                         static_cast<const float*>(B), static_cast<const float*>(bias),
+                         static_cast<float*>(C), partial};
+        e = launch_simt(p, sp, st);
+        if (e != cudaSuccess) { set_err(p, "simt launch", e); return NK_ERR_CUDA; }
+    } else {
+        const void* Buse = B;
+        if (p->b_repack) {
+            dim3 grid(static_cast<unsigned>(d.K / 32), static_cast<unsigned>(d.N / 32));
+            unpack_vnni_b_kernel<<<grid, 256, 0, st>>>(static_cast<const uint32_t*>(B),
+                                                       reinterpret_cast<uint16_t*>(ws),
+                                                       static_cast<int>(d.N), static_cast<int>(d.K));
+            e = cudaGetLastError();
+            if (e != cudaSuccess) { set_err(p, "unpack launch", e); return NK_ERR_CUDA; }
+            Buse = ws;
+        }
+        nk_status_t s = encode_maps(p, A, Buse);
+        if (s != NK_OK) return s;
+        UmmaParams up;
+        memset(&up, 0, sizeof(up));
+        up.M = static_cast<int>(d.M); up.N = static_cast<int>(d.N); up.K = static_cast<int>(d.K);
+        up.tiles_m = ceil_div(d.M, UMMA_BM);
+        up.tiles_n = ceil_div(d.N, p->bn);
+        up.splits = p->splits;
+        up.kb_total = ceil_div(d.K, UMMA_BK);
+        up.kb_per_split = ceil_div(up.kb_total, p->splits);
+        up.group_m = p->group_m;
+        up.a_blocked = d.layout_a == NK_BLOCKED32;
+        up.epilogue = d.epilogue;
+        up.out_bf16 = d.out_dtype == NK_BF16;
+        up.idesc = make_idesc(UMMA_BM, p->bn, !p->b_vnni_inkernel);
+        up.bias = bias;
+        up.C = C;
+        up.partial = partial;
+        up.Bblk = p->b_vnni_inkernel ? static_cast<const uint32_t*>(B) : nullptr;
+        up.status = p->status_dev;
+        const int units = up.tiles_m * up.tiles_n * up.splits;
+        const int grid = units < p->sm_count ? units : p->sm_count;
+        e = launch_umma(p, up, grid, st);
+        if (e != cudaSuccess) { set_err(p, "umma launch", e); return NK_ERR_CUDA; }
+    }
+
+    if (p->splits > 1) {
+        ReduceParams rp = {static_cast<size_t>(d.M) * d.N, static_cast<int>(d.N), p->splits, d.epilogue,
+                           d.in_dtype == NK_BF16, d.out_dtype == NK_BF16, partial, bias, C};
+        const size_t quads = rp.MN / 4;
+        splitk_reduce_kernel<<<static_cast<unsigned>((quads + 255) / 256), 256, 0, st>>>(rp);
+        e = cudaGetLastError();
+        if (e != cudaSuccess) { set_err(p, "reduce launch", e); return NK_ERR_CUDA; }
+    }
+    return NK_OK;
+}
+
+nk_status_t nk_gemm_run_host(nk_gemm_t p, const void* hA, const void* hB, const void* hbias, void* hC,
+                             void* dA, void* dB, void* dbias, void* dC, void* workspace,
+                             size_t workspace_bytes, void* cuda_stream) {
+    if (!p || !hA || !hB || !hC || !dA || !dB || !dC) return NK_ERR_INVALID_ARG;
+    const nk_gemm_desc_t& d = p->d;
+    if (d.epilogue != NK_EPI_NONE && (!hbias || !dbias)) return NK_ERR_INVALID_ARG;
+    const size_t ein = d.in_dtype == NK_BF16 ? 2 : 4, eout = d.out_dtype == NK_BF16 ? 2 : 4;
+    cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+    DeviceGuard guard(d.device);
+    if (guard.err != cudaSuccess) { set_err(p, "cudaSetDevice", guard.err); return NK_ERR_DEVICE; }
+    cudaError_t e;
+    if ((e = cudaMemcpyAsync(dA, hA, ein * d.M * d.K, cudaMemcpyHostToDevice, st)) != cudaSuccess ||
+        (e = cudaMemcpyAsync(dB, hB, ein * d.K * d.N, cudaMemcpyHostToDevice, st)) != cudaSuccess) {
+        set_err(p, "H2D copy", e);
+        return NK_ERR_CUDA;
+    }
+    if (d.epilogue != NK_EPI_NONE &&
+        (e = cudaMemcpyAsync(dbias, hbias, ein * d.N, cudaMemcpyHostToDevice, st)) != cudaSuccess) {
+        set_err(p, "H2D copy", e);
+        return NK_ERR_CUDA;
+    }
+    nk_status_t s = nk_gemm_run(p, dA, dB, d.epilogue != NK_EPI_NONE ? dbias : nullptr, dC, workspace,
+                                workspace_bytes, cuda_stream);
+    if (s != NK_OK) return s;
+    if ((e = cudaMemcpyAsync(hC, dC, eout * d.M * d.N, cudaMemcpyDeviceToHost, st)) != cudaSuccess ||
+        (e = cudaStreamSynchronize(st)) != cudaSuccess) {
+        set_err(p, "D2H copy / sync", e);
+        return NK_ERR_CUDA;
+    }
+    return NK_OK;
+}
+
+nk_status_t nk_gemm_check(nk_gemm_t p) {
+    if (!p) return NK_ERR_INVALID_ARG;
+    DeviceGuard guard(p->d.device);
+    if (guard.err != cudaSuccess) return NK_ERR_DEVICE;
+    cudaError_t e = cudaDeviceSynchronize();
+    if (e != cudaSuccess) { set_err(p, "cudaDeviceSynchronize", e); return NK_ERR_CUDA; }
+    unsigned int w = 0;
+    e = cudaMemcpy(&w, p->status_dev, sizeof(w), cudaMemcpyDeviceToHost);
+    if (e != cudaSuccess) { set_err(p, "status read", e); return NK_ERR_CUDA; }
+    if (w != 0) {
+        snprintf(p->cuda_err, sizeof(p->cuda_err), "device wait gave up, code 0x%x", w);
+        unsigned int z = 0;
+        cudaMemcpy(p->status_dev, &z, sizeof(z), cudaMemcpyHostToDevice);
+        return NK_ERR_TIMEOUT;
+    }
+    return NK_OK;
+}
+
+nk_status_t nk_gemm_destroy(nk_gemm_t p) {
+    delete p;
+    return NK_OK;
+}
+
+}  // extern "C"

@@ -1,0 +1,162 @@
+// FP32 GEMM on the FMA pipe (B200 has no exact-FP32 tensor-core MMA).
+//
+// This is the FP32 body of the paper's Algorithm 1 ("broadcast the A sub-column,
+// load a B chunk, FMA into the resident accumulators") in its outer-product form:
+// each thread keeps a TM x TN block of C in registers for the whole K loop and,
+// per k, reads TM values of A and TN values of B from shared memory with 128-bit
+// loads.  Tiles are double-buffered through registers so the global loads of
+// k-tile t+1 are in flight while k-tile t is multiplied.
+#pragma once
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+namespace nk {
+
+constexpr int SIMT_BK = 16;
+
+struct SimtParams {
+    int M, N, K;
+    int splits;        // gridDim.z; > 1 writes partials
+    int kt_per_split;  // k-tiles (of 16) per split
+    int epilogue;      // 0 none, 1 bias + ReLU
+    const float* A;    // [M][K]
+    const float* B;    // [K][N]
+    const float* bias; // [N] or null
+    float* C;          // [M][N]
+    float* partial;    // [splits][M][N]
+};
+
+template <int BM, int BN, int TM, int TN>
+__global__ void __launch_bounds__((BM / TM) * (BN / TN))
+simt_f32_kernel(const SimtParams p) {
+    constexpr int THREADS = (BM / TM) * (BN / TN);
+    constexpr int TX = BN / TN;          // threads across N
+    constexpr int GM = TM / 4, GN = TN / 4;  // 4-wide groups per thread
+    constexpr int SM_STRIDE = BM / GM;   // row distance between a thread's groups
+    constexpr int SN_STRIDE = BN / GN;
+    constexpr int AP = BM + 4;           // padded row length of the transposed A tile
+    constexpr int A_V4 = BM * SIMT_BK / 4 / THREADS;  // float4 loads per thread per tile
+    constexpr int B_V4 = BN * SIMT_BK / 4 / THREADS;
+    static_assert(TM % 4 == 0 && TN % 4 == 0, "thread tile is built from 4-wide groups");
+    static_assert(A_V4 >= 1 && B_V4 >= 1, "tile too small for the thread count");
+
+    __shared__ __align__(16) float As[2][SIMT_BK][AP];  // As[k][m]
+    __shared__ __align__(16) float Bs[2][SIMT_BK][BN];  // Bs[k][n]
+
+    const int t = threadIdx.x;
+    const int ty = t / TX, tx = t % TX;
+    const int m0 = blockIdx.y * BM, n0 = blockIdx.x * BN;
+    const int ktiles = (p.K + SIMT_BK - 1) / SIMT_BK;
+    const int kt0 = blockIdx.z * p.kt_per_split;
+    const int kt1 = min(ktiles, kt0 + p.kt_per_split);
+
+    float acc[TM][TN];
+#pragma unroll
+    for (int i = 0; i < TM; ++i)
+#pragma unroll
+        for (int j = 0; j < TN; ++j) acc[i][j] = 0.0f;
+
+    float4 ra[A_V4], rb[B_V4];
+
+    auto load_global = [&](int kt) {
+        const int k0 = kt * SIMT_BK;
+#pragma unroll
+        for (int i = 0; i < A_V4; ++i) {
+            const int idx = t + i * THREADS;       // over BM x 4 float4s
+            const int row = idx >> 2, kq = (idx & 3) * 4;
+            const int gm = m0 + row, gk = k0 + kq;
+            ra[i] = (gm < p.M && gk < p.K)
+                        ? __ldg(reinterpret_cast<const float4*>(p.A + static_cast<size_t>(gm) * p.K + gk))
+                        : make_float4(0.f, 0.f, 0.f, 0.f);
+        }
+#pragma unroll
+        for (int i = 0; i < B_V4; ++i) {
+            const int idx = t + i * THREADS;       // over 16 x BN/4 float4s
+            const int kr = idx / (BN / 4), nq = (idx % (BN / 4)) * 4;
+            const int gk = k0 + kr, gn = n0 + nq;
+            rb[i] = (gk < p.K && gn < p.N)
+                        ? __ldg(reinterpret_cast<const float4*>(p.B + static_cast<size_t>(gk) * p.N + gn))
+                        : make_float4(0.f, 0.f, 0.f, 0.f);
+        }
+    };
+    auto store_shared = [&](int buf) {
+#pragma unroll
+        for (int i = 0; i < A_V4; ++i) {
+            const int idx = t + i * THREADS;
+            const int row = idx >> 2, kq = (idx & 3) * 4;
+            As[buf][kq + 0][row] = ra[i].x;
+            As[buf][kq + 1][row] = ra[i].y;
+            As[buf][kq + 2][row] = ra[i].z;
+            As[buf][kq + 3][row] = ra[i].w;
+        }
+#pragma unroll
+        for (int i = 0; i < B_V4; ++i) {
+            const int idx = t + i * THREADS;
+            const int kr = idx / (BN / 4), nq = (idx % (BN / 4)) * 4;
+            *reinterpret_cast<float4*>(&Bs[buf][kr][nq]) = rb[i];
+        }
+    };
+
+    int buf = 0;
+    if (kt0 < kt1) {
+        load_global(kt0);
+        store_shared(0);
+    }
+    __syncthreads();
+
+    for (int kt = kt0; kt < kt1; ++kt) {
+        const bool more = kt + 1 < kt1;
+        if (more) load_global(kt + 1);
+#pragma unroll
+        for (int k = 0; k < SIMT_BK; ++k) {
+            float a[TM], b[TN];
+#pragma unroll
+            for (int g = 0; g < GM; ++g) {
+                const float4 v = *reinterpret_cast<const float4*>(&As[buf][k][g * SM_STRIDE + ty * 4]);
+                a[4 * g] = v.x; a[4 * g + 1] = v.y; a[4 * g + 2] = v.z; a[4 * g + 3] = v.w;
+            }
+#pragma unroll
+            for (int g = 0; g < GN; ++g) {
+                const float4 v = *reinterpret_cast<const float4*>(&Bs[buf][k][g * SN_STRIDE + tx * 4]);
+                b[4 * g] = v.x; b[4 * g + 1] = v.y; b[4 * g + 2] = v.z; b[4 * g + 3] = v.w;
+            }
+#pragma unroll
+            for (int i = 0; i < TM; ++i)
+#pragma unroll
+                for (int j = 0; j < TN; ++j) acc[i][j] = fmaf(a[i], b[j], acc[i][j]);
+        }
+        if (more) {
+            store_shared(buf ^ 1);
+            __syncthreads();
+            buf ^= 1;
+        }
+    }
+
+    // Epilogue: bias + ReLU on the accumulator, then the single store of C.
+    const bool to_partial = p.splits > 1;
+    float* out = to_partial ? p.partial + static_cast<size_t>(blockIdx.z) * p.M * p.N : p.C;
+#pragma unroll
+    for (int gi = 0; gi < GM; ++gi)
+#pragma unroll
+        for (int ii = 0; ii < 4; ++ii) {
+            const int gm = m0 + gi * SM_STRIDE + ty * 4 + ii;
+            if (gm >= p.M) continue;
+#pragma unroll
+            for (int gj = 0; gj < GN; ++gj) {
+                const int gn = n0 + gj * SN_STRIDE + tx * 4;
+                if (gn >= p.N) continue;
+                float4 v = make_float4(acc[4 * gi + ii][4 * gj], acc[4 * gi + ii][4 * gj + 1],
+                                       acc[4 * gi + ii][4 * gj + 2], acc[4 * gi + ii][4 * gj + 3]);
+                if (!to_partial && p.epilogue) {
+                    const float4 bv = __ldg(reinterpret_cast<const float4*>(p.bias + gn));
+                    v.x = fmaxf(v.x + bv.x, 0.f);
+                    v.y = fmaxf(v.y + bv.y, 0.f);
+                    v.z = fmaxf(v.z + bv.z, 0.f);
+                    v.w = fmaxf(v.w + bv.w, 0.f);
+                }
+                *reinterpret_cast<float4*>(out + static_cast<size_t>(gm) * p.N + gn) = v;
+            }
+        }
+}
+
+}  // namespace nk

@@ -1,0 +1,378 @@
+// BF16 x BF16 -> FP32 GEMM on the 5th-generation tensor cores.
+//
+// Structure (Algorithm 1 of the paper, re-expressed for sm_100a): a persistent
+// CTA walks output tiles; for each tile the accumulator stays resident in tensor
+// memory over the whole K loop (Algorithm 1: the C sub-block is held across the
+// batch-reduce and K loops), operands are staged by TMA into a ring of swizzled
+// shared-memory tiles while earlier stages are being multiplied (the software
+// pipelining of Algorithm 3, AMX branch), and bias + ReLU are applied to the
+// accumulator before the single store of C (Section 6, "MLP").
+//
+// Warp roles (192 threads, +128 when B is VNNI-blocked):
+//   warp 0      TMA producer: A tile 128 x 64 (K-major), B tile 64 x BN (N-major)
+//   warp 1      MMA issuer and TMEM owner: 4 x tcgen05.mma 128 x BN x 16 per stage
+//   warps 2-5   epilogue: tcgen05.ld -> (+bias, ReLU, cvt) -> global stores; two
+//               TMEM accumulators so tile t's epilogue overlaps tile t+1's K loop
+//   warps 6-9   (VNNI-blocked B only) re-layout: read the [k/2][n][2] blocks from
+//               global memory as 32-bit words and write them word-transposed into
+//               the K-major swizzled stage (the in-kernel counterpart of the
+//               paper's software-pipelined pack step, in the opposite direction)
+//
+// Every mbarrier wait is bounded; a role that gives up raises the CTA's abort
+// flag and the device status word, the other roles fall out of their loops, and
+// the CTA frees its TMEM and exits.
+#pragma once
+#include <cuda.h>
+#include <cuda_bf16.h>
+#include "ptx.cuh"
+
+namespace nk {
+
+constexpr int UMMA_BM = 128;
+constexpr int UMMA_BK = 64;
+constexpr int UMMA_A_STAGE_BYTES = UMMA_BM * UMMA_BK * 2;  // 16 KB
+
+struct UmmaParams {
+    int M, N, K;
+    int tiles_m, tiles_n;
+    int splits;         // K splits; > 1 writes FP32 partials to `partial`
+    int kb_total;       // ceil(K / 64)
+    int kb_per_split;   // ceil(kb_total / splits)
+    int group_m;        // raster: this many M tiles sweep N together
+    int a_blocked;      // A tensor map is the 4-D blocked view
+    int epilogue;       // 0 none, 1 bias + ReLU
+    int out_bf16;       // C element type
+    uint32_t idesc;     // tcgen05 instruction descriptor
+    const void* bias;   // BF16 [N] or null
+    void* C;            // [M][N] FP32 or BF16
+    float* partial;     // [splits][M][N] when splits > 1
+    const uint32_t* Bblk;  // VNNI-blocked B as 32-bit words (B_VNNI kernels only)
+    unsigned int* status;
+};
+
+__host__ __device__ constexpr int umma_b_stage_bytes(int BN) { return BN * UMMA_BK * 2; }
+__host__ __device__ constexpr int umma_stage_bytes(int BN) {
+    return UMMA_A_STAGE_BYTES + umma_b_stage_bytes(BN);
+}
+__host__ __device__ constexpr int umma_smem_bytes(int BN, int stages) {
+    return stages * umma_stage_bytes(BN) + 1024 /*alignment slack*/ + 256 /*barriers*/;
+}
+
+// tile id -> (m block, n block): groups of `group_m` M tiles sweep across N so
+// that CTAs running at the same time share A rows and B columns in L2.
+__device__ __forceinline__ void umma_tile_coords(const UmmaParams& p, int tile, int& mb, int& nb) {
+    const int per_group = p.group_m * p.tiles_n;
+    const int g = tile / per_group;
+    const int within = tile - g * per_group;
+    const int first_m = g * p.group_m;
+    const int gm = min(p.group_m, p.tiles_m - first_m);
+    mb = first_m + within % gm;
+    nb = within / gm;
+}
+
+__device__ __forceinline__ float bf16_bits_to_f32(uint32_t h) { return __uint_as_float(h << 16); }
+
+__device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi) {
+    __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
+    return *reinterpret_cast<uint32_t*>(&v);
+}
+
+template <int BN, int STAGES, bool B_VNNI>
+__global__ void __launch_bounds__(B_VNNI ? 320 : 192, 1)
+umma_bf16_kernel(const __grid_constant__ CUtensorMap tmap_a,
+                 const __grid_constant__ CUtensorMap tmap_b, const UmmaParams p) {
+    static_assert(BN % 32 == 0 && BN >= 32 && BN <= 256, "tile N");
+    constexpr int B_STAGE = umma_b_stage_bytes(BN);
+    constexpr int STAGE = umma_stage_bytes(BN);
+    constexpr uint32_t TMEM_COLS = (2 * BN <= 32) ? 32 : (2 * BN <= 64) ? 64 : (2 * BN <= 128) ? 128
+                                   : (2 * BN <= 256) ? 256 : 512;
+
+    extern __shared__ uint8_t smem_raw[];
+    const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
+    const uint32_t bar_base = smem_base + STAGES * STAGE;
+    // barrier block: full[STAGES], empty[STAGES], tmem_full[2], tmem_empty[2], then 2 words
+    auto full_bar = [&](int s) { return bar_base + 8u * s; };
+    auto empty_bar = [&](int s) { return bar_base + 8u * (STAGES + s); };
+    auto tfull_bar = [&](int a) { return bar_base + 8u * (2 * STAGES + a); };
+    auto tempty_bar = [&](int a) { return bar_base + 8u * (2 * STAGES + 2 + a); };
+    uint8_t* gen_base = smem_raw + (smem_base - smem_u32(smem_raw));
+    volatile uint32_t* tmem_slot =
+        reinterpret_cast<volatile uint32_t*>(gen_base + STAGES * STAGE + 8 * (2 * STAGES + 4));
+    volatile uint32_t* abort_flag = tmem_slot + 1;
+
+    const int warp = threadIdx.x >> 5;
+    const int lane = threadIdx.x & 31;
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < STAGES; ++s) {
+            mbar_init(full_bar(s), B_VNNI ? 1 + 4 : 1);
+            mbar_init(empty_bar(s), 1);
+        }
+        for (int a = 0; a < 2; ++a) {
+            mbar_init(tfull_bar(a), 1);
+            mbar_init(tempty_bar(a), 128);
+        }
+        *abort_flag = 0;
+        fence_mbar_init();
+        tma_prefetch_desc(&tmap_a);
+        if (!B_VNNI) tma_prefetch_desc(&tmap_b);
+    }
+    if (warp == 1) {
+        tmem_alloc(smem_u32(const_cast<uint32_t*>(tmem_slot)), TMEM_COLS);
+        tmem_relinquish();
+    }
+    tc_fence_before_sync();
+    __syncthreads();
+    tc_fence_after_sync();
+    const uint32_t tmem_base = *tmem_slot;
+
+    const int total_units = p.tiles_m * p.tiles_n * p.splits;
+
+    auto give_up = [&](unsigned int code) {
+        *abort_flag = 1;
+        if (p.status) atomicCAS(p.status, 0u, code);
+    };
+
+    if (warp == 0) {
+        // ------------------------------------------------ TMA producer
+        int stage = 0;
+        uint32_t phase = 0;
+        bool ok = true;
+        for (int unit = blockIdx.x; ok && unit < total_units; unit += gridDim.x) {
+            const int tile = unit / p.splits, split = unit - tile * p.splits;
+            int mb, nb;
+            umma_tile_coords(p, tile, mb, nb);
+            const int kb0 = split * p.kb_per_split;
+            const int kb1 = min(p.kb_total, kb0 + p.kb_per_split);
+            for (int kb = kb0; kb < kb1; ++kb) {
+                if (!mbar_wait(empty_bar(stage), phase ^ 1u, abort_flag)) {
+                    if (lane == 0) give_up(0x100u + stage);
+                    ok = false;
+                    break;
+                }
+                if (lane == 0) {
+                    const uint32_t sa = smem_base + stage * STAGE;
+                    const uint32_t sb = sa + UMMA_A_STAGE_BYTES;
+                    mbar_arrive_expect_tx(full_bar(stage),
+                                          UMMA_A_STAGE_BYTES + (B_VNNI ? 0 : B_STAGE));
+                    if (p.a_blocked)
+                        tma_load_4d(sa, &tmap_a, full_bar(stage), 0, kb * 2, 0, mb * 4);
+                    else
+                        tma_load_2d(sa, &tmap_a, full_bar(stage), kb * UMMA_BK, mb * UMMA_BM);
+                    if (!B_VNNI) {
+#pragma unroll
+                        for (int j = 0; j < BN / 64; ++j)
+                            tma_load_2d(sb + j * 8192, &tmap_b, full_bar(stage), nb * BN + j * 64,
+                                        kb * UMMA_BK);
+                    }
+                }
+                __syncwarp();
+                if (++stage == STAGES) { stage = 0; phase ^= 1u; }
+            }
+        }
+        // Drain: wait (bounded) until the consumer has released every stage this warp
+        // filled, so no TMA write is in flight when the CTA's shared memory is freed.
+        if (ok) {
+            for (int s = 0; s < STAGES; ++s) {
+                if (!mbar_wait(empty_bar(stage), phase ^ 1u, abort_flag)) break;
+                if (++stage == STAGES) { stage = 0; phase ^= 1u; }
+            }
+        }
+    } else if (warp == 1) {
+        // ------------------------------------------------ MMA issuer
+        int stage = 0;
+        uint32_t phase = 0;
+        int local = 0;
+        bool ok = true;
+        for (int unit = blockIdx.x; ok && unit < total_units; unit += gridDim.x, ++local) {
+            const int tile = unit / p.splits, split = unit - tile * p.splits;
+            const int kb0 = split * p.kb_per_split;
+            const int kb1 = min(p.kb_total, kb0 + p.kb_per_split);
+            const int acc = local & 1;
+            if (!mbar_wait(tempty_bar(acc), ((local >> 1) & 1u) ^ 1u, abort_flag)) {
+                if (lane == 0) give_up(0x200u + acc);
+                ok = false;
+                break;
+            }
+            tc_fence_after_sync();
+            const uint32_t d_tmem = tmem_base + acc * BN;
+            for (int kb = kb0; kb < kb1; ++kb) {
+                if (!mbar_wait(full_bar(stage), phase, abort_flag)) {
+                    if (lane == 0) give_up(0x300u + stage);
+                    ok = false;
+                    break;
+                }
+                tc_fence_after_sync();
+                if (lane == 0) {
+                    const uint32_t sa = smem_base + stage * STAGE;
+                    const uint32_t sb = sa + UMMA_A_STAGE_BYTES;
+                    // A: K-major, 128-byte swizzle, 8-row groups 1024 B apart.
+                    const uint64_t da = make_smem_desc(sa, 16, 1024, 2);
+                    // B row-major [K][N]: N-major, 64-column atoms 8192 B apart (leading),
+                    // 8-k groups 1024 B apart (stride).  B re-laid from VNNI: K-major like A.
+                    const uint64_t db = B_VNNI ? make_smem_desc(sb, 16, 1024, 2)
+                                               : make_smem_desc(sb, 8192, 1024, 2);
+#pragma unroll
+                    for (int k4 = 0; k4 < UMMA_BK / 16; ++k4) {
+                        const uint64_t a_adv = static_cast<uint64_t>(k4 * 2);  // 32 B
+                        const uint64_t b_adv =
+                            static_cast<uint64_t>(B_VNNI ? k4 * 2 : k4 * 128);  // 32 B | 2048 B
+                        umma_f16(d_tmem, da + a_adv, db + b_adv, p.idesc,
+                                 (kb > kb0 || k4 > 0) ? 1u : 0u);
+                    }
+                    umma_commit(empty_bar(stage));
+                    if (kb == kb1 - 1) umma_commit(tfull_bar(acc));
+                }
+                __syncwarp();
+                if (++stage == STAGES) { stage = 0; phase ^= 1u; }
+            }
+            if (kb1 <= kb0 && lane == 0) umma_commit(tfull_bar(acc));  // empty K range
+            __syncwarp();
+        }
+    } else if (warp < 6) {
+        // ------------------------------------------------ epilogue
+        const int quarter = warp & 3;  // TMEM lanes 32*quarter .. +31 belong to this warp
+        int local = 0;
+        bool ok = true;
+        for (int unit = blockIdx.x; ok && unit < total_units; unit += gridDim.x, ++local) {
+            const int tile = unit / p.splits, split = unit - tile * p.splits;
+            int mb, nb;
+            umma_tile_coords(p, tile, mb, nb);
+            const int kb0 = split * p.kb_per_split;
+            const int kb1 = min(p.kb_total, kb0 + p.kb_per_split);
+            const int acc = local & 1;
+            if (!mbar_wait(tfull_bar(acc), (local >> 1) & 1u, abort_flag)) {
+                if (lane == 0) give_up(0x400u + acc);
+                ok = false;
+                break;
+            }
+            tc_fence_after_sync();
+            const int row = mb * UMMA_BM + quarter * 32 + lane;
+            const bool row_ok = row < p.M;
+            const bool to_partial = p.splits > 1;
+            const bool empty_k = kb1 <= kb0;
+            const size_t row_off = static_cast<size_t>(row) * p.N;
+#pragma unroll 1
+            for (int c0 = 0; c0 < BN; c0 += 32) {
+                uint32_t v[32];
+                tmem_ld_32x32(tmem_base + acc * BN + c0 + (static_cast<uint32_t>(quarter * 32) << 16),
+                              v);
+                tmem_ld_wait();
+                const int col0 = nb * BN + c0;
+                if (row_ok && col0 < p.N) {
+                if (empty_k) {
+#pragma unroll
+                    for (int i = 0; i < 32; ++i) v[i] = 0u;
+                }
+                if (to_partial) {
+                    float* dst = p.partial + static_cast<size_t>(split) * p.M * p.N + row_off + col0;
+#pragma unroll
+                    for (int g = 0; g < 8; ++g)
+                        if (col0 + 4 * g < p.N)
+                            *reinterpret_cast<uint4*>(dst + 4 * g) =
+                                make_uint4(v[4 * g], v[4 * g + 1], v[4 * g + 2], v[4 * g + 3]);
+                } else {
+                if (p.epilogue) {
+                    const uint4* bsrc = reinterpret_cast<const uint4*>(
+                        static_cast<const uint16_t*>(p.bias) + col0);
+#pragma unroll
+                    for (int g = 0; g < 4; ++g) {
+                        if (col0 + 8 * g >= p.N) break;
+                        const uint4 b = __ldg(bsrc + g);
+                        const uint32_t w[4] = {b.x, b.y, b.z, b.w};
+#pragma unroll
+                        for (int j = 0; j < 4; ++j) {
+                            float x0 = __uint_as_float(v[8 * g + 2 * j]) + bf16_bits_to_f32(w[j] & 0xFFFFu);
+                            float x1 = __uint_as_float(v[8 * g + 2 * j + 1]) + bf16_bits_to_f32(w[j] >> 16);
+                            v[8 * g + 2 * j] = __float_as_uint(fmaxf(x0, 0.0f));
+                            v[8 * g + 2 * j + 1] = __float_as_uint(fmaxf(x1, 0.0f));
+                        }
+                    }
+                }
+                if (p.out_bf16) {
+                    uint16_t* dst = static_cast<uint16_t*>(p.C) + row_off + col0;
+#pragma unroll
+                    for (int g = 0; g < 4; ++g)
+                        if (col0 + 8 * g < p.N) {
+                            uint4 o;
+                            o.x = pack_bf16x2(__uint_as_float(v[8 * g]), __uint_as_float(v[8 * g + 1]));
+                            o.y = pack_bf16x2(__uint_as_float(v[8 * g + 2]), __uint_as_float(v[8 * g + 3]));
+                            o.z = pack_bf16x2(__uint_as_float(v[8 * g + 4]), __uint_as_float(v[8 * g + 5]));
+                            o.w = pack_bf16x2(__uint_as_float(v[8 * g + 6]), __uint_as_float(v[8 * g + 7]));
+                            *reinterpret_cast<uint4*>(dst + 8 * g) = o;
+                        }
+                } else {
+                    float* dst = static_cast<float*>(p.C) + row_off + col0;
+#pragma unroll
+                    for (int g = 0; g < 8; ++g)
+                        if (col0 + 4 * g < p.N)
+                            *reinterpret_cast<uint4*>(dst + 4 * g) =
+                                make_uint4(v[4 * g], v[4 * g + 1], v[4 * g + 2], v[4 * g + 3]);
+                }
+                }  // direct store
+                }  // in range
+                __syncwarp();
+            }
+            tc_fence_before_sync();
+            mbar_arrive(tempty_bar(acc));
+        }
+    } else if (B_VNNI) {
+        // ------------------------------------------------ VNNI re-layout warps (6..9)
+        // Stage tile: BN rows (n) x 64 k, K-major, 128-byte rows, 16-byte chunk c of row n
+        // stored at chunk c ^ (n & 7).  A 32 x 32 block of B is 16 rows (k/2) of 32 words
+        // (n); word (k2, n) goes to row n, byte offset (kb_local*32 + 2*k2) * 2.
+        const int tw = warp - 6;
+        int stage = 0;
+        uint32_t phase = 0;
+        bool ok = true;
+        const int kblocks32 = p.K / 32;
+        for (int unit = blockIdx.x; ok && unit < total_units; unit += gridDim.x) {
+            const int tile = unit / p.splits, split = unit - tile * p.splits;
+            int mb, nb;
+            umma_tile_coords(p, tile, mb, nb);
+            const int kb0 = split * p.kb_per_split;
+            const int kb1 = min(p.kb_total, kb0 + p.kb_per_split);
+            for (int kb = kb0; kb < kb1; ++kb) {
+                if (!mbar_wait(empty_bar(stage), phase ^ 1u, abort_flag)) {
+                    if (lane == 0) give_up(0x500u + stage);
+                    ok = false;
+                    break;
+                }
+                uint8_t* sb = gen_base + stage * STAGE + UMMA_A_STAGE_BYTES;
+                // work items: (n-block j, k-block half h, quad q) -> 4 words k2 = 4q..4q+3 at n = lane
+                constexpr int ITEMS = (BN / 32) * 2 * 4;
+#pragma unroll 4
+                for (int it = tw; it < ITEMS; it += 4) {
+                    const int q = it & 3, h = (it >> 2) & 1, j = it >> 3;
+                    const int nblk = nb * (BN / 32) + j;
+                    const int kblk = kb * 2 + h;
+                    uint4 w = make_uint4(0u, 0u, 0u, 0u);
+                    if (nblk * 32 < p.N && kblk < kblocks32) {
+                        const uint32_t* src = p.Bblk +
+                            ((static_cast<size_t>(nblk) * kblocks32 + kblk) * 16 + 4 * q) * 32 + lane;
+                        w.x = __ldg(src);
+                        w.y = __ldg(src + 32);
+                        w.z = __ldg(src + 64);
+                        w.w = __ldg(src + 96);
+                    }
+                    const int n = j * 32 + lane;
+                    const int chunk = (h * 4 + q) ^ (n & 7);
+                    *reinterpret_cast<uint4*>(sb + n * 128 + chunk * 16) = w;
+                }
+                fence_proxy_async_smem();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(full_bar(stage));
+                if (++stage == STAGES) { stage = 0; phase ^= 1u; }
+            }
+        }
+    }
+
+    tc_fence_before_sync();
+    __syncthreads();
+    if (warp == 1) {
+        tc_fence_after_sync();
+        tmem_dealloc(tmem_base, TMEM_COLS);
+    }
+}
+
+}  // namespace nk

@@ -1,0 +1,183 @@
+"""GPU parity: every kernel variant through the C ABI against the CPU oracle.
+
+Small cases use integer-valued operands (exact in FP32 accumulation, so the
+comparison is bit-exact and any addressing mistake is unmistakable) and random
+operands under the acceptance bound; shapes span several tiles, ragged tails in
+M, N and K, and the degenerate sizes (one row, one k-block, K smaller than a
+stage)."""
+import numpy as np
+import pytest
+import torch
+
+import nk_inputs
+import paper_2511_13764_b200 as nk
+from nk_testlib import run_and_check, run_plan, check_against_oracle
+
+pytestmark = pytest.mark.gpu
+
+INT = ("int", 1.0)
+
+
+def W(name, M, N, K, in_dtype="bf16", out_dtype="f32", layout="row", epilogue="none", integer=False,
+      seed=1):
+    kw = {}
+    if integer:
+        kw = dict(dist_a=INT, dist_b=INT, dist_bias=INT)
+    return nk_inputs.Workload(name, M, N, K, in_dtype, out_dtype, layout, epilogue, seed=seed, **kw)
+
+
+# ---------------------------------------------------------------- naive (debug) kernel
+@pytest.mark.parametrize("in_dtype,layout,out_dtype,epi", [
+    ("f32", "row", "f32", "none"), ("f32", "row", "f32", "bias_relu"),
+    ("bf16", "row", "f32", "none"), ("bf16", "blocked32", "f32", "none"),
+    ("bf16", "blocked32", "bf16", "bias_relu"),
+])
+def test_naive_kernel(in_dtype, layout, out_dtype, epi):
+    w = W("naive", 64, 96, 160, in_dtype, out_dtype, layout, epi, integer=True)
+    run_and_check(w, flags=nk.FLAG_KERNEL_NAIVE, exact=(out_dtype == "f32"), expect_kernel="naive")
+    w = W("naive", 64, 96, 160, in_dtype, out_dtype, layout, epi)
+    run_and_check(w, flags=nk.FLAG_KERNEL_NAIVE)
+
+
+# ---------------------------------------------------------------- FP32 SIMT kernel
+SIMT_SHAPES = [(256, 256, 256), (1, 4, 4), (33, 132, 68), (128, 128, 16), (130, 260, 100),
+               (16, 1024, 1024), (300, 520, 40), (512, 384, 1000)]
+
+
+@pytest.mark.parametrize("tile", [1, 2, 3])
+@pytest.mark.parametrize("shape", SIMT_SHAPES)
+def test_simt_f32_exact_integer(shape, tile):
+    M, N, K = shape
+    w = W("simt", M, N, K, "f32", integer=True)
+    run_and_check(w, flags=nk.FLAG_KERNEL_SIMT | nk.flag_tile_n(tile), exact=True, expect_kernel="simt_f32")
+
+
+@pytest.mark.parametrize("shape", SIMT_SHAPES)
+def test_simt_f32_random_auto(shape):
+    M, N, K = shape
+    run_and_check(W("simt", M, N, K, "f32", seed=3))
+
+
+@pytest.mark.parametrize("splits", [2, 5])
+@pytest.mark.parametrize("epi", ["none", "bias_relu"])
+def test_simt_f32_splitk(splits, epi):
+    w = W("simt", 100, 200, 1000, "f32", epilogue=epi, integer=True)
+    err, plan = run_and_check(w, flags=nk.flag_splitk(splits) | nk.flag_tile_n(2), exact=True)
+    assert f"splitk{splits}" in plan.kernel_name and plan.workspace_bytes >= splits * 100 * 200 * 4
+    run_and_check(W("simt", 100, 200, 1000, "f32", epilogue=epi, seed=4), flags=nk.flag_splitk(splits))
+
+
+def test_simt_f32_bias_relu():
+    run_and_check(W("simt", 130, 260, 100, "f32", epilogue="bias_relu", integer=True), exact=True)
+    run_and_check(W("simt", 512, 1024, 1024, "f32", epilogue="bias_relu", seed=5))
+
+
+# ---------------------------------------------------------------- BF16 tcgen05 kernel
+UMMA_SHAPES = [(128, 64, 64), (128, 256, 64), (128, 64, 256), (256, 512, 1024), (100, 64, 64),
+               (1, 8, 8), (130, 72, 72), (384, 328, 200), (1024, 1024, 1024), (16, 2048, 512)]
+
+
+@pytest.mark.parametrize("tile", [2, 3, 4])
+@pytest.mark.parametrize("shape", UMMA_SHAPES)
+def test_umma_bf16_exact_integer(shape, tile):
+    M, N, K = shape
+    w = W("umma", M, N, K, "bf16", integer=True)
+    run_and_check(w, flags=nk.flag_tile_n(tile), exact=True, expect_kernel=f"umma_bf16_128x{32 << (tile - 1)}")
+
+
+@pytest.mark.parametrize("shape", UMMA_SHAPES)
+def test_umma_bf16_random_auto(shape):
+    M, N, K = shape
+    run_and_check(W("umma", M, N, K, "bf16", seed=7))
+
+
+@pytest.mark.parametrize("out_dtype", ["f32", "bf16"])
+@pytest.mark.parametrize("epi", ["none", "bias_relu"])
+def test_umma_bf16_epilogues(out_dtype, epi):
+    w = W("umma", 200, 328, 264, "bf16", out_dtype, epilogue=epi, integer=(out_dtype == "f32"))
+    run_and_check(w, exact=(out_dtype == "f32"))
+    run_and_check(W("umma", 256, 512, 512, "bf16", out_dtype, epilogue=epi, seed=8))
+
+
+@pytest.mark.parametrize("splits", [2, 3, 7])
+@pytest.mark.parametrize("out_dtype,epi", [("f32", "none"), ("bf16", "bias_relu")])
+def test_umma_bf16_splitk(splits, out_dtype, epi):
+    w = W("umma", 130, 200, 1096, "bf16", out_dtype, epilogue=epi, integer=(out_dtype == "f32"))
+    err, plan = run_and_check(w, flags=nk.flag_splitk(splits), exact=(out_dtype == "f32"))
+    assert "splitk" in plan.kernel_name and plan.workspace_bytes > 0
+    run_and_check(W("umma", 130, 200, 1096, "bf16", out_dtype, epilogue=epi, seed=9), flags=nk.flag_splitk(splits))
+
+
+@pytest.mark.parametrize("tile", [2, 3, 4])
+@pytest.mark.parametrize("flags", [0, nk.FLAG_REPACK_B], ids=["inkernel", "repack"])
+@pytest.mark.parametrize("shape", [(128, 64, 64), (32, 32, 32), (160, 224, 96), (512, 512, 512)])
+def test_umma_bf16_blocked(shape, flags, tile):
+    M, N, K = shape
+    w = W("blk", M, N, K, "bf16", layout="blocked32", integer=True)
+    err, plan = run_and_check(w, flags=flags | nk.flag_tile_n(tile), exact=True)
+    assert "_ablk" in plan.kernel_name
+    run_and_check(W("blk", M, N, K, "bf16", layout="blocked32", seed=10), flags=flags | nk.flag_tile_n(tile))
+
+
+def test_blocked_mixed_layouts():
+    """A blocked with B row-major, and A row-major with B blocked."""
+    import oracle
+    M, N, K = 160, 224, 96
+    w = W("mix", M, N, K, "bf16", integer=True)
+    A, B, _ = w.make()
+    for la, lb in ((nk.BLOCKED32, nk.ROW_MAJOR), (nk.ROW_MAJOR, nk.BLOCKED32)):
+        plan = nk.Plan(M, N, K, nk.BF16, nk.F32, la, lb)
+        got, _ = run_plan(w, A, B, None, plan=plan)
+        Y, _ = oracle.gemm(M, N, K, A, B, in_dtype=oracle.BF16, layout_a=la, layout_b=lb)
+        assert np.array_equal(got, Y)
+
+
+def test_repeatable_bit_for_bit():
+    w = W("rep", 512, 768, 2048, "bf16", seed=12)
+    A, B, bias = w.make()
+    c1, plan = run_plan(w, A, B, bias)
+    c2, _ = run_plan(w, A, B, bias, plan=plan)
+    assert np.array_equal(c1, c2)
+    w = W("rep", 256, 256, 512, "f32", seed=13)
+    A, B, bias = w.make()
+    c1, plan = run_plan(w, A, B, bias, flags=nk.flag_splitk(4))
+    c2, _ = run_plan(w, A, B, bias, plan=plan)
+    assert np.array_equal(c1, c2)
+
+
+def test_run_host_entry_point():
+    w = W("host", 256, 320, 192, "bf16", "bf16", epilogue="bias_relu", seed=14)
+    A, B, bias = w.make()
+    plan = nk.plan_for(w)
+    hA = torch.from_numpy(A).pin_memory()
+    hB = torch.from_numpy(B).pin_memory()
+    hb = torch.from_numpy(bias).pin_memory()
+    hC = torch.empty(w.M * w.N, dtype=torch.int16).pin_memory()
+    dA = torch.empty(A.size, dtype=torch.int16, device="cuda")
+    dB = torch.empty(B.size, dtype=torch.int16, device="cuda")
+    db = torch.empty(bias.size, dtype=torch.int16, device="cuda")
+    dC = torch.empty(w.M * w.N, dtype=torch.int16, device="cuda")
+    ws_bytes = plan.workspace_bytes
+    ws = torch.empty(max(ws_bytes, 16), dtype=torch.uint8, device="cuda")
+    plan.run_host(hA, hB, hC, dA, dB, dC, hbias=hb, dbias=db, workspace=ws, workspace_bytes=ws_bytes,
+                  stream=torch.cuda.current_stream().cuda_stream)
+    plan.check()
+    got = (hC.numpy().view(np.uint16).astype(np.uint32) << 16).view(np.float32).astype(np.float64)
+    check_against_oracle(w, got.reshape(w.M, w.N), A, B, bias)
+
+
+def test_runtime_argument_errors():
+    plan = nk.Plan(128, 128, 128, nk.BF16, nk.F32, epilogue=nk.EPI_BIAS_RELU)
+    x = torch.zeros(128 * 128, dtype=torch.bfloat16, device="cuda")
+    c = torch.zeros(128 * 128, dtype=torch.float32, device="cuda")
+    with pytest.raises(nk.NkError) as e:
+        plan.run(x, x, c, bias=None)
+    assert e.value.status == 1
+    with pytest.raises(nk.NkError) as e:
+        plan.run(x.data_ptr() + 2, x, c, bias=x)
+    assert e.value.status == 3
+    plan2 = nk.Plan(128, 128, 1024, nk.BF16, nk.F32, flags=nk.flag_splitk(4))
+    assert plan2.workspace_bytes > 0
+    with pytest.raises(nk.NkError) as e:
+        plan2.run(x, x, c)
+    assert e.value.status == 4
