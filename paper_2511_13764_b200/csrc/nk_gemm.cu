@@ -178,14 +178,14 @@ static nk_status_t encode_maps(nk_gemm_s* p, const void* A, const void* B) {
     const nk_gemm_desc_t& d = p->d;
     CUresult r;
     if (d.layout_a == NK_BLOCKED32) {
-        // [M/32][K/32][32][32] viewed with dims (k, k-block, m, m-block): a box of
-        // 32 x 2 x 32 x 4 lands in shared memory as 128 rows of 64 consecutive k.
-        cuuint64_t dims[4] = {32, static_cast<cuuint64_t>(d.K / 32), 32, static_cast<cuuint64_t>(d.M / 32)};
-        cuuint64_t strides[3] = {1024 * 2, 32 * 2, static_cast<cuuint64_t>(d.K / 32) * 1024 * 2};
-        cuuint32_t box[4] = {32, 2, 32, 4};
+        // [M/32][K/32][32][32] as a 4-D tensor (k, m, k-block, m-block): a box of
+        // 32 x 32 x 1 x 4 lands in shared memory as 128 rows of 32 consecutive k (64 B).
+        cuuint64_t dims[4] = {32, 32, static_cast<cuuint64_t>(d.K / 32), static_cast<cuuint64_t>(d.M / 32)};
+        cuuint64_t strides[3] = {32 * 2, 1024 * 2, static_cast<cuuint64_t>(d.K / 32) * 1024 * 2};
+        cuuint32_t box[4] = {32, 32, 1, 4};
         cuuint32_t es[4] = {1, 1, 1, 1};
         r = p->encode(&p->tmap_a, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void*>(A), dims, strides,
-                      box, es, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+                      box, es, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_64B,
                       CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
     } else {
         cuuint64_t dims[2] = {static_cast<cuuint64_t>(d.K), static_cast<cuuint64_t>(d.M)};

@@ -155,9 +155,11 @@ umma_bf16_kernel(const __grid_constant__ CUtensorMap tmap_a,
                     const uint32_t sb = sa + UMMA_A_STAGE_BYTES;
                     mbar_arrive_expect_tx(full_bar(stage),
                                           UMMA_A_STAGE_BYTES + (B_VNNI ? 0 : B_STAGE));
-                    if (p.a_blocked)
-                        tma_load_4d(sa, &tmap_a, full_bar(stage), 0, kb * 2, 0, mb * 4);
-                    else
+                    if (p.a_blocked) {
+                        // two 32-wide K slabs, each 128 rows x 64 B (64-byte swizzle)
+                        tma_load_4d(sa, &tmap_a, full_bar(stage), 0, 0, kb * 2, mb * 4);
+                        tma_load_4d(sa + 8192, &tmap_a, full_bar(stage), 0, 0, kb * 2 + 1, mb * 4);
+                    } else
                         tma_load_2d(sa, &tmap_a, full_bar(stage), kb * UMMA_BK, mb * UMMA_BM);
                     if (!B_VNNI) {
 #pragma unroll
@@ -206,15 +208,18 @@ umma_bf16_kernel(const __grid_constant__ CUtensorMap tmap_a,
                 if (lane == 0) {
                     const uint32_t sa = smem_base + stage * STAGE;
                     const uint32_t sb = sa + UMMA_A_STAGE_BYTES;
-                    // A: K-major, 128-byte swizzle, 8-row groups 1024 B apart.
-                    const uint64_t da = make_smem_desc(sa, 16, 1024, 2);
+                    // A row-major: K-major tile, 128-byte swizzle, 8-row groups 1024 B apart.
+                    // A blocked: two K-major slabs of 32 k, 64-byte swizzle, 8-row groups 512 B apart.
+                    const uint64_t da = p.a_blocked ? make_smem_desc(sa, 16, 512, 4)
+                                                    : make_smem_desc(sa, 16, 1024, 2);
                     // B row-major [K][N]: N-major, 64-column atoms 8192 B apart (leading),
                     // 8-k groups 1024 B apart (stride).  B re-laid from VNNI: K-major like A.
                     const uint64_t db = B_VNNI ? make_smem_desc(sb, 16, 1024, 2)
                                                : make_smem_desc(sb, 8192, 1024, 2);
 #pragma unroll
                     for (int k4 = 0; k4 < UMMA_BK / 16; ++k4) {
-                        const uint64_t a_adv = static_cast<uint64_t>(k4 * 2);  // 32 B
+                        const uint64_t a_adv = static_cast<uint64_t>(
+                            p.a_blocked ? (k4 >> 1) * 512 + (k4 & 1) * 2 : k4 * 2);  // 32 B steps
                         const uint64_t b_adv =
                             static_cast<uint64_t>(B_VNNI ? k4 * 2 : k4 * 128);  // 32 B | 2048 B
                         umma_f16(d_tmem, da + a_adv, db + b_adv, p.idesc,
