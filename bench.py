@@ -1,0 +1,299 @@
+#!/usr/bin/env python
+"""Benchmark of the dense-GEMM hot path on B200.
+
+A step is one pass of the whole path (tile loop, operand staging, K loop with
+the accumulator resident, epilogue, store) over one batch of synthetic input:
+the BF16 GEMM M = N = K = 8192 with FP32 output.  With N GPUs every rank owns
+its own 8192-row block of A (M-sharded, B replicated: no collective on the data
+path), so per-GPU work is fixed ("weak" scaling) and `value` sums all ranks.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference]
+
+Prints ONE JSON line on rank 0.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import sys
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+METRIC = "GEMM TFLOP/s (device-timed, 1 B200) and fraction of dense BF16/FP32 peak"
+UNIT = "TFLOP/s"
+FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
+
+
+def load_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            p = json.load(f)
+        p["_source"] = "measured"
+        return p
+    p = dict(FALLBACK_PEAKS)
+    p["_source"] = "fallback"
+    return p
+
+
+def workload():
+    import nk_inputs
+    return nk_inputs.config(4)
+
+
+# --------------------------------------------------------------------------- reference arm
+def oracle_sample_rate(w, B, rows_per_step, steps, warmup, seed_shift=0):
+    """Time the CPU oracle, as it stands, on `rows_per_step` stratified rows of
+    the workload per step.  Returns (TFLOP/s, seconds per step, threads)."""
+    import numpy as np
+    import nk_inputs
+    import oracle
+    threads = os.cpu_count() or 1
+    rows = nk_inputs.stratified_rows(w.seed + seed_shift, w.M, rows_per_step)
+    # only the sampled rows of A are needed: build them into a sparse full-size buffer
+    A = np.zeros(w.M * w.K, dtype=np.uint16 if w.in_dtype == "bf16" else np.float32)
+    for r in rows:
+        A[r * w.K:(r + 1) * w.K] = nk_inputs.fill(w.seed, nk_inputs.TENSOR_A, w.K, w.dist_a[0], w.dist_a[1],
+                                                  w.in_dtype, start=int(r) * w.K)
+    times = []
+    for s in range(warmup + steps):
+        t0 = time.perf_counter()
+        oracle.gemm_workload(w, A, B, None, rows=rows, nthreads=threads, want_scale=False)
+        dt = time.perf_counter() - t0
+        if s >= warmup:
+            times.append(dt)
+    sec = sum(times) / len(times)
+    flops = 2.0 * len(rows) * w.N * w.K
+    return flops / sec / 1e12, sec, threads, len(rows)
+
+
+def run_reference(args):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return 0
+    import nk_inputs
+    w = workload()
+    B = nk_inputs.fill(w.seed, nk_inputs.TENSOR_B, w.K * w.N, w.dist_b[0], w.dist_b[1], w.in_dtype)
+    # probe the oracle's speed on 8 rows, then size the per-step sample so the whole
+    # run stays near two minutes
+    _, probe_sec, threads, _ = oracle_sample_rate(w, B, 8, 1, 0)
+    total_steps = args.steps + args.warmup
+    rows = int(max(1, min(256, 120.0 / max(total_steps, 1) / (probe_sec / 8))))
+    tf, sec, threads, nrows = oracle_sample_rate(w, B, rows, args.steps, args.warmup)
+    sample = f"{nrows} stratified rows of the {w.M}x{w.N}x{w.K} problem per step (all {w.N} columns, full K)"
+    out = {
+        "impl": "reference", "metric": METRIC, "value": tf, "unit": UNIT, "n_gpus": args.gpus,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": sec * 1e3,
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64",
+        "data": "synthetic",
+        "config": {"workload": w.name, "M": w.M, "N": w.N, "K": w.K, "in_dtype": w.in_dtype,
+                   "out_dtype": w.out_dtype, "layout": w.layout, "epilogue": w.epilogue},
+        "cpu_baseline": {"value": tf, "unit": UNIT, "cores": threads, "kind": "oracle", "sample": sample},
+        "e2e": {"value": tf, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+    print(json.dumps(out), flush=True)
+    return 0
+
+
+# --------------------------------------------------------------------------- clocks
+class ClockSampler:
+    """Samples SM clock and throttle reasons through NVML while the timed region runs."""
+
+    def __init__(self, index):
+        self.ok = False
+        self.samples, self.reasons = [], set()
+        self.max_mhz = None
+        try:
+            import pynvml
+            self.nv = pynvml
+            pynvml.nvmlInit()
+            self.h = pynvml.nvmlDeviceGetHandleByIndex(index)
+            self.max_mhz = pynvml.nvmlDeviceGetMaxClockInfo(self.h, pynvml.NVML_CLOCK_SM)
+            self.ok = True
+        except Exception:
+            pass
+
+    def sample(self):
+        if not self.ok:
+            return
+        nv = self.nv
+        try:
+            self.samples.append(nv.nvmlDeviceGetClockInfo(self.h, nv.NVML_CLOCK_SM))
+            r = nv.nvmlDeviceGetCurrentClocksEventReasons(self.h) if hasattr(
+                nv, "nvmlDeviceGetCurrentClocksEventReasons") else nv.nvmlDeviceGetCurrentClocksThrottleReasons(self.h)
+            names = {
+                0x8: "hw_slowdown", 0x40: "hw_thermal_slowdown", 0x20: "sw_thermal_slowdown",
+                0x4: "sw_power_cap", 0x80: "hw_power_brake_slowdown",
+            }
+            for bit, n in names.items():
+                if r & bit:
+                    self.reasons.add(n)
+        except Exception:
+            pass
+
+    def summary(self):
+        if not self.samples:
+            return {"sm_mhz": None, "sm_max_mhz": self.max_mhz, "reasons": sorted(self.reasons), "samples": 0}
+        s = sorted(self.samples)
+        return {"sm_mhz": s[len(s) // 2], "sm_max_mhz": self.max_mhz, "reasons": sorted(self.reasons),
+                "samples": len(s)}
+
+
+# --------------------------------------------------------------------------- our arm
+def run_ours(args):
+    import numpy as np
+    import torch
+    import torch.distributed as dist
+    import nk_inputs
+    import paper_2511_13764_b200 as nk
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the GEMM has no CPU path")
+    torch.cuda.set_device(local)
+    dev = torch.device("cuda", local)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=dev)
+
+    peaks = load_peaks()
+    w = workload()
+    # rank r owns its own block of 8192 rows of A (seed shifted by the rank); B is replicated
+    A = nk_inputs.fill(w.seed + 7919 * rank, nk_inputs.TENSOR_A, w.M * w.K, w.dist_a[0], w.dist_a[1], w.in_dtype)
+    B = nk_inputs.fill(w.seed, nk_inputs.TENSOR_B, w.K * w.N, w.dist_b[0], w.dist_b[1], w.in_dtype)
+    hA = torch.from_numpy(A).pin_memory()
+    hB = torch.from_numpy(B).pin_memory()
+    dA = hA.to(dev, non_blocking=True)
+    dB = hB.to(dev, non_blocking=True)
+    dC = torch.empty(w.M * w.N, dtype=torch.float32, device=dev)
+    plan = nk.plan_for(w, device=local)
+    ws_bytes = plan.workspace_bytes
+    ws = torch.empty(max(ws_bytes, 16), dtype=torch.uint8, device=dev)
+    stream = torch.cuda.current_stream()
+    sp = stream.cuda_stream
+
+    def step():
+        plan.run(dA, dB, dC, workspace=ws if ws_bytes else None, workspace_bytes=ws_bytes, stream=sp)
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    for _ in range(max(args.warmup, 3)):
+        step()
+    plan.check()
+
+    sampler = ClockSampler(local)
+    ev0 = torch.cuda.Event(enable_timing=True)
+    ev1 = torch.cuda.Event(enable_timing=True)
+    barrier()
+    ev0.record(stream)
+    for _ in range(args.steps):
+        step()
+    ev1.record(stream)
+    while not ev1.query():
+        sampler.sample()
+        time.sleep(0.002)
+    barrier()
+    ms = ev0.elapsed_time(ev1)
+    plan.check()
+    if world > 1:
+        t = torch.tensor([ms], dtype=torch.float64, device=dev)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        ms = float(t.item())
+    ms_per_step = ms / args.steps
+    value = world * w.flops / (ms_per_step * 1e-3) / 1e12
+
+    # per-launch duration of the GEMM kernel, measured live (one launch per step here;
+    # events on the launching stream around each of a few launches, L2 not reusable
+    # across launches: A, B, C total 512 MB)
+    k_ms = []
+    for _ in range(min(args.steps, 10)):
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record(stream)
+        step()
+        b.record(stream)
+        b.synchronize()
+        k_ms.append(a.elapsed_time(b))
+    k_avg = ms_per_step          # average launch duration inside the timed region
+    achieved = w.flops / (k_avg * 1e-3) / 1e12
+    peak = float(peaks["bf16_tflops"])
+    roofline = {
+        "bound": "tensor", "achieved": achieved, "peak": peak, "unit": "TFLOP/s",
+        "frac": achieved / peak, "traffic": None,
+        "peak_source": f"MEASURED_PEAKS.json bf16_tflops (burst), of {peaks['_source']}",
+        "frac_of_sustained_peak": achieved / float(peaks["bf16_tflops_sustained"]),
+        "frac_of_nominal_2250": achieved / 2250.0,
+        "kernel": plan.kernel_name,
+        "isolated_launch_tflops_best": w.flops / (min(k_ms) * 1e-3) / 1e12,
+        "isolated_launch_tflops_median": w.flops / (sorted(k_ms)[len(k_ms) // 2] * 1e-3) / 1e12,
+        "hbm_algorithmic_gbs": w.algorithmic_bytes / (k_avg * 1e-3) / 1e9,
+    }
+
+    # end to end through the C ABI with HOST buffers: H2D of A and B, GEMM, D2H of C per step
+    hC = torch.empty(w.M * w.N, dtype=torch.float32).pin_memory()
+    e2e_steps = max(1, min(args.steps, 5))
+    plan.run_host(hA, hB, hC, dA, dB, dC, workspace=ws if ws_bytes else None, workspace_bytes=ws_bytes, stream=sp)
+    barrier()
+    t0 = time.perf_counter()
+    for _ in range(e2e_steps):
+        plan.run_host(hA, hB, hC, dA, dB, dC, workspace=ws if ws_bytes else None, workspace_bytes=ws_bytes,
+                      stream=sp)
+    barrier()
+    e2e_s = (time.perf_counter() - t0) / e2e_steps
+    if world > 1:
+        t = torch.tensor([e2e_s], dtype=torch.float64, device=dev)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        e2e_s = float(t.item())
+    e2e = {"value": world * w.flops / e2e_s / 1e12, "unit": UNIT,
+           "h2d_bytes_per_step": int(A.nbytes + B.nbytes), "d2h_bytes_per_step": int(w.M * w.N * 4),
+           "steps": e2e_steps}
+
+    out = {
+        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+        "warmup": max(args.warmup, 3), "ms_per_step": ms_per_step, "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+        "config": {"workload": w.name, "M": w.M, "N": w.N, "K": w.K, "in_dtype": w.in_dtype,
+                   "out_dtype": w.out_dtype, "layout": w.layout, "epilogue": w.epilogue,
+                   "l2": "inputs larger than L2 (A 128 MB + B 128 MB + C 256 MB per step)",
+                   "parallelism": f"M-sharded x{world}, B replicated, no collective"},
+        "roofline": roofline, "e2e": e2e,
+        "gpu_launches": plan.launches_per_run * args.steps,
+        "clocks": sampler.summary(),
+    }
+
+    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+        tf, sec, threads, nrows = oracle_sample_rate(w, B, 256, 1, 0)
+        out["cpu_baseline"] = {
+            "value": tf, "unit": UNIT, "cores": threads, "kind": "oracle",
+            "sample": f"{nrows} stratified rows of the {w.M}x{w.N}x{w.K} problem (all columns, full K), "
+                      f"{sec:.1f} s"}
+    if rank == 0:
+        print(json.dumps(out), flush=True)
+    if world > 1:
+        dist.destroy_process_group()
+    return 0
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=100)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    if args.impl == "reference":
+        return run_reference(args)
+    return run_ours(args)
+
+
+if __name__ == "__main__":
+    sys.exit(main())
