@@ -40,9 +40,15 @@ def load_peaks():
     return p
 
 
-def workload():
+def workload(size=None):
+    """The benchmark workload: configuration 4 (BF16 8192^3, FP32 output).  `size`
+    shrinks M = N = K for profiler captures, which must stay small."""
+    import dataclasses
     import nk_inputs
-    return nk_inputs.config(4)
+    w = nk_inputs.config(4)
+    if size:
+        w = dataclasses.replace(w, name=f"c4_bf16_{size}_profiling_size", M=size, N=size, K=size)
+    return w
 
 
 # --------------------------------------------------------------------------- reference arm
@@ -76,7 +82,7 @@ def run_reference(args):
     if rank != 0:
         return 0
     import nk_inputs
-    w = workload()
+    w = workload(args.size)
     B = nk_inputs.fill(w.seed, nk_inputs.TENSOR_B, w.K * w.N, w.dist_b[0], w.dist_b[1], w.in_dtype)
     # probe the oracle's speed on 8 rows, then size the per-step sample so the whole
     # run stays near two minutes
@@ -163,7 +169,7 @@ def run_ours(args):
         dist.init_process_group("nccl", device_id=dev)
 
     peaks = load_peaks()
-    w = workload()
+    w = workload(args.size)
     # rank r owns its own block of 8192 rows of A (seed shifted by the rank); B is replicated
     A = nk_inputs.fill(w.seed + 7919 * rank, nk_inputs.TENSOR_A, w.M * w.K, w.dist_a[0], w.dist_a[1], w.in_dtype)
     B = nk_inputs.fill(w.seed, nk_inputs.TENSOR_B, w.K * w.N, w.dist_b[0], w.dist_b[1], w.in_dtype)
@@ -262,7 +268,7 @@ def run_ours(args):
         "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
         "config": {"workload": w.name, "M": w.M, "N": w.N, "K": w.K, "in_dtype": w.in_dtype,
                    "out_dtype": w.out_dtype, "layout": w.layout, "epilogue": w.epilogue,
-                   "l2": "inputs larger than L2 (A 128 MB + B 128 MB + C 256 MB per step)",
+                   "l2": f"inputs larger than L2 (A {A.nbytes >> 20} MB + B {B.nbytes >> 20} MB + C {(w.M * w.N * 4) >> 20} MB per step)",
                    "parallelism": f"M-sharded x{world}, B replicated, no collective"},
         "roofline": roofline, "e2e": e2e,
         "gpu_launches": plan.launches_per_run * args.steps,
@@ -289,6 +295,8 @@ def main():
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--size", type=int, default=None,
+                    help="shrink M=N=K (profiler captures only; not a benchmark number)")
     args = ap.parse_args()
     if args.impl == "reference":
         return run_reference(args)
