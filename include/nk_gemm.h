@@ -132,6 +132,41 @@ nk_status_t nk_gemm_run_host(nk_gemm_t plan, const void* hA, const void* hB, con
  */
 nk_status_t nk_gemm_check(nk_gemm_t plan);
 
+/*
+ * nk_gemm_run for callers that cannot allocate device memory.  (The paper has
+ * no counterpart; this is a convenience of the library.)
+ *
+ * Some callers of a GEMM library may not call cudaMalloc when they need the
+ * result: code running inside a region where device allocation is forbidden
+ * or would stall (a latency-critical serving loop, a plug-in that is handed
+ * buffers but owns no allocator, a process whose memory pool was sized up
+ * front and is now full).  A plan that splits K needs scratch for its FP32
+ * partial tiles, and nk_gemm_run makes the caller provide it.  This entry
+ * point runs the same plan with the scratch taken from a fixed array that is
+ * part of the library image instead: NK_STATIC_SCRATCH_BYTES (16 MiB) of
+ * device memory, present on every GPU that loads the library, from load until
+ * the process exits.  The caller passes only inputs and outputs.
+ *
+ * - Plans whose nk_gemm_workspace_bytes() exceeds NK_STATIC_SCRATCH_BYTES are
+ *   refused with NK_ERR_WORKSPACE and nothing is launched.  Plans that need no
+ *   scratch run exactly as with nk_gemm_run.
+ * - No cudaMalloc, cudaFree or other allocating call is made, here or in
+ *   anything this calls.
+ * - The first call on each device looks up the array's device address (once
+ *   per device, with that device current).  Make that first call outside any
+ *   stream capture.
+ * - All calls on a device share the one array, and it keeps whatever the last
+ *   call left in it.  The kernels overwrite every partial they later read, so
+ *   nothing has to be cleared between calls; but two calls whose GPU work can
+ *   overlap (different streams, or different plans run concurrently) race on
+ *   it.  Serialise them on one stream.
+ * Arguments, alignment rules, asynchrony and error codes are otherwise those of
+ * nk_gemm_run.
+ */
+#define NK_STATIC_SCRATCH_BYTES (16u << 20)
+nk_status_t nk_gemm_run_static(nk_gemm_t plan, const void* A, const void* B, const void* bias,
+                               void* C, void* cuda_stream);
+
 /* Free the plan's host state.  NULL is accepted. */
 nk_status_t nk_gemm_destroy(nk_gemm_t plan);
 

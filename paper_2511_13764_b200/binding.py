@@ -18,7 +18,9 @@ FLAG_REPACK_B = 0x10
 
 EXPORTS = ["nk_gemm_create", "nk_gemm_workspace_bytes", "nk_gemm_run", "nk_gemm_run_host",
            "nk_gemm_check", "nk_gemm_destroy", "nk_status_str", "nk_gemm_kernel_name",
-           "nk_gemm_launches_per_run", "nk_gemm_last_cuda_error"]
+           "nk_gemm_launches_per_run", "nk_gemm_last_cuda_error", "nk_gemm_run_static"]
+
+STATIC_SCRATCH_BYTES = 16 << 20
 
 
 def flag_splitk(n: int) -> int:
@@ -66,6 +68,8 @@ def lib():
         L.nk_gemm_workspace_bytes.argtypes = [vp]
         L.nk_gemm_run.restype = ctypes.c_int
         L.nk_gemm_run.argtypes = [vp, vp, vp, vp, vp, vp, sz, vp]
+        L.nk_gemm_run_static.restype = ctypes.c_int
+        L.nk_gemm_run_static.argtypes = [vp, vp, vp, vp, vp, vp]
         L.nk_gemm_run_host.restype = ctypes.c_int
         L.nk_gemm_run_host.argtypes = [vp, vp, vp, vp, vp, vp, vp, vp, vp, vp, sz, vp]
         L.nk_gemm_check.restype = ctypes.c_int
@@ -135,6 +139,11 @@ class Plan:
             workspace_bytes = 0 if workspace is None else workspace.numel() * workspace.element_size()
         _check(lib().nk_gemm_run(self._h, _ptr(A), _ptr(B), _ptr(bias), _ptr(C), _ptr(workspace),
                                  workspace_bytes, stream), self._h)
+
+    def run_static(self, A, B, C, bias=None, stream=None):
+        """nk_gemm_run_static: same GEMM, scratch taken from the library's built-in
+        16 MiB device array, so the caller allocates nothing."""
+        _check(lib().nk_gemm_run_static(self._h, _ptr(A), _ptr(B), _ptr(bias), _ptr(C), stream), self._h)
 
     def run_host(self, hA, hB, hC, dA, dB, dC, hbias=None, dbias=None, workspace=None,
                  workspace_bytes=None, stream=None):

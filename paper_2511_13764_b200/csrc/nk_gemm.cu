@@ -9,6 +9,7 @@
 #include <cstdio>
 #include <cstdlib>
 #include <cstring>
+#include <mutex>
 #include <new>
 
 #include "aux_kernels.cuh"
@@ -487,6 +488,47 @@ nk_status_t nk_gemm_run_host(nk_gemm_t p, const void* hA, const void* hB, const 
         return NK_ERR_CUDA;
     }
     return NK_OK;
+}
+
+// ---------------------------------------------------------------------------
+// Scratch for callers that cannot allocate: a fixed array inside the library
+// image.  In host code the symbol below is only a handle, not a device address;
+// the address each device gave it is looked up once per device and cached.
+static __device__ __align__(256) unsigned char g_static_scratch[NK_STATIC_SCRATCH_BYTES];
+
+namespace nk {
+constexpr int kMaxDevices = 64;
+static std::mutex g_scratch_mu;
+static void* g_scratch_addr[kMaxDevices];   // device address of g_static_scratch, per device
+}  // namespace nk
+
+nk_status_t nk_gemm_run_static(nk_gemm_t p, const void* A, const void* B, const void* bias, void* C,
+                               void* cuda_stream) {
+    if (!p) return NK_ERR_INVALID_ARG;
+    const size_t need = p->ws_repack_bytes + p->ws_partial_bytes;
+    if (need > NK_STATIC_SCRATCH_BYTES) {
+        snprintf(p->cuda_err, sizeof(p->cuda_err),
+                 "plan needs %zu bytes of scratch; the built-in array holds %u", need,
+                 (unsigned)NK_STATIC_SCRATCH_BYTES);
+        return NK_ERR_WORKSPACE;
+    }
+    if (need == 0) return nk_gemm_run(p, A, B, bias, C, nullptr, 0, cuda_stream);
+    const int dev = p->d.device;
+    if (dev < 0 || dev >= kMaxDevices) return NK_ERR_DEVICE;
+    void* scratch = nullptr;
+    {
+        std::lock_guard<std::mutex> lock(g_scratch_mu);
+        if (!g_scratch_addr[dev]) {
+            DeviceGuard guard(dev);   // the lookup answers for the current device
+            if (guard.err != cudaSuccess) { set_err(p, "cudaSetDevice", guard.err); return NK_ERR_DEVICE; }
+            void* addr = nullptr;
+            cudaError_t e = cudaGetSymbolAddress(&addr, g_static_scratch);
+            if (e != cudaSuccess || !addr) { set_err(p, "cudaGetSymbolAddress", e); return NK_ERR_CUDA; }
+            g_scratch_addr[dev] = addr;
+        }
+        scratch = g_scratch_addr[dev];
+    }
+    return nk_gemm_run(p, A, B, bias, C, scratch, NK_STATIC_SCRATCH_BYTES, cuda_stream);
 }
 
 nk_status_t nk_gemm_check(nk_gemm_t p) {
