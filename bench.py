@@ -106,6 +106,39 @@ def run_reference(args):
     return 0
 
 
+# --------------------------------------------------------------------------- multi-rank plumbing
+def shard_seed(seed: int, rank: int) -> int:
+    """Seed of rank `rank`'s block of A rows (B keeps the workload's seed on every rank)."""
+    return seed + 7919 * rank
+
+
+def init_distributed(world: int, device=None):
+    """One process per GPU: NCCL when a CUDA device is given, gloo otherwise (CPU tests)."""
+    import torch.distributed as dist
+    if world <= 1 or dist.is_initialized():
+        return
+    if device is not None:
+        dist.init_process_group("nccl", device_id=device)
+    else:
+        dist.init_process_group("gloo")
+
+
+def max_over_ranks(x: float, world: int, device=None) -> float:
+    """MAX all-reduce of one float (the step time every rank measured)."""
+    if world <= 1:
+        return float(x)
+    import torch
+    import torch.distributed as dist
+    t = torch.tensor([x], dtype=torch.float64, device=device if device is not None else "cpu")
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def whole_job_tflops(flops_per_rank: float, world: int, ms_per_step: float) -> float:
+    """Aggregate over all ranks: every rank does `flops_per_rank` per step (weak scaling)."""
+    return world * flops_per_rank / (ms_per_step * 1e-3) / 1e12
+
+
 # --------------------------------------------------------------------------- clocks
 class ClockSampler:
     """Samples SM clock and throttle reasons through NVML while the timed region runs."""
@@ -165,13 +198,12 @@ def run_ours(args):
         raise SystemExit("bench.py needs a CUDA device: the GEMM has no CPU path")
     torch.cuda.set_device(local)
     dev = torch.device("cuda", local)
-    if world > 1:
-        dist.init_process_group("nccl", device_id=dev)
+    init_distributed(world, dev)
 
     peaks = load_peaks()
     w = workload(args.size)
     # rank r owns its own block of 8192 rows of A (seed shifted by the rank); B is replicated
-    A = nk_inputs.fill(w.seed + 7919 * rank, nk_inputs.TENSOR_A, w.M * w.K, w.dist_a[0], w.dist_a[1], w.in_dtype)
+    A = nk_inputs.fill(shard_seed(w.seed, rank), nk_inputs.TENSOR_A, w.M * w.K, w.dist_a[0], w.dist_a[1], w.in_dtype)
     B = nk_inputs.fill(w.seed, nk_inputs.TENSOR_B, w.K * w.N, w.dist_b[0], w.dist_b[1], w.in_dtype)
     hA = torch.from_numpy(A).pin_memory()
     hB = torch.from_numpy(B).pin_memory()
@@ -210,12 +242,9 @@ def run_ours(args):
     barrier()
     ms = ev0.elapsed_time(ev1)
     plan.check()
-    if world > 1:
-        t = torch.tensor([ms], dtype=torch.float64, device=dev)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        ms = float(t.item())
+    ms = max_over_ranks(ms, world, dev)
     ms_per_step = ms / args.steps
-    value = world * w.flops / (ms_per_step * 1e-3) / 1e12
+    value = whole_job_tflops(w.flops, world, ms_per_step)
 
     # per-launch duration of the GEMM kernel, measured live (one launch per step here;
     # events on the launching stream around each of a few launches, L2 not reusable
@@ -254,11 +283,8 @@ def run_ours(args):
                       stream=sp)
     barrier()
     e2e_s = (time.perf_counter() - t0) / e2e_steps
-    if world > 1:
-        t = torch.tensor([e2e_s], dtype=torch.float64, device=dev)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        e2e_s = float(t.item())
-    e2e = {"value": world * w.flops / e2e_s / 1e12, "unit": UNIT,
+    e2e_s = max_over_ranks(e2e_s, world, dev)
+    e2e = {"value": whole_job_tflops(w.flops, world, e2e_s * 1e3), "unit": UNIT,
            "h2d_bytes_per_step": int(A.nbytes + B.nbytes), "d2h_bytes_per_step": int(w.M * w.N * 4),
            "steps": e2e_steps}
 
