@@ -15,6 +15,7 @@
 #include "aux_kernels.cuh"
 #include "simt_f32.cuh"
 #include "umma_bf16.cuh"
+#include "umma_bf16_pair.cuh"
 
 namespace nk {
 
@@ -37,6 +38,8 @@ struct nk_gemm_s {
     int sm_count;
     // UMMA
     int bn, stages, splits, group_m;
+    bool pair;             // CTA pairs: 256-row tiles, cta_group::2
+    int max_pairs;         // co-resident clusters of 2 for the chosen pair kernel
     bool b_vnni_inkernel;  // blocked B re-laid inside the GEMM kernel
     bool b_repack;         // blocked B unpacked to row-major scratch first
     // SIMT
@@ -104,27 +107,35 @@ static int umma_stages_for(int bn) { return bn == 256 ? 4 : bn == 128 ? 6 : 8; }
 static void choose_umma(nk_gemm_s* p) {
     const nk_gemm_desc_t& d = p->d;
     const int sms = p->sm_count;
-    const int tiles_m = ceil_div(d.M, UMMA_BM);
     const int kb_total = ceil_div(d.K, UMMA_BK);
-    int bn = 64;
     const int forced = (d.flags >> NK_FLAG_TILE_N_SHIFT) & 0xF;
+    // CTA pairs (256-row tiles) whenever there are at least two 128-row tiles of M.
+    bool pair = d.M > UMMA_BM;
+    if (d.flags & NK_FLAG_SINGLE_CTA) pair = false;
+    if (d.flags & NK_FLAG_CTA_PAIR) pair = true;
+    if (pair && forced == 2) pair = false;            // 64-wide tiles exist only single-CTA
+    const int workers = pair ? sms / 2 : sms;         // CTAs or CTA pairs
+    const int tiles_m = ceil_div(d.M, pair ? 2 * UMMA_BM : UMMA_BM);
+    int bn = pair ? 128 : 64;
     if (forced >= 2 && forced <= 4) {
         bn = 32 << (forced - 1);
     } else {
         const int cands[3] = {256, 128, 64};
         for (int c : cands) {
-            if (static_cast<int64_t>(tiles_m) * ceil_div(d.N, c) >= sms) { bn = c; break; }
+            if (pair && c == 64) break;
+            if (static_cast<int64_t>(tiles_m) * ceil_div(d.N, c) >= workers) { bn = c; break; }
         }
     }
+    p->pair = pair;
     p->bn = bn;
-    p->stages = umma_stages_for(bn);
+    p->stages = pair ? (bn == 256 ? 6 : 8) : umma_stages_for(bn);
     const int tiles = tiles_m * ceil_div(d.N, bn);
     int splits = 1;
     const int forced_s = (d.flags >> NK_FLAG_SPLITK_SHIFT) & 0xFF;
     if (forced_s > 0) {
         splits = forced_s;
-    } else if (tiles * 2 <= sms) {
-        splits = sms / tiles;
+    } else if (tiles * 2 <= workers) {
+        splits = workers / tiles;
         const int max_by_k = kb_total / 4 > 0 ? kb_total / 4 : 1;  // >= 4 k-blocks per split
         if (splits > max_by_k) splits = max_by_k;
         if (splits > 32) splits = 32;
@@ -240,7 +251,53 @@ static cudaError_t launch_umma(nk_gemm_s* p, const UmmaParams& up, int grid, cud
     }
 }
 
+template <int BN, int STAGES, bool VNNI>
+static cudaError_t launch_pair_t(nk_gemm_s* p, const UmmaParams& up, int pairs, cudaStream_t st) {
+    cudaLaunchConfig_t cfg;
+    memset(&cfg, 0, sizeof(cfg));
+    cfg.gridDim = dim3(static_cast<unsigned>(2 * pairs));
+    cfg.blockDim = dim3(VNNI ? 320 : 192);
+    cfg.dynamicSmemBytes = pair_smem_bytes(BN, STAGES);
+    cfg.stream = st;
+    cudaLaunchAttribute attr;
+    attr.id = cudaLaunchAttributeClusterDimension;
+    attr.val.clusterDim.x = 2;
+    attr.val.clusterDim.y = 1;
+    attr.val.clusterDim.z = 1;
+    cfg.attrs = &attr;
+    cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, umma_bf16_pair_kernel<BN, STAGES, VNNI>, p->tmap_a, p->tmap_b, up);
+}
+
+static cudaError_t launch_pair(nk_gemm_s* p, const UmmaParams& up, int pairs, cudaStream_t st) {
+    const bool v = p->b_vnni_inkernel;
+    if (p->bn == 256) return v ? launch_pair_t<256, 6, true>(p, up, pairs, st) : launch_pair_t<256, 6, false>(p, up, pairs, st);
+    return v ? launch_pair_t<128, 8, true>(p, up, pairs, st) : launch_pair_t<128, 8, false>(p, up, pairs, st);
+}
+
+template <int BN, int STAGES, bool VNNI>
+static cudaError_t pair_occupancy(int* out) {
+    cudaLaunchConfig_t cfg;
+    memset(&cfg, 0, sizeof(cfg));
+    cfg.gridDim = dim3(2);
+    cfg.blockDim = dim3(VNNI ? 320 : 192);
+    cfg.dynamicSmemBytes = pair_smem_bytes(BN, STAGES);
+    cudaLaunchAttribute attr;
+    attr.id = cudaLaunchAttributeClusterDimension;
+    attr.val.clusterDim.x = 2;
+    attr.val.clusterDim.y = 1;
+    attr.val.clusterDim.z = 1;
+    cfg.attrs = &attr;
+    cfg.numAttrs = 1;
+    return cudaOccupancyMaxActiveClusters(out, umma_bf16_pair_kernel<BN, STAGES, VNNI>, &cfg);
+}
+
 static cudaError_t prepare_umma_attrs() {
+    cudaError_t e2;
+    if ((e2 = allow_smem(umma_bf16_pair_kernel<256, 6, false>, pair_smem_bytes(256, 6))) != cudaSuccess) return e2;
+    if ((e2 = allow_smem(umma_bf16_pair_kernel<128, 8, false>, pair_smem_bytes(128, 8))) != cudaSuccess) return e2;
+    if ((e2 = allow_smem(umma_bf16_pair_kernel<256, 6, true>, pair_smem_bytes(256, 6))) != cudaSuccess) return e2;
+    if ((e2 = allow_smem(umma_bf16_pair_kernel<128, 8, true>, pair_smem_bytes(128, 8))) != cudaSuccess) return e2;
     cudaError_t e;
     if ((e = allow_smem(umma_bf16_kernel<256, 4, false>, umma_smem_bytes(256, 4))) != cudaSuccess) return e;
     if ((e = allow_smem(umma_bf16_kernel<128, 6, false>, umma_smem_bytes(128, 6))) != cudaSuccess) return e;
@@ -354,10 +411,20 @@ nk_status_t nk_gemm_create(const nk_gemm_desc_t* desc, nk_gemm_t* out) {
             p->b_repack = (d.flags & NK_FLAG_REPACK_B) != 0;
             p->b_vnni_inkernel = !p->b_repack;
         }
+        if (p->pair) {
+            const bool v = p->b_vnni_inkernel;
+            int n = 0;
+            cudaError_t oe = p->bn == 256
+                ? (v ? pair_occupancy<256, 6, true>(&n) : pair_occupancy<256, 6, false>(&n))
+                : (v ? pair_occupancy<128, 8, true>(&n) : pair_occupancy<128, 8, false>(&n));
+            if (oe != cudaSuccess || n <= 0) { cudaGetLastError(); delete p; return NK_ERR_CUDA; }
+            p->max_pairs = n;
+        }
         p->ws_repack_bytes = p->b_repack ? align_up(static_cast<size_t>(d.K) * d.N * 2, 256) : 0;
         p->ws_partial_bytes = p->splits > 1 ? static_cast<size_t>(p->splits) * d.M * d.N * 4 : 0;
         p->launches = 1 + (p->splits > 1 ? 1 : 0) + (p->b_repack ? 1 : 0);
-        snprintf(p->name, sizeof(p->name), "umma_bf16_128x%dx64_s%d_splitk%d%s%s", p->bn, p->stages,
+        snprintf(p->name, sizeof(p->name), "umma_bf16_%s%dx64_s%d_splitk%d%s%s",
+                 p->pair ? "pair_256x" : "128x", p->bn, p->stages,
                  p->splits, d.layout_a == NK_BLOCKED32 ? "_ablk" : "",
                  p->b_vnni_inkernel ? "_bvnni" : (p->b_repack ? "_brepack" : ""));
     }
@@ -426,7 +493,7 @@ nk_status_t nk_gemm_run(nk_gemm_t p, const void* A, const void* B, const void* b
         UmmaParams up;
         memset(&up, 0, sizeof(up));
         up.M = static_cast<int>(d.M); up.N = static_cast<int>(d.N); up.K = static_cast<int>(d.K);
-        up.tiles_m = ceil_div(d.M, UMMA_BM);
+        up.tiles_m = ceil_div(d.M, p->pair ? 2 * UMMA_BM : UMMA_BM);
         up.tiles_n = ceil_div(d.N, p->bn);
         up.splits = p->splits;
         up.kb_total = ceil_div(d.K, UMMA_BK);
@@ -435,15 +502,20 @@ nk_status_t nk_gemm_run(nk_gemm_t p, const void* A, const void* B, const void* b
         up.a_blocked = d.layout_a == NK_BLOCKED32;
         up.epilogue = d.epilogue;
         up.out_bf16 = d.out_dtype == NK_BF16;
-        up.idesc = make_idesc(UMMA_BM, p->bn, !p->b_vnni_inkernel);
+        up.idesc = make_idesc(p->pair ? 2 * UMMA_BM : UMMA_BM, p->bn, !p->b_vnni_inkernel);
         up.bias = bias;
         up.C = C;
         up.partial = partial;
         up.Bblk = p->b_vnni_inkernel ? static_cast<const uint32_t*>(B) : nullptr;
         up.status = p->status_dev;
         const int units = up.tiles_m * up.tiles_n * up.splits;
-        const int grid = units < p->sm_count ? units : p->sm_count;
-        e = launch_umma(p, up, grid, st);
+        if (p->pair) {
+            const int pairs = units < p->max_pairs ? units : p->max_pairs;
+            e = launch_pair(p, up, pairs, st);
+        } else {
+            const int grid = units < p->sm_count ? units : p->sm_count;
+            e = launch_umma(p, up, grid, st);
+        }
         if (e != cudaSuccess) { set_err(p, "umma launch", e); return NK_ERR_CUDA; }
     }
 

@@ -77,6 +77,65 @@ __device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi) {
     return *reinterpret_cast<uint32_t*>(&v);
 }
 
+// Epilogue for one 32-column chunk of one row held in registers (FP32 bit patterns):
+// either the raw FP32 partial of a K split, or bias + ReLU (Section 6, "MLP") followed by
+// the single store of C as FP32 or BF16 (one RNE rounding).  16-byte stores; columns are
+// predicated in groups (N is a multiple of 8).
+__device__ __forceinline__ void umma_store_chunk(const UmmaParams& p, uint32_t (&v)[32], int row,
+                                                 int col0, int split, bool empty_k) {
+    if (row >= p.M || col0 >= p.N) return;
+    const size_t row_off = static_cast<size_t>(row) * p.N;
+    if (empty_k) {
+#pragma unroll
+        for (int i = 0; i < 32; ++i) v[i] = 0u;
+    }
+    if (p.splits > 1) {
+        float* dst = p.partial + static_cast<size_t>(split) * p.M * p.N + row_off + col0;
+#pragma unroll
+        for (int g = 0; g < 8; ++g)
+            if (col0 + 4 * g < p.N)
+                *reinterpret_cast<uint4*>(dst + 4 * g) =
+                    make_uint4(v[4 * g], v[4 * g + 1], v[4 * g + 2], v[4 * g + 3]);
+        return;
+    }
+    if (p.epilogue) {
+        const uint4* bsrc = reinterpret_cast<const uint4*>(static_cast<const uint16_t*>(p.bias) + col0);
+#pragma unroll
+        for (int g = 0; g < 4; ++g) {
+            if (col0 + 8 * g >= p.N) break;
+            const uint4 b = __ldg(bsrc + g);
+            const uint32_t w[4] = {b.x, b.y, b.z, b.w};
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+                float x0 = __uint_as_float(v[8 * g + 2 * j]) + bf16_bits_to_f32(w[j] & 0xFFFFu);
+                float x1 = __uint_as_float(v[8 * g + 2 * j + 1]) + bf16_bits_to_f32(w[j] >> 16);
+                v[8 * g + 2 * j] = __float_as_uint(fmaxf(x0, 0.0f));
+                v[8 * g + 2 * j + 1] = __float_as_uint(fmaxf(x1, 0.0f));
+            }
+        }
+    }
+    if (p.out_bf16) {
+        uint16_t* dst = static_cast<uint16_t*>(p.C) + row_off + col0;
+#pragma unroll
+        for (int g = 0; g < 4; ++g)
+            if (col0 + 8 * g < p.N) {
+                uint4 o;
+                o.x = pack_bf16x2(__uint_as_float(v[8 * g]), __uint_as_float(v[8 * g + 1]));
+                o.y = pack_bf16x2(__uint_as_float(v[8 * g + 2]), __uint_as_float(v[8 * g + 3]));
+                o.z = pack_bf16x2(__uint_as_float(v[8 * g + 4]), __uint_as_float(v[8 * g + 5]));
+                o.w = pack_bf16x2(__uint_as_float(v[8 * g + 6]), __uint_as_float(v[8 * g + 7]));
+                *reinterpret_cast<uint4*>(dst + 8 * g) = o;
+            }
+    } else {
+        float* dst = static_cast<float*>(p.C) + row_off + col0;
+#pragma unroll
+        for (int g = 0; g < 8; ++g)
+            if (col0 + 4 * g < p.N)
+                *reinterpret_cast<uint4*>(dst + 4 * g) =
+                    make_uint4(v[4 * g], v[4 * g + 1], v[4 * g + 2], v[4 * g + 3]);
+    }
+}
+
 template <int BN, int STAGES, bool B_VNNI>
 __global__ void __launch_bounds__(B_VNNI ? 320 : 192, 1)
 umma_bf16_kernel(const __grid_constant__ CUtensorMap tmap_a,
@@ -182,8 +241,28 @@ umma_bf16_kernel(const __grid_constant__ CUtensorMap tmap_a,
         }
     } else if (warp == 1) {
         // ------------------------------------------------ MMA issuer
+        // One lane issues; its instruction stream is the critical path of the K loop, so the
+        // descriptors are kept as 32-bit halves and advanced with adds, and everything that
+        // does not change per stage is computed here, once.
+        //   A row-major: K-major tile, 128-byte swizzle, 8-row groups 1024 B apart; the four
+        //     k-steps of a stage are 32 B apart.
+        //   A blocked: two K-major slabs of 32 k (8192 B apart), 64-byte swizzle, 8-row groups
+        //     512 B apart; k-steps at 0, 32 B, 8192 B, 8192 + 32 B.
+        //   B row-major [K][N]: N-major, 64-column atoms 8192 B apart (leading), 8-k groups
+        //     1024 B apart (stride); k-steps 2048 B apart.  B re-laid from VNNI: K-major like A.
+        const bool a_blk = p.a_blocked != 0;
+        const uint64_t da0 = a_blk ? make_smem_desc(smem_base, 16, 512, 4) : make_smem_desc(smem_base, 16, 1024, 2);
+        const uint64_t db0 = B_VNNI ? make_smem_desc(smem_base + UMMA_A_STAGE_BYTES, 16, 1024, 2)
+                                    : make_smem_desc(smem_base + UMMA_A_STAGE_BYTES, 8192, 1024, 2);
+        const uint32_t a_hi = static_cast<uint32_t>(da0 >> 32), b_hi = static_cast<uint32_t>(db0 >> 32);
+        const uint32_t a_lo0 = static_cast<uint32_t>(da0), b_lo0 = static_cast<uint32_t>(db0);
+        const uint32_t a_s1 = 2u, a_s2 = a_blk ? 512u : 4u, a_s3 = a_blk ? 514u : 6u;
+        constexpr uint32_t b_s = B_VNNI ? 2u : 128u;
+        constexpr uint32_t STAGE16 = STAGE >> 4;
+        const uint32_t idesc = p.idesc;
         int stage = 0;
         uint32_t phase = 0;
+        uint32_t soff = 0;  // stage * STAGE / 16
         int local = 0;
         bool ok = true;
         for (int unit = blockIdx.x; ok && unit < total_units; unit += gridDim.x, ++local) {
@@ -198,6 +277,7 @@ umma_bf16_kernel(const __grid_constant__ CUtensorMap tmap_a,
             }
             tc_fence_after_sync();
             const uint32_t d_tmem = tmem_base + acc * BN;
+            uint32_t accumulate = 0u;
             for (int kb = kb0; kb < kb1; ++kb) {
                 if (!mbar_wait(full_bar(stage), phase, abort_flag)) {
                     if (lane == 0) give_up(0x300u + stage);
@@ -206,30 +286,18 @@ umma_bf16_kernel(const __grid_constant__ CUtensorMap tmap_a,
                 }
                 tc_fence_after_sync();
                 if (lane == 0) {
-                    const uint32_t sa = smem_base + stage * STAGE;
-                    const uint32_t sb = sa + UMMA_A_STAGE_BYTES;
-                    // A row-major: K-major tile, 128-byte swizzle, 8-row groups 1024 B apart.
-                    // A blocked: two K-major slabs of 32 k, 64-byte swizzle, 8-row groups 512 B apart.
-                    const uint64_t da = p.a_blocked ? make_smem_desc(sa, 16, 512, 4)
-                                                    : make_smem_desc(sa, 16, 1024, 2);
-                    // B row-major [K][N]: N-major, 64-column atoms 8192 B apart (leading),
-                    // 8-k groups 1024 B apart (stride).  B re-laid from VNNI: K-major like A.
-                    const uint64_t db = B_VNNI ? make_smem_desc(sb, 16, 1024, 2)
-                                               : make_smem_desc(sb, 8192, 1024, 2);
-#pragma unroll
-                    for (int k4 = 0; k4 < UMMA_BK / 16; ++k4) {
-                        const uint64_t a_adv = static_cast<uint64_t>(
-                            p.a_blocked ? (k4 >> 1) * 512 + (k4 & 1) * 2 : k4 * 2);  // 32 B steps
-                        const uint64_t b_adv =
-                            static_cast<uint64_t>(B_VNNI ? k4 * 2 : k4 * 128);  // 32 B | 2048 B
-                        umma_f16(d_tmem, da + a_adv, db + b_adv, p.idesc,
-                                 (kb > kb0 || k4 > 0) ? 1u : 0u);
-                    }
+                    const uint32_t a_lo = a_lo0 + soff, b_lo = b_lo0 + soff;
+                    umma_f16_lohi(d_tmem, a_lo, a_hi, b_lo, b_hi, idesc, accumulate);
+                    umma_f16_lohi(d_tmem, a_lo + a_s1, a_hi, b_lo + b_s, b_hi, idesc, 1u);
+                    umma_f16_lohi(d_tmem, a_lo + a_s2, a_hi, b_lo + 2 * b_s, b_hi, idesc, 1u);
+                    umma_f16_lohi(d_tmem, a_lo + a_s3, a_hi, b_lo + 3 * b_s, b_hi, idesc, 1u);
                     umma_commit(empty_bar(stage));
                     if (kb == kb1 - 1) umma_commit(tfull_bar(acc));
                 }
+                accumulate = 1u;
                 __syncwarp();
-                if (++stage == STAGES) { stage = 0; phase ^= 1u; }
+                soff += STAGE16;
+                if (++stage == STAGES) { stage = 0; phase ^= 1u; soff = 0; }
             }
             if (kb1 <= kb0 && lane == 0) umma_commit(tfull_bar(acc));  // empty K range
             __syncwarp();
@@ -253,69 +321,14 @@ umma_bf16_kernel(const __grid_constant__ CUtensorMap tmap_a,
             }
             tc_fence_after_sync();
             const int row = mb * UMMA_BM + quarter * 32 + lane;
-            const bool row_ok = row < p.M;
-            const bool to_partial = p.splits > 1;
             const bool empty_k = kb1 <= kb0;
-            const size_t row_off = static_cast<size_t>(row) * p.N;
 #pragma unroll 1
             for (int c0 = 0; c0 < BN; c0 += 32) {
                 uint32_t v[32];
                 tmem_ld_32x32(tmem_base + acc * BN + c0 + (static_cast<uint32_t>(quarter * 32) << 16),
                               v);
                 tmem_ld_wait();
-                const int col0 = nb * BN + c0;
-                if (row_ok && col0 < p.N) {
-                if (empty_k) {
-#pragma unroll
-                    for (int i = 0; i < 32; ++i) v[i] = 0u;
-                }
-                if (to_partial) {
-                    float* dst = p.partial + static_cast<size_t>(split) * p.M * p.N + row_off + col0;
-#pragma unroll
-                    for (int g = 0; g < 8; ++g)
-                        if (col0 + 4 * g < p.N)
-                            *reinterpret_cast<uint4*>(dst + 4 * g) =
-                                make_uint4(v[4 * g], v[4 * g + 1], v[4 * g + 2], v[4 * g + 3]);
-                } else {
-                if (p.epilogue) {
-                    const uint4* bsrc = reinterpret_cast<const uint4*>(
-                        static_cast<const uint16_t*>(p.bias) + col0);
-#pragma unroll
-                    for (int g = 0; g < 4; ++g) {
-                        if (col0 + 8 * g >= p.N) break;
-                        const uint4 b = __ldg(bsrc + g);
-                        const uint32_t w[4] = {b.x, b.y, b.z, b.w};
-#pragma unroll
-                        for (int j = 0; j < 4; ++j) {
-                            float x0 = __uint_as_float(v[8 * g + 2 * j]) + bf16_bits_to_f32(w[j] & 0xFFFFu);
-                            float x1 = __uint_as_float(v[8 * g + 2 * j + 1]) + bf16_bits_to_f32(w[j] >> 16);
-                            v[8 * g + 2 * j] = __float_as_uint(fmaxf(x0, 0.0f));
-                            v[8 * g + 2 * j + 1] = __float_as_uint(fmaxf(x1, 0.0f));
-                        }
-                    }
-                }
-                if (p.out_bf16) {
-                    uint16_t* dst = static_cast<uint16_t*>(p.C) + row_off + col0;
-#pragma unroll
-                    for (int g = 0; g < 4; ++g)
-                        if (col0 + 8 * g < p.N) {
-                            uint4 o;
-                            o.x = pack_bf16x2(__uint_as_float(v[8 * g]), __uint_as_float(v[8 * g + 1]));
-                            o.y = pack_bf16x2(__uint_as_float(v[8 * g + 2]), __uint_as_float(v[8 * g + 3]));
-                            o.z = pack_bf16x2(__uint_as_float(v[8 * g + 4]), __uint_as_float(v[8 * g + 5]));
-                            o.w = pack_bf16x2(__uint_as_float(v[8 * g + 6]), __uint_as_float(v[8 * g + 7]));
-                            *reinterpret_cast<uint4*>(dst + 8 * g) = o;
-                        }
-                } else {
-                    float* dst = static_cast<float*>(p.C) + row_off + col0;
-#pragma unroll
-                    for (int g = 0; g < 8; ++g)
-                        if (col0 + 4 * g < p.N)
-                            *reinterpret_cast<uint4*>(dst + 4 * g) =
-                                make_uint4(v[4 * g], v[4 * g + 1], v[4 * g + 2], v[4 * g + 3]);
-                }
-                }  // direct store
-                }  // in range
+                umma_store_chunk(p, v, row, nb * BN + c0, split, empty_k);
                 __syncwarp();
             }
             tc_fence_before_sync();

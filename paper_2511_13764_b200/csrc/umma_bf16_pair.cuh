@@ -1,0 +1,285 @@
+// BF16 GEMM on CTA pairs: two CTAs (a cluster of 2, neighbouring SMs) compute one
+// 256 x BN output tile with a single tcgen05.mma.cta_group::2 per k-step.
+//
+// Why: with one CTA per tile every SM has to pull 128 rows of A and BN columns of B per
+// k-block from L2, and that operand feed, not the tensor pipe, bounds the single-CTA
+// kernel.  In a pair each CTA loads its own 128 rows of A and only HALF of the B tile; the
+// tensor cores of both SMs read both halves.  Bytes per flop per SM drop by a third at
+// BN = 256 and the freed shared memory buys two more pipeline stages.  No TMA multicast is
+// used: every CTA fetches its own boxes; only the mbarrier signals cross the pair.
+//
+// The structure is that of the single-CTA kernel (Algorithm 1 of the paper: tile loop,
+// accumulator resident over the K loop, fused epilogue, one store).  Differences:
+//   - both CTAs' TMA loads complete on the LEADER's (rank 0) full[] barrier, which expects
+//     the bytes of both;
+//   - only the leader issues MMAs; tcgen05.commit signals empty[] and tmem_full[] in both CTAs;
+//   - each CTA drains its own 128 accumulator rows; tmem_empty[] lives in the leader and
+//     counts the epilogue threads of both CTAs (the peer arrives remotely);
+//   - cluster-wide barriers fence the start (barriers initialised) and the end (nobody
+//     leaves while its peer may still touch its shared memory or barriers).
+#pragma once
+#include "umma_bf16.cuh"
+
+namespace nk {
+
+__host__ __device__ constexpr int pair_stage_bytes(int BN) { return UMMA_A_STAGE_BYTES + (BN / 2) * UMMA_BK * 2; }
+__host__ __device__ constexpr int pair_smem_bytes(int BN, int stages) {
+    return stages * pair_stage_bytes(BN) + 1024 + 256;
+}
+
+// UmmaParams as for the single-CTA kernel, with tiles_m counted in 256-row tiles.
+template <int BN, int STAGES, bool B_VNNI>
+__global__ void __launch_bounds__(B_VNNI ? 320 : 192, 1)
+umma_bf16_pair_kernel(const __grid_constant__ CUtensorMap tmap_a,
+                      const __grid_constant__ CUtensorMap tmap_b, const UmmaParams p) {
+    static_assert(BN == 128 || BN == 256, "pair tile N");
+    constexpr int HALF = BN / 2;                       // B columns held by each CTA
+    constexpr int B_STAGE = HALF * UMMA_BK * 2;
+    constexpr int STAGE = pair_stage_bytes(BN);
+    constexpr uint32_t TMEM_COLS = 2 * BN;             // two accumulators of BN columns
+    constexpr int BM2 = 2 * UMMA_BM;
+
+    extern __shared__ uint8_t smem_raw[];
+    const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
+    const uint32_t bar_base = smem_base + STAGES * STAGE;
+    auto full_bar = [&](int s) { return bar_base + 8u * s; };
+    auto empty_bar = [&](int s) { return bar_base + 8u * (STAGES + s); };
+    auto tfull_bar = [&](int a) { return bar_base + 8u * (2 * STAGES + a); };
+    auto tempty_bar = [&](int a) { return bar_base + 8u * (2 * STAGES + 2 + a); };
+    uint8_t* gen_base = smem_raw + (smem_base - smem_u32(smem_raw));
+    volatile uint32_t* tmem_slot =
+        reinterpret_cast<volatile uint32_t*>(gen_base + STAGES * STAGE + 8 * (2 * STAGES + 4));
+    volatile uint32_t* abort_flag = tmem_slot + 1;
+
+    const int warp = threadIdx.x >> 5;
+    const int lane = threadIdx.x & 31;
+    const uint32_t rank = cluster_ctarank();           // 0 = leader
+    const int pair_id = blockIdx.x >> 1;
+    const int num_pairs = gridDim.x >> 1;
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < STAGES; ++s) {
+            mbar_init(full_bar(s), B_VNNI ? 1 + 8 : 1);  // leader's producer (+ 4 re-layout warps per CTA)
+            mbar_init(empty_bar(s), 1);
+        }
+        for (int a = 0; a < 2; ++a) {
+            mbar_init(tfull_bar(a), 1);
+            mbar_init(tempty_bar(a), 256);               // epilogue threads of both CTAs
+        }
+        *abort_flag = 0;
+        fence_mbar_init();
+        tma_prefetch_desc(&tmap_a);
+        if (!B_VNNI) tma_prefetch_desc(&tmap_b);
+    }
+    if (warp == 1) {
+        tmem_alloc_pair(smem_u32(const_cast<uint32_t*>(tmem_slot)), TMEM_COLS);
+        tmem_relinquish_pair();
+    }
+    tc_fence_before_sync();
+    __syncthreads();
+    cluster_sync_all();
+    tc_fence_after_sync();
+    const uint32_t tmem_base = *tmem_slot;
+
+    const int total_units = p.tiles_m * p.tiles_n * p.splits;
+    auto give_up = [&](unsigned int code) {
+        *abort_flag = 1;
+        if (p.status) atomicCAS(p.status, 0u, code);
+    };
+
+    if (warp == 0) {
+        // ------------------------------------------------ TMA producer (both CTAs)
+        int stage = 0;
+        uint32_t phase = 0;
+        bool ok = true;
+        for (int unit = pair_id; ok && unit < total_units; unit += num_pairs) {
+            const int tile = unit / p.splits, split = unit - tile * p.splits;
+            int mb, nb;
+            umma_tile_coords(p, tile, mb, nb);
+            const int kb0 = split * p.kb_per_split;
+            const int kb1 = min(p.kb_total, kb0 + p.kb_per_split);
+            const int row0 = mb * BM2 + static_cast<int>(rank) * UMMA_BM;
+            const int col0 = nb * BN + static_cast<int>(rank) * HALF;
+            for (int kb = kb0; kb < kb1; ++kb) {
+                if (!mbar_wait(empty_bar(stage), phase ^ 1u, abort_flag)) {
+                    if (lane == 0) give_up(0x100u + stage);
+                    ok = false;
+                    break;
+                }
+                if (lane == 0) {
+                    const uint32_t sa = smem_base + stage * STAGE;
+                    const uint32_t sb = sa + UMMA_A_STAGE_BYTES;
+                    const uint32_t lead_full = map_to_cta(full_bar(stage), 0);
+                    if (rank == 0)
+                        mbar_arrive_expect_tx(full_bar(stage),
+                                              2u * (UMMA_A_STAGE_BYTES + (B_VNNI ? 0 : B_STAGE)));
+                    if (p.a_blocked) {
+                        tma_load_4d_pair(sa, &tmap_a, lead_full, 0, 0, kb * 2, row0 / 32);
+                        tma_load_4d_pair(sa + 8192, &tmap_a, lead_full, 0, 0, kb * 2 + 1, row0 / 32);
+                    } else {
+                        tma_load_2d_pair(sa, &tmap_a, lead_full, kb * UMMA_BK, row0);
+                    }
+                    if (!B_VNNI) {
+#pragma unroll
+                        for (int j = 0; j < HALF / 64; ++j)
+                            tma_load_2d_pair(sb + j * 8192, &tmap_b, lead_full, col0 + j * 64, kb * UMMA_BK);
+                    }
+                }
+                __syncwarp();
+                if (++stage == STAGES) { stage = 0; phase ^= 1u; }
+            }
+        }
+        if (ok) {   // drain: every stage this CTA filled has been consumed
+            for (int s = 0; s < STAGES; ++s) {
+                if (!mbar_wait(empty_bar(stage), phase ^ 1u, abort_flag)) break;
+                if (++stage == STAGES) { stage = 0; phase ^= 1u; }
+            }
+        }
+    } else if (warp == 1) {
+        // ------------------------------------------------ MMA issuer (leader only)
+        // Lean issue loop: see the single-CTA kernel for the descriptor layouts.  Descriptor
+        // addresses are CTA-relative, so the leader's offsets name the same tiles in the peer.
+        if (rank == 0) {
+            const bool a_blk = p.a_blocked != 0;
+            const uint64_t da0 = a_blk ? make_smem_desc(smem_base, 16, 512, 4) : make_smem_desc(smem_base, 16, 1024, 2);
+            const uint64_t db0 = B_VNNI ? make_smem_desc(smem_base + UMMA_A_STAGE_BYTES, 16, 1024, 2)
+                                        : make_smem_desc(smem_base + UMMA_A_STAGE_BYTES, 8192, 1024, 2);
+            const uint32_t a_hi = static_cast<uint32_t>(da0 >> 32), b_hi = static_cast<uint32_t>(db0 >> 32);
+            const uint32_t a_lo0 = static_cast<uint32_t>(da0), b_lo0 = static_cast<uint32_t>(db0);
+            const uint32_t a_s1 = 2u, a_s2 = a_blk ? 512u : 4u, a_s3 = a_blk ? 514u : 6u;
+            constexpr uint32_t b_s = B_VNNI ? 2u : 128u;
+            constexpr uint32_t STAGE16 = STAGE >> 4;
+            const uint32_t idesc = p.idesc;
+            int stage = 0;
+            uint32_t phase = 0;
+            uint32_t soff = 0;
+            int local = 0;
+            bool ok = true;
+            for (int unit = pair_id; ok && unit < total_units; unit += num_pairs, ++local) {
+                const int tile = unit / p.splits, split = unit - tile * p.splits;
+                const int kb0 = split * p.kb_per_split;
+                const int kb1 = min(p.kb_total, kb0 + p.kb_per_split);
+                const int acc = local & 1;
+                if (!mbar_wait(tempty_bar(acc), ((local >> 1) & 1u) ^ 1u, abort_flag)) {
+                    if (lane == 0) give_up(0x200u + acc);
+                    ok = false;
+                    break;
+                }
+                tc_fence_after_sync();
+                const uint32_t d_tmem = tmem_base + acc * BN;
+                uint32_t accumulate = 0u;
+                for (int kb = kb0; kb < kb1; ++kb) {
+                    if (!mbar_wait(full_bar(stage), phase, abort_flag)) {
+                        if (lane == 0) give_up(0x300u + stage);
+                        ok = false;
+                        break;
+                    }
+                    tc_fence_after_sync();
+                    if (lane == 0) {
+                        const uint32_t a_lo = a_lo0 + soff, b_lo = b_lo0 + soff;
+                        umma_f16_pair_lohi(d_tmem, a_lo, a_hi, b_lo, b_hi, idesc, accumulate);
+                        umma_f16_pair_lohi(d_tmem, a_lo + a_s1, a_hi, b_lo + b_s, b_hi, idesc, 1u);
+                        umma_f16_pair_lohi(d_tmem, a_lo + a_s2, a_hi, b_lo + 2 * b_s, b_hi, idesc, 1u);
+                        umma_f16_pair_lohi(d_tmem, a_lo + a_s3, a_hi, b_lo + 3 * b_s, b_hi, idesc, 1u);
+                        umma_commit_pair(empty_bar(stage), 3);
+                        if (kb == kb1 - 1) umma_commit_pair(tfull_bar(acc), 3);
+                    }
+                    accumulate = 1u;
+                    __syncwarp();
+                    soff += STAGE16;
+                    if (++stage == STAGES) { stage = 0; phase ^= 1u; soff = 0; }
+                }
+                if (kb1 <= kb0 && lane == 0) umma_commit_pair(tfull_bar(acc), 3);
+                __syncwarp();
+            }
+        }
+    } else if (warp < 6) {
+        // ------------------------------------------------ epilogue (both CTAs, own 128 rows)
+        const int quarter = warp & 3;
+        int local = 0;
+        bool ok = true;
+        for (int unit = pair_id; ok && unit < total_units; unit += num_pairs, ++local) {
+            const int tile = unit / p.splits, split = unit - tile * p.splits;
+            int mb, nb;
+            umma_tile_coords(p, tile, mb, nb);
+            const int kb0 = split * p.kb_per_split;
+            const int kb1 = min(p.kb_total, kb0 + p.kb_per_split);
+            const int acc = local & 1;
+            if (!mbar_wait(tfull_bar(acc), (local >> 1) & 1u, abort_flag)) {
+                if (lane == 0) give_up(0x400u + acc);
+                ok = false;
+                break;
+            }
+            tc_fence_after_sync();
+            const int row = mb * BM2 + static_cast<int>(rank) * UMMA_BM + quarter * 32 + lane;
+            const bool empty_k = kb1 <= kb0;
+#pragma unroll 1
+            for (int c0 = 0; c0 < BN; c0 += 32) {
+                uint32_t v[32];
+                tmem_ld_32x32(tmem_base + acc * BN + c0 + (static_cast<uint32_t>(quarter * 32) << 16), v);
+                tmem_ld_wait();
+                umma_store_chunk(p, v, row, nb * BN + c0, split, empty_k);
+                __syncwarp();
+            }
+            tc_fence_before_sync();
+            mbar_arrive_cluster(map_to_cta(tempty_bar(acc), 0));
+        }
+    } else if (B_VNNI) {
+        // ------------------------------------------------ VNNI re-layout warps (both CTAs)
+        // Each CTA re-lays its HALF columns: rows n of a K-major tile, 128-byte rows, 16-byte
+        // chunk c of row n at chunk c ^ (n & 7) (see the single-CTA kernel).
+        const int tw = warp - 6;
+        int stage = 0;
+        uint32_t phase = 0;
+        bool ok = true;
+        const int kblocks32 = p.K / 32;
+        for (int unit = pair_id; ok && unit < total_units; unit += num_pairs) {
+            const int tile = unit / p.splits, split = unit - tile * p.splits;
+            int mb, nb;
+            umma_tile_coords(p, tile, mb, nb);
+            const int kb0 = split * p.kb_per_split;
+            const int kb1 = min(p.kb_total, kb0 + p.kb_per_split);
+            for (int kb = kb0; kb < kb1; ++kb) {
+                if (!mbar_wait(empty_bar(stage), phase ^ 1u, abort_flag)) {
+                    if (lane == 0) give_up(0x500u + stage);
+                    ok = false;
+                    break;
+                }
+                uint8_t* sb = gen_base + stage * STAGE + UMMA_A_STAGE_BYTES;
+                constexpr int ITEMS = (HALF / 32) * 2 * 4;
+#pragma unroll 4
+                for (int it = tw; it < ITEMS; it += 4) {
+                    const int q = it & 3, h = (it >> 2) & 1, j = it >> 3;
+                    const int nblk = (nb * BN + static_cast<int>(rank) * HALF) / 32 + j;
+                    const int kblk = kb * 2 + h;
+                    uint4 w = make_uint4(0u, 0u, 0u, 0u);
+                    if (nblk * 32 < p.N && kblk < kblocks32) {
+                        const uint32_t* src = p.Bblk +
+                            ((static_cast<size_t>(nblk) * kblocks32 + kblk) * 16 + 4 * q) * 32 + lane;
+                        w.x = __ldg(src);
+                        w.y = __ldg(src + 32);
+                        w.z = __ldg(src + 64);
+                        w.w = __ldg(src + 96);
+                    }
+                    const int n = j * 32 + lane;
+                    const int chunk = (h * 4 + q) ^ (n & 7);
+                    *reinterpret_cast<uint4*>(sb + n * 128 + chunk * 16) = w;
+                }
+                fence_proxy_async_smem();
+                __syncwarp();
+                if (lane == 0) mbar_arrive_cluster(map_to_cta(full_bar(stage), 0));
+                if (++stage == STAGES) { stage = 0; phase ^= 1u; }
+            }
+        }
+    }
+
+    tc_fence_before_sync();
+    __syncthreads();
+    cluster_sync_all();
+    if (warp == 1) {
+        tc_fence_after_sync();
+        tmem_dealloc_pair(tmem_base, TMEM_COLS);
+    }
+}
+
+}  // namespace nk

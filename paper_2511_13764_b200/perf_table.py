@@ -1,0 +1,113 @@
+"""Times every benchmark configuration through the C ABI and prints a table.
+
+    python -m paper_2511_13764_b200.perf_table [--iters 20] [--only c3] [--json out.json]
+
+Each launch is timed on its own with CUDA events on the launching stream, after
+warm-up, with L2 flushed in between (a 512 MB buffer is overwritten), so
+operands come from HBM as they would in a real pipeline.  Per configuration the
+table gives the median time, TFLOP/s, the algorithmic HBM GB/s, and the
+fraction of the roofline that binds it: the measured BF16 tensor peak, the
+measured HBM copy bandwidth, or the FP32 FMA-pipe peak (SMs x 128 x 2 x max SM
+clock).  It only measures; parity is the tests' business.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import sys
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+
+def peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            p = json.load(f)
+        return float(p["bf16_tflops"]), float(p["hbm_gbs"]), "measured"
+    return 1590.0, 6650.0, "fallback"
+
+
+def time_workload(w, iters, flags=0, flush=None):
+    import torch
+    import paper_2511_13764_b200 as nk
+    dev = torch.device("cuda", 0)
+    ein = torch.float32 if w.in_dtype == "f32" else torch.bfloat16
+    eout = torch.float32 if w.out_dtype == "f32" else torch.bfloat16
+    g = torch.Generator(device=dev).manual_seed(w.seed)
+    A = (torch.rand(w.M * w.K, device=dev, generator=g) * 2 - 1).to(ein)
+    B = (torch.rand(w.K * w.N, device=dev, generator=g) * 2 - 1).to(ein)
+    bias = (torch.randn(w.N, device=dev, generator=g) * 0.02).to(ein) if w.epilogue != "none" else None
+    C = torch.empty(w.M * w.N, dtype=eout, device=dev)
+    plan = nk.plan_for(w, flags=flags)
+    wsb = plan.workspace_bytes
+    ws = torch.empty(max(wsb, 16), dtype=torch.uint8, device=dev)
+    st = torch.cuda.current_stream()
+
+    def run():
+        plan.run(A, B, C, bias=bias, workspace=ws if wsb else None, workspace_bytes=wsb, stream=st.cuda_stream)
+
+    for _ in range(3):
+        run()
+    plan.check()
+    times = []
+    for _ in range(iters):
+        if flush is not None:
+            flush.fill_(1)
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record(st)
+        run()
+        b.record(st)
+        b.synchronize()
+        times.append(a.elapsed_time(b))
+    plan.check()
+    times.sort()
+    return times[len(times) // 2], times[0], plan.kernel_name, plan.launches_per_run
+
+
+def main():
+    import torch
+    import nk_inputs
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--iters", type=int, default=20)
+    ap.add_argument("--only", default=None, help="substring of the workload name")
+    ap.add_argument("--json", default=None)
+    ap.add_argument("--no-flush", action="store_true")
+    args = ap.parse_args()
+    if not torch.cuda.is_available():
+        raise SystemExit("needs a CUDA device")
+    tensor_peak, hbm_peak, src = peaks()
+    prop = torch.cuda.get_device_properties(0)
+    fma_peak = prop.multi_processor_count * 128 * 2 * 1.965e9 / 1e12
+    flush = None if args.no_flush else torch.empty(512 << 20, dtype=torch.uint8, device="cuda")
+    works = [nk_inputs.config(i) for i in (1, 2, 3, 4)] + nk_inputs.sweep() + nk_inputs.paper_mlp()
+    rows = []
+    print(f"| workload | kernel | launches | median us | TFLOP/s | alg. GB/s | bound | frac ({src}) |")
+    print("|---|---|---|---|---|---|---|---|")
+    for w in works:
+        if args.only and args.only not in w.name:
+            continue
+        med, best, kname, launches = time_workload(w, args.iters, flush=flush)
+        tf = w.flops / (med * 1e-3) / 1e12
+        gbs = w.algorithmic_bytes / (med * 1e-3) / 1e9
+        compute_peak = tensor_peak if w.in_dtype == "bf16" else fma_peak
+        t_compute = w.flops / (compute_peak * 1e12)
+        t_hbm = w.algorithmic_bytes / (hbm_peak * 1e9)
+        if t_hbm >= t_compute:
+            bound, frac = "hbm", gbs / hbm_peak
+        else:
+            bound, frac = ("tensor" if w.in_dtype == "bf16" else "alu"), tf / compute_peak
+        rows.append(dict(workload=w.name, kernel=kname, launches=launches, median_us=med * 1e3,
+                         best_us=best * 1e3, tflops=tf, gbs=gbs, bound=bound, frac=frac))
+        print(f"| {w.name} | {kname} | {launches} | {med * 1e3:.1f} | {tf:.1f} | {gbs:.0f} | {bound} | {frac:.3f} |",
+              flush=True)
+    if args.json:
+        with open(args.json, "w") as f:
+            json.dump(rows, f, indent=1)
+
+
+if __name__ == "__main__":
+    main()

@@ -96,7 +96,7 @@ def test_config3_bf16_mlp_bias_relu():
 
 def test_config4_bf16_8192():
     err, plan = check_workload(nk_inputs.config(4))
-    assert "umma_bf16_128x256" in plan.kernel_name
+    assert "umma_bf16_pair_256x256" in plan.kernel_name
 
 
 @pytest.mark.parametrize("w", nk_inputs.sweep(), ids=lambda w: w.name)

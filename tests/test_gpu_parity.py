@@ -77,12 +77,21 @@ UMMA_SHAPES = [(128, 64, 64), (128, 256, 64), (128, 64, 256), (256, 512, 1024), 
                (1, 8, 8), (130, 72, 72), (384, 328, 200), (1024, 1024, 1024), (16, 2048, 512)]
 
 
-@pytest.mark.parametrize("tile", [2, 3, 4])
+MODES = {"single": nk.FLAG_SINGLE_CTA, "pair": nk.FLAG_CTA_PAIR}
+
+
+def _kernel_prefix(mode, tile):
+    bn = 32 << (tile - 1)
+    return f"umma_bf16_pair_256x{bn}" if mode == "pair" else f"umma_bf16_128x{bn}"
+
+
+@pytest.mark.parametrize("mode,tile", [("single", 2), ("single", 3), ("single", 4), ("pair", 3), ("pair", 4)])
 @pytest.mark.parametrize("shape", UMMA_SHAPES)
-def test_umma_bf16_exact_integer(shape, tile):
+def test_umma_bf16_exact_integer(shape, tile, mode):
     M, N, K = shape
     w = W("umma", M, N, K, "bf16", integer=True)
-    run_and_check(w, flags=nk.flag_tile_n(tile), exact=True, expect_kernel=f"umma_bf16_128x{32 << (tile - 1)}")
+    run_and_check(w, flags=MODES[mode] | nk.flag_tile_n(tile), exact=True,
+                  expect_kernel=_kernel_prefix(mode, tile))
 
 
 @pytest.mark.parametrize("shape", UMMA_SHAPES)
@@ -91,32 +100,37 @@ def test_umma_bf16_random_auto(shape):
     run_and_check(W("umma", M, N, K, "bf16", seed=7))
 
 
+@pytest.mark.parametrize("mode", ["single", "pair"])
 @pytest.mark.parametrize("out_dtype", ["f32", "bf16"])
 @pytest.mark.parametrize("epi", ["none", "bias_relu"])
-def test_umma_bf16_epilogues(out_dtype, epi):
+def test_umma_bf16_epilogues(out_dtype, epi, mode):
     w = W("umma", 200, 328, 264, "bf16", out_dtype, epilogue=epi, integer=(out_dtype == "f32"))
-    run_and_check(w, exact=(out_dtype == "f32"))
-    run_and_check(W("umma", 256, 512, 512, "bf16", out_dtype, epilogue=epi, seed=8))
+    run_and_check(w, flags=MODES[mode], exact=(out_dtype == "f32"))
+    run_and_check(W("umma", 256, 512, 512, "bf16", out_dtype, epilogue=epi, seed=8), flags=MODES[mode])
 
 
+@pytest.mark.parametrize("mode", ["single", "pair"])
 @pytest.mark.parametrize("splits", [2, 3, 7])
 @pytest.mark.parametrize("out_dtype,epi", [("f32", "none"), ("bf16", "bias_relu")])
-def test_umma_bf16_splitk(splits, out_dtype, epi):
+def test_umma_bf16_splitk(splits, out_dtype, epi, mode):
+    f = MODES[mode] | nk.flag_splitk(splits)
     w = W("umma", 130, 200, 1096, "bf16", out_dtype, epilogue=epi, integer=(out_dtype == "f32"))
-    err, plan = run_and_check(w, flags=nk.flag_splitk(splits), exact=(out_dtype == "f32"))
+    err, plan = run_and_check(w, flags=f, exact=(out_dtype == "f32"))
     assert "splitk" in plan.kernel_name and plan.workspace_bytes > 0
-    run_and_check(W("umma", 130, 200, 1096, "bf16", out_dtype, epilogue=epi, seed=9), flags=nk.flag_splitk(splits))
+    assert ("pair" in plan.kernel_name) == (mode == "pair")
+    run_and_check(W("umma", 130, 200, 1096, "bf16", out_dtype, epilogue=epi, seed=9), flags=f)
 
 
-@pytest.mark.parametrize("tile", [2, 3, 4])
+@pytest.mark.parametrize("mode,tile", [("single", 2), ("single", 3), ("single", 4), ("pair", 3), ("pair", 4)])
 @pytest.mark.parametrize("flags", [0, nk.FLAG_REPACK_B], ids=["inkernel", "repack"])
 @pytest.mark.parametrize("shape", [(128, 64, 64), (32, 32, 32), (160, 224, 96), (512, 512, 512)])
-def test_umma_bf16_blocked(shape, flags, tile):
+def test_umma_bf16_blocked(shape, flags, tile, mode):
     M, N, K = shape
+    f = flags | MODES[mode] | nk.flag_tile_n(tile)
     w = W("blk", M, N, K, "bf16", layout="blocked32", integer=True)
-    err, plan = run_and_check(w, flags=flags | nk.flag_tile_n(tile), exact=True)
+    err, plan = run_and_check(w, flags=f, exact=True, expect_kernel=_kernel_prefix(mode, tile))
     assert "_ablk" in plan.kernel_name
-    run_and_check(W("blk", M, N, K, "bf16", layout="blocked32", seed=10), flags=flags | nk.flag_tile_n(tile))
+    run_and_check(W("blk", M, N, K, "bf16", layout="blocked32", seed=10), flags=f)
 
 
 def test_blocked_mixed_layouts():
