@@ -104,47 +104,72 @@ static cudaError_t allow_smem(K kernel, int bytes) {
 
 static int umma_stages_for(int bn) { return bn == 256 ? 4 : bn == 128 ? 6 : 8; }
 
+// Plan-time choice of (single CTA | CTA pair) x tile N x K splits for the BF16 kernel: the
+// counterpart of the paper's tile-size selection (Section 5a, found there by manual search).
+// A small cost model, fitted to timings on B200, is evaluated for every candidate:
+//   time = fixed + rounds * k-blocks-per-unit * t_kb(variant) [+ split-K partials and reduce],
+// floored by the HBM time of the operands.  t_kb is nearly independent of the tile width
+// (the stage pipeline is latency bound), so wide tiles win whenever they do not cost rounds.
+struct UmmaChoice { bool pair; int bn; int splits; double us; };
+
+static double umma_model_us(const nk_gemm_desc_t& d, int sms, bool pair, int bn, int splits) {
+    const int kb_total = ceil_div(d.K, UMMA_BK);
+    const int per = ceil_div(kb_total, splits);
+    const int eff_splits = ceil_div(kb_total, per);
+    const int64_t tiles = static_cast<int64_t>(ceil_div(d.M, pair ? 256 : 128)) * ceil_div(d.N, bn);
+    const int64_t units = tiles * eff_splits;
+    const int workers = pair ? sms / 2 : sms;
+    const double rounds = static_cast<double>((units + workers - 1) / workers);
+    double t_kb;  // microseconds per 64-wide k-block of one unit
+    if (pair) t_kb = bn == 256 ? 0.385 : 0.348;
+    else t_kb = bn == 256 ? 0.44 : bn == 128 ? 0.352 : 0.37;
+    const double eo = d.out_dtype == NK_BF16 ? 2.0 : 4.0;
+    const double mn = static_cast<double>(d.M) * d.N;
+    double us = (pair ? 12.0 : 10.0) + rounds * per * t_kb;
+    if (eff_splits > 1) us += 3.0 + eff_splits * mn * 4.0 / 3.0e6 + (eff_splits * 4.0 + eo) * mn / 5.0e6;
+    const double bytes = 2.0 * (static_cast<double>(d.M) * d.K + static_cast<double>(d.K) * d.N) + eo * mn;
+    const double hbm_us = bytes / 5.2e6;  // ~80 % of the copy bandwidth, bytes per microsecond
+    return us > hbm_us ? us : hbm_us;
+}
+
 static void choose_umma(nk_gemm_s* p) {
     const nk_gemm_desc_t& d = p->d;
     const int sms = p->sm_count;
     const int kb_total = ceil_div(d.K, UMMA_BK);
-    const int forced = (d.flags >> NK_FLAG_TILE_N_SHIFT) & 0xF;
-    // CTA pairs (256-row tiles) whenever there are at least two 128-row tiles of M.
-    bool pair = d.M > UMMA_BM;
-    if (d.flags & NK_FLAG_SINGLE_CTA) pair = false;
-    if (d.flags & NK_FLAG_CTA_PAIR) pair = true;
-    if (pair && forced == 2) pair = false;            // 64-wide tiles exist only single-CTA
-    const int workers = pair ? sms / 2 : sms;         // CTAs or CTA pairs
-    const int tiles_m = ceil_div(d.M, pair ? 2 * UMMA_BM : UMMA_BM);
-    int bn = pair ? 128 : 64;
-    if (forced >= 2 && forced <= 4) {
-        bn = 32 << (forced - 1);
-    } else {
-        const int cands[3] = {256, 128, 64};
-        for (int c : cands) {
-            if (pair && c == 64) break;
-            if (static_cast<int64_t>(tiles_m) * ceil_div(d.N, c) >= workers) { bn = c; break; }
+    const int forced_bn = (d.flags >> NK_FLAG_TILE_N_SHIFT) & 0xF;
+    const int forced_s = (d.flags >> NK_FLAG_SPLITK_SHIFT) & 0xFF;
+    const int split_cands[8] = {1, 2, 3, 4, 6, 8, 12, 16};
+    UmmaChoice best = {false, 64, 1, 1e30};
+    for (int pr = 0; pr < 2; ++pr) {
+        const bool pair = pr == 1;
+        if (pair && (d.flags & NK_FLAG_SINGLE_CTA)) continue;
+        if (!pair && (d.flags & NK_FLAG_CTA_PAIR) && forced_bn != 2) continue;
+        if (pair && d.M <= UMMA_BM && !(d.flags & NK_FLAG_CTA_PAIR)) continue;
+        for (int bn = 64; bn <= 256; bn *= 2) {
+            if (pair && bn == 64) continue;
+            if (forced_bn >= 2 && forced_bn <= 4 && bn != (32 << (forced_bn - 1))) continue;
+            for (int si = 0; si < 8; ++si) {
+                int splits = forced_s > 0 ? forced_s : split_cands[si];
+                if (forced_s > 0 && si > 0) break;
+                if (splits > kb_total) splits = kb_total;
+                if (forced_s == 0 && splits > 1) {
+                    if (kb_total / splits < 4) continue;  // >= 4 k-blocks per split
+                    if (static_cast<double>(splits) * d.M * d.N * 4.0 > 256.0 * 1024 * 1024) continue;
+                }
+                const double us = umma_model_us(d, sms, pair, bn, splits);
+                if (us < best.us) best = {pair, bn, splits, us};
+            }
         }
     }
-    p->pair = pair;
-    p->bn = bn;
-    p->stages = pair ? (bn == 256 ? 6 : 8) : umma_stages_for(bn);
-    const int tiles = tiles_m * ceil_div(d.N, bn);
-    int splits = 1;
-    const int forced_s = (d.flags >> NK_FLAG_SPLITK_SHIFT) & 0xFF;
-    if (forced_s > 0) {
-        splits = forced_s;
-    } else if (tiles * 2 <= workers) {
-        splits = workers / tiles;
-        const int max_by_k = kb_total / 4 > 0 ? kb_total / 4 : 1;  // >= 4 k-blocks per split
-        if (splits > max_by_k) splits = max_by_k;
-        if (splits > 32) splits = 32;
-    }
+    if (best.us >= 1e30) best = {false, 64, forced_s > 0 ? forced_s : 1, 0.0};  // contradictory overrides
+    int splits = best.splits;
     if (splits > kb_total) splits = kb_total;
     if (splits < 1) splits = 1;
-    // no empty split: shrink until the last one starts inside the K range
-    int per = ceil_div(kb_total, splits);
-    splits = ceil_div(kb_total, per);
+    const int per = ceil_div(kb_total, splits);
+    splits = ceil_div(kb_total, per);  // no empty split
+    p->pair = best.pair;
+    p->bn = best.bn;
+    p->stages = best.pair ? (best.bn == 256 ? 6 : 8) : umma_stages_for(best.bn);
     p->splits = splits;
     p->group_m = 8;
 }
