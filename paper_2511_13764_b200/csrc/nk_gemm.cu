@@ -42,6 +42,7 @@ struct nk_gemm_s {
     int max_pairs;         // co-resident clusters of 2 for the chosen pair kernel
     bool b_vnni_inkernel;  // blocked B re-laid inside the GEMM kernel
     bool b_repack;         // blocked B unpacked to row-major scratch first
+    bool b_3d;             // B tensor map is the 3-D slab view
     // SIMT
     int simt_tile;  // 128, 64 or 32
     int kt_per_split;
@@ -238,14 +239,30 @@ static nk_status_t encode_maps(nk_gemm_s* p, const void* A, const void* B) {
         return NK_ERR_CUDA;
     }
     if (!p->b_vnni_inkernel) {
-        // B row-major [K][N]: 64 (n) x 64 (k) boxes, N contiguous.
-        cuuint64_t dims[2] = {static_cast<cuuint64_t>(d.N), static_cast<cuuint64_t>(d.K)};
-        cuuint64_t strides[1] = {static_cast<cuuint64_t>(d.N) * 2};
-        cuuint32_t box[2] = {64, UMMA_BK};
-        cuuint32_t es[2] = {1, 1};
-        r = p->encode(&p->tmap_b, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(B), dims, strides,
-                      box, es, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
-                      CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+        // B row-major [K][N], N contiguous.  When N is a multiple of 64 the map is the 3-D view
+        // (n within a 64-column slab, k, slab): one box brings all the slabs of a stage, each
+        // as 64 k-rows of 128 B.  Otherwise 64 (n) x 64 (k) boxes, one per slab.
+        p->b_3d = d.N % 64 == 0;
+        const int slabs = (p->pair ? p->bn / 2 : p->bn) / 64;
+        if (p->b_3d) {
+            cuuint64_t dims[3] = {64, static_cast<cuuint64_t>(d.K), static_cast<cuuint64_t>(d.N / 64)};
+            cuuint64_t strides[2] = {static_cast<cuuint64_t>(d.N) * 2, 128};
+            cuuint32_t box[3] = {64, UMMA_BK, static_cast<cuuint32_t>(slabs)};
+            cuuint32_t es[3] = {1, 1, 1};
+            r = p->encode(&p->tmap_b, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(B), dims, strides,
+                          box, es, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+                          CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+            if (r != CUDA_SUCCESS) p->b_3d = false;   // fall back to per-slab boxes
+        }
+        if (!p->b_3d) {
+            cuuint64_t dims[2] = {static_cast<cuuint64_t>(d.N), static_cast<cuuint64_t>(d.K)};
+            cuuint64_t strides[1] = {static_cast<cuuint64_t>(d.N) * 2};
+            cuuint32_t box[2] = {64, UMMA_BK};
+            cuuint32_t es[2] = {1, 1};
+            r = p->encode(&p->tmap_b, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(B), dims, strides,
+                          box, es, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+                          CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+        }
         if (r != CUDA_SUCCESS) {
             snprintf(p->cuda_err, sizeof(p->cuda_err), "cuTensorMapEncodeTiled(B) failed: %d", (int)r);
             return NK_ERR_CUDA;
@@ -525,6 +542,7 @@ nk_status_t nk_gemm_run(nk_gemm_t p, const void* A, const void* B, const void* b
         up.kb_per_split = ceil_div(up.kb_total, p->splits);
         up.group_m = p->group_m;
         up.a_blocked = d.layout_a == NK_BLOCKED32;
+        up.b_3d = p->b_3d ? 1 : 0;
         up.epilogue = d.epilogue;
         up.out_bf16 = d.out_dtype == NK_BF16;
         up.idesc = make_idesc(p->pair ? 2 * UMMA_BM : UMMA_BM, p->bn, !p->b_vnni_inkernel);

@@ -13,8 +13,8 @@
 //   warp 1      MMA issuer and TMEM owner: 4 x tcgen05.mma 128 x BN x 16 per stage
 //   warps 2-5   epilogue: tcgen05.ld -> (+bias, ReLU, cvt) -> global stores; two
 //               TMEM accumulators so tile t's epilogue overlaps tile t+1's K loop
-//   warps 6-9   (VNNI-blocked B only) re-layout: read the [k/2][n][2] blocks from
-//               global memory as 32-bit words and write them word-transposed into
+//   warps 6-9   (VNNI-blocked B only) re-layout: copy the [k/2][n][2] blocks from
+//               global memory as 32-bit words, word-transposed (4-byte cp.async), into
 //               the K-major swizzled stage (the in-kernel counterpart of the
 //               paper's software-pipelined pack step, in the opposite direction)
 //
@@ -40,6 +40,7 @@ struct UmmaParams {
     int kb_per_split;   // ceil(kb_total / splits)
     int group_m;        // raster: this many M tiles sweep N together
     int a_blocked;      // A tensor map is the 4-D blocked view
+    int b_3d;           // B tensor map is the 3-D (n-in-slab, k, slab) view: one box per stage
     int epilogue;       // 0 none, 1 bias + ReLU
     int out_bf16;       // C element type
     uint32_t idesc;     // tcgen05 instruction descriptor
@@ -136,6 +137,52 @@ __device__ __forceinline__ void umma_store_chunk(const UmmaParams& p, uint32_t (
     }
 }
 
+// Re-layout of a VNNI-blocked B operand (Figure 1 of the paper: [k/2][n][2] inside every 32 x 32
+// block) into the K-major stage tile the tensor core reads: ROWS columns n x 64 k, 128-byte
+// rows, 16-byte chunk c of row n stored at chunk c ^ (n & 7) (the 128-byte swizzle).  Seen as
+// 32-bit words a block is 16 rows (k/2) x 32 words (n), and word (k2, n) belongs at row n, byte
+// (32 * half + 2 * k2) * 2: a word transpose.  Each lane copies one word per item with a 4-byte
+// cp.async (the scatter happens in the copy), so the copies of
+// several stages are in flight at once and no thread waits on global memory: the paper's
+// software-pipelined pack (Algorithm 3, AMX branch), in the opposite direction.
+constexpr int VNNI_LOOKAHEAD = 3;  // stages of copies in flight per warp before the oldest is awaited
+
+template <int ROWS>
+__device__ __forceinline__ void vnni_issue_stage(const UmmaParams& p, uint32_t sb, int n0, int kb,
+                                                 int tw, int lane) {
+    // Warp tw owns column octet tw of every 32-column block.  One warp instruction copies
+    // 8 columns x 4 consecutive word rows: its 32 destinations are 8 different swizzled
+    // chunks x 4 words (32 different banks) and its 4 source segments are whole 32-byte
+    // sectors.  Everything that depends only on the lane is computed once; the loops over
+    // (n-block j, k half h, word-row quad q) unroll into address adds.
+    const int kblocks32 = p.K / 32;
+    const int ln = lane & 7, lr = lane >> 3;
+    const int nn = tw * 8 + ln;                                  // column inside a block
+    const uint32_t dst_lane = sb + nn * 128 + lr * 4;
+    const uint32_t swz = static_cast<uint32_t>(nn & 7);
+    const int kblk0 = kb * 2;
+    const bool k_in0 = kblk0 < kblocks32, k_in1 = kblk0 + 1 < kblocks32;
+    const uint32_t* src_lane = p.Bblk + (static_cast<size_t>(kblk0) * 16 + lr) * 32 + nn;
+    const size_t nblk_stride = static_cast<size_t>(kblocks32) * 512;   // words per n-block
+#pragma unroll
+    for (int j = 0; j < ROWS / 32; ++j) {
+        const int nblk = n0 / 32 + j;
+        const bool n_in = nblk * 32 < p.N;
+        const uint32_t* src_j = src_lane + (n_in ? nblk * nblk_stride : 0);
+        const uint32_t dst_j = dst_lane + j * 4096;
+#pragma unroll
+        for (int h = 0; h < 2; ++h) {
+            const bool in = n_in && (h ? k_in1 : k_in0);
+            const uint32_t bytes = in ? 4u : 0u;
+            const uint32_t* src_h = in ? src_j + h * 512 : p.Bblk;
+#pragma unroll
+            for (int q = 0; q < 4; ++q)
+                cp_async_4(dst_j + (((h * 4 + q) ^ swz) << 4), src_h + (in ? q * 128 : 0), bytes);
+        }
+    }
+    cp_async_commit();
+}
+
 template <int BN, int STAGES, bool B_VNNI>
 __global__ void __launch_bounds__(B_VNNI ? 320 : 192, 1)
 umma_bf16_kernel(const __grid_constant__ CUtensorMap tmap_a,
@@ -194,8 +241,13 @@ umma_bf16_kernel(const __grid_constant__ CUtensorMap tmap_a,
 
     if (warp == 0) {
         // ------------------------------------------------ TMA producer
+        // One lane issues; like the MMA issuer its instruction stream paces the pipeline, so
+        // addresses advance by adds and the layout decisions are taken outside the loops.
+        const bool a_blk = p.a_blocked != 0;
+        const bool b3d = p.b_3d != 0;
         int stage = 0;
         uint32_t phase = 0;
+        uint32_t sa = smem_base, fb = full_bar(0);
         bool ok = true;
         for (int unit = blockIdx.x; ok && unit < total_units; unit += gridDim.x) {
             const int tile = unit / p.splits, split = unit - tile * p.splits;
@@ -203,32 +255,38 @@ umma_bf16_kernel(const __grid_constant__ CUtensorMap tmap_a,
             umma_tile_coords(p, tile, mb, nb);
             const int kb0 = split * p.kb_per_split;
             const int kb1 = min(p.kb_total, kb0 + p.kb_per_split);
-            for (int kb = kb0; kb < kb1; ++kb) {
+            const int row0 = mb * UMMA_BM, col0 = nb * BN;
+            int kx = kb0 * UMMA_BK;
+            for (int kb = kb0; kb < kb1; ++kb, kx += UMMA_BK) {
                 if (!mbar_wait(empty_bar(stage), phase ^ 1u, abort_flag)) {
                     if (lane == 0) give_up(0x100u + stage);
                     ok = false;
                     break;
                 }
                 if (lane == 0) {
-                    const uint32_t sa = smem_base + stage * STAGE;
                     const uint32_t sb = sa + UMMA_A_STAGE_BYTES;
-                    mbar_arrive_expect_tx(full_bar(stage),
-                                          UMMA_A_STAGE_BYTES + (B_VNNI ? 0 : B_STAGE));
-                    if (p.a_blocked) {
+                    mbar_arrive_expect_tx(fb, UMMA_A_STAGE_BYTES + (B_VNNI ? 0 : B_STAGE));
+                    if (a_blk) {
                         // two 32-wide K slabs, each 128 rows x 64 B (64-byte swizzle)
-                        tma_load_4d(sa, &tmap_a, full_bar(stage), 0, 0, kb * 2, mb * 4);
-                        tma_load_4d(sa + 8192, &tmap_a, full_bar(stage), 0, 0, kb * 2 + 1, mb * 4);
-                    } else
-                        tma_load_2d(sa, &tmap_a, full_bar(stage), kb * UMMA_BK, mb * UMMA_BM);
+                        tma_load_4d(sa, &tmap_a, fb, 0, 0, kb * 2, mb * 4);
+                        tma_load_4d(sa + 8192, &tmap_a, fb, 0, 0, kb * 2 + 1, mb * 4);
+                    } else {
+                        tma_load_2d(sa, &tmap_a, fb, kx, row0);
+                    }
                     if (!B_VNNI) {
+                        if (b3d) {
+                            tma_load_3d(sb, &tmap_b, fb, 0, kx, col0 >> 6);
+                        } else {
 #pragma unroll
-                        for (int j = 0; j < BN / 64; ++j)
-                            tma_load_2d(sb + j * 8192, &tmap_b, full_bar(stage), nb * BN + j * 64,
-                                        kb * UMMA_BK);
+                            for (int j = 0; j < BN / 64; ++j)
+                                tma_load_2d(sb + j * 8192, &tmap_b, fb, col0 + j * 64, kx);
+                        }
                     }
                 }
                 __syncwarp();
-                if (++stage == STAGES) { stage = 0; phase ^= 1u; }
+                sa += STAGE;
+                fb += 8;
+                if (++stage == STAGES) { stage = 0; phase ^= 1u; sa = smem_base; fb = full_bar(0); }
             }
         }
         // Drain: wait (bounded) until the consumer has released every stage this warp
@@ -336,14 +394,11 @@ umma_bf16_kernel(const __grid_constant__ CUtensorMap tmap_a,
         }
     } else if (B_VNNI) {
         // ------------------------------------------------ VNNI re-layout warps (6..9)
-        // Stage tile: BN rows (n) x 64 k, K-major, 128-byte rows, 16-byte chunk c of row n
-        // stored at chunk c ^ (n & 7).  A 32 x 32 block of B is 16 rows (k/2) of 32 words
-        // (n); word (k2, n) goes to row n, byte offset (kb_local*32 + 2*k2) * 2.
+        static_assert(VNNI_LOOKAHEAD < STAGES, "copies in flight must fit the ring");
         const int tw = warp - 6;
-        int stage = 0;
+        int stage = 0, astage = 0, pending = 0;
         uint32_t phase = 0;
         bool ok = true;
-        const int kblocks32 = p.K / 32;
         for (int unit = blockIdx.x; ok && unit < total_units; unit += gridDim.x) {
             const int tile = unit / p.splits, split = unit - tile * p.splits;
             int mb, nb;
@@ -356,32 +411,24 @@ umma_bf16_kernel(const __grid_constant__ CUtensorMap tmap_a,
                     ok = false;
                     break;
                 }
-                uint8_t* sb = gen_base + stage * STAGE + UMMA_A_STAGE_BYTES;
-                // work items: (n-block j, k-block half h, quad q) -> 4 words k2 = 4q..4q+3 at n = lane
-                constexpr int ITEMS = (BN / 32) * 2 * 4;
-#pragma unroll 4
-                for (int it = tw; it < ITEMS; it += 4) {
-                    const int q = it & 3, h = (it >> 2) & 1, j = it >> 3;
-                    const int nblk = nb * (BN / 32) + j;
-                    const int kblk = kb * 2 + h;
-                    uint4 w = make_uint4(0u, 0u, 0u, 0u);
-                    if (nblk * 32 < p.N && kblk < kblocks32) {
-                        const uint32_t* src = p.Bblk +
-                            ((static_cast<size_t>(nblk) * kblocks32 + kblk) * 16 + 4 * q) * 32 + lane;
-                        w.x = __ldg(src);
-                        w.y = __ldg(src + 32);
-                        w.z = __ldg(src + 64);
-                        w.w = __ldg(src + 96);
-                    }
-                    const int n = j * 32 + lane;
-                    const int chunk = (h * 4 + q) ^ (n & 7);
-                    *reinterpret_cast<uint4*>(sb + n * 128 + chunk * 16) = w;
-                }
-                fence_proxy_async_smem();
-                __syncwarp();
-                if (lane == 0) mbar_arrive(full_bar(stage));
+                vnni_issue_stage<BN>(p, smem_base + stage * STAGE + UMMA_A_STAGE_BYTES, nb * BN, kb, tw, lane);
                 if (++stage == STAGES) { stage = 0; phase ^= 1u; }
+                if (++pending > VNNI_LOOKAHEAD) {
+                    cp_async_wait_group<VNNI_LOOKAHEAD>();     // the oldest stage has landed
+                    fence_proxy_async_smem();
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(full_bar(astage));
+                    if (++astage == STAGES) astage = 0;
+                    --pending;
+                }
             }
+        }
+        cp_async_wait_group<0>();
+        fence_proxy_async_smem();
+        __syncwarp();
+        for (; ok && pending > 0; --pending) {
+            if (lane == 0) mbar_arrive(full_bar(astage));
+            if (++astage == STAGES) astage = 0;
         }
     }
 

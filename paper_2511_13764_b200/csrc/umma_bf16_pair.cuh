@@ -89,8 +89,12 @@ umma_bf16_pair_kernel(const __grid_constant__ CUtensorMap tmap_a,
 
     if (warp == 0) {
         // ------------------------------------------------ TMA producer (both CTAs)
+        const bool a_blk = p.a_blocked != 0;
+        const bool b3d = p.b_3d != 0;
+        const uint32_t lead_full0 = map_to_cta(full_bar(0), 0);  // leader's full[0], cluster address
         int stage = 0;
         uint32_t phase = 0;
+        uint32_t sa = smem_base, fb = full_bar(0), lfb = lead_full0;
         bool ok = true;
         for (int unit = pair_id; ok && unit < total_units; unit += num_pairs) {
             const int tile = unit / p.splits, split = unit - tile * p.splits;
@@ -100,33 +104,38 @@ umma_bf16_pair_kernel(const __grid_constant__ CUtensorMap tmap_a,
             const int kb1 = min(p.kb_total, kb0 + p.kb_per_split);
             const int row0 = mb * BM2 + static_cast<int>(rank) * UMMA_BM;
             const int col0 = nb * BN + static_cast<int>(rank) * HALF;
-            for (int kb = kb0; kb < kb1; ++kb) {
+            int kx = kb0 * UMMA_BK;
+            for (int kb = kb0; kb < kb1; ++kb, kx += UMMA_BK) {
                 if (!mbar_wait(empty_bar(stage), phase ^ 1u, abort_flag)) {
                     if (lane == 0) give_up(0x100u + stage);
                     ok = false;
                     break;
                 }
                 if (lane == 0) {
-                    const uint32_t sa = smem_base + stage * STAGE;
                     const uint32_t sb = sa + UMMA_A_STAGE_BYTES;
-                    const uint32_t lead_full = map_to_cta(full_bar(stage), 0);
                     if (rank == 0)
-                        mbar_arrive_expect_tx(full_bar(stage),
-                                              2u * (UMMA_A_STAGE_BYTES + (B_VNNI ? 0 : B_STAGE)));
-                    if (p.a_blocked) {
-                        tma_load_4d_pair(sa, &tmap_a, lead_full, 0, 0, kb * 2, row0 / 32);
-                        tma_load_4d_pair(sa + 8192, &tmap_a, lead_full, 0, 0, kb * 2 + 1, row0 / 32);
+                        mbar_arrive_expect_tx(fb, 2u * (UMMA_A_STAGE_BYTES + (B_VNNI ? 0 : B_STAGE)));
+                    if (a_blk) {
+                        tma_load_4d_pair(sa, &tmap_a, lfb, 0, 0, kb * 2, row0 / 32);
+                        tma_load_4d_pair(sa + 8192, &tmap_a, lfb, 0, 0, kb * 2 + 1, row0 / 32);
                     } else {
-                        tma_load_2d_pair(sa, &tmap_a, lead_full, kb * UMMA_BK, row0);
+                        tma_load_2d_pair(sa, &tmap_a, lfb, kx, row0);
                     }
                     if (!B_VNNI) {
+                        if (b3d) {
+                            tma_load_3d_pair(sb, &tmap_b, lfb, 0, kx, col0 >> 6);
+                        } else {
 #pragma unroll
-                        for (int j = 0; j < HALF / 64; ++j)
-                            tma_load_2d_pair(sb + j * 8192, &tmap_b, lead_full, col0 + j * 64, kb * UMMA_BK);
+                            for (int j = 0; j < HALF / 64; ++j)
+                                tma_load_2d_pair(sb + j * 8192, &tmap_b, lfb, col0 + j * 64, kx);
+                        }
                     }
                 }
                 __syncwarp();
-                if (++stage == STAGES) { stage = 0; phase ^= 1u; }
+                sa += STAGE;
+                fb += 8;
+                lfb += 8;
+                if (++stage == STAGES) { stage = 0; phase ^= 1u; sa = smem_base; fb = full_bar(0); lfb = lead_full0; }
             }
         }
         if (ok) {   // drain: every stage this CTA filled has been consumed
@@ -226,13 +235,14 @@ umma_bf16_pair_kernel(const __grid_constant__ CUtensorMap tmap_a,
         }
     } else if (B_VNNI) {
         // ------------------------------------------------ VNNI re-layout warps (both CTAs)
-        // Each CTA re-lays its HALF columns: rows n of a K-major tile, 128-byte rows, 16-byte
-        // chunk c of row n at chunk c ^ (n & 7) (see the single-CTA kernel).
+        // Each CTA re-lays its own HALF columns (see vnni_issue_stage) and reports each landed
+        // stage to the leader's full[] barrier.
+        static_assert(VNNI_LOOKAHEAD < STAGES, "copies in flight must fit the ring");
         const int tw = warp - 6;
-        int stage = 0;
+        const uint32_t lead_full0 = map_to_cta(full_bar(0), 0);
+        int stage = 0, astage = 0, pending = 0;
         uint32_t phase = 0;
         bool ok = true;
-        const int kblocks32 = p.K / 32;
         for (int unit = pair_id; ok && unit < total_units; unit += num_pairs) {
             const int tile = unit / p.splits, split = unit - tile * p.splits;
             int mb, nb;
@@ -245,31 +255,25 @@ umma_bf16_pair_kernel(const __grid_constant__ CUtensorMap tmap_a,
                     ok = false;
                     break;
                 }
-                uint8_t* sb = gen_base + stage * STAGE + UMMA_A_STAGE_BYTES;
-                constexpr int ITEMS = (HALF / 32) * 2 * 4;
-#pragma unroll 4
-                for (int it = tw; it < ITEMS; it += 4) {
-                    const int q = it & 3, h = (it >> 2) & 1, j = it >> 3;
-                    const int nblk = (nb * BN + static_cast<int>(rank) * HALF) / 32 + j;
-                    const int kblk = kb * 2 + h;
-                    uint4 w = make_uint4(0u, 0u, 0u, 0u);
-                    if (nblk * 32 < p.N && kblk < kblocks32) {
-                        const uint32_t* src = p.Bblk +
-                            ((static_cast<size_t>(nblk) * kblocks32 + kblk) * 16 + 4 * q) * 32 + lane;
-                        w.x = __ldg(src);
-                        w.y = __ldg(src + 32);
-                        w.z = __ldg(src + 64);
-                        w.w = __ldg(src + 96);
-                    }
-                    const int n = j * 32 + lane;
-                    const int chunk = (h * 4 + q) ^ (n & 7);
-                    *reinterpret_cast<uint4*>(sb + n * 128 + chunk * 16) = w;
-                }
-                fence_proxy_async_smem();
-                __syncwarp();
-                if (lane == 0) mbar_arrive_cluster(map_to_cta(full_bar(stage), 0));
+                vnni_issue_stage<HALF>(p, smem_base + stage * STAGE + UMMA_A_STAGE_BYTES,
+                                       nb * BN + static_cast<int>(rank) * HALF, kb, tw, lane);
                 if (++stage == STAGES) { stage = 0; phase ^= 1u; }
+                if (++pending > VNNI_LOOKAHEAD) {
+                    cp_async_wait_group<VNNI_LOOKAHEAD>();
+                    fence_proxy_async_smem();
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive_cluster(lead_full0 + 8u * astage);
+                    if (++astage == STAGES) astage = 0;
+                    --pending;
+                }
             }
+        }
+        cp_async_wait_group<0>();
+        fence_proxy_async_smem();
+        __syncwarp();
+        for (; ok && pending > 0; --pending) {
+            if (lane == 0) mbar_arrive_cluster(lead_full0 + 8u * astage);
+            if (++astage == STAGES) astage = 0;
         }
     }
 
