@@ -175,38 +175,66 @@ static void choose_umma(nk_gemm_s* p) {
     p->group_m = 8;
 }
 
+// Plan-time choice of tile and K splits for the FP32 kernel (the counterpart of the paper's
+// register-tile selection, Section 5a).  Model, fitted to B200 timings: an SM holds `res`
+// CTAs of a variant; a CTA's 16-wide k-tile costs tile^2 * 16 FMAs on 128 lanes, slowed by
+// the CTAs sharing the SM and by the variant's efficiency (wide thread tiles need fewer
+// shared-memory loads per FMA); units are scheduled in waves of sms * res.
+static double simt_model_us(const nk_gemm_desc_t& d, int sms, int tile, int splits) {
+    const int ktiles = ceil_div(d.K, SIMT_BK);
+    const int per = ceil_div(ktiles, splits);
+    const int eff_splits = ceil_div(ktiles, per);
+    const int64_t tiles = static_cast<int64_t>(ceil_div(d.M, tile)) * ceil_div(d.N, tile);
+    const int64_t units = tiles * eff_splits;
+    const int res = tile == 128 ? 2 : tile == 64 ? 4 : 16;
+    const double eff = tile == 128 ? 0.75 : tile == 64 ? 0.50 : 0.37;
+    const int64_t slots = static_cast<int64_t>(sms) * res;
+    const int64_t full_waves = units / slots;
+    const int64_t rest = units - full_waves * slots;
+    const double clk_per_kt = static_cast<double>(tile) * tile * SIMT_BK / 128.0;   // one CTA alone on an SM
+    const double us_per_kt = clk_per_kt / 1965.0 / eff;
+    // a CTA prefetches one k-tile only, so a k-tile never takes less than a global-load round trip
+    const double lat_us = 0.85;
+    auto kt_us = [&](double sharing) { const double t = us_per_kt * sharing; return t > lat_us ? t : lat_us; };
+    double us = 8.0 + full_waves * per * kt_us(res);
+    if (rest > 0) us += per * kt_us(static_cast<double>((rest + sms - 1) / sms));
+    const double mn = static_cast<double>(d.M) * d.N;
+    if (eff_splits > 1) us += 3.0 + (2.0 * eff_splits + 1.0) * mn * 4.0 / 4.0e6;
+    const double bytes = 4.0 * (static_cast<double>(d.M) * d.K + static_cast<double>(d.K) * d.N + mn);
+    // small tiles keep few bytes in flight: they reach a fraction of the HBM bandwidth only
+    const double hbm_us = bytes / (tile == 128 ? 5.0e6 : tile == 64 ? 3.5e6 : 1.8e6);
+    return us > hbm_us ? us : hbm_us;
+}
+
 static void choose_simt(nk_gemm_s* p) {
     const nk_gemm_desc_t& d = p->d;
     const int sms = p->sm_count;
     const int ktiles = ceil_div(d.K, SIMT_BK);
-    const int64_t t128 = static_cast<int64_t>(ceil_div(d.M, 128)) * ceil_div(d.N, 128);
-    const int64_t t64 = static_cast<int64_t>(ceil_div(d.M, 64)) * ceil_div(d.N, 64);
-    const int64_t t32 = static_cast<int64_t>(ceil_div(d.M, 32)) * ceil_div(d.N, 32);
-    int tile;
-    int64_t tiles;
-    int resident;  // CTAs of this variant one SM holds
-    if (t128 >= 2 * sms && d.M >= 96) { tile = 128; tiles = t128; resident = 2; }
-    else if (t64 >= sms && d.M >= 48) { tile = 64; tiles = t64; resident = 6; }
-    else { tile = 32; tiles = t32; resident = 16; }
     const int forced = (d.flags >> NK_FLAG_TILE_N_SHIFT) & 0xF;
-    if (forced == 1) { tile = 32; tiles = t32; resident = 16; }
-    if (forced == 2) { tile = 64; tiles = t64; resident = 6; }
-    if (forced == 3) { tile = 128; tiles = t128; resident = 2; }
-    p->simt_tile = tile;
-    int splits = 1;
     const int forced_s = (d.flags >> NK_FLAG_SPLITK_SHIFT) & 0xFF;
-    if (forced_s > 0) {
-        splits = forced_s;
-    } else if (tiles < static_cast<int64_t>(sms) * resident / 2) {
-        splits = static_cast<int>(static_cast<int64_t>(sms) * resident / tiles);
-        const int max_by_k = ktiles / 8 > 0 ? ktiles / 8 : 1;  // >= 8 k-tiles (128 k) per split
-        if (splits > max_by_k) splits = max_by_k;
-        if (splits > 64) splits = 64;
+    const int split_cands[10] = {1, 2, 3, 4, 6, 8, 12, 16, 24, 32};
+    int best_tile = 32, best_splits = 1;
+    double best_us = 1e30;
+    for (int tile = 32; tile <= 128; tile *= 2) {
+        if (forced >= 1 && forced <= 3 && tile != (16 << forced)) continue;
+        for (int si = 0; si < 10; ++si) {
+            int splits = forced_s > 0 ? forced_s : split_cands[si];
+            if (forced_s > 0 && si > 0) break;
+            if (splits > ktiles) splits = ktiles;
+            if (forced_s == 0 && splits > 1) {
+                if (ktiles / splits < 8) continue;   // >= 8 k-tiles (128 k) per split
+                if (static_cast<double>(splits) * d.M * d.N * 4.0 > 256.0 * 1024 * 1024) continue;
+            }
+            const double us = simt_model_us(d, sms, tile, splits);
+            if (us < best_us) { best_us = us; best_tile = tile; best_splits = splits; }
+        }
     }
+    int splits = best_splits;
     if (splits > ktiles) splits = ktiles;
     if (splits < 1) splits = 1;
-    int per = ceil_div(ktiles, splits);
+    const int per = ceil_div(ktiles, splits);
     splits = ceil_div(ktiles, per);
+    p->simt_tile = best_tile;
     p->splits = splits;
     p->kt_per_split = per;
 }

@@ -27,7 +27,7 @@ struct SimtParams {
 };
 
 template <int BM, int BN, int TM, int TN>
-__global__ void __launch_bounds__((BM / TM) * (BN / TN))
+__global__ void __launch_bounds__((BM / TM) * (BN / TN), (BM >= 128 ? 2 : 1))
 simt_f32_kernel(const SimtParams p) {
     constexpr int THREADS = (BM / TM) * (BN / TN);
     constexpr int TX = BN / TN;          // threads across N
