@@ -23,7 +23,7 @@ namespace nk {
 // loads the library).  Kernels receive its device address as a parameter.
 __device__ unsigned int g_status_word[4];
 
-enum Variant { V_NAIVE = 0, V_SIMT = 1, V_UMMA = 2 };
+enum Variant { V_NAIVE = 0, V_SIMT = 1, V_UMMA = 2, V_SKINNY = 3 };
 
 typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*,
                                   const cuuint64_t*, const cuuint64_t*, const cuuint32_t*,
@@ -46,6 +46,7 @@ struct nk_gemm_s {
     // SIMT
     int simt_tile;  // 128, 64 or 32
     int kt_per_split;
+    int skinny_kc;  // FP32 skinny kernel: k per CTA
     // workspace layout
     size_t ws_repack_bytes, ws_partial_bytes;
     // device status word
@@ -237,6 +238,24 @@ static void choose_simt(nk_gemm_s* p) {
     p->simt_tile = best_tile;
     p->splits = splits;
     p->kt_per_split = per;
+}
+
+// FP32, M <= 32: the streaming kernel.  K is cut so that about four CTAs per SM stream B at
+// once; a CTA's slice of A (rows x k-chunk) must fit its 32 KB of shared memory.
+static void choose_skinny(nk_gemm_s* p) {
+    const nk_gemm_desc_t& d = p->d;
+    const int mr = d.M <= 16 ? 16 : 32;
+    const int kc_max = SKINNY_A_FLOATS / mr;
+    const int col_tiles = ceil_div(d.N, SKINNY_COLS);
+    const int forced_s = (d.flags >> NK_FLAG_SPLITK_SHIFT) & 0xFF;
+    int want = forced_s > 0 ? forced_s : ceil_div(4 * p->sm_count, col_tiles);
+    if (want < 1) want = 1;
+    int kc = ceil_div(ceil_div(d.K, want), 8) * 8;
+    if (kc < 64 && forced_s == 0) kc = 64;
+    if (kc > kc_max) kc = kc_max;
+    if (kc > ceil_div(d.K, 8) * 8) kc = ceil_div(d.K, 8) * 8;
+    p->skinny_kc = kc;
+    p->splits = ceil_div(d.K, kc);
 }
 
 static nk_status_t encode_maps(nk_gemm_s* p, const void* A, const void* B) {
@@ -459,6 +478,13 @@ nk_status_t nk_gemm_create(const nk_gemm_desc_t* desc, nk_gemm_t* out) {
         p->variant = V_NAIVE;
         p->launches = 1;
         snprintf(p->name, sizeof(p->name), "naive");
+    } else if (d.in_dtype == NK_F32 && d.M <= 32 && force != NK_FLAG_KERNEL_SIMT) {
+        p->variant = V_SKINNY;
+        choose_skinny(p);
+        p->ws_partial_bytes = p->splits > 1 ? static_cast<size_t>(p->splits) * d.M * d.N * 4 : 0;
+        p->launches = p->splits > 1 ? 2 : 1;
+        snprintf(p->name, sizeof(p->name), "simt_f32_skinny_%dx512_kc%d_splitk%d", d.M <= 16 ? 16 : 32,
+                 p->skinny_kc, p->splits);
     } else if (d.in_dtype == NK_F32) {
         p->variant = V_SIMT;
         choose_simt(p);
@@ -540,7 +566,16 @@ nk_status_t nk_gemm_run(nk_gemm_t p, const void* A, const void* B, const void* b
     uint8_t* ws = static_cast<uint8_t*>(workspace);
     float* partial = p->ws_partial_bytes ? reinterpret_cast<float*>(ws + p->ws_repack_bytes) : nullptr;
 
-    if (p->variant == V_SIMT) {
+    if (p->variant == V_SKINNY) {
+        SkinnyParams kp = {static_cast<int>(d.M), static_cast<int>(d.N), static_cast<int>(d.K), p->skinny_kc,
+                           p->splits, d.epilogue, static_cast<const float*>(A), static_cast<const float*>(B),
+                           static_cast<const float*>(bias), static_cast<float*>(C), partial};
+        dim3 grid(ceil_div(d.N, SKINNY_COLS), p->splits);
+        if (d.M <= 16) simt_f32_skinny_kernel<16><<<grid, SKINNY_THREADS, 0, st>>>(kp);
+        else simt_f32_skinny_kernel<32><<<grid, SKINNY_THREADS, 0, st>>>(kp);
+        e = cudaGetLastError();
+        if (e != cudaSuccess) { set_err(p, "skinny launch", e); return NK_ERR_CUDA; }
+    } else if (p->variant == V_SIMT) {
         SimtParams sp = {static_cast<int>(d.M), static_cast<int>(d.N), static_cast<int>(d.K), p->splits,
                          p->kt_per_split, d.epilogue, static_cast<const float*>(A),
                          static_cast<const float*>(B), static_cast<const float*>(bias),

@@ -160,3 +160,108 @@ simt_f32_kernel(const SimtParams p) {
 }
 
 }  // namespace nk
+
+namespace nk {
+
+// Skinny FP32 GEMM (M <= MR rows): bound by the one pass over B, not by the FMA pipe.
+// A CTA of 128 threads owns 512 consecutive columns and a chunk of K: it parks its slice of A
+// in shared memory once (transposed, so the MR values of one k are read with broadcast
+// 128-bit loads), then streams B with no barrier in the loop: every thread keeps 8 independent
+// 16-byte loads in flight (row segments of 512 B per warp) and holds an MR x 4 block of C in
+// registers (Algorithm 1's resident accumulator).  K chunks are combined by the split-K reduce.
+constexpr int SKINNY_COLS = 512;
+constexpr int SKINNY_THREADS = 128;
+constexpr int SKINNY_A_FLOATS = 8192;   // MR * k-chunk <= this (32 KB of shared memory)
+
+struct SkinnyParams {
+    int M, N, K;
+    int kc;            // k per CTA (multiple of 8)
+    int splits;        // gridDim.y
+    int epilogue;
+    const float* A;
+    const float* B;
+    const float* bias;
+    float* C;
+    float* partial;
+};
+
+template <int MR>
+__global__ void __launch_bounds__(SKINNY_THREADS, MR == 16 ? 4 : 2) simt_f32_skinny_kernel(const SkinnyParams p) {
+    __shared__ __align__(16) float As[SKINNY_A_FLOATS];   // As[kk][MR]
+    const int t = threadIdx.x;
+    const int n = blockIdx.x * SKINNY_COLS + t * 4;
+    const int k0 = blockIdx.y * p.kc;
+    const int k1 = min(p.K, k0 + p.kc);
+    const int klen = k1 - k0;
+
+    // A slice: rows 0..MR-1 (zero beyond M), k0..k1, four k per load
+    for (int idx = t; idx < MR * (p.kc / 4); idx += SKINNY_THREADS) {
+        const int m = idx % MR, kq = (idx / MR) * 4;
+        float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
+        if (m < p.M && k0 + kq < k1)
+            v = __ldg(reinterpret_cast<const float4*>(p.A + static_cast<size_t>(m) * p.K + k0 + kq));
+        As[(kq + 0) * MR + m] = v.x;
+        As[(kq + 1) * MR + m] = v.y;
+        As[(kq + 2) * MR + m] = v.z;
+        As[(kq + 3) * MR + m] = v.w;
+    }
+    __syncthreads();
+
+    float acc[MR][4];
+#pragma unroll
+    for (int m = 0; m < MR; ++m) acc[m][0] = acc[m][1] = acc[m][2] = acc[m][3] = 0.f;
+
+    const bool col_ok = n < p.N;
+    const float* bptr = p.B + static_cast<size_t>(k0) * p.N + (col_ok ? n : 0);
+    float4 bnext[8];
+    auto load_group = [&](int kk) {
+#pragma unroll
+        for (int i = 0; i < 8; ++i)
+            bnext[i] = (col_ok && kk + i < klen)
+                           ? __ldcs(reinterpret_cast<const float4*>(bptr + static_cast<size_t>(kk + i) * p.N))
+                           : make_float4(0.f, 0.f, 0.f, 0.f);
+    };
+    load_group(0);
+    for (int kk = 0; kk < klen; kk += 8) {
+        float4 b[8];
+#pragma unroll
+        for (int i = 0; i < 8; ++i) b[i] = bnext[i];
+        if (kk + 8 < klen) load_group(kk + 8);
+#pragma unroll
+        for (int i = 0; i < 8; ++i) {
+            const float* arow = &As[(kk + i) * MR];
+#pragma unroll
+            for (int mq = 0; mq < MR; mq += 4) {
+                const float4 a = *reinterpret_cast<const float4*>(arow + mq);
+                const float av[4] = {a.x, a.y, a.z, a.w};
+#pragma unroll
+                for (int j = 0; j < 4; ++j) {
+                    acc[mq + j][0] = fmaf(av[j], b[i].x, acc[mq + j][0]);
+                    acc[mq + j][1] = fmaf(av[j], b[i].y, acc[mq + j][1]);
+                    acc[mq + j][2] = fmaf(av[j], b[i].z, acc[mq + j][2]);
+                    acc[mq + j][3] = fmaf(av[j], b[i].w, acc[mq + j][3]);
+                }
+            }
+        }
+    }
+
+    if (!col_ok) return;
+    const bool to_partial = p.splits > 1;
+    float* out = to_partial ? p.partial + static_cast<size_t>(blockIdx.y) * p.M * p.N : p.C;
+    float4 bv = make_float4(0.f, 0.f, 0.f, 0.f);
+    if (!to_partial && p.epilogue) bv = __ldg(reinterpret_cast<const float4*>(p.bias + n));
+#pragma unroll
+    for (int m = 0; m < MR; ++m) {
+        if (m >= p.M) break;
+        float4 v = make_float4(acc[m][0], acc[m][1], acc[m][2], acc[m][3]);
+        if (!to_partial && p.epilogue) {
+            v.x = fmaxf(v.x + bv.x, 0.f);
+            v.y = fmaxf(v.y + bv.y, 0.f);
+            v.z = fmaxf(v.z + bv.z, 0.f);
+            v.w = fmaxf(v.w + bv.w, 0.f);
+        }
+        *reinterpret_cast<float4*>(out + static_cast<size_t>(m) * p.N + n) = v;
+    }
+}
+
+}  // namespace nk

@@ -55,8 +55,9 @@ __host__ __device__ constexpr int umma_b_stage_bytes(int BN) { return BN * UMMA_
 __host__ __device__ constexpr int umma_stage_bytes(int BN) {
     return UMMA_A_STAGE_BYTES + umma_b_stage_bytes(BN);
 }
+constexpr int UMMA_EPI_STAGING = 4 * 4096;   // one 32 x 32 FP32 chunk per epilogue warp
 __host__ __device__ constexpr int umma_smem_bytes(int BN, int stages) {
-    return stages * umma_stage_bytes(BN) + 1024 /*alignment slack*/ + 256 /*barriers*/;
+    return stages * umma_stage_bytes(BN) + 1024 /*alignment slack*/ + 256 /*barriers*/ + UMMA_EPI_STAGING;
 }
 
 // tile id -> (m block, n block): groups of `group_m` M tiles sweep across N so
@@ -78,28 +79,23 @@ __device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi) {
     return *reinterpret_cast<uint32_t*>(&v);
 }
 
-// Epilogue for one 32-column chunk of one row held in registers (FP32 bit patterns):
-// either the raw FP32 partial of a K split, or bias + ReLU (Section 6, "MLP") followed by
-// the single store of C as FP32 or BF16 (one RNE rounding).  16-byte stores; columns are
-// predicated in groups (N is a multiple of 8).
-__device__ __forceinline__ void umma_store_chunk(const UmmaParams& p, uint32_t (&v)[32], int row,
-                                                 int col0, int split, bool empty_k) {
-    if (row >= p.M || col0 >= p.N) return;
-    const size_t row_off = static_cast<size_t>(row) * p.N;
+// Epilogue for one 32 x 32 chunk of the accumulator: lane t holds row `row0 + t`, columns
+// col0 .. col0+31 as FP32 bit patterns.  Either the raw FP32 partial of a K split, or bias +
+// ReLU (Section 6, "MLP") followed by the single store of C as FP32 or BF16 (one RNE rounding).
+// FP32 rows are transposed through a 4 KB per-warp shared-memory buffer (16-byte chunk g of
+// row t kept at chunk g ^ (t & 7): conflict-free both ways) so that every store instruction
+// writes four whole 128-byte row segments instead of 32 scattered 16-byte pieces.  BF16 rows
+// (64 bytes each) are stored directly.  Columns are predicated in groups (N is a multiple of 8).
+__device__ __forceinline__ void umma_store_chunk(const UmmaParams& p, uint32_t (&v)[32], int row0, int lane,
+                                                 int col0, int split, bool empty_k, uint8_t* staging) {
+    if (col0 >= p.N || row0 >= p.M) return;           // warp-uniform
+    const int row = row0 + lane;
     if (empty_k) {
 #pragma unroll
         for (int i = 0; i < 32; ++i) v[i] = 0u;
     }
-    if (p.splits > 1) {
-        float* dst = p.partial + static_cast<size_t>(split) * p.M * p.N + row_off + col0;
-#pragma unroll
-        for (int g = 0; g < 8; ++g)
-            if (col0 + 4 * g < p.N)
-                *reinterpret_cast<uint4*>(dst + 4 * g) =
-                    make_uint4(v[4 * g], v[4 * g + 1], v[4 * g + 2], v[4 * g + 3]);
-        return;
-    }
-    if (p.epilogue) {
+    const bool to_partial = p.splits > 1;
+    if (!to_partial && p.epilogue) {
         const uint4* bsrc = reinterpret_cast<const uint4*>(static_cast<const uint16_t*>(p.bias) + col0);
 #pragma unroll
         for (int g = 0; g < 4; ++g) {
@@ -115,8 +111,9 @@ __device__ __forceinline__ void umma_store_chunk(const UmmaParams& p, uint32_t (
             }
         }
     }
-    if (p.out_bf16) {
-        uint16_t* dst = static_cast<uint16_t*>(p.C) + row_off + col0;
+    if (!to_partial && p.out_bf16) {
+        if (row >= p.M) return;
+        uint16_t* dst = static_cast<uint16_t*>(p.C) + static_cast<size_t>(row) * p.N + col0;
 #pragma unroll
         for (int g = 0; g < 4; ++g)
             if (col0 + 8 * g < p.N) {
@@ -127,14 +124,25 @@ __device__ __forceinline__ void umma_store_chunk(const UmmaParams& p, uint32_t (
                 o.w = pack_bf16x2(__uint_as_float(v[8 * g + 6]), __uint_as_float(v[8 * g + 7]));
                 *reinterpret_cast<uint4*>(dst + 8 * g) = o;
             }
-    } else {
-        float* dst = static_cast<float*>(p.C) + row_off + col0;
-#pragma unroll
-        for (int g = 0; g < 8; ++g)
-            if (col0 + 4 * g < p.N)
-                *reinterpret_cast<uint4*>(dst + 4 * g) =
-                    make_uint4(v[4 * g], v[4 * g + 1], v[4 * g + 2], v[4 * g + 3]);
+        return;
     }
+    // FP32: registers -> staging (row per lane) -> global (4 row segments per instruction)
+#pragma unroll
+    for (int g = 0; g < 8; ++g)
+        *reinterpret_cast<uint4*>(staging + lane * 128 + ((g ^ (lane & 7)) << 4)) =
+            make_uint4(v[4 * g], v[4 * g + 1], v[4 * g + 2], v[4 * g + 3]);
+    __syncwarp();
+    float* out = to_partial ? p.partial + static_cast<size_t>(split) * p.M * p.N : static_cast<float*>(p.C);
+    const int c = lane & 7, rsub = lane >> 3;
+    const bool col_ok = col0 + 4 * c < p.N;
+#pragma unroll
+    for (int i = 0; i < 8; ++i) {
+        const int r = 4 * i + rsub;
+        const uint4 val = *reinterpret_cast<const uint4*>(staging + r * 128 + ((c ^ (r & 7)) << 4));
+        if (col_ok && row0 + r < p.M)
+            *reinterpret_cast<uint4*>(out + static_cast<size_t>(row0 + r) * p.N + col0 + 4 * c) = val;
+    }
+    __syncwarp();   // the buffer is reused by the next chunk
 }
 
 // Re-layout of a VNNI-blocked B operand (Figure 1 of the paper: [k/2][n][2] inside every 32 x 32
@@ -378,15 +386,16 @@ umma_bf16_kernel(const __grid_constant__ CUtensorMap tmap_a,
                 break;
             }
             tc_fence_after_sync();
-            const int row = mb * UMMA_BM + quarter * 32 + lane;
+            const int row0 = mb * UMMA_BM + quarter * 32;
             const bool empty_k = kb1 <= kb0;
+            uint8_t* staging = gen_base + STAGES * STAGE + 256 + (warp - 2) * 4096;
 #pragma unroll 1
             for (int c0 = 0; c0 < BN; c0 += 32) {
                 uint32_t v[32];
                 tmem_ld_32x32(tmem_base + acc * BN + c0 + (static_cast<uint32_t>(quarter * 32) << 16),
                               v);
                 tmem_ld_wait();
-                umma_store_chunk(p, v, row, nb * BN + c0, split, empty_k);
+                umma_store_chunk(p, v, row0, lane, nb * BN + c0, split, empty_k, staging);
                 __syncwarp();
             }
             tc_fence_before_sync();

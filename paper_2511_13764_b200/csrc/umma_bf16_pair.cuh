@@ -24,7 +24,7 @@ namespace nk {
 
 __host__ __device__ constexpr int pair_stage_bytes(int BN) { return UMMA_A_STAGE_BYTES + (BN / 2) * UMMA_BK * 2; }
 __host__ __device__ constexpr int pair_smem_bytes(int BN, int stages) {
-    return stages * pair_stage_bytes(BN) + 1024 + 256;
+    return stages * pair_stage_bytes(BN) + 1024 + 256 + UMMA_EPI_STAGING;
 }
 
 // UmmaParams as for the single-CTA kernel, with tiles_m counted in 256-row tiles.
@@ -220,14 +220,15 @@ umma_bf16_pair_kernel(const __grid_constant__ CUtensorMap tmap_a,
                 break;
             }
             tc_fence_after_sync();
-            const int row = mb * BM2 + static_cast<int>(rank) * UMMA_BM + quarter * 32 + lane;
+            const int row0 = mb * BM2 + static_cast<int>(rank) * UMMA_BM + quarter * 32;
             const bool empty_k = kb1 <= kb0;
+            uint8_t* staging = gen_base + STAGES * STAGE + 256 + (warp - 2) * 4096;
 #pragma unroll 1
             for (int c0 = 0; c0 < BN; c0 += 32) {
                 uint32_t v[32];
                 tmem_ld_32x32(tmem_base + acc * BN + c0 + (static_cast<uint32_t>(quarter * 32) << 16), v);
                 tmem_ld_wait();
-                umma_store_chunk(p, v, row, nb * BN + c0, split, empty_k);
+                umma_store_chunk(p, v, row0, lane, nb * BN + c0, split, empty_k, staging);
                 __syncwarp();
             }
             tc_fence_before_sync();

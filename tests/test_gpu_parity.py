@@ -72,6 +72,24 @@ def test_simt_f32_bias_relu():
     run_and_check(W("simt", 512, 1024, 1024, "f32", epilogue="bias_relu", seed=5))
 
 
+@pytest.mark.parametrize("epi", ["none", "bias_relu"])
+@pytest.mark.parametrize("shape", [(16, 1024, 1024), (1, 4, 4), (7, 520, 100), (32, 2052, 1000),
+                                   (17, 512, 64), (16, 4096, 4096)])
+def test_simt_f32_skinny(shape, epi):
+    """M <= 32 goes to the streaming kernel (one pass over B, K chunks reduced afterwards)."""
+    M, N, K = shape
+    err, plan = run_and_check(W("skinny", M, N, K, "f32", epilogue=epi, integer=True), exact=True,
+                              expect_kernel="simt_f32_skinny")
+    run_and_check(W("skinny", M, N, K, "f32", epilogue=epi, seed=6), expect_kernel="simt_f32_skinny")
+
+
+@pytest.mark.parametrize("splits", [1, 3])
+def test_simt_f32_skinny_forced_splits(splits):
+    w = W("skinny", 16, 1032, 600, "f32", integer=True)
+    err, plan = run_and_check(w, flags=nk.flag_splitk(splits), exact=True, expect_kernel="simt_f32_skinny")
+    assert (plan.workspace_bytes > 0) == (plan.launches_per_run == 2)
+
+
 # ---------------------------------------------------------------- BF16 tcgen05 kernel
 UMMA_SHAPES = [(128, 64, 64), (128, 256, 64), (128, 64, 256), (256, 512, 1024), (100, 64, 64),
                (1, 8, 8), (130, 72, 72), (384, 328, 200), (1024, 1024, 1024), (16, 2048, 512)]

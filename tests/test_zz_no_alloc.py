@@ -32,10 +32,14 @@ def _run_both(plan, w, seed):
     ref = torch.full((w.M * w.N,), float("nan"), dtype=out_dt, device="cuda")
     plan.run(dA, dB, ref, bias=db, workspace=ws, stream=sp)
     got = torch.full((w.M * w.N,), float("nan"), dtype=out_dt, device="cuda")
-    before = torch.cuda.memory_allocated()
+    torch.cuda.synchronize()
+    free_before = torch.cuda.mem_get_info()[0]
+    allocs_before = torch.cuda.memory_stats().get("allocation.all.allocated", 0)
     plan.run_static(dA, dB, got, bias=db, stream=sp)
     plan.check()
-    assert torch.cuda.memory_allocated() == before
+    # nothing was allocated on the device: neither through torch's allocator nor behind its back
+    assert torch.cuda.memory_stats().get("allocation.all.allocated", 0) == allocs_before
+    assert torch.cuda.mem_get_info()[0] >= free_before
     return c_to_f64(got), c_to_f64(ref)
 
 
