@@ -257,12 +257,17 @@ def run_ours(args):
         b.record(stream)
         b.synchronize()
         k_ms.append(a.elapsed_time(b))
+    # DRAM bytes per launch of the benchmark kernel at this size, from the ncu capture summarised in
+    # profiles/bench_c4_bf16_8192_dram_traffic.md; None for any other kernel or size.
+    traffic = None
+    if plan.kernel_name == "umma_bf16_pair_256x256x64_s6_splitk1" and (w.M, w.N, w.K) == (8192, 8192, 8192):
+        traffic = 1.12e9 + 250.9e6
     k_avg = ms_per_step          # average launch duration inside the timed region
     achieved = w.flops / (k_avg * 1e-3) / 1e12
     peak = float(peaks["bf16_tflops"])
     roofline = {
         "bound": "tensor", "achieved": achieved, "peak": peak, "unit": "TFLOP/s",
-        "frac": achieved / peak, "traffic": None,
+        "frac": achieved / peak, "traffic": traffic,
         "peak_source": f"MEASURED_PEAKS.json bf16_tflops (burst), of {peaks['_source']}",
         "frac_of_sustained_peak": achieved / float(peaks["bf16_tflops_sustained"]),
         "frac_of_nominal_2250": achieved / 2250.0,
