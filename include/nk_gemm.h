@@ -169,6 +169,15 @@ nk_status_t nk_gemm_check(nk_gemm_t plan);
 nk_status_t nk_gemm_run_static(nk_gemm_t plan, const void* A, const void* B, const void* bias,
                                void* C, void* cuda_stream);
 
+/*
+ * Self-test of the failure path, without a failure: enqueues a one-warp kernel that waits on
+ * a barrier nothing signals, with a limit of a few milliseconds.  The wait runs out, the
+ * kernel records it in the status word and exits normally, so the next nk_gemm_check
+ * returns NK_ERR_TIMEOUT (once) and the context stays usable.  This is how the bounded waits
+ * of the GEMM kernels (Algorithm 1's K loop, re-expressed as an mbarrier pipeline) report.
+ */
+nk_status_t nk_gemm_selftest_timeout(nk_gemm_t plan, void* cuda_stream);
+
 /* Free the plan's host state.  NULL is accepted. */
 nk_status_t nk_gemm_destroy(nk_gemm_t plan);
 

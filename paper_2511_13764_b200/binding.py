@@ -19,7 +19,8 @@ FLAG_SINGLE_CTA, FLAG_CTA_PAIR = 0x20, 0x40
 
 EXPORTS = ["nk_gemm_create", "nk_gemm_workspace_bytes", "nk_gemm_run", "nk_gemm_run_host",
            "nk_gemm_check", "nk_gemm_destroy", "nk_status_str", "nk_gemm_kernel_name",
-           "nk_gemm_launches_per_run", "nk_gemm_last_cuda_error", "nk_gemm_run_static"]
+           "nk_gemm_launches_per_run", "nk_gemm_last_cuda_error", "nk_gemm_run_static",
+           "nk_gemm_selftest_timeout"]
 
 STATIC_SCRATCH_BYTES = 16 << 20
 
@@ -73,6 +74,8 @@ def lib():
         L.nk_gemm_run_static.argtypes = [vp, vp, vp, vp, vp, vp]
         L.nk_gemm_run_host.restype = ctypes.c_int
         L.nk_gemm_run_host.argtypes = [vp, vp, vp, vp, vp, vp, vp, vp, vp, vp, sz, vp]
+        L.nk_gemm_selftest_timeout.restype = ctypes.c_int
+        L.nk_gemm_selftest_timeout.argtypes = [vp, vp]
         L.nk_gemm_check.restype = ctypes.c_int
         L.nk_gemm_check.argtypes = [vp]
         L.nk_gemm_destroy.restype = ctypes.c_int
@@ -153,6 +156,9 @@ class Plan:
         _check(lib().nk_gemm_run_host(self._h, _ptr(hA), _ptr(hB), _ptr(hbias), _ptr(hC), _ptr(dA),
                                       _ptr(dB), _ptr(dbias), _ptr(dC), _ptr(workspace),
                                       workspace_bytes, stream), self._h)
+
+    def selftest_timeout(self, stream=None):
+        _check(lib().nk_gemm_selftest_timeout(self._h, stream), self._h)
 
     def check(self):
         _check(lib().nk_gemm_check(self._h), self._h)

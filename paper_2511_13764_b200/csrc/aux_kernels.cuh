@@ -6,6 +6,8 @@
 #include <cuda_runtime.h>
 #include <stdint.h>
 
+#include "ptx.cuh"
+
 namespace nk {
 
 struct NaiveParams {
@@ -105,6 +107,23 @@ __global__ void unpack_vnni_b_kernel(const uint32_t* __restrict__ Bblk, uint16_t
         Brow[row0] = static_cast<uint16_t>(w & 0xFFFFu);       // even k: low half
         Brow[row0 + N] = static_cast<uint16_t>(w >> 16);       // odd k: high half
     }
+}
+
+// Self-test of the bounded-wait path: one warp waits on an mbarrier that nothing ever
+// arrives on, with a short limit; the wait gives up, the kernel records the code in the
+// status word and returns normally (no trap, no fault, the context stays usable).
+__global__ void wait_timeout_probe_kernel(unsigned int* status, long long limit_clocks) {
+    __shared__ __align__(8) unsigned long long bar;
+    __shared__ uint32_t abort_flag;
+    const uint32_t b = smem_u32(&bar);
+    if (threadIdx.x == 0) {
+        mbar_init(b, 1);
+        abort_flag = 0;
+        fence_mbar_init();
+    }
+    __syncwarp();
+    const bool done = mbar_wait(b, 0u, &abort_flag, limit_clocks);
+    if (!done && threadIdx.x == 0 && status) atomicCAS(status, 0u, 0x900u);
 }
 
 }  // namespace nk

@@ -727,6 +727,16 @@ nk_status_t nk_gemm_check(nk_gemm_t p) {
     return NK_OK;
 }
 
+nk_status_t nk_gemm_selftest_timeout(nk_gemm_t p, void* cuda_stream) {
+    if (!p) return NK_ERR_INVALID_ARG;
+    DeviceGuard guard(p->d.device);
+    if (guard.err != cudaSuccess) return NK_ERR_DEVICE;
+    wait_timeout_probe_kernel<<<1, 32, 0, static_cast<cudaStream_t>(cuda_stream)>>>(p->status_dev, 1ll << 22);
+    cudaError_t e = cudaGetLastError();
+    if (e != cudaSuccess) { set_err(p, "probe launch", e); return NK_ERR_CUDA; }
+    return NK_OK;
+}
+
 nk_status_t nk_gemm_destroy(nk_gemm_t p) {
     delete p;
     return NK_OK;

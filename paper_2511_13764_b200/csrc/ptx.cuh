@@ -42,7 +42,8 @@ __device__ __forceinline__ uint32_t mbar_try_wait(uint32_t bar, uint32_t parity)
 // Bounded wait: gives up after ~2^31 clock ticks (about a second), or as soon as
 // another role of the CTA has raised `*abort_flag`.  Returns false on give-up.
 __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity,
-                                          volatile uint32_t* abort_flag) {
+                                          volatile uint32_t* abort_flag,
+                                          long long limit_clocks = (1ll << 31)) {
     if (mbar_try_wait(bar, parity)) return true;
     const long long t0 = clock64();
     uint32_t polls = 0;
@@ -50,7 +51,7 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity,
         if (mbar_try_wait(bar, parity)) return true;
         if ((++polls & 255u) == 0u) {
             if (*abort_flag) return false;
-            if (clock64() - t0 > (1ll << 31)) return false;
+            if (clock64() - t0 > limit_clocks) return false;
         }
     }
 }

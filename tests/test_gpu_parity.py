@@ -213,3 +213,18 @@ def test_runtime_argument_errors():
     with pytest.raises(nk.NkError) as e:
         plan2.run(x, x, c)
     assert e.value.status == 4
+
+
+def test_bounded_wait_reports_timeout_and_context_survives():
+    """A wait that can never complete gives up after its limit, the kernel exits normally and
+    nk_gemm_check reports NK_ERR_TIMEOUT once; the same plan then runs a correct GEMM."""
+    w = W("after_timeout", 128, 128, 128, "bf16", integer=True)
+    plan = nk.plan_for(w)
+    plan.selftest_timeout(stream=torch.cuda.current_stream().cuda_stream)
+    with pytest.raises(nk.NkError) as e:
+        plan.check()
+    assert e.value.status == 7
+    plan.check()                                   # the word was cleared
+    A, B, bias = w.make()
+    got, _ = run_plan(w, A, B, bias, plan=plan)
+    check_against_oracle(w, got, A, B, bias, exact=True)
