@@ -381,6 +381,10 @@ static cudaError_t pair_occupancy(int* out) {
     return cudaOccupancyMaxActiveClusters(out, umma_bf16_pair_kernel<BN, STAGES, VNNI>, &cfg);
 }
 
+static cudaError_t prepare_simt_attrs() {
+    return allow_smem(simt_f32_async_kernel<128, 128, 8, 8>, simt_async_smem_bytes<128, 128>());
+}
+
 static cudaError_t prepare_umma_attrs() {
     cudaError_t e2;
     if ((e2 = allow_smem(umma_bf16_pair_kernel<256, 6, false>, pair_smem_bytes(256, 6))) != cudaSuccess) return e2;
@@ -400,9 +404,11 @@ static cudaError_t prepare_umma_attrs() {
 static cudaError_t launch_simt(nk_gemm_s* p, const SimtParams& sp, cudaStream_t st) {
     const int t = p->simt_tile;
     dim3 grid(ceil_div(sp.N, t), ceil_div(sp.M, t), sp.splits);
+    // 128-tile: register-staged double buffer (a little faster when the FMA pipe is the limit);
+    // smaller tiles: three-stage cp.async pipeline (their K loops are latency bound).
     if (t == 128) simt_f32_kernel<128, 128, 8, 8><<<grid, 256, 0, st>>>(sp);
-    else if (t == 64) simt_f32_kernel<64, 64, 4, 4><<<grid, 256, 0, st>>>(sp);
-    else simt_f32_kernel<32, 32, 4, 4><<<grid, 64, 0, st>>>(sp);
+    else if (t == 64) simt_f32_async_kernel<64, 64, 4, 4><<<grid, 256, simt_async_smem_bytes<64, 64>(), st>>>(sp);
+    else simt_f32_async_kernel<32, 32, 4, 4><<<grid, 64, simt_async_smem_bytes<32, 32>(), st>>>(sp);
     return cudaGetLastError();
 }
 
@@ -487,6 +493,7 @@ nk_status_t nk_gemm_create(const nk_gemm_desc_t* desc, nk_gemm_t* out) {
                  p->skinny_kc, p->splits);
     } else if (d.in_dtype == NK_F32) {
         p->variant = V_SIMT;
+        if (prepare_simt_attrs() != cudaSuccess) { cudaGetLastError(); delete p; return NK_ERR_CUDA; }
         choose_simt(p);
         p->ws_partial_bytes = p->splits > 1 ? static_cast<size_t>(p->splits) * d.M * d.N * 4 : 0;
         p->launches = p->splits > 1 ? 2 : 1;

@@ -120,10 +120,14 @@ simt_f32_kernel(const SimtParams p) {
                 const float4 v = *reinterpret_cast<const float4*>(&Bs[buf][k][g * SN_STRIDE + tx * 4]);
                 b[4 * g] = v.x; b[4 * g + 1] = v.y; b[4 * g + 2] = v.z; b[4 * g + 3] = v.w;
             }
+            // serpentine order over the thread tile: consecutive FMAs share an operand register
 #pragma unroll
             for (int i = 0; i < TM; ++i)
 #pragma unroll
-                for (int j = 0; j < TN; ++j) acc[i][j] = fmaf(a[i], b[j], acc[i][j]);
+                for (int jj = 0; jj < TN; ++jj) {
+                    const int j = (i & 1) ? TN - 1 - jj : jj;
+                    acc[i][j] = fmaf(a[i], b[j], acc[i][j]);
+                }
         }
         if (more) {
             store_shared(buf ^ 1);
@@ -262,6 +266,138 @@ __global__ void __launch_bounds__(SKINNY_THREADS, MR == 16 ? 4 : 2) simt_f32_ski
         }
         *reinterpret_cast<float4*>(out + static_cast<size_t>(m) * p.N + n) = v;
     }
+}
+
+}  // namespace nk
+
+#include "ptx.cuh"
+
+namespace nk {
+
+// The same FP32 GEMM with the operand staging done by cp.async instead of registers: tiles of
+// k-block t+2 and t+1 are in flight while k-block t is multiplied (three shared-memory stages),
+// nothing is held in registers for staging, and the transpose of A into As[k][m] happens in
+// the copy itself (4-byte copies, one element each; B rows go as 16-byte copies).
+constexpr int SIMT_STAGES = 3;
+
+template <int BM, int BN>
+__host__ __device__ constexpr int simt_async_smem_bytes() {
+    return SIMT_STAGES * SIMT_BK * ((BM + 4) + BN) * 4;
+}
+
+template <int BM, int BN, int TM, int TN>
+__global__ void __launch_bounds__((BM / TM) * (BN / TN), (BM >= 128 ? 2 : 1))
+simt_f32_async_kernel(const SimtParams p) {
+    constexpr int THREADS = (BM / TM) * (BN / TN);
+    constexpr int TX = BN / TN;
+    constexpr int GM = TM / 4, GN = TN / 4;
+    constexpr int SM_STRIDE = BM / GM;
+    constexpr int SN_STRIDE = BN / GN;
+    constexpr int AP = BM + 4;
+    constexpr int A_ELEMS = BM * SIMT_BK / THREADS;        // 4-byte copies per thread per tile
+    constexpr int B_V4 = BN * SIMT_BK / 4 / THREADS;       // 16-byte copies per thread per tile
+    constexpr int A_STAGE = SIMT_BK * AP, B_STAGE = SIMT_BK * BN;   // floats
+    static_assert(A_ELEMS >= 1 && B_V4 >= 1, "tile too small for the thread count");
+
+    extern __shared__ __align__(16) float simt_smem[];
+    float* As = simt_smem;                                  // [stage][k][AP]
+    float* Bs = simt_smem + SIMT_STAGES * A_STAGE;          // [stage][k][BN]
+    const uint32_t as_u32 = smem_u32(As), bs_u32 = smem_u32(Bs);
+
+    const int t = threadIdx.x;
+    const int ty = t / TX, tx = t % TX;
+    const int m0 = blockIdx.y * BM, n0 = blockIdx.x * BN;
+    const int ktiles = (p.K + SIMT_BK - 1) / SIMT_BK;
+    const int kt0 = blockIdx.z * p.kt_per_split;
+    const int kt1 = min(ktiles, kt0 + p.kt_per_split);
+
+    float acc[TM][TN];
+#pragma unroll
+    for (int i = 0; i < TM; ++i)
+#pragma unroll
+        for (int j = 0; j < TN; ++j) acc[i][j] = 0.0f;
+
+    auto issue_tile = [&](int kt, int stage) {
+        if (kt < kt1) {
+            const int k0 = kt * SIMT_BK;
+#pragma unroll
+            for (int i = 0; i < A_ELEMS; ++i) {
+                const int e = t + i * THREADS;             // 16 consecutive lanes = one row's 16 k
+                const int k = e & (SIMT_BK - 1), row = e / SIMT_BK;
+                const bool ok = m0 + row < p.M && k0 + k < p.K;
+                const float* src = p.A + (ok ? static_cast<size_t>(m0 + row) * p.K + k0 + k : 0);
+                cp_async_4(as_u32 + (stage * A_STAGE + k * AP + row) * 4, src, ok ? 4u : 0u);
+            }
+#pragma unroll
+            for (int i = 0; i < B_V4; ++i) {
+                const int idx = t + i * THREADS;
+                const int kr = idx / (BN / 4), nq = (idx % (BN / 4)) * 4;
+                const bool ok = k0 + kr < p.K && n0 + nq < p.N;
+                const float* src = p.B + (ok ? static_cast<size_t>(k0 + kr) * p.N + n0 + nq : 0);
+                cp_async_16(bs_u32 + (stage * B_STAGE + kr * BN + nq) * 4, src, ok ? 16u : 0u);
+            }
+        }
+        cp_async_commit();                                  // an empty group keeps the counts aligned
+    };
+
+#pragma unroll
+    for (int s = 0; s < SIMT_STAGES - 1; ++s) issue_tile(kt0 + s, s);
+
+    int stage = 0;
+    for (int kt = kt0; kt < kt1; ++kt) {
+        cp_async_wait_group<SIMT_STAGES - 2>();             // tile kt has landed (this thread's copies)
+        __syncthreads();                                    // ... everyone's; and tile kt-1 is consumed
+        int nstage = stage + SIMT_STAGES - 1;
+        if (nstage >= SIMT_STAGES) nstage -= SIMT_STAGES;
+        issue_tile(kt + SIMT_STAGES - 1, nstage);
+        const float* as = As + stage * A_STAGE;
+        const float* bs = Bs + stage * B_STAGE;
+#pragma unroll
+        for (int k = 0; k < SIMT_BK; ++k) {
+            float a[TM], b[TN];
+#pragma unroll
+            for (int g = 0; g < GM; ++g) {
+                const float4 v = *reinterpret_cast<const float4*>(as + k * AP + g * SM_STRIDE + ty * 4);
+                a[4 * g] = v.x; a[4 * g + 1] = v.y; a[4 * g + 2] = v.z; a[4 * g + 3] = v.w;
+            }
+#pragma unroll
+            for (int g = 0; g < GN; ++g) {
+                const float4 v = *reinterpret_cast<const float4*>(bs + k * BN + g * SN_STRIDE + tx * 4);
+                b[4 * g] = v.x; b[4 * g + 1] = v.y; b[4 * g + 2] = v.z; b[4 * g + 3] = v.w;
+            }
+#pragma unroll
+            for (int i = 0; i < TM; ++i)
+#pragma unroll
+                for (int j = 0; j < TN; ++j) acc[i][j] = fmaf(a[i], b[j], acc[i][j]);
+        }
+        if (++stage == SIMT_STAGES) stage = 0;
+    }
+    cp_async_wait_group<0>();
+
+    const bool to_partial = p.splits > 1;
+    float* out = to_partial ? p.partial + static_cast<size_t>(blockIdx.z) * p.M * p.N : p.C;
+#pragma unroll
+    for (int gi = 0; gi < GM; ++gi)
+#pragma unroll
+        for (int ii = 0; ii < 4; ++ii) {
+            const int gm = m0 + gi * SM_STRIDE + ty * 4 + ii;
+            if (gm >= p.M) continue;
+#pragma unroll
+            for (int gj = 0; gj < GN; ++gj) {
+                const int gn = n0 + gj * SN_STRIDE + tx * 4;
+                if (gn >= p.N) continue;
+                float4 v = make_float4(acc[4 * gi + ii][4 * gj], acc[4 * gi + ii][4 * gj + 1],
+                                       acc[4 * gi + ii][4 * gj + 2], acc[4 * gi + ii][4 * gj + 3]);
+                if (!to_partial && p.epilogue) {
+                    const float4 bv = __ldg(reinterpret_cast<const float4*>(p.bias + gn));
+                    v.x = fmaxf(v.x + bv.x, 0.f);
+                    v.y = fmaxf(v.y + bv.y, 0.f);
+                    v.z = fmaxf(v.z + bv.z, 0.f);
+                    v.w = fmaxf(v.w + bv.w, 0.f);
+                }
+                *reinterpret_cast<float4*>(out + static_cast<size_t>(gm) * p.N + gn) = v;
+            }
+        }
 }
 
 }  // namespace nk
