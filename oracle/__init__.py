@@ -61,6 +61,10 @@ def lib():
         L.nko_gemm.argtypes = [ctypes.POINTER(Desc), ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p,
                                ctypes.c_void_p, ctypes.c_int64, ctypes.c_void_p, ctypes.c_int64,
                                ctypes.c_void_p, ctypes.c_void_p, ctypes.c_int]
+        L.nko_brgemm.restype = ctypes.c_int
+        L.nko_brgemm.argtypes = [ctypes.c_int64] * 6 + [ctypes.c_int32, ctypes.c_int32, ctypes.c_double,
+                                 ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p,
+                                 ctypes.c_void_p, ctypes.c_void_p]
         _lib = L
     return _lib
 
@@ -169,3 +173,33 @@ def gemm_workload(w, A, B, bias, rows=None, cols=None, **kw):
                 layout_a=lay, layout_b=lay,
                 epilogue=EPI_BIAS_RELU if w.epilogue == "bias_relu" else EPI_NONE,
                 rows=rows, cols=cols, **kw)
+
+
+def brgemm(M, N, K, batch, A, B, bias=None, C0=None, *, in_dtype=F32, epilogue=EPI_NONE, beta=0.0,
+           stride_a=None, stride_b=None):
+    """Batch-reduce GEMM (Algorithm 1's output line): beta*C0 + sum_b A_b.B_b, row-major.
+    A and B are storage buffers holding all batch items (item b of A starts at b*stride_a
+    elements; default M*K and K*N).  C0: float64 [M][N] (the stored C widened) when beta = 1.
+    Returns (Y, S) float64 [M][N]."""
+    dt = _np_dtype(in_dtype)
+    A = np.ascontiguousarray(A, dtype=dt)
+    B = np.ascontiguousarray(B, dtype=dt)
+    stride_a = M * K if stride_a is None else stride_a
+    stride_b = K * N if stride_b is None else stride_b
+    assert A.size >= (batch - 1) * stride_a + M * K and B.size >= (batch - 1) * stride_b + K * N
+    bp = None
+    if bias is not None:
+        bias = np.ascontiguousarray(bias, dtype=dt)
+        bp = bias.ctypes.data
+    cp = None
+    if C0 is not None:
+        C0 = np.ascontiguousarray(C0, dtype=np.float64)
+        assert C0.size == M * N
+        cp = C0.ctypes.data
+    Y = np.empty((M, N), dtype=np.float64)
+    S = np.empty((M, N), dtype=np.float64)
+    rc = lib().nko_brgemm(M, N, K, batch, stride_a, stride_b, in_dtype, epilogue, float(beta),
+                          A.ctypes.data, B.ctypes.data, bp, cp, Y.ctypes.data, S.ctypes.data)
+    if rc != 0:
+        raise ValueError("oracle rejected the arguments")
+    return Y, S

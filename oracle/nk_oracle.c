@@ -173,3 +173,47 @@ int nko_gemm(const nko_desc_t* d, const void* A, const void* B, const void* bias
     free(jobs);
     return 0;
 }
+
+/*
+ * Batch-reduce GEMM, the output line of Algorithm 1 written out:
+ *
+ *     C[i][j] = beta * C0[i][j] + sum_{b=0}^{batch-1} sum_{k=0}^{K-1} a_b(i,k) * b_b(k,j)
+ *
+ * with the batch-reduce loop outside the K loop, as in the algorithm.  Row-major
+ * operands; A_b starts stride_a elements after A_{b-1}, B_b stride_b after B_{b-1} (the
+ * tiles need not be contiguous, Section 2.1).  beta is 0 or 1 (C0 may be NULL when 0);
+ * C0 holds the stored values of C widened to double.  FP64 accumulation, then the same
+ * epilogue as nko_gemm.  S receives sum |a.b| + |beta.C0| (+ |bias|).  Plain loops, one
+ * thread: this is the definition, used on test sizes only.
+ */
+int nko_brgemm(int64_t M, int64_t N, int64_t K, int64_t batch, int64_t stride_a, int64_t stride_b,
+               int32_t in_dtype, int32_t epilogue, double beta, const void* A, const void* B,
+               const void* bias, const double* C0, double* Y, double* S) {
+    if (!A || !B || !Y || M <= 0 || N <= 0 || K <= 0 || batch <= 0) return -1;
+    if (beta != 0.0 && beta != 1.0) return -1;
+    if (beta != 0.0 && !C0) return -1;
+    if (epilogue == NKO_EPI_BIAS_RELU && !bias) return -1;
+    for (int64_t i = 0; i < M; ++i) {
+        for (int64_t j = 0; j < N; ++j) {
+            double acc = beta != 0.0 ? beta * C0[i * N + j] : 0.0;
+            double s = fabs(acc);
+            for (int64_t b = 0; b < batch; ++b) {
+                for (int64_t k = 0; k < K; ++k) {
+                    double p = load(A, in_dtype, b * stride_a + i * K + k) *
+                               load(B, in_dtype, b * stride_b + k * N + j);
+                    acc += p;
+                    s += fabs(p);
+                }
+            }
+            if (epilogue == NKO_EPI_BIAS_RELU) {
+                double bv = load(bias, in_dtype, j);
+                acc += bv;
+                s += fabs(bv);
+                if (!(acc > 0.0)) acc = 0.0;
+            }
+            Y[i * N + j] = acc;
+            if (S) S[i * N + j] = s;
+        }
+    }
+    return 0;
+}

@@ -332,3 +332,69 @@ def test_generator_golden_and_ranges():
     assert np.array_equal(nk_inputs.fill(1, 0, 100), u[:100])
     rows = nk_inputs.stratified_rows(4017, 8192, 64)
     assert len(rows) == 64 and np.array_equal(rows // 128, np.arange(64))
+
+
+# ---------------------------------------------------------------- batch-reduce GEMM, beta
+@pytest.mark.parametrize("case", list(_shapes()), ids=lambda c: c[0])
+def test_brgemm_paper_shapes_against_k_concatenation(case):
+    """sum_b A_b.B_b over the paper's example shapes, through the batch interface, equals the
+    plain GEMM on K-concatenated operands bit for bit (same products, same order) and a
+    brute-force sum written in another loop order."""
+    name, batch, M, N, K, dt, lay = case
+    As = [_rand_int((M, K), 300 + i) for i in range(batch)]
+    Bs = [_rand_int((K, N), 400 + i) for i in range(batch)]
+    A = np.stack(As).reshape(-1)
+    B = np.stack(Bs).reshape(-1)
+    if dt == "bf16":
+        Y, S = oracle.brgemm(M, N, K, batch, _bits(A), _bits(B), in_dtype=BF16)
+        Yc, Sc = oracle.gemm(M, N, batch * K, _bits(np.concatenate(As, axis=1)), _bits(np.concatenate(Bs, axis=0)),
+                             in_dtype=BF16)
+    else:
+        Y, S = oracle.brgemm(M, N, K, batch, A, B)
+        Yc, Sc = oracle.gemm(M, N, batch * K, np.concatenate(As, axis=1), np.concatenate(Bs, axis=0))
+    assert np.array_equal(Y, Yc) and np.array_equal(S, Sc)
+    want = np.zeros((M, N))
+    for n in range(N):
+        for b in reversed(range(batch)):
+            want[:, n] += As[b].astype(np.float64) @ Bs[b][:, n].astype(np.float64)
+    assert np.array_equal(Y, want)          # integers: exact in any order
+
+
+def test_brgemm_beta_and_strides():
+    M, N, K, batch = 5, 7, 6, 3
+    sa, sb = M * K + 11, K * N + 5                      # non-contiguous batch items
+    rng = np.random.default_rng(50)
+    A = rng.integers(-4, 5, size=(batch - 1) * sa + M * K).astype(np.float32)
+    B = rng.integers(-4, 5, size=(batch - 1) * sb + K * N).astype(np.float32)
+    ref = np.zeros((M, N))
+    for b in range(batch):
+        ref += A[b * sa:b * sa + M * K].reshape(M, K).astype(np.float64) @ \
+               B[b * sb:b * sb + K * N].reshape(K, N).astype(np.float64)
+    Y, _ = oracle.brgemm(M, N, K, batch, A, B, stride_a=sa, stride_b=sb)
+    assert np.array_equal(Y, ref)
+    C0 = rng.integers(-9, 10, size=(M, N)).astype(np.float64)
+    Y1, S1 = oracle.brgemm(M, N, K, batch, A, B, C0=C0, beta=1.0, stride_a=sa, stride_b=sb)
+    assert np.array_equal(Y1, ref + C0)                 # beta = 1 adds the old C
+    Y0, S0 = oracle.brgemm(M, N, K, batch, A, B, C0=C0, beta=0.0, stride_a=sa, stride_b=sb)
+    assert np.array_equal(Y0, ref)                      # beta = 0 ignores it
+    assert np.array_equal(S1, S0 + np.abs(C0))
+    Yz, _ = oracle.brgemm(M, N, K, batch, A, B, C0=-ref, beta=1.0, stride_a=sa, stride_b=sb)
+    assert np.all(Yz == 0.0)                            # C0 = -(sum) cancels exactly
+    Ya, _ = oracle.brgemm(M, N, K, batch, np.zeros_like(A), B, C0=C0, beta=1.0, stride_a=sa, stride_b=sb)
+    assert np.array_equal(Ya, C0)                       # zero A leaves C0
+    bias = np.full(N, -1000.0, dtype=np.float32)
+    Yr, _ = oracle.brgemm(M, N, K, batch, A, B, bias, C0=C0, beta=1.0, epilogue=EPI_BIAS_RELU, stride_a=sa, stride_b=sb)
+    assert np.all(Yr == 0.0)
+    with pytest.raises(ValueError):
+        oracle.brgemm(M, N, K, batch, A, B, beta=1.0, stride_a=sa, stride_b=sb)      # beta = 1 needs C0
+    with pytest.raises(ValueError):
+        oracle.brgemm(M, N, K, batch, A, B, C0=C0, beta=0.5, stride_a=sa, stride_b=sb)
+
+
+def test_brgemm_batch_one_is_gemm():
+    M, N, K = 9, 12, 20
+    A = nk_inputs.fill(60, 0, M * K)
+    B = nk_inputs.fill(60, 1, K * N)
+    Y, S = oracle.brgemm(M, N, K, 1, A, B)
+    Yg, Sg = oracle.gemm(M, N, K, A, B)
+    assert np.array_equal(Y, Yg) and np.array_equal(S, Sg)
