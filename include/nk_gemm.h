@@ -77,6 +77,11 @@ typedef struct {
     int32_t epilogue;  /* nk_epilogue_t                                       */
     int32_t device;    /* CUDA device ordinal                                 */
     uint32_t flags;    /* NK_FLAG_*                                           */
+    /* Batch-reduce form of Algorithm 1, C = beta*C + sum_b A_b . B_b (all zero = plain GEMM): */
+    int32_t beta;      /* 0: C's old contents are never read; 1: they are added (FP32)  */
+    int64_t batch;     /* number of (A_b, B_b) pairs reduced into C; 0 means 1          */
+    int64_t stride_a;  /* elements from A_b to A_b+1; 0 means M*K (contiguous)          */
+    int64_t stride_b;  /* elements from B_b to B_b+1; 0 means K*N                       */
 } nk_gemm_desc_t;
 
 /*
@@ -86,7 +91,10 @@ typedef struct {
  * state.  Requirements: M, N, K > 0; blocked layouts need BF16 and the blocked
  * operand's two dimensions to be multiples of 32; row-major BF16 needs N and K
  * to be multiples of 8, row-major FP32 needs N and K to be multiples of 4
- * (16-byte rows); BF16 output needs BF16 inputs.  On failure *out is NULL.
+ * (16-byte rows); BF16 output needs BF16 inputs.  batch > 1 and beta = 1 (Section 2.1:
+ * the source tiles of a batch-reduce GEMM need not be contiguous, the accumulation tile is
+ * C) need row-major operands and strides that are multiples of 8 (BF16) or 4 (FP32)
+ * elements; with beta = 1, y = epilogue(C_old + sum_b A_b.B_b).  On failure *out is NULL.
  */
 nk_status_t nk_gemm_create(const nk_gemm_desc_t* desc, nk_gemm_t* out);
 

@@ -45,7 +45,8 @@ class Desc(ctypes.Structure):
                 ("in_dtype", ctypes.c_int32), ("out_dtype", ctypes.c_int32),
                 ("layout_a", ctypes.c_int32), ("layout_b", ctypes.c_int32),
                 ("epilogue", ctypes.c_int32), ("device", ctypes.c_int32),
-                ("flags", ctypes.c_uint32)]
+                ("flags", ctypes.c_uint32), ("beta", ctypes.c_int32), ("batch", ctypes.c_int64),
+                ("stride_a", ctypes.c_int64), ("stride_b", ctypes.c_int64)]
 
 
 _lib = None
@@ -121,8 +122,10 @@ class Plan:
     their pointers; the caller owns every buffer."""
 
     def __init__(self, M, N, K, in_dtype=BF16, out_dtype=F32, layout_a=ROW_MAJOR,
-                 layout_b=ROW_MAJOR, epilogue=EPI_NONE, device=0, flags=0):
-        self.desc = Desc(M, N, K, in_dtype, out_dtype, layout_a, layout_b, epilogue, device, flags)
+                 layout_b=ROW_MAJOR, epilogue=EPI_NONE, device=0, flags=0, beta=0, batch=0,
+                 stride_a=0, stride_b=0):
+        self.desc = Desc(M, N, K, in_dtype, out_dtype, layout_a, layout_b, epilogue, device, flags,
+                         beta, batch, stride_a, stride_b)
         self._h = ctypes.c_void_p()
         _check(lib().nk_gemm_create(ctypes.byref(self.desc), ctypes.byref(self._h)))
 

@@ -13,6 +13,8 @@ namespace nk {
 struct NaiveParams {
     int M, N, K;
     int in_bf16, out_bf16, a_blocked, b_blocked, epilogue;
+    int batch, beta;
+    long long stride_a, stride_b;
     const void *A, *B, *bias;
     void* C;
 };
@@ -29,7 +31,10 @@ __global__ void naive_gemm_kernel(const NaiveParams p) {
     const int i = blockIdx.y;
     if (j >= p.N || i >= p.M) return;
     const size_t kb32 = p.K / 32;
+    const size_t o = static_cast<size_t>(i) * p.N + j;
     float acc = 0.f;
+    if (p.beta) acc = ld_elem(p.C, p.out_bf16, o);
+    for (int b = 0; b < p.batch; ++b)
     for (int k = 0; k < p.K; ++k) {
         const size_t ia = p.a_blocked
             ? (((static_cast<size_t>(i / 32) * kb32 + k / 32) * 32 + i % 32) * 32 + k % 32)
@@ -37,10 +42,9 @@ __global__ void naive_gemm_kernel(const NaiveParams p) {
         const size_t ib = p.b_blocked
             ? (((((static_cast<size_t>(j / 32) * kb32 + k / 32) * 16 + (k % 32) / 2) * 32 + j % 32) * 2) + k % 2)
             : static_cast<size_t>(k) * p.N + j;
-        acc = fmaf(ld_elem(p.A, p.in_bf16, ia), ld_elem(p.B, p.in_bf16, ib), acc);
+        acc = fmaf(ld_elem(p.A, p.in_bf16, b * p.stride_a + ia), ld_elem(p.B, p.in_bf16, b * p.stride_b + ib), acc);
     }
     if (p.epilogue) acc = fmaxf(acc + ld_elem(p.bias, p.in_bf16, j), 0.f);
-    const size_t o = static_cast<size_t>(i) * p.N + j;
     if (p.out_bf16)
         static_cast<__nv_bfloat16*>(p.C)[o] = __float2bfloat16_rn(acc);
     else
@@ -52,6 +56,7 @@ struct ReduceParams {
     int N;
     int splits;
     int epilogue, bias_bf16, out_bf16;
+    int beta;              // 1: add the old C before the epilogue
     const float* partial;  // [splits][M][N]
     const void* bias;
     void* C;
@@ -67,6 +72,16 @@ __global__ void splitk_reduce_kernel(const ReduceParams p) {
     for (int sp = 1; sp < p.splits; ++sp) {
         const float4 v = __ldcs(reinterpret_cast<const float4*>(p.partial + sp * p.MN + e));
         s.x += v.x; s.y += v.y; s.z += v.z; s.w += v.w;
+    }
+    if (p.beta) {
+        if (p.out_bf16) {
+            const uint2 w = *reinterpret_cast<const uint2*>(static_cast<const uint16_t*>(p.C) + e);
+            s.x += __uint_as_float(w.x << 16); s.y += __uint_as_float(w.x & 0xFFFF0000u);
+            s.z += __uint_as_float(w.y << 16); s.w += __uint_as_float(w.y & 0xFFFF0000u);
+        } else {
+            const float4 c = *reinterpret_cast<const float4*>(static_cast<const float*>(p.C) + e);
+            s.x += c.x; s.y += c.y; s.z += c.z; s.w += c.w;
+        }
     }
     if (p.epilogue) {
         const int n = static_cast<int>(e % p.N);

@@ -47,6 +47,9 @@ struct nk_gemm_s {
     int simt_tile;  // 128, 64 or 32
     int kt_per_split;
     int skinny_kc;  // FP32 skinny kernel: k per CTA
+    // batch-reduce (normalised: batch >= 1, strides in elements)
+    int batch;
+    long long stride_a, stride_b;
     // workspace layout
     size_t ws_repack_bytes, ws_partial_bytes;
     // device status word
@@ -114,8 +117,10 @@ static int umma_stages_for(int bn) { return bn == 256 ? 4 : bn == 128 ? 6 : 8; }
 // (the stage pipeline is latency bound), so wide tiles win whenever they do not cost rounds.
 struct UmmaChoice { bool pair; int bn; int splits; double us; };
 
+static int desc_batch(const nk_gemm_desc_t& d) { return d.batch > 1 ? static_cast<int>(d.batch) : 1; }
+
 static double umma_model_us(const nk_gemm_desc_t& d, int sms, bool pair, int bn, int splits) {
-    const int kb_total = ceil_div(d.K, UMMA_BK);
+    const int kb_total = desc_batch(d) * ceil_div(d.K, UMMA_BK);
     const int per = ceil_div(kb_total, splits);
     const int eff_splits = ceil_div(kb_total, per);
     const int64_t tiles = static_cast<int64_t>(ceil_div(d.M, pair ? 256 : 128)) * ceil_div(d.N, bn);
@@ -129,7 +134,7 @@ static double umma_model_us(const nk_gemm_desc_t& d, int sms, bool pair, int bn,
     const double mn = static_cast<double>(d.M) * d.N;
     double us = (pair ? 12.0 : 10.0) + rounds * per * t_kb;
     if (eff_splits > 1) us += 3.0 + eff_splits * mn * 4.0 / 3.0e6 + (eff_splits * 4.0 + eo) * mn / 5.0e6;
-    const double bytes = 2.0 * (static_cast<double>(d.M) * d.K + static_cast<double>(d.K) * d.N) + eo * mn;
+    const double bytes = 2.0 * desc_batch(d) * (static_cast<double>(d.M) * d.K + static_cast<double>(d.K) * d.N) + eo * mn;
     const double hbm_us = bytes / 5.2e6;  // ~80 % of the copy bandwidth, bytes per microsecond
     return us > hbm_us ? us : hbm_us;
 }
@@ -137,7 +142,7 @@ static double umma_model_us(const nk_gemm_desc_t& d, int sms, bool pair, int bn,
 static void choose_umma(nk_gemm_s* p) {
     const nk_gemm_desc_t& d = p->d;
     const int sms = p->sm_count;
-    const int kb_total = ceil_div(d.K, UMMA_BK);
+    const int kb_total = desc_batch(d) * ceil_div(d.K, UMMA_BK);
     const int forced_bn = (d.flags >> NK_FLAG_TILE_N_SHIFT) & 0xF;
     const int forced_s = (d.flags >> NK_FLAG_SPLITK_SHIFT) & 0xFF;
     const int split_cands[8] = {1, 2, 3, 4, 6, 8, 12, 16};
@@ -182,7 +187,7 @@ static void choose_umma(nk_gemm_s* p) {
 // the CTAs sharing the SM and by the variant's efficiency (wide thread tiles need fewer
 // shared-memory loads per FMA); units are scheduled in waves of sms * res.
 static double simt_model_us(const nk_gemm_desc_t& d, int sms, int tile, int splits) {
-    const int ktiles = ceil_div(d.K, SIMT_BK);
+    const int ktiles = desc_batch(d) * ceil_div(d.K, SIMT_BK);
     const int per = ceil_div(ktiles, splits);
     const int eff_splits = ceil_div(ktiles, per);
     const int64_t tiles = static_cast<int64_t>(ceil_div(d.M, tile)) * ceil_div(d.N, tile);
@@ -201,7 +206,7 @@ static double simt_model_us(const nk_gemm_desc_t& d, int sms, int tile, int spli
     if (rest > 0) us += per * kt_us(static_cast<double>((rest + sms - 1) / sms));
     const double mn = static_cast<double>(d.M) * d.N;
     if (eff_splits > 1) us += 3.0 + (2.0 * eff_splits + 1.0) * mn * 4.0 / 4.0e6;
-    const double bytes = 4.0 * (static_cast<double>(d.M) * d.K + static_cast<double>(d.K) * d.N + mn);
+    const double bytes = 4.0 * (desc_batch(d) * (static_cast<double>(d.M) * d.K + static_cast<double>(d.K) * d.N) + mn);
     // small tiles keep few bytes in flight: they reach a fraction of the HBM bandwidth only
     const double hbm_us = bytes / (tile == 128 ? 5.0e6 : tile == 64 ? 3.5e6 : 1.8e6);
     return us > hbm_us ? us : hbm_us;
@@ -210,7 +215,7 @@ static double simt_model_us(const nk_gemm_desc_t& d, int sms, int tile, int spli
 static void choose_simt(nk_gemm_s* p) {
     const nk_gemm_desc_t& d = p->d;
     const int sms = p->sm_count;
-    const int ktiles = ceil_div(d.K, SIMT_BK);
+    const int ktiles = desc_batch(d) * ceil_div(d.K, SIMT_BK);
     const int forced = (d.flags >> NK_FLAG_TILE_N_SHIFT) & 0xF;
     const int forced_s = (d.flags >> NK_FLAG_SPLITK_SHIFT) & 0xFF;
     const int split_cands[10] = {1, 2, 3, 4, 6, 8, 12, 16, 24, 32};
@@ -273,11 +278,13 @@ static nk_status_t encode_maps(nk_gemm_s* p, const void* A, const void* B) {
                       box, es, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_64B,
                       CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
     } else {
-        cuuint64_t dims[2] = {static_cast<cuuint64_t>(d.K), static_cast<cuuint64_t>(d.M)};
-        cuuint64_t strides[1] = {static_cast<cuuint64_t>(d.K) * 2};
-        cuuint32_t box[2] = {UMMA_BK, UMMA_BM};
-        cuuint32_t es[2] = {1, 1};
-        r = p->encode(&p->tmap_a, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(A), dims, strides,
+        // A row-major [batch][M][K] (batch items stride_a elements apart): (k, m, item)
+        cuuint64_t dims[3] = {static_cast<cuuint64_t>(d.K), static_cast<cuuint64_t>(d.M),
+                              static_cast<cuuint64_t>(p->batch)};
+        cuuint64_t strides[2] = {static_cast<cuuint64_t>(d.K) * 2, static_cast<cuuint64_t>(p->stride_a) * 2};
+        cuuint32_t box[3] = {UMMA_BK, UMMA_BM, 1};
+        cuuint32_t es[3] = {1, 1, 1};
+        r = p->encode(&p->tmap_a, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(A), dims, strides,
                       box, es, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
                       CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
     }
@@ -292,21 +299,25 @@ static nk_status_t encode_maps(nk_gemm_s* p, const void* A, const void* B) {
         p->b_3d = d.N % 64 == 0;
         const int slabs = (p->pair ? p->bn / 2 : p->bn) / 64;
         if (p->b_3d) {
-            cuuint64_t dims[3] = {64, static_cast<cuuint64_t>(d.K), static_cast<cuuint64_t>(d.N / 64)};
-            cuuint64_t strides[2] = {static_cast<cuuint64_t>(d.N) * 2, 128};
-            cuuint32_t box[3] = {64, UMMA_BK, static_cast<cuuint32_t>(slabs)};
-            cuuint32_t es[3] = {1, 1, 1};
-            r = p->encode(&p->tmap_b, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(B), dims, strides,
+            // (n within slab, k, slab, item)
+            cuuint64_t dims[4] = {64, static_cast<cuuint64_t>(d.K), static_cast<cuuint64_t>(d.N / 64),
+                                  static_cast<cuuint64_t>(p->batch)};
+            cuuint64_t strides[3] = {static_cast<cuuint64_t>(d.N) * 2, 128, static_cast<cuuint64_t>(p->stride_b) * 2};
+            cuuint32_t box[4] = {64, UMMA_BK, static_cast<cuuint32_t>(slabs), 1};
+            cuuint32_t es[4] = {1, 1, 1, 1};
+            r = p->encode(&p->tmap_b, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void*>(B), dims, strides,
                           box, es, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
                           CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
             if (r != CUDA_SUCCESS) p->b_3d = false;   // fall back to per-slab boxes
         }
         if (!p->b_3d) {
-            cuuint64_t dims[2] = {static_cast<cuuint64_t>(d.N), static_cast<cuuint64_t>(d.K)};
-            cuuint64_t strides[1] = {static_cast<cuuint64_t>(d.N) * 2};
-            cuuint32_t box[2] = {64, UMMA_BK};
-            cuuint32_t es[2] = {1, 1};
-            r = p->encode(&p->tmap_b, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(B), dims, strides,
+            // (n, k, item)
+            cuuint64_t dims[3] = {static_cast<cuuint64_t>(d.N), static_cast<cuuint64_t>(d.K),
+                                  static_cast<cuuint64_t>(p->batch)};
+            cuuint64_t strides[2] = {static_cast<cuuint64_t>(d.N) * 2, static_cast<cuuint64_t>(p->stride_b) * 2};
+            cuuint32_t box[3] = {64, UMMA_BK, 1};
+            cuuint32_t es[3] = {1, 1, 1};
+            r = p->encode(&p->tmap_b, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(B), dims, strides,
                           box, es, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
                           CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
         }
@@ -449,6 +460,19 @@ nk_status_t nk_gemm_create(const nk_gemm_desc_t* desc, nk_gemm_t* out) {
     if (blocked && d.in_dtype != NK_BF16) return NK_ERR_UNSUPPORTED;
     if (d.layout_a == NK_BLOCKED32 && (d.M % 32 || d.K % 32)) return NK_ERR_MISALIGNED;
     if (d.layout_b == NK_BLOCKED32 && (d.N % 32 || d.K % 32)) return NK_ERR_MISALIGNED;
+    if (d.beta != 0 && d.beta != 1) return NK_ERR_INVALID_ARG;
+    if (d.batch < 0 || d.stride_a < 0 || d.stride_b < 0) return NK_ERR_INVALID_ARG;
+    const int64_t nbatch = d.batch > 1 ? d.batch : 1;
+    const int64_t str_a = d.stride_a > 0 ? d.stride_a : d.M * d.K;
+    const int64_t str_b = d.stride_b > 0 ? d.stride_b : d.K * d.N;
+    if (nbatch > 1) {
+        if (blocked) return NK_ERR_UNSUPPORTED;          // batch-reduce: row-major operands only
+        if (nbatch > 65535 || nbatch * d.K >= (1ll << 24)) return NK_ERR_UNSUPPORTED;
+        const int64_t gran = d.in_dtype == NK_BF16 ? 8 : 4;
+        if (str_a % gran || str_b % gran) return NK_ERR_MISALIGNED;
+        if (str_a < d.M * d.K || str_b < d.K * d.N) return NK_ERR_INVALID_ARG;   // items must not overlap
+    }
+    if (d.beta == 1 && blocked) return NK_ERR_UNSUPPORTED;
     const uint32_t force = d.flags & NK_FLAG_KERNEL_MASK;
     if (force > NK_FLAG_KERNEL_UMMA) return NK_ERR_INVALID_ARG;
     if (force != NK_FLAG_KERNEL_NAIVE) {
@@ -473,6 +497,9 @@ nk_status_t nk_gemm_create(const nk_gemm_desc_t* desc, nk_gemm_t* out) {
     memset(p, 0, sizeof(*p));
     p->d = d;
     p->sm_count = prop.multiProcessorCount;
+    p->batch = static_cast<int>(nbatch);
+    p->stride_a = str_a;
+    p->stride_b = str_b;
 
     DeviceGuard guard(d.device);
     if (guard.err != cudaSuccess) { delete p; return NK_ERR_DEVICE; }
@@ -484,7 +511,7 @@ nk_status_t nk_gemm_create(const nk_gemm_desc_t* desc, nk_gemm_t* out) {
         p->variant = V_NAIVE;
         p->launches = 1;
         snprintf(p->name, sizeof(p->name), "naive");
-    } else if (d.in_dtype == NK_F32 && d.M <= 32 && force != NK_FLAG_KERNEL_SIMT) {
+    } else if (d.in_dtype == NK_F32 && d.M <= 32 && force != NK_FLAG_KERNEL_SIMT && nbatch == 1 && d.beta == 0) {
         p->variant = V_SKINNY;
         choose_skinny(p);
         p->ws_partial_bytes = p->splits > 1 ? static_cast<size_t>(p->splits) * d.M * d.N * 4 : 0;
@@ -531,6 +558,10 @@ nk_status_t nk_gemm_create(const nk_gemm_desc_t* desc, nk_gemm_t* out) {
                  p->splits, d.layout_a == NK_BLOCKED32 ? "_ablk" : "",
                  p->b_vnni_inkernel ? "_bvnni" : (p->b_repack ? "_brepack" : ""));
     }
+    if (p->batch > 1 || d.beta) {
+        const size_t len = strlen(p->name);
+        snprintf(p->name + len, sizeof(p->name) - len, "_br%d%s", p->batch, d.beta ? "_beta1" : "");
+    }
     *out = p;
     return NK_OK;
 }
@@ -561,7 +592,8 @@ nk_status_t nk_gemm_run(nk_gemm_t p, const void* A, const void* B, const void* b
     if (p->variant == V_NAIVE) {
         NaiveParams np = {static_cast<int>(d.M), static_cast<int>(d.N), static_cast<int>(d.K),
                           d.in_dtype == NK_BF16, d.out_dtype == NK_BF16, d.layout_a == NK_BLOCKED32,
-                          d.layout_b == NK_BLOCKED32, d.epilogue, A, B, bias, C};
+                          d.layout_b == NK_BLOCKED32, d.epilogue, p->batch, d.beta, p->stride_a, p->stride_b,
+                          A, B, bias, C};
         dim3 grid(ceil_div(d.N, 128), static_cast<unsigned>(d.M));
         if (d.M > 65535) return NK_ERR_UNSUPPORTED;
         naive_gemm_kernel<<<grid, 128, 0, st>>>(np);
@@ -584,7 +616,8 @@ nk_status_t nk_gemm_run(nk_gemm_t p, const void* A, const void* B, const void* b
         if (e != cudaSuccess) { set_err(p, "skinny launch", e); return NK_ERR_CUDA; }
     } else if (p->variant == V_SIMT) {
         SimtParams sp = {static_cast<int>(d.M), static_cast<int>(d.N), static_cast<int>(d.K), p->splits,
-                         p->kt_per_split, d.epilogue, static_cast<const float*>(A),
+                         p->kt_per_split, p->batch, ceil_div(d.K, SIMT_BK), p->stride_a, p->stride_b, d.beta,
+                         d.epilogue, static_cast<const float*>(A),
                          static_cast<const float*>(B), static_cast<const float*>(bias),
                          static_cast<float*>(C), partial};
         e = launch_simt(p, sp, st);
@@ -608,7 +641,9 @@ nk_status_t nk_gemm_run(nk_gemm_t p, const void* A, const void* B, const void* b
         up.tiles_m = ceil_div(d.M, p->pair ? 2 * UMMA_BM : UMMA_BM);
         up.tiles_n = ceil_div(d.N, p->bn);
         up.splits = p->splits;
-        up.kb_total = ceil_div(d.K, UMMA_BK);
+        up.kb_per_item = ceil_div(d.K, UMMA_BK);
+        up.kb_total = p->batch * up.kb_per_item;
+        up.beta = d.beta;
         up.kb_per_split = ceil_div(up.kb_total, p->splits);
         up.group_m = p->group_m;
         up.a_blocked = d.layout_a == NK_BLOCKED32;
@@ -634,7 +669,7 @@ nk_status_t nk_gemm_run(nk_gemm_t p, const void* A, const void* B, const void* b
 
     if (p->splits > 1) {
         ReduceParams rp = {static_cast<size_t>(d.M) * d.N, static_cast<int>(d.N), p->splits, d.epilogue,
-                           d.in_dtype == NK_BF16, d.out_dtype == NK_BF16, partial, bias, C};
+                           d.in_dtype == NK_BF16, d.out_dtype == NK_BF16, d.beta, partial, bias, C};
         const size_t quads = rp.MN / 4;
         splitk_reduce_kernel<<<static_cast<unsigned>((quads + 255) / 256), 256, 0, st>>>(rp);
         e = cudaGetLastError();
@@ -654,8 +689,14 @@ nk_status_t nk_gemm_run_host(nk_gemm_t p, const void* hA, const void* hB, const 
     DeviceGuard guard(d.device);
     if (guard.err != cudaSuccess) { set_err(p, "cudaSetDevice", guard.err); return NK_ERR_DEVICE; }
     cudaError_t e;
-    if ((e = cudaMemcpyAsync(dA, hA, ein * d.M * d.K, cudaMemcpyHostToDevice, st)) != cudaSuccess ||
-        (e = cudaMemcpyAsync(dB, hB, ein * d.K * d.N, cudaMemcpyHostToDevice, st)) != cudaSuccess) {
+    const size_t a_elems = static_cast<size_t>(p->batch - 1) * p->stride_a + static_cast<size_t>(d.M) * d.K;
+    const size_t b_elems = static_cast<size_t>(p->batch - 1) * p->stride_b + static_cast<size_t>(d.K) * d.N;
+    if (d.beta && (e = cudaMemcpyAsync(dC, hC, eout * d.M * d.N, cudaMemcpyHostToDevice, st)) != cudaSuccess) {
+        set_err(p, "H2D copy", e);
+        return NK_ERR_CUDA;
+    }
+    if ((e = cudaMemcpyAsync(dA, hA, ein * a_elems, cudaMemcpyHostToDevice, st)) != cudaSuccess ||
+        (e = cudaMemcpyAsync(dB, hB, ein * b_elems, cudaMemcpyHostToDevice, st)) != cudaSuccess) {
         set_err(p, "H2D copy", e);
         return NK_ERR_CUDA;
     }

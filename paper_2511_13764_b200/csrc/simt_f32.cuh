@@ -18,6 +18,10 @@ struct SimtParams {
     int M, N, K;
     int splits;        // gridDim.z; > 1 writes partials
     int kt_per_split;  // k-tiles (of 16) per split
+    int batch;         // batch-reduce: number of (A_b, B_b) pairs summed into C (>= 1)
+    int kt_per_item;   // ceil(K / 16): k-tiles of one pair
+    long long stride_a, stride_b;  // elements between consecutive A_b / B_b
+    int beta;          // 1: the old C is added before the epilogue
     int epilogue;      // 0 none, 1 bias + ReLU
     const float* A;    // [M][K]
     const float* B;    // [K][N]
@@ -46,7 +50,7 @@ simt_f32_kernel(const SimtParams p) {
     const int t = threadIdx.x;
     const int ty = t / TX, tx = t % TX;
     const int m0 = blockIdx.y * BM, n0 = blockIdx.x * BN;
-    const int ktiles = (p.K + SIMT_BK - 1) / SIMT_BK;
+    const int ktiles = p.batch * p.kt_per_item;   // k-tiles of the whole batch-reduce
     const int kt0 = blockIdx.z * p.kt_per_split;
     const int kt1 = min(ktiles, kt0 + p.kt_per_split);
 
@@ -59,14 +63,17 @@ simt_f32_kernel(const SimtParams p) {
     float4 ra[A_V4], rb[B_V4];
 
     auto load_global = [&](int kt) {
-        const int k0 = kt * SIMT_BK;
+        const int item = kt / p.kt_per_item;               // which (A_b, B_b) pair
+        const int k0 = (kt - item * p.kt_per_item) * SIMT_BK;
+        const float* Ab = p.A + item * p.stride_a;
+        const float* Bb = p.B + item * p.stride_b;
 #pragma unroll
         for (int i = 0; i < A_V4; ++i) {
             const int idx = t + i * THREADS;       // over BM x 4 float4s
             const int row = idx >> 2, kq = (idx & 3) * 4;
             const int gm = m0 + row, gk = k0 + kq;
             ra[i] = (gm < p.M && gk < p.K)
-                        ? __ldg(reinterpret_cast<const float4*>(p.A + static_cast<size_t>(gm) * p.K + gk))
+                        ? __ldg(reinterpret_cast<const float4*>(Ab + static_cast<size_t>(gm) * p.K + gk))
                         : make_float4(0.f, 0.f, 0.f, 0.f);
         }
 #pragma unroll
@@ -75,7 +82,7 @@ simt_f32_kernel(const SimtParams p) {
             const int kr = idx / (BN / 4), nq = (idx % (BN / 4)) * 4;
             const int gk = k0 + kr, gn = n0 + nq;
             rb[i] = (gk < p.K && gn < p.N)
-                        ? __ldg(reinterpret_cast<const float4*>(p.B + static_cast<size_t>(gk) * p.N + gn))
+                        ? __ldg(reinterpret_cast<const float4*>(Bb + static_cast<size_t>(gk) * p.N + gn))
                         : make_float4(0.f, 0.f, 0.f, 0.f);
         }
     };
@@ -151,6 +158,10 @@ simt_f32_kernel(const SimtParams p) {
                 if (gn >= p.N) continue;
                 float4 v = make_float4(acc[4 * gi + ii][4 * gj], acc[4 * gi + ii][4 * gj + 1],
                                        acc[4 * gi + ii][4 * gj + 2], acc[4 * gi + ii][4 * gj + 3]);
+                if (!to_partial && p.beta) {       // beta = 1: the accumulation tile starts from the stored C
+                    const float4 cv = *reinterpret_cast<const float4*>(out + static_cast<size_t>(gm) * p.N + gn);
+                    v.x += cv.x; v.y += cv.y; v.z += cv.z; v.w += cv.w;
+                }
                 if (!to_partial && p.epilogue) {
                     const float4 bv = __ldg(reinterpret_cast<const float4*>(p.bias + gn));
                     v.x = fmaxf(v.x + bv.x, 0.f);
@@ -307,7 +318,7 @@ simt_f32_async_kernel(const SimtParams p) {
     const int t = threadIdx.x;
     const int ty = t / TX, tx = t % TX;
     const int m0 = blockIdx.y * BM, n0 = blockIdx.x * BN;
-    const int ktiles = (p.K + SIMT_BK - 1) / SIMT_BK;
+    const int ktiles = p.batch * p.kt_per_item;   // k-tiles of the whole batch-reduce
     const int kt0 = blockIdx.z * p.kt_per_split;
     const int kt1 = min(ktiles, kt0 + p.kt_per_split);
 
@@ -319,13 +330,16 @@ simt_f32_async_kernel(const SimtParams p) {
 
     auto issue_tile = [&](int kt, int stage) {
         if (kt < kt1) {
-            const int k0 = kt * SIMT_BK;
+            const int item = kt / p.kt_per_item;
+            const int k0 = (kt - item * p.kt_per_item) * SIMT_BK;
+            const float* Ab = p.A + item * p.stride_a;
+            const float* Bb = p.B + item * p.stride_b;
 #pragma unroll
             for (int i = 0; i < A_ELEMS; ++i) {
                 const int e = t + i * THREADS;             // 16 consecutive lanes = one row's 16 k
                 const int k = e & (SIMT_BK - 1), row = e / SIMT_BK;
                 const bool ok = m0 + row < p.M && k0 + k < p.K;
-                const float* src = p.A + (ok ? static_cast<size_t>(m0 + row) * p.K + k0 + k : 0);
+                const float* src = Ab + (ok ? static_cast<size_t>(m0 + row) * p.K + k0 + k : 0);
                 cp_async_4(as_u32 + (stage * A_STAGE + k * AP + row) * 4, src, ok ? 4u : 0u);
             }
 #pragma unroll
@@ -333,7 +347,7 @@ simt_f32_async_kernel(const SimtParams p) {
                 const int idx = t + i * THREADS;
                 const int kr = idx / (BN / 4), nq = (idx % (BN / 4)) * 4;
                 const bool ok = k0 + kr < p.K && n0 + nq < p.N;
-                const float* src = p.B + (ok ? static_cast<size_t>(k0 + kr) * p.N + n0 + nq : 0);
+                const float* src = Bb + (ok ? static_cast<size_t>(k0 + kr) * p.N + n0 + nq : 0);
                 cp_async_16(bs_u32 + (stage * B_STAGE + kr * BN + nq) * 4, src, ok ? 16u : 0u);
             }
         }
@@ -388,6 +402,10 @@ simt_f32_async_kernel(const SimtParams p) {
                 if (gn >= p.N) continue;
                 float4 v = make_float4(acc[4 * gi + ii][4 * gj], acc[4 * gi + ii][4 * gj + 1],
                                        acc[4 * gi + ii][4 * gj + 2], acc[4 * gi + ii][4 * gj + 3]);
+                if (!to_partial && p.beta) {       // beta = 1: the accumulation tile starts from the stored C
+                    const float4 cv = *reinterpret_cast<const float4*>(out + static_cast<size_t>(gm) * p.N + gn);
+                    v.x += cv.x; v.y += cv.y; v.z += cv.z; v.w += cv.w;
+                }
                 if (!to_partial && p.epilogue) {
                     const float4 bv = __ldg(reinterpret_cast<const float4*>(p.bias + gn));
                     v.x = fmaxf(v.x + bv.x, 0.f);

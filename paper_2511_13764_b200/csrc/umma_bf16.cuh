@@ -36,7 +36,9 @@ struct UmmaParams {
     int M, N, K;
     int tiles_m, tiles_n;
     int splits;         // K splits; > 1 writes FP32 partials to `partial`
-    int kb_total;       // ceil(K / 64)
+    int kb_total;       // batch * kb_per_item: k-blocks of the whole reduction
+    int kb_per_item;    // ceil(K / 64): k-blocks of one (A_b, B_b) pair of the batch-reduce
+    int beta;           // 1: the old C is added before the epilogue (Algorithm 1's beta.C)
     int kb_per_split;   // ceil(kb_total / splits)
     int group_m;        // raster: this many M tiles sweep N together
     int a_blocked;      // A tensor map is the 4-D blocked view
@@ -95,6 +97,37 @@ __device__ __forceinline__ void umma_store_chunk(const UmmaParams& p, uint32_t (
         for (int i = 0; i < 32; ++i) v[i] = 0u;
     }
     const bool to_partial = p.splits > 1;
+    if (!to_partial && p.beta && row < p.M) {
+        // beta = 1: the accumulation tile starts from the stored C (Algorithm 1 loads the C
+        // sub-block before the K loop; adding it here, in FP32, gives the same sum)
+        if (p.out_bf16) {
+            const uint4* csrc = reinterpret_cast<const uint4*>(static_cast<const uint16_t*>(p.C) +
+                                                               static_cast<size_t>(row) * p.N + col0);
+#pragma unroll
+            for (int g = 0; g < 4; ++g) {
+                if (col0 + 8 * g >= p.N) break;
+                const uint4 c = csrc[g];
+                const uint32_t w[4] = {c.x, c.y, c.z, c.w};
+#pragma unroll
+                for (int j = 0; j < 4; ++j) {
+                    v[8 * g + 2 * j] = __float_as_uint(__uint_as_float(v[8 * g + 2 * j]) + bf16_bits_to_f32(w[j] & 0xFFFFu));
+                    v[8 * g + 2 * j + 1] = __float_as_uint(__uint_as_float(v[8 * g + 2 * j + 1]) + bf16_bits_to_f32(w[j] >> 16));
+                }
+            }
+        } else {
+            const uint4* csrc = reinterpret_cast<const uint4*>(static_cast<const float*>(p.C) +
+                                                               static_cast<size_t>(row) * p.N + col0);
+#pragma unroll
+            for (int g = 0; g < 8; ++g) {
+                if (col0 + 4 * g >= p.N) break;
+                const uint4 c = csrc[g];
+                v[4 * g] = __float_as_uint(__uint_as_float(v[4 * g]) + __uint_as_float(c.x));
+                v[4 * g + 1] = __float_as_uint(__uint_as_float(v[4 * g + 1]) + __uint_as_float(c.y));
+                v[4 * g + 2] = __float_as_uint(__uint_as_float(v[4 * g + 2]) + __uint_as_float(c.z));
+                v[4 * g + 3] = __float_as_uint(__uint_as_float(v[4 * g + 3]) + __uint_as_float(c.w));
+            }
+        }
+    }
     if (!to_partial && p.epilogue) {
         const uint4* bsrc = reinterpret_cast<const uint4*>(static_cast<const uint16_t*>(p.bias) + col0);
 #pragma unroll
@@ -264,8 +297,11 @@ umma_bf16_kernel(const __grid_constant__ CUtensorMap tmap_a,
             const int kb0 = split * p.kb_per_split;
             const int kb1 = min(p.kb_total, kb0 + p.kb_per_split);
             const int row0 = mb * UMMA_BM, col0 = nb * BN;
-            int kx = kb0 * UMMA_BK;
-            for (int kb = kb0; kb < kb1; ++kb, kx += UMMA_BK) {
+            // k-block kb of the reduction = k-block (kb % kb_per_item) of batch item kb / kb_per_item
+            int item = kb0 / p.kb_per_item;
+            int kbl = kb0 - item * p.kb_per_item;
+            for (int kb = kb0; kb < kb1; ++kb) {
+                const int kx = kbl * UMMA_BK;
                 if (!mbar_wait(empty_bar(stage), phase ^ 1u, abort_flag)) {
                     if (lane == 0) give_up(0x100u + stage);
                     ok = false;
@@ -276,21 +312,22 @@ umma_bf16_kernel(const __grid_constant__ CUtensorMap tmap_a,
                     mbar_arrive_expect_tx(fb, UMMA_A_STAGE_BYTES + (B_VNNI ? 0 : B_STAGE));
                     if (a_blk) {
                         // two 32-wide K slabs, each 128 rows x 64 B (64-byte swizzle)
-                        tma_load_4d(sa, &tmap_a, fb, 0, 0, kb * 2, mb * 4);
-                        tma_load_4d(sa + 8192, &tmap_a, fb, 0, 0, kb * 2 + 1, mb * 4);
+                        tma_load_4d(sa, &tmap_a, fb, 0, 0, kbl * 2, mb * 4);
+                        tma_load_4d(sa + 8192, &tmap_a, fb, 0, 0, kbl * 2 + 1, mb * 4);
                     } else {
-                        tma_load_2d(sa, &tmap_a, fb, kx, row0);
+                        tma_load_3d(sa, &tmap_a, fb, kx, row0, item);
                     }
                     if (!B_VNNI) {
                         if (b3d) {
-                            tma_load_3d(sb, &tmap_b, fb, 0, kx, col0 >> 6);
+                            tma_load_4d(sb, &tmap_b, fb, 0, kx, col0 >> 6, item);
                         } else {
 #pragma unroll
                             for (int j = 0; j < BN / 64; ++j)
-                                tma_load_2d(sb + j * 8192, &tmap_b, fb, col0 + j * 64, kx);
+                                tma_load_3d(sb + j * 8192, &tmap_b, fb, col0 + j * 64, kx, item);
                         }
                     }
                 }
+                if (++kbl == p.kb_per_item) { kbl = 0; ++item; }
                 __syncwarp();
                 sa += STAGE;
                 fb += 8;

@@ -104,8 +104,10 @@ umma_bf16_pair_kernel(const __grid_constant__ CUtensorMap tmap_a,
             const int kb1 = min(p.kb_total, kb0 + p.kb_per_split);
             const int row0 = mb * BM2 + static_cast<int>(rank) * UMMA_BM;
             const int col0 = nb * BN + static_cast<int>(rank) * HALF;
-            int kx = kb0 * UMMA_BK;
-            for (int kb = kb0; kb < kb1; ++kb, kx += UMMA_BK) {
+            int item = kb0 / p.kb_per_item;
+            int kbl = kb0 - item * p.kb_per_item;
+            for (int kb = kb0; kb < kb1; ++kb) {
+                const int kx = kbl * UMMA_BK;
                 if (!mbar_wait(empty_bar(stage), phase ^ 1u, abort_flag)) {
                     if (lane == 0) give_up(0x100u + stage);
                     ok = false;
@@ -116,21 +118,22 @@ umma_bf16_pair_kernel(const __grid_constant__ CUtensorMap tmap_a,
                     if (rank == 0)
                         mbar_arrive_expect_tx(fb, 2u * (UMMA_A_STAGE_BYTES + (B_VNNI ? 0 : B_STAGE)));
                     if (a_blk) {
-                        tma_load_4d_pair(sa, &tmap_a, lfb, 0, 0, kb * 2, row0 / 32);
-                        tma_load_4d_pair(sa + 8192, &tmap_a, lfb, 0, 0, kb * 2 + 1, row0 / 32);
+                        tma_load_4d_pair(sa, &tmap_a, lfb, 0, 0, kbl * 2, row0 / 32);
+                        tma_load_4d_pair(sa + 8192, &tmap_a, lfb, 0, 0, kbl * 2 + 1, row0 / 32);
                     } else {
-                        tma_load_2d_pair(sa, &tmap_a, lfb, kx, row0);
+                        tma_load_3d_pair(sa, &tmap_a, lfb, kx, row0, item);
                     }
                     if (!B_VNNI) {
                         if (b3d) {
-                            tma_load_3d_pair(sb, &tmap_b, lfb, 0, kx, col0 >> 6);
+                            tma_load_4d_pair(sb, &tmap_b, lfb, 0, kx, col0 >> 6, item);
                         } else {
 #pragma unroll
                             for (int j = 0; j < HALF / 64; ++j)
-                                tma_load_2d_pair(sb + j * 8192, &tmap_b, lfb, col0 + j * 64, kx);
+                                tma_load_3d_pair(sb + j * 8192, &tmap_b, lfb, col0 + j * 64, kx, item);
                         }
                     }
                 }
+                if (++kbl == p.kb_per_item) { kbl = 0; ++item; }
                 __syncwarp();
                 sa += STAGE;
                 fb += 8;
