@@ -82,6 +82,10 @@ typedef struct {
     int64_t batch;     /* number of (A_b, B_b) pairs reduced into C; 0 means 1          */
     int64_t stride_a;  /* elements from A_b to A_b+1; 0 means M*K (contiguous)          */
     int64_t stride_b;  /* elements from B_b to B_b+1; 0 means K*N                       */
+    /* Batched matmul (Section 5(b): the same nanokernels serve batch.matmul): */
+    int64_t stride_c;  /* elements from C_b to C_b+1; 0 means M*N                       */
+    int32_t batch_independent; /* 0: the batch is reduced into one C; 1: C_b = A_b . B_b for
+                                  every b (bias shared; beta applies to each C_b)        */
 } nk_gemm_desc_t;
 
 /*

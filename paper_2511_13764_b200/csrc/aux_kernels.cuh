@@ -15,6 +15,8 @@ struct NaiveParams {
     int in_bf16, out_bf16, a_blocked, b_blocked, epilogue;
     int batch, beta;
     long long stride_a, stride_b;
+    int gemms;             // batched matmul: gridDim.z independent GEMMs
+    long long stride_c;
     const void *A, *B, *bias;
     void* C;
 };
@@ -31,7 +33,8 @@ __global__ void naive_gemm_kernel(const NaiveParams p) {
     const int i = blockIdx.y;
     if (j >= p.N || i >= p.M) return;
     const size_t kb32 = p.K / 32;
-    const size_t o = static_cast<size_t>(i) * p.N + j;
+    const int g = blockIdx.z;
+    const size_t o = static_cast<size_t>(g) * p.stride_c + static_cast<size_t>(i) * p.N + j;
     float acc = 0.f;
     if (p.beta) acc = ld_elem(p.C, p.out_bf16, o);
     for (int b = 0; b < p.batch; ++b)
@@ -42,7 +45,7 @@ __global__ void naive_gemm_kernel(const NaiveParams p) {
         const size_t ib = p.b_blocked
             ? (((((static_cast<size_t>(j / 32) * kb32 + k / 32) * 16 + (k % 32) / 2) * 32 + j % 32) * 2) + k % 2)
             : static_cast<size_t>(k) * p.N + j;
-        acc = fmaf(ld_elem(p.A, p.in_bf16, b * p.stride_a + ia), ld_elem(p.B, p.in_bf16, b * p.stride_b + ib), acc);
+        acc = fmaf(ld_elem(p.A, p.in_bf16, (g + b) * p.stride_a + ia), ld_elem(p.B, p.in_bf16, (g + b) * p.stride_b + ib), acc);
     }
     if (p.epilogue) acc = fmaxf(acc + ld_elem(p.bias, p.in_bf16, j), 0.f);
     if (p.out_bf16)

@@ -48,8 +48,10 @@ struct nk_gemm_s {
     int kt_per_split;
     int skinny_kc;  // FP32 skinny kernel: k per CTA
     // batch-reduce (normalised: batch >= 1, strides in elements)
-    int batch;
+    int batch;              // items reduced into one C (1 in a batched matmul)
     long long stride_a, stride_b;
+    int gemms;              // independent GEMMs per run (batched matmul), else 1
+    long long stride_c;
     // workspace layout
     size_t ws_repack_bytes, ws_partial_bytes;
     // device status word
@@ -117,13 +119,14 @@ static int umma_stages_for(int bn) { return bn == 256 ? 4 : bn == 128 ? 6 : 8; }
 // (the stage pipeline is latency bound), so wide tiles win whenever they do not cost rounds.
 struct UmmaChoice { bool pair; int bn; int splits; double us; };
 
-static int desc_batch(const nk_gemm_desc_t& d) { return d.batch > 1 ? static_cast<int>(d.batch) : 1; }
+static int desc_batch(const nk_gemm_desc_t& d) { return (d.batch > 1 && !d.batch_independent) ? static_cast<int>(d.batch) : 1; }
+static int desc_gemms(const nk_gemm_desc_t& d) { return (d.batch > 1 && d.batch_independent) ? static_cast<int>(d.batch) : 1; }
 
 static double umma_model_us(const nk_gemm_desc_t& d, int sms, bool pair, int bn, int splits) {
     const int kb_total = desc_batch(d) * ceil_div(d.K, UMMA_BK);
     const int per = ceil_div(kb_total, splits);
     const int eff_splits = ceil_div(kb_total, per);
-    const int64_t tiles = static_cast<int64_t>(ceil_div(d.M, pair ? 256 : 128)) * ceil_div(d.N, bn);
+    const int64_t tiles = static_cast<int64_t>(desc_gemms(d)) * ceil_div(d.M, pair ? 256 : 128) * ceil_div(d.N, bn);
     const int64_t units = tiles * eff_splits;
     const int workers = pair ? sms / 2 : sms;
     const double rounds = static_cast<double>((units + workers - 1) / workers);
@@ -161,7 +164,7 @@ static void choose_umma(nk_gemm_s* p) {
                 if (splits > kb_total) splits = kb_total;
                 if (forced_s == 0 && splits > 1) {
                     if (kb_total / splits < 4) continue;  // >= 4 k-blocks per split
-                    if (static_cast<double>(splits) * d.M * d.N * 4.0 > 256.0 * 1024 * 1024) continue;
+                    if (static_cast<double>(splits) * desc_gemms(d) * d.M * d.N * 4.0 > 256.0 * 1024 * 1024) continue;
                 }
                 const double us = umma_model_us(d, sms, pair, bn, splits);
                 if (us < best.us) best = {pair, bn, splits, us};
@@ -190,7 +193,7 @@ static double simt_model_us(const nk_gemm_desc_t& d, int sms, int tile, int spli
     const int ktiles = desc_batch(d) * ceil_div(d.K, SIMT_BK);
     const int per = ceil_div(ktiles, splits);
     const int eff_splits = ceil_div(ktiles, per);
-    const int64_t tiles = static_cast<int64_t>(ceil_div(d.M, tile)) * ceil_div(d.N, tile);
+    const int64_t tiles = static_cast<int64_t>(desc_gemms(d)) * ceil_div(d.M, tile) * ceil_div(d.N, tile);
     const int64_t units = tiles * eff_splits;
     const int res = tile == 128 ? 2 : tile == 64 ? 4 : 16;
     const double eff = tile == 128 ? 0.75 : tile == 64 ? 0.50 : 0.37;
@@ -229,7 +232,7 @@ static void choose_simt(nk_gemm_s* p) {
             if (splits > ktiles) splits = ktiles;
             if (forced_s == 0 && splits > 1) {
                 if (ktiles / splits < 8) continue;   // >= 8 k-tiles (128 k) per split
-                if (static_cast<double>(splits) * d.M * d.N * 4.0 > 256.0 * 1024 * 1024) continue;
+                if (static_cast<double>(splits) * desc_gemms(d) * d.M * d.N * 4.0 > 256.0 * 1024 * 1024) continue;
             }
             const double us = simt_model_us(d, sms, tile, splits);
             if (us < best_us) { best_us = us; best_tile = tile; best_splits = splits; }
@@ -280,7 +283,7 @@ static nk_status_t encode_maps(nk_gemm_s* p, const void* A, const void* B) {
     } else {
         // A row-major [batch][M][K] (batch items stride_a elements apart): (k, m, item)
         cuuint64_t dims[3] = {static_cast<cuuint64_t>(d.K), static_cast<cuuint64_t>(d.M),
-                              static_cast<cuuint64_t>(p->batch)};
+                              static_cast<cuuint64_t>(p->batch * p->gemms)};
         cuuint64_t strides[2] = {static_cast<cuuint64_t>(d.K) * 2, static_cast<cuuint64_t>(p->stride_a) * 2};
         cuuint32_t box[3] = {UMMA_BK, UMMA_BM, 1};
         cuuint32_t es[3] = {1, 1, 1};
@@ -301,7 +304,7 @@ static nk_status_t encode_maps(nk_gemm_s* p, const void* A, const void* B) {
         if (p->b_3d) {
             // (n within slab, k, slab, item)
             cuuint64_t dims[4] = {64, static_cast<cuuint64_t>(d.K), static_cast<cuuint64_t>(d.N / 64),
-                                  static_cast<cuuint64_t>(p->batch)};
+                                  static_cast<cuuint64_t>(p->batch * p->gemms)};
             cuuint64_t strides[3] = {static_cast<cuuint64_t>(d.N) * 2, 128, static_cast<cuuint64_t>(p->stride_b) * 2};
             cuuint32_t box[4] = {64, UMMA_BK, static_cast<cuuint32_t>(slabs), 1};
             cuuint32_t es[4] = {1, 1, 1, 1};
@@ -313,7 +316,7 @@ static nk_status_t encode_maps(nk_gemm_s* p, const void* A, const void* B) {
         if (!p->b_3d) {
             // (n, k, item)
             cuuint64_t dims[3] = {static_cast<cuuint64_t>(d.N), static_cast<cuuint64_t>(d.K),
-                                  static_cast<cuuint64_t>(p->batch)};
+                                  static_cast<cuuint64_t>(p->batch * p->gemms)};
             cuuint64_t strides[2] = {static_cast<cuuint64_t>(d.N) * 2, static_cast<cuuint64_t>(p->stride_b) * 2};
             cuuint32_t box[3] = {64, UMMA_BK, 1};
             cuuint32_t es[3] = {1, 1, 1};
@@ -414,7 +417,7 @@ static cudaError_t prepare_umma_attrs() {
 
 static cudaError_t launch_simt(nk_gemm_s* p, const SimtParams& sp, cudaStream_t st) {
     const int t = p->simt_tile;
-    dim3 grid(ceil_div(sp.N, t), ceil_div(sp.M, t), sp.splits);
+    dim3 grid(ceil_div(sp.N, t), ceil_div(sp.M, t), sp.splits * sp.gemms);
     // 128-tile: register-staged double buffer (a little faster when the FMA pipe is the limit);
     // smaller tiles: three-stage cp.async pipeline (their K loops are latency bound).
     if (t == 128) simt_f32_kernel<128, 128, 8, 8><<<grid, 256, 0, st>>>(sp);
@@ -473,6 +476,16 @@ nk_status_t nk_gemm_create(const nk_gemm_desc_t* desc, nk_gemm_t* out) {
         if (str_a < d.M * d.K || str_b < d.K * d.N) return NK_ERR_INVALID_ARG;   // items must not overlap
     }
     if (d.beta == 1 && blocked) return NK_ERR_UNSUPPORTED;
+    if (d.batch_independent != 0 && d.batch_independent != 1) return NK_ERR_INVALID_ARG;
+    if (d.stride_c < 0) return NK_ERR_INVALID_ARG;
+    const int64_t str_c = d.stride_c > 0 ? d.stride_c : d.M * d.N;
+    const bool indep = d.batch_independent == 1 && nbatch > 1;
+    if (indep) {
+        const int64_t gran_c = d.out_dtype == NK_BF16 ? 8 : 4;
+        if (str_c % gran_c) return NK_ERR_MISALIGNED;
+        if (str_c < d.M * d.N) return NK_ERR_INVALID_ARG;
+        if (nbatch * d.M * d.N >= (1ll << 31)) return NK_ERR_UNSUPPORTED;
+    }
     const uint32_t force = d.flags & NK_FLAG_KERNEL_MASK;
     if (force > NK_FLAG_KERNEL_UMMA) return NK_ERR_INVALID_ARG;
     if (force != NK_FLAG_KERNEL_NAIVE) {
@@ -497,9 +510,14 @@ nk_status_t nk_gemm_create(const nk_gemm_desc_t* desc, nk_gemm_t* out) {
     memset(p, 0, sizeof(*p));
     p->d = d;
     p->sm_count = prop.multiProcessorCount;
-    p->batch = static_cast<int>(nbatch);
+    p->batch = indep ? 1 : static_cast<int>(nbatch);
+    p->gemms = indep ? static_cast<int>(nbatch) : 1;
     p->stride_a = str_a;
     p->stride_b = str_b;
+    p->stride_c = str_c;
+    // a batched matmul whose C's are not contiguous cannot use the flat split-K reduction
+    if (indep && str_c != d.M * d.N && ((d.flags >> NK_FLAG_SPLITK_SHIFT) & 0xFF) == 0)
+        p->d.flags |= 1u << NK_FLAG_SPLITK_SHIFT;
 
     DeviceGuard guard(d.device);
     if (guard.err != cudaSuccess) { delete p; return NK_ERR_DEVICE; }
@@ -514,7 +532,7 @@ nk_status_t nk_gemm_create(const nk_gemm_desc_t* desc, nk_gemm_t* out) {
     } else if (d.in_dtype == NK_F32 && d.M <= 32 && force != NK_FLAG_KERNEL_SIMT && nbatch == 1 && d.beta == 0) {
         p->variant = V_SKINNY;
         choose_skinny(p);
-        p->ws_partial_bytes = p->splits > 1 ? static_cast<size_t>(p->splits) * d.M * d.N * 4 : 0;
+        p->ws_partial_bytes = p->splits > 1 ? static_cast<size_t>(p->splits) * p->gemms * d.M * d.N * 4 : 0;
         p->launches = p->splits > 1 ? 2 : 1;
         snprintf(p->name, sizeof(p->name), "simt_f32_skinny_%dx512_kc%d_splitk%d", d.M <= 16 ? 16 : 32,
                  p->skinny_kc, p->splits);
@@ -522,7 +540,7 @@ nk_status_t nk_gemm_create(const nk_gemm_desc_t* desc, nk_gemm_t* out) {
         p->variant = V_SIMT;
         if (prepare_simt_attrs() != cudaSuccess) { cudaGetLastError(); delete p; return NK_ERR_CUDA; }
         choose_simt(p);
-        p->ws_partial_bytes = p->splits > 1 ? static_cast<size_t>(p->splits) * d.M * d.N * 4 : 0;
+        p->ws_partial_bytes = p->splits > 1 ? static_cast<size_t>(p->splits) * p->gemms * d.M * d.N * 4 : 0;
         p->launches = p->splits > 1 ? 2 : 1;
         snprintf(p->name, sizeof(p->name), "simt_f32_%dx%dx16_splitk%d", p->simt_tile, p->simt_tile, p->splits);
     } else {
@@ -551,16 +569,24 @@ nk_status_t nk_gemm_create(const nk_gemm_desc_t* desc, nk_gemm_t* out) {
             p->max_pairs = n;
         }
         p->ws_repack_bytes = p->b_repack ? align_up(static_cast<size_t>(d.K) * d.N * 2, 256) : 0;
-        p->ws_partial_bytes = p->splits > 1 ? static_cast<size_t>(p->splits) * d.M * d.N * 4 : 0;
+        p->ws_partial_bytes = p->splits > 1 ? static_cast<size_t>(p->splits) * p->gemms * d.M * d.N * 4 : 0;
         p->launches = 1 + (p->splits > 1 ? 1 : 0) + (p->b_repack ? 1 : 0);
         snprintf(p->name, sizeof(p->name), "umma_bf16_%s%dx64_s%d_splitk%d%s%s",
                  p->pair ? "pair_256x" : "128x", p->bn, p->stages,
                  p->splits, d.layout_a == NK_BLOCKED32 ? "_ablk" : "",
                  p->b_vnni_inkernel ? "_bvnni" : (p->b_repack ? "_brepack" : ""));
     }
-    if (p->batch > 1 || d.beta) {
+    if (p->batch > 1 || p->gemms > 1 || d.beta) {
         const size_t len = strlen(p->name);
-        snprintf(p->name + len, sizeof(p->name) - len, "_br%d%s", p->batch, d.beta ? "_beta1" : "");
+        if (p->gemms > 1) snprintf(p->name + len, sizeof(p->name) - len, "_bmm%d%s", p->gemms, d.beta ? "_beta1" : "");
+        else snprintf(p->name + len, sizeof(p->name) - len, "_br%d%s", p->batch, d.beta ? "_beta1" : "");
+    }
+    // split-K partials are laid out [split][gemm][M][N] and reduced as one flat array: that
+    // needs the C of a batched matmul to be contiguous
+    if (p->gemms > 1 && p->splits > 1 && p->stride_c != d.M * d.N) {
+        delete p;
+        *out = nullptr;
+        return NK_ERR_UNSUPPORTED;
     }
     *out = p;
     return NK_OK;
@@ -593,8 +619,8 @@ nk_status_t nk_gemm_run(nk_gemm_t p, const void* A, const void* B, const void* b
         NaiveParams np = {static_cast<int>(d.M), static_cast<int>(d.N), static_cast<int>(d.K),
                           d.in_dtype == NK_BF16, d.out_dtype == NK_BF16, d.layout_a == NK_BLOCKED32,
                           d.layout_b == NK_BLOCKED32, d.epilogue, p->batch, d.beta, p->stride_a, p->stride_b,
-                          A, B, bias, C};
-        dim3 grid(ceil_div(d.N, 128), static_cast<unsigned>(d.M));
+                          p->gemms, p->stride_c, A, B, bias, C};
+        dim3 grid(ceil_div(d.N, 128), static_cast<unsigned>(d.M), static_cast<unsigned>(p->gemms));
         if (d.M > 65535) return NK_ERR_UNSUPPORTED;
         naive_gemm_kernel<<<grid, 128, 0, st>>>(np);
         e = cudaGetLastError();
@@ -617,7 +643,7 @@ nk_status_t nk_gemm_run(nk_gemm_t p, const void* A, const void* B, const void* b
     } else if (p->variant == V_SIMT) {
         SimtParams sp = {static_cast<int>(d.M), static_cast<int>(d.N), static_cast<int>(d.K), p->splits,
                          p->kt_per_split, p->batch, ceil_div(d.K, SIMT_BK), p->stride_a, p->stride_b, d.beta,
-                         d.epilogue, static_cast<const float*>(A),
+                         p->gemms, p->stride_c, d.epilogue, static_cast<const float*>(A),
                          static_cast<const float*>(B), static_cast<const float*>(bias),
                          static_cast<float*>(C), partial};
         e = launch_simt(p, sp, st);
@@ -644,6 +670,8 @@ nk_status_t nk_gemm_run(nk_gemm_t p, const void* A, const void* B, const void* b
         up.kb_per_item = ceil_div(d.K, UMMA_BK);
         up.kb_total = p->batch * up.kb_per_item;
         up.beta = d.beta;
+        up.gemms = p->gemms;
+        up.stride_c = p->stride_c;
         up.kb_per_split = ceil_div(up.kb_total, p->splits);
         up.group_m = p->group_m;
         up.a_blocked = d.layout_a == NK_BLOCKED32;
@@ -656,7 +684,7 @@ nk_status_t nk_gemm_run(nk_gemm_t p, const void* A, const void* B, const void* b
         up.partial = partial;
         up.Bblk = p->b_vnni_inkernel ? static_cast<const uint32_t*>(B) : nullptr;
         up.status = p->status_dev;
-        const int units = up.tiles_m * up.tiles_n * up.splits;
+        const int units = up.gemms * up.tiles_m * up.tiles_n * up.splits;
         if (p->pair) {
             const int pairs = units < p->max_pairs ? units : p->max_pairs;
             e = launch_pair(p, up, pairs, st);
@@ -668,7 +696,7 @@ nk_status_t nk_gemm_run(nk_gemm_t p, const void* A, const void* B, const void* b
     }
 
     if (p->splits > 1) {
-        ReduceParams rp = {static_cast<size_t>(d.M) * d.N, static_cast<int>(d.N), p->splits, d.epilogue,
+        ReduceParams rp = {static_cast<size_t>(p->gemms) * d.M * d.N, static_cast<int>(d.N), p->splits, d.epilogue,
                            d.in_dtype == NK_BF16, d.out_dtype == NK_BF16, d.beta, partial, bias, C};
         const size_t quads = rp.MN / 4;
         splitk_reduce_kernel<<<static_cast<unsigned>((quads + 255) / 256), 256, 0, st>>>(rp);
@@ -689,9 +717,11 @@ nk_status_t nk_gemm_run_host(nk_gemm_t p, const void* hA, const void* hB, const 
     DeviceGuard guard(d.device);
     if (guard.err != cudaSuccess) { set_err(p, "cudaSetDevice", guard.err); return NK_ERR_DEVICE; }
     cudaError_t e;
-    const size_t a_elems = static_cast<size_t>(p->batch - 1) * p->stride_a + static_cast<size_t>(d.M) * d.K;
-    const size_t b_elems = static_cast<size_t>(p->batch - 1) * p->stride_b + static_cast<size_t>(d.K) * d.N;
-    if (d.beta && (e = cudaMemcpyAsync(dC, hC, eout * d.M * d.N, cudaMemcpyHostToDevice, st)) != cudaSuccess) {
+    const size_t items = static_cast<size_t>(p->batch) * p->gemms;
+    const size_t a_elems = (items - 1) * p->stride_a + static_cast<size_t>(d.M) * d.K;
+    const size_t b_elems = (items - 1) * p->stride_b + static_cast<size_t>(d.K) * d.N;
+    const size_t c_elems = static_cast<size_t>(p->gemms - 1) * p->stride_c + static_cast<size_t>(d.M) * d.N;
+    if (d.beta && (e = cudaMemcpyAsync(dC, hC, eout * c_elems, cudaMemcpyHostToDevice, st)) != cudaSuccess) {
         set_err(p, "H2D copy", e);
         return NK_ERR_CUDA;
     }
@@ -708,7 +738,7 @@ nk_status_t nk_gemm_run_host(nk_gemm_t p, const void* hA, const void* hB, const 
     nk_status_t s = nk_gemm_run(p, dA, dB, d.epilogue != NK_EPI_NONE ? dbias : nullptr, dC, workspace,
                                 workspace_bytes, cuda_stream);
     if (s != NK_OK) return s;
-    if ((e = cudaMemcpyAsync(hC, dC, eout * d.M * d.N, cudaMemcpyDeviceToHost, st)) != cudaSuccess ||
+    if ((e = cudaMemcpyAsync(hC, dC, eout * c_elems, cudaMemcpyDeviceToHost, st)) != cudaSuccess ||
         (e = cudaStreamSynchronize(st)) != cudaSuccess) {
         set_err(p, "D2H copy / sync", e);
         return NK_ERR_CUDA;

@@ -22,6 +22,8 @@ struct SimtParams {
     int kt_per_item;   // ceil(K / 16): k-tiles of one pair
     long long stride_a, stride_b;  // elements between consecutive A_b / B_b
     int beta;          // 1: the old C is added before the epilogue
+    int gemms;         // independent GEMMs in one launch (batched matmul), else 1; gridDim.z = splits * gemms
+    long long stride_c;  // elements from C_g to C_g+1
     int epilogue;      // 0 none, 1 bias + ReLU
     const float* A;    // [M][K]
     const float* B;    // [K][N]
@@ -51,7 +53,8 @@ simt_f32_kernel(const SimtParams p) {
     const int ty = t / TX, tx = t % TX;
     const int m0 = blockIdx.y * BM, n0 = blockIdx.x * BN;
     const int ktiles = p.batch * p.kt_per_item;   // k-tiles of the whole batch-reduce
-    const int kt0 = blockIdx.z * p.kt_per_split;
+    const int gemm = blockIdx.z / p.splits, split = blockIdx.z - gemm * p.splits;
+    const int kt0 = split * p.kt_per_split;
     const int kt1 = min(ktiles, kt0 + p.kt_per_split);
 
     float acc[TM][TN];
@@ -63,8 +66,9 @@ simt_f32_kernel(const SimtParams p) {
     float4 ra[A_V4], rb[B_V4];
 
     auto load_global = [&](int kt) {
-        const int item = kt / p.kt_per_item;               // which (A_b, B_b) pair
-        const int k0 = (kt - item * p.kt_per_item) * SIMT_BK;
+        const int item_l = kt / p.kt_per_item;             // which (A_b, B_b) pair of the reduction
+        const int item = gemm + item_l;                    // (+ this GEMM's own pair in a batched matmul)
+        const int k0 = (kt - item_l * p.kt_per_item) * SIMT_BK;
         const float* Ab = p.A + item * p.stride_a;
         const float* Bb = p.B + item * p.stride_b;
 #pragma unroll
@@ -145,7 +149,8 @@ simt_f32_kernel(const SimtParams p) {
 
     // Epilogue: bias + ReLU on the accumulator, then the single store of C.
     const bool to_partial = p.splits > 1;
-    float* out = to_partial ? p.partial + static_cast<size_t>(blockIdx.z) * p.M * p.N : p.C;
+    float* out = to_partial ? p.partial + (static_cast<size_t>(split) * p.gemms + gemm) * p.M * p.N
+                            : p.C + gemm * p.stride_c;
 #pragma unroll
     for (int gi = 0; gi < GM; ++gi)
 #pragma unroll
@@ -319,7 +324,8 @@ simt_f32_async_kernel(const SimtParams p) {
     const int ty = t / TX, tx = t % TX;
     const int m0 = blockIdx.y * BM, n0 = blockIdx.x * BN;
     const int ktiles = p.batch * p.kt_per_item;   // k-tiles of the whole batch-reduce
-    const int kt0 = blockIdx.z * p.kt_per_split;
+    const int gemm = blockIdx.z / p.splits, split = blockIdx.z - gemm * p.splits;
+    const int kt0 = split * p.kt_per_split;
     const int kt1 = min(ktiles, kt0 + p.kt_per_split);
 
     float acc[TM][TN];
@@ -330,8 +336,9 @@ simt_f32_async_kernel(const SimtParams p) {
 
     auto issue_tile = [&](int kt, int stage) {
         if (kt < kt1) {
-            const int item = kt / p.kt_per_item;
-            const int k0 = (kt - item * p.kt_per_item) * SIMT_BK;
+            const int item_l = kt / p.kt_per_item;
+            const int item = gemm + item_l;
+            const int k0 = (kt - item_l * p.kt_per_item) * SIMT_BK;
             const float* Ab = p.A + item * p.stride_a;
             const float* Bb = p.B + item * p.stride_b;
 #pragma unroll
@@ -389,7 +396,8 @@ simt_f32_async_kernel(const SimtParams p) {
     cp_async_wait_group<0>();
 
     const bool to_partial = p.splits > 1;
-    float* out = to_partial ? p.partial + static_cast<size_t>(blockIdx.z) * p.M * p.N : p.C;
+    float* out = to_partial ? p.partial + (static_cast<size_t>(split) * p.gemms + gemm) * p.M * p.N
+                            : p.C + gemm * p.stride_c;
 #pragma unroll
     for (int gi = 0; gi < GM; ++gi)
 #pragma unroll

@@ -39,6 +39,8 @@ struct UmmaParams {
     int kb_total;       // batch * kb_per_item: k-blocks of the whole reduction
     int kb_per_item;    // ceil(K / 64): k-blocks of one (A_b, B_b) pair of the batch-reduce
     int beta;           // 1: the old C is added before the epilogue (Algorithm 1's beta.C)
+    int gemms;          // independent GEMMs in one launch (batched matmul): C_g = A_g . B_g; else 1
+    long long stride_c; // elements from C_g to C_g+1
     int kb_per_split;   // ceil(kb_total / splits)
     int group_m;        // raster: this many M tiles sweep N together
     int a_blocked;      // A tensor map is the 4-D blocked view
@@ -74,6 +76,15 @@ __device__ __forceinline__ void umma_tile_coords(const UmmaParams& p, int tile, 
     nb = within / gm;
 }
 
+// unit id -> (independent GEMM, tile, K split)
+__device__ __forceinline__ void umma_decode_unit(const UmmaParams& p, int unit, int& tile, int& split, int& gemm) {
+    const int per_gemm = p.tiles_m * p.tiles_n * p.splits;
+    gemm = unit / per_gemm;
+    const int u = unit - gemm * per_gemm;
+    tile = u / p.splits;
+    split = u - tile * p.splits;
+}
+
 __device__ __forceinline__ float bf16_bits_to_f32(uint32_t h) { return __uint_as_float(h << 16); }
 
 __device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi) {
@@ -89,9 +100,10 @@ __device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi) {
 // writes four whole 128-byte row segments instead of 32 scattered 16-byte pieces.  BF16 rows
 // (64 bytes each) are stored directly.  Columns are predicated in groups (N is a multiple of 8).
 __device__ __forceinline__ void umma_store_chunk(const UmmaParams& p, uint32_t (&v)[32], int row0, int lane,
-                                                 int col0, int split, bool empty_k, uint8_t* staging) {
+                                                 int col0, int split, int gemm, bool empty_k, uint8_t* staging) {
     if (col0 >= p.N || row0 >= p.M) return;           // warp-uniform
     const int row = row0 + lane;
+    const size_t c_base = static_cast<size_t>(gemm) * p.stride_c;   // this GEMM's C inside the batch
     if (empty_k) {
 #pragma unroll
         for (int i = 0; i < 32; ++i) v[i] = 0u;
@@ -101,7 +113,7 @@ __device__ __forceinline__ void umma_store_chunk(const UmmaParams& p, uint32_t (
         // beta = 1: the accumulation tile starts from the stored C (Algorithm 1 loads the C
         // sub-block before the K loop; adding it here, in FP32, gives the same sum)
         if (p.out_bf16) {
-            const uint4* csrc = reinterpret_cast<const uint4*>(static_cast<const uint16_t*>(p.C) +
+            const uint4* csrc = reinterpret_cast<const uint4*>(static_cast<const uint16_t*>(p.C) + c_base +
                                                                static_cast<size_t>(row) * p.N + col0);
 #pragma unroll
             for (int g = 0; g < 4; ++g) {
@@ -115,7 +127,7 @@ __device__ __forceinline__ void umma_store_chunk(const UmmaParams& p, uint32_t (
                 }
             }
         } else {
-            const uint4* csrc = reinterpret_cast<const uint4*>(static_cast<const float*>(p.C) +
+            const uint4* csrc = reinterpret_cast<const uint4*>(static_cast<const float*>(p.C) + c_base +
                                                                static_cast<size_t>(row) * p.N + col0);
 #pragma unroll
             for (int g = 0; g < 8; ++g) {
@@ -146,7 +158,7 @@ __device__ __forceinline__ void umma_store_chunk(const UmmaParams& p, uint32_t (
     }
     if (!to_partial && p.out_bf16) {
         if (row >= p.M) return;
-        uint16_t* dst = static_cast<uint16_t*>(p.C) + static_cast<size_t>(row) * p.N + col0;
+        uint16_t* dst = static_cast<uint16_t*>(p.C) + c_base + static_cast<size_t>(row) * p.N + col0;
 #pragma unroll
         for (int g = 0; g < 4; ++g)
             if (col0 + 8 * g < p.N) {
@@ -165,7 +177,8 @@ __device__ __forceinline__ void umma_store_chunk(const UmmaParams& p, uint32_t (
         *reinterpret_cast<uint4*>(staging + lane * 128 + ((g ^ (lane & 7)) << 4)) =
             make_uint4(v[4 * g], v[4 * g + 1], v[4 * g + 2], v[4 * g + 3]);
     __syncwarp();
-    float* out = to_partial ? p.partial + static_cast<size_t>(split) * p.M * p.N : static_cast<float*>(p.C);
+    float* out = to_partial ? p.partial + (static_cast<size_t>(split) * p.gemms + gemm) * p.M * p.N
+                            : static_cast<float*>(p.C) + c_base;
     const int c = lane & 7, rsub = lane >> 3;
     const bool col_ok = col0 + 4 * c < p.N;
 #pragma unroll
@@ -273,7 +286,7 @@ umma_bf16_kernel(const __grid_constant__ CUtensorMap tmap_a,
     tc_fence_after_sync();
     const uint32_t tmem_base = *tmem_slot;
 
-    const int total_units = p.tiles_m * p.tiles_n * p.splits;
+    const int total_units = p.gemms * p.tiles_m * p.tiles_n * p.splits;
 
     auto give_up = [&](unsigned int code) {
         *abort_flag = 1;
@@ -291,7 +304,8 @@ umma_bf16_kernel(const __grid_constant__ CUtensorMap tmap_a,
         uint32_t sa = smem_base, fb = full_bar(0);
         bool ok = true;
         for (int unit = blockIdx.x; ok && unit < total_units; unit += gridDim.x) {
-            const int tile = unit / p.splits, split = unit - tile * p.splits;
+            int tile, split, gemm;
+            umma_decode_unit(p, unit, tile, split, gemm);
             int mb, nb;
             umma_tile_coords(p, tile, mb, nb);
             const int kb0 = split * p.kb_per_split;
@@ -300,6 +314,7 @@ umma_bf16_kernel(const __grid_constant__ CUtensorMap tmap_a,
             // k-block kb of the reduction = k-block (kb % kb_per_item) of batch item kb / kb_per_item
             int item = kb0 / p.kb_per_item;
             int kbl = kb0 - item * p.kb_per_item;
+            item += gemm;   // independent batch: the unit's own (A, B) pair
             for (int kb = kb0; kb < kb1; ++kb) {
                 const int kx = kbl * UMMA_BK;
                 if (!mbar_wait(empty_bar(stage), phase ^ 1u, abort_flag)) {
@@ -369,7 +384,8 @@ umma_bf16_kernel(const __grid_constant__ CUtensorMap tmap_a,
         int local = 0;
         bool ok = true;
         for (int unit = blockIdx.x; ok && unit < total_units; unit += gridDim.x, ++local) {
-            const int tile = unit / p.splits, split = unit - tile * p.splits;
+            int tile, split, gemm;
+            umma_decode_unit(p, unit, tile, split, gemm);
             const int kb0 = split * p.kb_per_split;
             const int kb1 = min(p.kb_total, kb0 + p.kb_per_split);
             const int acc = local & 1;
@@ -411,7 +427,8 @@ umma_bf16_kernel(const __grid_constant__ CUtensorMap tmap_a,
         int local = 0;
         bool ok = true;
         for (int unit = blockIdx.x; ok && unit < total_units; unit += gridDim.x, ++local) {
-            const int tile = unit / p.splits, split = unit - tile * p.splits;
+            int tile, split, gemm;
+            umma_decode_unit(p, unit, tile, split, gemm);
             int mb, nb;
             umma_tile_coords(p, tile, mb, nb);
             const int kb0 = split * p.kb_per_split;
@@ -432,7 +449,7 @@ umma_bf16_kernel(const __grid_constant__ CUtensorMap tmap_a,
                 tmem_ld_32x32(tmem_base + acc * BN + c0 + (static_cast<uint32_t>(quarter * 32) << 16),
                               v);
                 tmem_ld_wait();
-                umma_store_chunk(p, v, row0, lane, nb * BN + c0, split, empty_k, staging);
+                umma_store_chunk(p, v, row0, lane, nb * BN + c0, split, gemm, empty_k, staging);
                 __syncwarp();
             }
             tc_fence_before_sync();
@@ -446,7 +463,8 @@ umma_bf16_kernel(const __grid_constant__ CUtensorMap tmap_a,
         uint32_t phase = 0;
         bool ok = true;
         for (int unit = blockIdx.x; ok && unit < total_units; unit += gridDim.x) {
-            const int tile = unit / p.splits, split = unit - tile * p.splits;
+            int tile, split, gemm;
+            umma_decode_unit(p, unit, tile, split, gemm);
             int mb, nb;
             umma_tile_coords(p, tile, mb, nb);
             const int kb0 = split * p.kb_per_split;

@@ -81,7 +81,7 @@ umma_bf16_pair_kernel(const __grid_constant__ CUtensorMap tmap_a,
     tc_fence_after_sync();
     const uint32_t tmem_base = *tmem_slot;
 
-    const int total_units = p.tiles_m * p.tiles_n * p.splits;
+    const int total_units = p.gemms * p.tiles_m * p.tiles_n * p.splits;
     auto give_up = [&](unsigned int code) {
         *abort_flag = 1;
         if (p.status) atomicCAS(p.status, 0u, code);
@@ -97,7 +97,8 @@ umma_bf16_pair_kernel(const __grid_constant__ CUtensorMap tmap_a,
         uint32_t sa = smem_base, fb = full_bar(0), lfb = lead_full0;
         bool ok = true;
         for (int unit = pair_id; ok && unit < total_units; unit += num_pairs) {
-            const int tile = unit / p.splits, split = unit - tile * p.splits;
+            int tile, split, gemm;
+            umma_decode_unit(p, unit, tile, split, gemm);
             int mb, nb;
             umma_tile_coords(p, tile, mb, nb);
             const int kb0 = split * p.kb_per_split;
@@ -106,6 +107,7 @@ umma_bf16_pair_kernel(const __grid_constant__ CUtensorMap tmap_a,
             const int col0 = nb * BN + static_cast<int>(rank) * HALF;
             int item = kb0 / p.kb_per_item;
             int kbl = kb0 - item * p.kb_per_item;
+            item += gemm;   // independent batch: the unit's own (A, B) pair
             for (int kb = kb0; kb < kb1; ++kb) {
                 const int kx = kbl * UMMA_BK;
                 if (!mbar_wait(empty_bar(stage), phase ^ 1u, abort_flag)) {
@@ -168,7 +170,8 @@ umma_bf16_pair_kernel(const __grid_constant__ CUtensorMap tmap_a,
             int local = 0;
             bool ok = true;
             for (int unit = pair_id; ok && unit < total_units; unit += num_pairs, ++local) {
-                const int tile = unit / p.splits, split = unit - tile * p.splits;
+                int tile, split, gemm;
+            umma_decode_unit(p, unit, tile, split, gemm);
                 const int kb0 = split * p.kb_per_split;
                 const int kb1 = min(p.kb_total, kb0 + p.kb_per_split);
                 const int acc = local & 1;
@@ -211,7 +214,8 @@ umma_bf16_pair_kernel(const __grid_constant__ CUtensorMap tmap_a,
         int local = 0;
         bool ok = true;
         for (int unit = pair_id; ok && unit < total_units; unit += num_pairs, ++local) {
-            const int tile = unit / p.splits, split = unit - tile * p.splits;
+            int tile, split, gemm;
+            umma_decode_unit(p, unit, tile, split, gemm);
             int mb, nb;
             umma_tile_coords(p, tile, mb, nb);
             const int kb0 = split * p.kb_per_split;
@@ -231,7 +235,7 @@ umma_bf16_pair_kernel(const __grid_constant__ CUtensorMap tmap_a,
                 uint32_t v[32];
                 tmem_ld_32x32(tmem_base + acc * BN + c0 + (static_cast<uint32_t>(quarter * 32) << 16), v);
                 tmem_ld_wait();
-                umma_store_chunk(p, v, row0, lane, nb * BN + c0, split, empty_k, staging);
+                umma_store_chunk(p, v, row0, lane, nb * BN + c0, split, gemm, empty_k, staging);
                 __syncwarp();
             }
             tc_fence_before_sync();
@@ -248,7 +252,8 @@ umma_bf16_pair_kernel(const __grid_constant__ CUtensorMap tmap_a,
         uint32_t phase = 0;
         bool ok = true;
         for (int unit = pair_id; ok && unit < total_units; unit += num_pairs) {
-            const int tile = unit / p.splits, split = unit - tile * p.splits;
+            int tile, split, gemm;
+            umma_decode_unit(p, unit, tile, split, gemm);
             int mb, nb;
             umma_tile_coords(p, tile, mb, nb);
             const int kb0 = split * p.kb_per_split;

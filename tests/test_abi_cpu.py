@@ -74,7 +74,7 @@ def test_null_arguments():
     L = nk.lib()
     h = ctypes.c_void_p()
     assert L.nk_gemm_create(None, ctypes.byref(h)) == 1
-    assert L.nk_gemm_create(ctypes.byref(binding.Desc(8, 8, 8, 0, 0, 0, 0, 0, 0, 0, 0, 0, 0, 0)), None) == 1
+    assert L.nk_gemm_create(ctypes.byref(binding.Desc(8, 8, 8, 0, 0, 0, 0, 0, 0, 0, 0, 0, 0, 0, 0, 0)), None) == 1
     assert L.nk_gemm_destroy(None) == 0
     assert L.nk_gemm_workspace_bytes(None) == 0
     assert L.nk_gemm_run(None, None, None, None, None, None, 0, None) == 1

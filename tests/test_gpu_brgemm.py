@@ -78,3 +78,63 @@ def test_brgemm_naive_cross_check():
 def test_beta_one_plain_gemm_auto():
     _run(512, 512, 1024, 1, "bf16", "f32", False, 1, integer=False, seed=5)
     _run(16, 1024, 512, 1, "f32", "f32", False, 1)          # M <= 32 with beta goes to the tiled kernel
+
+
+# ---------------------------------------------------------------- batched matmul: C_g = A_g . B_g
+def _run_bmm(M, N, K, gemms, dt, out_dt, epi, beta, pad_a=0, pad_b=0, pad_c=0, flags=0, integer=True, seed=2):
+    sa, sb, sc = M * K + pad_a, K * N + pad_b, M * N + pad_c
+    dist = "int" if integer else "uniform"
+    A = nk_inputs.fill(seed, nk_inputs.TENSOR_A, (gemms - 1) * sa + M * K, dist, dtype=dt)
+    B = nk_inputs.fill(seed, nk_inputs.TENSOR_B, (gemms - 1) * sb + K * N, dist, dtype=dt)
+    bias = nk_inputs.fill(seed, nk_inputs.TENSOR_BIAS, N, dist, dtype=dt) if epi else None
+    C0 = nk_inputs.fill(seed, 5, (gemms - 1) * sc + M * N, dist, dtype=out_dt)
+    plan = nk.Plan(M, N, K, nk.BF16 if dt == "bf16" else nk.F32, nk.BF16 if out_dt == "bf16" else nk.F32,
+                   epilogue=nk.EPI_BIAS_RELU if epi else nk.EPI_NONE, flags=flags, beta=beta, batch=gemms,
+                   stride_a=sa if pad_a else 0, stride_b=sb if pad_b else 0, stride_c=sc if pad_c else 0,
+                   batch_independent=1)
+    assert f"_bmm{gemms}" in plan.kernel_name
+    dA, dB = to_device(A), to_device(B)
+    dbias = to_device(bias) if epi else None
+    dC = to_device(C0).clone()
+    ws = torch.empty(max(plan.workspace_bytes, 16), dtype=torch.uint8, device="cuda")
+    plan.run(dA, dB, dC, bias=dbias, workspace=ws if plan.workspace_bytes else None,
+             workspace_bytes=plan.workspace_bytes, stream=torch.cuda.current_stream().cuda_stream)
+    plan.check()
+    got = c_to_f64(dC)
+    c0 = ((C0.astype(np.uint32) << 16).view(np.float32) if out_dt == "bf16" else C0).astype(np.float64)
+    for g in range(gemms):
+        Y, S = oracle.brgemm(M, N, K, 1, A[g * sa:g * sa + M * K], B[g * sb:g * sb + K * N], bias,
+                             C0=c0[g * sc:g * sc + M * N].reshape(M, N) if beta else None,
+                             in_dtype=oracle.BF16 if dt == "bf16" else oracle.F32,
+                             epilogue=oracle.EPI_BIAS_RELU if epi else oracle.EPI_NONE, beta=float(beta))
+        gg = got[g * sc:g * sc + M * N].reshape(M, N)
+        if integer and out_dt == "f32":
+            assert np.array_equal(gg, Y), (plan.kernel_name, g)
+        else:
+            tol = TOL_REL_SMAX * S.max() + (TOL_BF16_REL * np.abs(Y) if out_dt == "bf16" else 0.0)
+            assert np.all(np.abs(gg - Y) <= tol), (plan.kernel_name, g)
+    if pad_c:   # the gaps between the C's are untouched
+        for g in range(gemms - 1):
+            assert np.array_equal(got[g * sc + M * N:(g + 1) * sc], c0[g * sc + M * N:(g + 1) * sc])
+    return plan
+
+
+@pytest.mark.parametrize("mode", ["single", "pair"])
+@pytest.mark.parametrize("beta", [0, 1])
+def test_batched_matmul_bf16(mode, beta):
+    f = nk.FLAG_SINGLE_CTA if mode == "single" else nk.FLAG_CTA_PAIR
+    _run_bmm(200, 136, 72, 5, "bf16", "f32", False, beta, pad_a=8, pad_b=16, pad_c=12, flags=f)
+    _run_bmm(130, 256, 192, 3, "bf16", "bf16", True, beta, flags=f | nk.flag_splitk(3), integer=False)
+
+
+@pytest.mark.parametrize("beta", [0, 1])
+@pytest.mark.parametrize("tile", [1, 2, 3])
+def test_batched_matmul_f32(beta, tile):
+    _run_bmm(70, 132, 52, 4, "f32", "f32", True, beta, pad_a=4, pad_c=8, flags=nk.FLAG_KERNEL_SIMT | nk.flag_tile_n(tile))
+    _run_bmm(64, 64, 256, 6, "f32", "f32", False, beta, flags=nk.flag_tile_n(tile) | nk.flag_splitk(2), integer=False)
+
+
+def test_batched_matmul_auto_and_naive():
+    _run_bmm(256, 256, 256, 16, "bf16", "f32", False, 0, integer=False)
+    _run_bmm(24, 40, 16, 3, "f32", "f32", True, 1, pad_c=4, flags=nk.FLAG_KERNEL_NAIVE)
+    _run_bmm(16, 64, 64, 4, "f32", "f32", False, 0)      # small M, batched: tiled kernel, not the streaming one
