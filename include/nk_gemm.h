@@ -20,7 +20,8 @@
  *                  B[N/32][K/32][16][32][2]              (n-block, k-block, k/2, n, k%2):
  *                  every 32x32 block of B is VNNI-2 packed as in Figure 1,
  *                  packed[k/2][n][k%2] = flat[k][n]; BF16 only.
- * C is row-major [M][N] in every case; bias is [N] in the operand type.
+ * C is row-major [M][N] unless desc.layout_c asks for the blocked form; bias is [N] in the
+ * operand type.
  *
  * All data pointers are DEVICE pointers on the plan's device unless a function
  * says otherwise.  The library never allocates or frees device memory, never
@@ -86,6 +87,9 @@ typedef struct {
     int64_t stride_c;  /* elements from C_b to C_b+1; 0 means M*N                       */
     int32_t batch_independent; /* 0: the batch is reduced into one C; 1: C_b = A_b . B_b for
                                   every b (bias shared; beta applies to each C_b)        */
+    int32_t layout_c;  /* nk_layout_t of C: NK_ROW_MAJOR, or NK_BLOCKED32 = C[M/32][N/32][32][32],
+                          the layout a following layer reads as its blocked A (BF16 operands;
+                          M and N multiples of 32)                                        */
 } nk_gemm_desc_t;
 
 /*
@@ -95,10 +99,11 @@ typedef struct {
  * state.  Requirements: M, N, K > 0; blocked layouts need BF16 and the blocked
  * operand's two dimensions to be multiples of 32; row-major BF16 needs N and K
  * to be multiples of 8, row-major FP32 needs N and K to be multiples of 4
- * (16-byte rows); BF16 output needs BF16 inputs.  batch > 1 and beta = 1 (Section 2.1:
- * the source tiles of a batch-reduce GEMM need not be contiguous, the accumulation tile is
- * C) need row-major operands and strides that are multiples of 8 (BF16) or 4 (FP32)
- * elements; with beta = 1, y = epilogue(C_old + sum_b A_b.B_b).  On failure *out is NULL.
+ * (16-byte rows); BF16 output needs BF16 inputs.  batch > 1 (Section 2.1: the source tiles
+ * of a batch-reduce GEMM need not be contiguous, the accumulation tile is C) needs
+ * row-major operands and strides that are multiples of 8 (BF16) or 4 (FP32) elements; with
+ * beta = 1, y = epilogue(C_old + sum_b A_b.B_b), C_old read in C's own layout.  A blocked C
+ * needs BF16 operands and M, N multiples of 32.  On failure *out is NULL.
  */
 nk_status_t nk_gemm_create(const nk_gemm_desc_t* desc, nk_gemm_t* out);
 

@@ -47,7 +47,7 @@ class Desc(ctypes.Structure):
                 ("epilogue", ctypes.c_int32), ("device", ctypes.c_int32),
                 ("flags", ctypes.c_uint32), ("beta", ctypes.c_int32), ("batch", ctypes.c_int64),
                 ("stride_a", ctypes.c_int64), ("stride_b", ctypes.c_int64), ("stride_c", ctypes.c_int64),
-                ("batch_independent", ctypes.c_int32)]
+                ("batch_independent", ctypes.c_int32), ("layout_c", ctypes.c_int32)]
 
 
 _lib = None
@@ -124,9 +124,10 @@ class Plan:
 
     def __init__(self, M, N, K, in_dtype=BF16, out_dtype=F32, layout_a=ROW_MAJOR,
                  layout_b=ROW_MAJOR, epilogue=EPI_NONE, device=0, flags=0, beta=0, batch=0,
-                 stride_a=0, stride_b=0, stride_c=0, batch_independent=0):
+                 stride_a=0, stride_b=0, stride_c=0, batch_independent=0,
+                 layout_c=ROW_MAJOR):
         self.desc = Desc(M, N, K, in_dtype, out_dtype, layout_a, layout_b, epilogue, device, flags,
-                         beta, batch, stride_a, stride_b, stride_c, batch_independent)
+                         beta, batch, stride_a, stride_b, stride_c, batch_independent, layout_c)
         self._h = ctypes.c_void_p()
         _check(lib().nk_gemm_create(ctypes.byref(self.desc), ctypes.byref(self._h)))
 

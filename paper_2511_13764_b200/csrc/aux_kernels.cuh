@@ -17,6 +17,7 @@ struct NaiveParams {
     long long stride_a, stride_b;
     int gemms;             // batched matmul: gridDim.z independent GEMMs
     long long stride_c;
+    int c_blocked;         // C stored as [M/32][N/32][32][32]
     const void *A, *B, *bias;
     void* C;
 };
@@ -34,7 +35,9 @@ __global__ void naive_gemm_kernel(const NaiveParams p) {
     if (j >= p.N || i >= p.M) return;
     const size_t kb32 = p.K / 32;
     const int g = blockIdx.z;
-    const size_t o = static_cast<size_t>(g) * p.stride_c + static_cast<size_t>(i) * p.N + j;
+    const size_t o = static_cast<size_t>(g) * p.stride_c +
+                     (p.c_blocked ? ((static_cast<size_t>(i / 32) * (p.N / 32) + j / 32) * 32 + i % 32) * 32 + j % 32
+                                  : static_cast<size_t>(i) * p.N + j);
     float acc = 0.f;
     if (p.beta) acc = ld_elem(p.C, p.out_bf16, o);
     for (int b = 0; b < p.batch; ++b)
@@ -60,6 +63,8 @@ struct ReduceParams {
     int splits;
     int epilogue, bias_bf16, out_bf16;
     int beta;              // 1: add the old C before the epilogue
+    int c_blocked;         // C stored as [M/32][N/32][32][32] (per GEMM of M_rows rows)
+    int M;                 // rows of one GEMM
     const float* partial;  // [splits][M][N]
     const void* bias;
     void* C;
@@ -71,6 +76,14 @@ __global__ void splitk_reduce_kernel(const ReduceParams p) {
     const size_t q = static_cast<size_t>(blockIdx.x) * blockDim.x + threadIdx.x;
     const size_t e = q * 4;
     if (e >= p.MN) return;
+    // where the four elements live in C: same index, or inside their 32 x 32 block
+    size_t ce = e;
+    if (p.c_blocked) {
+        const size_t per = static_cast<size_t>(p.M) * p.N;
+        const size_t g = e / per, r = e - g * per;
+        const size_t i = r / p.N, j = r - i * p.N;
+        ce = g * per + ((i / 32 * (p.N / 32) + j / 32) * 32 + i % 32) * 32 + j % 32;
+    }
     float4 s = __ldcs(reinterpret_cast<const float4*>(p.partial + e));
     for (int sp = 1; sp < p.splits; ++sp) {
         const float4 v = __ldcs(reinterpret_cast<const float4*>(p.partial + sp * p.MN + e));
@@ -78,11 +91,11 @@ __global__ void splitk_reduce_kernel(const ReduceParams p) {
     }
     if (p.beta) {
         if (p.out_bf16) {
-            const uint2 w = *reinterpret_cast<const uint2*>(static_cast<const uint16_t*>(p.C) + e);
+            const uint2 w = *reinterpret_cast<const uint2*>(static_cast<const uint16_t*>(p.C) + ce);
             s.x += __uint_as_float(w.x << 16); s.y += __uint_as_float(w.x & 0xFFFF0000u);
             s.z += __uint_as_float(w.y << 16); s.w += __uint_as_float(w.y & 0xFFFF0000u);
         } else {
-            const float4 c = *reinterpret_cast<const float4*>(static_cast<const float*>(p.C) + e);
+            const float4 c = *reinterpret_cast<const float4*>(static_cast<const float*>(p.C) + ce);
             s.x += c.x; s.y += c.y; s.z += c.z; s.w += c.w;
         }
     }
@@ -105,9 +118,9 @@ __global__ void splitk_reduce_kernel(const ReduceParams p) {
         uint2 o;
         o.x = *reinterpret_cast<uint32_t*>(&lo);
         o.y = *reinterpret_cast<uint32_t*>(&hi);
-        *reinterpret_cast<uint2*>(static_cast<uint16_t*>(p.C) + e) = o;
+        *reinterpret_cast<uint2*>(static_cast<uint16_t*>(p.C) + ce) = o;
     } else {
-        *reinterpret_cast<float4*>(static_cast<float*>(p.C) + e) = s;
+        *reinterpret_cast<float4*>(static_cast<float*>(p.C) + ce) = s;
     }
 }
 

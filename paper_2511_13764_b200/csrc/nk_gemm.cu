@@ -475,7 +475,11 @@ nk_status_t nk_gemm_create(const nk_gemm_desc_t* desc, nk_gemm_t* out) {
         if (str_a % gran || str_b % gran) return NK_ERR_MISALIGNED;
         if (str_a < d.M * d.K || str_b < d.K * d.N) return NK_ERR_INVALID_ARG;   // items must not overlap
     }
-    if (d.beta == 1 && blocked) return NK_ERR_UNSUPPORTED;
+    if (d.layout_c != NK_ROW_MAJOR && d.layout_c != NK_BLOCKED32) return NK_ERR_INVALID_ARG;
+    if (d.layout_c == NK_BLOCKED32) {
+        if (d.in_dtype != NK_BF16) return NK_ERR_UNSUPPORTED;
+        if (d.M % 32 || d.N % 32) return NK_ERR_MISALIGNED;
+    }
     if (d.batch_independent != 0 && d.batch_independent != 1) return NK_ERR_INVALID_ARG;
     if (d.stride_c < 0) return NK_ERR_INVALID_ARG;
     const int64_t str_c = d.stride_c > 0 ? d.stride_c : d.M * d.N;
@@ -581,6 +585,10 @@ nk_status_t nk_gemm_create(const nk_gemm_desc_t* desc, nk_gemm_t* out) {
         if (p->gemms > 1) snprintf(p->name + len, sizeof(p->name) - len, "_bmm%d%s", p->gemms, d.beta ? "_beta1" : "");
         else snprintf(p->name + len, sizeof(p->name) - len, "_br%d%s", p->batch, d.beta ? "_beta1" : "");
     }
+    if (d.layout_c == NK_BLOCKED32) {
+        const size_t len = strlen(p->name);
+        snprintf(p->name + len, sizeof(p->name) - len, "_cblk");
+    }
     // split-K partials are laid out [split][gemm][M][N] and reduced as one flat array: that
     // needs the C of a batched matmul to be contiguous
     if (p->gemms > 1 && p->splits > 1 && p->stride_c != d.M * d.N) {
@@ -619,7 +627,7 @@ nk_status_t nk_gemm_run(nk_gemm_t p, const void* A, const void* B, const void* b
         NaiveParams np = {static_cast<int>(d.M), static_cast<int>(d.N), static_cast<int>(d.K),
                           d.in_dtype == NK_BF16, d.out_dtype == NK_BF16, d.layout_a == NK_BLOCKED32,
                           d.layout_b == NK_BLOCKED32, d.epilogue, p->batch, d.beta, p->stride_a, p->stride_b,
-                          p->gemms, p->stride_c, A, B, bias, C};
+                          p->gemms, p->stride_c, d.layout_c == NK_BLOCKED32, A, B, bias, C};
         dim3 grid(ceil_div(d.N, 128), static_cast<unsigned>(d.M), static_cast<unsigned>(p->gemms));
         if (d.M > 65535) return NK_ERR_UNSUPPORTED;
         naive_gemm_kernel<<<grid, 128, 0, st>>>(np);
@@ -672,6 +680,7 @@ nk_status_t nk_gemm_run(nk_gemm_t p, const void* A, const void* B, const void* b
         up.beta = d.beta;
         up.gemms = p->gemms;
         up.stride_c = p->stride_c;
+        up.c_blocked = d.layout_c == NK_BLOCKED32;
         up.kb_per_split = ceil_div(up.kb_total, p->splits);
         up.group_m = p->group_m;
         up.a_blocked = d.layout_a == NK_BLOCKED32;
@@ -697,7 +706,8 @@ nk_status_t nk_gemm_run(nk_gemm_t p, const void* A, const void* B, const void* b
 
     if (p->splits > 1) {
         ReduceParams rp = {static_cast<size_t>(p->gemms) * d.M * d.N, static_cast<int>(d.N), p->splits, d.epilogue,
-                           d.in_dtype == NK_BF16, d.out_dtype == NK_BF16, d.beta, partial, bias, C};
+                           d.in_dtype == NK_BF16, d.out_dtype == NK_BF16, d.beta, d.layout_c == NK_BLOCKED32,
+                           static_cast<int>(d.M), partial, bias, C};
         const size_t quads = rp.MN / 4;
         splitk_reduce_kernel<<<static_cast<unsigned>((quads + 255) / 256), 256, 0, st>>>(rp);
         e = cudaGetLastError();

@@ -41,6 +41,7 @@ struct UmmaParams {
     int beta;           // 1: the old C is added before the epilogue (Algorithm 1's beta.C)
     int gemms;          // independent GEMMs in one launch (batched matmul): C_g = A_g . B_g; else 1
     long long stride_c; // elements from C_g to C_g+1
+    int c_blocked;      // C is stored as [M/32][N/32][32][32]: each 32 x 32 chunk is one block
     int kb_per_split;   // ceil(kb_total / splits)
     int group_m;        // raster: this many M tiles sweep N together
     int a_blocked;      // A tensor map is the 4-D blocked view
@@ -104,6 +105,11 @@ __device__ __forceinline__ void umma_store_chunk(const UmmaParams& p, uint32_t (
     if (col0 >= p.N || row0 >= p.M) return;           // warp-uniform
     const int row = row0 + lane;
     const size_t c_base = static_cast<size_t>(gemm) * p.stride_c;   // this GEMM's C inside the batch
+    // element offset of (row0 + r, col0 + c) inside C: row-major, or one 32 x 32 block per chunk
+    const size_t blk_base = (static_cast<size_t>(row0 >> 5) * (p.N >> 5) + (col0 >> 5)) * 1024;
+    auto c_off = [&](int r, int c) -> size_t {
+        return p.c_blocked ? blk_base + r * 32 + c : static_cast<size_t>(row0 + r) * p.N + col0 + c;
+    };
     if (empty_k) {
 #pragma unroll
         for (int i = 0; i < 32; ++i) v[i] = 0u;
@@ -113,8 +119,7 @@ __device__ __forceinline__ void umma_store_chunk(const UmmaParams& p, uint32_t (
         // beta = 1: the accumulation tile starts from the stored C (Algorithm 1 loads the C
         // sub-block before the K loop; adding it here, in FP32, gives the same sum)
         if (p.out_bf16) {
-            const uint4* csrc = reinterpret_cast<const uint4*>(static_cast<const uint16_t*>(p.C) + c_base +
-                                                               static_cast<size_t>(row) * p.N + col0);
+            const uint4* csrc = reinterpret_cast<const uint4*>(static_cast<const uint16_t*>(p.C) + c_base + c_off(lane, 0));
 #pragma unroll
             for (int g = 0; g < 4; ++g) {
                 if (col0 + 8 * g >= p.N) break;
@@ -127,8 +132,7 @@ __device__ __forceinline__ void umma_store_chunk(const UmmaParams& p, uint32_t (
                 }
             }
         } else {
-            const uint4* csrc = reinterpret_cast<const uint4*>(static_cast<const float*>(p.C) + c_base +
-                                                               static_cast<size_t>(row) * p.N + col0);
+            const uint4* csrc = reinterpret_cast<const uint4*>(static_cast<const float*>(p.C) + c_base + c_off(lane, 0));
 #pragma unroll
             for (int g = 0; g < 8; ++g) {
                 if (col0 + 4 * g >= p.N) break;
@@ -158,7 +162,7 @@ __device__ __forceinline__ void umma_store_chunk(const UmmaParams& p, uint32_t (
     }
     if (!to_partial && p.out_bf16) {
         if (row >= p.M) return;
-        uint16_t* dst = static_cast<uint16_t*>(p.C) + c_base + static_cast<size_t>(row) * p.N + col0;
+        uint16_t* dst = static_cast<uint16_t*>(p.C) + c_base + c_off(lane, 0);
 #pragma unroll
         for (int g = 0; g < 4; ++g)
             if (col0 + 8 * g < p.N) {
@@ -186,7 +190,8 @@ __device__ __forceinline__ void umma_store_chunk(const UmmaParams& p, uint32_t (
         const int r = 4 * i + rsub;
         const uint4 val = *reinterpret_cast<const uint4*>(staging + r * 128 + ((c ^ (r & 7)) << 4));
         if (col_ok && row0 + r < p.M)
-            *reinterpret_cast<uint4*>(out + static_cast<size_t>(row0 + r) * p.N + col0 + 4 * c) = val;
+            *reinterpret_cast<uint4*>(out + (to_partial ? static_cast<size_t>(row0 + r) * p.N + col0 + 4 * c
+                                                        : c_off(r, 4 * c))) = val;
     }
     __syncwarp();   // the buffer is reused by the next chunk
 }

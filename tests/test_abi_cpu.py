@@ -57,10 +57,12 @@ def test_status_strings():
     (dict(M=8, N=12, K=8, in_dtype=1), 3),                       # BF16 rows must be 16-byte multiples
     (dict(M=8, N=8, K=6, in_dtype=0), 3),
     (dict(M=32, N=32, K=32, in_dtype=1, layout_a=1, batch=2), 2),       # batch-reduce needs row-major
-    (dict(M=32, N=32, K=32, in_dtype=1, layout_b=1, beta=1), 2),
+    (dict(M=32, N=32, K=32, in_dtype=1, layout_b=1, batch=2), 2),
     (dict(M=8, N=8, K=8, in_dtype=1, batch=2, stride_a=68), 3),           # stride not a multiple of 8
     (dict(M=8, N=8, K=8, in_dtype=0, batch=2, stride_b=32), 1),           # items overlap
     (dict(M=8, N=8, K=8, in_dtype=0, beta=2), 1),
+    (dict(M=32, N=32, K=32, in_dtype=0, layout_c=1), 2),                 # blocked C needs BF16 operands
+    (dict(M=32, N=40, K=32, in_dtype=1, layout_c=1), 3),
     (dict(M=8, N=8, K=8, in_dtype=1, flags=nk.FLAG_KERNEL_SIMT), 2),
     (dict(M=8, N=8, K=8, in_dtype=0, flags=nk.FLAG_KERNEL_UMMA), 2),
 ])
@@ -74,7 +76,7 @@ def test_null_arguments():
     L = nk.lib()
     h = ctypes.c_void_p()
     assert L.nk_gemm_create(None, ctypes.byref(h)) == 1
-    assert L.nk_gemm_create(ctypes.byref(binding.Desc(8, 8, 8, 0, 0, 0, 0, 0, 0, 0, 0, 0, 0, 0, 0, 0)), None) == 1
+    assert L.nk_gemm_create(ctypes.byref(binding.Desc(8, 8, 8, 0, 0, 0, 0, 0, 0, 0, 0, 0, 0, 0, 0, 0, 0)), None) == 1
     assert L.nk_gemm_destroy(None) == 0
     assert L.nk_gemm_workspace_bytes(None) == 0
     assert L.nk_gemm_run(None, None, None, None, None, None, 0, None) == 1
