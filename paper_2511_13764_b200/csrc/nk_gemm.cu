@@ -196,7 +196,7 @@ static double simt_model_us(const nk_gemm_desc_t& d, int sms, int tile, int spli
     const int64_t tiles = static_cast<int64_t>(desc_gemms(d)) * ceil_div(d.M, tile) * ceil_div(d.N, tile);
     const int64_t units = tiles * eff_splits;
     const int res = tile == 128 ? 2 : tile == 64 ? 4 : 16;
-    const double eff = tile == 128 ? 0.75 : tile == 64 ? 0.50 : 0.37;
+    const double eff = tile == 128 ? ((d.flags & NK_FLAG_SCALAR_FMA) ? 0.68 : 0.82) : tile == 64 ? 0.50 : 0.37;
     const int64_t slots = static_cast<int64_t>(sms) * res;
     const int64_t full_waves = units / slots;
     const int64_t rest = units - full_waves * slots;
@@ -396,7 +396,7 @@ static cudaError_t pair_occupancy(int* out) {
 }
 
 static cudaError_t prepare_simt_attrs() {
-    return allow_smem(simt_f32_async_kernel<128, 128, 8, 8>, simt_async_smem_bytes<128, 128>());
+    return allow_smem(simt_f32_async_kernel<128, 128, 8, 16, true>, simt_async_smem_bytes<128, 128>());
 }
 
 static cudaError_t prepare_umma_attrs() {
@@ -418,11 +418,13 @@ static cudaError_t prepare_umma_attrs() {
 static cudaError_t launch_simt(nk_gemm_s* p, const SimtParams& sp, cudaStream_t st) {
     const int t = p->simt_tile;
     dim3 grid(ceil_div(sp.N, t), ceil_div(sp.M, t), sp.splits * sp.gemms);
-    // 128-tile: register-staged double buffer (a little faster when the FMA pipe is the limit);
-    // smaller tiles: three-stage cp.async pipeline (their K loops are latency bound).
-    if (t == 128) simt_f32_kernel<128, 128, 8, 8><<<grid, 256, 0, st>>>(sp);
-    else if (t == 64) simt_f32_async_kernel<64, 64, 4, 4><<<grid, 256, simt_async_smem_bytes<64, 64>(), st>>>(sp);
-    else simt_f32_async_kernel<32, 32, 4, 4><<<grid, 64, simt_async_smem_bytes<32, 32>(), st>>>(sp);
+    // 128-tile: 128 threads with 8 x 16 thread tiles and packed FMAs (or, on request, the 256-thread
+    // scalar-FFMA kernel with a register-staged double buffer); all through a three-stage cp.async
+    // pipeline except the scalar one.
+    if (t == 128 && (p->d.flags & NK_FLAG_SCALAR_FMA)) simt_f32_kernel<128, 128, 8, 8><<<grid, 256, 0, st>>>(sp);
+    else if (t == 128) simt_f32_async_kernel<128, 128, 8, 16, true><<<grid, 128, simt_async_smem_bytes<128, 128>(), st>>>(sp);
+    else if (t == 64) simt_f32_async_kernel<64, 64, 4, 4, false><<<grid, 256, simt_async_smem_bytes<64, 64>(), st>>>(sp);
+    else simt_f32_async_kernel<32, 32, 4, 4, false><<<grid, 64, simt_async_smem_bytes<32, 32>(), st>>>(sp);
     return cudaGetLastError();
 }
 
@@ -546,7 +548,9 @@ nk_status_t nk_gemm_create(const nk_gemm_desc_t* desc, nk_gemm_t* out) {
         choose_simt(p);
         p->ws_partial_bytes = p->splits > 1 ? static_cast<size_t>(p->splits) * p->gemms * d.M * d.N * 4 : 0;
         p->launches = p->splits > 1 ? 2 : 1;
-        snprintf(p->name, sizeof(p->name), "simt_f32_%dx%dx16_splitk%d", p->simt_tile, p->simt_tile, p->splits);
+        snprintf(p->name, sizeof(p->name), "simt_f32%s_%dx%dx16_splitk%d",
+                 (p->simt_tile == 128 && !(d.flags & NK_FLAG_SCALAR_FMA)) ? "x2" : "", p->simt_tile, p->simt_tile,
+                 p->splits);
     } else {
         p->variant = V_UMMA;
         void* fn = nullptr;

@@ -65,29 +65,37 @@ simt_f32_kernel(const SimtParams p) {
 
     float4 ra[A_V4], rb[B_V4];
 
-    auto load_global = [&](int kt) {
-        const int item_l = kt / p.kt_per_item;             // which (A_b, B_b) pair of the reduction
-        const int item = gemm + item_l;                    // (+ this GEMM's own pair in a batched matmul)
-        const int k0 = (kt - item_l * p.kt_per_item) * SIMT_BK;
-        const float* Ab = p.A + item * p.stride_a;
-        const float* Bb = p.B + item * p.stride_b;
+    // Where this thread's share of the next k-tile lives in global memory.  The position is
+    // kept as two running pointers that step by one k-tile per load (and by the item stride at
+    // the end of a batch-reduce item), so the K loop carries no divisions or 64-bit multiplies.
+    const int item0 = kt0 / p.kt_per_item;
+    int kin = kt0 - item0 * p.kt_per_item;                 // k-tile inside the current (A_b, B_b) pair
+    const int a_row = t >> 2, a_kq = (t & 3) * 4;          // A: rows a_row + i * THREADS / 4, 4 k per load
+    const int b_kr = t / (BN / 4), b_nq = (t % (BN / 4)) * 4;   // B: k rows b_kr + i * THREADS / (BN / 4)
+    const float* pa = p.A + (gemm + item0) * p.stride_a + static_cast<size_t>(m0 + a_row) * p.K + kin * SIMT_BK + a_kq;
+    const float* pb = p.B + (gemm + item0) * p.stride_b + static_cast<size_t>(kin * SIMT_BK + b_kr) * p.N + n0 + b_nq;
+    const int a_step_i = (THREADS / 4) * p.K, b_step_i = (THREADS / (BN / 4)) * p.N;   // K, N < 2^24: these fit 32 bits
+    const int b_step_kt = SIMT_BK * p.N;
+    const bool b_col_ok = n0 + b_nq < p.N;
+
+    auto load_global = [&]() {
+        const int k0 = kin * SIMT_BK;
 #pragma unroll
-        for (int i = 0; i < A_V4; ++i) {
-            const int idx = t + i * THREADS;       // over BM x 4 float4s
-            const int row = idx >> 2, kq = (idx & 3) * 4;
-            const int gm = m0 + row, gk = k0 + kq;
-            ra[i] = (gm < p.M && gk < p.K)
-                        ? __ldg(reinterpret_cast<const float4*>(Ab + static_cast<size_t>(gm) * p.K + gk))
+        for (int i = 0; i < A_V4; ++i)
+            ra[i] = (m0 + a_row + i * (THREADS / 4) < p.M && k0 + a_kq < p.K)
+                        ? __ldg(reinterpret_cast<const float4*>(pa + i * a_step_i))
                         : make_float4(0.f, 0.f, 0.f, 0.f);
-        }
 #pragma unroll
-        for (int i = 0; i < B_V4; ++i) {
-            const int idx = t + i * THREADS;       // over 16 x BN/4 float4s
-            const int kr = idx / (BN / 4), nq = (idx % (BN / 4)) * 4;
-            const int gk = k0 + kr, gn = n0 + nq;
-            rb[i] = (gk < p.K && gn < p.N)
-                        ? __ldg(reinterpret_cast<const float4*>(Bb + static_cast<size_t>(gk) * p.N + gn))
+        for (int i = 0; i < B_V4; ++i)
+            rb[i] = (b_col_ok && k0 + b_kr + i * (THREADS / (BN / 4)) < p.K)
+                        ? __ldg(reinterpret_cast<const float4*>(pb + i * b_step_i))
                         : make_float4(0.f, 0.f, 0.f, 0.f);
+        pa += SIMT_BK;
+        pb += b_step_kt;
+        if (++kin == p.kt_per_item) {   // next item of the batch-reduce
+            kin = 0;
+            pa += p.stride_a - static_cast<long long>(p.kt_per_item) * SIMT_BK;
+            pb += p.stride_b - static_cast<long long>(p.kt_per_item) * SIMT_BK * p.N;
         }
     };
     auto store_shared = [&](int buf) {
@@ -110,14 +118,14 @@ simt_f32_kernel(const SimtParams p) {
 
     int buf = 0;
     if (kt0 < kt1) {
-        load_global(kt0);
+        load_global();
         store_shared(0);
     }
     __syncthreads();
 
     for (int kt = kt0; kt < kt1; ++kt) {
         const bool more = kt + 1 < kt1;
-        if (more) load_global(kt + 1);
+        if (more) load_global();
 #pragma unroll
         for (int k = 0; k < SIMT_BK; ++k) {
             float a[TM], b[TN];
@@ -301,7 +309,15 @@ __host__ __device__ constexpr int simt_async_smem_bytes() {
     return SIMT_STAGES * SIMT_BK * ((BM + 4) + BN) * 4;
 }
 
-template <int BM, int BN, int TM, int TN>
+//
+// X2 selects packed FMAs (fma.rn.f32x2, new with sm_100: two IEEE FP32 FMAs per instruction on an
+// aligned register pair).  The FMA pipe's peak is the same, but a k-step needs half the issue
+// slots, which is what makes an 8 x 16 thread tile pay: a thread then reads (8 + 16) operands
+// from shared memory per 128 FMAs instead of 16 per 64, and shared-memory bandwidth (128 B per
+// clock per SM against 128 FMA lanes) is the other limit of this kernel.  Accumulators are
+// paired along N, the way a 128-bit load of B delivers them; the A value of a row is copied
+// into both halves of a register pair.
+template <int BM, int BN, int TM, int TN, bool X2>
 __global__ void __launch_bounds__((BM / TM) * (BN / TN), (BM >= 128 ? 2 : 1))
 simt_f32_async_kernel(const SimtParams p) {
     constexpr int THREADS = (BM / TM) * (BN / TN);
@@ -334,29 +350,39 @@ simt_f32_async_kernel(const SimtParams p) {
 #pragma unroll
         for (int j = 0; j < TN; ++j) acc[i][j] = 0.0f;
 
+    // running global positions of this thread's copies (see simt_f32_kernel)
+    const int item0 = kt0 / p.kt_per_item;
+    int kin = kt0 - item0 * p.kt_per_item;
+    const int a_k = t & (SIMT_BK - 1), a_row = t / SIMT_BK;     // A: rows a_row + i * THREADS / 16
+    const int b_kr = t / (BN / 4), b_nq = (t % (BN / 4)) * 4;   // B: k rows b_kr + i * THREADS / (BN / 4)
+    const float* pa = p.A + (gemm + item0) * p.stride_a + static_cast<size_t>(m0 + a_row) * p.K + kin * SIMT_BK + a_k;
+    const float* pb = p.B + (gemm + item0) * p.stride_b + static_cast<size_t>(kin * SIMT_BK + b_kr) * p.N + n0 + b_nq;
+    const int a_step_i = (THREADS / SIMT_BK) * p.K, b_step_i = (THREADS / (BN / 4)) * p.N;   // fit 32 bits
+    const int b_step_kt = SIMT_BK * p.N;
+    const bool b_col_ok = n0 + b_nq < p.N;
+
     auto issue_tile = [&](int kt, int stage) {
         if (kt < kt1) {
-            const int item_l = kt / p.kt_per_item;
-            const int item = gemm + item_l;
-            const int k0 = (kt - item_l * p.kt_per_item) * SIMT_BK;
-            const float* Ab = p.A + item * p.stride_a;
-            const float* Bb = p.B + item * p.stride_b;
+            const int k0 = kin * SIMT_BK;
 #pragma unroll
             for (int i = 0; i < A_ELEMS; ++i) {
-                const int e = t + i * THREADS;             // 16 consecutive lanes = one row's 16 k
-                const int k = e & (SIMT_BK - 1), row = e / SIMT_BK;
-                const bool ok = m0 + row < p.M && k0 + k < p.K;
-                const float* src = Ab + (ok ? static_cast<size_t>(m0 + row) * p.K + k0 + k : 0);
-                cp_async_4(as_u32 + (stage * A_STAGE + k * AP + row) * 4, src, ok ? 4u : 0u);
+                const int row = a_row + i * (THREADS / SIMT_BK);   // 16 consecutive lanes = one row's 16 k
+                const bool ok = m0 + row < p.M && k0 + a_k < p.K;
+                cp_async_4(as_u32 + (stage * A_STAGE + a_k * AP + row) * 4, ok ? pa + i * a_step_i : p.A, ok ? 4u : 0u);
             }
 #pragma unroll
             for (int i = 0; i < B_V4; ++i) {
-                const int idx = t + i * THREADS;
-                const int kr = idx / (BN / 4), nq = (idx % (BN / 4)) * 4;
-                const bool ok = k0 + kr < p.K && n0 + nq < p.N;
-                const float* src = Bb + (ok ? static_cast<size_t>(k0 + kr) * p.N + n0 + nq : 0);
-                cp_async_16(bs_u32 + (stage * B_STAGE + kr * BN + nq) * 4, src, ok ? 16u : 0u);
+                const int kr = b_kr + i * (THREADS / (BN / 4));
+                const bool ok = b_col_ok && k0 + kr < p.K;
+                cp_async_16(bs_u32 + (stage * B_STAGE + kr * BN + b_nq) * 4, ok ? pb + i * b_step_i : p.B, ok ? 16u : 0u);
             }
+            pa += SIMT_BK;
+            pb += b_step_kt;
+            if (++kin == p.kt_per_item) {   // next item of the batch-reduce
+            kin = 0;
+            pa += p.stride_a - static_cast<long long>(p.kt_per_item) * SIMT_BK;
+            pb += p.stride_b - static_cast<long long>(p.kt_per_item) * SIMT_BK * p.N;
+        }
         }
         cp_async_commit();                                  // an empty group keeps the counts aligned
     };
@@ -386,10 +412,22 @@ simt_f32_async_kernel(const SimtParams p) {
                 const float4 v = *reinterpret_cast<const float4*>(bs + k * BN + g * SN_STRIDE + tx * 4);
                 b[4 * g] = v.x; b[4 * g + 1] = v.y; b[4 * g + 2] = v.z; b[4 * g + 3] = v.w;
             }
+            if (X2) {
 #pragma unroll
-            for (int i = 0; i < TM; ++i)
+                for (int i = 0; i < TM; ++i) {
+                    const float2 a2 = make_float2(a[i], a[i]);
 #pragma unroll
-                for (int j = 0; j < TN; ++j) acc[i][j] = fmaf(a[i], b[j], acc[i][j]);
+                    for (int j = 0; j < TN; j += 2) {
+                        float2* c = reinterpret_cast<float2*>(&acc[i][j]);
+                        *c = __ffma2_rn(a2, make_float2(b[j], b[j + 1]), *c);
+                    }
+                }
+            } else {
+#pragma unroll
+                for (int i = 0; i < TM; ++i)
+#pragma unroll
+                    for (int j = 0; j < TN; ++j) acc[i][j] = fmaf(a[i], b[j], acc[i][j]);
+            }
         }
         if (++stage == SIMT_STAGES) stage = 0;
     }

@@ -76,6 +76,7 @@ def main():
     ap.add_argument("--only", default=None, help="substring of the workload name")
     ap.add_argument("--json", default=None)
     ap.add_argument("--no-flush", action="store_true")
+    ap.add_argument("--flags", type=lambda x: int(x, 0), default=0, help="NK_FLAG_* bits given to every plan")
     args = ap.parse_args()
     if not torch.cuda.is_available():
         raise SystemExit("needs a CUDA device")
@@ -90,7 +91,7 @@ def main():
     for w in works:
         if args.only and args.only not in w.name:
             continue
-        med, best, kname, launches = time_workload(w, args.iters, flush=flush)
+        med, best, kname, launches = time_workload(w, args.iters, flags=args.flags, flush=flush)
         tf = w.flops / (med * 1e-3) / 1e12
         gbs = w.algorithmic_bytes / (med * 1e-3) / 1e9
         compute_peak = tensor_peak if w.in_dtype == "bf16" else fma_peak
