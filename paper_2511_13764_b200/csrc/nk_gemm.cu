@@ -43,6 +43,7 @@ struct nk_gemm_s {
     bool b_vnni_inkernel;  // blocked B re-laid inside the GEMM kernel
     bool b_repack;         // blocked B unpacked to row-major scratch first
     bool b_3d;             // B tensor map is the 3-D slab view
+    bool cluster_reduce;   // K splits of a tile = the CTAs of one cluster; partial sums meet in shared memory
     // SIMT
     int simt_tile;  // 128, 64 or 32
     int kt_per_split;
@@ -110,6 +111,7 @@ static cudaError_t allow_smem(K kernel, int bytes) {
 }
 
 static int umma_stages_for(int bn) { return bn == 256 ? 4 : bn == 128 ? 6 : 8; }
+static int cluster_stages_for(int bn) { return bn == 128 ? 4 : 6; }   // the receive slots take the room of the other stages
 
 // Plan-time choice of (single CTA | CTA pair) x tile N x K splits for the BF16 kernel: the
 // counterpart of the paper's tile-size selection (Section 5a, found there by manual search).
@@ -121,6 +123,17 @@ struct UmmaChoice { bool pair; int bn; int splits; double us; };
 
 static int desc_batch(const nk_gemm_desc_t& d) { return (d.batch > 1 && !d.batch_independent) ? static_cast<int>(d.batch) : 1; }
 static int desc_gemms(const nk_gemm_desc_t& d) { return (d.batch > 1 && d.batch_independent) ? static_cast<int>(d.batch) : 1; }
+
+// K splits can meet inside a cluster (no partials in global memory, no second kernel) when the
+// plan is one CTA per 128-row tile, at most 128 columns wide, 2, 4 or 8 splits, and all its units
+// fit the GPU at once (clusters of 8 leave a few SMs of every GPC unused: allow for that).
+static bool cluster_reduce_fits(const nk_gemm_desc_t& d, int sms, bool pair, int bn, int eff_splits) {
+    if (pair || bn > 128 || (d.flags & NK_FLAG_SEPARATE_REDUCE)) return false;
+    if (eff_splits != 2 && eff_splits != 4 && eff_splits != 8) return false;
+    const int64_t units = static_cast<int64_t>(desc_gemms(d)) * ceil_div(d.M, UMMA_BM) * ceil_div(d.N, bn) * eff_splits;
+    const int usable = eff_splits == 8 ? sms - sms / 9 : eff_splits == 4 ? sms - 4 : sms;
+    return units <= usable;
+}
 
 static double umma_model_us(const nk_gemm_desc_t& d, int sms, bool pair, int bn, int splits) {
     const int kb_total = desc_batch(d) * ceil_div(d.K, UMMA_BK);
@@ -136,7 +149,10 @@ static double umma_model_us(const nk_gemm_desc_t& d, int sms, bool pair, int bn,
     const double eo = d.out_dtype == NK_BF16 ? 2.0 : 4.0;
     const double mn = static_cast<double>(d.M) * d.N;
     double us = (pair ? 12.0 : 10.0) + rounds * per * t_kb;
-    if (eff_splits > 1) us += 3.0 + eff_splits * mn * 4.0 / 3.0e6 + (eff_splits * 4.0 + eo) * mn / 5.0e6;
+    if (eff_splits > 1) {
+        if (cluster_reduce_fits(d, sms, pair, bn, eff_splits)) us += 1.5;
+        else us += 3.0 + eff_splits * mn * 4.0 / 3.0e6 + (eff_splits * 4.0 + eo) * mn / 5.0e6;
+    }
     const double bytes = 2.0 * desc_batch(d) * (static_cast<double>(d.M) * d.K + static_cast<double>(d.K) * d.N) + eo * mn;
     const double hbm_us = bytes / 5.2e6;  // ~80 % of the copy bandwidth, bytes per microsecond
     return us > hbm_us ? us : hbm_us;
@@ -182,6 +198,8 @@ static void choose_umma(nk_gemm_s* p) {
     p->stages = best.pair ? (best.bn == 256 ? 6 : 8) : umma_stages_for(best.bn);
     p->splits = splits;
     p->group_m = 8;
+    p->cluster_reduce = splits > 1 && cluster_reduce_fits(d, sms, best.pair, best.bn, splits);
+    if (p->cluster_reduce) p->stages = cluster_stages_for(best.bn);
 }
 
 // Plan-time choice of tile and K splits for the FP32 kernel (the counterpart of the paper's
@@ -354,6 +372,41 @@ static cudaError_t launch_umma(nk_gemm_s* p, const UmmaParams& up, int grid, cud
     }
 }
 
+// Cluster split-K variants: BN = 128 with 4 stages, BN = 64 with 6 (the receive slots take the
+// room of the other stages); the cluster is `splits` CTAs wide and the grid is exactly the units.
+template <int BN, int STAGES, bool VNNI>
+static cudaError_t launch_cluster_t(nk_gemm_s* p, const UmmaParams& up, int units, int splits, cudaStream_t st,
+                                    int* max_clusters) {
+    cudaLaunchConfig_t cfg;
+    memset(&cfg, 0, sizeof(cfg));
+    cfg.gridDim = dim3(static_cast<unsigned>(units));
+    cfg.blockDim = dim3(VNNI ? 320 : 192);
+    cfg.dynamicSmemBytes = umma_cluster_smem_bytes(BN, STAGES);
+    cfg.stream = st;
+    cudaLaunchAttribute attr;
+    attr.id = cudaLaunchAttributeClusterDimension;
+    attr.val.clusterDim.x = static_cast<unsigned>(splits);
+    attr.val.clusterDim.y = 1;
+    attr.val.clusterDim.z = 1;
+    cfg.attrs = &attr;
+    cfg.numAttrs = 1;
+    if (max_clusters) {   // occupancy query only
+        cfg.gridDim = dim3(static_cast<unsigned>(splits));
+        return cudaOccupancyMaxActiveClusters(max_clusters, umma_bf16_kernel<BN, STAGES, VNNI, true>, &cfg);
+    }
+    return cudaLaunchKernelEx(&cfg, umma_bf16_kernel<BN, STAGES, VNNI, true>, p->tmap_a, p->tmap_b, up);
+}
+
+static cudaError_t launch_cluster(nk_gemm_s* p, const UmmaParams& up, int units, int splits, cudaStream_t st,
+                                  int* max_clusters) {
+    const bool v = p->b_vnni_inkernel;
+    if (p->bn == 128)
+        return v ? launch_cluster_t<128, 4, true>(p, up, units, splits, st, max_clusters)
+                 : launch_cluster_t<128, 4, false>(p, up, units, splits, st, max_clusters);
+    return v ? launch_cluster_t<64, 6, true>(p, up, units, splits, st, max_clusters)
+             : launch_cluster_t<64, 6, false>(p, up, units, splits, st, max_clusters);
+}
+
 template <int BN, int STAGES, bool VNNI>
 static cudaError_t launch_pair_t(nk_gemm_s* p, const UmmaParams& up, int pairs, cudaStream_t st) {
     cudaLaunchConfig_t cfg;
@@ -412,6 +465,10 @@ static cudaError_t prepare_umma_attrs() {
     if ((e = allow_smem(umma_bf16_kernel<256, 4, true>, umma_smem_bytes(256, 4))) != cudaSuccess) return e;
     if ((e = allow_smem(umma_bf16_kernel<128, 6, true>, umma_smem_bytes(128, 6))) != cudaSuccess) return e;
     if ((e = allow_smem(umma_bf16_kernel<64, 8, true>, umma_smem_bytes(64, 8))) != cudaSuccess) return e;
+    if ((e = allow_smem(umma_bf16_kernel<128, 4, false, true>, umma_cluster_smem_bytes(128, 4))) != cudaSuccess) return e;
+    if ((e = allow_smem(umma_bf16_kernel<128, 4, true, true>, umma_cluster_smem_bytes(128, 4))) != cudaSuccess) return e;
+    if ((e = allow_smem(umma_bf16_kernel<64, 6, false, true>, umma_cluster_smem_bytes(64, 6))) != cudaSuccess) return e;
+    if ((e = allow_smem(umma_bf16_kernel<64, 6, true, true>, umma_cluster_smem_bytes(64, 6))) != cudaSuccess) return e;
     return cudaSuccess;
 }
 
@@ -576,12 +633,22 @@ nk_status_t nk_gemm_create(const nk_gemm_desc_t* desc, nk_gemm_t* out) {
             if (oe != cudaSuccess || n <= 0) { cudaGetLastError(); delete p; return NK_ERR_CUDA; }
             p->max_pairs = n;
         }
+        if (p->cluster_reduce) {
+            // every cluster of the plan must be resident at once (one unit per CTA): ask the driver
+            int n = 0;
+            const int clusters = p->gemms * ceil_div(d.M, UMMA_BM) * ceil_div(d.N, p->bn);
+            if (launch_cluster(p, UmmaParams(), 0, p->splits, nullptr, &n) != cudaSuccess || n < clusters) {
+                cudaGetLastError();
+                p->cluster_reduce = false;
+                p->stages = umma_stages_for(p->bn);
+            }
+        }
         p->ws_repack_bytes = p->b_repack ? align_up(static_cast<size_t>(d.K) * d.N * 2, 256) : 0;
-        p->ws_partial_bytes = p->splits > 1 ? static_cast<size_t>(p->splits) * p->gemms * d.M * d.N * 4 : 0;
-        p->launches = 1 + (p->splits > 1 ? 1 : 0) + (p->b_repack ? 1 : 0);
-        snprintf(p->name, sizeof(p->name), "umma_bf16_%s%dx64_s%d_splitk%d%s%s",
+        p->ws_partial_bytes = (p->splits > 1 && !p->cluster_reduce) ? static_cast<size_t>(p->splits) * p->gemms * d.M * d.N * 4 : 0;
+        p->launches = 1 + ((p->splits > 1 && !p->cluster_reduce) ? 1 : 0) + (p->b_repack ? 1 : 0);
+        snprintf(p->name, sizeof(p->name), "umma_bf16_%s%dx64_s%d_splitk%d%s%s%s",
                  p->pair ? "pair_256x" : "128x", p->bn, p->stages,
-                 p->splits, d.layout_a == NK_BLOCKED32 ? "_ablk" : "",
+                 p->splits, p->cluster_reduce ? "_cluster" : "", d.layout_a == NK_BLOCKED32 ? "_ablk" : "",
                  p->b_vnni_inkernel ? "_bvnni" : (p->b_repack ? "_brepack" : ""));
     }
     if (p->batch > 1 || p->gemms > 1 || d.beta) {
@@ -595,7 +662,7 @@ nk_status_t nk_gemm_create(const nk_gemm_desc_t* desc, nk_gemm_t* out) {
     }
     // split-K partials are laid out [split][gemm][M][N] and reduced as one flat array: that
     // needs the C of a batched matmul to be contiguous
-    if (p->gemms > 1 && p->splits > 1 && p->stride_c != d.M * d.N) {
+    if (p->gemms > 1 && p->splits > 1 && p->stride_c != d.M * d.N && !p->cluster_reduce) {
         delete p;
         *out = nullptr;
         return NK_ERR_UNSUPPORTED;
@@ -698,7 +765,9 @@ nk_status_t nk_gemm_run(nk_gemm_t p, const void* A, const void* B, const void* b
         up.Bblk = p->b_vnni_inkernel ? static_cast<const uint32_t*>(B) : nullptr;
         up.status = p->status_dev;
         const int units = up.gemms * up.tiles_m * up.tiles_n * up.splits;
-        if (p->pair) {
+        if (p->cluster_reduce) {
+            e = launch_cluster(p, up, units, p->splits, st, nullptr);
+        } else if (p->pair) {
             const int pairs = units < p->max_pairs ? units : p->max_pairs;
             e = launch_pair(p, up, pairs, st);
         } else {
@@ -708,7 +777,7 @@ nk_status_t nk_gemm_run(nk_gemm_t p, const void* A, const void* B, const void* b
         if (e != cudaSuccess) { set_err(p, "umma launch", e); return NK_ERR_CUDA; }
     }
 
-    if (p->splits > 1) {
+    if (p->splits > 1 && !p->cluster_reduce) {
         ReduceParams rp = {static_cast<size_t>(p->gemms) * d.M * d.N, static_cast<int>(d.N), p->splits, d.epilogue,
                            d.in_dtype == NK_BF16, d.out_dtype == NK_BF16, d.beta, d.layout_c == NK_BLOCKED32,
                            static_cast<int>(d.M), partial, bias, C};

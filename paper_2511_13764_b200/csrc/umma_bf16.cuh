@@ -21,6 +21,13 @@
 // Every mbarrier wait is bounded; a role that gives up raises the CTA's abort
 // flag and the device status word, the other roles fall out of their loops, and
 // the CTA frees its TMEM and exits.
+//
+// Split-K inside a thread-block cluster (CLUSTER_REDUCE): the K splits of one tile are the CTAs
+// of one cluster, one unit per CTA.  After its K loop every CTA scatters its accumulator, in
+// 32 x 32 pieces, straight into the shared memory of the CTA that owns each piece (distributed
+// shared memory); after a cluster barrier every CTA adds the pieces it owns in split order,
+// applies the epilogue and stores them.  No partial ever goes to global memory and there is no
+// second kernel.
 #pragma once
 #include <cuda.h>
 #include <cuda_bf16.h>
@@ -63,6 +70,12 @@ __host__ __device__ constexpr int umma_stage_bytes(int BN) {
 constexpr int UMMA_EPI_STAGING = 4 * 4096;   // one 32 x 32 FP32 chunk per epilogue warp
 __host__ __device__ constexpr int umma_smem_bytes(int BN, int stages) {
     return stages * umma_stage_bytes(BN) + 1024 /*alignment slack*/ + 256 /*barriers*/ + UMMA_EPI_STAGING;
+}
+// cluster split-K: one 4 KB slot per (32 x 32 piece this CTA owns, split it comes from); a tile has
+// 4 * BN / 32 pieces shared out over the cluster, so the slots of a CTA always add up to the tile
+__host__ __device__ constexpr int umma_recv_bytes(int BN) { return 4 * (BN / 32) * 4096; }
+__host__ __device__ constexpr int umma_cluster_smem_bytes(int BN, int stages) {
+    return umma_smem_bytes(BN, stages) + umma_recv_bytes(BN);
 }
 
 // tile id -> (m block, n block): groups of `group_m` M tiles sweep across N so
@@ -196,6 +209,54 @@ __device__ __forceinline__ void umma_store_chunk(const UmmaParams& p, uint32_t (
     __syncwarp();   // the buffer is reused by the next chunk
 }
 
+// Tail of the cluster split-K reduction: lane (rsub = lane / 8, cg = lane % 8) holds the summed
+// FP32 values of rows row0 + 4 i + rsub (i = 0..7), columns col0 + 4 cg .. + 3 of one 32 x 32
+// piece; beta, bias + ReLU, the conversion and the store of C follow (Section 6, "MLP").
+__device__ __forceinline__ void umma_finish_piece(const UmmaParams& p, float4 (&s)[8], int row0, int col0, int gemm,
+                                                  int lane) {
+    const int cg = lane & 7, rsub = lane >> 3;
+    const int col = col0 + 4 * cg;
+    if (col >= p.N || row0 >= p.M) return;
+    const size_t c_base = static_cast<size_t>(gemm) * p.stride_c;
+    float4 bv = make_float4(0.f, 0.f, 0.f, 0.f);
+    if (p.epilogue) {
+        const uint2 w = __ldg(reinterpret_cast<const uint2*>(static_cast<const uint16_t*>(p.bias) + col));
+        bv = make_float4(bf16_bits_to_f32(w.x & 0xFFFFu), bf16_bits_to_f32(w.x >> 16),
+                         bf16_bits_to_f32(w.y & 0xFFFFu), bf16_bits_to_f32(w.y >> 16));
+    }
+    const size_t blk_base = (static_cast<size_t>(row0 >> 5) * (p.N >> 5) + (col0 >> 5)) * 1024;
+#pragma unroll
+    for (int i = 0; i < 8; ++i) {
+        const int r = 4 * i + rsub;
+        if (row0 + r >= p.M) continue;
+        const size_t off = c_base + (p.c_blocked ? blk_base + r * 32 + 4 * cg
+                                                 : static_cast<size_t>(row0 + r) * p.N + col);
+        float4 v = s[i];
+        if (p.beta) {
+            if (p.out_bf16) {
+                const uint2 w = *reinterpret_cast<const uint2*>(static_cast<const uint16_t*>(p.C) + off);
+                v.x += bf16_bits_to_f32(w.x & 0xFFFFu); v.y += bf16_bits_to_f32(w.x >> 16);
+                v.z += bf16_bits_to_f32(w.y & 0xFFFFu); v.w += bf16_bits_to_f32(w.y >> 16);
+            } else {
+                const float4 cv = *reinterpret_cast<const float4*>(static_cast<const float*>(p.C) + off);
+                v.x += cv.x; v.y += cv.y; v.z += cv.z; v.w += cv.w;
+            }
+        }
+        if (p.epilogue) {
+            v.x = fmaxf(v.x + bv.x, 0.f); v.y = fmaxf(v.y + bv.y, 0.f);
+            v.z = fmaxf(v.z + bv.z, 0.f); v.w = fmaxf(v.w + bv.w, 0.f);
+        }
+        if (p.out_bf16) {
+            uint2 o;
+            o.x = pack_bf16x2(v.x, v.y);
+            o.y = pack_bf16x2(v.z, v.w);
+            *reinterpret_cast<uint2*>(static_cast<uint16_t*>(p.C) + off) = o;
+        } else {
+            *reinterpret_cast<float4*>(static_cast<float*>(p.C) + off) = v;
+        }
+    }
+}
+
 // Re-layout of a VNNI-blocked B operand (Figure 1 of the paper: [k/2][n][2] inside every 32 x 32
 // block) into the K-major stage tile the tensor core reads: ROWS columns n x 64 k, 128-byte
 // rows, 16-byte chunk c of row n stored at chunk c ^ (n & 7) (the 128-byte swizzle).  Seen as
@@ -242,7 +303,7 @@ __device__ __forceinline__ void vnni_issue_stage(const UmmaParams& p, uint32_t s
     cp_async_commit();
 }
 
-template <int BN, int STAGES, bool B_VNNI>
+template <int BN, int STAGES, bool B_VNNI, bool CLUSTER_REDUCE = false>
 __global__ void __launch_bounds__(B_VNNI ? 320 : 192, 1)
 umma_bf16_kernel(const __grid_constant__ CUtensorMap tmap_a,
                  const __grid_constant__ CUtensorMap tmap_b, const UmmaParams p) {
@@ -290,6 +351,9 @@ umma_bf16_kernel(const __grid_constant__ CUtensorMap tmap_a,
     __syncthreads();
     tc_fence_after_sync();
     const uint32_t tmem_base = *tmem_slot;
+    // cluster split-K, barrier phase A ("this CTA is running: its shared memory may be written"):
+    // arrive now, wait only just before the first remote store
+    if (CLUSTER_REDUCE) cluster_arrive();
 
     const int total_units = p.gemms * p.tiles_m * p.tiles_n * p.splits;
 
@@ -426,6 +490,65 @@ umma_bf16_kernel(const __grid_constant__ CUtensorMap tmap_a,
             if (kb1 <= kb0 && lane == 0) umma_commit(tfull_bar(acc));  // empty K range
             __syncwarp();
         }
+    } else if (warp < 6 && CLUSTER_REDUCE) {
+        // ------------------------------------------------ epilogue, K splits reduced inside the cluster
+        // One unit per CTA (grid = units); cluster rank = K split.  Piece u = quarter * NC + chunk of
+        // the 128 x BN tile is owned by CTA u % S and kept there in slot (u / S, source split).
+        constexpr int NC = BN / 32;
+        const int quarter = warp & 3;
+        const uint32_t S = static_cast<uint32_t>(p.splits), rank = cluster_ctarank();
+        const uint32_t recv = bar_base + 256 + UMMA_EPI_STAGING;   // shared-memory offset of the slots, same in every CTA
+        int tile, split, gemm;
+        umma_decode_unit(p, blockIdx.x, tile, split, gemm);
+        int mb, nb;
+        umma_tile_coords(p, tile, mb, nb);
+        bool ok = blockIdx.x < total_units;
+        if (ok && !mbar_wait(tfull_bar(0), 0u, abort_flag)) {
+            if (lane == 0) give_up(0x400u);
+            ok = false;
+        }
+        tc_fence_after_sync();
+        cluster_wait();                                  // phase A: every CTA of the cluster is running
+        if (ok) {
+#pragma unroll 1
+            for (int c = 0; c < NC; ++c) {
+                uint32_t v[32];
+                tmem_ld_32x32(tmem_base + c * 32 + (static_cast<uint32_t>(quarter * 32) << 16), v);
+                tmem_ld_wait();
+                const uint32_t u = quarter * NC + c, owner = u % S, slot = (u / S) * S + rank;
+                const uint32_t dst = map_to_cta(recv + slot * 4096u + lane * 128u, owner);
+#pragma unroll
+                for (int g = 0; g < 8; ++g)
+                    st_cluster_v4(dst + ((g ^ (lane & 7)) << 4), v[4 * g], v[4 * g + 1], v[4 * g + 2], v[4 * g + 3]);
+            }
+        }
+        cluster_arrive();                                // phase B: this thread's pieces are delivered
+        cluster_wait();                                  //          ... and so are everybody else's
+        if (ok) {
+            const uint8_t* recv_gen = gen_base + STAGES * STAGE + 256 + UMMA_EPI_STAGING;
+            const int cg = lane & 7, rsub = lane >> 3;
+#pragma unroll 1
+            for (int c = 0; c < NC; ++c) {
+                const uint32_t u = quarter * NC + c;
+                if (u % S != rank) continue;             // warp-uniform
+                const uint8_t* slot0 = recv_gen + (u / S) * S * 4096u;
+                float4 acc4[8];
+#pragma unroll
+                for (int i = 0; i < 8; ++i) {
+                    const int r = 4 * i + rsub;
+                    acc4[i] = *reinterpret_cast<const float4*>(slot0 + r * 128 + ((cg ^ (r & 7)) << 4));
+                }
+                for (uint32_t sp = 1; sp < S; ++sp) {     // split order: the sum does not depend on timing
+#pragma unroll
+                    for (int i = 0; i < 8; ++i) {
+                        const int r = 4 * i + rsub;
+                        const float4 t4 = *reinterpret_cast<const float4*>(slot0 + sp * 4096u + r * 128 + ((cg ^ (r & 7)) << 4));
+                        acc4[i].x += t4.x; acc4[i].y += t4.y; acc4[i].z += t4.z; acc4[i].w += t4.w;
+                    }
+                }
+                umma_finish_piece(p, acc4, mb * UMMA_BM + quarter * 32, nb * BN + c * 32, gemm, lane);
+            }
+        }
     } else if (warp < 6) {
         // ------------------------------------------------ epilogue
         const int quarter = warp & 3;  // TMEM lanes 32*quarter .. +31 belong to this warp
@@ -501,6 +624,12 @@ umma_bf16_kernel(const __grid_constant__ CUtensorMap tmap_a,
         }
     }
 
+    if (CLUSTER_REDUCE && !(warp >= 2 && warp < 6)) {
+        // the cluster barrier counts every thread: the other roles pass both phases here
+        cluster_wait();
+        cluster_arrive();
+        cluster_wait();
+    }
     tc_fence_before_sync();
     __syncthreads();
     if (warp == 1) {
