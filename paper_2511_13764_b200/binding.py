@@ -18,6 +18,7 @@ FLAG_REPACK_B = 0x10
 FLAG_SINGLE_CTA, FLAG_CTA_PAIR = 0x20, 0x40
 FLAG_SCALAR_FMA = 0x80
 FLAG_SEPARATE_REDUCE = 0x100000
+FLAG_LSU_STORE = 0x200000
 
 EXPORTS = ["nk_gemm_create", "nk_gemm_workspace_bytes", "nk_gemm_run", "nk_gemm_run_host",
            "nk_gemm_check", "nk_gemm_destroy", "nk_status_str", "nk_gemm_kernel_name",

@@ -58,8 +58,9 @@ struct nk_gemm_s {
     // device status word
     unsigned int* status_dev;
     // cached tensor maps
-    CUtensorMap tmap_a, tmap_b;
-    const void *cached_a, *cached_b;
+    CUtensorMap tmap_a, tmap_b, tmap_c;
+    const void *cached_a, *cached_b, *cached_c;
+    bool tma_store;        // FP32 row-major C without beta or K split: stored by TMA, 32 x 32 boxes
     nk::EncodeTiledFn encode;
     char name[96];
     char cuda_err[256];
@@ -354,11 +355,31 @@ static nk_status_t encode_maps(nk_gemm_s* p, const void* A, const void* B) {
     return NK_OK;
 }
 
+// C row-major FP32 [gemms][M][N] as (n, m, gemm): the epilogue stores 32 x 32 boxes from a
+// 128-byte-swizzled staging tile; the TMA unit drops whatever lies beyond M or N.
+static nk_status_t encode_c_map(nk_gemm_s* p, void* C) {
+    if (!p->tma_store || p->cached_c == C) return NK_OK;
+    const nk_gemm_desc_t& d = p->d;
+    cuuint64_t dims[3] = {static_cast<cuuint64_t>(d.N), static_cast<cuuint64_t>(d.M), static_cast<cuuint64_t>(p->gemms)};
+    cuuint64_t strides[2] = {static_cast<cuuint64_t>(d.N) * 4, static_cast<cuuint64_t>(p->stride_c) * 4};
+    cuuint32_t box[3] = {32, 32, 1};
+    cuuint32_t es[3] = {1, 1, 1};
+    CUresult r = p->encode(&p->tmap_c, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 3, C, dims, strides, box, es,
+                           CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+                           CU_TENSOR_MAP_L2_PROMOTION_NONE, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    if (r != CUDA_SUCCESS) {
+        snprintf(p->cuda_err, sizeof(p->cuda_err), "cuTensorMapEncodeTiled(C) failed: %d", (int)r);
+        return NK_ERR_CUDA;
+    }
+    p->cached_c = C;
+    return NK_OK;
+}
+
 template <int BN, int STAGES, bool VNNI>
 static cudaError_t launch_umma_t(nk_gemm_s* p, const UmmaParams& up, int grid, cudaStream_t st) {
     auto k = umma_bf16_kernel<BN, STAGES, VNNI>;
     umma_bf16_kernel<BN, STAGES, VNNI><<<grid, VNNI ? 320 : 192, umma_smem_bytes(BN, STAGES), st>>>(
-        p->tmap_a, p->tmap_b, up);
+        p->tmap_a, p->tmap_b, p->tmap_c, up);
     (void)k;
     return cudaGetLastError();
 }
@@ -394,7 +415,7 @@ static cudaError_t launch_cluster_t(nk_gemm_s* p, const UmmaParams& up, int unit
         cfg.gridDim = dim3(static_cast<unsigned>(splits));
         return cudaOccupancyMaxActiveClusters(max_clusters, umma_bf16_kernel<BN, STAGES, VNNI, true>, &cfg);
     }
-    return cudaLaunchKernelEx(&cfg, umma_bf16_kernel<BN, STAGES, VNNI, true>, p->tmap_a, p->tmap_b, up);
+    return cudaLaunchKernelEx(&cfg, umma_bf16_kernel<BN, STAGES, VNNI, true>, p->tmap_a, p->tmap_b, p->tmap_c, up);
 }
 
 static cudaError_t launch_cluster(nk_gemm_s* p, const UmmaParams& up, int units, int splits, cudaStream_t st,
@@ -422,7 +443,7 @@ static cudaError_t launch_pair_t(nk_gemm_s* p, const UmmaParams& up, int pairs, 
     attr.val.clusterDim.z = 1;
     cfg.attrs = &attr;
     cfg.numAttrs = 1;
-    return cudaLaunchKernelEx(&cfg, umma_bf16_pair_kernel<BN, STAGES, VNNI>, p->tmap_a, p->tmap_b, up);
+    return cudaLaunchKernelEx(&cfg, umma_bf16_pair_kernel<BN, STAGES, VNNI>, p->tmap_a, p->tmap_b, p->tmap_c, up);
 }
 
 static cudaError_t launch_pair(nk_gemm_s* p, const UmmaParams& up, int pairs, cudaStream_t st) {
@@ -643,6 +664,8 @@ nk_status_t nk_gemm_create(const nk_gemm_desc_t* desc, nk_gemm_t* out) {
                 p->stages = umma_stages_for(p->bn);
             }
         }
+        p->tma_store = d.out_dtype == NK_F32 && d.layout_c == NK_ROW_MAJOR && d.beta == 0 && p->splits == 1 &&
+                       !(d.flags & NK_FLAG_LSU_STORE);
         p->ws_repack_bytes = p->b_repack ? align_up(static_cast<size_t>(d.K) * d.N * 2, 256) : 0;
         p->ws_partial_bytes = (p->splits > 1 && !p->cluster_reduce) ? static_cast<size_t>(p->splits) * p->gemms * d.M * d.N * 4 : 0;
         p->launches = 1 + ((p->splits > 1 && !p->cluster_reduce) ? 1 : 0) + (p->b_repack ? 1 : 0);
@@ -740,6 +763,7 @@ nk_status_t nk_gemm_run(nk_gemm_t p, const void* A, const void* B, const void* b
         }
         nk_status_t s = encode_maps(p, A, Buse);
         if (s != NK_OK) return s;
+        if ((s = encode_c_map(p, C)) != NK_OK) return s;
         UmmaParams up;
         memset(&up, 0, sizeof(up));
         up.M = static_cast<int>(d.M); up.N = static_cast<int>(d.N); up.K = static_cast<int>(d.K);
@@ -752,6 +776,7 @@ nk_status_t nk_gemm_run(nk_gemm_t p, const void* A, const void* B, const void* b
         up.gemms = p->gemms;
         up.stride_c = p->stride_c;
         up.c_blocked = d.layout_c == NK_BLOCKED32;
+        up.tma_store = p->tma_store ? 1 : 0;
         up.kb_per_split = ceil_div(up.kb_total, p->splits);
         up.group_m = p->group_m;
         up.a_blocked = d.layout_a == NK_BLOCKED32;

@@ -49,6 +49,7 @@ struct UmmaParams {
     int gemms;          // independent GEMMs in one launch (batched matmul): C_g = A_g . B_g; else 1
     long long stride_c; // elements from C_g to C_g+1
     int c_blocked;      // C is stored as [M/32][N/32][32][32]: each 32 x 32 chunk is one block
+    int tma_store;      // C (FP32, row-major, no beta, no K split) leaves through TMA stores of 32 x 32 boxes
     int kb_per_split;   // ceil(kb_total / splits)
     int group_m;        // raster: this many M tiles sweep N together
     int a_blocked;      // A tensor map is the 4-D blocked view
@@ -67,9 +68,9 @@ __host__ __device__ constexpr int umma_b_stage_bytes(int BN) { return BN * UMMA_
 __host__ __device__ constexpr int umma_stage_bytes(int BN) {
     return UMMA_A_STAGE_BYTES + umma_b_stage_bytes(BN);
 }
-constexpr int UMMA_EPI_STAGING = 4 * 4096;   // one 32 x 32 FP32 chunk per epilogue warp
+constexpr int UMMA_EPI_STAGING = 4 * 2 * 4096;   // two 32 x 32 FP32 chunks per epilogue warp (1024-byte aligned: TMA store source)
 __host__ __device__ constexpr int umma_smem_bytes(int BN, int stages) {
-    return stages * umma_stage_bytes(BN) + 1024 /*alignment slack*/ + 256 /*barriers*/ + UMMA_EPI_STAGING;
+    return stages * umma_stage_bytes(BN) + 1024 /*alignment slack*/ + UMMA_EPI_STAGING + 256 /*barriers*/;
 }
 // cluster split-K: one 4 KB slot per (32 x 32 piece this CTA owns, split it comes from); a tile has
 // 4 * BN / 32 pieces shared out over the cluster, so the slots of a CTA always add up to the tile
@@ -113,8 +114,9 @@ __device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi) {
 // row t kept at chunk g ^ (t & 7): conflict-free both ways) so that every store instruction
 // writes four whole 128-byte row segments instead of 32 scattered 16-byte pieces.  BF16 rows
 // (64 bytes each) are stored directly.  Columns are predicated in groups (N is a multiple of 8).
-__device__ __forceinline__ void umma_store_chunk(const UmmaParams& p, uint32_t (&v)[32], int row0, int lane,
-                                                 int col0, int split, int gemm, bool empty_k, uint8_t* staging) {
+__device__ __forceinline__ void umma_store_chunk(const UmmaParams& p, const CUtensorMap* tmap_c, uint32_t (&v)[32],
+                                                 int row0, int lane, int col0, int split, int gemm, bool empty_k,
+                                                 uint8_t* staging) {
     if (col0 >= p.N || row0 >= p.M) return;           // warp-uniform
     const int row = row0 + lane;
     const size_t c_base = static_cast<size_t>(gemm) * p.stride_c;   // this GEMM's C inside the batch
@@ -188,11 +190,28 @@ __device__ __forceinline__ void umma_store_chunk(const UmmaParams& p, uint32_t (
             }
         return;
     }
-    // FP32: registers -> staging (row per lane) -> global (4 row segments per instruction)
+    // FP32: registers -> staging (row per lane, 16-byte chunk g of row t at chunk g ^ (t & 7): the
+    // 128-byte swizzle) -> global, either as one TMA store of the 32 x 32 box (the TMA unit writes
+    // whole lines and clips the ragged edge; the warp only pays eight shared-memory stores), or with
+    // per-thread stores of four 128-byte row segments per instruction.
+    if (p.tma_store) {
+        // the caller alternates two buffers: the store issued two chunks ago has read this one
+        if (lane == 0) bulk_wait_read<1>();
+        __syncwarp();
+    }
 #pragma unroll
     for (int g = 0; g < 8; ++g)
         *reinterpret_cast<uint4*>(staging + lane * 128 + ((g ^ (lane & 7)) << 4)) =
             make_uint4(v[4 * g], v[4 * g + 1], v[4 * g + 2], v[4 * g + 3]);
+    if (p.tma_store) {
+        fence_proxy_async_smem();
+        __syncwarp();
+        if (lane == 0) {
+            tma_store_3d(tmap_c, smem_u32(staging), col0, row0, gemm);
+            bulk_commit();
+        }
+        return;
+    }
     __syncwarp();
     float* out = to_partial ? p.partial + (static_cast<size_t>(split) * p.gemms + gemm) * p.M * p.N
                             : static_cast<float*>(p.C) + c_base;
@@ -305,8 +324,8 @@ __device__ __forceinline__ void vnni_issue_stage(const UmmaParams& p, uint32_t s
 
 template <int BN, int STAGES, bool B_VNNI, bool CLUSTER_REDUCE = false>
 __global__ void __launch_bounds__(B_VNNI ? 320 : 192, 1)
-umma_bf16_kernel(const __grid_constant__ CUtensorMap tmap_a,
-                 const __grid_constant__ CUtensorMap tmap_b, const UmmaParams p) {
+umma_bf16_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ CUtensorMap tmap_b,
+                 const __grid_constant__ CUtensorMap tmap_c, const UmmaParams p) {
     static_assert(BN % 32 == 0 && BN >= 32 && BN <= 256, "tile N");
     constexpr int B_STAGE = umma_b_stage_bytes(BN);
     constexpr int STAGE = umma_stage_bytes(BN);
@@ -315,15 +334,16 @@ umma_bf16_kernel(const __grid_constant__ CUtensorMap tmap_a,
 
     extern __shared__ uint8_t smem_raw[];
     const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
-    const uint32_t bar_base = smem_base + STAGES * STAGE;
-    // barrier block: full[STAGES], empty[STAGES], tmem_full[2], tmem_empty[2], then 2 words
+    const uint32_t bar_base = smem_base + STAGES * STAGE + UMMA_EPI_STAGING;
+    // after the stages: epilogue staging, then the barrier block: full[STAGES], empty[STAGES],
+    // tmem_full[2], tmem_empty[2], then 2 words
     auto full_bar = [&](int s) { return bar_base + 8u * s; };
     auto empty_bar = [&](int s) { return bar_base + 8u * (STAGES + s); };
     auto tfull_bar = [&](int a) { return bar_base + 8u * (2 * STAGES + a); };
     auto tempty_bar = [&](int a) { return bar_base + 8u * (2 * STAGES + 2 + a); };
     uint8_t* gen_base = smem_raw + (smem_base - smem_u32(smem_raw));
     volatile uint32_t* tmem_slot =
-        reinterpret_cast<volatile uint32_t*>(gen_base + STAGES * STAGE + 8 * (2 * STAGES + 4));
+        reinterpret_cast<volatile uint32_t*>(gen_base + STAGES * STAGE + UMMA_EPI_STAGING + 8 * (2 * STAGES + 4));
     volatile uint32_t* abort_flag = tmem_slot + 1;
 
     const int warp = threadIdx.x >> 5;
@@ -342,15 +362,26 @@ umma_bf16_kernel(const __grid_constant__ CUtensorMap tmap_a,
         fence_mbar_init();
         tma_prefetch_desc(&tmap_a);
         if (!B_VNNI) tma_prefetch_desc(&tmap_b);
+        if (p.tma_store) tma_prefetch_desc(&tmap_c);
     }
     if (warp == 1) {
         tmem_alloc(smem_u32(const_cast<uint32_t*>(tmem_slot)), TMEM_COLS);
         tmem_relinquish();
     }
-    tc_fence_before_sync();
-    __syncthreads();
-    tc_fence_after_sync();
-    const uint32_t tmem_base = *tmem_slot;
+    // The producer warp needs nothing but the barriers its own lane 0 has just initialised: it
+    // signals the CTA barrier without waiting on it and starts fetching while tensor memory is
+    // still being allocated (on a short problem this start-up is a visible part of the run).
+    const uint32_t nthreads = blockDim.x;
+    uint32_t tmem_base = 0;
+    if (warp == 0) {
+        __syncwarp();
+        asm volatile("bar.arrive 0, %0;" ::"r"(nthreads) : "memory");
+    } else {
+        tc_fence_before_sync();
+        asm volatile("bar.sync 0, %0;" ::"r"(nthreads) : "memory");
+        tc_fence_after_sync();
+        tmem_base = *tmem_slot;
+    }
     // cluster split-K, barrier phase A ("this CTA is running: its shared memory may be written"):
     // arrive now, wait only just before the first remote store
     if (CLUSTER_REDUCE) cluster_arrive();
@@ -497,7 +528,7 @@ umma_bf16_kernel(const __grid_constant__ CUtensorMap tmap_a,
         constexpr int NC = BN / 32;
         const int quarter = warp & 3;
         const uint32_t S = static_cast<uint32_t>(p.splits), rank = cluster_ctarank();
-        const uint32_t recv = bar_base + 256 + UMMA_EPI_STAGING;   // shared-memory offset of the slots, same in every CTA
+        const uint32_t recv = bar_base + 256;   // shared-memory offset of the slots, same in every CTA
         int tile, split, gemm;
         umma_decode_unit(p, blockIdx.x, tile, split, gemm);
         int mb, nb;
@@ -510,22 +541,32 @@ umma_bf16_kernel(const __grid_constant__ CUtensorMap tmap_a,
         tc_fence_after_sync();
         cluster_wait();                                  // phase A: every CTA of the cluster is running
         if (ok) {
+            // Slot layout: 16-byte group g (columns 4g..4g+3) of row t at g * 512 + (t ^ g) * 16, so one
+            // warp instruction writes 512 contiguous bytes of the remote slot (rows scattered over
+            // 32 different 128-byte lines made the remote stores several times slower) and both the
+            // writes and the reads below stay free of bank conflicts.
 #pragma unroll 1
-            for (int c = 0; c < NC; ++c) {
-                uint32_t v[32];
-                tmem_ld_32x32(tmem_base + c * 32 + (static_cast<uint32_t>(quarter * 32) << 16), v);
+            for (int c = 0; c < NC; c += 2) {
+                uint32_t v0[32], v1[32];
+                const uint32_t taddr = tmem_base + c * 32 + (static_cast<uint32_t>(quarter * 32) << 16);
+                tmem_ld_32x32(taddr, v0);
+                tmem_ld_32x32(taddr + 32, v1);
                 tmem_ld_wait();
-                const uint32_t u = quarter * NC + c, owner = u % S, slot = (u / S) * S + rank;
-                const uint32_t dst = map_to_cta(recv + slot * 4096u + lane * 128u, owner);
+                const uint32_t u0 = quarter * NC + c, u1 = u0 + 1;
+                const uint32_t d0 = map_to_cta(recv + ((u0 / S) * S + rank) * 4096u, u0 % S);
+                const uint32_t d1 = map_to_cta(recv + ((u1 / S) * S + rank) * 4096u, u1 % S);
 #pragma unroll
                 for (int g = 0; g < 8; ++g)
-                    st_cluster_v4(dst + ((g ^ (lane & 7)) << 4), v[4 * g], v[4 * g + 1], v[4 * g + 2], v[4 * g + 3]);
+                    st_cluster_v4(d0 + g * 512 + ((lane ^ g) << 4), v0[4 * g], v0[4 * g + 1], v0[4 * g + 2], v0[4 * g + 3]);
+#pragma unroll
+                for (int g = 0; g < 8; ++g)
+                    st_cluster_v4(d1 + g * 512 + ((lane ^ g) << 4), v1[4 * g], v1[4 * g + 1], v1[4 * g + 2], v1[4 * g + 3]);
             }
         }
         cluster_arrive();                                // phase B: this thread's pieces are delivered
         cluster_wait();                                  //          ... and so are everybody else's
         if (ok) {
-            const uint8_t* recv_gen = gen_base + STAGES * STAGE + 256 + UMMA_EPI_STAGING;
+            const uint8_t* recv_gen = gen_base + STAGES * STAGE + UMMA_EPI_STAGING + 256;
             const int cg = lane & 7, rsub = lane >> 3;
 #pragma unroll 1
             for (int c = 0; c < NC; ++c) {
@@ -536,13 +577,13 @@ umma_bf16_kernel(const __grid_constant__ CUtensorMap tmap_a,
 #pragma unroll
                 for (int i = 0; i < 8; ++i) {
                     const int r = 4 * i + rsub;
-                    acc4[i] = *reinterpret_cast<const float4*>(slot0 + r * 128 + ((cg ^ (r & 7)) << 4));
+                    acc4[i] = *reinterpret_cast<const float4*>(slot0 + cg * 512 + ((r ^ cg) << 4));
                 }
                 for (uint32_t sp = 1; sp < S; ++sp) {     // split order: the sum does not depend on timing
 #pragma unroll
                     for (int i = 0; i < 8; ++i) {
                         const int r = 4 * i + rsub;
-                        const float4 t4 = *reinterpret_cast<const float4*>(slot0 + sp * 4096u + r * 128 + ((cg ^ (r & 7)) << 4));
+                        const float4 t4 = *reinterpret_cast<const float4*>(slot0 + sp * 4096u + cg * 512 + ((r ^ cg) << 4));
                         acc4[i].x += t4.x; acc4[i].y += t4.y; acc4[i].z += t4.z; acc4[i].w += t4.w;
                     }
                 }
@@ -570,19 +611,27 @@ umma_bf16_kernel(const __grid_constant__ CUtensorMap tmap_a,
             tc_fence_after_sync();
             const int row0 = mb * UMMA_BM + quarter * 32;
             const bool empty_k = kb1 <= kb0;
-            uint8_t* staging = gen_base + STAGES * STAGE + 256 + (warp - 2) * 4096;
+            uint8_t* staging = gen_base + STAGES * STAGE + (warp - 2) * 8192;
+            // two 32-column chunks per round: one wait for both tensor-memory loads
 #pragma unroll 1
-            for (int c0 = 0; c0 < BN; c0 += 32) {
-                uint32_t v[32];
-                tmem_ld_32x32(tmem_base + acc * BN + c0 + (static_cast<uint32_t>(quarter * 32) << 16),
-                              v);
+            for (int c0 = 0; c0 < BN; c0 += 64) {
+                uint32_t v0[32], v1[32];
+                const uint32_t taddr = tmem_base + acc * BN + c0 + (static_cast<uint32_t>(quarter * 32) << 16);
+                tmem_ld_32x32(taddr, v0);
+                tmem_ld_32x32(taddr + 32, v1);
                 tmem_ld_wait();
-                umma_store_chunk(p, v, row0, lane, nb * BN + c0, split, gemm, empty_k, staging);
+                umma_store_chunk(p, &tmap_c, v0, row0, lane, nb * BN + c0, split, gemm, empty_k, staging);
+                __syncwarp();
+                umma_store_chunk(p, &tmap_c, v1, row0, lane, nb * BN + c0 + 32, split, gemm, empty_k, staging + 4096);
                 __syncwarp();
             }
             tc_fence_before_sync();
             mbar_arrive(tempty_bar(acc));
         }
+        // the TMA stores of this warp must have read their staging buffers (and, to be safe, be
+        // complete) before the CTA's shared memory goes away
+        if (lane == 0) bulk_wait_all();
+        __syncwarp();
     } else if (B_VNNI) {
         // ------------------------------------------------ VNNI re-layout warps (6..9)
         static_assert(VNNI_LOOKAHEAD < STAGES, "copies in flight must fit the ring");

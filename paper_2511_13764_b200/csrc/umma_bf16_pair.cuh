@@ -24,14 +24,14 @@ namespace nk {
 
 __host__ __device__ constexpr int pair_stage_bytes(int BN) { return UMMA_A_STAGE_BYTES + (BN / 2) * UMMA_BK * 2; }
 __host__ __device__ constexpr int pair_smem_bytes(int BN, int stages) {
-    return stages * pair_stage_bytes(BN) + 1024 + 256 + UMMA_EPI_STAGING;
+    return stages * pair_stage_bytes(BN) + 1024 + UMMA_EPI_STAGING + 256;
 }
 
 // UmmaParams as for the single-CTA kernel, with tiles_m counted in 256-row tiles.
 template <int BN, int STAGES, bool B_VNNI>
 __global__ void __launch_bounds__(B_VNNI ? 320 : 192, 1)
-umma_bf16_pair_kernel(const __grid_constant__ CUtensorMap tmap_a,
-                      const __grid_constant__ CUtensorMap tmap_b, const UmmaParams p) {
+umma_bf16_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ CUtensorMap tmap_b,
+                      const __grid_constant__ CUtensorMap tmap_c, const UmmaParams p) {
     static_assert(BN == 128 || BN == 256, "pair tile N");
     constexpr int HALF = BN / 2;                       // B columns held by each CTA
     constexpr int B_STAGE = HALF * UMMA_BK * 2;
@@ -41,14 +41,14 @@ umma_bf16_pair_kernel(const __grid_constant__ CUtensorMap tmap_a,
 
     extern __shared__ uint8_t smem_raw[];
     const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
-    const uint32_t bar_base = smem_base + STAGES * STAGE;
+    const uint32_t bar_base = smem_base + STAGES * STAGE + UMMA_EPI_STAGING;   // stages, epilogue staging, barriers
     auto full_bar = [&](int s) { return bar_base + 8u * s; };
     auto empty_bar = [&](int s) { return bar_base + 8u * (STAGES + s); };
     auto tfull_bar = [&](int a) { return bar_base + 8u * (2 * STAGES + a); };
     auto tempty_bar = [&](int a) { return bar_base + 8u * (2 * STAGES + 2 + a); };
     uint8_t* gen_base = smem_raw + (smem_base - smem_u32(smem_raw));
     volatile uint32_t* tmem_slot =
-        reinterpret_cast<volatile uint32_t*>(gen_base + STAGES * STAGE + 8 * (2 * STAGES + 4));
+        reinterpret_cast<volatile uint32_t*>(gen_base + STAGES * STAGE + UMMA_EPI_STAGING + 8 * (2 * STAGES + 4));
     volatile uint32_t* abort_flag = tmem_slot + 1;
 
     const int warp = threadIdx.x >> 5;
@@ -70,6 +70,7 @@ umma_bf16_pair_kernel(const __grid_constant__ CUtensorMap tmap_a,
         fence_mbar_init();
         tma_prefetch_desc(&tmap_a);
         if (!B_VNNI) tma_prefetch_desc(&tmap_b);
+        if (p.tma_store) tma_prefetch_desc(&tmap_c);
     }
     if (warp == 1) {
         tmem_alloc_pair(smem_u32(const_cast<uint32_t*>(tmem_slot)), TMEM_COLS);
@@ -229,18 +230,24 @@ umma_bf16_pair_kernel(const __grid_constant__ CUtensorMap tmap_a,
             tc_fence_after_sync();
             const int row0 = mb * BM2 + static_cast<int>(rank) * UMMA_BM + quarter * 32;
             const bool empty_k = kb1 <= kb0;
-            uint8_t* staging = gen_base + STAGES * STAGE + 256 + (warp - 2) * 4096;
+            uint8_t* staging = gen_base + STAGES * STAGE + (warp - 2) * 8192;
 #pragma unroll 1
-            for (int c0 = 0; c0 < BN; c0 += 32) {
-                uint32_t v[32];
-                tmem_ld_32x32(tmem_base + acc * BN + c0 + (static_cast<uint32_t>(quarter * 32) << 16), v);
+            for (int c0 = 0; c0 < BN; c0 += 64) {   // two 32-column chunks per round
+                uint32_t v0[32], v1[32];
+                const uint32_t taddr = tmem_base + acc * BN + c0 + (static_cast<uint32_t>(quarter * 32) << 16);
+                tmem_ld_32x32(taddr, v0);
+                tmem_ld_32x32(taddr + 32, v1);
                 tmem_ld_wait();
-                umma_store_chunk(p, v, row0, lane, nb * BN + c0, split, gemm, empty_k, staging);
+                umma_store_chunk(p, &tmap_c, v0, row0, lane, nb * BN + c0, split, gemm, empty_k, staging);
+                __syncwarp();
+                umma_store_chunk(p, &tmap_c, v1, row0, lane, nb * BN + c0 + 32, split, gemm, empty_k, staging + 4096);
                 __syncwarp();
             }
             tc_fence_before_sync();
             mbar_arrive_cluster(map_to_cta(tempty_bar(acc), 0));
         }
+        if (lane == 0) bulk_wait_all();   // this warp's TMA stores are done with the staging buffers
+        __syncwarp();
     } else if (B_VNNI) {
         // ------------------------------------------------ VNNI re-layout warps (both CTAs)
         // Each CTA re-lays its own HALF columns (see vnni_issue_stage) and reports each landed
