@@ -69,7 +69,7 @@ typedef enum { NK_EPI_NONE = 0, NK_EPI_BIAS_RELU = 1 } nk_epilogue_t;
 #define NK_FLAG_SCALAR_FMA 0x80u  /* FP32 128 x 128 tile: scalar FFMA instead of packed fma.f32x2   */
 #define NK_FLAG_SEPARATE_REDUCE 0x100000u /* BF16 split-K: always write FP32 partials to the workspace and sum
                                              them in a second kernel, never inside a thread-block cluster  */
-#define NK_FLAG_LSU_STORE 0x200000u /* BF16 kernels: store FP32 C with per-thread stores, never by TMA        */
+#define NK_FLAG_LSU_STORE 0x200000u /* BF16 kernels: store C with per-thread stores, never by TMA             */
 #define NK_FLAG_SPLITK_SHIFT 8    /* bits 8..15: force this many K splits (0 = auto)          */
 #define NK_FLAG_TILE_N_SHIFT 16   /* bits 16..19: force tile N: 1=32 2=64 3=128 4=256 (0 = auto) */
 

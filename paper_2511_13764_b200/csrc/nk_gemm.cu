@@ -60,7 +60,7 @@ struct nk_gemm_s {
     // cached tensor maps
     CUtensorMap tmap_a, tmap_b, tmap_c;
     const void *cached_a, *cached_b, *cached_c;
-    bool tma_store;        // FP32 row-major C without beta or K split: stored by TMA, 32 x 32 boxes
+    bool tma_store;        // row-major C without beta or K split: stored by TMA, 32 x 32 boxes
     nk::EncodeTiledFn encode;
     char name[96];
     char cuda_err[256];
@@ -355,17 +355,21 @@ static nk_status_t encode_maps(nk_gemm_s* p, const void* A, const void* B) {
     return NK_OK;
 }
 
-// C row-major FP32 [gemms][M][N] as (n, m, gemm): the epilogue stores 32 x 32 boxes from a
-// 128-byte-swizzled staging tile; the TMA unit drops whatever lies beyond M or N.
+// C row-major [gemms][M][N] as (n, m, gemm): the epilogue stores 32 x 32 boxes from a swizzled
+// staging tile; the TMA unit drops whatever lies beyond M or N.
 static nk_status_t encode_c_map(nk_gemm_s* p, void* C) {
     if (!p->tma_store || p->cached_c == C) return NK_OK;
     const nk_gemm_desc_t& d = p->d;
+    const bool bf16 = d.out_dtype == NK_BF16;
+    const cuuint64_t es_bytes = bf16 ? 2 : 4;
     cuuint64_t dims[3] = {static_cast<cuuint64_t>(d.N), static_cast<cuuint64_t>(d.M), static_cast<cuuint64_t>(p->gemms)};
-    cuuint64_t strides[2] = {static_cast<cuuint64_t>(d.N) * 4, static_cast<cuuint64_t>(p->stride_c) * 4};
+    cuuint64_t strides[2] = {static_cast<cuuint64_t>(d.N) * es_bytes, static_cast<cuuint64_t>(p->stride_c) * es_bytes};
     cuuint32_t box[3] = {32, 32, 1};
     cuuint32_t es[3] = {1, 1, 1};
-    CUresult r = p->encode(&p->tmap_c, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 3, C, dims, strides, box, es,
-                           CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+    // a box row is 128 bytes of FP32 (128-byte swizzle) or 64 bytes of BF16 (64-byte swizzle)
+    CUresult r = p->encode(&p->tmap_c, bf16 ? CU_TENSOR_MAP_DATA_TYPE_BFLOAT16 : CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 3, C,
+                           dims, strides, box, es, CU_TENSOR_MAP_INTERLEAVE_NONE,
+                           bf16 ? CU_TENSOR_MAP_SWIZZLE_64B : CU_TENSOR_MAP_SWIZZLE_128B,
                            CU_TENSOR_MAP_L2_PROMOTION_NONE, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
     if (r != CUDA_SUCCESS) {
         snprintf(p->cuda_err, sizeof(p->cuda_err), "cuTensorMapEncodeTiled(C) failed: %d", (int)r);
@@ -664,7 +668,7 @@ nk_status_t nk_gemm_create(const nk_gemm_desc_t* desc, nk_gemm_t* out) {
                 p->stages = umma_stages_for(p->bn);
             }
         }
-        p->tma_store = d.out_dtype == NK_F32 && d.layout_c == NK_ROW_MAJOR && d.beta == 0 && p->splits == 1 &&
+        p->tma_store = d.layout_c == NK_ROW_MAJOR && d.beta == 0 && p->splits == 1 &&
                        !(d.flags & NK_FLAG_LSU_STORE);
         p->ws_repack_bytes = p->b_repack ? align_up(static_cast<size_t>(d.K) * d.N * 2, 256) : 0;
         p->ws_partial_bytes = (p->splits > 1 && !p->cluster_reduce) ? static_cast<size_t>(p->splits) * p->gemms * d.M * d.N * 4 : 0;

@@ -49,7 +49,7 @@ struct UmmaParams {
     int gemms;          // independent GEMMs in one launch (batched matmul): C_g = A_g . B_g; else 1
     long long stride_c; // elements from C_g to C_g+1
     int c_blocked;      // C is stored as [M/32][N/32][32][32]: each 32 x 32 chunk is one block
-    int tma_store;      // C (FP32, row-major, no beta, no K split) leaves through TMA stores of 32 x 32 boxes
+    int tma_store;      // C (row-major, no beta, no K split) leaves through TMA stores of 32 x 32 boxes
     int kb_per_split;   // ceil(kb_total / splits)
     int group_m;        // raster: this many M tiles sweep N together
     int a_blocked;      // A tensor map is the 4-D blocked view
@@ -114,9 +114,14 @@ __device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi) {
 // row t kept at chunk g ^ (t & 7): conflict-free both ways) so that every store instruction
 // writes four whole 128-byte row segments instead of 32 scattered 16-byte pieces.  BF16 rows
 // (64 bytes each) are stored directly.  Columns are predicated in groups (N is a multiple of 8).
+//
+// `staging` is the warp's 8 KB of shared memory: two 4 KB (FP32) or two 2 KB (BF16) tiles used
+// alternately (`parity`) as TMA-store sources; with BF16 output the bias slice of the tile
+// (`bias_smem`, one value per tile column, fetched while the K loop was still running) sits
+// behind them.
 __device__ __forceinline__ void umma_store_chunk(const UmmaParams& p, const CUtensorMap* tmap_c, uint32_t (&v)[32],
                                                  int row0, int lane, int col0, int split, int gemm, bool empty_k,
-                                                 uint8_t* staging) {
+                                                 uint8_t* staging, int parity, const uint16_t* bias_smem) {
     if (col0 >= p.N || row0 >= p.M) return;           // warp-uniform
     const int row = row0 + lane;
     const size_t c_base = static_cast<size_t>(gemm) * p.stride_c;   // this GEMM's C inside the batch
@@ -164,7 +169,7 @@ __device__ __forceinline__ void umma_store_chunk(const UmmaParams& p, const CUte
 #pragma unroll
         for (int g = 0; g < 4; ++g) {
             if (col0 + 8 * g >= p.N) break;
-            const uint4 b = __ldg(bsrc + g);
+            const uint4 b = bias_smem ? reinterpret_cast<const uint4*>(bias_smem)[g] : __ldg(bsrc + g);
             const uint32_t w[4] = {b.x, b.y, b.z, b.w};
 #pragma unroll
             for (int j = 0; j < 4; ++j) {
@@ -174,6 +179,29 @@ __device__ __forceinline__ void umma_store_chunk(const UmmaParams& p, const CUte
                 v[8 * g + 2 * j + 1] = __float_as_uint(fmaxf(x1, 0.0f));
             }
         }
+    }
+    if (!to_partial && p.out_bf16 && p.tma_store) {
+        // BF16 rows (64 bytes) -> staging, 16-byte chunk g of row t at chunk g ^ ((t >> 1) & 3) (the
+        // 64-byte swizzle: conflict-free stores) -> one TMA store of the 32 x 32 box
+        uint8_t* tile = staging + parity * 2048;
+        if (lane == 0) bulk_wait_read<1>();          // the store issued two chunks ago has read this tile
+        __syncwarp();
+#pragma unroll
+        for (int g = 0; g < 4; ++g) {
+            uint4 o;
+            o.x = pack_bf16x2(__uint_as_float(v[8 * g]), __uint_as_float(v[8 * g + 1]));
+            o.y = pack_bf16x2(__uint_as_float(v[8 * g + 2]), __uint_as_float(v[8 * g + 3]));
+            o.z = pack_bf16x2(__uint_as_float(v[8 * g + 4]), __uint_as_float(v[8 * g + 5]));
+            o.w = pack_bf16x2(__uint_as_float(v[8 * g + 6]), __uint_as_float(v[8 * g + 7]));
+            *reinterpret_cast<uint4*>(tile + lane * 64 + ((g ^ ((lane >> 1) & 3)) << 4)) = o;
+        }
+        fence_proxy_async_smem();
+        __syncwarp();
+        if (lane == 0) {
+            tma_store_3d(tmap_c, smem_u32(tile), col0, row0, gemm);
+            bulk_commit();
+        }
+        return;
     }
     if (!to_partial && p.out_bf16) {
         if (row >= p.M) return;
@@ -194,8 +222,9 @@ __device__ __forceinline__ void umma_store_chunk(const UmmaParams& p, const CUte
     // 128-byte swizzle) -> global, either as one TMA store of the 32 x 32 box (the TMA unit writes
     // whole lines and clips the ragged edge; the warp only pays eight shared-memory stores), or with
     // per-thread stores of four 128-byte row segments per instruction.
+    staging += parity * 4096;
     if (p.tma_store) {
-        // the caller alternates two buffers: the store issued two chunks ago has read this one
+        // two tiles used alternately: the store issued two chunks ago has read this one
         if (lane == 0) bulk_wait_read<1>();
         __syncwarp();
     }
@@ -274,6 +303,22 @@ __device__ __forceinline__ void umma_finish_piece(const UmmaParams& p, float4 (&
             *reinterpret_cast<float4*>(static_cast<float*>(p.C) + off) = v;
         }
     }
+}
+
+// With BF16 output the warp's staging tiles take 4 KB of its 8 KB: the bias slice of the tile
+// (BN values) is parked behind them before the wait for the accumulator, so that its global
+// latency is hidden behind the K loop instead of being paid in every chunk.
+template <int BN>
+__device__ __forceinline__ const uint16_t* umma_fetch_bias(const UmmaParams& p, uint8_t* staging, int col_tile0, int lane) {
+    if (!p.epilogue || !p.out_bf16 || p.splits > 1) return nullptr;
+    uint4* dst = reinterpret_cast<uint4*>(staging + 4096);
+    if (lane < BN / 8) {
+        const int col = col_tile0 + 8 * lane;
+        dst[lane] = col < p.N ? __ldg(reinterpret_cast<const uint4*>(static_cast<const uint16_t*>(p.bias) + col))
+                              : make_uint4(0u, 0u, 0u, 0u);
+    }
+    __syncwarp();
+    return reinterpret_cast<const uint16_t*>(dst);
 }
 
 // Re-layout of a VNNI-blocked B operand (Figure 1 of the paper: [k/2][n][2] inside every 32 x 32
@@ -603,6 +648,8 @@ umma_bf16_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_consta
             const int kb0 = split * p.kb_per_split;
             const int kb1 = min(p.kb_total, kb0 + p.kb_per_split);
             const int acc = local & 1;
+            uint8_t* staging = gen_base + STAGES * STAGE + (warp - 2) * 8192;
+            const uint16_t* bias_smem = umma_fetch_bias<BN>(p, staging, nb * BN, lane);
             if (!mbar_wait(tfull_bar(acc), (local >> 1) & 1u, abort_flag)) {
                 if (lane == 0) give_up(0x400u + acc);
                 ok = false;
@@ -611,7 +658,6 @@ umma_bf16_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_consta
             tc_fence_after_sync();
             const int row0 = mb * UMMA_BM + quarter * 32;
             const bool empty_k = kb1 <= kb0;
-            uint8_t* staging = gen_base + STAGES * STAGE + (warp - 2) * 8192;
             // two 32-column chunks per round: one wait for both tensor-memory loads
 #pragma unroll 1
             for (int c0 = 0; c0 < BN; c0 += 64) {
@@ -620,9 +666,11 @@ umma_bf16_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_consta
                 tmem_ld_32x32(taddr, v0);
                 tmem_ld_32x32(taddr + 32, v1);
                 tmem_ld_wait();
-                umma_store_chunk(p, &tmap_c, v0, row0, lane, nb * BN + c0, split, gemm, empty_k, staging);
+                umma_store_chunk(p, &tmap_c, v0, row0, lane, nb * BN + c0, split, gemm, empty_k, staging, 0,
+                                 bias_smem ? bias_smem + c0 : nullptr);
                 __syncwarp();
-                umma_store_chunk(p, &tmap_c, v1, row0, lane, nb * BN + c0 + 32, split, gemm, empty_k, staging + 4096);
+                umma_store_chunk(p, &tmap_c, v1, row0, lane, nb * BN + c0 + 32, split, gemm, empty_k, staging, 1,
+                                 bias_smem ? bias_smem + c0 + 32 : nullptr);
                 __syncwarp();
             }
             tc_fence_before_sync();

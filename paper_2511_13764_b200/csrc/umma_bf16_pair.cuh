@@ -222,6 +222,8 @@ umma_bf16_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_c
             const int kb0 = split * p.kb_per_split;
             const int kb1 = min(p.kb_total, kb0 + p.kb_per_split);
             const int acc = local & 1;
+            uint8_t* staging = gen_base + STAGES * STAGE + (warp - 2) * 8192;
+            const uint16_t* bias_smem = umma_fetch_bias<BN>(p, staging, nb * BN, lane);
             if (!mbar_wait(tfull_bar(acc), (local >> 1) & 1u, abort_flag)) {
                 if (lane == 0) give_up(0x400u + acc);
                 ok = false;
@@ -230,7 +232,6 @@ umma_bf16_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_c
             tc_fence_after_sync();
             const int row0 = mb * BM2 + static_cast<int>(rank) * UMMA_BM + quarter * 32;
             const bool empty_k = kb1 <= kb0;
-            uint8_t* staging = gen_base + STAGES * STAGE + (warp - 2) * 8192;
 #pragma unroll 1
             for (int c0 = 0; c0 < BN; c0 += 64) {   // two 32-column chunks per round
                 uint32_t v0[32], v1[32];
@@ -238,9 +239,11 @@ umma_bf16_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_c
                 tmem_ld_32x32(taddr, v0);
                 tmem_ld_32x32(taddr + 32, v1);
                 tmem_ld_wait();
-                umma_store_chunk(p, &tmap_c, v0, row0, lane, nb * BN + c0, split, gemm, empty_k, staging);
+                umma_store_chunk(p, &tmap_c, v0, row0, lane, nb * BN + c0, split, gemm, empty_k, staging, 0,
+                                 bias_smem ? bias_smem + c0 : nullptr);
                 __syncwarp();
-                umma_store_chunk(p, &tmap_c, v1, row0, lane, nb * BN + c0 + 32, split, gemm, empty_k, staging + 4096);
+                umma_store_chunk(p, &tmap_c, v1, row0, lane, nb * BN + c0 + 32, split, gemm, empty_k, staging, 1,
+                                 bias_smem ? bias_smem + c0 + 32 : nullptr);
                 __syncwarp();
             }
             tc_fence_before_sync();
