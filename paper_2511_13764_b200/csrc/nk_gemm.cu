@@ -112,7 +112,6 @@ static cudaError_t allow_smem(K kernel, int bytes) {
 }
 
 static int umma_stages_for(int bn) { return bn == 256 ? 4 : bn == 128 ? 6 : 8; }
-static int cluster_stages_for(int bn) { return bn == 128 ? 4 : 6; }   // the receive slots take the room of the other stages
 
 // Plan-time choice of (single CTA | CTA pair) x tile N x K splits for the BF16 kernel: the
 // counterpart of the paper's tile-size selection (Section 5a, found there by manual search).
@@ -125,15 +124,16 @@ struct UmmaChoice { bool pair; int bn; int splits; double us; };
 static int desc_batch(const nk_gemm_desc_t& d) { return (d.batch > 1 && !d.batch_independent) ? static_cast<int>(d.batch) : 1; }
 static int desc_gemms(const nk_gemm_desc_t& d) { return (d.batch > 1 && d.batch_independent) ? static_cast<int>(d.batch) : 1; }
 
-// K splits can meet inside a cluster (no partials in global memory, no second kernel) when the
-// plan is one CTA per 128-row tile, at most 128 columns wide, 2, 4 or 8 splits, and all its units
-// fit the GPU at once (clusters of 8 leave a few SMs of every GPC unused: allow for that).
+// K splits can meet inside a cluster (no partials in global memory, no second kernel) when there
+// are 2, 4 or 8 of them (2 or 4 pairs), and all the units of the plan fit the GPU at once (large
+// clusters leave a few SMs of every GPC unused: allow for that; the driver is asked at creation).
 static bool cluster_reduce_fits(const nk_gemm_desc_t& d, int sms, bool pair, int bn, int eff_splits) {
-    if (pair || bn > 128 || (d.flags & NK_FLAG_SEPARATE_REDUCE)) return false;
-    if (eff_splits != 2 && eff_splits != 4 && eff_splits != 8) return false;
-    const int64_t units = static_cast<int64_t>(desc_gemms(d)) * ceil_div(d.M, UMMA_BM) * ceil_div(d.N, bn) * eff_splits;
-    const int usable = eff_splits == 8 ? sms - sms / 9 : eff_splits == 4 ? sms - 4 : sms;
-    return units <= usable;
+    if (d.flags & NK_FLAG_SEPARATE_REDUCE) return false;
+    if (eff_splits != 2 && eff_splits != 4 && !(eff_splits == 8 && !pair)) return false;
+    const int cluster = pair ? 2 * eff_splits : eff_splits;
+    const int64_t ctas = static_cast<int64_t>(desc_gemms(d)) * ceil_div(d.M, pair ? 2 * UMMA_BM : UMMA_BM) * ceil_div(d.N, bn) * cluster;
+    const int usable = cluster == 8 ? sms - sms / 9 : cluster == 4 ? sms - 4 : sms;
+    return ctas <= usable;
 }
 
 static double umma_model_us(const nk_gemm_desc_t& d, int sms, bool pair, int bn, int splits) {
@@ -200,7 +200,6 @@ static void choose_umma(nk_gemm_s* p) {
     p->splits = splits;
     p->group_m = 8;
     p->cluster_reduce = splits > 1 && cluster_reduce_fits(d, sms, best.pair, best.bn, splits);
-    if (p->cluster_reduce) p->stages = cluster_stages_for(best.bn);
 }
 
 // Plan-time choice of tile and K splits for the FP32 kernel (the counterpart of the paper's
@@ -397,39 +396,50 @@ static cudaError_t launch_umma(nk_gemm_s* p, const UmmaParams& up, int grid, cud
     }
 }
 
-// Cluster split-K variants: BN = 128 with 4 stages, BN = 64 with 6 (the receive slots take the
-// room of the other stages); the cluster is `splits` CTAs wide and the grid is exactly the units.
-template <int BN, int STAGES, bool VNNI>
-static cudaError_t launch_cluster_t(nk_gemm_s* p, const UmmaParams& up, int units, int splits, cudaStream_t st,
-                                    int* max_clusters) {
+// Cluster split-K variants of both kernels: the cluster is `splits` CTAs (or pairs) wide and the
+// grid is exactly the units; with `max_clusters` set only the occupancy of one cluster is queried.
+template <typename Kernel>
+static cudaError_t launch_clustered(Kernel kernel, nk_gemm_s* p, const UmmaParams& up, int ctas, int cluster, int threads,
+                                    int smem, cudaStream_t st, int* max_clusters) {
     cudaLaunchConfig_t cfg;
     memset(&cfg, 0, sizeof(cfg));
-    cfg.gridDim = dim3(static_cast<unsigned>(units));
-    cfg.blockDim = dim3(VNNI ? 320 : 192);
-    cfg.dynamicSmemBytes = umma_cluster_smem_bytes(BN, STAGES);
+    cfg.gridDim = dim3(static_cast<unsigned>(max_clusters ? cluster : ctas));
+    cfg.blockDim = dim3(static_cast<unsigned>(threads));
+    cfg.dynamicSmemBytes = static_cast<size_t>(smem);
     cfg.stream = st;
     cudaLaunchAttribute attr;
     attr.id = cudaLaunchAttributeClusterDimension;
-    attr.val.clusterDim.x = static_cast<unsigned>(splits);
+    attr.val.clusterDim.x = static_cast<unsigned>(cluster);
     attr.val.clusterDim.y = 1;
     attr.val.clusterDim.z = 1;
     cfg.attrs = &attr;
     cfg.numAttrs = 1;
-    if (max_clusters) {   // occupancy query only
-        cfg.gridDim = dim3(static_cast<unsigned>(splits));
-        return cudaOccupancyMaxActiveClusters(max_clusters, umma_bf16_kernel<BN, STAGES, VNNI, true>, &cfg);
-    }
-    return cudaLaunchKernelEx(&cfg, umma_bf16_kernel<BN, STAGES, VNNI, true>, p->tmap_a, p->tmap_b, p->tmap_c, up);
+    if (max_clusters) return cudaOccupancyMaxActiveClusters(max_clusters, kernel, &cfg);
+    return cudaLaunchKernelEx(&cfg, kernel, p->tmap_a, p->tmap_b, p->tmap_c, up);
 }
 
+// `units` = tiles x splits; the single-CTA kernel runs one CTA per unit, the pair kernel two.
 static cudaError_t launch_cluster(nk_gemm_s* p, const UmmaParams& up, int units, int splits, cudaStream_t st,
                                   int* max_clusters) {
     const bool v = p->b_vnni_inkernel;
+    const int th = v ? 320 : 192;
+#define NK_CL(K, ctas, cl, smem) launch_clustered(K, p, up, ctas, cl, th, smem, st, max_clusters)
+    if (p->pair) {
+        if (p->bn == 256)
+            return v ? NK_CL((umma_bf16_pair_kernel<256, 6, true, true>), 2 * units, 2 * splits, pair_smem_bytes(256, 6))
+                     : NK_CL((umma_bf16_pair_kernel<256, 6, false, true>), 2 * units, 2 * splits, pair_smem_bytes(256, 6));
+        return v ? NK_CL((umma_bf16_pair_kernel<128, 8, true, true>), 2 * units, 2 * splits, pair_smem_bytes(128, 8))
+                 : NK_CL((umma_bf16_pair_kernel<128, 8, false, true>), 2 * units, 2 * splits, pair_smem_bytes(128, 8));
+    }
+    if (p->bn == 256)
+        return v ? NK_CL((umma_bf16_kernel<256, 4, true, true>), units, splits, umma_smem_bytes(256, 4))
+                 : NK_CL((umma_bf16_kernel<256, 4, false, true>), units, splits, umma_smem_bytes(256, 4));
     if (p->bn == 128)
-        return v ? launch_cluster_t<128, 4, true>(p, up, units, splits, st, max_clusters)
-                 : launch_cluster_t<128, 4, false>(p, up, units, splits, st, max_clusters);
-    return v ? launch_cluster_t<64, 6, true>(p, up, units, splits, st, max_clusters)
-             : launch_cluster_t<64, 6, false>(p, up, units, splits, st, max_clusters);
+        return v ? NK_CL((umma_bf16_kernel<128, 6, true, true>), units, splits, umma_smem_bytes(128, 6))
+                 : NK_CL((umma_bf16_kernel<128, 6, false, true>), units, splits, umma_smem_bytes(128, 6));
+    return v ? NK_CL((umma_bf16_kernel<64, 8, true, true>), units, splits, umma_smem_bytes(64, 8))
+             : NK_CL((umma_bf16_kernel<64, 8, false, true>), units, splits, umma_smem_bytes(64, 8));
+#undef NK_CL
 }
 
 template <int BN, int STAGES, bool VNNI>
@@ -490,10 +500,16 @@ static cudaError_t prepare_umma_attrs() {
     if ((e = allow_smem(umma_bf16_kernel<256, 4, true>, umma_smem_bytes(256, 4))) != cudaSuccess) return e;
     if ((e = allow_smem(umma_bf16_kernel<128, 6, true>, umma_smem_bytes(128, 6))) != cudaSuccess) return e;
     if ((e = allow_smem(umma_bf16_kernel<64, 8, true>, umma_smem_bytes(64, 8))) != cudaSuccess) return e;
-    if ((e = allow_smem(umma_bf16_kernel<128, 4, false, true>, umma_cluster_smem_bytes(128, 4))) != cudaSuccess) return e;
-    if ((e = allow_smem(umma_bf16_kernel<128, 4, true, true>, umma_cluster_smem_bytes(128, 4))) != cudaSuccess) return e;
-    if ((e = allow_smem(umma_bf16_kernel<64, 6, false, true>, umma_cluster_smem_bytes(64, 6))) != cudaSuccess) return e;
-    if ((e = allow_smem(umma_bf16_kernel<64, 6, true, true>, umma_cluster_smem_bytes(64, 6))) != cudaSuccess) return e;
+    if ((e = allow_smem(umma_bf16_kernel<256, 4, false, true>, umma_smem_bytes(256, 4))) != cudaSuccess) return e;
+    if ((e = allow_smem(umma_bf16_kernel<256, 4, true, true>, umma_smem_bytes(256, 4))) != cudaSuccess) return e;
+    if ((e = allow_smem(umma_bf16_kernel<128, 6, false, true>, umma_smem_bytes(128, 6))) != cudaSuccess) return e;
+    if ((e = allow_smem(umma_bf16_kernel<128, 6, true, true>, umma_smem_bytes(128, 6))) != cudaSuccess) return e;
+    if ((e = allow_smem(umma_bf16_kernel<64, 8, false, true>, umma_smem_bytes(64, 8))) != cudaSuccess) return e;
+    if ((e = allow_smem(umma_bf16_kernel<64, 8, true, true>, umma_smem_bytes(64, 8))) != cudaSuccess) return e;
+    if ((e = allow_smem(umma_bf16_pair_kernel<256, 6, false, true>, pair_smem_bytes(256, 6))) != cudaSuccess) return e;
+    if ((e = allow_smem(umma_bf16_pair_kernel<256, 6, true, true>, pair_smem_bytes(256, 6))) != cudaSuccess) return e;
+    if ((e = allow_smem(umma_bf16_pair_kernel<128, 8, false, true>, pair_smem_bytes(128, 8))) != cudaSuccess) return e;
+    if ((e = allow_smem(umma_bf16_pair_kernel<128, 8, true, true>, pair_smem_bytes(128, 8))) != cudaSuccess) return e;
     return cudaSuccess;
 }
 
@@ -661,14 +677,13 @@ nk_status_t nk_gemm_create(const nk_gemm_desc_t* desc, nk_gemm_t* out) {
         if (p->cluster_reduce) {
             // every cluster of the plan must be resident at once (one unit per CTA): ask the driver
             int n = 0;
-            const int clusters = p->gemms * ceil_div(d.M, UMMA_BM) * ceil_div(d.N, p->bn);
+            const int clusters = p->gemms * ceil_div(d.M, p->pair ? 2 * UMMA_BM : UMMA_BM) * ceil_div(d.N, p->bn);
             if (launch_cluster(p, UmmaParams(), 0, p->splits, nullptr, &n) != cudaSuccess || n < clusters) {
                 cudaGetLastError();
                 p->cluster_reduce = false;
-                p->stages = umma_stages_for(p->bn);
             }
         }
-        p->tma_store = d.layout_c == NK_ROW_MAJOR && d.beta == 0 && p->splits == 1 &&
+        p->tma_store = d.layout_c == NK_ROW_MAJOR && d.beta == 0 && (p->splits == 1 || p->cluster_reduce) &&
                        !(d.flags & NK_FLAG_LSU_STORE);
         p->ws_repack_bytes = p->b_repack ? align_up(static_cast<size_t>(d.K) * d.N * 2, 256) : 0;
         p->ws_partial_bytes = (p->splits > 1 && !p->cluster_reduce) ? static_cast<size_t>(p->splits) * p->gemms * d.M * d.N * 4 : 0;
@@ -781,6 +796,7 @@ nk_status_t nk_gemm_run(nk_gemm_t p, const void* A, const void* B, const void* b
         up.stride_c = p->stride_c;
         up.c_blocked = d.layout_c == NK_BLOCKED32;
         up.tma_store = p->tma_store ? 1 : 0;
+        up.cluster_reduce = p->cluster_reduce ? 1 : 0;
         up.kb_per_split = ceil_div(up.kb_total, p->splits);
         up.group_m = p->group_m;
         up.a_blocked = d.layout_a == NK_BLOCKED32;

@@ -23,11 +23,11 @@
 // the CTA frees its TMEM and exits.
 //
 // Split-K inside a thread-block cluster (CLUSTER_REDUCE): the K splits of one tile are the CTAs
-// of one cluster, one unit per CTA.  After its K loop every CTA scatters its accumulator, in
-// 32 x 32 pieces, straight into the shared memory of the CTA that owns each piece (distributed
-// shared memory); after a cluster barrier every CTA adds the pieces it owns in split order,
-// applies the epilogue and stores them.  No partial ever goes to global memory and there is no
-// second kernel.
+// of one cluster, one unit per CTA.  After its K loop every CTA sends the 32 x 32 pieces of its
+// accumulator that other CTAs own straight into their shared memory (distributed shared memory;
+// they land in the stage ring, which is idle by then); after a cluster barrier every CTA adds
+// the pieces it owns in split order, applies the epilogue and stores them.  No partial ever
+// goes to global memory and there is no second kernel.
 #pragma once
 #include <cuda.h>
 #include <cuda_bf16.h>
@@ -49,7 +49,8 @@ struct UmmaParams {
     int gemms;          // independent GEMMs in one launch (batched matmul): C_g = A_g . B_g; else 1
     long long stride_c; // elements from C_g to C_g+1
     int c_blocked;      // C is stored as [M/32][N/32][32][32]: each 32 x 32 chunk is one block
-    int tma_store;      // C (row-major, no beta, no K split) leaves through TMA stores of 32 x 32 boxes
+    int tma_store;      // C (row-major, no beta, no partials) leaves through TMA stores of 32 x 32 boxes
+    int cluster_reduce; // the K splits of a tile are the CTAs of one cluster and meet in shared memory
     int kb_per_split;   // ceil(kb_total / splits)
     int group_m;        // raster: this many M tiles sweep N together
     int a_blocked;      // A tensor map is the 4-D blocked view
@@ -72,12 +73,9 @@ constexpr int UMMA_EPI_STAGING = 4 * 2 * 4096;   // two 32 x 32 FP32 chunks per 
 __host__ __device__ constexpr int umma_smem_bytes(int BN, int stages) {
     return stages * umma_stage_bytes(BN) + 1024 /*alignment slack*/ + UMMA_EPI_STAGING + 256 /*barriers*/;
 }
-// cluster split-K: one 4 KB slot per (32 x 32 piece this CTA owns, split it comes from); a tile has
-// 4 * BN / 32 pieces shared out over the cluster, so the slots of a CTA always add up to the tile
-__host__ __device__ constexpr int umma_recv_bytes(int BN) { return 4 * (BN / 32) * 4096; }
-__host__ __device__ constexpr int umma_cluster_smem_bytes(int BN, int stages) {
-    return umma_smem_bytes(BN, stages) + umma_recv_bytes(BN);
-}
+// cluster split-K: one 4 KB slot per (32 x 32 piece this CTA owns, split it comes from); the pieces of
+// a CTA's 128 x BN accumulator are shared out over the splits, so a CTA's slots never exceed one
+// accumulator (BN * 512 bytes), which fits the stage ring of every variant
 
 // tile id -> (m block, n block): groups of `group_m` M tiles sweep across N so
 // that CTAs running at the same time share A rows and B columns in L2.
@@ -121,7 +119,8 @@ __device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi) {
 // behind them.
 __device__ __forceinline__ void umma_store_chunk(const UmmaParams& p, const CUtensorMap* tmap_c, uint32_t (&v)[32],
                                                  int row0, int lane, int col0, int split, int gemm, bool empty_k,
-                                                 uint8_t* staging, int parity, const uint16_t* bias_smem) {
+                                                 uint8_t* staging, int parity, const uint16_t* bias_smem,
+                                                 bool to_partial) {
     if (col0 >= p.N || row0 >= p.M) return;           // warp-uniform
     const int row = row0 + lane;
     const size_t c_base = static_cast<size_t>(gemm) * p.stride_c;   // this GEMM's C inside the batch
@@ -134,7 +133,6 @@ __device__ __forceinline__ void umma_store_chunk(const UmmaParams& p, const CUte
 #pragma unroll
         for (int i = 0; i < 32; ++i) v[i] = 0u;
     }
-    const bool to_partial = p.splits > 1;
     if (!to_partial && p.beta && row < p.M) {
         // beta = 1: the accumulation tile starts from the stored C (Algorithm 1 loads the C
         // sub-block before the K loop; adding it here, in FP32, gives the same sum)
@@ -257,60 +255,12 @@ __device__ __forceinline__ void umma_store_chunk(const UmmaParams& p, const CUte
     __syncwarp();   // the buffer is reused by the next chunk
 }
 
-// Tail of the cluster split-K reduction: lane (rsub = lane / 8, cg = lane % 8) holds the summed
-// FP32 values of rows row0 + 4 i + rsub (i = 0..7), columns col0 + 4 cg .. + 3 of one 32 x 32
-// piece; beta, bias + ReLU, the conversion and the store of C follow (Section 6, "MLP").
-__device__ __forceinline__ void umma_finish_piece(const UmmaParams& p, float4 (&s)[8], int row0, int col0, int gemm,
-                                                  int lane) {
-    const int cg = lane & 7, rsub = lane >> 3;
-    const int col = col0 + 4 * cg;
-    if (col >= p.N || row0 >= p.M) return;
-    const size_t c_base = static_cast<size_t>(gemm) * p.stride_c;
-    float4 bv = make_float4(0.f, 0.f, 0.f, 0.f);
-    if (p.epilogue) {
-        const uint2 w = __ldg(reinterpret_cast<const uint2*>(static_cast<const uint16_t*>(p.bias) + col));
-        bv = make_float4(bf16_bits_to_f32(w.x & 0xFFFFu), bf16_bits_to_f32(w.x >> 16),
-                         bf16_bits_to_f32(w.y & 0xFFFFu), bf16_bits_to_f32(w.y >> 16));
-    }
-    const size_t blk_base = (static_cast<size_t>(row0 >> 5) * (p.N >> 5) + (col0 >> 5)) * 1024;
-#pragma unroll
-    for (int i = 0; i < 8; ++i) {
-        const int r = 4 * i + rsub;
-        if (row0 + r >= p.M) continue;
-        const size_t off = c_base + (p.c_blocked ? blk_base + r * 32 + 4 * cg
-                                                 : static_cast<size_t>(row0 + r) * p.N + col);
-        float4 v = s[i];
-        if (p.beta) {
-            if (p.out_bf16) {
-                const uint2 w = *reinterpret_cast<const uint2*>(static_cast<const uint16_t*>(p.C) + off);
-                v.x += bf16_bits_to_f32(w.x & 0xFFFFu); v.y += bf16_bits_to_f32(w.x >> 16);
-                v.z += bf16_bits_to_f32(w.y & 0xFFFFu); v.w += bf16_bits_to_f32(w.y >> 16);
-            } else {
-                const float4 cv = *reinterpret_cast<const float4*>(static_cast<const float*>(p.C) + off);
-                v.x += cv.x; v.y += cv.y; v.z += cv.z; v.w += cv.w;
-            }
-        }
-        if (p.epilogue) {
-            v.x = fmaxf(v.x + bv.x, 0.f); v.y = fmaxf(v.y + bv.y, 0.f);
-            v.z = fmaxf(v.z + bv.z, 0.f); v.w = fmaxf(v.w + bv.w, 0.f);
-        }
-        if (p.out_bf16) {
-            uint2 o;
-            o.x = pack_bf16x2(v.x, v.y);
-            o.y = pack_bf16x2(v.z, v.w);
-            *reinterpret_cast<uint2*>(static_cast<uint16_t*>(p.C) + off) = o;
-        } else {
-            *reinterpret_cast<float4*>(static_cast<float*>(p.C) + off) = v;
-        }
-    }
-}
-
 // With BF16 output the warp's staging tiles take 4 KB of its 8 KB: the bias slice of the tile
 // (BN values) is parked behind them before the wait for the accumulator, so that its global
 // latency is hidden behind the K loop instead of being paid in every chunk.
 template <int BN>
 __device__ __forceinline__ const uint16_t* umma_fetch_bias(const UmmaParams& p, uint8_t* staging, int col_tile0, int lane) {
-    if (!p.epilogue || !p.out_bf16 || p.splits > 1) return nullptr;
+    if (!p.epilogue || !p.out_bf16 || (p.splits > 1 && !p.cluster_reduce)) return nullptr;
     uint4* dst = reinterpret_cast<uint4*>(staging + 4096);
     if (lane < BN / 8) {
         const int col = col_tile0 + 8 * lane;
@@ -319,6 +269,91 @@ __device__ __forceinline__ const uint16_t* umma_fetch_bias(const UmmaParams& p, 
     }
     __syncwarp();
     return reinterpret_cast<const uint16_t*>(dst);
+}
+
+// Epilogue of a cluster split-K CTA.  Its accumulator (128 rows x BN columns, tensor-memory
+// columns 0..BN-1) is cut into 4 * BN / 32 pieces, piece u = quarter * (BN / 32) + chunk; the CTAs
+// that hold the S splits of the same rows have cluster ranks rank0 + s * rank_step.  Piece u
+// belongs to split u % S; the other splits send theirs into slot (u / S) * S + source split of
+// the owner's stage ring (idle by then), the owner's own contribution stays in tensor memory.
+//   phase A  every CTA of the cluster has finished its K loop: the rings may be overwritten
+//   send     tcgen05.ld -> 16-byte stores into the owner's ring (group g of row t at
+//            g * 512 + (t ^ g) * 16: a warp instruction writes 512 contiguous bytes, and both
+//            sides stay free of bank conflicts)
+//   phase B  all pieces have arrived
+//   reduce   every owned piece is summed in split order (the result does not depend on timing)
+//            and leaves through the ordinary chunk epilogue: beta, bias + ReLU, conversion, store
+// Every thread of the cluster passes both barrier phases, also after a wait that gave up.
+template <int BN>
+__device__ __forceinline__ void umma_cluster_epilogue(const UmmaParams& p, const CUtensorMap* tmap_c, uint32_t tmem_base,
+                                                      uint32_t ring, const uint8_t* ring_gen, uint8_t* staging,
+                                                      const uint16_t* bias_smem, int quarter, int lane, uint32_t S,
+                                                      uint32_t split, uint32_t rank0, uint32_t rank_step, int row_cta0,
+                                                      int col_tile0, int gemm, bool ok) {
+    constexpr uint32_t NC = BN / 32;
+    const uint32_t lane_tmem = static_cast<uint32_t>(quarter * 32) << 16;
+    cluster_arrive();
+    cluster_wait();                                      // phase A
+    if (ok) {
+#pragma unroll 1
+        for (uint32_t c = 0; c < NC; ++c) {
+            const uint32_t u = quarter * NC + c, owner = u % S;
+            if (owner == split) continue;                // mine: stays in tensor memory (warp-uniform)
+            uint32_t v[32];
+            tmem_ld_32x32(tmem_base + c * 32 + lane_tmem, v);
+            tmem_ld_wait();
+            const uint32_t dst = map_to_cta(ring + ((u / S) * S + split) * 4096u, rank0 + owner * rank_step);
+#pragma unroll
+            for (int g = 0; g < 8; ++g)
+                st_cluster_v4(dst + g * 512 + ((lane ^ g) << 4), v[4 * g], v[4 * g + 1], v[4 * g + 2], v[4 * g + 3]);
+        }
+    }
+    cluster_arrive();
+    cluster_wait();                                      // phase B
+    if (!ok) return;
+    int parity = 0;
+#pragma unroll 1
+    for (uint32_t c = 0; c < NC; ++c) {
+        const uint32_t u = quarter * NC + c;
+        if (u % S != split) continue;                    // warp-uniform
+        uint32_t own[32], v[32];
+        tmem_ld_32x32(tmem_base + c * 32 + lane_tmem, own);
+        tmem_ld_wait();
+        const uint8_t* slot0 = ring_gen + (u / S) * S * 4096u;
+        // split order s = 0, 1, .., S-1, this CTA's own accumulator taking its place in the row
+#pragma unroll 1
+        for (uint32_t sp = 0; sp < S; ++sp) {
+            if (sp == split) {
+                if (sp == 0) {
+#pragma unroll
+                    for (int i = 0; i < 32; ++i) v[i] = own[i];
+                } else {
+#pragma unroll
+                    for (int i = 0; i < 32; ++i) v[i] = __float_as_uint(__uint_as_float(v[i]) + __uint_as_float(own[i]));
+                }
+                continue;
+            }
+            const uint8_t* slot = slot0 + sp * 4096u;
+#pragma unroll
+            for (int g = 0; g < 8; ++g) {
+                const uint4 t4 = *reinterpret_cast<const uint4*>(slot + g * 512 + ((lane ^ g) << 4));
+                if (sp == 0) {
+                    v[4 * g] = t4.x; v[4 * g + 1] = t4.y; v[4 * g + 2] = t4.z; v[4 * g + 3] = t4.w;
+                } else {
+                    v[4 * g] = __float_as_uint(__uint_as_float(v[4 * g]) + __uint_as_float(t4.x));
+                    v[4 * g + 1] = __float_as_uint(__uint_as_float(v[4 * g + 1]) + __uint_as_float(t4.y));
+                    v[4 * g + 2] = __float_as_uint(__uint_as_float(v[4 * g + 2]) + __uint_as_float(t4.z));
+                    v[4 * g + 3] = __float_as_uint(__uint_as_float(v[4 * g + 3]) + __uint_as_float(t4.w));
+                }
+            }
+        }
+        umma_store_chunk(p, tmap_c, v, row_cta0 + quarter * 32, lane, col_tile0 + static_cast<int>(c) * 32, 0, gemm,
+                         false, staging, parity, bias_smem ? bias_smem + c * 32 : nullptr, false);
+        __syncwarp();
+        parity ^= 1;
+    }
+    if (lane == 0) bulk_wait_all();
+    __syncwarp();
 }
 
 // Re-layout of a VNNI-blocked B operand (Figure 1 of the paper: [k/2][n][2] inside every 32 x 32
@@ -427,9 +462,6 @@ umma_bf16_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_consta
         tc_fence_after_sync();
         tmem_base = *tmem_slot;
     }
-    // cluster split-K, barrier phase A ("this CTA is running: its shared memory may be written"):
-    // arrive now, wait only just before the first remote store
-    if (CLUSTER_REDUCE) cluster_arrive();
 
     const int total_units = p.gemms * p.tiles_m * p.tiles_n * p.splits;
 
@@ -568,73 +600,22 @@ umma_bf16_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_consta
         }
     } else if (warp < 6 && CLUSTER_REDUCE) {
         // ------------------------------------------------ epilogue, K splits reduced inside the cluster
-        // One unit per CTA (grid = units); cluster rank = K split.  Piece u = quarter * NC + chunk of
-        // the 128 x BN tile is owned by CTA u % S and kept there in slot (u / S, source split).
-        constexpr int NC = BN / 32;
-        const int quarter = warp & 3;
-        const uint32_t S = static_cast<uint32_t>(p.splits), rank = cluster_ctarank();
-        const uint32_t recv = bar_base + 256;   // shared-memory offset of the slots, same in every CTA
+        // One unit per CTA (grid = units); cluster rank = K split.
         int tile, split, gemm;
         umma_decode_unit(p, blockIdx.x, tile, split, gemm);
         int mb, nb;
         umma_tile_coords(p, tile, mb, nb);
         bool ok = blockIdx.x < total_units;
+        uint8_t* staging = gen_base + STAGES * STAGE + (warp - 2) * 8192;
+        const uint16_t* bias_smem = umma_fetch_bias<BN>(p, staging, nb * BN, lane);
         if (ok && !mbar_wait(tfull_bar(0), 0u, abort_flag)) {
             if (lane == 0) give_up(0x400u);
             ok = false;
         }
         tc_fence_after_sync();
-        cluster_wait();                                  // phase A: every CTA of the cluster is running
-        if (ok) {
-            // Slot layout: 16-byte group g (columns 4g..4g+3) of row t at g * 512 + (t ^ g) * 16, so one
-            // warp instruction writes 512 contiguous bytes of the remote slot (rows scattered over
-            // 32 different 128-byte lines made the remote stores several times slower) and both the
-            // writes and the reads below stay free of bank conflicts.
-#pragma unroll 1
-            for (int c = 0; c < NC; c += 2) {
-                uint32_t v0[32], v1[32];
-                const uint32_t taddr = tmem_base + c * 32 + (static_cast<uint32_t>(quarter * 32) << 16);
-                tmem_ld_32x32(taddr, v0);
-                tmem_ld_32x32(taddr + 32, v1);
-                tmem_ld_wait();
-                const uint32_t u0 = quarter * NC + c, u1 = u0 + 1;
-                const uint32_t d0 = map_to_cta(recv + ((u0 / S) * S + rank) * 4096u, u0 % S);
-                const uint32_t d1 = map_to_cta(recv + ((u1 / S) * S + rank) * 4096u, u1 % S);
-#pragma unroll
-                for (int g = 0; g < 8; ++g)
-                    st_cluster_v4(d0 + g * 512 + ((lane ^ g) << 4), v0[4 * g], v0[4 * g + 1], v0[4 * g + 2], v0[4 * g + 3]);
-#pragma unroll
-                for (int g = 0; g < 8; ++g)
-                    st_cluster_v4(d1 + g * 512 + ((lane ^ g) << 4), v1[4 * g], v1[4 * g + 1], v1[4 * g + 2], v1[4 * g + 3]);
-            }
-        }
-        cluster_arrive();                                // phase B: this thread's pieces are delivered
-        cluster_wait();                                  //          ... and so are everybody else's
-        if (ok) {
-            const uint8_t* recv_gen = gen_base + STAGES * STAGE + UMMA_EPI_STAGING + 256;
-            const int cg = lane & 7, rsub = lane >> 3;
-#pragma unroll 1
-            for (int c = 0; c < NC; ++c) {
-                const uint32_t u = quarter * NC + c;
-                if (u % S != rank) continue;             // warp-uniform
-                const uint8_t* slot0 = recv_gen + (u / S) * S * 4096u;
-                float4 acc4[8];
-#pragma unroll
-                for (int i = 0; i < 8; ++i) {
-                    const int r = 4 * i + rsub;
-                    acc4[i] = *reinterpret_cast<const float4*>(slot0 + cg * 512 + ((r ^ cg) << 4));
-                }
-                for (uint32_t sp = 1; sp < S; ++sp) {     // split order: the sum does not depend on timing
-#pragma unroll
-                    for (int i = 0; i < 8; ++i) {
-                        const int r = 4 * i + rsub;
-                        const float4 t4 = *reinterpret_cast<const float4*>(slot0 + sp * 4096u + cg * 512 + ((r ^ cg) << 4));
-                        acc4[i].x += t4.x; acc4[i].y += t4.y; acc4[i].z += t4.z; acc4[i].w += t4.w;
-                    }
-                }
-                umma_finish_piece(p, acc4, mb * UMMA_BM + quarter * 32, nb * BN + c * 32, gemm, lane);
-            }
-        }
+        umma_cluster_epilogue<BN>(p, &tmap_c, tmem_base, smem_base, gen_base, staging, bias_smem, warp & 3, lane,
+                                  static_cast<uint32_t>(p.splits), cluster_ctarank(), 0u, 1u, mb * UMMA_BM, nb * BN,
+                                  gemm, ok);
     } else if (warp < 6) {
         // ------------------------------------------------ epilogue
         const int quarter = warp & 3;  // TMEM lanes 32*quarter .. +31 belong to this warp
@@ -667,10 +648,10 @@ umma_bf16_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_consta
                 tmem_ld_32x32(taddr + 32, v1);
                 tmem_ld_wait();
                 umma_store_chunk(p, &tmap_c, v0, row0, lane, nb * BN + c0, split, gemm, empty_k, staging, 0,
-                                 bias_smem ? bias_smem + c0 : nullptr);
+                                 bias_smem ? bias_smem + c0 : nullptr, p.splits > 1);
                 __syncwarp();
                 umma_store_chunk(p, &tmap_c, v1, row0, lane, nb * BN + c0 + 32, split, gemm, empty_k, staging, 1,
-                                 bias_smem ? bias_smem + c0 + 32 : nullptr);
+                                 bias_smem ? bias_smem + c0 + 32 : nullptr, p.splits > 1);
                 __syncwarp();
             }
             tc_fence_before_sync();
@@ -722,7 +703,9 @@ umma_bf16_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_consta
     }
 
     if (CLUSTER_REDUCE && !(warp >= 2 && warp < 6)) {
-        // the cluster barrier counts every thread: the other roles pass both phases here
+        // the cluster barrier counts every thread: the other roles pass both phases here, once
+        // their part of the K loop is over (the producer has seen every stage consumed)
+        cluster_arrive();
         cluster_wait();
         cluster_arrive();
         cluster_wait();

@@ -17,6 +17,11 @@
 //     counts the epilogue threads of both CTAs (the peer arrives remotely);
 //   - cluster-wide barriers fence the start (barriers initialised) and the end (nobody
 //     leaves while its peer may still touch its shared memory or barriers).
+//
+// With CLUSTER_REDUCE the cluster holds S pairs, one per K split of the same 256-row tile
+// (ranks 2s and 2s + 1 are the pair of split s; a pair's leader is its even rank); the
+// accumulators of the S CTAs that own the same 128 rows are summed through distributed shared
+// memory exactly as in the single-CTA kernel (umma_cluster_epilogue).
 #pragma once
 #include "umma_bf16.cuh"
 
@@ -28,7 +33,7 @@ __host__ __device__ constexpr int pair_smem_bytes(int BN, int stages) {
 }
 
 // UmmaParams as for the single-CTA kernel, with tiles_m counted in 256-row tiles.
-template <int BN, int STAGES, bool B_VNNI>
+template <int BN, int STAGES, bool B_VNNI, bool CLUSTER_REDUCE = false>
 __global__ void __launch_bounds__(B_VNNI ? 320 : 192, 1)
 umma_bf16_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ CUtensorMap tmap_b,
                       const __grid_constant__ CUtensorMap tmap_c, const UmmaParams p) {
@@ -53,7 +58,10 @@ umma_bf16_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_c
 
     const int warp = threadIdx.x >> 5;
     const int lane = threadIdx.x & 31;
-    const uint32_t rank = cluster_ctarank();           // 0 = leader
+    const uint32_t crank = cluster_ctarank();          // rank in the cluster (0, 1 unless CLUSTER_REDUCE)
+    const uint32_t rank = crank & 1u;                  // half of the pair: 0 = leader
+    const uint32_t leader = crank & ~1u;               // cluster rank of this pair's leader
+    const uint16_t pair_mask = static_cast<uint16_t>(3u << leader);   // both CTAs of this pair
     const int pair_id = blockIdx.x >> 1;
     const int num_pairs = gridDim.x >> 1;
 
@@ -92,7 +100,7 @@ umma_bf16_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_c
         // ------------------------------------------------ TMA producer (both CTAs)
         const bool a_blk = p.a_blocked != 0;
         const bool b3d = p.b_3d != 0;
-        const uint32_t lead_full0 = map_to_cta(full_bar(0), 0);  // leader's full[0], cluster address
+        const uint32_t lead_full0 = map_to_cta(full_bar(0), leader);  // leader's full[0], cluster address
         int stage = 0;
         uint32_t phase = 0;
         uint32_t sa = smem_base, fb = full_bar(0), lfb = lead_full0;
@@ -197,18 +205,37 @@ umma_bf16_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_c
                         umma_f16_pair_lohi(d_tmem, a_lo + a_s1, a_hi, b_lo + b_s, b_hi, idesc, 1u);
                         umma_f16_pair_lohi(d_tmem, a_lo + a_s2, a_hi, b_lo + 2 * b_s, b_hi, idesc, 1u);
                         umma_f16_pair_lohi(d_tmem, a_lo + a_s3, a_hi, b_lo + 3 * b_s, b_hi, idesc, 1u);
-                        umma_commit_pair(empty_bar(stage), 3);
-                        if (kb == kb1 - 1) umma_commit_pair(tfull_bar(acc), 3);
+                        umma_commit_pair(empty_bar(stage), pair_mask);
+                        if (kb == kb1 - 1) umma_commit_pair(tfull_bar(acc), pair_mask);
                     }
                     accumulate = 1u;
                     __syncwarp();
                     soff += STAGE16;
                     if (++stage == STAGES) { stage = 0; phase ^= 1u; soff = 0; }
                 }
-                if (kb1 <= kb0 && lane == 0) umma_commit_pair(tfull_bar(acc), 3);
+                if (kb1 <= kb0 && lane == 0) umma_commit_pair(tfull_bar(acc), pair_mask);
                 __syncwarp();
             }
         }
+    } else if (warp < 6 && CLUSTER_REDUCE) {
+        // ------------------------------------------------ epilogue, K splits reduced inside the cluster
+        // One unit per pair (grid = 2 x units); this pair's split = its index in the cluster.  The
+        // other splits of this CTA's 128 rows are the CTAs with the same parity of cluster rank.
+        int tile, split, gemm;
+        umma_decode_unit(p, pair_id, tile, split, gemm);
+        int mb, nb;
+        umma_tile_coords(p, tile, mb, nb);
+        bool ok = pair_id < total_units;
+        uint8_t* staging = gen_base + STAGES * STAGE + (warp - 2) * 8192;
+        const uint16_t* bias_smem = umma_fetch_bias<BN>(p, staging, nb * BN, lane);
+        if (ok && !mbar_wait(tfull_bar(0), 0u, abort_flag)) {
+            if (lane == 0) give_up(0x400u);
+            ok = false;
+        }
+        tc_fence_after_sync();
+        umma_cluster_epilogue<BN>(p, &tmap_c, tmem_base, smem_base, gen_base, staging, bias_smem, warp & 3, lane,
+                                  static_cast<uint32_t>(p.splits), crank >> 1, rank, 2u,
+                                  mb * BM2 + static_cast<int>(rank) * UMMA_BM, nb * BN, gemm, ok);
     } else if (warp < 6) {
         // ------------------------------------------------ epilogue (both CTAs, own 128 rows)
         const int quarter = warp & 3;
@@ -240,14 +267,14 @@ umma_bf16_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_c
                 tmem_ld_32x32(taddr + 32, v1);
                 tmem_ld_wait();
                 umma_store_chunk(p, &tmap_c, v0, row0, lane, nb * BN + c0, split, gemm, empty_k, staging, 0,
-                                 bias_smem ? bias_smem + c0 : nullptr);
+                                 bias_smem ? bias_smem + c0 : nullptr, p.splits > 1);
                 __syncwarp();
                 umma_store_chunk(p, &tmap_c, v1, row0, lane, nb * BN + c0 + 32, split, gemm, empty_k, staging, 1,
-                                 bias_smem ? bias_smem + c0 + 32 : nullptr);
+                                 bias_smem ? bias_smem + c0 + 32 : nullptr, p.splits > 1);
                 __syncwarp();
             }
             tc_fence_before_sync();
-            mbar_arrive_cluster(map_to_cta(tempty_bar(acc), 0));
+            mbar_arrive_cluster(map_to_cta(tempty_bar(acc), leader));
         }
         if (lane == 0) bulk_wait_all();   // this warp's TMA stores are done with the staging buffers
         __syncwarp();
@@ -257,7 +284,7 @@ umma_bf16_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_c
         // stage to the leader's full[] barrier.
         static_assert(VNNI_LOOKAHEAD < STAGES, "copies in flight must fit the ring");
         const int tw = warp - 6;
-        const uint32_t lead_full0 = map_to_cta(full_bar(0), 0);
+        const uint32_t lead_full0 = map_to_cta(full_bar(0), leader);
         int stage = 0, astage = 0, pending = 0;
         uint32_t phase = 0;
         bool ok = true;
@@ -296,6 +323,13 @@ umma_bf16_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_c
         }
     }
 
+    if (CLUSTER_REDUCE && !(warp >= 2 && warp < 6)) {
+        // the cluster barrier counts every thread: the other roles pass both reduction phases here
+        cluster_arrive();
+        cluster_wait();
+        cluster_arrive();
+        cluster_wait();
+    }
     tc_fence_before_sync();
     __syncthreads();
     cluster_sync_all();

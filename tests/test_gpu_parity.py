@@ -137,32 +137,34 @@ def test_umma_bf16_splitk(splits, out_dtype, epi, mode):
     assert "splitk" in plan.kernel_name
     # partials either meet in shared memory (splits = the CTAs of a cluster) or go through the workspace
     assert ("_cluster" in plan.kernel_name) == (plan.workspace_bytes == 0)
-    assert ("_cluster" in plan.kernel_name) == (mode == "single" and splits in (2, 4, 8))
+    if mode == "single":
+        assert ("_cluster" in plan.kernel_name) == (splits in (2, 4, 8))
     assert ("pair" in plan.kernel_name) == (mode == "pair")
     run_and_check(W("umma", 130, 200, 1096, "bf16", out_dtype, epilogue=epi, seed=9), flags=f)
 
 
-@pytest.mark.parametrize("tile", [2, 3])
+@pytest.mark.parametrize("mode,tile", [("single", 2), ("single", 3), ("single", 4), ("pair", 3), ("pair", 4)])
 @pytest.mark.parametrize("out_dtype,epi", [("f32", "none"), ("bf16", "bias_relu")])
-@pytest.mark.parametrize("shape,splits", [((130, 200, 1096), 2), ((130, 200, 1096), 8), ((520, 776, 2048), 4),
-                                          ((256, 4096, 1024), 4), ((16, 1024, 1024), 8), ((100, 72, 64), 2)])
-def test_umma_splitk_cluster_reduce_equals_reduce_kernel(shape, splits, out_dtype, epi, tile):
-    """K splits as the CTAs of one cluster: the partial sums meet in shared memory and are added in
-    split order, exactly as the separate reduce kernel adds them: same bits, one launch, no workspace."""
+@pytest.mark.parametrize("shape,splits", [((130, 200, 1096), 2), ((520, 776, 2048), 4), ((256, 4096, 1024), 4),
+                                          ((16, 1024, 1024), 8), ((100, 72, 64), 2), ((300, 520, 512), 2)])
+def test_umma_splitk_cluster_reduce_equals_reduce_kernel(shape, splits, out_dtype, epi, mode, tile):
+    """K splits as the CTAs (or CTA pairs) of one cluster: the partial sums meet in shared memory and
+    are added in split order, exactly as the separate reduce kernel adds them: same bits, one
+    launch, no workspace."""
     M, N, K = shape
     w = W("cluster", M, N, K, "bf16", out_dtype, epilogue=epi, seed=21)
     A, B, bias = w.make()
-    f = nk.FLAG_SINGLE_CTA | nk.flag_splitk(splits) | nk.flag_tile_n(tile)
-    c_two, p_two = run_plan(w, A, B, bias, flags=f | nk.FLAG_SEPARATE_REDUCE)
+    f = MODES[mode] | nk.flag_splitk(splits) | nk.flag_tile_n(tile)
     c_one, p_one = run_plan(w, A, B, bias, flags=f)
-    nsplit = int(p_one.kernel_name.split("splitk")[1].split("_")[0])   # the plan drops empty splits
-    if nsplit not in (2, 4, 8):
-        pytest.skip(f"{nsplit} splits do not form a cluster")
     if "_cluster" not in p_one.kernel_name:
-        assert nsplit * -(-M // 128) * -(-N // (32 << (tile - 1))) > 100, p_one.kernel_name
-        pytest.skip("the clusters of this plan are not all resident at once")
+        # not a cluster size (the plan drops empty splits), or the clusters are not all resident at once
+        nsplit = int(p_one.kernel_name.split("splitk")[1].split("_")[0])
+        ctas = nsplit * -(-M // 128) * -(-N // (32 << (tile - 1)))
+        assert nsplit not in (2, 4, 8) or ctas > 100 or (mode == "pair" and nsplit == 8), p_one.kernel_name
+        pytest.skip("no cluster for this plan")
+    c_two, p_two = run_plan(w, A, B, bias, flags=f | nk.FLAG_SEPARATE_REDUCE)
     assert p_two.launches_per_run == 2 and p_one.launches_per_run == 1
-    assert "_cluster" in p_one.kernel_name and "_cluster" not in p_two.kernel_name
+    assert "_cluster" not in p_two.kernel_name and ("pair" in p_one.kernel_name) == (mode == "pair")
     assert p_one.workspace_bytes == 0 and p_two.workspace_bytes > 0
     assert np.array_equal(c_one, c_two)
     c_again, _ = run_plan(w, A, B, bias, plan=p_one)
@@ -170,12 +172,14 @@ def test_umma_splitk_cluster_reduce_equals_reduce_kernel(shape, splits, out_dtyp
     check_against_oracle(w, c_one, A, B, bias)
 
 
+@pytest.mark.parametrize("mode", ["single", "pair"])
 @pytest.mark.parametrize("splits", [2, 4])
-def test_umma_splitk_cluster_blocked_operands(splits):
+def test_umma_splitk_cluster_blocked_operands(splits, mode):
     """Cluster split-K with blocked A, VNNI-blocked B (re-laid in the kernel) and exact integer data."""
     w = W("cluster_blk", 256, 256, 1024, "bf16", layout="blocked32", integer=True)
-    err, plan = run_and_check(w, flags=nk.FLAG_SINGLE_CTA | nk.flag_splitk(splits) | nk.flag_tile_n(3), exact=True)
+    err, plan = run_and_check(w, flags=MODES[mode] | nk.flag_splitk(splits) | nk.flag_tile_n(3), exact=True)
     assert "_cluster" in plan.kernel_name and "_bvnni" in plan.kernel_name and plan.workspace_bytes == 0
+    assert ("pair" in plan.kernel_name) == (mode == "pair")
 
 
 @pytest.mark.parametrize("mode,tile", [("single", 2), ("single", 3), ("single", 4), ("pair", 3), ("pair", 4)])
