@@ -144,15 +144,28 @@ static double umma_model_us(const nk_gemm_desc_t& d, int sms, bool pair, int bn,
     const int64_t units = tiles * eff_splits;
     const int workers = pair ? sms / 2 : sms;
     const double rounds = static_cast<double>((units + workers - 1) / workers);
+    // Fitted to timelines taken inside the kernels on B200: a k-block costs about the same whatever
+    // the tile width (the SM's operand feed from L2, ~50 bytes per clock, or the MMA itself at
+    // N = 256); the epilogue of the last tile is not hidden and is bound by the SM's store path
+    // (~0.35 us per 32 columns, 0.5 us in a pair); a cluster reduction costs two cluster barriers
+    // plus the accumulator pieces that cross to other SMs (~14 KB per microsecond per CTA).
     double t_kb;  // microseconds per 64-wide k-block of one unit
-    if (pair) t_kb = bn == 256 ? 0.385 : 0.348;
-    else t_kb = bn == 256 ? 0.44 : bn == 128 ? 0.352 : 0.37;
+    if (pair) t_kb = bn == 256 ? (rounds > 1 ? 0.385 : 0.36) : 0.345;
+    else t_kb = bn == 256 ? 0.46 : bn == 128 ? 0.345 : 0.31;
+    if (d.layout_b == NK_BLOCKED32 && !(d.flags & NK_FLAG_REPACK_B)) {
+        // VNNI-blocked B is re-laid by four warps through the LSU: its cost grows with the columns a CTA covers
+        const double vnni = 0.14 + bn * 0.0042;
+        if (vnni > t_kb) t_kb = vnni;
+    }
     const double eo = d.out_dtype == NK_BF16 ? 2.0 : 4.0;
     const double mn = static_cast<double>(d.M) * d.N;
-    double us = (pair ? 12.0 : 10.0) + rounds * per * t_kb;
-    if (eff_splits > 1) {
-        if (cluster_reduce_fits(d, sms, pair, bn, eff_splits)) us += 1.5;
-        else us += 3.0 + eff_splits * mn * 4.0 / 3.0e6 + (eff_splits * 4.0 + eo) * mn / 5.0e6;
+    const double chunks = bn / 32.0;
+    double us = (pair ? 7.0 : 6.0) + rounds * per * t_kb;
+    if (eff_splits > 1 && cluster_reduce_fits(d, sms, pair, bn, eff_splits)) {
+        us += 2.0 + bn * 512.0 * (eff_splits - 1) / eff_splits / 14.0e3 + chunks / eff_splits * (pair ? 0.5 : 0.4);
+    } else {
+        us += chunks * (pair ? 0.5 : 0.35);
+        if (eff_splits > 1) us += 3.0 + eff_splits * mn * 4.0 / 3.0e6 + (eff_splits * 4.0 + eo) * mn / 5.0e6;
     }
     const double bytes = 2.0 * desc_batch(d) * (static_cast<double>(d.M) * d.K + static_cast<double>(d.K) * d.N) + eo * mn;
     const double hbm_us = bytes / 5.2e6;  // ~80 % of the copy bandwidth, bytes per microsecond
@@ -172,6 +185,8 @@ static void choose_umma(nk_gemm_s* p) {
         if (pair && (d.flags & NK_FLAG_SINGLE_CTA)) continue;
         if (!pair && (d.flags & NK_FLAG_CTA_PAIR) && forced_bn != 2) continue;
         if (pair && d.M <= UMMA_BM && !(d.flags & NK_FLAG_CTA_PAIR)) continue;
+        // measured: with the in-kernel VNNI re-layout a pair is far slower than two single CTAs
+        if (pair && d.layout_b == NK_BLOCKED32 && !(d.flags & (NK_FLAG_REPACK_B | NK_FLAG_CTA_PAIR))) continue;
         for (int bn = 64; bn <= 256; bn *= 2) {
             if (pair && bn == 64) continue;
             if (forced_bn >= 2 && forced_bn <= 4 && bn != (32 << (forced_bn - 1))) continue;
