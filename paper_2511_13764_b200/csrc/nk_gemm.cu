@@ -148,7 +148,7 @@ static double umma_model_us(const nk_gemm_desc_t& d, int sms, bool pair, int bn,
     // the tile width (the SM's operand feed from L2, ~50 bytes per clock, or the MMA itself at
     // N = 256); the epilogue of the last tile is not hidden and is bound by the SM's store path
     // (~0.35 us per 32 columns, 0.5 us in a pair); a cluster reduction costs two cluster barriers
-    // plus the accumulator pieces that cross to other SMs (~14 KB per microsecond per CTA).
+    // plus the accumulator pieces that cross to other SMs as 4 KB bulk copies (~40 KB per microsecond per CTA).
     double t_kb;  // microseconds per 64-wide k-block of one unit
     if (pair) t_kb = bn == 256 ? (rounds > 1 ? 0.385 : 0.36) : 0.345;
     else t_kb = bn == 256 ? 0.46 : bn == 128 ? 0.345 : 0.31;
@@ -162,7 +162,7 @@ static double umma_model_us(const nk_gemm_desc_t& d, int sms, bool pair, int bn,
     const double chunks = bn / 32.0;
     double us = (pair ? 7.0 : 6.0) + rounds * per * t_kb;
     if (eff_splits > 1 && cluster_reduce_fits(d, sms, pair, bn, eff_splits)) {
-        us += 2.0 + bn * 512.0 * (eff_splits - 1) / eff_splits / 14.0e3 + chunks / eff_splits * (pair ? 0.5 : 0.4);
+        us += 2.0 + bn * 512.0 * (eff_splits - 1) / eff_splits / 40.0e3 + chunks / eff_splits * (pair ? 0.5 : 0.4);
     } else {
         us += chunks * (pair ? 0.5 : 0.35);
         if (eff_splits > 1) us += 3.0 + eff_splits * mn * 4.0 / 3.0e6 + (eff_splits * 4.0 + eo) * mn / 5.0e6;

@@ -221,6 +221,17 @@ __device__ __forceinline__ void st_cluster_v4(uint32_t cluster_addr, uint32_t a,
                  "r"(d)
                  : "memory");
 }
+// Bulk copy of `bytes` (a multiple of 16) from this CTA's shared memory into the shared memory of a
+// CTA of the cluster; the bytes are counted in on the mbarrier `cluster_bar` of the receiving CTA
+// (both given as cluster-window addresses).  Tracked by the issuing thread's bulk group.
+__device__ __forceinline__ void bulk_copy_to_cluster(uint32_t cluster_dst, uint32_t src, uint32_t bytes,
+                                                     uint32_t cluster_bar) {
+    asm volatile(
+        "cp.async.bulk.shared::cluster.shared::cta.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(
+            cluster_dst),
+        "r"(src), "r"(bytes), "r"(cluster_bar)
+        : "memory");
+}
 // Arrive on an mbarrier given by a cluster-window address (possibly in the peer CTA).
 __device__ __forceinline__ void mbar_arrive_cluster(uint32_t cluster_bar) {
     asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(cluster_bar)

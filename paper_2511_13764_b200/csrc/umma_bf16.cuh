@@ -271,30 +271,56 @@ __device__ __forceinline__ const uint16_t* umma_fetch_bias(const UmmaParams& p, 
     return reinterpret_cast<const uint16_t*>(dst);
 }
 
+// The lane's 16 bytes of the tile's bias slice (lanes 0 .. BN/8-1), for the cluster epilogue.
+template <int BN>
+__device__ __forceinline__ uint4 umma_load_bias_reg(const UmmaParams& p, int col_tile0, int lane, bool& have) {
+    have = p.epilogue && p.out_bf16;
+    uint4 r = make_uint4(0u, 0u, 0u, 0u);
+    const int col = col_tile0 + 8 * lane;
+    if (have && lane < BN / 8 && col < p.N)
+        r = __ldg(reinterpret_cast<const uint4*>(static_cast<const uint16_t*>(p.bias) + col));
+    return r;
+}
+
 // Epilogue of a cluster split-K CTA.  Its accumulator (128 rows x BN columns, tensor-memory
 // columns 0..BN-1) is cut into 4 * BN / 32 pieces, piece u = quarter * (BN / 32) + chunk; the CTAs
 // that hold the S splits of the same rows have cluster ranks rank0 + s * rank_step.  Piece u
 // belongs to split u % S; the other splits send theirs into slot (u / S) * S + source split of
 // the owner's stage ring (idle by then), the owner's own contribution stays in tensor memory.
-//   phase A  every CTA of the cluster has finished its K loop: the rings may be overwritten
-//   send     tcgen05.ld -> 16-byte stores into the owner's ring (group g of row t at
-//            g * 512 + (t ^ g) * 16: a warp instruction writes 512 contiguous bytes, and both
-//            sides stay free of bank conflicts)
-//   phase B  all pieces have arrived
+//   barrier  every CTA of the cluster has finished its K loop: the rings may be overwritten
+//   send     tcgen05.ld -> the warp's staging tile (16-byte group g of row t at g * 512 +
+//            (t ^ g) * 16: conflict-free on both sides) -> one 4 KB bulk copy into the owner's
+//            slot, counted in on the owner's `recv` mbarrier (per-thread remote stores were
+//            several times slower)
+//   wait     the owner's mbarrier has seen all the bytes it expects (bounded wait)
 //   reduce   every owned piece is summed in split order (the result does not depend on timing)
 //            and leaves through the ordinary chunk epilogue: beta, bias + ReLU, conversion, store
-// Every thread of the cluster passes both barrier phases, also after a wait that gave up.
+// Every thread of the cluster passes the barrier, also after a wait that gave up.
 template <int BN>
-__device__ __forceinline__ void umma_cluster_epilogue(const UmmaParams& p, const CUtensorMap* tmap_c, uint32_t tmem_base,
-                                                      uint32_t ring, const uint8_t* ring_gen, uint8_t* staging,
-                                                      const uint16_t* bias_smem, int quarter, int lane, uint32_t S,
+__host__ __device__ constexpr uint32_t umma_cluster_recv_bytes(uint32_t S) { return (4u * (BN / 32) / S) * (S - 1u) * 4096u; }
+
+template <int BN>
+__device__ __forceinline__ bool umma_cluster_epilogue(const UmmaParams& p, const CUtensorMap* tmap_c, uint32_t tmem_base,
+                                                      uint32_t ring, const uint8_t* ring_gen, uint32_t recv_bar,
+                                                      volatile uint32_t* abort_flag, uint8_t* staging, uint8_t* bias_park,
+                                                      uint4 bias_reg, bool have_bias, int quarter, int lane, uint32_t S,
                                                       uint32_t split, uint32_t rank0, uint32_t rank_step, int row_cta0,
                                                       int col_tile0, int gemm, bool ok) {
     constexpr uint32_t NC = BN / 32;
     const uint32_t lane_tmem = static_cast<uint32_t>(quarter * 32) << 16;
     cluster_arrive();
-    cluster_wait();                                      // phase A
+    cluster_wait();
+    // The bias slice of the tile was loaded into a register per lane before the accumulator was
+    // ready; it is parked behind the receive slots of the ring now that the ring is free (the
+    // staging tiles, where the ordinary epilogue keeps it, are the send buffers here).
+    const uint16_t* bias_smem = nullptr;
+    if (have_bias) {
+        if (lane < BN / 8) reinterpret_cast<uint4*>(bias_park)[lane] = bias_reg;
+        __syncwarp();
+        bias_smem = reinterpret_cast<const uint16_t*>(bias_park);
+    }
     if (ok) {
+        uint32_t parity = 0;
 #pragma unroll 1
         for (uint32_t c = 0; c < NC; ++c) {
             const uint32_t u = quarter * NC + c, owner = u % S;
@@ -302,15 +328,31 @@ __device__ __forceinline__ void umma_cluster_epilogue(const UmmaParams& p, const
             uint32_t v[32];
             tmem_ld_32x32(tmem_base + c * 32 + lane_tmem, v);
             tmem_ld_wait();
-            const uint32_t dst = map_to_cta(ring + ((u / S) * S + split) * 4096u, rank0 + owner * rank_step);
+            uint8_t* tile = staging + parity * 4096;
+            if (lane == 0) bulk_wait_read<1>();          // the copy issued two pieces ago has read this tile
+            __syncwarp();
 #pragma unroll
             for (int g = 0; g < 8; ++g)
-                st_cluster_v4(dst + g * 512 + ((lane ^ g) << 4), v[4 * g], v[4 * g + 1], v[4 * g + 2], v[4 * g + 3]);
+                *reinterpret_cast<uint4*>(tile + g * 512 + ((lane ^ g) << 4)) =
+                    make_uint4(v[4 * g], v[4 * g + 1], v[4 * g + 2], v[4 * g + 3]);
+            fence_proxy_async_smem();
+            __syncwarp();
+            if (lane == 0) {
+                const uint32_t peer = rank0 + owner * rank_step;
+                bulk_copy_to_cluster(map_to_cta(ring + ((u / S) * S + split) * 4096u, peer), smem_u32(tile), 4096u,
+                                     map_to_cta(recv_bar, peer));
+                bulk_commit();
+            }
+            parity ^= 1u;
         }
+        if (!mbar_wait(recv_bar, 0u, abort_flag)) ok = false;   // every piece sent to this CTA has landed
+    } else {
+        // this CTA gave up, but healthy peers may still be copying into it: let their copies land
+        mbar_wait(recv_bar, 0u, abort_flag, 1ll << 24);
     }
-    cluster_arrive();
-    cluster_wait();                                      // phase B
-    if (!ok) return;
+    if (lane == 0) bulk_wait_read<0>();                  // the staging tiles are free again
+    __syncwarp();
+    if (!ok) return false;
     int parity = 0;
 #pragma unroll 1
     for (uint32_t c = 0; c < NC; ++c) {
@@ -354,6 +396,7 @@ __device__ __forceinline__ void umma_cluster_epilogue(const UmmaParams& p, const
     }
     if (lane == 0) bulk_wait_all();
     __syncwarp();
+    return true;
 }
 
 // Re-layout of a VNNI-blocked B operand (Figure 1 of the paper: [k/2][n][2] inside every 32 x 32
@@ -439,7 +482,13 @@ umma_bf16_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_consta
             mbar_init(tempty_bar(a), 128);
         }
         *abort_flag = 0;
+        if (CLUSTER_REDUCE) {
+            // the pieces other CTAs will send to this one are counted in on this barrier
+            mbar_init(bar_base + 192u, 1);
+        }
         fence_mbar_init();
+        if (CLUSTER_REDUCE)
+            mbar_arrive_expect_tx(bar_base + 192u, umma_cluster_recv_bytes<BN>(static_cast<uint32_t>(p.splits)));
         tma_prefetch_desc(&tmap_a);
         if (!B_VNNI) tma_prefetch_desc(&tmap_b);
         if (p.tma_store) tma_prefetch_desc(&tmap_c);
@@ -607,15 +656,17 @@ umma_bf16_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_consta
         umma_tile_coords(p, tile, mb, nb);
         bool ok = blockIdx.x < total_units;
         uint8_t* staging = gen_base + STAGES * STAGE + (warp - 2) * 8192;
-        const uint16_t* bias_smem = umma_fetch_bias<BN>(p, staging, nb * BN, lane);
+        bool have_bias;
+        const uint4 bias_reg = umma_load_bias_reg<BN>(p, nb * BN, lane, have_bias);
         if (ok && !mbar_wait(tfull_bar(0), 0u, abort_flag)) {
             if (lane == 0) give_up(0x400u);
             ok = false;
         }
         tc_fence_after_sync();
-        umma_cluster_epilogue<BN>(p, &tmap_c, tmem_base, smem_base, gen_base, staging, bias_smem, warp & 3, lane,
-                                  static_cast<uint32_t>(p.splits), cluster_ctarank(), 0u, 1u, mb * UMMA_BM, nb * BN,
-                                  gemm, ok);
+        if (!umma_cluster_epilogue<BN>(p, &tmap_c, tmem_base, smem_base, gen_base, bar_base + 192u, abort_flag, staging,
+                                       gen_base + BN * 512 + (warp - 2) * 512, bias_reg, have_bias, warp & 3, lane, static_cast<uint32_t>(p.splits), cluster_ctarank(), 0u,
+                                       1u, mb * UMMA_BM, nb * BN, gemm, ok) && ok && lane == 0)
+            give_up(0x600u);
     } else if (warp < 6) {
         // ------------------------------------------------ epilogue
         const int quarter = warp & 3;  // TMEM lanes 32*quarter .. +31 belong to this warp
@@ -703,10 +754,8 @@ umma_bf16_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_consta
     }
 
     if (CLUSTER_REDUCE && !(warp >= 2 && warp < 6)) {
-        // the cluster barrier counts every thread: the other roles pass both phases here, once
-        // their part of the K loop is over (the producer has seen every stage consumed)
-        cluster_arrive();
-        cluster_wait();
+        // the cluster barrier counts every thread: the other roles pass it here, once their part
+        // of the K loop is over (the producer has seen every stage consumed)
         cluster_arrive();
         cluster_wait();
     }

@@ -75,7 +75,10 @@ umma_bf16_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_c
             mbar_init(tempty_bar(a), 256);               // epilogue threads of both CTAs
         }
         *abort_flag = 0;
+        if (CLUSTER_REDUCE) mbar_init(bar_base + 192u, 1);   // counts in the pieces other CTAs send to this one
         fence_mbar_init();
+        if (CLUSTER_REDUCE)
+            mbar_arrive_expect_tx(bar_base + 192u, umma_cluster_recv_bytes<BN>(static_cast<uint32_t>(p.splits)));
         tma_prefetch_desc(&tmap_a);
         if (!B_VNNI) tma_prefetch_desc(&tmap_b);
         if (p.tma_store) tma_prefetch_desc(&tmap_c);
@@ -227,15 +230,17 @@ umma_bf16_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_c
         umma_tile_coords(p, tile, mb, nb);
         bool ok = pair_id < total_units;
         uint8_t* staging = gen_base + STAGES * STAGE + (warp - 2) * 8192;
-        const uint16_t* bias_smem = umma_fetch_bias<BN>(p, staging, nb * BN, lane);
+        bool have_bias;
+        const uint4 bias_reg = umma_load_bias_reg<BN>(p, nb * BN, lane, have_bias);
         if (ok && !mbar_wait(tfull_bar(0), 0u, abort_flag)) {
             if (lane == 0) give_up(0x400u);
             ok = false;
         }
         tc_fence_after_sync();
-        umma_cluster_epilogue<BN>(p, &tmap_c, tmem_base, smem_base, gen_base, staging, bias_smem, warp & 3, lane,
-                                  static_cast<uint32_t>(p.splits), crank >> 1, rank, 2u,
-                                  mb * BM2 + static_cast<int>(rank) * UMMA_BM, nb * BN, gemm, ok);
+        if (!umma_cluster_epilogue<BN>(p, &tmap_c, tmem_base, smem_base, gen_base, bar_base + 192u, abort_flag, staging,
+                                       gen_base + BN * 512 + (warp - 2) * 512, bias_reg, have_bias, warp & 3, lane, static_cast<uint32_t>(p.splits), crank >> 1, rank, 2u,
+                                       mb * BM2 + static_cast<int>(rank) * UMMA_BM, nb * BN, gemm, ok) && ok && lane == 0)
+            give_up(0x600u);
     } else if (warp < 6) {
         // ------------------------------------------------ epilogue (both CTAs, own 128 rows)
         const int quarter = warp & 3;
@@ -324,9 +329,7 @@ umma_bf16_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_c
     }
 
     if (CLUSTER_REDUCE && !(warp >= 2 && warp < 6)) {
-        // the cluster barrier counts every thread: the other roles pass both reduction phases here
-        cluster_arrive();
-        cluster_wait();
+        // the cluster barrier counts every thread: the other roles pass it here
         cluster_arrive();
         cluster_wait();
     }
