@@ -65,6 +65,11 @@ def f32_to_bf16_bits(x: np.ndarray) -> np.ndarray:
     return (r >> np.uint32(16)).astype(np.uint16)
 
 
+def f32_to_f16_bits(x: np.ndarray) -> np.ndarray:
+    """Round finite FP32 values to IEEE binary16 (nearest, ties to even); returns uint16."""
+    return np.ascontiguousarray(x, dtype=np.float32).astype(np.float16).view(np.uint16)
+
+
 def _uniform_f32(seed, tensor_id, start, count):
     t = (raw_bits(seed, tensor_id, start, count) >> np.uint64(40)).astype(np.float64)
     return (t * 2.0 ** -23 - 1.0).astype(np.float32)
@@ -85,7 +90,7 @@ def fill(seed: int, tensor_id: int, count: int, dist: str = "uniform",
 
     dist: "uniform" (U[-1,1) on the 2**-23 grid), "normal" (N(0, sigma**2)),
           "int" (integers in [-4, 4], exact in every precision used here).
-    dtype: "f32" -> float32 array; "bf16" -> uint16 bit patterns.
+    dtype: "f32" -> float32 array; "bf16" / "f16" -> uint16 bit patterns.
     """
     out = np.empty(count, dtype=np.float32 if dtype == "f32" else np.uint16)
     for s in range(0, count, _CHUNK):
@@ -99,7 +104,7 @@ def fill(seed: int, tensor_id: int, count: int, dist: str = "uniform",
                  ).astype(np.float32) - 4.0
         else:
             raise ValueError(dist)
-        out[s:s + n] = v if dtype == "f32" else f32_to_bf16_bits(v)
+        out[s:s + n] = v if dtype == "f32" else (f32_to_f16_bits(v) if dtype == "f16" else f32_to_bf16_bits(v))
     return out
 
 
@@ -130,8 +135,8 @@ class Workload:
     M: int
     N: int
     K: int
-    in_dtype: str = "bf16"          # "f32" | "bf16"
-    out_dtype: str = "f32"          # "f32" | "bf16"
+    in_dtype: str = "bf16"          # "f32" | "bf16" | "f16"
+    out_dtype: str = "f32"          # "f32" | "bf16" | "f16" (a 16-bit output has the input's type)
     layout: str = "row"             # "row" | "blocked32" (A and B both)
     epilogue: str = "none"          # "none" | "bias_relu"
     dist_a: tuple = ("uniform", 1.0)

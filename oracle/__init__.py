@@ -17,7 +17,7 @@ _HERE = os.path.dirname(os.path.abspath(__file__))
 _SRC = os.path.join(_HERE, "nk_oracle.c")
 _LIB = os.path.join(_HERE, "libnk_oracle.so")
 
-F32, BF16 = 0, 1
+F32, BF16, F16 = 0, 1, 2
 ROW, BLOCKED32 = 0, 1
 EPI_NONE, EPI_BIAS_RELU = 0, 1
 ACC_F64, ACC_F32_SEQ = 0, 1
@@ -49,6 +49,8 @@ def lib():
         L = ctypes.CDLL(build())
         L.nko_bf16_to_f32.restype = ctypes.c_float
         L.nko_bf16_to_f32.argtypes = [ctypes.c_uint16]
+        L.nko_f16_to_f32.restype = ctypes.c_float
+        L.nko_f16_to_f32.argtypes = [ctypes.c_uint16]
         L.nko_f32_to_bf16_rne.restype = ctypes.c_uint16
         L.nko_f32_to_bf16_rne.argtypes = [ctypes.c_float]
         for f in (L.nko_pack_vnni2, L.nko_unpack_vnni2):
@@ -74,6 +76,14 @@ def bf16_to_f32(bits: np.ndarray) -> np.ndarray:
     L = lib()
     flat = np.ascontiguousarray(bits, dtype=np.uint16).ravel()
     out = np.fromiter((L.nko_bf16_to_f32(int(h)) for h in flat), dtype=np.float32, count=flat.size)
+    return out.reshape(np.shape(bits))
+
+
+def f16_to_f32(bits: np.ndarray) -> np.ndarray:
+    """Decode uint16 IEEE binary16 patterns element by element through the C routine."""
+    L = lib()
+    flat = np.ascontiguousarray(bits, dtype=np.uint16).ravel()
+    out = np.fromiter((L.nko_f16_to_f32(int(h)) for h in flat), dtype=np.float32, count=flat.size)
     return out.reshape(np.shape(bits))
 
 
@@ -169,7 +179,7 @@ def gemm_workload(w, A, B, bias, rows=None, cols=None, **kw):
     in_dtype, layout, epilogue attributes)."""
     lay = BLOCKED32 if w.layout == "blocked32" else ROW
     return gemm(w.M, w.N, w.K, A, B, bias,
-                in_dtype=F32 if w.in_dtype == "f32" else BF16,
+                in_dtype={"f32": F32, "bf16": BF16, "f16": F16}[w.in_dtype],
                 layout_a=lay, layout_b=lay,
                 epilogue=EPI_BIAS_RELU if w.epilogue == "bias_relu" else EPI_NONE,
                 rows=rows, cols=cols, **kw)

@@ -13,8 +13,10 @@
  *     S[i][j] = sum_k |a(i,k) * b(k,j)| (+ |bias[j]|) (scale of the error bound)
  *
  * a, b are the stored operand values: FP32, or BF16 widened exactly to FP32 (the
- * appendix kernels' scalar body: extf, extf, mulf, addf).  y is returned
- * unrounded, as double; a BF16-storing implementation rounds once afterwards.
+ * appendix kernels' scalar body: extf, extf, mulf, addf), or FP16 (IEEE binary16, the
+ * other 16-bit type the paper's Section 5 names as the next packed type) widened
+ * exactly.  y is returned unrounded, as double; a BF16- or FP16-storing
+ * implementation rounds once afterwards.
  *
  * Layouts: row-major A[M][K], B[K][N]; or 32x32-blocked with the VNNI-2
  * interleave of Figure 1 inside each B block:
@@ -24,7 +26,8 @@
  * Pins (tests/test_oracle_*.py): Figure 1's printed packing, identity /
  * permutation / diagonal / rank-1 / all-ones closed forms, brute force in a
  * different loop order, numpy float64 matmul on small shapes, blocked-vs-flat
- * bit equality, epilogue closed forms, exhaustive BF16 codec round trip.
+ * bit equality, epilogue closed forms, exhaustive BF16 codec round trip, exhaustive FP16
+ * decode against the IEEE reading.
  */
 #include <math.h>
 #include <pthread.h>
@@ -32,14 +35,14 @@
 #include <stdlib.h>
 #include <string.h>
 
-enum { NKO_F32 = 0, NKO_BF16 = 1 };
+enum { NKO_F32 = 0, NKO_BF16 = 1, NKO_F16 = 2 };
 enum { NKO_ROW = 0, NKO_BLOCKED32 = 1 };
 enum { NKO_EPI_NONE = 0, NKO_EPI_BIAS_RELU = 1 };
 enum { NKO_ACC_F64 = 0, NKO_ACC_F32_SEQ = 1 };
 
 typedef struct {
     int64_t M, N, K;
-    int32_t in_dtype;   /* NKO_F32 | NKO_BF16: element type of A, B and bias */
+    int32_t in_dtype;   /* NKO_F32 | NKO_BF16 | NKO_F16: element type of A, B and bias */
     int32_t layout_a;   /* NKO_ROW | NKO_BLOCKED32 */
     int32_t layout_b;
     int32_t epilogue;
@@ -52,6 +55,19 @@ float nko_bf16_to_f32(uint16_t h) {
     float f;
     memcpy(&f, &u, 4);
     return f;
+}
+
+/* IEEE 754 binary16 -> FP32, written from the format's definition: 1 sign bit, 5 exponent bits
+   (bias 15), 10 fraction bits; exponent 0 is zero or a subnormal (fraction * 2^-24), exponent 31
+   is infinity or NaN, otherwise (1 + fraction / 1024) * 2^(exponent - 15).  Every binary16 value
+   is exactly representable in FP32. */
+float nko_f16_to_f32(uint16_t h) {
+    int sign = (h >> 15) & 1, e = (h >> 10) & 0x1F, m = h & 0x3FF;
+    double v;
+    if (e == 0) v = ldexp((double)m, -24);
+    else if (e == 31) v = m ? NAN : INFINITY;
+    else v = ldexp(1.0 + (double)m / 1024.0, e - 15);
+    return (float)(sign ? -v : v);
 }
 
 /* FP32 -> BF16, round to nearest, ties to even (finite inputs). */
@@ -92,6 +108,7 @@ int64_t nko_b_index(const nko_desc_t* d, int64_t k, int64_t j) { return b_index(
 
 static double load(const void* p, int32_t dtype, int64_t idx) {
     if (dtype == NKO_F32) return (double)((const float*)p)[idx];
+    if (dtype == NKO_F16) return (double)nko_f16_to_f32(((const uint16_t*)p)[idx]);
     return (double)nko_bf16_to_f32(((const uint16_t*)p)[idx]);
 }
 

@@ -398,3 +398,66 @@ def test_brgemm_batch_one_is_gemm():
     Y, S = oracle.brgemm(M, N, K, 1, A, B)
     Yg, Sg = oracle.gemm(M, N, K, A, B)
     assert np.array_equal(Y, Yg) and np.array_equal(S, Sg)
+
+
+# ---------------------------------------------------------------- FP16 operands (Section 5: the next packed type)
+def test_f16_decode_exhaustive_against_ieee_and_numpy():
+    bits = np.arange(65536, dtype=np.uint16)
+    e = ((bits >> 10) & 0x1F).astype(np.int64)
+    finite = bits[e != 31]
+    f = oracle.f16_to_f32(finite).astype(np.float64)
+    ef = ((finite >> 10) & 0x1F).astype(np.int64)
+    m = (finite & 0x3FF).astype(np.float64)
+    sign = np.where(finite >> 15, -1.0, 1.0)
+    want = np.where(ef == 0, sign * m * 2.0 ** -24, sign * (1 + m / 1024) * 2.0 ** (ef - 15))
+    assert np.array_equal(f, want)
+    # the same through the library's binary16 type (a separate implementation of the format)
+    assert np.array_equal(f, finite.view(np.float16).astype(np.float64))
+    # landmarks of the format: 1, -2, the smallest subnormal, the largest finite value, 1/3 rounded
+    marks = np.array([0x3C00, 0xC000, 0x0001, 0x7BFF, 0x3555], dtype=np.uint16)
+    assert np.array_equal(oracle.f16_to_f32(marks).astype(np.float64),
+                          np.array([1.0, -2.0, 2.0 ** -24, 65504.0, 1365 / 4096]))
+    inf = oracle.f16_to_f32(np.array([0x7C00, 0xFC00], dtype=np.uint16))
+    assert np.isposinf(inf[0]) and np.isneginf(inf[1])
+
+
+def test_f16_generator_rounds_to_nearest_even():
+    v = nk_inputs.fill(4, 0, 20000, "uniform", dtype="f32")
+    h = nk_inputs.f32_to_f16_bits(v)
+    back = oracle.f16_to_f32(h).astype(np.float64)
+    x = v.astype(np.float64)
+    ulp = np.where(np.abs(back) >= 2.0 ** -14, 2.0 ** (np.floor(np.log2(np.maximum(np.abs(back), 2.0 ** -14))) - 10), 2.0 ** -24)
+    assert np.all(np.abs(back - x) <= ulp / 2 * (1 + 1e-12))
+    ties = np.array([1 + 2.0 ** -11, 1 + 3 * 2.0 ** -11, -(1 + 3 * 2.0 ** -11), 1 + 2.0 ** -11 + 2.0 ** -20], dtype=np.float32)
+    got = oracle.f16_to_f32(nk_inputs.f32_to_f16_bits(ties)).astype(np.float64)
+    assert np.array_equal(got, np.array([1.0, 1 + 2.0 ** -9, -(1 + 2.0 ** -9), 1 + 2.0 ** -10]))
+    assert np.array_equal(nk_inputs.fill(4, 0, 100, "uniform", dtype="f16"), nk_inputs.f32_to_f16_bits(v[:100]))
+
+
+def test_f16_gemm_equals_gemm_of_the_widened_operands():
+    """FP16 operands, row-major and blocked, with bias: the oracle on the 16-bit storage equals, bit
+    for bit, the oracle on the same values stored as FP32 (widening is exact, the order is the same)."""
+    M, N, K = 64, 96, 128
+    for layout in ("row", "blocked32"):
+        w = nk_inputs.Workload("t", M, N, K, "f16", "f32", layout=layout, epilogue="bias_relu", seed=9)
+        A, B, bias = w.make()
+        Y, S = oracle.gemm_workload(w, A, B, bias)
+        widen = lambda x: x.view(np.float16).astype(np.float32)
+        lay = BLOCKED32 if layout == "blocked32" else ROW
+        if layout == "blocked32":
+            # blocked storage of FP32 is not a product layout, but the oracle's index functions do not care
+            Y2, S2 = oracle.gemm(M, N, K, widen(A), widen(B), widen(bias), in_dtype=F32, layout_a=lay, layout_b=lay,
+                                 epilogue=EPI_BIAS_RELU)
+        else:
+            Y2, S2 = oracle.gemm(M, N, K, widen(A), widen(B), widen(bias), in_dtype=F32, epilogue=EPI_BIAS_RELU)
+        assert np.array_equal(Y, Y2) and np.array_equal(S, S2)
+    # integer data: exact closed form through numpy
+    w = nk_inputs.Workload("t", 40, 48, 64, "f16", "f32", dist_a=("int", 1.0), dist_b=("int", 1.0), seed=10)
+    A, B, _ = w.make()
+    Y, _ = oracle.gemm_workload(w, A, B, None)
+    Af = A.view(np.float16).astype(np.float64).reshape(40, 64)
+    Bf = B.view(np.float16).astype(np.float64).reshape(64, 48)
+    assert np.array_equal(Y, Af @ Bf)
+    # a BF16 reading of the same bits gives something else: the dtype switch is live
+    Yb, _ = oracle.gemm(40, 48, 64, A, B, in_dtype=BF16)
+    assert not np.array_equal(Y, Yb)
