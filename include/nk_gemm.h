@@ -19,7 +19,7 @@
  *   NK_BLOCKED32   A[M/32][K/32][32][32]                 (m-block, k-block, m, k)
  *                  B[N/32][K/32][16][32][2]              (n-block, k-block, k/2, n, k%2):
  *                  every 32x32 block of B is VNNI-2 packed as in Figure 1,
- *                  packed[k/2][n][k%2] = flat[k][n]; BF16 only.
+ *                  packed[k/2][n][k%2] = flat[k][n]; 16-bit operands (BF16, FP16) only.
  * C is row-major [M][N] unless desc.layout_c asks for the blocked form; bias is [N] in the
  * operand type.
  *
@@ -52,7 +52,12 @@ typedef enum {
     NK_ERR_TIMEOUT = 7      /* a bounded device-side wait ran out (see nk_gemm_check)    */
 } nk_status_t;
 
-typedef enum { NK_F32 = 0, NK_BF16 = 1 } nk_dtype_t;
+typedef enum {
+    NK_F32 = 0,
+    NK_BF16 = 1,
+    NK_F16 = 2 /* IEEE binary16: the other 16-bit packed type (Section 5 names FP16 as the next one); same
+                  kernels, layouts and rules as BF16, FP32 accumulation, one RNE rounding of a 16-bit C */
+} nk_dtype_t;
 typedef enum { NK_ROW_MAJOR = 0, NK_BLOCKED32 = 1 } nk_layout_t;
 typedef enum { NK_EPI_NONE = 0, NK_EPI_BIAS_RELU = 1 } nk_epilogue_t;
 
@@ -76,7 +81,7 @@ typedef enum { NK_EPI_NONE = 0, NK_EPI_BIAS_RELU = 1 } nk_epilogue_t;
 typedef struct {
     int64_t M, N, K;
     int32_t in_dtype;  /* nk_dtype_t of A, B and bias                        */
-    int32_t out_dtype; /* nk_dtype_t of C: NK_F32, or NK_BF16 with BF16 inputs */
+    int32_t out_dtype; /* nk_dtype_t of C: NK_F32, or the operands' 16-bit type      */
     int32_t layout_a;  /* nk_layout_t                                         */
     int32_t layout_b;  /* nk_layout_t                                         */
     int32_t epilogue;  /* nk_epilogue_t                                       */

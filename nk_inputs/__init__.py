@@ -208,3 +208,15 @@ def paper_mlp() -> list:
         out.append(Workload(f"mlp_bf16_flat_{n}", 512, n, n, "bf16", "bf16", epilogue="bias_relu",
                             dist_a=("normal", 1.0), dist_b=("normal", 0.02), seed=6002 + n))
     return out
+
+
+def f16_set() -> list:
+    """FP16 (IEEE binary16) counterparts of the headline shapes: the large square GEMM, the MLP
+    layer of configuration 3, and the paper's 4096-wide MLP layer."""
+    return [
+        Workload("x_f16_8192", 8192, 8192, 8192, "f16", "f32", seed=7017),
+        Workload("x_f16_mlp_256x4096x4096", 256, 4096, 4096, "f16", "f16", epilogue="bias_relu",
+                 dist_a=("normal", 1.0), dist_b=("normal", 0.02), seed=7018),
+        Workload("x_f16_mlp_512x4096x4096", 512, 4096, 4096, "f16", "f16", epilogue="bias_relu",
+                 dist_a=("normal", 1.0), dist_b=("normal", 0.02), seed=7019),
+    ]

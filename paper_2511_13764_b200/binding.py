@@ -10,7 +10,7 @@ import os
 
 from . import _build
 
-F32, BF16 = 0, 1
+F32, BF16, F16 = 0, 1, 2
 ROW_MAJOR, BLOCKED32 = 0, 1
 EPI_NONE, EPI_BIAS_RELU = 0, 1
 FLAG_KERNEL_NAIVE, FLAG_KERNEL_SIMT, FLAG_KERNEL_UMMA = 0x1, 0x2, 0x3
@@ -184,12 +184,12 @@ class Plan:
 
 
 def plan_for(w, device=0, flags=0) -> Plan:
-    """Plan for a workload record with M, N, K, in_dtype ("f32"/"bf16"), out_dtype,
+    """Plan for a workload record with M, N, K, in_dtype ("f32"/"bf16"/"f16"), out_dtype,
     layout ("row"/"blocked32") and epilogue ("none"/"bias_relu") attributes."""
     lay = BLOCKED32 if w.layout == "blocked32" else ROW_MAJOR
     return Plan(w.M, w.N, w.K,
-                in_dtype=F32 if w.in_dtype == "f32" else BF16,
-                out_dtype=F32 if w.out_dtype == "f32" else BF16,
+                in_dtype={"f32": F32, "bf16": BF16, "f16": F16}[w.in_dtype],
+                out_dtype={"f32": F32, "bf16": BF16, "f16": F16}[w.out_dtype],
                 layout_a=lay, layout_b=lay,
                 epilogue=EPI_BIAS_RELU if w.epilogue == "bias_relu" else EPI_NONE,
                 device=device, flags=flags)

@@ -3,6 +3,7 @@
 // unpacking of a VNNI-blocked B operand into row-major scratch.
 #pragma once
 #include <cuda_bf16.h>
+#include <cuda_fp16.h>
 #include <cuda_runtime.h>
 #include <stdint.h>
 
@@ -10,9 +11,23 @@
 
 namespace nk {
 
+// A 16-bit element is BF16 (its bits are the upper half of the FP32 pattern) or, with `f16`
+// set, IEEE binary16.  Both widen exactly to FP32; a result is rounded once (RNE) on the way out.
+__device__ __forceinline__ float half_bits_to_f32(uint32_t h, int f16) {
+    return f16 ? __half2float(__ushort_as_half(static_cast<unsigned short>(h))) : __uint_as_float(h << 16);
+}
+__device__ __forceinline__ uint32_t pack_half2(float lo, float hi, int f16) {
+    if (f16) {
+        const __half2 v = __floats2half2_rn(lo, hi);
+        return *reinterpret_cast<const uint32_t*>(&v);
+    }
+    const __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
+    return *reinterpret_cast<const uint32_t*>(&v);
+}
+
 struct NaiveParams {
     int M, N, K;
-    int in_bf16, out_bf16, a_blocked, b_blocked, epilogue;
+    int in_bf16, out_bf16, a_blocked, b_blocked, epilogue;   // in_bf16 / out_bf16: 16-bit elements (BF16 or FP16)
     int batch, beta;
     long long stride_a, stride_b;
     int gemms;             // batched matmul: gridDim.z independent GEMMs
@@ -20,11 +35,11 @@ struct NaiveParams {
     int c_blocked;         // C stored as [M/32][N/32][32][32]
     const void *A, *B, *bias;
     void* C;
+    int f16;               // the 16-bit type is IEEE binary16, not BF16
 };
 
-__device__ __forceinline__ float ld_elem(const void* p, int bf16, size_t i) {
-    return bf16 ? __uint_as_float(static_cast<uint32_t>(static_cast<const uint16_t*>(p)[i]) << 16)
-                : static_cast<const float*>(p)[i];
+__device__ __forceinline__ float ld_elem(const void* p, int is16, int f16, size_t i) {
+    return is16 ? half_bits_to_f32(static_cast<const uint16_t*>(p)[i], f16) : static_cast<const float*>(p)[i];
 }
 
 // Debug cross-check only: one thread per C element, FP32 accumulation in k order,
@@ -39,7 +54,7 @@ __global__ void naive_gemm_kernel(const NaiveParams p) {
                      (p.c_blocked ? ((static_cast<size_t>(i / 32) * (p.N / 32) + j / 32) * 32 + i % 32) * 32 + j % 32
                                   : static_cast<size_t>(i) * p.N + j);
     float acc = 0.f;
-    if (p.beta) acc = ld_elem(p.C, p.out_bf16, o);
+    if (p.beta) acc = ld_elem(p.C, p.out_bf16, p.f16, o);
     for (int b = 0; b < p.batch; ++b)
     for (int k = 0; k < p.K; ++k) {
         const size_t ia = p.a_blocked
@@ -48,11 +63,11 @@ __global__ void naive_gemm_kernel(const NaiveParams p) {
         const size_t ib = p.b_blocked
             ? (((((static_cast<size_t>(j / 32) * kb32 + k / 32) * 16 + (k % 32) / 2) * 32 + j % 32) * 2) + k % 2)
             : static_cast<size_t>(k) * p.N + j;
-        acc = fmaf(ld_elem(p.A, p.in_bf16, (g + b) * p.stride_a + ia), ld_elem(p.B, p.in_bf16, (g + b) * p.stride_b + ib), acc);
+        acc = fmaf(ld_elem(p.A, p.in_bf16, p.f16, (g + b) * p.stride_a + ia), ld_elem(p.B, p.in_bf16, p.f16, (g + b) * p.stride_b + ib), acc);
     }
-    if (p.epilogue) acc = fmaxf(acc + ld_elem(p.bias, p.in_bf16, j), 0.f);
+    if (p.epilogue) acc = fmaxf(acc + ld_elem(p.bias, p.in_bf16, p.f16, j), 0.f);
     if (p.out_bf16)
-        static_cast<__nv_bfloat16*>(p.C)[o] = __float2bfloat16_rn(acc);
+        static_cast<uint16_t*>(p.C)[o] = static_cast<uint16_t>(pack_half2(acc, 0.f, p.f16) & 0xFFFFu);
     else
         static_cast<float*>(p.C)[o] = acc;
 }
@@ -68,6 +83,7 @@ struct ReduceParams {
     const float* partial;  // [splits][M][N]
     const void* bias;
     void* C;
+    int f16;               // the 16-bit type (bias_bf16 / out_bf16) is IEEE binary16, not BF16
 };
 
 // C = epilogue(sum over splits, in split order): fixed order, so the result does
@@ -92,8 +108,8 @@ __global__ void splitk_reduce_kernel(const ReduceParams p) {
     if (p.beta) {
         if (p.out_bf16) {
             const uint2 w = *reinterpret_cast<const uint2*>(static_cast<const uint16_t*>(p.C) + ce);
-            s.x += __uint_as_float(w.x << 16); s.y += __uint_as_float(w.x & 0xFFFF0000u);
-            s.z += __uint_as_float(w.y << 16); s.w += __uint_as_float(w.y & 0xFFFF0000u);
+            s.x += half_bits_to_f32(w.x & 0xFFFFu, p.f16); s.y += half_bits_to_f32(w.x >> 16, p.f16);
+            s.z += half_bits_to_f32(w.y & 0xFFFFu, p.f16); s.w += half_bits_to_f32(w.y >> 16, p.f16);
         } else {
             const float4 c = *reinterpret_cast<const float4*>(static_cast<const float*>(p.C) + ce);
             s.x += c.x; s.y += c.y; s.z += c.z; s.w += c.w;
@@ -104,8 +120,8 @@ __global__ void splitk_reduce_kernel(const ReduceParams p) {
         float b0, b1, b2, b3;
         if (p.bias_bf16) {
             const uint2 w = __ldg(reinterpret_cast<const uint2*>(static_cast<const uint16_t*>(p.bias) + n));
-            b0 = __uint_as_float(w.x << 16); b1 = __uint_as_float(w.x & 0xFFFF0000u);
-            b2 = __uint_as_float(w.y << 16); b3 = __uint_as_float(w.y & 0xFFFF0000u);
+            b0 = half_bits_to_f32(w.x & 0xFFFFu, p.f16); b1 = half_bits_to_f32(w.x >> 16, p.f16);
+            b2 = half_bits_to_f32(w.y & 0xFFFFu, p.f16); b3 = half_bits_to_f32(w.y >> 16, p.f16);
         } else {
             const float4 w = __ldg(reinterpret_cast<const float4*>(static_cast<const float*>(p.bias) + n));
             b0 = w.x; b1 = w.y; b2 = w.z; b3 = w.w;
@@ -114,10 +130,9 @@ __global__ void splitk_reduce_kernel(const ReduceParams p) {
         s.z = fmaxf(s.z + b2, 0.f); s.w = fmaxf(s.w + b3, 0.f);
     }
     if (p.out_bf16) {
-        __nv_bfloat162 lo = __floats2bfloat162_rn(s.x, s.y), hi = __floats2bfloat162_rn(s.z, s.w);
         uint2 o;
-        o.x = *reinterpret_cast<uint32_t*>(&lo);
-        o.y = *reinterpret_cast<uint32_t*>(&hi);
+        o.x = pack_half2(s.x, s.y, p.f16);
+        o.y = pack_half2(s.z, s.w, p.f16);
         *reinterpret_cast<uint2*>(static_cast<uint16_t*>(p.C) + ce) = o;
     } else {
         *reinterpret_cast<float4*>(static_cast<float*>(p.C) + ce) = s;

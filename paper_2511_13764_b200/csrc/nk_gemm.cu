@@ -89,17 +89,18 @@ struct DeviceGuard {
     }
 };
 
+static inline bool is16(int dt) { return dt == NK_BF16 || dt == NK_F16; }   // a 16-bit element type
 static inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 static inline int ceil_div(int64_t a, int64_t b) { return static_cast<int>((a + b - 1) / b); }
 
-// tcgen05 instruction descriptor, kind::f16: D format FP32 (bit 4), A and B format
-// BF16 (bits 7, 10), B major-ness (bit 16: 0 = K-major, 1 = N-major), N/8 at bit 17,
+// tcgen05 instruction descriptor, kind::f16: D format FP32 (bit 4), A and B format at bits 7 and
+// 10 (0 = FP16, 1 = BF16), B major-ness (bit 16: 0 = K-major, 1 = N-major), N/8 at bit 17,
 // M/16 at bit 24.  A is always K-major.
-static uint32_t make_idesc(int m, int n, bool b_n_major) {
+static uint32_t make_idesc(int m, int n, bool b_n_major, bool f16) {
     uint32_t d = 0;
     d |= 1u << 4;
-    d |= 1u << 7;
-    d |= 1u << 10;
+    d |= (f16 ? 0u : 1u) << 7;
+    d |= (f16 ? 0u : 1u) << 10;
     d |= (b_n_major ? 1u : 0u) << 16;
     d |= static_cast<uint32_t>(n >> 3) << 17;
     d |= static_cast<uint32_t>(m >> 4) << 24;
@@ -157,7 +158,7 @@ static double umma_model_us(const nk_gemm_desc_t& d, int sms, bool pair, int bn,
         const double vnni = 0.14 + bn * 0.0042;
         if (vnni > t_kb) t_kb = vnni;
     }
-    const double eo = d.out_dtype == NK_BF16 ? 2.0 : 4.0;
+    const double eo = is16(d.out_dtype) ? 2.0 : 4.0;
     const double mn = static_cast<double>(d.M) * d.N;
     const double chunks = bn / 32.0;
     double us = (pair ? 7.0 : 6.0) + rounds * per * t_kb;
@@ -302,6 +303,7 @@ static void choose_skinny(nk_gemm_s* p) {
 static nk_status_t encode_maps(nk_gemm_s* p, const void* A, const void* B) {
     if (p->cached_a == A && p->cached_b == B) return NK_OK;
     const nk_gemm_desc_t& d = p->d;
+    const CUtensorMapDataType half_type = d.in_dtype == NK_F16 ? CU_TENSOR_MAP_DATA_TYPE_FLOAT16 : CU_TENSOR_MAP_DATA_TYPE_BFLOAT16;
     CUresult r;
     if (d.layout_a == NK_BLOCKED32) {
         // [M/32][K/32][32][32] as a 4-D tensor (k, m, k-block, m-block): a box of
@@ -310,7 +312,7 @@ static nk_status_t encode_maps(nk_gemm_s* p, const void* A, const void* B) {
         cuuint64_t strides[3] = {32 * 2, 1024 * 2, static_cast<cuuint64_t>(d.K / 32) * 1024 * 2};
         cuuint32_t box[4] = {32, 32, 1, 4};
         cuuint32_t es[4] = {1, 1, 1, 1};
-        r = p->encode(&p->tmap_a, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void*>(A), dims, strides,
+        r = p->encode(&p->tmap_a, half_type, 4, const_cast<void*>(A), dims, strides,
                       box, es, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_64B,
                       CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
     } else {
@@ -320,7 +322,7 @@ static nk_status_t encode_maps(nk_gemm_s* p, const void* A, const void* B) {
         cuuint64_t strides[2] = {static_cast<cuuint64_t>(d.K) * 2, static_cast<cuuint64_t>(p->stride_a) * 2};
         cuuint32_t box[3] = {UMMA_BK, UMMA_BM, 1};
         cuuint32_t es[3] = {1, 1, 1};
-        r = p->encode(&p->tmap_a, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(A), dims, strides,
+        r = p->encode(&p->tmap_a, half_type, 3, const_cast<void*>(A), dims, strides,
                       box, es, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
                       CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
     }
@@ -341,7 +343,7 @@ static nk_status_t encode_maps(nk_gemm_s* p, const void* A, const void* B) {
             cuuint64_t strides[3] = {static_cast<cuuint64_t>(d.N) * 2, 128, static_cast<cuuint64_t>(p->stride_b) * 2};
             cuuint32_t box[4] = {64, UMMA_BK, static_cast<cuuint32_t>(slabs), 1};
             cuuint32_t es[4] = {1, 1, 1, 1};
-            r = p->encode(&p->tmap_b, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void*>(B), dims, strides,
+            r = p->encode(&p->tmap_b, half_type, 4, const_cast<void*>(B), dims, strides,
                           box, es, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
                           CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
             if (r != CUDA_SUCCESS) p->b_3d = false;   // fall back to per-slab boxes
@@ -353,7 +355,7 @@ static nk_status_t encode_maps(nk_gemm_s* p, const void* A, const void* B) {
             cuuint64_t strides[2] = {static_cast<cuuint64_t>(d.N) * 2, static_cast<cuuint64_t>(p->stride_b) * 2};
             cuuint32_t box[3] = {64, UMMA_BK, 1};
             cuuint32_t es[3] = {1, 1, 1};
-            r = p->encode(&p->tmap_b, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(B), dims, strides,
+            r = p->encode(&p->tmap_b, half_type, 3, const_cast<void*>(B), dims, strides,
                           box, es, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
                           CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
         }
@@ -374,14 +376,14 @@ static nk_status_t encode_maps(nk_gemm_s* p, const void* A, const void* B) {
 static nk_status_t encode_c_map(nk_gemm_s* p, void* C) {
     if (!p->tma_store || p->cached_c == C) return NK_OK;
     const nk_gemm_desc_t& d = p->d;
-    const bool bf16 = d.out_dtype == NK_BF16;
+    const bool bf16 = is16(d.out_dtype);
     const cuuint64_t es_bytes = bf16 ? 2 : 4;
     cuuint64_t dims[3] = {static_cast<cuuint64_t>(d.N), static_cast<cuuint64_t>(d.M), static_cast<cuuint64_t>(p->gemms)};
     cuuint64_t strides[2] = {static_cast<cuuint64_t>(d.N) * es_bytes, static_cast<cuuint64_t>(p->stride_c) * es_bytes};
     cuuint32_t box[3] = {32, 32, 1};
     cuuint32_t es[3] = {1, 1, 1};
     // a box row is 128 bytes of FP32 (128-byte swizzle) or 64 bytes of BF16 (64-byte swizzle)
-    CUresult r = p->encode(&p->tmap_c, bf16 ? CU_TENSOR_MAP_DATA_TYPE_BFLOAT16 : CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 3, C,
+    CUresult r = p->encode(&p->tmap_c, !bf16 ? CU_TENSOR_MAP_DATA_TYPE_FLOAT32 : d.out_dtype == NK_F16 ? CU_TENSOR_MAP_DATA_TYPE_FLOAT16 : CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, C,
                            dims, strides, box, es, CU_TENSOR_MAP_INTERLEAVE_NONE,
                            bf16 ? CU_TENSOR_MAP_SWIZZLE_64B : CU_TENSOR_MAP_SWIZZLE_128B,
                            CU_TENSOR_MAP_L2_PROMOTION_NONE, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
@@ -568,14 +570,14 @@ nk_status_t nk_gemm_create(const nk_gemm_desc_t* desc, nk_gemm_t* out) {
     if (d.M <= 0 || d.N <= 0 || d.K <= 0) return NK_ERR_INVALID_ARG;
     if (d.M > (1 << 24) || d.N > (1 << 24) || d.K > (1 << 24)) return NK_ERR_UNSUPPORTED;
     if (d.M * d.N >= (1ll << 31) || d.M * d.K >= (1ll << 33) || d.K * d.N >= (1ll << 33)) return NK_ERR_UNSUPPORTED;
-    if (d.in_dtype != NK_F32 && d.in_dtype != NK_BF16) return NK_ERR_INVALID_ARG;
-    if (d.out_dtype != NK_F32 && d.out_dtype != NK_BF16) return NK_ERR_INVALID_ARG;
+    if (d.in_dtype != NK_F32 && !is16(d.in_dtype)) return NK_ERR_INVALID_ARG;
+    if (d.out_dtype != NK_F32 && !is16(d.out_dtype)) return NK_ERR_INVALID_ARG;
     if (d.layout_a != NK_ROW_MAJOR && d.layout_a != NK_BLOCKED32) return NK_ERR_INVALID_ARG;
     if (d.layout_b != NK_ROW_MAJOR && d.layout_b != NK_BLOCKED32) return NK_ERR_INVALID_ARG;
     if (d.epilogue != NK_EPI_NONE && d.epilogue != NK_EPI_BIAS_RELU) return NK_ERR_INVALID_ARG;
-    if (d.out_dtype == NK_BF16 && d.in_dtype != NK_BF16) return NK_ERR_INVALID_ARG;
+    if (is16(d.out_dtype) && d.in_dtype != d.out_dtype) return NK_ERR_INVALID_ARG;   // a 16-bit C has the operands' type
     const bool blocked = d.layout_a == NK_BLOCKED32 || d.layout_b == NK_BLOCKED32;
-    if (blocked && d.in_dtype != NK_BF16) return NK_ERR_UNSUPPORTED;
+    if (blocked && !is16(d.in_dtype)) return NK_ERR_UNSUPPORTED;
     if (d.layout_a == NK_BLOCKED32 && (d.M % 32 || d.K % 32)) return NK_ERR_MISALIGNED;
     if (d.layout_b == NK_BLOCKED32 && (d.N % 32 || d.K % 32)) return NK_ERR_MISALIGNED;
     if (d.beta != 0 && d.beta != 1) return NK_ERR_INVALID_ARG;
@@ -586,13 +588,13 @@ nk_status_t nk_gemm_create(const nk_gemm_desc_t* desc, nk_gemm_t* out) {
     if (nbatch > 1) {
         if (blocked) return NK_ERR_UNSUPPORTED;          // batch-reduce: row-major operands only
         if (nbatch > 65535 || nbatch * d.K >= (1ll << 24)) return NK_ERR_UNSUPPORTED;
-        const int64_t gran = d.in_dtype == NK_BF16 ? 8 : 4;
+        const int64_t gran = is16(d.in_dtype) ? 8 : 4;
         if (str_a % gran || str_b % gran) return NK_ERR_MISALIGNED;
         if (str_a < d.M * d.K || str_b < d.K * d.N) return NK_ERR_INVALID_ARG;   // items must not overlap
     }
     if (d.layout_c != NK_ROW_MAJOR && d.layout_c != NK_BLOCKED32) return NK_ERR_INVALID_ARG;
     if (d.layout_c == NK_BLOCKED32) {
-        if (d.in_dtype != NK_BF16) return NK_ERR_UNSUPPORTED;
+        if (!is16(d.in_dtype)) return NK_ERR_UNSUPPORTED;
         if (d.M % 32 || d.N % 32) return NK_ERR_MISALIGNED;
     }
     if (d.batch_independent != 0 && d.batch_independent != 1) return NK_ERR_INVALID_ARG;
@@ -600,7 +602,7 @@ nk_status_t nk_gemm_create(const nk_gemm_desc_t* desc, nk_gemm_t* out) {
     const int64_t str_c = d.stride_c > 0 ? d.stride_c : d.M * d.N;
     const bool indep = d.batch_independent == 1 && nbatch > 1;
     if (indep) {
-        const int64_t gran_c = d.out_dtype == NK_BF16 ? 8 : 4;
+        const int64_t gran_c = is16(d.out_dtype) ? 8 : 4;
         if (str_c % gran_c) return NK_ERR_MISALIGNED;
         if (str_c < d.M * d.N) return NK_ERR_INVALID_ARG;
         if (nbatch * d.M * d.N >= (1ll << 31)) return NK_ERR_UNSUPPORTED;
@@ -608,10 +610,10 @@ nk_status_t nk_gemm_create(const nk_gemm_desc_t* desc, nk_gemm_t* out) {
     const uint32_t force = d.flags & NK_FLAG_KERNEL_MASK;
     if (force > NK_FLAG_KERNEL_UMMA) return NK_ERR_INVALID_ARG;
     if (force != NK_FLAG_KERNEL_NAIVE) {
-        if (d.in_dtype == NK_BF16 && (d.N % 8 || d.K % 8)) return NK_ERR_MISALIGNED;
+        if (is16(d.in_dtype) && (d.N % 8 || d.K % 8)) return NK_ERR_MISALIGNED;
         if (d.in_dtype == NK_F32 && (d.N % 4 || d.K % 4)) return NK_ERR_MISALIGNED;
         if (force == NK_FLAG_KERNEL_SIMT && d.in_dtype != NK_F32) return NK_ERR_UNSUPPORTED;
-        if (force == NK_FLAG_KERNEL_UMMA && d.in_dtype != NK_BF16) return NK_ERR_UNSUPPORTED;
+        if (force == NK_FLAG_KERNEL_UMMA && !is16(d.in_dtype)) return NK_ERR_UNSUPPORTED;
     }
 
     int ndev = 0;
@@ -717,6 +719,10 @@ nk_status_t nk_gemm_create(const nk_gemm_desc_t* desc, nk_gemm_t* out) {
         const size_t len = strlen(p->name);
         snprintf(p->name + len, sizeof(p->name) - len, "_cblk");
     }
+    if (d.in_dtype == NK_F16) {
+        const size_t len = strlen(p->name);
+        snprintf(p->name + len, sizeof(p->name) - len, "_f16");
+    }
     // split-K partials are laid out [split][gemm][M][N] and reduced as one flat array: that
     // needs the C of a batched matmul to be contiguous
     if (p->gemms > 1 && p->splits > 1 && p->stride_c != d.M * d.N && !p->cluster_reduce) {
@@ -753,9 +759,9 @@ nk_status_t nk_gemm_run(nk_gemm_t p, const void* A, const void* B, const void* b
 
     if (p->variant == V_NAIVE) {
         NaiveParams np = {static_cast<int>(d.M), static_cast<int>(d.N), static_cast<int>(d.K),
-                          d.in_dtype == NK_BF16, d.out_dtype == NK_BF16, d.layout_a == NK_BLOCKED32,
+                          is16(d.in_dtype), is16(d.out_dtype), d.layout_a == NK_BLOCKED32,
                           d.layout_b == NK_BLOCKED32, d.epilogue, p->batch, d.beta, p->stride_a, p->stride_b,
-                          p->gemms, p->stride_c, d.layout_c == NK_BLOCKED32, A, B, bias, C};
+                          p->gemms, p->stride_c, d.layout_c == NK_BLOCKED32, A, B, bias, C, d.in_dtype == NK_F16};
         dim3 grid(ceil_div(d.N, 128), static_cast<unsigned>(d.M), static_cast<unsigned>(p->gemms));
         if (d.M > 65535) return NK_ERR_UNSUPPORTED;
         naive_gemm_kernel<<<grid, 128, 0, st>>>(np);
@@ -817,8 +823,9 @@ nk_status_t nk_gemm_run(nk_gemm_t p, const void* A, const void* B, const void* b
         up.a_blocked = d.layout_a == NK_BLOCKED32;
         up.b_3d = p->b_3d ? 1 : 0;
         up.epilogue = d.epilogue;
-        up.out_bf16 = d.out_dtype == NK_BF16;
-        up.idesc = make_idesc(p->pair ? 2 * UMMA_BM : UMMA_BM, p->bn, !p->b_vnni_inkernel);
+        up.out_bf16 = is16(d.out_dtype);
+        up.idesc = make_idesc(p->pair ? 2 * UMMA_BM : UMMA_BM, p->bn, !p->b_vnni_inkernel, d.in_dtype == NK_F16);
+        up.f16 = d.in_dtype == NK_F16;
         up.bias = bias;
         up.C = C;
         up.partial = partial;
@@ -839,8 +846,8 @@ nk_status_t nk_gemm_run(nk_gemm_t p, const void* A, const void* B, const void* b
 
     if (p->splits > 1 && !p->cluster_reduce) {
         ReduceParams rp = {static_cast<size_t>(p->gemms) * d.M * d.N, static_cast<int>(d.N), p->splits, d.epilogue,
-                           d.in_dtype == NK_BF16, d.out_dtype == NK_BF16, d.beta, d.layout_c == NK_BLOCKED32,
-                           static_cast<int>(d.M), partial, bias, C};
+                           is16(d.in_dtype), is16(d.out_dtype), d.beta, d.layout_c == NK_BLOCKED32,
+                           static_cast<int>(d.M), partial, bias, C, d.in_dtype == NK_F16};
         const size_t quads = rp.MN / 4;
         splitk_reduce_kernel<<<static_cast<unsigned>((quads + 255) / 256), 256, 0, st>>>(rp);
         e = cudaGetLastError();
@@ -855,7 +862,7 @@ nk_status_t nk_gemm_run_host(nk_gemm_t p, const void* hA, const void* hB, const 
     if (!p || !hA || !hB || !hC || !dA || !dB || !dC) return NK_ERR_INVALID_ARG;
     const nk_gemm_desc_t& d = p->d;
     if (d.epilogue != NK_EPI_NONE && (!hbias || !dbias)) return NK_ERR_INVALID_ARG;
-    const size_t ein = d.in_dtype == NK_BF16 ? 2 : 4, eout = d.out_dtype == NK_BF16 ? 2 : 4;
+    const size_t ein = is16(d.in_dtype) ? 2 : 4, eout = is16(d.out_dtype) ? 2 : 4;
     cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
     DeviceGuard guard(d.device);
     if (guard.err != cudaSuccess) { set_err(p, "cudaSetDevice", guard.err); return NK_ERR_DEVICE; }

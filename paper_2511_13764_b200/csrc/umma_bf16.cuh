@@ -31,6 +31,7 @@
 #pragma once
 #include <cuda.h>
 #include <cuda_bf16.h>
+#include "aux_kernels.cuh"
 #include "ptx.cuh"
 
 namespace nk {
@@ -56,7 +57,8 @@ struct UmmaParams {
     int a_blocked;      // A tensor map is the 4-D blocked view
     int b_3d;           // B tensor map is the 3-D (n-in-slab, k, slab) view: one box per stage
     int epilogue;       // 0 none, 1 bias + ReLU
-    int out_bf16;       // C element type
+    int out_bf16;       // C is 16 bits wide (the operands' type), else FP32
+    int f16;            // the 16-bit type of A, B, bias (and C) is IEEE binary16 instead of BF16
     uint32_t idesc;     // tcgen05 instruction descriptor
     const void* bias;   // BF16 [N] or null
     void* C;            // [M][N] FP32 or BF16
@@ -96,13 +98,6 @@ __device__ __forceinline__ void umma_decode_unit(const UmmaParams& p, int unit, 
     const int u = unit - gemm * per_gemm;
     tile = u / p.splits;
     split = u - tile * p.splits;
-}
-
-__device__ __forceinline__ float bf16_bits_to_f32(uint32_t h) { return __uint_as_float(h << 16); }
-
-__device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi) {
-    __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
-    return *reinterpret_cast<uint32_t*>(&v);
 }
 
 // Epilogue for one 32 x 32 chunk of the accumulator: lane t holds row `row0 + t`, columns
@@ -145,8 +140,8 @@ __device__ __forceinline__ void umma_store_chunk(const UmmaParams& p, const CUte
                 const uint32_t w[4] = {c.x, c.y, c.z, c.w};
 #pragma unroll
                 for (int j = 0; j < 4; ++j) {
-                    v[8 * g + 2 * j] = __float_as_uint(__uint_as_float(v[8 * g + 2 * j]) + bf16_bits_to_f32(w[j] & 0xFFFFu));
-                    v[8 * g + 2 * j + 1] = __float_as_uint(__uint_as_float(v[8 * g + 2 * j + 1]) + bf16_bits_to_f32(w[j] >> 16));
+                    v[8 * g + 2 * j] = __float_as_uint(__uint_as_float(v[8 * g + 2 * j]) + half_bits_to_f32(w[j] & 0xFFFFu, p.f16));
+                    v[8 * g + 2 * j + 1] = __float_as_uint(__uint_as_float(v[8 * g + 2 * j + 1]) + half_bits_to_f32(w[j] >> 16, p.f16));
                 }
             }
         } else {
@@ -171,8 +166,8 @@ __device__ __forceinline__ void umma_store_chunk(const UmmaParams& p, const CUte
             const uint32_t w[4] = {b.x, b.y, b.z, b.w};
 #pragma unroll
             for (int j = 0; j < 4; ++j) {
-                float x0 = __uint_as_float(v[8 * g + 2 * j]) + bf16_bits_to_f32(w[j] & 0xFFFFu);
-                float x1 = __uint_as_float(v[8 * g + 2 * j + 1]) + bf16_bits_to_f32(w[j] >> 16);
+                float x0 = __uint_as_float(v[8 * g + 2 * j]) + half_bits_to_f32(w[j] & 0xFFFFu, p.f16);
+                float x1 = __uint_as_float(v[8 * g + 2 * j + 1]) + half_bits_to_f32(w[j] >> 16, p.f16);
                 v[8 * g + 2 * j] = __float_as_uint(fmaxf(x0, 0.0f));
                 v[8 * g + 2 * j + 1] = __float_as_uint(fmaxf(x1, 0.0f));
             }
@@ -187,10 +182,10 @@ __device__ __forceinline__ void umma_store_chunk(const UmmaParams& p, const CUte
 #pragma unroll
         for (int g = 0; g < 4; ++g) {
             uint4 o;
-            o.x = pack_bf16x2(__uint_as_float(v[8 * g]), __uint_as_float(v[8 * g + 1]));
-            o.y = pack_bf16x2(__uint_as_float(v[8 * g + 2]), __uint_as_float(v[8 * g + 3]));
-            o.z = pack_bf16x2(__uint_as_float(v[8 * g + 4]), __uint_as_float(v[8 * g + 5]));
-            o.w = pack_bf16x2(__uint_as_float(v[8 * g + 6]), __uint_as_float(v[8 * g + 7]));
+            o.x = pack_half2(__uint_as_float(v[8 * g]), __uint_as_float(v[8 * g + 1]), p.f16);
+            o.y = pack_half2(__uint_as_float(v[8 * g + 2]), __uint_as_float(v[8 * g + 3]), p.f16);
+            o.z = pack_half2(__uint_as_float(v[8 * g + 4]), __uint_as_float(v[8 * g + 5]), p.f16);
+            o.w = pack_half2(__uint_as_float(v[8 * g + 6]), __uint_as_float(v[8 * g + 7]), p.f16);
             *reinterpret_cast<uint4*>(tile + lane * 64 + ((g ^ ((lane >> 1) & 3)) << 4)) = o;
         }
         fence_proxy_async_smem();
@@ -208,10 +203,10 @@ __device__ __forceinline__ void umma_store_chunk(const UmmaParams& p, const CUte
         for (int g = 0; g < 4; ++g)
             if (col0 + 8 * g < p.N) {
                 uint4 o;
-                o.x = pack_bf16x2(__uint_as_float(v[8 * g]), __uint_as_float(v[8 * g + 1]));
-                o.y = pack_bf16x2(__uint_as_float(v[8 * g + 2]), __uint_as_float(v[8 * g + 3]));
-                o.z = pack_bf16x2(__uint_as_float(v[8 * g + 4]), __uint_as_float(v[8 * g + 5]));
-                o.w = pack_bf16x2(__uint_as_float(v[8 * g + 6]), __uint_as_float(v[8 * g + 7]));
+                o.x = pack_half2(__uint_as_float(v[8 * g]), __uint_as_float(v[8 * g + 1]), p.f16);
+                o.y = pack_half2(__uint_as_float(v[8 * g + 2]), __uint_as_float(v[8 * g + 3]), p.f16);
+                o.z = pack_half2(__uint_as_float(v[8 * g + 4]), __uint_as_float(v[8 * g + 5]), p.f16);
+                o.w = pack_half2(__uint_as_float(v[8 * g + 6]), __uint_as_float(v[8 * g + 7]), p.f16);
                 *reinterpret_cast<uint4*>(dst + 8 * g) = o;
             }
         return;

@@ -35,8 +35,8 @@ def time_workload(w, iters, flags=0, flush=None):
     import torch
     import paper_2511_13764_b200 as nk
     dev = torch.device("cuda", 0)
-    ein = torch.float32 if w.in_dtype == "f32" else torch.bfloat16
-    eout = torch.float32 if w.out_dtype == "f32" else torch.bfloat16
+    tt = {"f32": torch.float32, "bf16": torch.bfloat16, "f16": torch.float16}
+    ein, eout = tt[w.in_dtype], tt[w.out_dtype]
     g = torch.Generator(device=dev).manual_seed(w.seed)
     A = (torch.rand(w.M * w.K, device=dev, generator=g) * 2 - 1).to(ein)
     B = (torch.rand(w.K * w.N, device=dev, generator=g) * 2 - 1).to(ein)
@@ -84,7 +84,7 @@ def main():
     prop = torch.cuda.get_device_properties(0)
     fma_peak = prop.multi_processor_count * 128 * 2 * 1.965e9 / 1e12
     flush = None if args.no_flush else torch.empty(512 << 20, dtype=torch.uint8, device="cuda")
-    works = [nk_inputs.config(i) for i in (1, 2, 3, 4)] + nk_inputs.sweep() + nk_inputs.paper_mlp()
+    works = [nk_inputs.config(i) for i in (1, 2, 3, 4)] + nk_inputs.sweep() + nk_inputs.paper_mlp() + nk_inputs.f16_set()
     rows = []
     print(f"| workload | kernel | launches | median us | TFLOP/s | alg. GB/s | bound | frac ({src}) |")
     print("|---|---|---|---|---|---|---|---|")
@@ -94,13 +94,13 @@ def main():
         med, best, kname, launches = time_workload(w, args.iters, flags=args.flags, flush=flush)
         tf = w.flops / (med * 1e-3) / 1e12
         gbs = w.algorithmic_bytes / (med * 1e-3) / 1e9
-        compute_peak = tensor_peak if w.in_dtype == "bf16" else fma_peak
+        compute_peak = tensor_peak if w.in_dtype != "f32" else fma_peak
         t_compute = w.flops / (compute_peak * 1e12)
         t_hbm = w.algorithmic_bytes / (hbm_peak * 1e9)
         if t_hbm >= t_compute:
             bound, frac = "hbm", gbs / hbm_peak
         else:
-            bound, frac = ("tensor" if w.in_dtype == "bf16" else "alu"), tf / compute_peak
+            bound, frac = ("tensor" if w.in_dtype != "f32" else "alu"), tf / compute_peak
         rows.append(dict(workload=w.name, kernel=kname, launches=launches, median_us=med * 1e3,
                          best_us=best * 1e3, tflops=tf, gbs=gbs, bound=bound, frac=frac))
         print(f"| {w.name} | {kname} | {launches} | {med * 1e3:.1f} | {tf:.1f} | {gbs:.0f} | {bound} | {frac:.3f} |",

@@ -11,9 +11,12 @@ import paper_2511_13764_b200 as nk
 
 TOL_REL_SMAX = 1e-5         # |c - y| <= 1e-5 * max sum_k |a.b|      (FP32 output)
 TOL_BF16_REL = 2.0 ** -8    # + 2^-8 * |y| for a BF16-stored output  (one final RNE)
+TOL_F16_REL = 2.0 ** -11    # + 2^-11 * |y| for an FP16-stored output (half an ulp of 11 significant bits)
+TOL_F16_ABS = 2.0 ** -25    # + half the spacing of FP16 subnormals, for results below 2^-14
 
 
 def to_device(buf: np.ndarray, device="cuda:0") -> torch.Tensor:
+    """16-bit patterns travel as bfloat16 tensors whatever they encode: only the bytes matter."""
     t = torch.from_numpy(buf)
     if buf.dtype == np.uint16:
         t = t.view(torch.bfloat16)
@@ -21,6 +24,8 @@ def to_device(buf: np.ndarray, device="cuda:0") -> torch.Tensor:
 
 
 def c_to_f64(C: torch.Tensor) -> np.ndarray:
+    if C.dtype == torch.float16:
+        return C.cpu().numpy().astype(np.float64)
     if C.dtype == torch.bfloat16:
         bits = C.cpu().view(torch.int16).numpy().view(np.uint16)
         return (bits.astype(np.uint32) << 16).view(np.float32).astype(np.float64)
@@ -35,7 +40,7 @@ def run_plan(w, A, B, bias, flags=0, poison=True, device="cuda:0", plan=None):
         plan = nk.plan_for(w, device=torch.device(device).index or 0, flags=flags)
     dA, dB = to_device(A, device), to_device(B, device)
     dbias = to_device(bias, device) if bias is not None else None
-    out_dt = torch.float32 if w.out_dtype == "f32" else torch.bfloat16
+    out_dt = {"f32": torch.float32, "bf16": torch.bfloat16, "f16": torch.float16}[w.out_dtype]
     pad = 1024
     Cbuf = torch.full((w.M * w.N + 2 * pad,), float("nan") if poison else 0.0, dtype=out_dt, device=device)
     Cbuf[:pad] = 7.0
@@ -80,6 +85,8 @@ def check_against_oracle(w, got, A, B, bias, rows=None, cols=None, exact=False):
     tol = TOL_REL_SMAX * smax
     if w.out_dtype == "bf16":
         tol = tol + TOL_BF16_REL * np.abs(Y)
+    if w.out_dtype == "f16":
+        tol = tol + TOL_F16_REL * np.abs(Y) + TOL_F16_ABS
     err = np.abs(g - Y)
     bad = err > tol
     assert not bad.any(), describe_mismatch(g, Y, bad) + f" (Smax={smax:.4g})"

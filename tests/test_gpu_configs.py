@@ -37,6 +37,8 @@ def _make(w):
 def _as_f64(buf, dtype):
     if dtype == "bf16":
         return (buf.astype(np.uint32) << 16).view(np.float32).astype(np.float64)
+    if dtype == "f16":
+        return buf.view(np.float16).astype(np.float64)
     return buf.astype(np.float64)
 
 
@@ -107,3 +109,12 @@ def test_config5_sweep(w):
 @pytest.mark.parametrize("w", nk_inputs.paper_mlp(), ids=lambda w: w.name)
 def test_paper_mlp_grid(w):
     check_workload(w)
+
+
+@pytest.mark.parametrize("i", [0, 1, 2])
+def test_f16_headline_shapes(i):
+    """FP16 operands at full size: 8192^3 on 64 stratified rows plus the Freivalds identity, the two
+    MLP layers element by element."""
+    w = nk_inputs.f16_set()[i]
+    err, plan = check_workload(w)
+    assert plan.kernel_name.endswith("_f16")
