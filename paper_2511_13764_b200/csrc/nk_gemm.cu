@@ -125,16 +125,21 @@ struct UmmaChoice { bool pair; int bn; int splits; double us; };
 static int desc_batch(const nk_gemm_desc_t& d) { return (d.batch > 1 && !d.batch_independent) ? static_cast<int>(d.batch) : 1; }
 static int desc_gemms(const nk_gemm_desc_t& d) { return (d.batch > 1 && d.batch_independent) ? static_cast<int>(d.batch) : 1; }
 
+// Co-resident clusters of the cluster split-K variant (pair?, tile N, VNNI?, splits), as the driver
+// reports them for this device; asked once per variant and remembered.
+static int max_clusters_for(bool pair, int bn, bool vnni, int splits);
+
 // K splits can meet inside a cluster (no partials in global memory, no second kernel) when there
-// are 2, 4 or 8 of them (2 or 4 pairs), and all the units of the plan fit the GPU at once (large
-// clusters leave a few SMs of every GPC unused: allow for that; the driver is asked at creation).
+// are 2, 4 or 8 of them (2 or 4 pairs) and all the units of the plan are resident at once (one
+// unit per CTA; large clusters leave a few SMs of every GPC unused, which the driver's answer
+// accounts for).
 static bool cluster_reduce_fits(const nk_gemm_desc_t& d, int sms, bool pair, int bn, int eff_splits) {
+    (void)sms;
     if (d.flags & NK_FLAG_SEPARATE_REDUCE) return false;
     if (eff_splits != 2 && eff_splits != 4 && !(eff_splits == 8 && !pair)) return false;
-    const int cluster = pair ? 2 * eff_splits : eff_splits;
-    const int64_t ctas = static_cast<int64_t>(desc_gemms(d)) * ceil_div(d.M, pair ? 2 * UMMA_BM : UMMA_BM) * ceil_div(d.N, bn) * cluster;
-    const int usable = cluster == 8 ? sms - sms / 9 : cluster == 4 ? sms - 4 : sms;
-    return ctas <= usable;
+    const int64_t clusters = static_cast<int64_t>(desc_gemms(d)) * ceil_div(d.M, pair ? 2 * UMMA_BM : UMMA_BM) * ceil_div(d.N, bn);
+    const bool vnni = d.layout_b == NK_BLOCKED32 && !(d.flags & NK_FLAG_REPACK_B);
+    return clusters <= max_clusters_for(pair, bn, vnni, eff_splits);
 }
 
 static double umma_model_us(const nk_gemm_desc_t& d, int sms, bool pair, int bn, int splits) {
@@ -145,28 +150,37 @@ static double umma_model_us(const nk_gemm_desc_t& d, int sms, bool pair, int bn,
     const int64_t units = tiles * eff_splits;
     const int workers = pair ? sms / 2 : sms;
     const double rounds = static_cast<double>((units + workers - 1) / workers);
-    // Fitted to timelines taken inside the kernels on B200: a k-block costs about the same whatever
-    // the tile width (the SM's operand feed from L2, ~50 bytes per clock, or the MMA itself at
-    // N = 256); the epilogue of the last tile is not hidden and is bound by the SM's store path
-    // (~0.35 us per 32 columns, 0.5 us in a pair); a cluster reduction costs two cluster barriers
-    // plus the accumulator pieces that cross to other SMs as 4 KB bulk copies (~40 KB per microsecond per CTA).
-    double t_kb;  // microseconds per 64-wide k-block of one unit
-    if (pair) t_kb = bn == 256 ? (rounds > 1 ? 0.385 : 0.36) : 0.345;
-    else t_kb = bn == 256 ? 0.46 : bn == 128 ? 0.345 : 0.31;
+    // Fitted to kernel-only durations (one-pass ncu captures, cold L2) of every variant on the MLP
+    // shapes.  A k-block costs 0.33-0.38 us whatever the tile (the SM's operand feed from L2, or
+    // the MMA at N = 256), a little more when nearly every SM streams at once; start-up is
+    // 5.4-7.3 us; the epilogue of the last tile is not hidden (0.35 us per 32 columns, 0.5 in a
+    // pair: the SM's store path); a cluster reduction costs 2.4 us (barrier, receive wait) plus
+    // 1.2 us per 32 x 32 piece a warp sends: the SM-to-SM path moves only ~13 KB per microsecond
+    // per CTA, so two splits (half of the pieces stay at home) beat four.
+    const bool busy = units > 100;
+    double t_kb, start;  // microseconds per 64-wide k-block of one unit; start-up of the kernel
+    if (pair) {
+        t_kb = bn == 256 ? (rounds > 1 ? 0.385 : busy ? 0.34 : 0.325) : (busy ? 0.35 : 0.335);
+        start = bn == 256 ? 7.3 : 6.4;
+    } else {
+        t_kb = bn == 256 ? (busy ? 0.42 : 0.37) : bn == 128 ? (busy ? 0.35 : 0.335) : 0.33;
+        start = bn == 256 ? 6.0 : bn == 128 ? 5.4 : 5.8;
+    }
     if (d.layout_b == NK_BLOCKED32 && !(d.flags & NK_FLAG_REPACK_B)) {
         // VNNI-blocked B is re-laid by four warps through the LSU: its cost grows with the columns a CTA covers
         const double vnni = 0.14 + bn * 0.0042;
         if (vnni > t_kb) t_kb = vnni;
     }
-    const double eo = is16(d.out_dtype) ? 2.0 : 4.0;
+    const double eo = d.out_dtype == NK_F32 ? 4.0 : 2.0;
     const double mn = static_cast<double>(d.M) * d.N;
     const double chunks = bn / 32.0;
-    double us = (pair ? 7.0 : 6.0) + rounds * per * t_kb;
+    double us = start + rounds * per * t_kb;
     if (eff_splits > 1 && cluster_reduce_fits(d, sms, pair, bn, eff_splits)) {
-        us += 2.0 + bn * 512.0 * (eff_splits - 1) / eff_splits / 40.0e3 + chunks / eff_splits * (pair ? 0.5 : 0.4);
+        us += 2.4 + 1.2 * chunks * (eff_splits - 1) / eff_splits + (pair ? 0.5 : 0.0);
     } else {
         us += chunks * (pair ? 0.5 : 0.35);
-        if (eff_splits > 1) us += 3.0 + eff_splits * mn * 4.0 / 3.0e6 + (eff_splits * 4.0 + eo) * mn / 5.0e6;
+        // two kernels: the reduce kernel, the gap before it, and the partials written and read back
+        if (eff_splits > 1) us += 5.5 + eff_splits * mn * 4.0 / 3.0e6 + (eff_splits * 4.0 + eo) * mn / 5.0e6;
     }
     const double bytes = 2.0 * desc_batch(d) * (static_cast<double>(d.M) * d.K + static_cast<double>(d.K) * d.N) + eo * mn;
     const double hbm_us = bytes / 5.2e6;  // ~80 % of the copy bandwidth, bytes per microsecond
@@ -457,6 +471,29 @@ static cudaError_t launch_cluster(nk_gemm_s* p, const UmmaParams& up, int units,
     return v ? NK_CL((umma_bf16_kernel<64, 8, true, true>), units, splits, umma_smem_bytes(64, 8))
              : NK_CL((umma_bf16_kernel<64, 8, false, true>), units, splits, umma_smem_bytes(64, 8));
 #undef NK_CL
+}
+
+static int max_clusters_for(bool pair, int bn, bool vnni, int splits) {
+    static std::mutex mu;
+    static int cache[2][3][2][9];   // 0 = not asked yet, -1 = none
+    const int bi = bn == 256 ? 2 : bn == 128 ? 1 : 0;
+    if (splits < 2 || splits > 8) return 0;
+    std::lock_guard<std::mutex> lock(mu);
+    int& c = cache[pair ? 1 : 0][bi][vnni ? 1 : 0][splits];
+    if (c == 0) {
+        nk_gemm_s tmp;
+        memset(&tmp, 0, sizeof(tmp));
+        tmp.pair = pair;
+        tmp.bn = bn;
+        tmp.b_vnni_inkernel = vnni;
+        int n = 0;
+        if (launch_cluster(&tmp, UmmaParams(), 0, splits, nullptr, &n) != cudaSuccess || n <= 0) {
+            cudaGetLastError();
+            n = -1;
+        }
+        c = n;
+    }
+    return c > 0 ? c : 0;
 }
 
 template <int BN, int STAGES, bool VNNI>
