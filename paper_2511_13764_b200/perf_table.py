@@ -31,7 +31,58 @@ def peaks():
     return 1590.0, 6650.0, "fallback"
 
 
-def time_workload(w, iters, flags=0, flush=None):
+def time_launch(launch, st, iters, flush, graph_pairs):
+    """Median (and best) time in ms of `launch(cuda_stream)`, each call timed on its own after an
+    L2 flush.  With `graph_pairs` a CUDA graph of that many (flush, launch) pairs is replayed and a
+    graph of the flushes alone subtracted: CUDA-event stamps are a microsecond or two coarse on
+    some boxes, the graph difference resolves a fraction of a microsecond, and the launches come
+    without host gaps, as they would inside a captured pipeline."""
+    import torch
+    for _ in range(3):
+        launch(st.cuda_stream)
+    torch.cuda.synchronize()
+    if graph_pairs and flush is not None:
+        side = torch.cuda.Stream()
+        side.wait_stream(st)
+        mids = []
+        for with_launch in (True, False):
+            g = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(g, stream=side):
+                cs = torch.cuda.current_stream().cuda_stream
+                for _ in range(graph_pairs):
+                    flush.fill_(1)
+                    if with_launch:
+                        launch(cs)
+            ts = []
+            for _ in range(max(3, iters // 3)):
+                a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                a.record(st)
+                g.replay()
+                b.record(st)
+                b.synchronize()
+                ts.append(a.elapsed_time(b))
+            ts.sort()
+            mids.append(ts[len(ts) // 2])
+        per = (mids[0] - mids[1]) / graph_pairs
+        return per, per
+    times = []
+    for _ in range(iters):
+        if flush is not None:
+            flush.fill_(1)
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record(st)
+        launch(st.cuda_stream)
+        b.record(st)
+        b.synchronize()
+        times.append(a.elapsed_time(b))
+    times.sort()
+    return times[len(times) // 2], times[0]
+
+
+def time_workload(w, iters, flags=0, flush=None, graph_pairs=0, library=False):
+    """Returns (median ms, best ms, kernel name, launches per run, library ms or None).  `library`
+    also times torch.matmul (cuBLAS) on the same shape and element type (row-major operands, no
+    epilogue, FP32 without TF32): context for the table, never part of the product path."""
     import torch
     import paper_2511_13764_b200 as nk
     dev = torch.device("cuda", 0)
@@ -47,25 +98,18 @@ def time_workload(w, iters, flags=0, flush=None):
     ws = torch.empty(max(wsb, 16), dtype=torch.uint8, device=dev)
     st = torch.cuda.current_stream()
 
-    def run():
-        plan.run(A, B, C, bias=bias, workspace=ws if wsb else None, workspace_bytes=wsb, stream=st.cuda_stream)
+    def run(cs):
+        plan.run(A, B, C, bias=bias, workspace=ws if wsb else None, workspace_bytes=wsb, stream=cs)
 
-    for _ in range(3):
-        run()
+    med, best = time_launch(run, st, iters, flush, graph_pairs)
     plan.check()
-    times = []
-    for _ in range(iters):
-        if flush is not None:
-            flush.fill_(1)
-        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        a.record(st)
-        run()
-        b.record(st)
-        b.synchronize()
-        times.append(a.elapsed_time(b))
-    plan.check()
-    times.sort()
-    return times[len(times) // 2], times[0], plan.kernel_name, plan.launches_per_run
+    lib_ms = None
+    if library:
+        torch.backends.cuda.matmul.allow_tf32 = False
+        A2, B2 = A.view(w.M, w.K), B.view(w.K, w.N)
+        C2 = torch.empty(w.M, w.N, dtype=ein, device=dev)
+        lib_ms, _ = time_launch(lambda cs: torch.matmul(A2, B2, out=C2), st, iters, flush, graph_pairs)
+    return med, best, plan.kernel_name, plan.launches_per_run, lib_ms
 
 
 def main():
@@ -77,6 +121,9 @@ def main():
     ap.add_argument("--json", default=None)
     ap.add_argument("--no-flush", action="store_true")
     ap.add_argument("--flags", type=lambda x: int(x, 0), default=0, help="NK_FLAG_* bits given to every plan")
+    ap.add_argument("--graph", type=int, default=0,
+                    help="time N (flush, GEMM) pairs per CUDA-graph replay against N flushes (finer than event stamps)")
+    ap.add_argument("--library", action="store_true", help="add a column with torch.matmul (cuBLAS) on the same shape")
     args = ap.parse_args()
     if not torch.cuda.is_available():
         raise SystemExit("needs a CUDA device")
@@ -86,12 +133,15 @@ def main():
     flush = None if args.no_flush else torch.empty(512 << 20, dtype=torch.uint8, device="cuda")
     works = [nk_inputs.config(i) for i in (1, 2, 3, 4)] + nk_inputs.sweep() + nk_inputs.paper_mlp() + nk_inputs.f16_set()
     rows = []
-    print(f"| workload | kernel | launches | median us | TFLOP/s | alg. GB/s | bound | frac ({src}) |")
-    print("|---|---|---|---|---|---|---|---|")
+    print(f"| workload | kernel | launches | median us | TFLOP/s | alg. GB/s | bound | frac ({src}) |"
+          + (" cuBLAS us |" if args.library else ""))
+    print("|---|---|---|---|---|---|---|---|" + ("---|" if args.library else ""))
     for w in works:
         if args.only and args.only not in w.name:
             continue
-        med, best, kname, launches = time_workload(w, args.iters, flags=args.flags, flush=flush)
+        med, best, kname, launches, lib_ms = time_workload(w, args.iters, flags=args.flags, flush=flush,
+                                                           graph_pairs=args.graph if w.flops < 5e11 else 0,
+                                                           library=args.library)
         tf = w.flops / (med * 1e-3) / 1e12
         gbs = w.algorithmic_bytes / (med * 1e-3) / 1e9
         compute_peak = tensor_peak if w.in_dtype != "f32" else fma_peak
@@ -102,9 +152,10 @@ def main():
         else:
             bound, frac = ("tensor" if w.in_dtype != "f32" else "alu"), tf / compute_peak
         rows.append(dict(workload=w.name, kernel=kname, launches=launches, median_us=med * 1e3,
-                         best_us=best * 1e3, tflops=tf, gbs=gbs, bound=bound, frac=frac))
-        print(f"| {w.name} | {kname} | {launches} | {med * 1e3:.1f} | {tf:.1f} | {gbs:.0f} | {bound} | {frac:.3f} |",
-              flush=True)
+                         best_us=best * 1e3, tflops=tf, gbs=gbs, bound=bound, frac=frac,
+                         library_us=None if lib_ms is None else lib_ms * 1e3))
+        print(f"| {w.name} | {kname} | {launches} | {med * 1e3:.1f} | {tf:.1f} | {gbs:.0f} | {bound} | {frac:.3f} |"
+              + (f" {lib_ms * 1e3:.1f} |" if lib_ms is not None else ""), flush=True)
     if args.json:
         with open(args.json, "w") as f:
             json.dump(rows, f, indent=1)
