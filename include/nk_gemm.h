@@ -10,9 +10,11 @@
  *                                                     (Section 6, "MLP": bias and ReLU are
  *                                                     applied before the single store of C)
  *
- * Element types (Section 2.3): FP32 operands, or BF16 operands widened exactly to
- * FP32 with the products accumulated in FP32.  C is FP32, or BF16 (BF16 operands
- * only) rounded to nearest-even once, after the epilogue.
+ * Element types (Section 2.3): FP32 operands, or 16-bit operands (BF16; or FP16, the
+ * packed type Section 5 names next) widened exactly to FP32 with the products
+ * accumulated in FP32.  C is FP32, or has the operands' 16-bit type, rounded to
+ * nearest-even once, after the epilogue.  Wherever a rule below says BF16 it holds
+ * for FP16 as well.
  *
  * Operand layouts (Section 2.3, Figure 1 and Listing 1):
  *   NK_ROW_MAJOR   A[M][K], B[K][N]                      ("flat")
@@ -118,8 +120,10 @@ nk_status_t nk_gemm_create(const nk_gemm_desc_t* desc, nk_gemm_t* out);
 
 /*
  * Bytes of device scratch nk_gemm_run needs for this plan: 0 unless the plan
- * splits K (FP32 partial tiles, reduced in a fixed order: deterministic) or
- * unpacks a blocked operand first.  The caller allocates it; contents need not
+ * splits K through global memory (FP32 partial tiles, reduced by a second kernel
+ * in a fixed order: deterministic; 16-bit plans whose K splits are the CTAs of one
+ * thread-block cluster sum them in shared memory instead, in the same order, and
+ * need none) or unpacks a blocked operand first.  The caller allocates it; contents need not
  * be initialised and are undefined afterwards.
  */
 size_t nk_gemm_workspace_bytes(nk_gemm_t plan);

@@ -255,7 +255,7 @@ __device__ __forceinline__ void umma_store_chunk(const UmmaParams& p, const CUte
 // latency is hidden behind the K loop instead of being paid in every chunk.
 template <int BN>
 __device__ __forceinline__ const uint16_t* umma_fetch_bias(const UmmaParams& p, uint8_t* staging, int col_tile0, int lane) {
-    if (!p.epilogue || !p.out_bf16 || (p.splits > 1 && !p.cluster_reduce)) return nullptr;
+    if (!p.epilogue || !p.out_bf16 || p.splits > 1) return nullptr;   // (cluster plans park the slice in the ring)
     uint4* dst = reinterpret_cast<uint4*>(staging + 4096);
     if (lane < BN / 8) {
         const int col = col_tile0 + 8 * lane;
