@@ -77,6 +77,8 @@ typedef enum { NK_EPI_NONE = 0, NK_EPI_BIAS_RELU = 1 } nk_epilogue_t;
 #define NK_FLAG_SEPARATE_REDUCE 0x100000u /* BF16 split-K: always write FP32 partials to the workspace and sum
                                              them in a second kernel, never inside a thread-block cluster  */
 #define NK_FLAG_LSU_STORE 0x200000u /* BF16 kernels: store C with per-thread stores, never by TMA             */
+#define NK_FLAG_NO_TAIL_SPLIT 0x400000u /* BF16 pair kernel: never cut the tiles of the last, partial wave along K */
+#define NK_FLAG_TAIL_SPLIT_SHIFT 24 /* bits 24..27: force this many K splits (2..8) for the last wave's tiles */
 #define NK_FLAG_SPLITK_SHIFT 8    /* bits 8..15: force this many K splits (0 = auto)          */
 #define NK_FLAG_TILE_N_SHIFT 16   /* bits 16..19: force tile N: 1=32 2=64 3=128 4=256 (0 = auto) */
 

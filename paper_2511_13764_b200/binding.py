@@ -19,6 +19,7 @@ FLAG_SINGLE_CTA, FLAG_CTA_PAIR = 0x20, 0x40
 FLAG_SCALAR_FMA = 0x80
 FLAG_SEPARATE_REDUCE = 0x100000
 FLAG_LSU_STORE = 0x200000
+FLAG_NO_TAIL_SPLIT = 0x400000
 
 EXPORTS = ["nk_gemm_create", "nk_gemm_workspace_bytes", "nk_gemm_run", "nk_gemm_run_host",
            "nk_gemm_check", "nk_gemm_destroy", "nk_status_str", "nk_gemm_kernel_name",
@@ -30,6 +31,11 @@ STATIC_SCRATCH_BYTES = 16 << 20
 
 def flag_splitk(n: int) -> int:
     return (n & 0xFF) << 8
+
+
+def flag_tail_split(n: int) -> int:
+    """Force n K splits (2..8) for the tiles of the last, partial wave (pair kernel)."""
+    return (n & 0xF) << 24
 
 
 def flag_tile_n(code: int) -> int:

@@ -139,6 +139,69 @@ __global__ void splitk_reduce_kernel(const ReduceParams p) {
     }
 }
 
+struct TailReduceParams {
+    int M, N;
+    int tile_rows, tile_cols;   // 256 x BN
+    int tiles_m, tiles_n, group_m, first_tile;   // raster of the GEMM kernel; first_tile = id of tail tile 0
+    int splits;
+    int epilogue, bias_bf16, out_bf16, beta, c_blocked, f16;
+    const float* partial;       // [tail tile][split][tile_rows][tile_cols]
+    const void* bias;
+    void* C;
+};
+
+// Sums the K splits of the tail tiles (the last, partial wave of a large GEMM, see the pair
+// kernel) in split order and applies the epilogue: blockIdx.y = tail tile, four consecutive
+// columns per thread.
+__global__ void tail_reduce_kernel(const TailReduceParams p) {
+    const int q = blockIdx.x * blockDim.x + threadIdx.x;
+    const int per_row = p.tile_cols / 4;
+    const int r = q / per_row, c = (q - r * per_row) * 4;
+    if (r >= p.tile_rows) return;
+    // tile id -> (m block, n block), as in the GEMM kernel's raster
+    const int tile = p.first_tile + blockIdx.y;
+    const int per_group = p.group_m * p.tiles_n;
+    const int g = tile / per_group;
+    const int within = tile - g * per_group;
+    const int first_m = g * p.group_m;
+    const int gm = min(p.group_m, p.tiles_m - first_m);
+    const int mb = first_m + within % gm, nb = within / gm;
+    const int i = mb * p.tile_rows + r, j = nb * p.tile_cols + c;
+    if (i >= p.M || j >= p.N) return;
+    const size_t slab = static_cast<size_t>(p.tile_rows) * p.tile_cols;
+    const float* src = p.partial + static_cast<size_t>(blockIdx.y) * p.splits * slab + static_cast<size_t>(r) * p.tile_cols + c;
+    float4 s = __ldcs(reinterpret_cast<const float4*>(src));
+    for (int sp = 1; sp < p.splits; ++sp) {
+        const float4 v = __ldcs(reinterpret_cast<const float4*>(src + sp * slab));
+        s.x += v.x; s.y += v.y; s.z += v.z; s.w += v.w;
+    }
+    const size_t ce = p.c_blocked ? ((static_cast<size_t>(i / 32) * (p.N / 32) + j / 32) * 32 + i % 32) * 32 + j % 32
+                                  : static_cast<size_t>(i) * p.N + j;
+    if (p.beta) {
+        if (p.out_bf16) {
+            const uint2 w = *reinterpret_cast<const uint2*>(static_cast<const uint16_t*>(p.C) + ce);
+            s.x += half_bits_to_f32(w.x & 0xFFFFu, p.f16); s.y += half_bits_to_f32(w.x >> 16, p.f16);
+            s.z += half_bits_to_f32(w.y & 0xFFFFu, p.f16); s.w += half_bits_to_f32(w.y >> 16, p.f16);
+        } else {
+            const float4 cv = *reinterpret_cast<const float4*>(static_cast<const float*>(p.C) + ce);
+            s.x += cv.x; s.y += cv.y; s.z += cv.z; s.w += cv.w;
+        }
+    }
+    if (p.epilogue) {
+        const uint2 w = __ldg(reinterpret_cast<const uint2*>(static_cast<const uint16_t*>(p.bias) + j));
+        s.x = fmaxf(s.x + half_bits_to_f32(w.x & 0xFFFFu, p.f16), 0.f); s.y = fmaxf(s.y + half_bits_to_f32(w.x >> 16, p.f16), 0.f);
+        s.z = fmaxf(s.z + half_bits_to_f32(w.y & 0xFFFFu, p.f16), 0.f); s.w = fmaxf(s.w + half_bits_to_f32(w.y >> 16, p.f16), 0.f);
+    }
+    if (p.out_bf16) {
+        uint2 o;
+        o.x = pack_half2(s.x, s.y, p.f16);
+        o.y = pack_half2(s.z, s.w, p.f16);
+        *reinterpret_cast<uint2*>(static_cast<uint16_t*>(p.C) + ce) = o;
+    } else {
+        *reinterpret_cast<float4*>(static_cast<float*>(p.C) + ce) = s;
+    }
+}
+
 // VNNI-blocked B[N/32][K/32][16][32][2] -> row-major B[K][N] (BF16).  One CTA per
 // 32 x 32 block; thread (r, lane) reads word (k2 = r.., n = lane) and writes the two
 // k rows.  Reads are 128-byte rows; writes are 64-byte row segments.

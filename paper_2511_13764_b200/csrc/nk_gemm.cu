@@ -44,6 +44,7 @@ struct nk_gemm_s {
     bool b_repack;         // blocked B unpacked to row-major scratch first
     bool b_3d;             // B tensor map is the 3-D slab view
     bool cluster_reduce;   // K splits of a tile = the CTAs of one cluster; partial sums meet in shared memory
+    int tail_from, tail_splits;   // pair kernel: tiles >= tail_from (the last, partial wave) are cut into K splits; -1: off
     // SIMT
     int simt_tile;  // 128, 64 or 32
     int kt_per_split;
@@ -737,11 +738,40 @@ nk_status_t nk_gemm_create(const nk_gemm_desc_t* desc, nk_gemm_t* out) {
                 p->cluster_reduce = false;
             }
         }
+        // Tail wave: when the tiles do not fill the last wave of pairs, cutting those tiles along K lets
+        // them use all the pairs for 1/s of a wave; worth it when the K loop saved outweighs the small
+        // reduce kernel and the partials (FP32, written and read once).
+        p->tail_from = -1;
+        p->tail_splits = 0;
+        if (p->pair && p->splits == 1 && p->gemms == 1 && !(d.flags & NK_FLAG_NO_TAIL_SPLIT)) {
+            const int tiles = ceil_div(d.M, 2 * UMMA_BM) * ceil_div(d.N, p->bn);
+            const int kb_total = p->batch * ceil_div(d.K, UMMA_BK);
+            const int tail = tiles % p->max_pairs;
+            if (tiles > p->max_pairs && tail > 0 && (2 * tail <= p->max_pairs || ((d.flags >> NK_FLAG_TAIL_SPLIT_SHIFT) & 0xF) >= 2)) {
+                int sp = p->max_pairs / tail;
+                if (sp > 4) sp = 4;
+                while (sp > 1 && kb_total / sp < 8) --sp;
+                const double t_kb = p->bn == 256 ? 0.385 : 0.35;
+                const double slab_bytes = static_cast<double>(tail) * sp * 2 * UMMA_BM * p->bn * 4;
+                const double saved_us = kb_total * t_kb * (1.0 - 1.0 / sp);
+                const double cost_us = 5.5 + 2.0 * slab_bytes / 7.0e6;   // measured: ~10 us for 18 MB of partials (they stay in L2)
+                const int forced_tail = (d.flags >> NK_FLAG_TAIL_SPLIT_SHIFT) & 0xF;
+                if (forced_tail >= 2 && forced_tail <= 8 && forced_tail <= kb_total) sp = forced_tail;
+                if (sp > 1 && (saved_us > cost_us || forced_tail >= 2)) {
+                    p->tail_from = tiles - tail;
+                    p->tail_splits = sp;
+                }
+            }
+        }
         p->tma_store = d.layout_c == NK_ROW_MAJOR && d.beta == 0 && (p->splits == 1 || p->cluster_reduce) &&
                        !(d.flags & NK_FLAG_LSU_STORE);
         p->ws_repack_bytes = p->b_repack ? align_up(static_cast<size_t>(d.K) * d.N * 2, 256) : 0;
         p->ws_partial_bytes = (p->splits > 1 && !p->cluster_reduce) ? static_cast<size_t>(p->splits) * p->gemms * d.M * d.N * 4 : 0;
-        p->launches = 1 + ((p->splits > 1 && !p->cluster_reduce) ? 1 : 0) + (p->b_repack ? 1 : 0);
+        if (p->tail_from >= 0) {
+            const int tiles = ceil_div(d.M, 2 * UMMA_BM) * ceil_div(d.N, p->bn);
+            p->ws_partial_bytes = static_cast<size_t>(tiles - p->tail_from) * p->tail_splits * 2 * UMMA_BM * p->bn * 4;
+        }
+        p->launches = 1 + ((p->splits > 1 && !p->cluster_reduce) || p->tail_from >= 0 ? 1 : 0) + (p->b_repack ? 1 : 0);
         snprintf(p->name, sizeof(p->name), "umma_bf16_%s%dx64_s%d_splitk%d%s%s%s",
                  p->pair ? "pair_256x" : "128x", p->bn, p->stages,
                  p->splits, p->cluster_reduce ? "_cluster" : "", d.layout_a == NK_BLOCKED32 ? "_ablk" : "",
@@ -755,6 +785,10 @@ nk_status_t nk_gemm_create(const nk_gemm_desc_t* desc, nk_gemm_t* out) {
     if (d.layout_c == NK_BLOCKED32) {
         const size_t len = strlen(p->name);
         snprintf(p->name + len, sizeof(p->name) - len, "_cblk");
+    }
+    if (p->variant == V_UMMA && p->tail_from >= 0) {
+        const size_t len = strlen(p->name);
+        snprintf(p->name + len, sizeof(p->name) - len, "_tail%d", p->tail_splits);
     }
     if (d.in_dtype == NK_F16) {
         const size_t len = strlen(p->name);
@@ -868,7 +902,10 @@ nk_status_t nk_gemm_run(nk_gemm_t p, const void* A, const void* B, const void* b
         up.partial = partial;
         up.Bblk = p->b_vnni_inkernel ? static_cast<const uint32_t*>(B) : nullptr;
         up.status = p->status_dev;
-        const int units = up.gemms * up.tiles_m * up.tiles_n * up.splits;
+        up.tail_from = p->tail_from;
+        up.tail_splits = p->tail_splits;
+        const int units = p->tail_from >= 0 ? p->tail_from + (up.tiles_m * up.tiles_n - p->tail_from) * p->tail_splits
+                                            : up.gemms * up.tiles_m * up.tiles_n * up.splits;
         if (p->cluster_reduce) {
             e = launch_cluster(p, up, units, p->splits, st, nullptr);
         } else if (p->pair) {
@@ -881,6 +918,17 @@ nk_status_t nk_gemm_run(nk_gemm_t p, const void* A, const void* B, const void* b
         if (e != cudaSuccess) { set_err(p, "umma launch", e); return NK_ERR_CUDA; }
     }
 
+    if (p->variant == V_UMMA && p->tail_from >= 0) {
+        const int tiles_m = ceil_div(d.M, 2 * UMMA_BM), tiles_n = ceil_div(d.N, p->bn);
+        TailReduceParams tp = {static_cast<int>(d.M), static_cast<int>(d.N), 2 * UMMA_BM, p->bn, tiles_m, tiles_n, p->group_m,
+                               p->tail_from, p->tail_splits, d.epilogue, 1, is16(d.out_dtype), d.beta,
+                               d.layout_c == NK_BLOCKED32, d.in_dtype == NK_F16, partial, bias, C};
+        const int quads = 2 * UMMA_BM * p->bn / 4;
+        dim3 grid(static_cast<unsigned>((quads + 255) / 256), static_cast<unsigned>(tiles_m * tiles_n - p->tail_from));
+        tail_reduce_kernel<<<grid, 256, 0, st>>>(tp);
+        e = cudaGetLastError();
+        if (e != cudaSuccess) { set_err(p, "tail reduce launch", e); return NK_ERR_CUDA; }
+    }
     if (p->splits > 1 && !p->cluster_reduce) {
         ReduceParams rp = {static_cast<size_t>(p->gemms) * d.M * d.N, static_cast<int>(d.N), p->splits, d.epilogue,
                            is16(d.in_dtype), is16(d.out_dtype), d.beta, d.layout_c == NK_BLOCKED32,

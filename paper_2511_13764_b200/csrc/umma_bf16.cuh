@@ -62,7 +62,9 @@ struct UmmaParams {
     uint32_t idesc;     // tcgen05 instruction descriptor
     const void* bias;   // BF16 [N] or null
     void* C;            // [M][N] FP32 or BF16
-    float* partial;     // [splits][M][N] when splits > 1
+    float* partial;     // [splits][M][N] when splits > 1; [tail tile][tail split][tile rows][BN] in tail mode
+    int tail_from;      // tail mode (pair kernel): units >= tail_from are K splits of the last, partial wave's tiles; else -1
+    int tail_splits;    // K splits of each tail tile
     const uint32_t* Bblk;  // VNNI-blocked B as 32-bit words (B_VNNI kernels only)
     unsigned int* status;
 };
@@ -100,6 +102,12 @@ __device__ __forceinline__ void umma_decode_unit(const UmmaParams& p, int unit, 
     split = u - tile * p.splits;
 }
 
+// Where the FP32 partial of a chunk goes: base[(row0 + r) * ld + col0 + c], clipped to rows x cols.
+struct PartialDst {
+    float* base;
+    int ld, row0, col0, rows, cols;
+};
+
 // Epilogue for one 32 x 32 chunk of the accumulator: lane t holds row `row0 + t`, columns
 // col0 .. col0+31 as FP32 bit patterns.  Either the raw FP32 partial of a K split, or bias +
 // ReLU (Section 6, "MLP") followed by the single store of C as FP32 or BF16 (one RNE rounding).
@@ -115,7 +123,9 @@ __device__ __forceinline__ void umma_decode_unit(const UmmaParams& p, int unit, 
 __device__ __forceinline__ void umma_store_chunk(const UmmaParams& p, const CUtensorMap* tmap_c, uint32_t (&v)[32],
                                                  int row0, int lane, int col0, int split, int gemm, bool empty_k,
                                                  uint8_t* staging, int parity, const uint16_t* bias_smem,
-                                                 bool to_partial) {
+                                                 const PartialDst* pd) {
+    const bool to_partial = pd != nullptr;      // a K split's FP32 partial instead of the final C
+    const bool tma_store = p.tma_store && !to_partial;
     if (col0 >= p.N || row0 >= p.M) return;           // warp-uniform
     const int row = row0 + lane;
     const size_t c_base = static_cast<size_t>(gemm) * p.stride_c;   // this GEMM's C inside the batch
@@ -173,7 +183,7 @@ __device__ __forceinline__ void umma_store_chunk(const UmmaParams& p, const CUte
             }
         }
     }
-    if (!to_partial && p.out_bf16 && p.tma_store) {
+    if (!to_partial && p.out_bf16 && tma_store) {
         // BF16 rows (64 bytes) -> staging, 16-byte chunk g of row t at chunk g ^ ((t >> 1) & 3) (the
         // 64-byte swizzle: conflict-free stores) -> one TMA store of the 32 x 32 box
         uint8_t* tile = staging + parity * 2048;
@@ -216,7 +226,7 @@ __device__ __forceinline__ void umma_store_chunk(const UmmaParams& p, const CUte
     // whole lines and clips the ragged edge; the warp only pays eight shared-memory stores), or with
     // per-thread stores of four 128-byte row segments per instruction.
     staging += parity * 4096;
-    if (p.tma_store) {
+    if (tma_store) {
         // two tiles used alternately: the store issued two chunks ago has read this one
         if (lane == 0) bulk_wait_read<1>();
         __syncwarp();
@@ -225,7 +235,7 @@ __device__ __forceinline__ void umma_store_chunk(const UmmaParams& p, const CUte
     for (int g = 0; g < 8; ++g)
         *reinterpret_cast<uint4*>(staging + lane * 128 + ((g ^ (lane & 7)) << 4)) =
             make_uint4(v[4 * g], v[4 * g + 1], v[4 * g + 2], v[4 * g + 3]);
-    if (p.tma_store) {
+    if (tma_store) {
         fence_proxy_async_smem();
         __syncwarp();
         if (lane == 0) {
@@ -235,17 +245,26 @@ __device__ __forceinline__ void umma_store_chunk(const UmmaParams& p, const CUte
         return;
     }
     __syncwarp();
-    float* out = to_partial ? p.partial + (static_cast<size_t>(split) * p.gemms + gemm) * p.M * p.N
-                            : static_cast<float*>(p.C) + c_base;
     const int c = lane & 7, rsub = lane >> 3;
+    if (to_partial) {
+        const bool col_in = pd->col0 + 4 * c < pd->cols;
+#pragma unroll
+        for (int i = 0; i < 8; ++i) {
+            const int r = 4 * i + rsub;
+            const uint4 val = *reinterpret_cast<const uint4*>(staging + r * 128 + ((c ^ (r & 7)) << 4));
+            if (col_in && pd->row0 + r < pd->rows)
+                *reinterpret_cast<uint4*>(pd->base + static_cast<size_t>(pd->row0 + r) * pd->ld + pd->col0 + 4 * c) = val;
+        }
+        __syncwarp();
+        return;
+    }
+    float* out = static_cast<float*>(p.C) + c_base;
     const bool col_ok = col0 + 4 * c < p.N;
 #pragma unroll
     for (int i = 0; i < 8; ++i) {
         const int r = 4 * i + rsub;
         const uint4 val = *reinterpret_cast<const uint4*>(staging + r * 128 + ((c ^ (r & 7)) << 4));
-        if (col_ok && row0 + r < p.M)
-            *reinterpret_cast<uint4*>(out + (to_partial ? static_cast<size_t>(row0 + r) * p.N + col0 + 4 * c
-                                                        : c_off(r, 4 * c))) = val;
+        if (col_ok && row0 + r < p.M) *reinterpret_cast<uint4*>(out + c_off(r, 4 * c)) = val;
     }
     __syncwarp();   // the buffer is reused by the next chunk
 }
@@ -385,7 +404,7 @@ __device__ __forceinline__ bool umma_cluster_epilogue(const UmmaParams& p, const
             }
         }
         umma_store_chunk(p, tmap_c, v, row_cta0 + quarter * 32, lane, col_tile0 + static_cast<int>(c) * 32, 0, gemm,
-                         false, staging, parity, bias_smem ? bias_smem + c * 32 : nullptr, false);
+                         false, staging, parity, bias_smem ? bias_smem + c * 32 : nullptr, nullptr);
         __syncwarp();
         parity ^= 1;
     }
@@ -685,6 +704,8 @@ umma_bf16_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_consta
             tc_fence_after_sync();
             const int row0 = mb * UMMA_BM + quarter * 32;
             const bool empty_k = kb1 <= kb0;
+            PartialDst pdst = {p.partial + (static_cast<size_t>(split) * p.gemms + gemm) * p.M * p.N, p.N, row0, 0, p.M, p.N};
+            const PartialDst* pd = p.splits > 1 ? &pdst : nullptr;
             // two 32-column chunks per round: one wait for both tensor-memory loads
 #pragma unroll 1
             for (int c0 = 0; c0 < BN; c0 += 64) {
@@ -693,11 +714,13 @@ umma_bf16_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_consta
                 tmem_ld_32x32(taddr, v0);
                 tmem_ld_32x32(taddr + 32, v1);
                 tmem_ld_wait();
+                pdst.col0 = nb * BN + c0;
                 umma_store_chunk(p, &tmap_c, v0, row0, lane, nb * BN + c0, split, gemm, empty_k, staging, 0,
-                                 bias_smem ? bias_smem + c0 : nullptr, p.splits > 1);
+                                 bias_smem ? bias_smem + c0 : nullptr, pd);
                 __syncwarp();
+                pdst.col0 = nb * BN + c0 + 32;
                 umma_store_chunk(p, &tmap_c, v1, row0, lane, nb * BN + c0 + 32, split, gemm, empty_k, staging, 1,
-                                 bias_smem ? bias_smem + c0 + 32 : nullptr, p.splits > 1);
+                                 bias_smem ? bias_smem + c0 + 32 : nullptr, pd);
                 __syncwarp();
             }
             tc_fence_before_sync();

@@ -18,6 +18,11 @@
 //   - cluster-wide barriers fence the start (barriers initialised) and the end (nobody
 //     leaves while its peer may still touch its shared memory or barriers).
 //
+// Tail mode (p.tail_from >= 0): the tiles of the last, partial wave are each cut into
+// p.tail_splits K splits so that they occupy all the pairs for a fraction of a wave instead
+// of a fraction of the pairs for a whole one; their FP32 partials go to the workspace and a
+// small kernel sums them (tail_reduce_kernel).  Units 0 .. tail_from-1 are whole tiles.
+//
 // With CLUSTER_REDUCE the cluster holds S pairs, one per K split of the same 256-row tile
 // (ranks 2s and 2s + 1 are the pair of split s; a pair's leader is its even rank); the
 // accumulators of the S CTAs that own the same 128 rows are summed through distributed shared
@@ -93,7 +98,31 @@ umma_bf16_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_c
     tc_fence_after_sync();
     const uint32_t tmem_base = *tmem_slot;
 
-    const int total_units = p.gemms * p.tiles_m * p.tiles_n * p.splits;
+    const bool tail_mode = p.tail_from >= 0;
+    const int total_units = tail_mode ? p.tail_from + (p.tiles_m * p.tiles_n - p.tail_from) * p.tail_splits
+                                      : p.gemms * p.tiles_m * p.tiles_n * p.splits;
+    // unit -> tile, K split, GEMM of the batch, k-block range; tail >= 0: index of the tail tile
+    auto decode = [&](int unit, int& tile, int& split, int& gemm, int& kb0, int& kb1, int& tail) {
+        tail = -1;
+        if (tail_mode) {
+            gemm = 0;
+            if (unit < p.tail_from) {
+                tile = unit; split = 0; kb0 = 0; kb1 = p.kb_total;
+            } else {
+                const int u = unit - p.tail_from;
+                tail = u / p.tail_splits;
+                split = u - tail * p.tail_splits;
+                tile = p.tail_from + tail;
+                const int per = (p.kb_total + p.tail_splits - 1) / p.tail_splits;
+                kb0 = split * per;
+                kb1 = min(p.kb_total, kb0 + per);
+            }
+            return;
+        }
+        umma_decode_unit(p, unit, tile, split, gemm);
+        kb0 = split * p.kb_per_split;
+        kb1 = min(p.kb_total, kb0 + p.kb_per_split);
+    };
     auto give_up = [&](unsigned int code) {
         *abort_flag = 1;
         if (p.status) atomicCAS(p.status, 0u, code);
@@ -109,12 +138,10 @@ umma_bf16_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_c
         uint32_t sa = smem_base, fb = full_bar(0), lfb = lead_full0;
         bool ok = true;
         for (int unit = pair_id; ok && unit < total_units; unit += num_pairs) {
-            int tile, split, gemm;
-            umma_decode_unit(p, unit, tile, split, gemm);
+            int tile, split, gemm, kb0, kb1, tail;
+            decode(unit, tile, split, gemm, kb0, kb1, tail);
             int mb, nb;
             umma_tile_coords(p, tile, mb, nb);
-            const int kb0 = split * p.kb_per_split;
-            const int kb1 = min(p.kb_total, kb0 + p.kb_per_split);
             const int row0 = mb * BM2 + static_cast<int>(rank) * UMMA_BM;
             const int col0 = nb * BN + static_cast<int>(rank) * HALF;
             int item = kb0 / p.kb_per_item;
@@ -182,10 +209,8 @@ umma_bf16_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_c
             int local = 0;
             bool ok = true;
             for (int unit = pair_id; ok && unit < total_units; unit += num_pairs, ++local) {
-                int tile, split, gemm;
-            umma_decode_unit(p, unit, tile, split, gemm);
-                const int kb0 = split * p.kb_per_split;
-                const int kb1 = min(p.kb_total, kb0 + p.kb_per_split);
+                int tile, split, gemm, kb0, kb1, tail;
+                decode(unit, tile, split, gemm, kb0, kb1, tail);
                 const int acc = local & 1;
                 if (!mbar_wait(tempty_bar(acc), ((local >> 1) & 1u) ^ 1u, abort_flag)) {
                     if (lane == 0) give_up(0x200u + acc);
@@ -247,12 +272,10 @@ umma_bf16_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_c
         int local = 0;
         bool ok = true;
         for (int unit = pair_id; ok && unit < total_units; unit += num_pairs, ++local) {
-            int tile, split, gemm;
-            umma_decode_unit(p, unit, tile, split, gemm);
+            int tile, split, gemm, kb0, kb1, tail;
+            decode(unit, tile, split, gemm, kb0, kb1, tail);
             int mb, nb;
             umma_tile_coords(p, tile, mb, nb);
-            const int kb0 = split * p.kb_per_split;
-            const int kb1 = min(p.kb_total, kb0 + p.kb_per_split);
             const int acc = local & 1;
             uint8_t* staging = gen_base + STAGES * STAGE + (warp - 2) * 8192;
             const uint16_t* bias_smem = umma_fetch_bias<BN>(p, staging, nb * BN, lane);
@@ -264,6 +287,13 @@ umma_bf16_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_c
             tc_fence_after_sync();
             const int row0 = mb * BM2 + static_cast<int>(rank) * UMMA_BM + quarter * 32;
             const bool empty_k = kb1 <= kb0;
+            // FP32 partial of a K split: the [split][M][N] workspace, or this tail tile's own slab
+            PartialDst pdst = {p.partial + (static_cast<size_t>(split) * p.gemms + gemm) * p.M * p.N, p.N, row0, 0, p.M, p.N};
+            if (tail >= 0)
+                pdst = {p.partial + (static_cast<size_t>(tail) * p.tail_splits + split) * (BM2 * BN), BN,
+                        static_cast<int>(rank) * UMMA_BM + quarter * 32, 0, BM2, BN};
+            const PartialDst* pd = (p.splits > 1 || tail >= 0) ? &pdst : nullptr;
+            const int pcol0 = tail >= 0 ? 0 : nb * BN;
 #pragma unroll 1
             for (int c0 = 0; c0 < BN; c0 += 64) {   // two 32-column chunks per round
                 uint32_t v0[32], v1[32];
@@ -271,11 +301,13 @@ umma_bf16_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_c
                 tmem_ld_32x32(taddr, v0);
                 tmem_ld_32x32(taddr + 32, v1);
                 tmem_ld_wait();
+                pdst.col0 = pcol0 + c0;
                 umma_store_chunk(p, &tmap_c, v0, row0, lane, nb * BN + c0, split, gemm, empty_k, staging, 0,
-                                 bias_smem ? bias_smem + c0 : nullptr, p.splits > 1);
+                                 bias_smem ? bias_smem + c0 : nullptr, pd);
                 __syncwarp();
+                pdst.col0 = pcol0 + c0 + 32;
                 umma_store_chunk(p, &tmap_c, v1, row0, lane, nb * BN + c0 + 32, split, gemm, empty_k, staging, 1,
-                                 bias_smem ? bias_smem + c0 + 32 : nullptr, p.splits > 1);
+                                 bias_smem ? bias_smem + c0 + 32 : nullptr, pd);
                 __syncwarp();
             }
             tc_fence_before_sync();
@@ -294,12 +326,10 @@ umma_bf16_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_c
         uint32_t phase = 0;
         bool ok = true;
         for (int unit = pair_id; ok && unit < total_units; unit += num_pairs) {
-            int tile, split, gemm;
-            umma_decode_unit(p, unit, tile, split, gemm);
+            int tile, split, gemm, kb0, kb1, tail;
+            decode(unit, tile, split, gemm, kb0, kb1, tail);
             int mb, nb;
             umma_tile_coords(p, tile, mb, nb);
-            const int kb0 = split * p.kb_per_split;
-            const int kb1 = min(p.kb_total, kb0 + p.kb_per_split);
             for (int kb = kb0; kb < kb1; ++kb) {
                 if (!mbar_wait(empty_bar(stage), phase ^ 1u, abort_flag)) {
                     if (lane == 0) give_up(0x500u + stage);

@@ -271,3 +271,24 @@ def test_bounded_wait_reports_timeout_and_context_survives():
     A, B, bias = w.make()
     got, _ = run_plan(w, A, B, bias, plan=plan)
     check_against_oracle(w, got, A, B, bias, exact=True)
+
+
+@pytest.mark.parametrize("bn", [3, 4])
+@pytest.mark.parametrize("out_dtype,epi,splits", [("f32", "none", 2), ("bf16", "bias_relu", 3), ("f32", "bias_relu", 4)])
+def test_pair_tail_wave_split(out_dtype, epi, splits, bn):
+    """More 256-row tiles than CTA pairs, and a partial last wave: its tiles are cut along K, their FP32
+    partials summed by the tail kernel.  Exact integer data, then random data; the plan without the tail
+    split gives the same bits when the tail tiles are summed in the same order (two halves of K)."""
+    # 10 x 10 (BN = 256) or 10 x 20 (BN = 128) tiles of 256 rows over 74 pairs; ragged M and N
+    M, N, K = 2500, 2520, 640
+    f = nk.FLAG_CTA_PAIR | nk.flag_tile_n(bn) | nk.flag_splitk(1) | nk.flag_tail_split(splits)
+    w = W("tail", M, N, K, "bf16", out_dtype, epilogue=epi, integer=True)
+    err, plan = run_and_check(w, flags=f, exact=(out_dtype == "f32"))
+    assert f"_tail{splits}" in plan.kernel_name and plan.launches_per_run == 2 and plan.workspace_bytes > 0
+    w = W("tail", M, N, K, "bf16", out_dtype, epilogue=epi, seed=31)
+    A, B, bias = w.make()
+    c_tail, _ = run_plan(w, A, B, bias, flags=f)
+    check_against_oracle(w, c_tail, A, B, bias)
+    c_plain, p_plain = run_plan(w, A, B, bias, flags=f & ~nk.flag_tail_split(15) | nk.FLAG_NO_TAIL_SPLIT)
+    assert "_tail" not in p_plain.kernel_name
+    check_against_oracle(w, c_plain, A, B, bias)
