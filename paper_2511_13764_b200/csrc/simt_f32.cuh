@@ -196,7 +196,10 @@ namespace nk {
 // in shared memory once (transposed, so the MR values of one k are read with broadcast
 // 128-bit loads), then streams B with no barrier in the loop: every thread keeps 8 independent
 // 16-byte loads in flight (row segments of 512 B per warp) and holds an MR x 4 block of C in
-// registers (Algorithm 1's resident accumulator).  K chunks are combined by the split-K reduce.
+// registers (Algorithm 1's resident accumulator), as MR / 2 x 4 register pairs along M that are
+// updated with packed FMAs (fma.rn.f32x2: the pair of A values comes straight from shared
+// memory, the B value is copied into both halves), which halves the issue slots the 16 FMAs
+// per loaded element need.  K chunks are combined by the split-K reduce.
 constexpr int SKINNY_COLS = 512;
 constexpr int SKINNY_THREADS = 128;
 constexpr int SKINNY_A_FLOATS = 8192;   // MR * k-chunk <= this (32 KB of shared memory)
@@ -235,9 +238,9 @@ __global__ void __launch_bounds__(SKINNY_THREADS, MR == 16 ? 4 : 2) simt_f32_ski
     }
     __syncthreads();
 
-    float acc[MR][4];
+    float2 acc[MR / 2][4];   // acc[mp][c] = rows 2 mp, 2 mp + 1 of column n + c
 #pragma unroll
-    for (int m = 0; m < MR; ++m) acc[m][0] = acc[m][1] = acc[m][2] = acc[m][3] = 0.f;
+    for (int m = 0; m < MR / 2; ++m) acc[m][0] = acc[m][1] = acc[m][2] = acc[m][3] = make_float2(0.f, 0.f);
 
     const bool col_ok = n < p.N;
     const float* bptr = p.B + static_cast<size_t>(k0) * p.N + (col_ok ? n : 0);
@@ -259,16 +262,18 @@ __global__ void __launch_bounds__(SKINNY_THREADS, MR == 16 ? 4 : 2) simt_f32_ski
         for (int i = 0; i < 8; ++i) {
             const float* arow = &As[(kk + i) * MR];
 #pragma unroll
+            const float2 bx = make_float2(b[i].x, b[i].x), by = make_float2(b[i].y, b[i].y);
+            const float2 bz = make_float2(b[i].z, b[i].z), bw = make_float2(b[i].w, b[i].w);
+#pragma unroll
             for (int mq = 0; mq < MR; mq += 4) {
                 const float4 a = *reinterpret_cast<const float4*>(arow + mq);
-                const float av[4] = {a.x, a.y, a.z, a.w};
-#pragma unroll
-                for (int j = 0; j < 4; ++j) {
-                    acc[mq + j][0] = fmaf(av[j], b[i].x, acc[mq + j][0]);
-                    acc[mq + j][1] = fmaf(av[j], b[i].y, acc[mq + j][1]);
-                    acc[mq + j][2] = fmaf(av[j], b[i].z, acc[mq + j][2]);
-                    acc[mq + j][3] = fmaf(av[j], b[i].w, acc[mq + j][3]);
-                }
+                const float2 alo = make_float2(a.x, a.y), ahi = make_float2(a.z, a.w);
+                float2* c0 = acc[mq / 2];
+                float2* c1 = acc[mq / 2 + 1];
+                c0[0] = __ffma2_rn(alo, bx, c0[0]); c0[1] = __ffma2_rn(alo, by, c0[1]);
+                c0[2] = __ffma2_rn(alo, bz, c0[2]); c0[3] = __ffma2_rn(alo, bw, c0[3]);
+                c1[0] = __ffma2_rn(ahi, bx, c1[0]); c1[1] = __ffma2_rn(ahi, by, c1[1]);
+                c1[2] = __ffma2_rn(ahi, bz, c1[2]); c1[3] = __ffma2_rn(ahi, bw, c1[3]);
             }
         }
     }
@@ -281,7 +286,8 @@ __global__ void __launch_bounds__(SKINNY_THREADS, MR == 16 ? 4 : 2) simt_f32_ski
 #pragma unroll
     for (int m = 0; m < MR; ++m) {
         if (m >= p.M) break;
-        float4 v = make_float4(acc[m][0], acc[m][1], acc[m][2], acc[m][3]);
+        const float2* r = acc[m / 2];
+        float4 v = (m & 1) ? make_float4(r[0].y, r[1].y, r[2].y, r[3].y) : make_float4(r[0].x, r[1].x, r[2].x, r[3].x);
         if (!to_partial && p.epilogue) {
             v.x = fmaxf(v.x + bv.x, 0.f);
             v.y = fmaxf(v.y + bv.y, 0.f);
