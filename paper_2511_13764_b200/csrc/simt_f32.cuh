@@ -217,7 +217,7 @@ struct SkinnyParams {
 };
 
 template <int MR>
-__global__ void __launch_bounds__(SKINNY_THREADS, MR == 16 ? 4 : 2) simt_f32_skinny_kernel(const SkinnyParams p) {
+__global__ void __launch_bounds__(SKINNY_THREADS, MR == 16 ? 3 : 2) simt_f32_skinny_kernel(const SkinnyParams p) {
     __shared__ __align__(16) float As[SKINNY_A_FLOATS];   // As[kk][MR]
     const int t = threadIdx.x;
     const int n = blockIdx.x * SKINNY_COLS + t * 4;
