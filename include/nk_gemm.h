@@ -149,7 +149,10 @@ nk_status_t nk_gemm_run(nk_gemm_t plan, const void* A, const void* B, const void
  * copies hA, hB (and hbias) into the caller-provided device staging buffers
  * dA, dB, dbias, runs the plan, copies dC back into hC, and waits for the
  * stream.  Sizes are those implied by the plan's descriptor.  Returns after the
- * result is in hC.
+ * result is in hC.  Large single GEMMs (no batch, no beta, row-major C, M a multiple
+ * of 2048) are cut into eight chunks of rows whose copies overlap the multiplication
+ * and each other on two internal copy streams (created on the first such call and
+ * kept by the plan; pinned host buffers are needed for the overlap to happen).
  */
 nk_status_t nk_gemm_run_host(nk_gemm_t plan, const void* hA, const void* hB, const void* hbias,
                              void* hC, void* dA, void* dB, void* dbias, void* dC, void* workspace,

@@ -66,6 +66,11 @@ struct nk_gemm_s {
     char name[96];
     char cuda_err[256];
     int launches;
+    // nk_gemm_run_host on large problems: M chunks pipelined over two copy streams (made on first use)
+    nk_gemm_s* chunk_plan;
+    int chunk_rows;
+    cudaStream_t h2d_stream, d2h_stream;
+    cudaEvent_t ev_start, ev_done, ev_a[8], ev_g[8];
 };
 
 namespace nk {
@@ -952,6 +957,79 @@ nk_status_t nk_gemm_run_host(nk_gemm_t p, const void* hA, const void* hB, const 
     DeviceGuard guard(d.device);
     if (guard.err != cudaSuccess) { set_err(p, "cudaSetDevice", guard.err); return NK_ERR_DEVICE; }
     cudaError_t e;
+    // Large single GEMMs: the host link, not the GPU, bounds this call, so rows of A and C travel in
+    // eight chunks over two internal copy streams: chunk i+1 of A goes up and chunk i-1 of C comes
+    // back (PCIe is full duplex) while chunk i is multiplied on the caller's stream.
+    constexpr int kChunks = 8;
+    if (d.beta == 0 && p->batch == 1 && p->gemms == 1 && d.layout_c == NK_ROW_MAJOR && d.M % (kChunks * 256) == 0 &&
+        2.0 * d.M * d.N * d.K >= 2.0e10 && !(d.flags & NK_FLAG_KERNEL_MASK)) {
+        if (!p->chunk_plan) {
+            nk_gemm_desc_t cd = d;
+            cd.M = d.M / kChunks;
+            cd.flags = (d.flags & ~(0xFFu << NK_FLAG_SPLITK_SHIFT)) | (1u << NK_FLAG_SPLITK_SHIFT) | NK_FLAG_NO_TAIL_SPLIT;
+            nk_gemm_t cp = nullptr;
+            nk_status_t cs = nk_gemm_create(&cd, &cp);
+            if (cs == NK_OK && nk_gemm_workspace_bytes(cp) == 0) {
+                bool ok = cudaStreamCreateWithFlags(&p->h2d_stream, cudaStreamNonBlocking) == cudaSuccess &&
+                          cudaStreamCreateWithFlags(&p->d2h_stream, cudaStreamNonBlocking) == cudaSuccess &&
+                          cudaEventCreateWithFlags(&p->ev_start, cudaEventDisableTiming) == cudaSuccess &&
+                          cudaEventCreateWithFlags(&p->ev_done, cudaEventDisableTiming) == cudaSuccess;
+                for (int i = 0; ok && i < kChunks; ++i)
+                    ok = cudaEventCreateWithFlags(&p->ev_a[i], cudaEventDisableTiming) == cudaSuccess &&
+                         cudaEventCreateWithFlags(&p->ev_g[i], cudaEventDisableTiming) == cudaSuccess;
+                if (ok) {
+                    p->chunk_plan = cp;
+                    p->chunk_rows = static_cast<int>(cd.M);
+                } else {
+                    cudaGetLastError();
+                    nk_gemm_destroy(cp);
+                }
+            } else if (cp) {
+                nk_gemm_destroy(cp);
+            }
+        }
+        if (p->chunk_plan) {
+            const size_t ein_b = is16(d.in_dtype) ? 2 : 4, eout_b = is16(d.out_dtype) ? 2 : 4;
+            const size_t a_chunk = static_cast<size_t>(p->chunk_rows) * d.K * ein_b;   // also right for blocked A
+            const size_t c_chunk = static_cast<size_t>(p->chunk_rows) * d.N * eout_b;
+            const bool has_bias = d.epilogue != NK_EPI_NONE;
+            bool ok = cudaEventRecord(p->ev_start, st) == cudaSuccess &&
+                      cudaStreamWaitEvent(p->h2d_stream, p->ev_start, 0) == cudaSuccess &&
+                      cudaStreamWaitEvent(p->d2h_stream, p->ev_start, 0) == cudaSuccess &&
+                      cudaMemcpyAsync(dB, hB, static_cast<size_t>(d.K) * d.N * ein_b, cudaMemcpyHostToDevice, p->h2d_stream) == cudaSuccess &&
+                      (!has_bias || cudaMemcpyAsync(dbias, hbias, static_cast<size_t>(d.N) * ein_b, cudaMemcpyHostToDevice, p->h2d_stream) == cudaSuccess);
+            for (int i = 0; ok && i < kChunks; ++i) {
+                const char* hA_i = static_cast<const char*>(hA) + i * a_chunk;
+                char* dA_i = static_cast<char*>(dA) + i * a_chunk;
+                char* dC_i = static_cast<char*>(dC) + i * c_chunk;
+                char* hC_i = static_cast<char*>(hC) + i * c_chunk;
+                ok = cudaMemcpyAsync(dA_i, hA_i, a_chunk, cudaMemcpyHostToDevice, p->h2d_stream) == cudaSuccess &&
+                     cudaEventRecord(p->ev_a[i], p->h2d_stream) == cudaSuccess &&
+                     cudaStreamWaitEvent(st, p->ev_a[i], 0) == cudaSuccess;
+                if (!ok) break;
+                nk_status_t rs = nk_gemm_run(p->chunk_plan, dA_i, dB, has_bias ? dbias : nullptr, dC_i, nullptr, 0, cuda_stream);
+                if (rs != NK_OK) {
+                    snprintf(p->cuda_err, sizeof(p->cuda_err), "chunk %d: %s", i, nk_gemm_last_cuda_error(p->chunk_plan));
+                    cudaStreamSynchronize(p->h2d_stream);
+                    cudaStreamSynchronize(st);
+                    return rs;
+                }
+                ok = cudaEventRecord(p->ev_g[i], st) == cudaSuccess &&
+                     cudaStreamWaitEvent(p->d2h_stream, p->ev_g[i], 0) == cudaSuccess &&
+                     cudaMemcpyAsync(hC_i, dC_i, c_chunk, cudaMemcpyDeviceToHost, p->d2h_stream) == cudaSuccess;
+            }
+            ok = ok && cudaEventRecord(p->ev_done, p->d2h_stream) == cudaSuccess &&
+                 cudaStreamWaitEvent(st, p->ev_done, 0) == cudaSuccess;
+            e = cudaStreamSynchronize(st);
+            if (!ok || e != cudaSuccess) {
+                cudaStreamSynchronize(p->h2d_stream);
+                cudaStreamSynchronize(p->d2h_stream);
+                set_err(p, "pipelined host run", e != cudaSuccess ? e : cudaGetLastError());
+                return NK_ERR_CUDA;
+            }
+            return NK_OK;
+        }
+    }
     const size_t items = static_cast<size_t>(p->batch) * p->gemms;
     const size_t a_elems = (items - 1) * p->stride_a + static_cast<size_t>(d.M) * d.K;
     const size_t b_elems = (items - 1) * p->stride_b + static_cast<size_t>(d.K) * d.N;
@@ -1051,6 +1129,15 @@ nk_status_t nk_gemm_selftest_timeout(nk_gemm_t p, void* cuda_stream) {
 }
 
 nk_status_t nk_gemm_destroy(nk_gemm_t p) {
+    if (p && p->chunk_plan) {
+        DeviceGuard guard(p->d.device);
+        nk_gemm_destroy(p->chunk_plan);
+        cudaStreamDestroy(p->h2d_stream);
+        cudaStreamDestroy(p->d2h_stream);
+        cudaEventDestroy(p->ev_start);
+        cudaEventDestroy(p->ev_done);
+        for (int i = 0; i < 8; ++i) { cudaEventDestroy(p->ev_a[i]); cudaEventDestroy(p->ev_g[i]); }
+    }
     delete p;
     return NK_OK;
 }

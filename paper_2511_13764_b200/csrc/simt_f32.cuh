@@ -261,7 +261,6 @@ __global__ void __launch_bounds__(SKINNY_THREADS, MR == 16 ? 3 : 2) simt_f32_ski
 #pragma unroll
         for (int i = 0; i < 8; ++i) {
             const float* arow = &As[(kk + i) * MR];
-#pragma unroll
             const float2 bx = make_float2(b[i].x, b[i].x), by = make_float2(b[i].y, b[i].y);
             const float2 bz = make_float2(b[i].z, b[i].z), bw = make_float2(b[i].w, b[i].w);
 #pragma unroll

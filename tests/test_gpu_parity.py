@@ -292,3 +292,34 @@ def test_pair_tail_wave_split(out_dtype, epi, splits, bn):
     c_plain, p_plain = run_plan(w, A, B, bias, flags=f & ~nk.flag_tail_split(15) | nk.FLAG_NO_TAIL_SPLIT)
     assert "_tail" not in p_plain.kernel_name
     check_against_oracle(w, c_plain, A, B, bias)
+
+
+@pytest.mark.parametrize("out_dtype,epi", [("f32", "none"), ("bf16", "bias_relu")])
+def test_run_host_pipelined_chunks(out_dtype, epi):
+    """Host buffers, a problem large enough for the chunked pipeline (rows of A and C in eight chunks over
+    two copy streams): the result on 64 stratified rows (every chunk is hit) against the oracle, twice."""
+    M, N, K = 2048, 2048, 2560
+    w = W("hostpipe", M, N, K, "bf16", out_dtype, epilogue=epi, seed=41)
+    A, B, bias = w.make()
+    plan = nk.plan_for(w)
+    odt = torch.float32 if out_dtype == "f32" else torch.int16
+    hA, hB = torch.from_numpy(A).pin_memory(), torch.from_numpy(B).pin_memory()
+    hb = torch.from_numpy(bias).pin_memory() if bias is not None else None
+    hC = torch.empty(M * N, dtype=odt).pin_memory()
+    dA = torch.empty(A.size, dtype=torch.int16, device="cuda")
+    dB = torch.empty(B.size, dtype=torch.int16, device="cuda")
+    db = torch.empty(N, dtype=torch.int16, device="cuda") if bias is not None else None
+    dC = torch.empty(M * N, dtype=odt, device="cuda")
+    ws_bytes = plan.workspace_bytes
+    ws = torch.empty(max(ws_bytes, 16), dtype=torch.uint8, device="cuda")
+    rows = nk_inputs.stratified_rows(w.seed, M, 64)
+    for call in range(2):
+        hC.fill_(0)
+        plan.run_host(hA, hB, hC, dA, dB, dC, hbias=hb, dbias=db, workspace=ws, workspace_bytes=ws_bytes,
+                      stream=torch.cuda.current_stream().cuda_stream)
+        plan.check()
+        if out_dtype == "f32":
+            got = hC.numpy().astype(np.float64)
+        else:
+            got = (hC.numpy().view(np.uint16).astype(np.uint32) << 16).view(np.float32).astype(np.float64)
+        check_against_oracle(w, got.reshape(M, N), A, B, bias, rows=rows)
