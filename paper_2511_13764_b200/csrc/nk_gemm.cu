@@ -160,21 +160,24 @@ static double umma_model_us(const nk_gemm_desc_t& d, int sms, bool pair, int bn,
     // shapes.  A k-block costs 0.33-0.38 us whatever the tile (the SM's operand feed from L2, or
     // the MMA at N = 256), a little more when nearly every SM streams at once; start-up is
     // 5.4-7.3 us; the epilogue of the last tile is not hidden (0.35 us per 32 columns, 0.5 in a
-    // pair: the SM's store path); a cluster reduction costs 2.4 us (barrier, receive wait) plus
-    // 1.2 us per 32 x 32 piece a warp sends: the SM-to-SM path moves only ~13 KB per microsecond
-    // per CTA, so two splits (half of the pieces stay at home) beat four.
+    // pair: the SM's store path); a cluster reduction costs 1.2 us (barrier, receive wait) plus
+    // 1.1 us per 32 x 32 piece a warp sends: the SM-to-SM path moves only ~13 KB per microsecond
+    // per CTA, so two splits (half of the pieces stay at home) usually beat four.
     const bool busy = units > 100;
     double t_kb, start;  // microseconds per 64-wide k-block of one unit; start-up of the kernel
     if (pair) {
         t_kb = bn == 256 ? (rounds > 1 ? 0.385 : busy ? 0.34 : 0.325) : (busy ? 0.35 : 0.335);
         start = bn == 256 ? 7.3 : 6.4;
     } else {
-        t_kb = bn == 256 ? (busy ? 0.42 : 0.37) : bn == 128 ? (busy ? 0.35 : 0.335) : 0.33;
-        start = bn == 256 ? 6.0 : bn == 128 ? 5.4 : 5.8;
+        t_kb = bn == 256 ? (busy ? 0.42 : 0.37) : bn == 128 ? (busy ? 0.35 : 0.335) : 0.31;
+        start = bn == 256 ? 6.0 : bn == 128 ? 5.4 : 5.5;
     }
     if (d.layout_b == NK_BLOCKED32 && !(d.flags & NK_FLAG_REPACK_B)) {
-        // VNNI-blocked B is re-laid by four warps through the LSU: its cost grows with the columns a CTA covers
-        const double vnni = 0.14 + bn * 0.0042;
+        // VNNI-blocked B is re-laid in place by four warps: the CTA's share of B crosses shared memory
+        // four times instead of twice (TMA write, re-layout read and write, MMA read), and a k-block
+        // then costs what the shared-memory port needs for all of a stage's traffic (~250 KB/us)
+        const int cols = pair ? bn / 2 : bn;
+        const double vnni = (32.0 + cols / 2.0) / 250.0;
         if (vnni > t_kb) t_kb = vnni;
     }
     const double eo = d.out_dtype == NK_F32 ? 4.0 : 2.0;
@@ -182,7 +185,7 @@ static double umma_model_us(const nk_gemm_desc_t& d, int sms, bool pair, int bn,
     const double chunks = bn / 32.0;
     double us = start + rounds * per * t_kb;
     if (eff_splits > 1 && cluster_reduce_fits(d, sms, pair, bn, eff_splits)) {
-        us += 2.4 + 1.2 * chunks * (eff_splits - 1) / eff_splits + (pair ? 0.5 : 0.0);
+        us += 1.2 + 1.1 * chunks * (eff_splits - 1) / eff_splits + (pair ? 0.5 : 0.0);
     } else {
         us += chunks * (pair ? 0.5 : 0.35);
         // two kernels: the reduce kernel, the gap before it, and the partials written and read back
@@ -206,8 +209,6 @@ static void choose_umma(nk_gemm_s* p) {
         if (pair && (d.flags & NK_FLAG_SINGLE_CTA)) continue;
         if (!pair && (d.flags & NK_FLAG_CTA_PAIR) && forced_bn != 2) continue;
         if (pair && d.M <= UMMA_BM && !(d.flags & NK_FLAG_CTA_PAIR)) continue;
-        // measured: with the in-kernel VNNI re-layout a pair is far slower than two single CTAs
-        if (pair && d.layout_b == NK_BLOCKED32 && !(d.flags & (NK_FLAG_REPACK_B | NK_FLAG_CTA_PAIR))) continue;
         for (int bn = 64; bn <= 256; bn *= 2) {
             if (pair && bn == 64) continue;
             if (forced_bn >= 2 && forced_bn <= 4 && bn != (32 << (forced_bn - 1))) continue;
@@ -384,7 +385,23 @@ static nk_status_t encode_maps(nk_gemm_s* p, const void* A, const void* B) {
             return NK_ERR_CUDA;
         }
     } else {
-        memset(&p->tmap_b, 0, sizeof(p->tmap_b));
+        // B VNNI-blocked [N/32][K/32][16][32][2]: a k-pair row of a block is 64 elements (128 B), the
+        // 16 rows of a block and the K/32 blocks of a column block follow one another, so the
+        // operand is the 3-D tensor (64, K/2, N/32).  One box brings the 32 pair rows of a 64-deep
+        // stage for all the column blocks a CTA covers, swizzled per 128-byte row; rows beyond
+        // K/2 and column blocks beyond N/32 arrive as zeros.
+        const int cols = p->pair ? p->bn / 2 : p->bn;
+        cuuint64_t dims[3] = {64, static_cast<cuuint64_t>(d.K / 2), static_cast<cuuint64_t>(d.N / 32)};
+        cuuint64_t strides[2] = {128, static_cast<cuuint64_t>(d.K) * 64};
+        cuuint32_t box[3] = {64, UMMA_BK / 2, static_cast<cuuint32_t>(cols / 32)};
+        cuuint32_t es[3] = {1, 1, 1};
+        r = p->encode(&p->tmap_b, half_type, 3, const_cast<void*>(B), dims, strides,
+                      box, es, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+                      CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+        if (r != CUDA_SUCCESS) {
+            snprintf(p->cuda_err, sizeof(p->cuda_err), "cuTensorMapEncodeTiled(B blocked) failed: %d", (int)r);
+            return NK_ERR_CUDA;
+        }
     }
     p->cached_a = A;
     p->cached_b = B;
@@ -905,7 +922,6 @@ nk_status_t nk_gemm_run(nk_gemm_t p, const void* A, const void* B, const void* b
         up.bias = bias;
         up.C = C;
         up.partial = partial;
-        up.Bblk = p->b_vnni_inkernel ? static_cast<const uint32_t*>(B) : nullptr;
         up.status = p->status_dev;
         up.tail_from = p->tail_from;
         up.tail_splits = p->tail_splits;

@@ -61,7 +61,16 @@ __device__ __forceinline__ void fence_proxy_async_smem() {
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
 }
 
-// ---------------------------------------------------------------- cp.async (4-byte scatter copies)
+// ---------------------------------------------------------------- 16-byte shared-memory accesses by address
+__device__ __forceinline__ void ld_shared_v4(uint32_t addr, uint32_t (&v)[4]) {
+    asm volatile("ld.shared.v4.b32 {%0, %1, %2, %3}, [%4];" : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]) : "r"(addr)
+                 : "memory");
+}
+__device__ __forceinline__ void st_shared_v4(uint32_t addr, uint32_t a, uint32_t b, uint32_t c, uint32_t d) {
+    asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(addr), "r"(a), "r"(b), "r"(c), "r"(d) : "memory");
+}
+
+// ---------------------------------------------------------------- cp.async
 // Asynchronous 4-byte copy global -> shared; `src_bytes` = 0 writes zeros instead.
 __device__ __forceinline__ void cp_async_4(uint32_t dst, const void* src, uint32_t src_bytes) {
     asm volatile("cp.async.ca.shared.global [%0], [%1], 4, %2;" ::"r"(dst), "l"(src), "r"(src_bytes)
@@ -232,10 +241,14 @@ __device__ __forceinline__ void bulk_copy_to_cluster(uint32_t cluster_dst, uint3
         "r"(src), "r"(bytes), "r"(cluster_bar)
         : "memory");
 }
-// Arrive on an mbarrier given by a cluster-window address (possibly in the peer CTA).
-__device__ __forceinline__ void mbar_arrive_cluster(uint32_t cluster_bar) {
-    asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(cluster_bar)
-                 : "memory");
+// Arrive on an mbarrier given by a cluster-window address (possibly in the peer CTA), with
+// CTA-scope release.  That is enough where what the arriving thread did before is not read
+// through another CTA's memory accesses: shared-memory writes that the tensor core reads as
+// this CTA's half of an operand (made visible to it by fence.proxy.async), or tensor-memory
+// loads (ordered by the tcgen05 fences).  A cluster-scope release costs about a microsecond
+// per arrive here, which a per-stage loop cannot afford.
+__device__ __forceinline__ void mbar_arrive_cluster_cta_release(uint32_t cluster_bar) {
+    asm volatile("mbarrier.arrive.shared::cluster.b64 _, [%0];" ::"r"(cluster_bar) : "memory");
 }
 // TMA loads issued by either CTA of a pair; completion bytes go to `cluster_bar`, which may
 // live in the other CTA of the pair (no multicast: each CTA fetches its own tile).

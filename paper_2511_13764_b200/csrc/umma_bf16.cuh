@@ -13,10 +13,11 @@
 //   warp 1      MMA issuer and TMEM owner: 4 x tcgen05.mma 128 x BN x 16 per stage
 //   warps 2-5   epilogue: tcgen05.ld -> (+bias, ReLU, cvt) -> global stores; two
 //               TMEM accumulators so tile t's epilogue overlaps tile t+1's K loop
-//   warps 6-9   (VNNI-blocked B only) re-layout: copy the [k/2][n][2] blocks from
-//               global memory as 32-bit words, word-transposed (4-byte cp.async), into
-//               the K-major swizzled stage (the in-kernel counterpart of the
-//               paper's software-pipelined pack step, in the opposite direction)
+//   warps 6-9   (VNNI-blocked B only) re-layout: the producer's TMA box brings the
+//               [k/2][n][2] blocks of a stage as they are; these warps transpose them
+//               as 32-bit words, in place, into the K-major swizzled stage (the
+//               in-kernel counterpart of the paper's software-pipelined pack step,
+//               in the opposite direction)
 //
 // Every mbarrier wait is bounded; a role that gives up raises the CTA's abort
 // flag and the device status word, the other roles fall out of their loops, and
@@ -65,7 +66,6 @@ struct UmmaParams {
     float* partial;     // [splits][M][N] when splits > 1; [tail tile][tail split][tile rows][BN] in tail mode
     int tail_from;      // tail mode (pair kernel): units >= tail_from are K splits of the last, partial wave's tiles; else -1
     int tail_splits;    // K splits of each tail tile
-    const uint32_t* Bblk;  // VNNI-blocked B as 32-bit words (B_VNNI kernels only)
     unsigned int* status;
 };
 
@@ -73,9 +73,10 @@ __host__ __device__ constexpr int umma_b_stage_bytes(int BN) { return BN * UMMA_
 __host__ __device__ constexpr int umma_stage_bytes(int BN) {
     return UMMA_A_STAGE_BYTES + umma_b_stage_bytes(BN);
 }
+constexpr uint32_t UMMA_RAW_BAR_OFFSET = 200;     // in the barrier block: after full/empty/tmem barriers (<= 168 B) and the cluster barrier (192)
 constexpr int UMMA_EPI_STAGING = 4 * 2 * 4096;   // two 32 x 32 FP32 chunks per epilogue warp (1024-byte aligned: TMA store source)
 __host__ __device__ constexpr int umma_smem_bytes(int BN, int stages) {
-    return stages * umma_stage_bytes(BN) + 1024 /*alignment slack*/ + UMMA_EPI_STAGING + 256 /*barriers*/;
+    return stages * umma_stage_bytes(BN) + 1024 /*alignment slack*/ + UMMA_EPI_STAGING + 320 /*barriers*/;
 }
 // cluster split-K: one 4 KB slot per (32 x 32 piece this CTA owns, split it comes from); the pieces of
 // a CTA's 128 x BN accumulator are shared out over the splits, so a CTA's slots never exceed one
@@ -414,49 +415,48 @@ __device__ __forceinline__ bool umma_cluster_epilogue(const UmmaParams& p, const
 }
 
 // Re-layout of a VNNI-blocked B operand (Figure 1 of the paper: [k/2][n][2] inside every 32 x 32
-// block) into the K-major stage tile the tensor core reads: ROWS columns n x 64 k, 128-byte
-// rows, 16-byte chunk c of row n stored at chunk c ^ (n & 7) (the 128-byte swizzle).  Seen as
-// 32-bit words a block is 16 rows (k/2) x 32 words (n), and word (k2, n) belongs at row n, byte
-// (32 * half + 2 * k2) * 2: a word transpose.  Each lane copies one word per item with a 4-byte
-// cp.async (the scatter happens in the copy), so the copies of
-// several stages are in flight at once and no thread waits on global memory: the paper's
-// software-pipelined pack (Algorithm 3, AMX branch), in the opposite direction.
-constexpr int VNNI_LOOKAHEAD = 3;  // stages of copies in flight per warp before the oldest is awaited
-
-template <int ROWS>
-__device__ __forceinline__ void vnni_issue_stage(const UmmaParams& p, uint32_t sb, int n0, int kb,
-                                                 int tw, int lane) {
-    // Warp tw owns column octet tw of every 32-column block.  One warp instruction copies
-    // 8 columns x 4 consecutive word rows: its 32 destinations are 8 different swizzled
-    // chunks x 4 words (32 different banks) and its 4 source segments are whole 32-byte
-    // sectors.  Everything that depends only on the lane is computed once; the loops over
-    // (n-block j, k half h, word-row quad q) unroll into address adds.
-    const int kblocks32 = p.K / 32;
-    const int ln = lane & 7, lr = lane >> 3;
-    const int nn = tw * 8 + ln;                                  // column inside a block
-    const uint32_t dst_lane = sb + nn * 128 + lr * 4;
-    const uint32_t swz = static_cast<uint32_t>(nn & 7);
-    const int kblk0 = kb * 2;
-    const bool k_in0 = kblk0 < kblocks32, k_in1 = kblk0 + 1 < kblocks32;
-    const uint32_t* src_lane = p.Bblk + (static_cast<size_t>(kblk0) * 16 + lr) * 32 + nn;
-    const size_t nblk_stride = static_cast<size_t>(kblocks32) * 512;   // words per n-block
+// block) into the K-major stage tile the tensor core reads: COLS columns n x 64 k, 128-byte
+// rows, 16-byte chunk c of row n stored at chunk c ^ (n & 7) (the 128-byte swizzle).
+//
+// The producer brings the blocks of a stage with one TMA box: seen as 16-bit elements the
+// operand is a 3-D tensor (64 elements = the 32 words of one k-pair row, K/2 pair rows, N/32
+// column blocks), and a box of 64 x 32 x COLS/32 lands as COLS/32 regions of 4 KB, region j
+// holding the 32 pair rows of column block j, 128 bytes each, 16-byte chunk c of row R at
+// chunk c ^ (R & 7).  Seen as 32-bit words a region is 32 rows (k/2) x 32 words (n), and the
+// stage tile wants its word transpose: word (R, n) belongs at row n, word R.  One warp
+// transposes one region in place: a lane reads eight 4 x 4 word blocks with 16-byte loads
+// (four rows R x four columns n each), the warp synchronises, and the lane writes each
+// block's four columns as 16-byte stores (one column n, four consecutive R = eight
+// consecutive k).  The lane -> block map below makes the eight lanes of a quarter warp touch
+// eight different 16-byte bank groups in the loads and in the stores, so neither side has
+// bank conflicts.  This is the paper's software-pipelined pack (Algorithm 3, AMX branch) in the
+// opposite direction: the copies of later stages are in flight while a stage is re-laid.
+template <int COLS>
+__device__ __forceinline__ void vnni_relayout_stage(uint32_t sb, int tw, int lane) {
+    // block (q, nq): pair rows 16h + 4q .. + 3 (h = 0, 1), columns 4nq .. 4nq + 3
+    const uint32_t l0 = lane & 1, l1 = (lane >> 1) & 1, l2 = (lane >> 2) & 1, l3 = (lane >> 3) & 1, l4 = lane >> 4;
+    const uint32_t q = l2 * 2 + l1;
+    const uint32_t nq = l3 * 4 + (l2 ^ l4) * 2 + l0;
 #pragma unroll
-    for (int j = 0; j < ROWS / 32; ++j) {
-        const int nblk = n0 / 32 + j;
-        const bool n_in = nblk * 32 < p.N;
-        const uint32_t* src_j = src_lane + (n_in ? nblk * nblk_stride : 0);
-        const uint32_t dst_j = dst_lane + j * 4096;
+    for (int j = tw; j < COLS / 32; j += 4) {
+        const uint32_t rb = sb + j * 4096;
+        uint32_t w[2][4][4];
 #pragma unroll
-        for (int h = 0; h < 2; ++h) {
-            const bool in = n_in && (h ? k_in1 : k_in0);
-            const uint32_t bytes = in ? 4u : 0u;
-            const uint32_t* src_h = in ? src_j + h * 512 : p.Bblk;
+        for (int h = 0; h < 2; ++h)
 #pragma unroll
-            for (int q = 0; q < 4; ++q)
-                cp_async_4(dst_j + (((h * 4 + q) ^ swz) << 4), src_h + (in ? q * 128 : 0), bytes);
-        }
+            for (int r = 0; r < 4; ++r) {
+                const uint32_t R = 16 * h + 4 * q + r;
+                ld_shared_v4(rb + R * 128 + ((nq ^ (R & 7)) << 4), w[h][r]);
+            }
+        __syncwarp();
+#pragma unroll
+        for (int h = 0; h < 2; ++h)
+#pragma unroll
+            for (int c = 0; c < 4; ++c) {
+                const uint32_t n = 4 * nq + c;
+                st_shared_v4(rb + n * 128 + (((4 * h + q) ^ (n & 7)) << 4), w[h][0][c], w[h][1][c], w[h][2][c], w[h][3][c]);
+            }
     }
-    cp_async_commit();
 }
 
 template <int BN, int STAGES, bool B_VNNI, bool CLUSTER_REDUCE = false>
@@ -478,6 +478,7 @@ umma_bf16_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_consta
     auto empty_bar = [&](int s) { return bar_base + 8u * (STAGES + s); };
     auto tfull_bar = [&](int a) { return bar_base + 8u * (2 * STAGES + a); };
     auto tempty_bar = [&](int a) { return bar_base + 8u * (2 * STAGES + 2 + a); };
+    auto raw_bar = [&](int s) { return bar_base + UMMA_RAW_BAR_OFFSET + 8u * s; };   // VNNI B: blocks of stage s have landed
     uint8_t* gen_base = smem_raw + (smem_base - smem_u32(smem_raw));
     volatile uint32_t* tmem_slot =
         reinterpret_cast<volatile uint32_t*>(gen_base + STAGES * STAGE + UMMA_EPI_STAGING + 8 * (2 * STAGES + 4));
@@ -490,6 +491,7 @@ umma_bf16_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_consta
         for (int s = 0; s < STAGES; ++s) {
             mbar_init(full_bar(s), B_VNNI ? 1 + 4 : 1);
             mbar_init(empty_bar(s), 1);
+            if (B_VNNI) mbar_init(raw_bar(s), 1);
         }
         for (int a = 0; a < 2; ++a) {
             mbar_init(tfull_bar(a), 1);
@@ -504,7 +506,7 @@ umma_bf16_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_consta
         if (CLUSTER_REDUCE)
             mbar_arrive_expect_tx(bar_base + 192u, umma_cluster_recv_bytes<BN>(static_cast<uint32_t>(p.splits)));
         tma_prefetch_desc(&tmap_a);
-        if (!B_VNNI) tma_prefetch_desc(&tmap_b);
+        tma_prefetch_desc(&tmap_b);
         if (p.tma_store) tma_prefetch_desc(&tmap_c);
     }
     if (warp == 1) {
@@ -572,7 +574,11 @@ umma_bf16_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_consta
                     } else {
                         tma_load_3d(sa, &tmap_a, fb, kx, row0, item);
                     }
-                    if (!B_VNNI) {
+                    if (B_VNNI) {
+                        // the stage's blocks as they are; warps 6-9 re-lay them in place
+                        mbar_arrive_expect_tx(raw_bar(stage), B_STAGE);
+                        tma_load_3d(sb, &tmap_b, raw_bar(stage), 0, kbl * (UMMA_BK / 2), col0 >> 5);
+                    } else {
                         if (b3d) {
                             tma_load_4d(sb, &tmap_b, fb, 0, kx, col0 >> 6, item);
                         } else {
@@ -732,42 +738,27 @@ umma_bf16_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_consta
         __syncwarp();
     } else if (B_VNNI) {
         // ------------------------------------------------ VNNI re-layout warps (6..9)
-        static_assert(VNNI_LOOKAHEAD < STAGES, "copies in flight must fit the ring");
         const int tw = warp - 6;
-        int stage = 0, astage = 0, pending = 0;
+        int stage = 0;
         uint32_t phase = 0;
         bool ok = true;
         for (int unit = blockIdx.x; ok && unit < total_units; unit += gridDim.x) {
             int tile, split, gemm;
             umma_decode_unit(p, unit, tile, split, gemm);
-            int mb, nb;
-            umma_tile_coords(p, tile, mb, nb);
             const int kb0 = split * p.kb_per_split;
             const int kb1 = min(p.kb_total, kb0 + p.kb_per_split);
             for (int kb = kb0; kb < kb1; ++kb) {
-                if (!mbar_wait(empty_bar(stage), phase ^ 1u, abort_flag)) {
+                if (!mbar_wait(raw_bar(stage), phase, abort_flag)) {
                     if (lane == 0) give_up(0x500u + stage);
                     ok = false;
                     break;
                 }
-                vnni_issue_stage<BN>(p, smem_base + stage * STAGE + UMMA_A_STAGE_BYTES, nb * BN, kb, tw, lane);
+                vnni_relayout_stage<BN>(smem_base + stage * STAGE + UMMA_A_STAGE_BYTES, tw, lane);
+                fence_proxy_async_smem();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(full_bar(stage));
                 if (++stage == STAGES) { stage = 0; phase ^= 1u; }
-                if (++pending > VNNI_LOOKAHEAD) {
-                    cp_async_wait_group<VNNI_LOOKAHEAD>();     // the oldest stage has landed
-                    fence_proxy_async_smem();
-                    __syncwarp();
-                    if (lane == 0) mbar_arrive(full_bar(astage));
-                    if (++astage == STAGES) astage = 0;
-                    --pending;
-                }
             }
-        }
-        cp_async_wait_group<0>();
-        fence_proxy_async_smem();
-        __syncwarp();
-        for (; ok && pending > 0; --pending) {
-            if (lane == 0) mbar_arrive(full_bar(astage));
-            if (++astage == STAGES) astage = 0;
         }
     }
 

@@ -34,7 +34,7 @@ namespace nk {
 
 __host__ __device__ constexpr int pair_stage_bytes(int BN) { return UMMA_A_STAGE_BYTES + (BN / 2) * UMMA_BK * 2; }
 __host__ __device__ constexpr int pair_smem_bytes(int BN, int stages) {
-    return stages * pair_stage_bytes(BN) + 1024 + UMMA_EPI_STAGING + 256;
+    return stages * pair_stage_bytes(BN) + 1024 + UMMA_EPI_STAGING + 320;
 }
 
 // UmmaParams as for the single-CTA kernel, with tiles_m counted in 256-row tiles.
@@ -56,6 +56,7 @@ umma_bf16_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_c
     auto empty_bar = [&](int s) { return bar_base + 8u * (STAGES + s); };
     auto tfull_bar = [&](int a) { return bar_base + 8u * (2 * STAGES + a); };
     auto tempty_bar = [&](int a) { return bar_base + 8u * (2 * STAGES + 2 + a); };
+    auto raw_bar = [&](int s) { return bar_base + UMMA_RAW_BAR_OFFSET + 8u * s; };   // VNNI B: this CTA's blocks of stage s have landed
     uint8_t* gen_base = smem_raw + (smem_base - smem_u32(smem_raw));
     volatile uint32_t* tmem_slot =
         reinterpret_cast<volatile uint32_t*>(gen_base + STAGES * STAGE + UMMA_EPI_STAGING + 8 * (2 * STAGES + 4));
@@ -74,6 +75,7 @@ umma_bf16_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_c
         for (int s = 0; s < STAGES; ++s) {
             mbar_init(full_bar(s), B_VNNI ? 1 + 8 : 1);  // leader's producer (+ 4 re-layout warps per CTA)
             mbar_init(empty_bar(s), 1);
+            if (B_VNNI) mbar_init(raw_bar(s), 1);
         }
         for (int a = 0; a < 2; ++a) {
             mbar_init(tfull_bar(a), 1);
@@ -85,7 +87,7 @@ umma_bf16_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_c
         if (CLUSTER_REDUCE)
             mbar_arrive_expect_tx(bar_base + 192u, umma_cluster_recv_bytes<BN>(static_cast<uint32_t>(p.splits)));
         tma_prefetch_desc(&tmap_a);
-        if (!B_VNNI) tma_prefetch_desc(&tmap_b);
+        tma_prefetch_desc(&tmap_b);
         if (p.tma_store) tma_prefetch_desc(&tmap_c);
     }
     if (warp == 1) {
@@ -164,7 +166,11 @@ umma_bf16_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_c
                     } else {
                         tma_load_3d_pair(sa, &tmap_a, lfb, kx, row0, item);
                     }
-                    if (!B_VNNI) {
+                    if (B_VNNI) {
+                        // this CTA's column blocks as they are, on its own barrier; its warps 6-9 re-lay them in place
+                        mbar_arrive_expect_tx(raw_bar(stage), B_STAGE);
+                        tma_load_3d(sb, &tmap_b, raw_bar(stage), 0, kbl * (UMMA_BK / 2), col0 >> 5);
+                    } else {
                         if (b3d) {
                             tma_load_4d_pair(sb, &tmap_b, lfb, 0, kx, col0 >> 6, item);
                         } else {
@@ -311,50 +317,34 @@ umma_bf16_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_c
                 __syncwarp();
             }
             tc_fence_before_sync();
-            mbar_arrive_cluster(map_to_cta(tempty_bar(acc), leader));
+            mbar_arrive_cluster_cta_release(map_to_cta(tempty_bar(acc), leader));
         }
         if (lane == 0) bulk_wait_all();   // this warp's TMA stores are done with the staging buffers
         __syncwarp();
     } else if (B_VNNI) {
         // ------------------------------------------------ VNNI re-layout warps (both CTAs)
-        // Each CTA re-lays its own HALF columns (see vnni_issue_stage) and reports each landed
-        // stage to the leader's full[] barrier.
-        static_assert(VNNI_LOOKAHEAD < STAGES, "copies in flight must fit the ring");
+        // Each CTA re-lays its own HALF columns in place (see vnni_relayout_stage) and reports
+        // each finished stage to the leader's full[] barrier.
         const int tw = warp - 6;
         const uint32_t lead_full0 = map_to_cta(full_bar(0), leader);
-        int stage = 0, astage = 0, pending = 0;
+        int stage = 0;
         uint32_t phase = 0;
         bool ok = true;
         for (int unit = pair_id; ok && unit < total_units; unit += num_pairs) {
             int tile, split, gemm, kb0, kb1, tail;
             decode(unit, tile, split, gemm, kb0, kb1, tail);
-            int mb, nb;
-            umma_tile_coords(p, tile, mb, nb);
             for (int kb = kb0; kb < kb1; ++kb) {
-                if (!mbar_wait(empty_bar(stage), phase ^ 1u, abort_flag)) {
+                if (!mbar_wait(raw_bar(stage), phase, abort_flag)) {
                     if (lane == 0) give_up(0x500u + stage);
                     ok = false;
                     break;
                 }
-                vnni_issue_stage<HALF>(p, smem_base + stage * STAGE + UMMA_A_STAGE_BYTES,
-                                       nb * BN + static_cast<int>(rank) * HALF, kb, tw, lane);
+                vnni_relayout_stage<HALF>(smem_base + stage * STAGE + UMMA_A_STAGE_BYTES, tw, lane);
+                fence_proxy_async_smem();
+                __syncwarp();
+                if (lane == 0) mbar_arrive_cluster_cta_release(lead_full0 + 8u * stage);
                 if (++stage == STAGES) { stage = 0; phase ^= 1u; }
-                if (++pending > VNNI_LOOKAHEAD) {
-                    cp_async_wait_group<VNNI_LOOKAHEAD>();
-                    fence_proxy_async_smem();
-                    __syncwarp();
-                    if (lane == 0) mbar_arrive_cluster(lead_full0 + 8u * astage);
-                    if (++astage == STAGES) astage = 0;
-                    --pending;
-                }
             }
-        }
-        cp_async_wait_group<0>();
-        fence_proxy_async_smem();
-        __syncwarp();
-        for (; ok && pending > 0; --pending) {
-            if (lane == 0) mbar_arrive_cluster(lead_full0 + 8u * astage);
-            if (++astage == STAGES) astage = 0;
         }
     }
 
