@@ -78,6 +78,18 @@ typedef enum { NK_EPI_NONE = 0, NK_EPI_BIAS_RELU = 1 } nk_epilogue_t;
                                              them in a second kernel, never inside a thread-block cluster  */
 #define NK_FLAG_LSU_STORE 0x200000u /* BF16 kernels: store C with per-thread stores, never by TMA             */
 #define NK_FLAG_NO_TAIL_SPLIT 0x400000u /* BF16 pair kernel: never cut the tiles of the last, partial wave along K */
+#define NK_FLAG_F32_TENSOR 0x800000u /* FP32 operands (row-major, no batch): multiply on the tensor cores.  A and B
+                                       are each split into three BF16 planes, x = hi + mid + lo to within 2^-27
+                                       of x (a first kernel; the planes take 6 bytes per element of A and B in the
+                                       workspace), and the six cross terms that weigh more than 2^-25 of |a||b|
+                                       are multiplied by the BF16 kernels as a batch-reduce GEMM with FP32
+                                       accumulation, smallest terms first.  BF16 x BF16 products are exact in
+                                       FP32, so the result differs from the FP32 product by the dropped terms
+                                       (< 2^-24 of sum |a||b|) and the accumulation's rounding: the same error
+                                       class as the FMA kernels, not bit-identical to them.  The paper's FP32
+                                       path is FMA arithmetic (Algorithm 1); this flag is an opt-in departure
+                                       for compute-bound shapes.  Needs N and K multiples of 8.  A value beyond
+                                       the largest BF16 (3.39e38) counts as infinite.                        */
 #define NK_FLAG_TAIL_SPLIT_SHIFT 24 /* bits 24..27: force this many K splits (2..8) for the last wave's tiles */
 #define NK_FLAG_SPLITK_SHIFT 8    /* bits 8..15: force this many K splits (0 = auto)          */
 #define NK_FLAG_TILE_N_SHIFT 16   /* bits 16..19: force tile N: 1=32 2=64 3=128 4=256 (0 = auto) */

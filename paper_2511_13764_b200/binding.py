@@ -20,6 +20,7 @@ FLAG_SCALAR_FMA = 0x80
 FLAG_SEPARATE_REDUCE = 0x100000
 FLAG_LSU_STORE = 0x200000
 FLAG_NO_TAIL_SPLIT = 0x400000
+FLAG_F32_TENSOR = 0x800000
 
 EXPORTS = ["nk_gemm_create", "nk_gemm_workspace_bytes", "nk_gemm_run", "nk_gemm_run_host",
            "nk_gemm_check", "nk_gemm_destroy", "nk_status_str", "nk_gemm_kernel_name",

@@ -187,7 +187,11 @@ __global__ void tail_reduce_kernel(const TailReduceParams p) {
             s.x += cv.x; s.y += cv.y; s.z += cv.z; s.w += cv.w;
         }
     }
-    if (p.epilogue) {
+    if (p.epilogue && !p.bias_bf16) {
+        const float4 w = __ldg(reinterpret_cast<const float4*>(static_cast<const float*>(p.bias) + j));
+        s.x = fmaxf(s.x + w.x, 0.f); s.y = fmaxf(s.y + w.y, 0.f);
+        s.z = fmaxf(s.z + w.z, 0.f); s.w = fmaxf(s.w + w.w, 0.f);
+    } else if (p.epilogue) {
         const uint2 w = __ldg(reinterpret_cast<const uint2*>(static_cast<const uint16_t*>(p.bias) + j));
         s.x = fmaxf(s.x + half_bits_to_f32(w.x & 0xFFFFu, p.f16), 0.f); s.y = fmaxf(s.y + half_bits_to_f32(w.x >> 16, p.f16), 0.f);
         s.z = fmaxf(s.z + half_bits_to_f32(w.y & 0xFFFFu, p.f16), 0.f); s.w = fmaxf(s.w + half_bits_to_f32(w.y >> 16, p.f16), 0.f);
@@ -199,6 +203,35 @@ __global__ void tail_reduce_kernel(const TailReduceParams p) {
         *reinterpret_cast<uint2*>(static_cast<uint16_t*>(p.C) + ce) = o;
     } else {
         *reinterpret_cast<float4*>(static_cast<float*>(p.C) + ce) = s;
+    }
+}
+
+// FP32 -> three BF16 planes whose sum is the FP32 value (to within 2^-27 of it): hi = bf16(x),
+// mid = bf16(x - hi), lo = bf16(x - hi - mid), every rounding to nearest even, the subtractions
+// exact in FP32.  Products of BF16 values are exact in FP32, so a GEMM over cross terms of the
+// planes of A and B, accumulated in FP32, reproduces the FP32 product on the tensor cores.  A
+// value whose hi plane is not finite (inf, NaN, or beyond the largest BF16, 3.39e38) keeps that
+// plane only (inf - inf would poison the others).
+// Plane q of element i is P[q * plane + i]; four elements per thread and iteration.
+__global__ void split_f32_bf16x3_kernel(const float* __restrict__ X, uint16_t* __restrict__ P, long long count,
+                                        long long plane) {
+    const long long step = static_cast<long long>(gridDim.x) * blockDim.x * 4;
+    for (long long i = (static_cast<long long>(blockIdx.x) * blockDim.x + threadIdx.x) * 4; i < count; i += step) {
+        const float4 x4 = __ldcs(reinterpret_cast<const float4*>(X + i));
+        const float x[4] = {x4.x, x4.y, x4.z, x4.w};
+        uint32_t hi[4], mid[4], lo[4];
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+            hi[j] = pack_half2(x[j], 0.f, false) & 0xFFFFu;
+            const float r1 = x[j] - __uint_as_float(hi[j] << 16);
+            mid[j] = pack_half2(r1, 0.f, false) & 0xFFFFu;
+            const float r2 = r1 - __uint_as_float(mid[j] << 16);
+            lo[j] = pack_half2(r2, 0.f, false) & 0xFFFFu;
+            if ((hi[j] & 0x7F80u) == 0x7F80u) mid[j] = lo[j] = 0u;
+        }
+        *reinterpret_cast<uint2*>(P + i) = make_uint2(hi[0] | (hi[1] << 16), hi[2] | (hi[3] << 16));
+        *reinterpret_cast<uint2*>(P + plane + i) = make_uint2(mid[0] | (mid[1] << 16), mid[2] | (mid[3] << 16));
+        *reinterpret_cast<uint2*>(P + 2 * plane + i) = make_uint2(lo[0] | (lo[1] << 16), lo[2] | (lo[3] << 16));
     }
 }
 

@@ -23,7 +23,7 @@ namespace nk {
 // loads the library).  Kernels receive its device address as a parameter.
 __device__ unsigned int g_status_word[4];
 
-enum Variant { V_NAIVE = 0, V_SIMT = 1, V_UMMA = 2, V_SKINNY = 3 };
+enum Variant { V_NAIVE = 0, V_SIMT = 1, V_UMMA = 2, V_SKINNY = 3, V_SPLIT3 = 4 };
 
 typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*,
                                   const cuuint64_t*, const cuuint64_t*, const cuuint32_t*,
@@ -63,9 +63,16 @@ struct nk_gemm_s {
     const void *cached_a, *cached_b, *cached_c;
     bool tma_store;        // row-major C without beta or K split: stored by TMA, 32 x 32 boxes
     nk::EncodeTiledFn encode;
-    char name[96];
+    char name[128];
     char cuda_err[256];
     int launches;
+    // FP32 operands on the tensor cores: A and B are split into three BF16 planes each (workspace) and
+    // `inner`, a BF16 batch-reduce plan over six (A plane, B plane) pairs, multiplies the cross terms
+    nk_gemm_s* inner;
+    long long plane_a, plane_b;   // elements per plane
+    // set on such an inner plan: FP32 bias with 16-bit operands; batch item -> (A item, B item)
+    bool bias_f32, item_remap;
+    uint32_t item_map_a, item_map_b;
     // nk_gemm_run_host on large problems: M chunks pipelined over two copy streams (made on first use)
     nk_gemm_s* chunk_plan;
     int chunk_rows;
@@ -669,6 +676,11 @@ nk_status_t nk_gemm_create(const nk_gemm_desc_t* desc, nk_gemm_t* out) {
     }
     const uint32_t force = d.flags & NK_FLAG_KERNEL_MASK;
     if (force > NK_FLAG_KERNEL_UMMA) return NK_ERR_INVALID_ARG;
+    if ((d.flags & NK_FLAG_F32_TENSOR) && d.in_dtype == NK_F32 && force != NK_FLAG_KERNEL_NAIVE) {
+        if (force == NK_FLAG_KERNEL_SIMT) return NK_ERR_INVALID_ARG;
+        if (nbatch > 1 || d.layout_c != NK_ROW_MAJOR) return NK_ERR_UNSUPPORTED;
+        if (d.N % 8 || d.K % 8) return NK_ERR_MISALIGNED;   // the BF16 planes are read by TMA
+    }
     if (force != NK_FLAG_KERNEL_NAIVE) {
         if (is16(d.in_dtype) && (d.N % 8 || d.K % 8)) return NK_ERR_MISALIGNED;
         if (d.in_dtype == NK_F32 && (d.N % 4 || d.K % 4)) return NK_ERR_MISALIGNED;
@@ -706,6 +718,36 @@ nk_status_t nk_gemm_create(const nk_gemm_desc_t* desc, nk_gemm_t* out) {
     if (cudaGetSymbolAddress(&sym, g_status_word) != cudaSuccess) { delete p; return NK_ERR_CUDA; }
     p->status_dev = static_cast<unsigned int*>(sym);
 
+    if (d.in_dtype == NK_F32 && (d.flags & NK_FLAG_F32_TENSOR) && force != NK_FLAG_KERNEL_NAIVE) {
+        // x = hi + mid + lo in BF16 (to 2^-27 of x); A.B = sum of the nine cross terms, of which the six
+        // whose weight is above 2^-25 of |a||b| are kept, smallest first, so the FP32 accumulator of the
+        // tensor core sees them in increasing size:  (lo,hi) (hi,lo) (mid,mid) (mid,hi) (hi,mid) (hi,hi)
+        p->variant = V_SPLIT3;
+        nk_gemm_desc_t id = d;
+        id.in_dtype = NK_BF16;
+        id.out_dtype = NK_F32;
+        id.batch = 6;
+        id.batch_independent = 0;
+        id.stride_a = static_cast<int64_t>(align_up(static_cast<size_t>(d.M) * d.K, 8));
+        id.stride_b = static_cast<int64_t>(align_up(static_cast<size_t>(d.K) * d.N, 8));
+        id.flags = d.flags & ~(NK_FLAG_F32_TENSOR | NK_FLAG_KERNEL_MASK | NK_FLAG_SCALAR_FMA);
+        nk_gemm_t inner = nullptr;
+        const nk_status_t is = nk_gemm_create(&id, &inner);
+        if (is != NK_OK) { delete p; return is; }
+        inner->bias_f32 = true;
+        inner->item_remap = true;
+        inner->item_map_a = 0x001102u;   // items 0..5: planes 2 0 1 1 0 0 (0 = hi)
+        inner->item_map_b = 0x010120u;   //             planes 0 2 1 0 1 0
+        p->inner = inner;
+        p->plane_a = id.stride_a;
+        p->plane_b = id.stride_b;
+        p->ws_repack_bytes = align_up(static_cast<size_t>(p->plane_a) * 6, 256) + align_up(static_cast<size_t>(p->plane_b) * 6, 256);
+        p->ws_partial_bytes = nk_gemm_workspace_bytes(inner);
+        p->launches = 2 + inner->launches;
+        snprintf(p->name, sizeof(p->name), "f32_as_bf16x3_%.100s", inner->name);
+        *out = p;
+        return NK_OK;
+    }
     if (force == NK_FLAG_KERNEL_NAIVE) {
         p->variant = V_NAIVE;
         p->launches = 1;
@@ -863,6 +905,26 @@ nk_status_t nk_gemm_run(nk_gemm_t p, const void* A, const void* B, const void* b
         return NK_OK;
     }
 
+    if (p->variant == V_SPLIT3) {
+        uint8_t* w8 = static_cast<uint8_t*>(workspace);
+        uint16_t* pa = reinterpret_cast<uint16_t*>(w8);
+        uint16_t* pb = reinterpret_cast<uint16_t*>(w8 + align_up(static_cast<size_t>(p->plane_a) * 6, 256));
+        const long long na = static_cast<long long>(d.M) * d.K, nb = static_cast<long long>(d.K) * d.N;
+        auto blocks = [&](long long n) {
+            const long long want = (n / 4 + 255) / 256;
+            const long long cap = static_cast<long long>(p->sm_count) * 16;
+            return static_cast<unsigned>(want < cap ? (want > 0 ? want : 1) : cap);
+        };
+        split_f32_bf16x3_kernel<<<blocks(na), 256, 0, st>>>(static_cast<const float*>(A), pa, na, p->plane_a);
+        split_f32_bf16x3_kernel<<<blocks(nb), 256, 0, st>>>(static_cast<const float*>(B), pb, nb, p->plane_b);
+        e = cudaGetLastError();
+        if (e != cudaSuccess) { set_err(p, "split launch", e); return NK_ERR_CUDA; }
+        const nk_status_t rs = nk_gemm_run(p->inner, pa, pb, bias, C, p->ws_partial_bytes ? w8 + p->ws_repack_bytes : nullptr,
+                                           p->ws_partial_bytes, cuda_stream);
+        if (rs != NK_OK) memcpy(p->cuda_err, p->inner->cuda_err, sizeof(p->cuda_err));
+        return rs;
+    }
+
     uint8_t* ws = static_cast<uint8_t*>(workspace);
     float* partial = p->ws_partial_bytes ? reinterpret_cast<float*>(ws + p->ws_repack_bytes) : nullptr;
 
@@ -923,6 +985,10 @@ nk_status_t nk_gemm_run(nk_gemm_t p, const void* A, const void* B, const void* b
         up.C = C;
         up.partial = partial;
         up.status = p->status_dev;
+        up.bias_f32 = p->bias_f32 ? 1 : 0;
+        up.item_remap = p->item_remap ? 1 : 0;
+        up.item_map_a = p->item_map_a;
+        up.item_map_b = p->item_map_b;
         up.tail_from = p->tail_from;
         up.tail_splits = p->tail_splits;
         const int units = p->tail_from >= 0 ? p->tail_from + (up.tiles_m * up.tiles_n - p->tail_from) * p->tail_splits
@@ -942,7 +1008,7 @@ nk_status_t nk_gemm_run(nk_gemm_t p, const void* A, const void* B, const void* b
     if (p->variant == V_UMMA && p->tail_from >= 0) {
         const int tiles_m = ceil_div(d.M, 2 * UMMA_BM), tiles_n = ceil_div(d.N, p->bn);
         TailReduceParams tp = {static_cast<int>(d.M), static_cast<int>(d.N), 2 * UMMA_BM, p->bn, tiles_m, tiles_n, p->group_m,
-                               p->tail_from, p->tail_splits, d.epilogue, 1, is16(d.out_dtype), d.beta,
+                               p->tail_from, p->tail_splits, d.epilogue, p->bias_f32 ? 0 : 1, is16(d.out_dtype), d.beta,
                                d.layout_c == NK_BLOCKED32, d.in_dtype == NK_F16, partial, bias, C};
         const int quads = 2 * UMMA_BM * p->bn / 4;
         dim3 grid(static_cast<unsigned>((quads + 255) / 256), static_cast<unsigned>(tiles_m * tiles_n - p->tail_from));
@@ -952,7 +1018,7 @@ nk_status_t nk_gemm_run(nk_gemm_t p, const void* A, const void* B, const void* b
     }
     if (p->splits > 1 && !p->cluster_reduce) {
         ReduceParams rp = {static_cast<size_t>(p->gemms) * d.M * d.N, static_cast<int>(d.N), p->splits, d.epilogue,
-                           is16(d.in_dtype), is16(d.out_dtype), d.beta, d.layout_c == NK_BLOCKED32,
+                           is16(d.in_dtype) && !p->bias_f32, is16(d.out_dtype), d.beta, d.layout_c == NK_BLOCKED32,
                            static_cast<int>(d.M), partial, bias, C, d.in_dtype == NK_F16};
         const size_t quads = rp.MN / 4;
         splitk_reduce_kernel<<<static_cast<unsigned>((quads + 255) / 256), 256, 0, st>>>(rp);
@@ -1145,6 +1211,7 @@ nk_status_t nk_gemm_selftest_timeout(nk_gemm_t p, void* cuda_stream) {
 }
 
 nk_status_t nk_gemm_destroy(nk_gemm_t p) {
+    if (p && p->inner) nk_gemm_destroy(p->inner);
     if (p && p->chunk_plan) {
         DeviceGuard guard(p->d.device);
         nk_gemm_destroy(p->chunk_plan);

@@ -66,8 +66,21 @@ struct UmmaParams {
     float* partial;     // [splits][M][N] when splits > 1; [tail tile][tail split][tile rows][BN] in tail mode
     int tail_from;      // tail mode (pair kernel): units >= tail_from are K splits of the last, partial wave's tiles; else -1
     int tail_splits;    // K splits of each tail tile
+    int bias_f32;       // the bias vector is FP32 although the operands are 16-bit (split-FP32 plans)
+    int item_remap;     // batch item i multiplies A item (item_map_a >> 4i) & 15 by B item (item_map_b >> 4i) & 15
+    uint32_t item_map_a, item_map_b;
     unsigned int* status;
 };
+
+// The (A item, B item) pair of batch item `item`: the item itself, or, for plans that multiply
+// cross terms of split operands, the pair the plan's 4-bit tables name.
+__device__ __forceinline__ void umma_item_pair(const UmmaParams& p, int item, int& ia, int& ib) {
+    ia = ib = item;
+    if (p.item_remap) {
+        ia = static_cast<int>((p.item_map_a >> (4 * item)) & 15u);
+        ib = static_cast<int>((p.item_map_b >> (4 * item)) & 15u);
+    }
+}
 
 __host__ __device__ constexpr int umma_b_stage_bytes(int BN) { return BN * UMMA_BK * 2; }
 __host__ __device__ constexpr int umma_stage_bytes(int BN) {
@@ -168,7 +181,18 @@ __device__ __forceinline__ void umma_store_chunk(const UmmaParams& p, const CUte
             }
         }
     }
-    if (!to_partial && p.epilogue) {
+    if (!to_partial && p.epilogue && p.bias_f32) {
+        const float4* bsrc = reinterpret_cast<const float4*>(static_cast<const float*>(p.bias) + col0);
+#pragma unroll
+        for (int g = 0; g < 8; ++g) {
+            if (col0 + 4 * g >= p.N) break;
+            const float4 b = __ldg(bsrc + g);
+            v[4 * g] = __float_as_uint(fmaxf(__uint_as_float(v[4 * g]) + b.x, 0.0f));
+            v[4 * g + 1] = __float_as_uint(fmaxf(__uint_as_float(v[4 * g + 1]) + b.y, 0.0f));
+            v[4 * g + 2] = __float_as_uint(fmaxf(__uint_as_float(v[4 * g + 2]) + b.z, 0.0f));
+            v[4 * g + 3] = __float_as_uint(fmaxf(__uint_as_float(v[4 * g + 3]) + b.w, 0.0f));
+        }
+    } else if (!to_partial && p.epilogue) {
         const uint4* bsrc = reinterpret_cast<const uint4*>(static_cast<const uint16_t*>(p.bias) + col0);
 #pragma unroll
         for (int g = 0; g < 4; ++g) {
@@ -557,6 +581,8 @@ umma_bf16_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_consta
             int item = kb0 / p.kb_per_item;
             int kbl = kb0 - item * p.kb_per_item;
             item += gemm;   // independent batch: the unit's own (A, B) pair
+            int ia, ib;
+            umma_item_pair(p, item, ia, ib);
             for (int kb = kb0; kb < kb1; ++kb) {
                 const int kx = kbl * UMMA_BK;
                 if (!mbar_wait(empty_bar(stage), phase ^ 1u, abort_flag)) {
@@ -572,7 +598,7 @@ umma_bf16_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_consta
                         tma_load_4d(sa, &tmap_a, fb, 0, 0, kbl * 2, mb * 4);
                         tma_load_4d(sa + 8192, &tmap_a, fb, 0, 0, kbl * 2 + 1, mb * 4);
                     } else {
-                        tma_load_3d(sa, &tmap_a, fb, kx, row0, item);
+                        tma_load_3d(sa, &tmap_a, fb, kx, row0, ia);
                     }
                     if (B_VNNI) {
                         // the stage's blocks as they are; warps 6-9 re-lay them in place
@@ -580,15 +606,15 @@ umma_bf16_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_consta
                         tma_load_3d(sb, &tmap_b, raw_bar(stage), 0, kbl * (UMMA_BK / 2), col0 >> 5);
                     } else {
                         if (b3d) {
-                            tma_load_4d(sb, &tmap_b, fb, 0, kx, col0 >> 6, item);
+                            tma_load_4d(sb, &tmap_b, fb, 0, kx, col0 >> 6, ib);
                         } else {
 #pragma unroll
                             for (int j = 0; j < BN / 64; ++j)
-                                tma_load_3d(sb + j * 8192, &tmap_b, fb, col0 + j * 64, kx, item);
+                                tma_load_3d(sb + j * 8192, &tmap_b, fb, col0 + j * 64, kx, ib);
                         }
                     }
                 }
-                if (++kbl == p.kb_per_item) { kbl = 0; ++item; }
+                if (++kbl == p.kb_per_item) { kbl = 0; ++item; umma_item_pair(p, item, ia, ib); }
                 __syncwarp();
                 sa += STAGE;
                 fb += 8;

@@ -149,6 +149,8 @@ umma_bf16_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_c
             int item = kb0 / p.kb_per_item;
             int kbl = kb0 - item * p.kb_per_item;
             item += gemm;   // independent batch: the unit's own (A, B) pair
+            int ia, ib;
+            umma_item_pair(p, item, ia, ib);
             for (int kb = kb0; kb < kb1; ++kb) {
                 const int kx = kbl * UMMA_BK;
                 if (!mbar_wait(empty_bar(stage), phase ^ 1u, abort_flag)) {
@@ -164,7 +166,7 @@ umma_bf16_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_c
                         tma_load_4d_pair(sa, &tmap_a, lfb, 0, 0, kbl * 2, row0 / 32);
                         tma_load_4d_pair(sa + 8192, &tmap_a, lfb, 0, 0, kbl * 2 + 1, row0 / 32);
                     } else {
-                        tma_load_3d_pair(sa, &tmap_a, lfb, kx, row0, item);
+                        tma_load_3d_pair(sa, &tmap_a, lfb, kx, row0, ia);
                     }
                     if (B_VNNI) {
                         // this CTA's column blocks as they are, on its own barrier; its warps 6-9 re-lay them in place
@@ -172,15 +174,15 @@ umma_bf16_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_c
                         tma_load_3d(sb, &tmap_b, raw_bar(stage), 0, kbl * (UMMA_BK / 2), col0 >> 5);
                     } else {
                         if (b3d) {
-                            tma_load_4d_pair(sb, &tmap_b, lfb, 0, kx, col0 >> 6, item);
+                            tma_load_4d_pair(sb, &tmap_b, lfb, 0, kx, col0 >> 6, ib);
                         } else {
 #pragma unroll
                             for (int j = 0; j < HALF / 64; ++j)
-                                tma_load_3d_pair(sb + j * 8192, &tmap_b, lfb, col0 + j * 64, kx, item);
+                                tma_load_3d_pair(sb + j * 8192, &tmap_b, lfb, col0 + j * 64, kx, ib);
                         }
                     }
                 }
-                if (++kbl == p.kb_per_item) { kbl = 0; ++item; }
+                if (++kbl == p.kb_per_item) { kbl = 0; ++item; umma_item_pair(p, item, ia, ib); }
                 __syncwarp();
                 sa += STAGE;
                 fb += 8;

@@ -118,3 +118,15 @@ def test_f16_headline_shapes(i):
     w = nk_inputs.f16_set()[i]
     err, plan = check_workload(w)
     assert plan.kernel_name.endswith("_f16")
+
+
+@pytest.mark.parametrize("name", ["c5_f32_1024x1024x1024", "c5_f32_4096x4096x4096", "c5_f32_128x16384x16384"])
+def test_f32_on_tensor_cores_full_size(name):
+    """FP32 sweep shapes through the three-plane BF16 split (NK_FLAG_F32_TENSOR): sampled rows against
+    the oracle and the Freivalds identity over the whole of C.  The tensor core's FP32 accumulation
+    truncates, so the error grows with K: measured 1.0e-6 of max sum |a.b| at K = 16384 (the FMA
+    kernels: 2e-8), a fifth of the acceptance bound at worst."""
+    w = next(x for x in nk_inputs.sweep() if x.name == name)
+    err, plan = check_workload(w, flags=nk.FLAG_F32_TENSOR)
+    assert plan.kernel_name.startswith("f32_as_bf16x3_")
+    assert err < 2e-6
