@@ -8,7 +8,9 @@ operands come from HBM as they would in a real pipeline.  Per configuration the
 table gives the median time, TFLOP/s, the algorithmic HBM GB/s, and the
 fraction of the roofline that binds it: the measured BF16 tensor peak, the
 measured HBM copy bandwidth, or the FP32 FMA-pipe peak (SMs x 128 x 2 x max SM
-clock).  It only measures; parity is the tests' business.
+clock); with --f32-tensor every FP32 row is followed by the same workload
+multiplied on the tensor cores (a sixth of the BF16 tensor peak: six BF16
+products per FP32 product).  It only measures; parity is the tests' business.
 """
 from __future__ import annotations
 
@@ -124,6 +126,9 @@ def main():
     ap.add_argument("--graph", type=int, default=0,
                     help="time N (flush, GEMM) pairs per CUDA-graph replay against N flushes (finer than event stamps)")
     ap.add_argument("--library", action="store_true", help="add a column with torch.matmul (cuBLAS) on the same shape")
+    ap.add_argument("--f32-tensor", action="store_true",
+                    help="after every FP32 row, the same workload with NK_FLAG_F32_TENSOR (three BF16 planes, six "
+                         "cross terms on the tensor cores); its roofline is a sixth of the BF16 tensor peak")
     args = ap.parse_args()
     if not torch.cuda.is_available():
         raise SystemExit("needs a CUDA device")
@@ -136,26 +141,32 @@ def main():
     print(f"| workload | kernel | launches | median us | TFLOP/s | alg. GB/s | bound | frac ({src}) |"
           + (" cuBLAS us |" if args.library else ""))
     print("|---|---|---|---|---|---|---|---|" + ("---|" if args.library else ""))
+    import paper_2511_13764_b200 as nk
+    todo = []
     for w in works:
         if args.only and args.only not in w.name:
             continue
-        med, best, kname, launches, lib_ms = time_workload(w, args.iters, flags=args.flags, flush=flush,
+        todo.append((w, w.name, args.flags, False))
+        if args.f32_tensor and w.in_dtype == "f32" and w.N % 8 == 0 and w.K % 8 == 0:
+            todo.append((w, w.name + " +tensor", args.flags | nk.FLAG_F32_TENSOR, True))
+    for w, label, flags, split in todo:
+        med, best, kname, launches, lib_ms = time_workload(w, args.iters, flags=flags, flush=flush,
                                                            graph_pairs=args.graph if w.flops < 5e11 else 0,
-                                                           library=args.library)
+                                                           library=args.library and not split)
         tf = w.flops / (med * 1e-3) / 1e12
         gbs = w.algorithmic_bytes / (med * 1e-3) / 1e9
-        compute_peak = tensor_peak if w.in_dtype != "f32" else fma_peak
+        compute_peak = tensor_peak / 6 if split else tensor_peak if w.in_dtype != "f32" else fma_peak
         t_compute = w.flops / (compute_peak * 1e12)
         t_hbm = w.algorithmic_bytes / (hbm_peak * 1e9)
         if t_hbm >= t_compute:
             bound, frac = "hbm", gbs / hbm_peak
         else:
-            bound, frac = ("tensor" if w.in_dtype != "f32" else "alu"), tf / compute_peak
-        rows.append(dict(workload=w.name, kernel=kname, launches=launches, median_us=med * 1e3,
+            bound, frac = ("tensor/6" if split else "tensor" if w.in_dtype != "f32" else "alu"), tf / compute_peak
+        rows.append(dict(workload=label, kernel=kname, launches=launches, median_us=med * 1e3,
                          best_us=best * 1e3, tflops=tf, gbs=gbs, bound=bound, frac=frac,
                          library_us=None if lib_ms is None else lib_ms * 1e3))
-        print(f"| {w.name} | {kname} | {launches} | {med * 1e3:.1f} | {tf:.1f} | {gbs:.0f} | {bound} | {frac:.3f} |"
-              + (f" {lib_ms * 1e3:.1f} |" if lib_ms is not None else ""), flush=True)
+        print(f"| {label} | {kname} | {launches} | {med * 1e3:.1f} | {tf:.1f} | {gbs:.0f} | {bound} | {frac:.3f} |"
+              + (f" {lib_ms * 1e3:.1f} |" if lib_ms is not None else " |" if args.library else ""), flush=True)
     if args.json:
         with open(args.json, "w") as f:
             json.dump(rows, f, indent=1)
