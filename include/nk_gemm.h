@@ -162,9 +162,14 @@ nk_status_t nk_gemm_run(nk_gemm_t plan, const void* A, const void* B, const void
  * dA, dB, dbias, runs the plan, copies dC back into hC, and waits for the
  * stream.  Sizes are those implied by the plan's descriptor.  Returns after the
  * result is in hC.  Large single GEMMs (no batch, no beta, row-major C, M a multiple
- * of 2048) are cut into eight chunks of rows whose copies overlap the multiplication
- * and each other on two internal copy streams (created on the first such call and
- * kept by the plan; pinned host buffers are needed for the overlap to happen).
+ * of 2048) are cut into eight chunks of rows and, when N is a multiple of 1024, four
+ * panels of columns: uploads of A chunks and B panels alternate, each of the 8 x 4
+ * blocks of C is multiplied as soon as its chunk and its panel are on the device and
+ * copied back while later uploads are still running, on two internal copy streams
+ * (created on the first such call and kept by the plan; pinned host buffers are
+ * needed for the overlap to happen).  The staging buffers are scratch: afterwards dB
+ * holds B as dense column panels and dC holds C as dense blocks, not the row-major
+ * matrices.
  */
 nk_status_t nk_gemm_run_host(nk_gemm_t plan, const void* hA, const void* hB, const void* hbias,
                              void* hC, void* dA, void* dB, void* dbias, void* dC, void* workspace,

@@ -73,11 +73,12 @@ struct nk_gemm_s {
     // set on such an inner plan: FP32 bias with 16-bit operands; batch item -> (A item, B item)
     bool bias_f32, item_remap;
     uint32_t item_map_a, item_map_b;
-    // nk_gemm_run_host on large problems: M chunks pipelined over two copy streams (made on first use)
+    // nk_gemm_run_host on large problems: 8 row chunks x up to 4 column panels pipelined over two copy
+    // streams (made on first use)
     nk_gemm_s* chunk_plan;
-    int chunk_rows;
+    int chunk_rows, chunk_panels;
     cudaStream_t h2d_stream, d2h_stream;
-    cudaEvent_t ev_start, ev_done, ev_a[8], ev_g[8];
+    cudaEvent_t ev_start, ev_done, ev_up[12], ev_g[32];
 };
 
 namespace nk {
@@ -1039,15 +1040,21 @@ nk_status_t nk_gemm_run_host(nk_gemm_t p, const void* hA, const void* hB, const 
     DeviceGuard guard(d.device);
     if (guard.err != cudaSuccess) { set_err(p, "cudaSetDevice", guard.err); return NK_ERR_DEVICE; }
     cudaError_t e;
-    // Large single GEMMs: the host link, not the GPU, bounds this call, so rows of A and C travel in
-    // eight chunks over two internal copy streams: chunk i+1 of A goes up and chunk i-1 of C comes
-    // back (PCIe is full duplex) while chunk i is multiplied on the caller's stream.
-    constexpr int kChunks = 8;
-    if (d.beta == 0 && p->batch == 1 && p->gemms == 1 && d.layout_c == NK_ROW_MAJOR && d.M % (kChunks * 256) == 0 &&
+    // Large single GEMMs: the host link, not the GPU, bounds this call.  A travels in eight chunks of
+    // rows, B in four panels of columns (one when N does not divide), C comes back as the 8 x 4
+    // blocks they span: uploads alternate between the two operands, every block is multiplied on
+    // the caller's stream as soon as its row chunk and its column panel have arrived, and goes
+    // down on a second copy stream while later uploads are still running (PCIe is full duplex).
+    // On the device the panels of B and the blocks of C are dense (the staging buffers are
+    // scratch); the copies convert between that and the row-major host matrices.
+    constexpr int kRowChunks = 8, kMaxPanels = 4;
+    if (d.beta == 0 && p->batch == 1 && p->gemms == 1 && d.layout_c == NK_ROW_MAJOR && d.M % (kRowChunks * 256) == 0 &&
         2.0 * d.M * d.N * d.K >= 2.0e10 && !(d.flags & NK_FLAG_KERNEL_MASK)) {
         if (!p->chunk_plan) {
+            const int panels = d.N % (kMaxPanels * 256) == 0 ? kMaxPanels : 1;
             nk_gemm_desc_t cd = d;
-            cd.M = d.M / kChunks;
+            cd.M = d.M / kRowChunks;
+            cd.N = d.N / panels;
             cd.flags = (d.flags & ~(0xFFu << NK_FLAG_SPLITK_SHIFT)) | (1u << NK_FLAG_SPLITK_SHIFT) | NK_FLAG_NO_TAIL_SPLIT;
             nk_gemm_t cp = nullptr;
             nk_status_t cs = nk_gemm_create(&cd, &cp);
@@ -1056,12 +1063,14 @@ nk_status_t nk_gemm_run_host(nk_gemm_t p, const void* hA, const void* hB, const 
                           cudaStreamCreateWithFlags(&p->d2h_stream, cudaStreamNonBlocking) == cudaSuccess &&
                           cudaEventCreateWithFlags(&p->ev_start, cudaEventDisableTiming) == cudaSuccess &&
                           cudaEventCreateWithFlags(&p->ev_done, cudaEventDisableTiming) == cudaSuccess;
-                for (int i = 0; ok && i < kChunks; ++i)
-                    ok = cudaEventCreateWithFlags(&p->ev_a[i], cudaEventDisableTiming) == cudaSuccess &&
-                         cudaEventCreateWithFlags(&p->ev_g[i], cudaEventDisableTiming) == cudaSuccess;
+                for (int i = 0; ok && i < kRowChunks + kMaxPanels; ++i)
+                    ok = cudaEventCreateWithFlags(&p->ev_up[i], cudaEventDisableTiming) == cudaSuccess;
+                for (int i = 0; ok && i < kRowChunks * kMaxPanels; ++i)
+                    ok = cudaEventCreateWithFlags(&p->ev_g[i], cudaEventDisableTiming) == cudaSuccess;
                 if (ok) {
                     p->chunk_plan = cp;
                     p->chunk_rows = static_cast<int>(cd.M);
+                    p->chunk_panels = panels;
                 } else {
                     cudaGetLastError();
                     nk_gemm_destroy(cp);
@@ -1072,33 +1081,61 @@ nk_status_t nk_gemm_run_host(nk_gemm_t p, const void* hA, const void* hB, const 
         }
         if (p->chunk_plan) {
             const size_t ein_b = is16(d.in_dtype) ? 2 : 4, eout_b = is16(d.out_dtype) ? 2 : 4;
-            const size_t a_chunk = static_cast<size_t>(p->chunk_rows) * d.K * ein_b;   // also right for blocked A
-            const size_t c_chunk = static_cast<size_t>(p->chunk_rows) * d.N * eout_b;
+            const int panels = p->chunk_panels;
+            const size_t rows = static_cast<size_t>(p->chunk_rows), cols = static_cast<size_t>(d.N) / panels;
+            const size_t a_chunk = rows * d.K * ein_b;                         // also right for blocked A
+            const size_t b_panel = static_cast<size_t>(d.K) * cols * ein_b;     // dense on the device
+            const size_t c_block = rows * cols * eout_b;                       // dense on the device
             const bool has_bias = d.epilogue != NK_EPI_NONE;
+            const bool b_rows_strided = d.layout_b == NK_ROW_MAJOR && panels > 1;   // a blocked B panel is contiguous
             bool ok = cudaEventRecord(p->ev_start, st) == cudaSuccess &&
                       cudaStreamWaitEvent(p->h2d_stream, p->ev_start, 0) == cudaSuccess &&
                       cudaStreamWaitEvent(p->d2h_stream, p->ev_start, 0) == cudaSuccess &&
-                      cudaMemcpyAsync(dB, hB, static_cast<size_t>(d.K) * d.N * ein_b, cudaMemcpyHostToDevice, p->h2d_stream) == cudaSuccess &&
                       (!has_bias || cudaMemcpyAsync(dbias, hbias, static_cast<size_t>(d.N) * ein_b, cudaMemcpyHostToDevice, p->h2d_stream) == cudaSuccess);
-            for (int i = 0; ok && i < kChunks; ++i) {
-                const char* hA_i = static_cast<const char*>(hA) + i * a_chunk;
-                char* dA_i = static_cast<char*>(dA) + i * a_chunk;
-                char* dC_i = static_cast<char*>(dC) + i * c_chunk;
-                char* hC_i = static_cast<char*>(hC) + i * c_chunk;
-                ok = cudaMemcpyAsync(dA_i, hA_i, a_chunk, cudaMemcpyHostToDevice, p->h2d_stream) == cudaSuccess &&
-                     cudaEventRecord(p->ev_a[i], p->h2d_stream) == cudaSuccess &&
-                     cudaStreamWaitEvent(st, p->ev_a[i], 0) == cudaSuccess;
-                if (!ok) break;
-                nk_status_t rs = nk_gemm_run(p->chunk_plan, dA_i, dB, has_bias ? dbias : nullptr, dC_i, nullptr, 0, cuda_stream);
-                if (rs != NK_OK) {
-                    snprintf(p->cuda_err, sizeof(p->cuda_err), "chunk %d: %s", i, nk_gemm_last_cuda_error(p->chunk_plan));
-                    cudaStreamSynchronize(p->h2d_stream);
-                    cudaStreamSynchronize(st);
-                    return rs;
+            int na = 0, nb = 0, nup = 0, ng = 0;     // row chunks and panels on the device; uploads and blocks so far
+            while (ok && (na < kRowChunks || nb < panels)) {
+                // A0, B0, then B and A in turn until one runs out
+                const bool up_a = nb >= panels || (na < kRowChunks && na < nb + (na == 0 ? 1 : 0));
+                if (up_a) {
+                    ok = cudaMemcpyAsync(static_cast<char*>(dA) + na * a_chunk, static_cast<const char*>(hA) + na * a_chunk, a_chunk,
+                                         cudaMemcpyHostToDevice, p->h2d_stream) == cudaSuccess;
+                } else if (b_rows_strided) {
+                    ok = cudaMemcpy2DAsync(static_cast<char*>(dB) + nb * b_panel, cols * ein_b,
+                                           static_cast<const char*>(hB) + nb * cols * ein_b, static_cast<size_t>(d.N) * ein_b,
+                                           cols * ein_b, static_cast<size_t>(d.K), cudaMemcpyHostToDevice, p->h2d_stream) == cudaSuccess;
+                } else {
+                    ok = cudaMemcpyAsync(static_cast<char*>(dB) + nb * b_panel, static_cast<const char*>(hB) + nb * b_panel, b_panel,
+                                         cudaMemcpyHostToDevice, p->h2d_stream) == cudaSuccess;
                 }
-                ok = cudaEventRecord(p->ev_g[i], st) == cudaSuccess &&
-                     cudaStreamWaitEvent(p->d2h_stream, p->ev_g[i], 0) == cudaSuccess &&
-                     cudaMemcpyAsync(hC_i, dC_i, c_chunk, cudaMemcpyDeviceToHost, p->d2h_stream) == cudaSuccess;
+                ok = ok && cudaEventRecord(p->ev_up[nup], p->h2d_stream) == cudaSuccess &&
+                     cudaStreamWaitEvent(st, p->ev_up[nup], 0) == cudaSuccess;
+                ++nup;
+                if (!ok) break;
+                // the blocks this upload completes: a new row chunk meets every panel present, and vice versa
+                const int i0 = up_a ? na : 0, i1 = up_a ? na + 1 : na;
+                const int j0 = up_a ? 0 : nb, j1 = up_a ? nb : nb + 1;
+                if (up_a) ++na; else ++nb;
+                for (int i = i0; ok && i < i1; ++i)
+                    for (int j = j0; ok && j < j1; ++j) {
+                        char* dC_ij = static_cast<char*>(dC) + (static_cast<size_t>(i) * panels + j) * c_block;
+                        nk_status_t rs = nk_gemm_run(p->chunk_plan, static_cast<char*>(dA) + i * a_chunk,
+                                                     static_cast<char*>(dB) + j * b_panel,
+                                                     has_bias ? static_cast<char*>(dbias) + j * cols * ein_b : nullptr, dC_ij,
+                                                     nullptr, 0, cuda_stream);
+                        if (rs != NK_OK) {
+                            snprintf(p->cuda_err, sizeof(p->cuda_err), "block %d,%d: %s", i, j, nk_gemm_last_cuda_error(p->chunk_plan));
+                            cudaStreamSynchronize(p->h2d_stream);
+                            cudaStreamSynchronize(p->d2h_stream);
+                            cudaStreamSynchronize(st);
+                            return rs;
+                        }
+                        char* hC_ij = static_cast<char*>(hC) + (static_cast<size_t>(i) * rows * d.N + j * cols) * eout_b;
+                        ok = cudaEventRecord(p->ev_g[ng], st) == cudaSuccess &&
+                             cudaStreamWaitEvent(p->d2h_stream, p->ev_g[ng], 0) == cudaSuccess &&
+                             cudaMemcpy2DAsync(hC_ij, static_cast<size_t>(d.N) * eout_b, dC_ij, cols * eout_b, cols * eout_b, rows,
+                                               cudaMemcpyDeviceToHost, p->d2h_stream) == cudaSuccess;
+                        ++ng;
+                    }
             }
             ok = ok && cudaEventRecord(p->ev_done, p->d2h_stream) == cudaSuccess &&
                  cudaStreamWaitEvent(st, p->ev_done, 0) == cudaSuccess;
@@ -1219,7 +1256,8 @@ nk_status_t nk_gemm_destroy(nk_gemm_t p) {
         cudaStreamDestroy(p->d2h_stream);
         cudaEventDestroy(p->ev_start);
         cudaEventDestroy(p->ev_done);
-        for (int i = 0; i < 8; ++i) { cudaEventDestroy(p->ev_a[i]); cudaEventDestroy(p->ev_g[i]); }
+        for (int i = 0; i < 12; ++i) cudaEventDestroy(p->ev_up[i]);
+        for (int i = 0; i < 32; ++i) cudaEventDestroy(p->ev_g[i]);
     }
     delete p;
     return NK_OK;

@@ -294,12 +294,14 @@ def test_pair_tail_wave_split(out_dtype, epi, splits, bn):
     check_against_oracle(w, c_plain, A, B, bias)
 
 
-@pytest.mark.parametrize("out_dtype,epi", [("f32", "none"), ("bf16", "bias_relu")])
-def test_run_host_pipelined_chunks(out_dtype, epi):
-    """Host buffers, a problem large enough for the chunked pipeline (rows of A and C in eight chunks over
-    two copy streams): the result on 64 stratified rows (every chunk is hit) against the oracle, twice."""
-    M, N, K = 2048, 2048, 2560
-    w = W("hostpipe", M, N, K, "bf16", out_dtype, epilogue=epi, seed=41)
+@pytest.mark.parametrize("out_dtype,epi,layout,N", [("f32", "none", "row", 2048), ("bf16", "bias_relu", "row", 2048),
+                                                    ("bf16", "bias_relu", "blocked32", 2048), ("f32", "none", "row", 2304)])
+def test_run_host_pipelined_chunks(out_dtype, epi, layout, N):
+    """Host buffers, a problem large enough for the chunked pipeline (eight row chunks of A, four column
+    panels of B when N divides, one otherwise, C back block by block over two copy streams): the result on
+    64 stratified rows (every row chunk is hit, all columns) against the oracle, twice."""
+    M, K = 2048, 2560
+    w = W("hostpipe", M, N, K, "bf16", out_dtype, layout=layout, epilogue=epi, seed=41)
     A, B, bias = w.make()
     plan = nk.plan_for(w)
     odt = torch.float32 if out_dtype == "f32" else torch.int16
