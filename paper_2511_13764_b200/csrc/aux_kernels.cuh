@@ -212,12 +212,22 @@ __global__ void tail_reduce_kernel(const TailReduceParams p) {
 // planes of A and B, accumulated in FP32, reproduces the FP32 product on the tensor cores.  A
 // value whose hi plane is not finite (inf, NaN, or beyond the largest BF16, 3.39e38) keeps that
 // plane only (inf - inf would poison the others).
-// Plane q of element i is P[q * plane + i]; four elements per thread and iteration.
-__global__ void split_f32_bf16x3_kernel(const float* __restrict__ X, uint16_t* __restrict__ P, long long count,
-                                        long long plane) {
-    const long long step = static_cast<long long>(gridDim.x) * blockDim.x * 4;
-    for (long long i = (static_cast<long long>(blockIdx.x) * blockDim.x + threadIdx.x) * 4; i < count; i += step) {
-        const float4 x4 = __ldcs(reinterpret_cast<const float4*>(X + i));
+// Plane q of element i is P[q * plane + i]; four elements per thread and iteration.  One launch
+// splits both operands: the first `blocks_a` CTAs take A, the others B.
+struct SplitOperand {
+    const float* X;
+    uint16_t* P;
+    long long count, plane;
+};
+
+__global__ void split_f32_bf16x3_kernel(const SplitOperand a, const SplitOperand b, unsigned blocks_a) {
+    const bool is_a = blockIdx.x < blocks_a;
+    const SplitOperand& o = is_a ? a : b;
+    const long long block = is_a ? blockIdx.x : blockIdx.x - blocks_a;
+    const long long nblocks = is_a ? blocks_a : gridDim.x - blocks_a;
+    const long long step = nblocks * blockDim.x * 4;
+    for (long long i = (block * blockDim.x + threadIdx.x) * 4; i < o.count; i += step) {
+        const float4 x4 = __ldcs(reinterpret_cast<const float4*>(o.X + i));
         const float x[4] = {x4.x, x4.y, x4.z, x4.w};
         uint32_t hi[4], mid[4], lo[4];
 #pragma unroll
@@ -229,9 +239,9 @@ __global__ void split_f32_bf16x3_kernel(const float* __restrict__ X, uint16_t* _
             lo[j] = pack_half2(r2, 0.f, false) & 0xFFFFu;
             if ((hi[j] & 0x7F80u) == 0x7F80u) mid[j] = lo[j] = 0u;
         }
-        *reinterpret_cast<uint2*>(P + i) = make_uint2(hi[0] | (hi[1] << 16), hi[2] | (hi[3] << 16));
-        *reinterpret_cast<uint2*>(P + plane + i) = make_uint2(mid[0] | (mid[1] << 16), mid[2] | (mid[3] << 16));
-        *reinterpret_cast<uint2*>(P + 2 * plane + i) = make_uint2(lo[0] | (lo[1] << 16), lo[2] | (lo[3] << 16));
+        *reinterpret_cast<uint2*>(o.P + i) = make_uint2(hi[0] | (hi[1] << 16), hi[2] | (hi[3] << 16));
+        *reinterpret_cast<uint2*>(o.P + o.plane + i) = make_uint2(mid[0] | (mid[1] << 16), mid[2] | (mid[3] << 16));
+        *reinterpret_cast<uint2*>(o.P + 2 * o.plane + i) = make_uint2(lo[0] | (lo[1] << 16), lo[2] | (lo[3] << 16));
     }
 }
 

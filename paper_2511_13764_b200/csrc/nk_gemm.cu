@@ -744,7 +744,7 @@ nk_status_t nk_gemm_create(const nk_gemm_desc_t* desc, nk_gemm_t* out) {
         p->plane_b = id.stride_b;
         p->ws_repack_bytes = align_up(static_cast<size_t>(p->plane_a) * 6, 256) + align_up(static_cast<size_t>(p->plane_b) * 6, 256);
         p->ws_partial_bytes = nk_gemm_workspace_bytes(inner);
-        p->launches = 2 + inner->launches;
+        p->launches = 1 + inner->launches;
         snprintf(p->name, sizeof(p->name), "f32_as_bf16x3_%.100s", inner->name);
         *out = p;
         return NK_OK;
@@ -916,8 +916,9 @@ nk_status_t nk_gemm_run(nk_gemm_t p, const void* A, const void* B, const void* b
             const long long cap = static_cast<long long>(p->sm_count) * 16;
             return static_cast<unsigned>(want < cap ? (want > 0 ? want : 1) : cap);
         };
-        split_f32_bf16x3_kernel<<<blocks(na), 256, 0, st>>>(static_cast<const float*>(A), pa, na, p->plane_a);
-        split_f32_bf16x3_kernel<<<blocks(nb), 256, 0, st>>>(static_cast<const float*>(B), pb, nb, p->plane_b);
+        const SplitOperand sa = {static_cast<const float*>(A), pa, na, p->plane_a};
+        const SplitOperand sb = {static_cast<const float*>(B), pb, nb, p->plane_b};
+        split_f32_bf16x3_kernel<<<blocks(na) + blocks(nb), 256, 0, st>>>(sa, sb, blocks(na));
         e = cudaGetLastError();
         if (e != cudaSuccess) { set_err(p, "split launch", e); return NK_ERR_CUDA; }
         const nk_status_t rs = nk_gemm_run(p->inner, pa, pb, bias, C, p->ws_partial_bytes ? w8 + p->ws_repack_bytes : nullptr,
