@@ -90,8 +90,17 @@ def fill(seed: int, tensor_id: int, count: int, dist: str = "uniform",
 
     dist: "uniform" (U[-1,1) on the 2**-23 grid), "normal" (N(0, sigma**2)),
           "int" (integers in [-4, 4], exact in every precision used here).
-    dtype: "f32" -> float32 array; "bf16" / "f16" -> uint16 bit patterns.
+    dtype: "f32" -> float32 array; "bf16" / "f16" -> uint16 bit patterns; "s8" -> int8, uniform over
+           all 256 values.
     """
+    if dtype == "s8":
+        # INT8 operands: the full range [-128, 127], uniformly, whatever `dist` says
+        out = np.empty(count, dtype=np.int8)
+        for s in range(0, count, _CHUNK):
+            n = min(_CHUNK, count - s)
+            out[s:s + n] = ((raw_bits(seed, tensor_id, start + s, n) >> np.uint64(40)) & np.uint64(0xFF)
+                            ).astype(np.uint8).view(np.int8)
+        return out
     out = np.empty(count, dtype=np.float32 if dtype == "f32" else np.uint16)
     for s in range(0, count, _CHUNK):
         n = min(_CHUNK, count - s)
@@ -135,9 +144,9 @@ class Workload:
     M: int
     N: int
     K: int
-    in_dtype: str = "bf16"          # "f32" | "bf16" | "f16"
-    out_dtype: str = "f32"          # "f32" | "bf16" | "f16" (a 16-bit output has the input's type)
-    layout: str = "row"             # "row" | "blocked32" (A and B both)
+    in_dtype: str = "bf16"          # "f32" | "bf16" | "f16" | "s8"
+    out_dtype: str = "f32"          # "f32" | "bf16" | "f16" (a 16-bit output has the input's type) | "s32" (INT8 operands)
+    layout: str = "row"             # "row" | "blocked32" (A and B both) | "b_blocked32" (A row-major, B blocked)
     epilogue: str = "none"          # "none" | "bias_relu"
     dist_a: tuple = ("uniform", 1.0)
     dist_b: tuple = ("uniform", 1.0)
@@ -150,8 +159,8 @@ class Workload:
 
     @property
     def algorithmic_bytes(self) -> int:
-        e_in = 4 if self.in_dtype == "f32" else 2
-        e_out = 4 if self.out_dtype == "f32" else 2
+        e_in = 4 if self.in_dtype == "f32" else 1 if self.in_dtype == "s8" else 2
+        e_out = 4 if self.out_dtype in ("f32", "s32") else 2
         b = e_in * (self.M * self.K + self.K * self.N) + e_out * self.M * self.N
         if self.epilogue != "none":
             b += e_in * self.N
@@ -208,6 +217,17 @@ def paper_mlp() -> list:
         out.append(Workload(f"mlp_bf16_flat_{n}", 512, n, n, "bf16", "bf16", epilogue="bias_relu",
                             dist_a=("normal", 1.0), dist_b=("normal", 0.02), seed=6002 + n))
     return out
+
+
+def s8_set() -> list:
+    """INT8 operands (the Int8 dot product Section 5 names as the next packed type), B packed in
+    groups of four inside 32 x 32 blocks, INT32 result: the large square GEMM, a mid-size one and
+    the paper's 4096-wide MLP layer shape."""
+    return [
+        Workload("x_s8_8192", 8192, 8192, 8192, "s8", "s32", layout="b_blocked32", seed=8017),
+        Workload("x_s8_4096", 4096, 4096, 4096, "s8", "s32", layout="b_blocked32", seed=8018),
+        Workload("x_s8_512x4096x4096", 512, 4096, 4096, "s8", "s32", layout="b_blocked32", seed=8019),
+    ]
 
 
 def f16_set() -> list:

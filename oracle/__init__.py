@@ -67,8 +67,63 @@ def lib():
         L.nko_brgemm.argtypes = [ctypes.c_int64] * 6 + [ctypes.c_int32, ctypes.c_int32, ctypes.c_double,
                                  ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p,
                                  ctypes.c_void_p, ctypes.c_void_p]
+        for f in (L.nko_pack_vnni4, L.nko_unpack_vnni4):
+            f.restype = None
+            f.argtypes = [ctypes.c_void_p, ctypes.c_int64, ctypes.c_int64, ctypes.c_void_p]
+        L.nko_b_index_s8.restype = ctypes.c_int64
+        L.nko_b_index_s8.argtypes = [ctypes.c_int64, ctypes.c_int64, ctypes.c_int32, ctypes.c_int64, ctypes.c_int64]
+        L.nko_gemm_s8.restype = ctypes.c_int
+        L.nko_gemm_s8.argtypes = [ctypes.c_int64, ctypes.c_int64, ctypes.c_int64, ctypes.c_int32, ctypes.c_void_p,
+                                  ctypes.c_void_p, ctypes.c_void_p, ctypes.c_int64, ctypes.c_void_p, ctypes.c_int]
         _lib = L
     return _lib
+
+
+def pack_vnni4(flat: np.ndarray) -> np.ndarray:
+    """[K][N] int8 -> [K/4][N][4]: Figure 1's rule with groups of four (Section 2)."""
+    flat = np.ascontiguousarray(flat, dtype=np.int8)
+    K, N = flat.shape
+    assert K % 4 == 0
+    out = np.empty((K // 4, N, 4), dtype=np.int8)
+    lib().nko_pack_vnni4(flat.ctypes.data, K, N, out.ctypes.data)
+    return out
+
+
+def unpack_vnni4(packed: np.ndarray) -> np.ndarray:
+    packed = np.ascontiguousarray(packed, dtype=np.int8)
+    K4, N, four = packed.shape
+    assert four == 4
+    out = np.empty((K4 * 4, N), dtype=np.int8)
+    lib().nko_unpack_vnni4(packed.ctypes.data, K4 * 4, N, out.ctypes.data)
+    return out
+
+
+def to_blocked_s8(flat_b: np.ndarray) -> np.ndarray:
+    """Scatter a row-major int8 B[K][N] into B_blk4[N/32][K/32][8][32][4] with the oracle's own
+    index function (Python loop; test sizes only)."""
+    K, N = flat_b.shape
+    L = lib()
+    B = np.empty(K * N, dtype=np.int8)
+    for k in range(K):
+        for j in range(N):
+            B[L.nko_b_index_s8(K, N, BLOCKED32, k, j)] = flat_b[k, j]
+    return B
+
+
+def gemm_s8(M, N, K, A, B, *, layout_b=ROW, rows=None, nthreads=None) -> np.ndarray:
+    """Exact integer product of int8 operands: int64 [rows][N] (all M rows by default)."""
+    A = np.ascontiguousarray(A, dtype=np.int8).ravel()
+    B = np.ascontiguousarray(B, dtype=np.int8).ravel()
+    assert A.size == M * K and B.size == K * N
+    r = None if rows is None else np.ascontiguousarray(rows, dtype=np.int64)
+    nr = M if r is None else r.size
+    Y = np.empty((nr, N), dtype=np.int64)
+    nt = nthreads or min(os.cpu_count() or 1, 32)
+    rc = lib().nko_gemm_s8(M, N, K, layout_b, A.ctypes.data, B.ctypes.data, None if r is None else r.ctypes.data,
+                           nr, Y.ctypes.data, nt)
+    if rc != 0:
+        raise ValueError("nko_gemm_s8: bad arguments")
+    return Y
 
 
 def bf16_to_f32(bits: np.ndarray) -> np.ndarray:

@@ -23,6 +23,12 @@
  *     A_blk[M/32][K/32][32][32]         (m-block, k-block, m-in-block, k-in-block)
  *     B_blk[N/32][K/32][16][32][2]      (n-block, k-block, k-pair, n-in-block, k-parity)
  *
+ * INT8 (Section 5c, "other packed types": the Int8 dot product, whose operands Section 2
+ * packs in groups of four): nko_gemm_s8 computes C[i][j] = sum_k a(i,k) * b(k,j) in integers,
+ * exactly (int64 accumulation; results fit int32 while K < 2^17).  A is row-major; B is
+ * row-major or 32x32-blocked with Figure 1's rule at group size four:
+ *     B_blk4[N/32][K/32][8][32][4]      (n-block, k-block, k-quad, n-in-block, k mod 4)
+ *
  * Pins (tests/test_oracle_*.py): Figure 1's printed packing, identity /
  * permutation / diagonal / rank-1 / all-ones closed forms, brute force in a
  * different loop order, numpy float64 matmul on small shapes, blocked-vs-flat
@@ -232,5 +238,72 @@ int nko_brgemm(int64_t M, int64_t N, int64_t K, int64_t batch, int64_t stride_a,
             if (S) S[i * N + j] = s;
         }
     }
+    return 0;
+}
+
+/* ------------------------------------------------------------------ INT8
+ * Figure 1's packing rule with groups of four along k (Section 2: "INT8 elements in groups
+ * of four"): packed[k/4][n][k%4] = flat[k][n]. */
+void nko_pack_vnni4(const int8_t* flat, int64_t K, int64_t N, int8_t* packed) {
+    for (int64_t k = 0; k < K; ++k)
+        for (int64_t n = 0; n < N; ++n)
+            packed[((k / 4) * N + n) * 4 + (k % 4)] = flat[k * N + n];
+}
+
+void nko_unpack_vnni4(const int8_t* packed, int64_t K, int64_t N, int8_t* flat) {
+    for (int64_t k = 0; k < K; ++k)
+        for (int64_t n = 0; n < N; ++n)
+            flat[k * N + n] = packed[((k / 4) * N + n) * 4 + (k % 4)];
+}
+
+/* Storage index of logical element (k,j) of an INT8 B operand. */
+int64_t nko_b_index_s8(int64_t K, int64_t N, int32_t layout_b, int64_t k, int64_t j) {
+    if (layout_b == NKO_ROW) return k * N + j;
+    return ((((j / 32) * (K / 32) + k / 32) * 8 + (k % 32) / 4) * 32 + j % 32) * 4 + k % 4;
+}
+
+typedef struct {
+    int64_t M, N, K;
+    int32_t layout_b;
+    const int8_t *A, *B;
+    const int64_t* rows;
+    int64_t r0, r1;
+    int64_t* Y;
+} job_s8_t;
+
+static void* worker_s8(void* arg) {
+    job_s8_t* w = (job_s8_t*)arg;
+    for (int64_t r = w->r0; r < w->r1; ++r) {
+        const int64_t i = w->rows ? w->rows[r] : r;
+        for (int64_t j = 0; j < w->N; ++j) {
+            int64_t acc = 0;
+            for (int64_t k = 0; k < w->K; ++k)
+                acc += (int64_t)w->A[i * w->K + k] * (int64_t)w->B[nko_b_index_s8(w->K, w->N, w->layout_b, k, j)];
+            w->Y[r * w->N + j] = acc;
+        }
+    }
+    return NULL;
+}
+
+/* Y[r][j] (int64) for the listed rows (all M rows when rows == NULL).  Returns 0, or -1 on bad arguments. */
+int nko_gemm_s8(int64_t M, int64_t N, int64_t K, int32_t layout_b, const int8_t* A, const int8_t* B,
+                const int64_t* rows, int64_t nrows, int64_t* Y, int nthreads) {
+    if (M <= 0 || N <= 0 || K <= 0 || !A || !B || !Y) return -1;
+    if (layout_b != NKO_ROW && (layout_b != NKO_BLOCKED32 || N % 32 || K % 32)) return -1;
+    const int64_t nr = rows ? nrows : M;
+    if (rows)
+        for (int64_t r = 0; r < nr; ++r)
+            if (rows[r] < 0 || rows[r] >= M) return -1;
+    if (nthreads < 1) nthreads = 1;
+    if (nthreads > 64) nthreads = 64;
+    if (nthreads > nr) nthreads = (int)nr;
+    pthread_t th[64];
+    job_s8_t jobs[64];
+    for (int t = 0; t < nthreads; ++t) {
+        job_s8_t j = {M, N, K, layout_b, A, B, rows, nr * t / nthreads, nr * (t + 1) / nthreads, Y};
+        jobs[t] = j;
+        if (pthread_create(&th[t], NULL, worker_s8, &jobs[t]) != 0) return -1;
+    }
+    for (int t = 0; t < nthreads; ++t) pthread_join(th[t], NULL);
     return 0;
 }

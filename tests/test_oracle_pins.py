@@ -461,3 +461,73 @@ def test_f16_gemm_equals_gemm_of_the_widened_operands():
     # a BF16 reading of the same bits gives something else: the dtype switch is live
     Yb, _ = oracle.gemm(40, 48, 64, A, B, in_dtype=BF16)
     assert not np.array_equal(Y, Yb)
+
+
+# ---------------------------------------------------------------- INT8 (Section 5c; packing in groups of four, Section 2)
+def test_vnni4_is_fig1_rule_with_groups_of_four():
+    """Figure 1's flat 4 x 4 matrix 0..15 under the same rule with four k per group: one row of
+    quadruples (0,4,8,12) (1,5,9,13) (2,6,10,14) (3,7,11,15); and the pair packing of Figure 1 is what
+    the quadruple packing gives when rows 2k, 2k+1 are read out of a quadruple's halves."""
+    flat = np.arange(16, dtype=np.int8).reshape(4, 4)
+    p4 = oracle.pack_vnni4(flat)
+    assert p4.tolist() == [[[0, 4, 8, 12], [1, 5, 9, 13], [2, 6, 10, 14], [3, 7, 11, 15]]]
+    with open(os.path.join(GOLD, "fig1_vnni2.txt")) as f:
+        printed = [[int(v) for v in line.split()[1:]] for line in f if line.startswith("packed")]
+    halves = [[v for q in p4[0].tolist() for v in q[0:2]], [v for q in p4[0].tolist() for v in q[2:4]]]
+    assert halves == printed
+    rng = np.random.default_rng(5)
+    x = rng.integers(-128, 128, (64, 96), dtype=np.int8)
+    assert np.array_equal(oracle.unpack_vnni4(oracle.pack_vnni4(x)), x)
+
+
+def test_s8_blocked_b_block_is_vnni4_packing_of_the_flat_block():
+    rng = np.random.default_rng(6)
+    K, N = 64, 96
+    flat = rng.integers(-128, 128, (K, N), dtype=np.int8)
+    blk = oracle.to_blocked_s8(flat).reshape(N // 32, K // 32, 8, 32, 4)
+    for nb in range(N // 32):
+        for kb in range(K // 32):
+            want = oracle.pack_vnni4(flat[kb * 32:(kb + 1) * 32, nb * 32:(nb + 1) * 32])
+            assert np.array_equal(blk[nb, kb], want)
+
+
+def test_s8_gemm_closed_forms_and_numpy():
+    rng = np.random.default_rng(7)
+    M, N, K = 37, 64, 96
+    A = rng.integers(-128, 128, (M, K), dtype=np.int8)
+    B = rng.integers(-128, 128, (K, N), dtype=np.int8)
+    want = A.astype(np.int64) @ B.astype(np.int64)            # library routine on a small case
+    got = oracle.gemm_s8(M, N, K, A, B)
+    assert got.dtype == np.int64 and np.array_equal(got, want)
+    # blocked B gives the same integers; so does any row subset and any thread count
+    Bb = oracle.to_blocked_s8(B)
+    assert np.array_equal(oracle.gemm_s8(M, N, K, A, Bb, layout_b=BLOCKED32), want)
+    rows = np.array([36, 0, 5, 5], dtype=np.int64)
+    assert np.array_equal(oracle.gemm_s8(M, N, K, A, Bb, layout_b=BLOCKED32, rows=rows, nthreads=3), want[rows])
+    # identity: A . I = A; extremes: (-128) . (-128) summed K times
+    eye = np.eye(K, dtype=np.int8)
+    assert np.array_equal(oracle.gemm_s8(M, K, K, A, eye), A.astype(np.int64))
+    lo = np.full((2, K), -128, dtype=np.int8)
+    assert np.array_equal(oracle.gemm_s8(2, N, K, lo, np.full((K, N), -128, dtype=np.int8)),
+                          np.full((2, N), 16384 * K, dtype=np.int64))
+    # non-square roles: a transposed operand is caught
+    assert not np.array_equal(oracle.gemm_s8(M, N, K, A, np.ascontiguousarray(B.T).reshape(K, N)), want)
+
+
+def test_s8_planted_mistake_in_the_quad_order_is_caught():
+    rng = np.random.default_rng(8)
+    K, N = 32, 32
+    A = rng.integers(-128, 128, (4, K), dtype=np.int8)
+    B = rng.integers(-128, 128, (K, N), dtype=np.int8)
+    good = oracle.to_blocked_s8(B)
+    bad = good.reshape(-1, 4)[:, [1, 0, 2, 3]].reshape(-1)        # first two k of every quadruple swapped
+    want = oracle.gemm_s8(4, N, K, A, B)
+    assert np.array_equal(oracle.gemm_s8(4, N, K, A, good, layout_b=BLOCKED32), want)
+    assert not np.array_equal(oracle.gemm_s8(4, N, K, A, np.ascontiguousarray(bad), layout_b=BLOCKED32), want)
+
+
+def test_s8_generator_covers_the_range():
+    v = nk_inputs.fill(11, nk_inputs.TENSOR_A, 1 << 16, dtype="s8")
+    assert v.dtype == np.int8 and v.min() == -128 and v.max() == 127
+    assert abs(float(v.astype(np.float64).mean())) < 1.5
+    assert np.array_equal(v[100:200], nk_inputs.fill(11, nk_inputs.TENSOR_A, 100, dtype="s8", start=100))
