@@ -57,8 +57,14 @@ typedef enum {
 typedef enum {
     NK_F32 = 0,
     NK_BF16 = 1,
-    NK_F16 = 2 /* IEEE binary16: the other 16-bit packed type (Section 5 names FP16 as the next one); same
-                  kernels, layouts and rules as BF16, FP32 accumulation, one RNE rounding of a 16-bit C */
+    NK_F16 = 2, /* IEEE binary16: the other 16-bit packed type (Section 5 names FP16 as the next one); same
+                   kernels, layouts and rules as BF16, FP32 accumulation, one RNE rounding of a 16-bit C */
+    NK_S8 = 3, /* signed 8-bit integers: the Int8 dot product Section 5 names among the next packed types.  A is
+                  row-major; B is NK_BLOCKED32 with four k per group (Section 2: "INT8 elements in groups of
+                  four"): B[N/32][K/32][8][32][4], packed[k/4][n][k%4] = flat[k][n] inside each 32 x 32 block.
+                  The result is exact: INT32 accumulation of at most 2^17 - 1 products.  No epilogue, no beta,
+                  no batch, no K split; N and K multiples of 32 */
+    NK_S32 = 4 /* signed 32-bit integers: the type of C for NK_S8 operands (and only for them) */
 } nk_dtype_t;
 typedef enum { NK_ROW_MAJOR = 0, NK_BLOCKED32 = 1 } nk_layout_t;
 typedef enum { NK_EPI_NONE = 0, NK_EPI_BIAS_RELU = 1 } nk_epilogue_t;

@@ -10,7 +10,7 @@ import os
 
 from . import _build
 
-F32, BF16, F16 = 0, 1, 2
+F32, BF16, F16, S8, S32 = 0, 1, 2, 3, 4
 ROW_MAJOR, BLOCKED32 = 0, 1
 EPI_NONE, EPI_BIAS_RELU = 0, 1
 FLAG_KERNEL_NAIVE, FLAG_KERNEL_SIMT, FLAG_KERNEL_UMMA = 0x1, 0x2, 0x3
@@ -191,12 +191,12 @@ class Plan:
 
 
 def plan_for(w, device=0, flags=0) -> Plan:
-    """Plan for a workload record with M, N, K, in_dtype ("f32"/"bf16"/"f16"), out_dtype,
+    """Plan for a workload record with M, N, K, in_dtype ("f32"/"bf16"/"f16"/"s8"), out_dtype,
     layout ("row"/"blocked32") and epilogue ("none"/"bias_relu") attributes."""
-    lay = BLOCKED32 if w.layout == "blocked32" else ROW_MAJOR
-    return Plan(w.M, w.N, w.K,
-                in_dtype={"f32": F32, "bf16": BF16, "f16": F16}[w.in_dtype],
-                out_dtype={"f32": F32, "bf16": BF16, "f16": F16}[w.out_dtype],
-                layout_a=lay, layout_b=lay,
+    lay_a = BLOCKED32 if w.layout == "blocked32" else ROW_MAJOR
+    lay_b = BLOCKED32 if w.layout in ("blocked32", "b_blocked32") else ROW_MAJOR
+    types = {"f32": F32, "bf16": BF16, "f16": F16, "s8": S8, "s32": S32}
+    return Plan(w.M, w.N, w.K, in_dtype=types[w.in_dtype], out_dtype=types[w.out_dtype],
+                layout_a=lay_a, layout_b=lay_b,
                 epilogue=EPI_BIAS_RELU if w.epilogue == "bias_relu" else EPI_NONE,
                 device=device, flags=flags)

@@ -104,14 +104,26 @@ struct DeviceGuard {
 };
 
 static inline bool is16(int dt) { return dt == NK_BF16 || dt == NK_F16; }   // a 16-bit element type
+static inline bool is_s8(const nk_gemm_desc_t& d) { return d.in_dtype == NK_S8; }
+// k elements in one stage row of the tensor-core kernels (128 bytes)
+static inline int kblock(const nk_gemm_desc_t& d) { return d.in_dtype == NK_S8 ? 2 * UMMA_BK : UMMA_BK; }
 static inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 static inline int ceil_div(int64_t a, int64_t b) { return static_cast<int>((a + b - 1) / b); }
 
 // tcgen05 instruction descriptor, kind::f16: D format FP32 (bit 4), A and B format at bits 7 and
 // 10 (0 = FP16, 1 = BF16), B major-ness (bit 16: 0 = K-major, 1 = N-major), N/8 at bit 17,
 // M/16 at bit 24.  A is always K-major.
-static uint32_t make_idesc(int m, int n, bool b_n_major, bool f16) {
+static uint32_t make_idesc(int m, int n, bool b_n_major, bool f16, bool s8 = false) {
     uint32_t d = 0;
+    if (s8) {
+        // kind::i8: D format INT32 (2 at bit 4), A and B format signed 8-bit (1 at bits 7 and 10)
+        d |= 2u << 4;
+        d |= 1u << 7;
+        d |= 1u << 10;
+        d |= static_cast<uint32_t>(n >> 3) << 17;
+        d |= static_cast<uint32_t>(m >> 4) << 24;
+        return d;   // both operands K-major
+    }
     d |= 1u << 4;
     d |= (f16 ? 0u : 1u) << 7;
     d |= (f16 ? 0u : 1u) << 10;
@@ -157,7 +169,7 @@ static bool cluster_reduce_fits(const nk_gemm_desc_t& d, int sms, bool pair, int
 }
 
 static double umma_model_us(const nk_gemm_desc_t& d, int sms, bool pair, int bn, int splits) {
-    const int kb_total = desc_batch(d) * ceil_div(d.K, UMMA_BK);
+    const int kb_total = desc_batch(d) * ceil_div(d.K, kblock(d));
     const int per = ceil_div(kb_total, splits);
     const int eff_splits = ceil_div(kb_total, per);
     const int64_t tiles = static_cast<int64_t>(desc_gemms(d)) * ceil_div(d.M, pair ? 256 : 128) * ceil_div(d.N, bn);
@@ -188,7 +200,7 @@ static double umma_model_us(const nk_gemm_desc_t& d, int sms, bool pair, int bn,
         const double vnni = (32.0 + cols / 2.0) / 250.0;
         if (vnni > t_kb) t_kb = vnni;
     }
-    const double eo = d.out_dtype == NK_F32 ? 4.0 : 2.0;
+    const double eo = is16(d.out_dtype) ? 2.0 : 4.0;
     const double mn = static_cast<double>(d.M) * d.N;
     const double chunks = bn / 32.0;
     double us = start + rounds * per * t_kb;
@@ -207,7 +219,7 @@ static double umma_model_us(const nk_gemm_desc_t& d, int sms, bool pair, int bn,
 static void choose_umma(nk_gemm_s* p) {
     const nk_gemm_desc_t& d = p->d;
     const int sms = p->sm_count;
-    const int kb_total = desc_batch(d) * ceil_div(d.K, UMMA_BK);
+    const int kb_total = desc_batch(d) * ceil_div(d.K, kblock(d));
     const int forced_bn = (d.flags >> NK_FLAG_TILE_N_SHIFT) & 0xF;
     const int forced_s = (d.flags >> NK_FLAG_SPLITK_SHIFT) & 0xFF;
     const int split_cands[8] = {1, 2, 3, 4, 6, 8, 12, 16};
@@ -224,6 +236,7 @@ static void choose_umma(nk_gemm_s* p) {
                 int splits = forced_s > 0 ? forced_s : split_cands[si];
                 if (forced_s > 0 && si > 0) break;
                 if (splits > kb_total) splits = kb_total;
+                if (is_s8(d) && splits > 1) continue;   // INT32 partial sums have no reduce path: one unit per tile
                 if (forced_s == 0 && splits > 1) {
                     if (kb_total / splits < 4) continue;  // >= 4 k-blocks per split
                     if (static_cast<double>(splits) * desc_gemms(d) * d.M * d.N * 4.0 > 256.0 * 1024 * 1024) continue;
@@ -233,7 +246,7 @@ static void choose_umma(nk_gemm_s* p) {
             }
         }
     }
-    if (best.us >= 1e30) best = {false, 64, forced_s > 0 ? forced_s : 1, 0.0};  // contradictory overrides
+    if (best.us >= 1e30) best = {false, 64, (forced_s > 0 && !is_s8(d)) ? forced_s : 1, 0.0};  // contradictory overrides
     int splits = best.splits;
     if (splits > kb_total) splits = kb_total;
     if (splits < 1) splits = 1;
@@ -332,7 +345,9 @@ static void choose_skinny(nk_gemm_s* p) {
 static nk_status_t encode_maps(nk_gemm_s* p, const void* A, const void* B) {
     if (p->cached_a == A && p->cached_b == B) return NK_OK;
     const nk_gemm_desc_t& d = p->d;
-    const CUtensorMapDataType half_type = d.in_dtype == NK_F16 ? CU_TENSOR_MAP_DATA_TYPE_FLOAT16 : CU_TENSOR_MAP_DATA_TYPE_BFLOAT16;
+    const CUtensorMapDataType half_type = d.in_dtype == NK_S8 ? CU_TENSOR_MAP_DATA_TYPE_UINT8
+                                          : d.in_dtype == NK_F16 ? CU_TENSOR_MAP_DATA_TYPE_FLOAT16 : CU_TENSOR_MAP_DATA_TYPE_BFLOAT16;
+    const cuuint64_t esz = d.in_dtype == NK_S8 ? 1 : 2;   // bytes per operand element
     CUresult r;
     if (d.layout_a == NK_BLOCKED32) {
         // [M/32][K/32][32][32] as a 4-D tensor (k, m, k-block, m-block): a box of
@@ -348,8 +363,8 @@ static nk_status_t encode_maps(nk_gemm_s* p, const void* A, const void* B) {
         // A row-major [batch][M][K] (batch items stride_a elements apart): (k, m, item)
         cuuint64_t dims[3] = {static_cast<cuuint64_t>(d.K), static_cast<cuuint64_t>(d.M),
                               static_cast<cuuint64_t>(p->batch * p->gemms)};
-        cuuint64_t strides[2] = {static_cast<cuuint64_t>(d.K) * 2, static_cast<cuuint64_t>(p->stride_a) * 2};
-        cuuint32_t box[3] = {UMMA_BK, UMMA_BM, 1};
+        cuuint64_t strides[2] = {static_cast<cuuint64_t>(d.K) * esz, static_cast<cuuint64_t>(p->stride_a) * esz};
+        cuuint32_t box[3] = {static_cast<cuuint32_t>(kblock(d)), UMMA_BM, 1};   // 128 bytes of k per row
         cuuint32_t es[3] = {1, 1, 1};
         r = p->encode(&p->tmap_a, half_type, 3, const_cast<void*>(A), dims, strides,
                       box, es, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
@@ -398,10 +413,12 @@ static nk_status_t encode_maps(nk_gemm_s* p, const void* A, const void* B) {
         // operand is the 3-D tensor (64, K/2, N/32).  One box brings the 32 pair rows of a 64-deep
         // stage for all the column blocks a CTA covers, swizzled per 128-byte row; rows beyond
         // K/2 and column blocks beyond N/32 arrive as zeros.
+        // INT8: the same bytes with four k per group: [N/32][K/32][8][32][4] is (128 elements, K/4, N/32).
         const int cols = p->pair ? p->bn / 2 : p->bn;
-        cuuint64_t dims[3] = {64, static_cast<cuuint64_t>(d.K / 2), static_cast<cuuint64_t>(d.N / 32)};
-        cuuint64_t strides[2] = {128, static_cast<cuuint64_t>(d.K) * 64};
-        cuuint32_t box[3] = {64, UMMA_BK / 2, static_cast<cuuint32_t>(cols / 32)};
+        const cuuint64_t group = 4 / esz;   // k per 32-bit word: 2 (16-bit) or 4 (8-bit)
+        cuuint64_t dims[3] = {128 / esz, static_cast<cuuint64_t>(d.K) / group, static_cast<cuuint64_t>(d.N / 32)};
+        cuuint64_t strides[2] = {128, static_cast<cuuint64_t>(d.K) * 32 * esz};
+        cuuint32_t box[3] = {static_cast<cuuint32_t>(128 / esz), UMMA_BK / 2, static_cast<cuuint32_t>(cols / 32)};
         cuuint32_t es[3] = {1, 1, 1};
         r = p->encode(&p->tmap_b, half_type, 3, const_cast<void*>(B), dims, strides,
                       box, es, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
@@ -428,7 +445,7 @@ static nk_status_t encode_c_map(nk_gemm_s* p, void* C) {
     cuuint32_t box[3] = {32, 32, 1};
     cuuint32_t es[3] = {1, 1, 1};
     // a box row is 128 bytes of FP32 (128-byte swizzle) or 64 bytes of BF16 (64-byte swizzle)
-    CUresult r = p->encode(&p->tmap_c, !bf16 ? CU_TENSOR_MAP_DATA_TYPE_FLOAT32 : d.out_dtype == NK_F16 ? CU_TENSOR_MAP_DATA_TYPE_FLOAT16 : CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, C,
+    CUresult r = p->encode(&p->tmap_c, d.out_dtype == NK_S32 ? CU_TENSOR_MAP_DATA_TYPE_INT32 : !bf16 ? CU_TENSOR_MAP_DATA_TYPE_FLOAT32 : d.out_dtype == NK_F16 ? CU_TENSOR_MAP_DATA_TYPE_FLOAT16 : CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, C,
                            dims, strides, box, es, CU_TENSOR_MAP_INTERLEAVE_NONE,
                            bf16 ? CU_TENSOR_MAP_SWIZZLE_64B : CU_TENSOR_MAP_SWIZZLE_128B,
                            CU_TENSOR_MAP_L2_PROMOTION_NONE, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
@@ -440,17 +457,22 @@ static nk_status_t encode_c_map(nk_gemm_s* p, void* C) {
     return NK_OK;
 }
 
-template <int BN, int STAGES, bool VNNI>
+template <int BN, int STAGES, bool VNNI, bool I8 = false>
 static cudaError_t launch_umma_t(nk_gemm_s* p, const UmmaParams& up, int grid, cudaStream_t st) {
-    auto k = umma_bf16_kernel<BN, STAGES, VNNI>;
-    umma_bf16_kernel<BN, STAGES, VNNI><<<grid, VNNI ? 320 : 192, umma_smem_bytes(BN, STAGES), st>>>(
+    umma_bf16_kernel<BN, STAGES, VNNI, false, I8><<<grid, VNNI ? 320 : 192, umma_smem_bytes(BN, STAGES), st>>>(
         p->tmap_a, p->tmap_b, p->tmap_c, up);
-    (void)k;
     return cudaGetLastError();
 }
 
 static cudaError_t launch_umma(nk_gemm_s* p, const UmmaParams& up, int grid, cudaStream_t st) {
     const bool v = p->b_vnni_inkernel;
+    if (is_s8(p->d)) {   // INT8 operands: B is always blocked and re-laid in the kernel
+        switch (p->bn) {
+            case 256: return launch_umma_t<256, 4, true, true>(p, up, grid, st);
+            case 128: return launch_umma_t<128, 6, true, true>(p, up, grid, st);
+            default:  return launch_umma_t<64, 8, true, true>(p, up, grid, st);
+        }
+    }
     switch (p->bn) {
         case 256: return v ? launch_umma_t<256, 4, true>(p, up, grid, st) : launch_umma_t<256, 4, false>(p, up, grid, st);
         case 128: return v ? launch_umma_t<128, 6, true>(p, up, grid, st) : launch_umma_t<128, 6, false>(p, up, grid, st);
@@ -527,7 +549,7 @@ static int max_clusters_for(bool pair, int bn, bool vnni, int splits) {
     return c > 0 ? c : 0;
 }
 
-template <int BN, int STAGES, bool VNNI>
+template <int BN, int STAGES, bool VNNI, bool I8 = false>
 static cudaError_t launch_pair_t(nk_gemm_s* p, const UmmaParams& up, int pairs, cudaStream_t st) {
     cudaLaunchConfig_t cfg;
     memset(&cfg, 0, sizeof(cfg));
@@ -542,11 +564,12 @@ static cudaError_t launch_pair_t(nk_gemm_s* p, const UmmaParams& up, int pairs, 
     attr.val.clusterDim.z = 1;
     cfg.attrs = &attr;
     cfg.numAttrs = 1;
-    return cudaLaunchKernelEx(&cfg, umma_bf16_pair_kernel<BN, STAGES, VNNI>, p->tmap_a, p->tmap_b, p->tmap_c, up);
+    return cudaLaunchKernelEx(&cfg, umma_bf16_pair_kernel<BN, STAGES, VNNI, false, I8>, p->tmap_a, p->tmap_b, p->tmap_c, up);
 }
 
 static cudaError_t launch_pair(nk_gemm_s* p, const UmmaParams& up, int pairs, cudaStream_t st) {
     const bool v = p->b_vnni_inkernel;
+    if (is_s8(p->d)) return p->bn == 256 ? launch_pair_t<256, 6, true, true>(p, up, pairs, st) : launch_pair_t<128, 8, true, true>(p, up, pairs, st);
     if (p->bn == 256) return v ? launch_pair_t<256, 6, true>(p, up, pairs, st) : launch_pair_t<256, 6, false>(p, up, pairs, st);
     return v ? launch_pair_t<128, 8, true>(p, up, pairs, st) : launch_pair_t<128, 8, false>(p, up, pairs, st);
 }
@@ -595,6 +618,11 @@ static cudaError_t prepare_umma_attrs() {
     if ((e = allow_smem(umma_bf16_pair_kernel<256, 6, true, true>, pair_smem_bytes(256, 6))) != cudaSuccess) return e;
     if ((e = allow_smem(umma_bf16_pair_kernel<128, 8, false, true>, pair_smem_bytes(128, 8))) != cudaSuccess) return e;
     if ((e = allow_smem(umma_bf16_pair_kernel<128, 8, true, true>, pair_smem_bytes(128, 8))) != cudaSuccess) return e;
+    if ((e = allow_smem(umma_bf16_kernel<256, 4, true, false, true>, umma_smem_bytes(256, 4))) != cudaSuccess) return e;
+    if ((e = allow_smem(umma_bf16_kernel<128, 6, true, false, true>, umma_smem_bytes(128, 6))) != cudaSuccess) return e;
+    if ((e = allow_smem(umma_bf16_kernel<64, 8, true, false, true>, umma_smem_bytes(64, 8))) != cudaSuccess) return e;
+    if ((e = allow_smem(umma_bf16_pair_kernel<256, 6, true, false, true>, pair_smem_bytes(256, 6))) != cudaSuccess) return e;
+    if ((e = allow_smem(umma_bf16_pair_kernel<128, 8, true, false, true>, pair_smem_bytes(128, 8))) != cudaSuccess) return e;
     return cudaSuccess;
 }
 
@@ -638,14 +666,24 @@ nk_status_t nk_gemm_create(const nk_gemm_desc_t* desc, nk_gemm_t* out) {
     if (d.M <= 0 || d.N <= 0 || d.K <= 0) return NK_ERR_INVALID_ARG;
     if (d.M > (1 << 24) || d.N > (1 << 24) || d.K > (1 << 24)) return NK_ERR_UNSUPPORTED;
     if (d.M * d.N >= (1ll << 31) || d.M * d.K >= (1ll << 33) || d.K * d.N >= (1ll << 33)) return NK_ERR_UNSUPPORTED;
-    if (d.in_dtype != NK_F32 && !is16(d.in_dtype)) return NK_ERR_INVALID_ARG;
-    if (d.out_dtype != NK_F32 && !is16(d.out_dtype)) return NK_ERR_INVALID_ARG;
+    if (d.in_dtype != NK_F32 && !is16(d.in_dtype) && d.in_dtype != NK_S8) return NK_ERR_INVALID_ARG;
+    if (d.out_dtype != NK_F32 && !is16(d.out_dtype) && d.out_dtype != NK_S32) return NK_ERR_INVALID_ARG;
+    if ((d.in_dtype == NK_S8) != (d.out_dtype == NK_S32)) return NK_ERR_INVALID_ARG;   // INT8 operands <-> INT32 result
+    if (d.in_dtype == NK_S8) {
+        // the Int8 dot product: A row-major, B packed in groups of four inside 32 x 32 blocks, exact INT32 C
+        if (d.layout_a != NK_ROW_MAJOR || d.layout_b != NK_BLOCKED32 || d.layout_c != NK_ROW_MAJOR) return NK_ERR_UNSUPPORTED;
+        if (d.epilogue != NK_EPI_NONE || d.beta != 0 || d.batch > 1) return NK_ERR_UNSUPPORTED;
+        if (d.flags & (NK_FLAG_REPACK_B | NK_FLAG_SEPARATE_REDUCE)) return NK_ERR_UNSUPPORTED;
+        const uint32_t fk = d.flags & NK_FLAG_KERNEL_MASK;
+        if (fk == NK_FLAG_KERNEL_NAIVE || fk == NK_FLAG_KERNEL_SIMT) return NK_ERR_UNSUPPORTED;
+        if (d.K >= (1ll << 17)) return NK_ERR_UNSUPPORTED;   // INT32 accumulation is exact below 2^17 terms
+    }
     if (d.layout_a != NK_ROW_MAJOR && d.layout_a != NK_BLOCKED32) return NK_ERR_INVALID_ARG;
     if (d.layout_b != NK_ROW_MAJOR && d.layout_b != NK_BLOCKED32) return NK_ERR_INVALID_ARG;
     if (d.epilogue != NK_EPI_NONE && d.epilogue != NK_EPI_BIAS_RELU) return NK_ERR_INVALID_ARG;
     if (is16(d.out_dtype) && d.in_dtype != d.out_dtype) return NK_ERR_INVALID_ARG;   // a 16-bit C has the operands' type
     const bool blocked = d.layout_a == NK_BLOCKED32 || d.layout_b == NK_BLOCKED32;
-    if (blocked && !is16(d.in_dtype)) return NK_ERR_UNSUPPORTED;
+    if (blocked && !is16(d.in_dtype) && d.in_dtype != NK_S8) return NK_ERR_UNSUPPORTED;
     if (d.layout_a == NK_BLOCKED32 && (d.M % 32 || d.K % 32)) return NK_ERR_MISALIGNED;
     if (d.layout_b == NK_BLOCKED32 && (d.N % 32 || d.K % 32)) return NK_ERR_MISALIGNED;
     if (d.beta != 0 && d.beta != 1) return NK_ERR_INVALID_ARG;
@@ -686,7 +724,7 @@ nk_status_t nk_gemm_create(const nk_gemm_desc_t* desc, nk_gemm_t* out) {
         if (is16(d.in_dtype) && (d.N % 8 || d.K % 8)) return NK_ERR_MISALIGNED;
         if (d.in_dtype == NK_F32 && (d.N % 4 || d.K % 4)) return NK_ERR_MISALIGNED;
         if (force == NK_FLAG_KERNEL_SIMT && d.in_dtype != NK_F32) return NK_ERR_UNSUPPORTED;
-        if (force == NK_FLAG_KERNEL_UMMA && !is16(d.in_dtype)) return NK_ERR_UNSUPPORTED;
+        if (force == NK_FLAG_KERNEL_UMMA && !is16(d.in_dtype) && d.in_dtype != NK_S8) return NK_ERR_UNSUPPORTED;
     }
 
     int ndev = 0;
@@ -808,9 +846,9 @@ nk_status_t nk_gemm_create(const nk_gemm_desc_t* desc, nk_gemm_t* out) {
         // reduce kernel and the partials (FP32, written and read once).
         p->tail_from = -1;
         p->tail_splits = 0;
-        if (p->pair && p->splits == 1 && p->gemms == 1 && !(d.flags & NK_FLAG_NO_TAIL_SPLIT)) {
+        if (p->pair && p->splits == 1 && p->gemms == 1 && !(d.flags & NK_FLAG_NO_TAIL_SPLIT) && !is_s8(d)) {
             const int tiles = ceil_div(d.M, 2 * UMMA_BM) * ceil_div(d.N, p->bn);
-            const int kb_total = p->batch * ceil_div(d.K, UMMA_BK);
+            const int kb_total = p->batch * ceil_div(d.K, kblock(d));
             const int tail = tiles % p->max_pairs;
             if (tiles > p->max_pairs && tail > 0 && (2 * tail <= p->max_pairs || ((d.flags >> NK_FLAG_TAIL_SPLIT_SHIFT) & 0xF) >= 2)) {
                 int sp = p->max_pairs / tail;
@@ -837,8 +875,8 @@ nk_status_t nk_gemm_create(const nk_gemm_desc_t* desc, nk_gemm_t* out) {
             p->ws_partial_bytes = static_cast<size_t>(tiles - p->tail_from) * p->tail_splits * 2 * UMMA_BM * p->bn * 4;
         }
         p->launches = 1 + ((p->splits > 1 && !p->cluster_reduce) || p->tail_from >= 0 ? 1 : 0) + (p->b_repack ? 1 : 0);
-        snprintf(p->name, sizeof(p->name), "umma_bf16_%s%dx64_s%d_splitk%d%s%s%s",
-                 p->pair ? "pair_256x" : "128x", p->bn, p->stages,
+        snprintf(p->name, sizeof(p->name), "umma_bf16_%s%dx%d_s%d_splitk%d%s%s%s",
+                 p->pair ? "pair_256x" : "128x", p->bn, kblock(d), p->stages,
                  p->splits, p->cluster_reduce ? "_cluster" : "", d.layout_a == NK_BLOCKED32 ? "_ablk" : "",
                  p->b_vnni_inkernel ? "_bvnni" : (p->b_repack ? "_brepack" : ""));
     }
@@ -858,6 +896,10 @@ nk_status_t nk_gemm_create(const nk_gemm_desc_t* desc, nk_gemm_t* out) {
     if (d.in_dtype == NK_F16) {
         const size_t len = strlen(p->name);
         snprintf(p->name + len, sizeof(p->name) - len, "_f16");
+    }
+    if (d.in_dtype == NK_S8) {
+        const size_t len = strlen(p->name);
+        snprintf(p->name + len, sizeof(p->name) - len, "_s8");
     }
     // split-K partials are laid out [split][gemm][M][N] and reduced as one flat array: that
     // needs the C of a batched matmul to be contiguous
@@ -967,7 +1009,7 @@ nk_status_t nk_gemm_run(nk_gemm_t p, const void* A, const void* B, const void* b
         up.tiles_m = ceil_div(d.M, p->pair ? 2 * UMMA_BM : UMMA_BM);
         up.tiles_n = ceil_div(d.N, p->bn);
         up.splits = p->splits;
-        up.kb_per_item = ceil_div(d.K, UMMA_BK);
+        up.kb_per_item = ceil_div(d.K, kblock(d));
         up.kb_total = p->batch * up.kb_per_item;
         up.beta = d.beta;
         up.gemms = p->gemms;
@@ -981,7 +1023,7 @@ nk_status_t nk_gemm_run(nk_gemm_t p, const void* A, const void* B, const void* b
         up.b_3d = p->b_3d ? 1 : 0;
         up.epilogue = d.epilogue;
         up.out_bf16 = is16(d.out_dtype);
-        up.idesc = make_idesc(p->pair ? 2 * UMMA_BM : UMMA_BM, p->bn, !p->b_vnni_inkernel, d.in_dtype == NK_F16);
+        up.idesc = make_idesc(p->pair ? 2 * UMMA_BM : UMMA_BM, p->bn, !p->b_vnni_inkernel, d.in_dtype == NK_F16, is_s8(d));
         up.f16 = d.in_dtype == NK_F16;
         up.bias = bias;
         up.C = C;
@@ -1036,7 +1078,7 @@ nk_status_t nk_gemm_run_host(nk_gemm_t p, const void* hA, const void* hB, const 
     if (!p || !hA || !hB || !hC || !dA || !dB || !dC) return NK_ERR_INVALID_ARG;
     const nk_gemm_desc_t& d = p->d;
     if (d.epilogue != NK_EPI_NONE && (!hbias || !dbias)) return NK_ERR_INVALID_ARG;
-    const size_t ein = is16(d.in_dtype) ? 2 : 4, eout = is16(d.out_dtype) ? 2 : 4;
+    const size_t ein = d.in_dtype == NK_S8 ? 1 : is16(d.in_dtype) ? 2 : 4, eout = is16(d.out_dtype) ? 2 : 4;
     cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
     DeviceGuard guard(d.device);
     if (guard.err != cudaSuccess) { set_err(p, "cudaSetDevice", guard.err); return NK_ERR_DEVICE; }
@@ -1081,7 +1123,7 @@ nk_status_t nk_gemm_run_host(nk_gemm_t p, const void* hA, const void* hB, const 
             }
         }
         if (p->chunk_plan) {
-            const size_t ein_b = is16(d.in_dtype) ? 2 : 4, eout_b = is16(d.out_dtype) ? 2 : 4;
+            const size_t ein_b = d.in_dtype == NK_S8 ? 1 : is16(d.in_dtype) ? 2 : 4, eout_b = is16(d.out_dtype) ? 2 : 4;
             const int panels = p->chunk_panels;
             const size_t rows = static_cast<size_t>(p->chunk_rows), cols = static_cast<size_t>(d.N) / panels;
             const size_t a_chunk = rows * d.K * ein_b;                         // also right for blocked A
