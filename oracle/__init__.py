@@ -72,6 +72,8 @@ def lib():
             f.argtypes = [ctypes.c_void_p, ctypes.c_int64, ctypes.c_int64, ctypes.c_void_p]
         L.nko_b_index_s8.restype = ctypes.c_int64
         L.nko_b_index_s8.argtypes = [ctypes.c_int64, ctypes.c_int64, ctypes.c_int32, ctypes.c_int64, ctypes.c_int64]
+        L.nko_quantize_s8.restype = None
+        L.nko_quantize_s8.argtypes = [ctypes.c_void_p, ctypes.c_int64, ctypes.c_float, ctypes.c_void_p]
         L.nko_gemm_s8.restype = ctypes.c_int
         L.nko_gemm_s8.argtypes = [ctypes.c_int64, ctypes.c_int64, ctypes.c_int64, ctypes.c_int32, ctypes.c_void_p,
                                   ctypes.c_void_p, ctypes.c_void_p, ctypes.c_int64, ctypes.c_void_p, ctypes.c_int]
@@ -268,3 +270,26 @@ def brgemm(M, N, K, batch, A, B, bias=None, C0=None, *, in_dtype=F32, epilogue=E
     if rc != 0:
         raise ValueError("oracle rejected the arguments")
     return Y, S
+
+
+def quantize_s8(x: np.ndarray, inv_scale: float) -> np.ndarray:
+    """FP32 -> INT8: saturate(round-half-even(fl32(x * inv_scale))); NaN -> 0."""
+    x = np.ascontiguousarray(x, dtype=np.float32)
+    q = np.empty(x.shape, dtype=np.int8)
+    lib().nko_quantize_s8(x.ctypes.data, x.size, float(np.float32(inv_scale)), q.ctypes.data)
+    return q
+
+
+def gemm_s8_scaled(M, N, K, A, B, scale, bias=None, *, layout_b=ROW, rows=None, relu=False):
+    """The quantised layer on top of the exact integer product: y = scale * (A.B) (+ bias, then
+    max(., 0)), in float64, with S = |scale * (A.B)| (+ |bias|) as the scale of the error bound."""
+    acc = gemm_s8(M, N, K, A, B, layout_b=layout_b, rows=rows).astype(np.float64)
+    y = float(np.float32(scale)) * acc
+    s = np.abs(y)
+    if bias is not None:
+        b = np.asarray(bias, dtype=np.float32).astype(np.float64)
+        y = y + b[None, :]
+        s = s + np.abs(b)[None, :]
+    if relu:
+        y = np.maximum(y, 0.0)
+    return y, s

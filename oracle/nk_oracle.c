@@ -307,3 +307,16 @@ int nko_gemm_s8(int64_t M, int64_t N, int64_t K, int32_t layout_b, const int8_t*
     for (int t = 0; t < nthreads; ++t) pthread_join(th[t], NULL);
     return 0;
 }
+
+/* Quantisation to INT8 (Section 5c leaves "quantization support" to future work; the reading taken
+ * here is the usual symmetric one): q = the FP32 product x * inv_scale, rounded to the nearest
+ * integer with ties to even, saturated to [-128, 127]; NaN gives 0. */
+void nko_quantize_s8(const float* x, int64_t n, float inv_scale, int8_t* q) {
+    for (int64_t i = 0; i < n; ++i) {
+        volatile float p = x[i] * inv_scale;      /* one FP32 rounding, kept out of wider registers */
+        if (p != p) { q[i] = 0; continue; }
+        if (p >= 127.0f) { q[i] = 127; continue; }
+        if (p <= -128.0f) { q[i] = -128; continue; }
+        q[i] = (int8_t)lrintf(p);                 /* default rounding mode: to nearest, ties to even */
+    }
+}

@@ -531,3 +531,33 @@ def test_s8_generator_covers_the_range():
     assert v.dtype == np.int8 and v.min() == -128 and v.max() == 127
     assert abs(float(v.astype(np.float64).mean())) < 1.5
     assert np.array_equal(v[100:200], nk_inputs.fill(11, nk_inputs.TENSOR_A, 100, dtype="s8", start=100))
+
+
+def test_quantize_s8_ties_saturation_and_nan():
+    x = np.array([0.5, 1.5, 2.5, -0.5, -1.5, -2.5, 0.49999997, 126.5, 127.5, 1e9, -128.5, -129.0, -1e9,
+                  np.nan, 3.0, -0.0], dtype=np.float32)
+    want = np.array([0, 2, 2, 0, -2, -2, 0, 126, 127, 127, -128, -128, -128, 0, 3, 0], dtype=np.int8)
+    assert np.array_equal(oracle.quantize_s8(x, 1.0), want)
+    # a power-of-two step is exact: x / 2^-4 = 16 x
+    v = np.array([0.0625, 0.09375, -0.15625, 7.9375, 8.0], dtype=np.float32)       # 1, 1.5, -2.5, 127, 128 steps
+    assert np.array_equal(oracle.quantize_s8(v, 16.0), np.array([1, 2, -2, 127, 127], dtype=np.int8))
+    # against numpy's own float32 product and rint (round half to even), on random data
+    rng = np.random.default_rng(9)
+    r = (rng.standard_normal(4096) * 60).astype(np.float32)
+    inv = np.float32(1.0 / 0.37)
+    ref = np.clip(np.rint(r * inv), -128, 127).astype(np.int8)
+    assert np.array_equal(oracle.quantize_s8(r, inv), ref)
+
+
+def test_s8_scaled_layer_closed_forms():
+    rng = np.random.default_rng(10)
+    M, N, K = 8, 32, 64
+    A = rng.integers(-128, 128, (M, K), dtype=np.int8)
+    B = rng.integers(-128, 128, (K, N), dtype=np.int8)
+    acc = A.astype(np.int64) @ B.astype(np.int64)
+    y, s = oracle.gemm_s8_scaled(M, N, K, A, B, 0.5)
+    assert np.array_equal(y, 0.5 * acc) and np.array_equal(s, np.abs(0.5 * acc))
+    bias = -(0.25 * acc[0]).astype(np.float32)                # exact in FP32: |acc| < 2^21
+    y, s = oracle.gemm_s8_scaled(M, N, K, A, B, 0.25, bias=bias, relu=True)
+    assert np.all(y[0] == 0.0) and np.all(y >= 0.0)
+    assert np.array_equal(s[0], 2 * np.abs(0.25 * acc[0]))
