@@ -64,7 +64,9 @@ typedef enum {
                   four"): B[N/32][K/32][8][32][4], packed[k/4][n][k%4] = flat[k][n] inside each 32 x 32 block.
                   The result is exact: INT32 accumulation of at most 2^17 - 1 products.  No epilogue, no beta,
                   no batch, no K split; N and K multiples of 32 */
-    NK_S32 = 4 /* signed 32-bit integers: the type of C for NK_S8 operands (and only for them) */
+    NK_S32 = 4 /* signed 32-bit integers: the type of C for NK_S8 operands (and only for them).  NK_S8
+                  operands may also have an NK_F32 C: the INT32 sum is converted (round to nearest even),
+                  multiplied by desc.scale and given the epilogue (FP32 bias + ReLU) before the store */
 } nk_dtype_t;
 typedef enum { NK_ROW_MAJOR = 0, NK_BLOCKED32 = 1 } nk_layout_t;
 typedef enum { NK_EPI_NONE = 0, NK_EPI_BIAS_RELU = 1 } nk_epilogue_t;
@@ -121,6 +123,10 @@ typedef struct {
     int32_t layout_c;  /* nk_layout_t of C: NK_ROW_MAJOR, or NK_BLOCKED32 = C[M/32][N/32][32][32],
                           the layout a following layer reads as its blocked A (BF16 operands;
                           M and N multiples of 32)                                        */
+    float scale;       /* NK_S8 operands with an NK_F32 C (quantised layer, Section 5c's "Int8 ... along
+                          with quantization support"): C = scale * (A.B), then the epilogue, in FP32;
+                          scale is the product of the two operands' quantisation steps and must be
+                          finite and non-zero.  The bias of such a plan is FP32.  Ignored otherwise. */
 } nk_gemm_desc_t;
 
 /*
@@ -191,6 +197,16 @@ nk_status_t nk_gemm_run_host(nk_gemm_t plan, const void* hA, const void* hB, con
  * plans on that device.
  */
 nk_status_t nk_gemm_check(nk_gemm_t plan);
+
+/*
+ * Quantise FP32 values to INT8 for an NK_S8 operand (the quantisation step Section 5c leaves to
+ * future work): q[i] = saturate_to_[-128,127](round_to_nearest_even(x[i] * inv_scale)), the product
+ * taken in FP32; NaN gives 0.  x and q are device pointers on `device` (x 16-byte aligned when
+ * n >= 4), n elements each, they must not overlap; the kernel is enqueued on `cuda_stream` and the
+ * call returns without synchronising.  Row-major values in, the same order out: packing B into
+ * its blocked layout is the caller's business, like every other operand layout.
+ */
+nk_status_t nk_quantize_s8(const float* x, int8_t* q, size_t n, float inv_scale, int device, void* cuda_stream);
 
 /*
  * nk_gemm_run for callers that cannot allocate device memory.  (The paper has

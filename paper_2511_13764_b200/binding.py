@@ -57,7 +57,7 @@ class Desc(ctypes.Structure):
                 ("epilogue", ctypes.c_int32), ("device", ctypes.c_int32),
                 ("flags", ctypes.c_uint32), ("beta", ctypes.c_int32), ("batch", ctypes.c_int64),
                 ("stride_a", ctypes.c_int64), ("stride_b", ctypes.c_int64), ("stride_c", ctypes.c_int64),
-                ("batch_independent", ctypes.c_int32), ("layout_c", ctypes.c_int32)]
+                ("batch_independent", ctypes.c_int32), ("layout_c", ctypes.c_int32), ("scale", ctypes.c_float)]
 
 
 _lib = None
@@ -100,6 +100,8 @@ def lib():
         L.nk_gemm_launches_per_run.argtypes = [vp]
         L.nk_gemm_last_cuda_error.restype = ctypes.c_char_p
         L.nk_gemm_last_cuda_error.argtypes = [vp]
+        L.nk_quantize_s8.restype = ctypes.c_int
+        L.nk_quantize_s8.argtypes = [vp, vp, sz, ctypes.c_float, ctypes.c_int, vp]
         _lib = L
     return _lib
 
@@ -135,9 +137,9 @@ class Plan:
     def __init__(self, M, N, K, in_dtype=BF16, out_dtype=F32, layout_a=ROW_MAJOR,
                  layout_b=ROW_MAJOR, epilogue=EPI_NONE, device=0, flags=0, beta=0, batch=0,
                  stride_a=0, stride_b=0, stride_c=0, batch_independent=0,
-                 layout_c=ROW_MAJOR):
+                 layout_c=ROW_MAJOR, scale=0.0):
         self.desc = Desc(M, N, K, in_dtype, out_dtype, layout_a, layout_b, epilogue, device, flags,
-                         beta, batch, stride_a, stride_b, stride_c, batch_independent, layout_c)
+                         beta, batch, stride_a, stride_b, stride_c, batch_independent, layout_c, scale)
         self._h = ctypes.c_void_p()
         _check(lib().nk_gemm_create(ctypes.byref(self.desc), ctypes.byref(self._h)))
 
@@ -188,6 +190,11 @@ class Plan:
             self.destroy()
         except Exception:
             pass
+
+
+def quantize_s8(x, q, n, inv_scale, device=0, stream=None):
+    """nk_quantize_s8: FP32 device values -> INT8 (round half to even of x * inv_scale, saturating)."""
+    _check(lib().nk_quantize_s8(_ptr(x), _ptr(q), n, inv_scale, device, stream))
 
 
 def plan_for(w, device=0, flags=0) -> Plan:

@@ -261,6 +261,25 @@ __global__ void unpack_vnni_b_kernel(const uint32_t* __restrict__ Bblk, uint16_t
     }
 }
 
+// FP32 -> INT8: q = saturate(round-to-nearest-even(x * inv_scale)), the product in FP32 (one
+// multiplication: nothing for the compiler to contract); NaN converts to 0.  Four elements per thread.
+__global__ void quantize_s8_kernel(const float* __restrict__ x, int8_t* __restrict__ q, size_t n, float inv_scale) {
+    const size_t i = (static_cast<size_t>(blockIdx.x) * blockDim.x + threadIdx.x) * 4;
+    if (i >= n) return;
+    auto one = [&](float v) { return static_cast<uint32_t>(max(-128, min(127, __float2int_rn(v * inv_scale))) & 0xFF); };
+    if (i + 4 <= n) {
+        const float4 v = __ldcs(reinterpret_cast<const float4*>(x + i));
+        const uint32_t w = one(v.x) | (one(v.y) << 8) | (one(v.z) << 16) | (one(v.w) << 24);
+        if ((reinterpret_cast<uintptr_t>(q + i) & 3u) == 0) {
+            *reinterpret_cast<uint32_t*>(q + i) = w;
+        } else {
+            for (int j = 0; j < 4; ++j) q[i + j] = static_cast<int8_t>((w >> (8 * j)) & 0xFF);
+        }
+    } else {
+        for (size_t j = i; j < n; ++j) q[j] = static_cast<int8_t>(one(x[j]));
+    }
+}
+
 // Self-test of the bounded-wait path: one warp waits on an mbarrier that nothing ever
 // arrives on, with a short limit; the wait gives up, the kernel records the code in the
 // status word and returns normally (no trap, no fault, the context stays usable).

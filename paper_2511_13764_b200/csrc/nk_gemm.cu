@@ -8,6 +8,7 @@
 
 #include <cstdio>
 #include <cstdlib>
+#include <cmath>
 #include <cstring>
 #include <mutex>
 #include <new>
@@ -668,11 +669,15 @@ nk_status_t nk_gemm_create(const nk_gemm_desc_t* desc, nk_gemm_t* out) {
     if (d.M * d.N >= (1ll << 31) || d.M * d.K >= (1ll << 33) || d.K * d.N >= (1ll << 33)) return NK_ERR_UNSUPPORTED;
     if (d.in_dtype != NK_F32 && !is16(d.in_dtype) && d.in_dtype != NK_S8) return NK_ERR_INVALID_ARG;
     if (d.out_dtype != NK_F32 && !is16(d.out_dtype) && d.out_dtype != NK_S32) return NK_ERR_INVALID_ARG;
-    if ((d.in_dtype == NK_S8) != (d.out_dtype == NK_S32)) return NK_ERR_INVALID_ARG;   // INT8 operands <-> INT32 result
+    if (d.out_dtype == NK_S32 && d.in_dtype != NK_S8) return NK_ERR_INVALID_ARG;   // an INT32 C belongs to INT8 operands
     if (d.in_dtype == NK_S8) {
-        // the Int8 dot product: A row-major, B packed in groups of four inside 32 x 32 blocks, exact INT32 C
+        // the Int8 dot product: A row-major, B packed in groups of four inside 32 x 32 blocks; C is the exact
+        // INT32 sum, or FP32 = scale * sum with the epilogue (quantised layer)
+        if (d.out_dtype != NK_S32 && d.out_dtype != NK_F32) return NK_ERR_INVALID_ARG;
         if (d.layout_a != NK_ROW_MAJOR || d.layout_b != NK_BLOCKED32 || d.layout_c != NK_ROW_MAJOR) return NK_ERR_UNSUPPORTED;
-        if (d.epilogue != NK_EPI_NONE || d.beta != 0 || d.batch > 1) return NK_ERR_UNSUPPORTED;
+        if (d.beta != 0 || d.batch > 1) return NK_ERR_UNSUPPORTED;
+        if (d.out_dtype == NK_S32 && d.epilogue != NK_EPI_NONE) return NK_ERR_UNSUPPORTED;
+        if (d.out_dtype == NK_F32 && !(std::isfinite(d.scale) && d.scale != 0.0f)) return NK_ERR_INVALID_ARG;
         if (d.flags & (NK_FLAG_REPACK_B | NK_FLAG_SEPARATE_REDUCE)) return NK_ERR_UNSUPPORTED;
         const uint32_t fk = d.flags & NK_FLAG_KERNEL_MASK;
         if (fk == NK_FLAG_KERNEL_NAIVE || fk == NK_FLAG_KERNEL_SIMT) return NK_ERR_UNSUPPORTED;
@@ -899,7 +904,7 @@ nk_status_t nk_gemm_create(const nk_gemm_desc_t* desc, nk_gemm_t* out) {
     }
     if (d.in_dtype == NK_S8) {
         const size_t len = strlen(p->name);
-        snprintf(p->name + len, sizeof(p->name) - len, "_s8");
+        snprintf(p->name + len, sizeof(p->name) - len, d.out_dtype == NK_F32 ? "_s8_dequant" : "_s8");
     }
     // split-K partials are laid out [split][gemm][M][N] and reduced as one flat array: that
     // needs the C of a batched matmul to be contiguous
@@ -1029,7 +1034,9 @@ nk_status_t nk_gemm_run(nk_gemm_t p, const void* A, const void* B, const void* b
         up.C = C;
         up.partial = partial;
         up.status = p->status_dev;
-        up.bias_f32 = p->bias_f32 ? 1 : 0;
+        up.bias_f32 = (p->bias_f32 || is_s8(d)) ? 1 : 0;
+        up.dequant = (is_s8(d) && d.out_dtype == NK_F32) ? 1 : 0;
+        up.scale = d.scale;
         up.item_remap = p->item_remap ? 1 : 0;
         up.item_map_a = p->item_map_a;
         up.item_map_b = p->item_map_b;
@@ -1288,6 +1295,20 @@ nk_status_t nk_gemm_selftest_timeout(nk_gemm_t p, void* cuda_stream) {
     cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess) { set_err(p, "probe launch", e); return NK_ERR_CUDA; }
     return NK_OK;
+}
+
+nk_status_t nk_quantize_s8(const float* x, int8_t* q, size_t n, float inv_scale, int device, void* cuda_stream) {
+    if (!x || !q) return NK_ERR_INVALID_ARG;
+    if (n == 0) return NK_OK;
+    if (n >= 4 && (reinterpret_cast<uintptr_t>(x) & 15u)) return NK_ERR_MISALIGNED;
+    int ndev = 0;
+    if (cudaGetDeviceCount(&ndev) != cudaSuccess || device < 0 || device >= ndev) { cudaGetLastError(); return NK_ERR_DEVICE; }
+    DeviceGuard guard(device);
+    if (guard.err != cudaSuccess) return NK_ERR_DEVICE;
+    const size_t blocks = (n / 4 + 1 + 255) / 256;
+    if (blocks > 0x7FFFFFFFull) return NK_ERR_UNSUPPORTED;
+    quantize_s8_kernel<<<static_cast<unsigned>(blocks), 256, 0, static_cast<cudaStream_t>(cuda_stream)>>>(x, q, n, inv_scale);
+    return cudaGetLastError() == cudaSuccess ? NK_OK : NK_ERR_CUDA;
 }
 
 nk_status_t nk_gemm_destroy(nk_gemm_t p) {

@@ -66,7 +66,9 @@ struct UmmaParams {
     float* partial;     // [splits][M][N] when splits > 1; [tail tile][tail split][tile rows][BN] in tail mode
     int tail_from;      // tail mode (pair kernel): units >= tail_from are K splits of the last, partial wave's tiles; else -1
     int tail_splits;    // K splits of each tail tile
-    int bias_f32;       // the bias vector is FP32 although the operands are 16-bit (split-FP32 plans)
+    int bias_f32;       // the bias vector is FP32 although the operands are not (split-FP32 and quantised plans)
+    int dequant;        // the accumulator holds INT32 sums: convert to FP32 and multiply by `scale` before the epilogue
+    float scale;
     int item_remap;     // batch item i multiplies A item (item_map_a >> 4i) & 15 by B item (item_map_b >> 4i) & 15
     uint32_t item_map_a, item_map_b;
     unsigned int* status;
@@ -151,6 +153,10 @@ __device__ __forceinline__ void umma_store_chunk(const UmmaParams& p, const CUte
     if (empty_k) {
 #pragma unroll
         for (int i = 0; i < 32; ++i) v[i] = 0u;
+    }
+    if (p.dequant) {
+#pragma unroll
+        for (int i = 0; i < 32; ++i) v[i] = __float_as_uint(__int2float_rn(static_cast<int>(v[i])) * p.scale);
     }
     if (!to_partial && p.beta && row < p.M) {
         // beta = 1: the accumulation tile starts from the stored C (Algorithm 1 loads the C

@@ -88,10 +88,77 @@ def test_s8_headline_shapes(i):
     assert np.array_equal(lhs, rhs)
 
 
+# ---------------------------------------------------------------- quantised layer: C = scale * (A.B) (+ FP32 bias, ReLU) in FP32
+DEQ_TOL = 2.0 ** -22    # int -> FP32, the scaling and the bias add each round once (2^-24 relative each)
+
+
+@pytest.mark.parametrize("mode,tile", [("single", 2), ("single", 4), ("pair", 3), ("pair", 4), ("auto", 0)])
+@pytest.mark.parametrize("epi", ["none", "bias_relu"])
+@pytest.mark.parametrize("shape", [(130, 160, 416), (512, 1024, 2048)])
+def test_s8_dequantised_output(shape, epi, mode, tile):
+    M, N, K = shape
+    seed = 5
+    A = nk_inputs.fill(seed, nk_inputs.TENSOR_A, M * K, dtype="s8")
+    B = nk_inputs.fill(seed, nk_inputs.TENSOR_B, K * N, dtype="s8")
+    bias = nk_inputs.fill(seed, nk_inputs.TENSOR_BIAS, N, "normal", 50.0, "f32") if epi != "none" else None
+    scale = 0.0123 * 0.0071
+    plan = nk.Plan(M, N, K, in_dtype=nk.S8, out_dtype=nk.F32, layout_a=nk.ROW_MAJOR, layout_b=nk.BLOCKED32,
+                   epilogue=nk.EPI_BIAS_RELU if bias is not None else nk.EPI_NONE, scale=scale,
+                   flags=MODES[mode] | (nk.flag_tile_n(tile) if tile else 0))
+    assert plan.kernel_name.endswith("_s8_dequant")
+    C = torch.full((M * N,), float("nan"), dtype=torch.float32, device="cuda")
+    plan.run(torch.from_numpy(A).cuda(), torch.from_numpy(B).cuda(), C,
+             bias=torch.from_numpy(bias).cuda() if bias is not None else None,
+             stream=torch.cuda.current_stream().cuda_stream)
+    plan.check()
+    got = C.cpu().numpy().astype(np.float64).reshape(M, N)
+    want, S = oracle.gemm_s8_scaled(M, N, K, A, B, scale, bias=bias, layout_b=oracle.BLOCKED32, relu=bias is not None)
+    assert not np.isnan(got).any()
+    bad = np.abs(got - want) > DEQ_TOL * S
+    assert not bad.any(), f"{bad.sum()} of {bad.size} out of tolerance; first at {np.argwhere(bad)[:4].tolist()}"
+    if bias is not None:
+        assert (got == 0).any() and (got > 0).any()      # the ReLU is active on part of the output
+
+
+@pytest.mark.parametrize("n", [1, 3, 4, 7, 1024, 1 << 20, (1 << 20) + 5])
+def test_quantize_s8_is_bit_exact(n):
+    rng = np.random.default_rng(n)
+    x = (rng.standard_normal(n) * 40).astype(np.float32)
+    x[: min(n, 8)] = np.array([0.5, 1.5, 2.5, -0.5, 1e9, -1e9, np.nan, -2.5], dtype=np.float32)[: min(n, 8)]
+    inv = float(np.float32(1.0 / 0.37))
+    dx = torch.from_numpy(x).cuda()
+    dq = torch.full((n + 16,), 77, dtype=torch.int8, device="cuda")
+    nk.quantize_s8(dx, dq[8:], n, inv, stream=torch.cuda.current_stream().cuda_stream)
+    torch.cuda.synchronize()
+    q = dq.cpu().numpy()
+    assert np.all(q[:8] == 77) and np.all(q[8 + n:] == 77)
+    assert np.array_equal(q[8:8 + n], oracle.quantize_s8(x, inv))
+
+
+def test_quantised_layer_end_to_end():
+    """FP32 activations -> nk_quantize_s8 -> INT8 GEMM with dequantising epilogue, against the oracle fed
+    with the oracle's own quantisation of the same activations."""
+    M, N, K = 256, 512, 1024
+    x = nk_inputs.fill(6, nk_inputs.TENSOR_A, M * K, "normal", 1.0, "f32")
+    sx, sw = 4.0 / 127, 0.02
+    W8 = nk_inputs.fill(6, nk_inputs.TENSOR_B, K * N, dtype="s8")
+    dq = torch.empty(M * K, dtype=torch.int8, device="cuda")
+    nk.quantize_s8(torch.from_numpy(x).cuda(), dq, M * K, 1.0 / sx, stream=torch.cuda.current_stream().cuda_stream)
+    plan = nk.Plan(M, N, K, in_dtype=nk.S8, out_dtype=nk.F32, layout_a=nk.ROW_MAJOR, layout_b=nk.BLOCKED32, scale=sx * sw)
+    C = torch.empty(M * N, dtype=torch.float32, device="cuda")
+    plan.run(dq, torch.from_numpy(W8).cuda(), C, stream=torch.cuda.current_stream().cuda_stream)
+    plan.check()
+    xq = oracle.quantize_s8(x, 1.0 / sx)
+    assert np.array_equal(dq.cpu().numpy(), xq)
+    want, S = oracle.gemm_s8_scaled(M, N, K, xq, W8, sx * sw, layout_b=oracle.BLOCKED32)
+    got = C.cpu().numpy().astype(np.float64).reshape(M, N)
+    assert np.all(np.abs(got - want) <= DEQ_TOL * S)
+
+
 def test_s8_rejects_what_it_cannot_do():
     ok = dict(in_dtype=nk.S8, out_dtype=nk.S32, layout_a=nk.ROW_MAJOR, layout_b=nk.BLOCKED32)
     nk.Plan(64, 64, 64, **ok)
-    for bad in (dict(ok, out_dtype=nk.F32), dict(ok, layout_b=nk.ROW_MAJOR), dict(ok, layout_a=nk.BLOCKED32),
+    for bad in (dict(ok, out_dtype=nk.BF16), dict(ok, out_dtype=nk.F32, scale=0.0), dict(ok, layout_b=nk.ROW_MAJOR), dict(ok, layout_a=nk.BLOCKED32),
                 dict(ok, epilogue=nk.EPI_BIAS_RELU), dict(ok, beta=1), dict(ok, batch=2),
                 dict(ok, flags=nk.FLAG_KERNEL_NAIVE), dict(ok, flags=nk.FLAG_REPACK_B)):
         with pytest.raises(nk.NkError):
