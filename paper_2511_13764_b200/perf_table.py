@@ -46,7 +46,7 @@ def time_launch(launch, st, iters, flush, graph_pairs):
     if graph_pairs and flush is not None:
         side = torch.cuda.Stream()
         side.wait_stream(st)
-        mids = []
+        graphs = []
         for with_launch in (True, False):
             g = torch.cuda.CUDAGraph()
             with torch.cuda.graph(g, stream=side):
@@ -55,18 +55,23 @@ def time_launch(launch, st, iters, flush, graph_pairs):
                     flush.fill_(1)
                     if with_launch:
                         launch(cs)
-            ts = []
-            for _ in range(max(3, iters // 3)):
-                a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-                a.record(st)
-                g.replay()
-                b.record(st)
-                b.synchronize()
-                ts.append(a.elapsed_time(b))
-            ts.sort()
-            mids.append(ts[len(ts) // 2])
-        per = (mids[0] - mids[1]) / graph_pairs
-        return per, per
+            graphs.append(g)
+
+        def replay_ms(g):
+            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a.record(st)
+            g.replay()
+            b.record(st)
+            b.synchronize()
+            return a.elapsed_time(b)
+
+        # The two graphs are timed in turn, so that a drift of the clocks (the previous row may have
+        # left the part power-throttled) hits both alike; the median of the differences is reported.
+        for g in graphs:
+            replay_ms(g)
+        diffs = sorted(replay_ms(graphs[0]) - replay_ms(graphs[1]) for _ in range(max(5, iters // 2)))
+        per = diffs[len(diffs) // 2] / graph_pairs
+        return per, diffs[0] / graph_pairs
     times = []
     for _ in range(iters):
         if flush is not None:
