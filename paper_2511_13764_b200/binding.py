@@ -25,7 +25,7 @@ FLAG_F32_TENSOR = 0x800000
 EXPORTS = ["nk_gemm_create", "nk_gemm_workspace_bytes", "nk_gemm_run", "nk_gemm_run_host",
            "nk_gemm_check", "nk_gemm_destroy", "nk_status_str", "nk_gemm_kernel_name",
            "nk_gemm_launches_per_run", "nk_gemm_last_cuda_error", "nk_gemm_run_static",
-           "nk_gemm_selftest_timeout"]
+           "nk_gemm_selftest_timeout", "nk_quantize_s8"]
 
 STATIC_SCRATCH_BYTES = 16 << 20
 
