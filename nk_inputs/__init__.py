@@ -84,6 +84,23 @@ def _normal_f32(seed, tensor_id, start, count, sigma):
     return (z * sigma).astype(np.float32)
 
 
+def f32_to_fp8_bits(v: np.ndarray, fmt: str) -> np.ndarray:
+    """FP32 -> 8-bit floating point ("e4m3": 4 exponent bits, bias 7, 3 fraction bits, largest finite
+    value 448; "e5m2": 5 exponent bits, bias 15, 2 fraction bits, largest finite value 57344), round to
+    nearest, ties to even, gradual underflow, finite inputs; magnitudes beyond the largest finite value
+    saturate to it."""
+    man, bias, emin, top = (3, 7, -6, 448.0) if fmt == "e4m3" else (2, 15, -14, 57344.0)
+    x = np.minimum(np.abs(v.astype(np.float64)), top)
+    _, E = np.frexp(x)                              # x = m * 2^E, m in [0.5, 1)
+    e = np.maximum(E - 1, emin)                     # exponent of the binade (subnormals share emin)
+    q = np.rint(x / np.exp2((e - man).astype(np.float64))).astype(np.int64)   # significand in units of 2^(e - man): ties to even
+    # q may reach 2^(man+1) (carry into the next binade): the bit arithmetic below absorbs it
+    bits = ((e - emin) << man) + q                  # subnormals: exponent field 0, q < 2^man; normals: field (e - emin + 1), q - 2^man
+    bits = np.where(x == 0, 0, bits)
+    sign = (np.signbit(v)).astype(np.int64) << 7
+    return (bits | sign).astype(np.uint8)
+
+
 def fill(seed: int, tensor_id: int, count: int, dist: str = "uniform",
          sigma: float = 1.0, dtype: str = "f32", start: int = 0) -> np.ndarray:
     """1-D storage-order buffer of ``count`` entries (storage indices start .. start+count-1).
@@ -91,7 +108,7 @@ def fill(seed: int, tensor_id: int, count: int, dist: str = "uniform",
     dist: "uniform" (U[-1,1) on the 2**-23 grid), "normal" (N(0, sigma**2)),
           "int" (integers in [-4, 4], exact in every precision used here).
     dtype: "f32" -> float32 array; "bf16" / "f16" -> uint16 bit patterns; "s8" -> int8, uniform over
-           all 256 values.
+           all 256 values; "e4m3" / "e5m2" -> uint8 bit patterns of the 8-bit floating-point formats.
     """
     if dtype == "s8":
         # INT8 operands: the full range [-128, 127], uniformly, whatever `dist` says
@@ -101,7 +118,7 @@ def fill(seed: int, tensor_id: int, count: int, dist: str = "uniform",
             out[s:s + n] = ((raw_bits(seed, tensor_id, start + s, n) >> np.uint64(40)) & np.uint64(0xFF)
                             ).astype(np.uint8).view(np.int8)
         return out
-    out = np.empty(count, dtype=np.float32 if dtype == "f32" else np.uint16)
+    out = np.empty(count, dtype=np.float32 if dtype == "f32" else np.uint8 if dtype in ("e4m3", "e5m2") else np.uint16)
     for s in range(0, count, _CHUNK):
         n = min(_CHUNK, count - s)
         if dist == "uniform":
@@ -113,7 +130,8 @@ def fill(seed: int, tensor_id: int, count: int, dist: str = "uniform",
                  ).astype(np.float32) - 4.0
         else:
             raise ValueError(dist)
-        out[s:s + n] = v if dtype == "f32" else (f32_to_f16_bits(v) if dtype == "f16" else f32_to_bf16_bits(v))
+        out[s:s + n] = (v if dtype == "f32" else f32_to_f16_bits(v) if dtype == "f16"
+                        else f32_to_fp8_bits(v, dtype) if dtype in ("e4m3", "e5m2") else f32_to_bf16_bits(v))
     return out
 
 
@@ -159,11 +177,11 @@ class Workload:
 
     @property
     def algorithmic_bytes(self) -> int:
-        e_in = 4 if self.in_dtype == "f32" else 1 if self.in_dtype == "s8" else 2
+        e_in = 4 if self.in_dtype == "f32" else 1 if self.in_dtype in ("s8", "e4m3", "e5m2") else 2
         e_out = 4 if self.out_dtype in ("f32", "s32") else 2
         b = e_in * (self.M * self.K + self.K * self.N) + e_out * self.M * self.N
         if self.epilogue != "none":
-            b += e_in * self.N
+            b += (4 if self.in_dtype in ("e4m3", "e5m2") else e_in) * self.N
         return b
 
     def make(self):
@@ -174,8 +192,13 @@ class Workload:
         B = fill(self.seed, TENSOR_B, self.K * self.N, self.dist_b[0], self.dist_b[1], self.in_dtype)
         bias = None
         if self.epilogue != "none":
-            bias = fill(self.seed, TENSOR_BIAS, self.N, self.dist_bias[0], self.dist_bias[1], self.in_dtype)
+            bias = fill(self.seed, TENSOR_BIAS, self.N, self.dist_bias[0], self.dist_bias[1], self.bias_dtype)
         return A, B, bias
+
+    @property
+    def bias_dtype(self) -> str:
+        """The bias has the operands' type, except with 8-bit floating-point operands (FP32 bias)."""
+        return "f32" if self.in_dtype in ("e4m3", "e5m2") else self.in_dtype
 
 
 def config(i: int) -> Workload:
@@ -227,6 +250,18 @@ def s8_set() -> list:
         Workload("x_s8_8192", 8192, 8192, 8192, "s8", "s32", layout="b_blocked32", seed=8017),
         Workload("x_s8_4096", 4096, 4096, 4096, "s8", "s32", layout="b_blocked32", seed=8018),
         Workload("x_s8_512x4096x4096", 512, 4096, 4096, "s8", "s32", layout="b_blocked32", seed=8019),
+    ]
+
+
+def fp8_set() -> list:
+    """8-bit floating-point operands (E4M3 / E5M2; the 8-bit floating-point counterpart, on B200, of the
+    packed types Section 5 lists), B packed in groups of four inside 32 x 32 blocks, FP32 accumulation
+    and output: the large square GEMM, a mid-size E5M2 one and the 4096-wide MLP layer with FP32 bias."""
+    return [
+        Workload("x_e4m3_8192", 8192, 8192, 8192, "e4m3", "f32", layout="b_blocked32", seed=9017),
+        Workload("x_e5m2_4096", 4096, 4096, 4096, "e5m2", "f32", layout="b_blocked32", seed=9018),
+        Workload("x_e4m3_mlp_512x4096x4096", 512, 4096, 4096, "e4m3", "f32", layout="b_blocked32", epilogue="bias_relu",
+                 dist_a=("normal", 1.0), dist_b=("normal", 0.02), seed=9019),
     ]
 
 

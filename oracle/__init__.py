@@ -18,6 +18,7 @@ _SRC = os.path.join(_HERE, "nk_oracle.c")
 _LIB = os.path.join(_HERE, "libnk_oracle.so")
 
 F32, BF16, F16 = 0, 1, 2
+E4M3, E5M2 = 5, 6
 ROW, BLOCKED32 = 0, 1
 EPI_NONE, EPI_BIAS_RELU = 0, 1
 ACC_F64, ACC_F32_SEQ = 0, 1
@@ -51,6 +52,9 @@ def lib():
         L.nko_bf16_to_f32.argtypes = [ctypes.c_uint16]
         L.nko_f16_to_f32.restype = ctypes.c_float
         L.nko_f16_to_f32.argtypes = [ctypes.c_uint16]
+        for f in (L.nko_e4m3_to_f32, L.nko_e5m2_to_f32):
+            f.restype = ctypes.c_float
+            f.argtypes = [ctypes.c_uint8]
         L.nko_f32_to_bf16_rne.restype = ctypes.c_uint16
         L.nko_f32_to_bf16_rne.argtypes = [ctypes.c_float]
         for f in (L.nko_pack_vnni2, L.nko_unpack_vnni2):
@@ -171,7 +175,16 @@ def unpack_vnni2(packed: np.ndarray) -> np.ndarray:
 
 
 def _np_dtype(in_dtype):
-    return np.float32 if in_dtype == F32 else np.uint16
+    return np.float32 if in_dtype == F32 else np.uint8 if in_dtype in (E4M3, E5M2) else np.uint16
+
+
+def fp8_to_f32(bits: np.ndarray, fmt: int) -> np.ndarray:
+    """Decode uint8 E4M3 / E5M2 patterns element by element through the C routines."""
+    L = lib()
+    f = L.nko_e4m3_to_f32 if fmt == E4M3 else L.nko_e5m2_to_f32
+    flat = np.ascontiguousarray(bits, dtype=np.uint8).ravel()
+    out = np.fromiter((f(int(h)) for h in flat), dtype=np.float32, count=flat.size)
+    return out.reshape(np.shape(bits))
 
 
 def to_blocked(flat_a: np.ndarray, flat_b: np.ndarray, in_dtype: int):
@@ -206,7 +219,7 @@ def gemm(M, N, K, A, B, bias=None, *, in_dtype=F32, layout_a=ROW, layout_b=ROW,
     assert A.size == M * K and B.size == K * N, "operand size mismatch"
     bp = None
     if bias is not None:
-        bias = np.ascontiguousarray(bias, dtype=dt)
+        bias = np.ascontiguousarray(bias, dtype=np.float32 if in_dtype in (E4M3, E5M2) else dt)
         assert bias.size == N
         bp = bias.ctypes.data
     rp, nrows = None, M
@@ -234,10 +247,11 @@ def gemm(M, N, K, A, B, bias=None, *, in_dtype=F32, layout_a=ROW, layout_b=ROW,
 def gemm_workload(w, A, B, bias, rows=None, cols=None, **kw):
     """Oracle on an ``nk_inputs.Workload``-shaped object (duck-typed: M, N, K,
     in_dtype, layout, epilogue attributes)."""
-    lay = BLOCKED32 if w.layout == "blocked32" else ROW
+    lay_a = BLOCKED32 if w.layout == "blocked32" else ROW
+    lay_b = BLOCKED32 if w.layout in ("blocked32", "b_blocked32") else ROW
     return gemm(w.M, w.N, w.K, A, B, bias,
-                in_dtype={"f32": F32, "bf16": BF16, "f16": F16}[w.in_dtype],
-                layout_a=lay, layout_b=lay,
+                in_dtype={"f32": F32, "bf16": BF16, "f16": F16, "e4m3": E4M3, "e5m2": E5M2}[w.in_dtype],
+                layout_a=lay_a, layout_b=lay_b,
                 epilogue=EPI_BIAS_RELU if w.epilogue == "bias_relu" else EPI_NONE,
                 rows=rows, cols=cols, **kw)
 

@@ -41,14 +41,15 @@
 #include <stdlib.h>
 #include <string.h>
 
-enum { NKO_F32 = 0, NKO_BF16 = 1, NKO_F16 = 2 };
+enum { NKO_F32 = 0, NKO_BF16 = 1, NKO_F16 = 2, NKO_E4M3 = 5, NKO_E5M2 = 6 };
 enum { NKO_ROW = 0, NKO_BLOCKED32 = 1 };
 enum { NKO_EPI_NONE = 0, NKO_EPI_BIAS_RELU = 1 };
 enum { NKO_ACC_F64 = 0, NKO_ACC_F32_SEQ = 1 };
 
 typedef struct {
     int64_t M, N, K;
-    int32_t in_dtype;   /* NKO_F32 | NKO_BF16 | NKO_F16: element type of A, B and bias */
+    int32_t in_dtype;   /* NKO_F32 | NKO_BF16 | NKO_F16: element type of A, B and bias;
+                           NKO_E4M3 | NKO_E5M2: 8-bit floating-point A and B, FP32 bias */
     int32_t layout_a;   /* NKO_ROW | NKO_BLOCKED32 */
     int32_t layout_b;
     int32_t epilogue;
@@ -73,6 +74,31 @@ float nko_f16_to_f32(uint16_t h) {
     if (e == 0) v = ldexp((double)m, -24);
     else if (e == 31) v = m ? NAN : INFINITY;
     else v = ldexp(1.0 + (double)m / 1024.0, e - 15);
+    return (float)(sign ? -v : v);
+}
+
+/* The two 8-bit floating-point formats of the OCP FP8 specification, written from their
+   definitions; every value is exactly representable in FP32.
+   E4M3: 1 sign bit, 4 exponent bits (bias 7), 3 fraction bits; exponent 0 is zero or a subnormal
+   (fraction * 2^-9); there are no infinities, and only exponent 15 with fraction 7 is NaN, so the
+   largest finite value is 1.75 * 2^8 = 448.
+   E5M2: 1 sign bit, 5 exponent bits (bias 15), 2 fraction bits, IEEE rules: exponent 0 is zero or
+   a subnormal (fraction * 2^-16), exponent 31 is infinity (fraction 0) or NaN. */
+float nko_e4m3_to_f32(uint8_t h) {
+    int sign = (h >> 7) & 1, e = (h >> 3) & 0xF, m = h & 7;
+    double v;
+    if (e == 0) v = ldexp((double)m, -9);
+    else if (e == 15 && m == 7) v = NAN;
+    else v = ldexp(1.0 + (double)m / 8.0, e - 7);
+    return (float)(sign ? -v : v);
+}
+
+float nko_e5m2_to_f32(uint8_t h) {
+    int sign = (h >> 7) & 1, e = (h >> 2) & 0x1F, m = h & 3;
+    double v;
+    if (e == 0) v = ldexp((double)m, -16);
+    else if (e == 31) v = m ? NAN : INFINITY;
+    else v = ldexp(1.0 + (double)m / 4.0, e - 15);
     return (float)(sign ? -v : v);
 }
 
@@ -103,8 +129,12 @@ static int64_t a_index(const nko_desc_t* d, int64_t i, int64_t k) {
     return (((i / 32) * (d->K / 32) + k / 32) * 32 + i % 32) * 32 + k % 32;
 }
 
+static int is_8bit(int32_t dtype) { return dtype == NKO_E4M3 || dtype == NKO_E5M2; }
+
 static int64_t b_index(const nko_desc_t* d, int64_t k, int64_t j) {
     if (d->layout_b == NKO_ROW) return k * d->N + j;
+    if (is_8bit(d->in_dtype))   /* 8-bit elements are packed in groups of four (Section 2) */
+        return ((((j / 32) * (d->K / 32) + k / 32) * 8 + (k % 32) / 4) * 32 + j % 32) * 4 + k % 4;
     return ((((j / 32) * (d->K / 32) + k / 32) * 16 + (k % 32) / 2) * 32 + j % 32) * 2 + k % 2;
 }
 
@@ -115,6 +145,8 @@ int64_t nko_b_index(const nko_desc_t* d, int64_t k, int64_t j) { return b_index(
 static double load(const void* p, int32_t dtype, int64_t idx) {
     if (dtype == NKO_F32) return (double)((const float*)p)[idx];
     if (dtype == NKO_F16) return (double)nko_f16_to_f32(((const uint16_t*)p)[idx]);
+    if (dtype == NKO_E4M3) return (double)nko_e4m3_to_f32(((const uint8_t*)p)[idx]);
+    if (dtype == NKO_E5M2) return (double)nko_e5m2_to_f32(((const uint8_t*)p)[idx]);
     return (double)nko_bf16_to_f32(((const uint16_t*)p)[idx]);
 }
 
@@ -154,7 +186,7 @@ static void* worker(void* arg) {
         if (d->epilogue == NKO_EPI_BIAS_RELU) {
             for (int64_t c = 0; c < nc; ++c) {
                 int64_t j = w->cols ? w->cols[c] : c;
-                double b = load(w->bias, d->in_dtype, j);
+                double b = load(w->bias, is_8bit(d->in_dtype) ? NKO_F32 : d->in_dtype, j);
                 double v = y[c] + b;
                 y[c] = v > 0.0 ? v : 0.0;
                 if (s) s[c] += fabs(b);

@@ -561,3 +561,73 @@ def test_s8_scaled_layer_closed_forms():
     y, s = oracle.gemm_s8_scaled(M, N, K, A, B, 0.25, bias=bias, relu=True)
     assert np.all(y[0] == 0.0) and np.all(y >= 0.0)
     assert np.array_equal(s[0], 2 * np.abs(0.25 * acc[0]))
+
+
+# ---------------------------------------------------------------- 8-bit floating point (E4M3, E5M2)
+def test_fp8_decode_exhaustive_against_the_format_and_a_library():
+    import torch
+    bits = np.arange(256, dtype=np.uint8)
+    sign = np.where(bits >> 7, -1.0, 1.0)
+    # E4M3: bias 7, 3 fraction bits, no infinities, NaN only at exponent 15 / fraction 7
+    e, m = ((bits >> 3) & 0xF).astype(np.int64), (bits & 7).astype(np.float64)
+    want = np.where(e == 0, sign * m * 2.0 ** -9, sign * (1 + m / 8) * 2.0 ** (e - 7))
+    got = oracle.fp8_to_f32(bits, oracle.E4M3).astype(np.float64)
+    nan = (e == 15) & (m == 7)
+    assert np.all(np.isnan(got[nan])) and np.array_equal(got[~nan], want[~nan])
+    lib8 = torch.from_numpy(bits).view(torch.float8_e4m3fn).to(torch.float32).numpy().astype(np.float64)
+    assert np.array_equal(got[~nan], lib8[~nan])
+    assert got[0x38] == 1.0 and got[0x7E] == 448.0 and got[0x01] == 2.0 ** -9 and got[0xC0] == -2.0
+    # E5M2: bias 15, 2 fraction bits, IEEE infinities and NaNs
+    e, m = ((bits >> 2) & 0x1F).astype(np.int64), (bits & 3).astype(np.float64)
+    want = np.where(e == 0, sign * m * 2.0 ** -16, sign * (1 + m / 4) * 2.0 ** (e - 15))
+    got = oracle.fp8_to_f32(bits, oracle.E5M2).astype(np.float64)
+    fin = e != 31
+    assert np.array_equal(got[fin], want[fin])
+    assert np.isposinf(got[0x7C]) and np.isneginf(got[0xFC]) and np.all(np.isnan(got[[0x7D, 0x7E, 0x7F, 0xFD]]))
+    lib8 = torch.from_numpy(bits).view(torch.float8_e5m2).to(torch.float32).numpy().astype(np.float64)
+    assert np.array_equal(got[fin], lib8[fin])
+    assert got[0x3C] == 1.0 and got[0x7B] == 57344.0 and got[0x01] == 2.0 ** -16
+
+
+@pytest.mark.parametrize("fmt", ["e4m3", "e5m2"])
+def test_fp8_generator_rounds_to_nearest_even(fmt):
+    import torch
+    of, td, top = (oracle.E4M3, torch.float8_e4m3fn, 448.0) if fmt == "e4m3" else (oracle.E5M2, torch.float8_e5m2, 57344.0)
+    rng = np.random.default_rng(12)
+    v = np.concatenate([(rng.standard_normal(50000) * sc).astype(np.float32) for sc in (1.0, 0.02, 30.0, 1e-3)]
+                       + [nk_inputs.fill(4, 0, 20000, "uniform", dtype="f32")])
+    h = nk_inputs.f32_to_fp8_bits(v, fmt)
+    # nearest: no other representable value is closer (checked through the decode of the neighbouring patterns)
+    back = oracle.fp8_to_f32(h, of).astype(np.float64)
+    mag = (h & 0x7F).astype(np.int64)
+    up = oracle.fp8_to_f32(np.minimum(mag + 1, 0x7E if fmt == "e4m3" else 0x7B).astype(np.uint8), of).astype(np.float64)
+    dn = oracle.fp8_to_f32(np.maximum(mag - 1, 0).astype(np.uint8), of).astype(np.float64)
+    x = np.abs(np.clip(v.astype(np.float64), -top, top))
+    assert np.all(np.abs(np.abs(back) - x) <= np.abs(up - x)) and np.all(np.abs(np.abs(back) - x) <= np.abs(dn - x))
+    # ties go to the even pattern; the library's conversion agrees everywhere
+    ref = torch.from_numpy(np.clip(v, -top, top)).to(td).view(torch.uint8).numpy()
+    assert np.array_equal(h, ref)
+    ties = np.array([1.0625, 1.1875, -1.1875], dtype=np.float32) if fmt == "e4m3" else np.array([1.125, 1.375, -1.375], dtype=np.float32)
+    want = np.array([1.0, 1.25, -1.25]) if fmt == "e4m3" else np.array([1.0, 1.5, -1.5])
+    assert np.array_equal(oracle.fp8_to_f32(nk_inputs.f32_to_fp8_bits(ties, fmt), of).astype(np.float64), want)
+
+
+@pytest.mark.parametrize("fmt", ["e4m3", "e5m2"])
+def test_fp8_gemm_equals_gemm_of_the_widened_operands(fmt):
+    """8-bit floating-point operands, B row-major and blocked in groups of four, FP32 bias: the oracle on the
+    8-bit storage equals, bit for bit, the oracle on the same values held as FP32 in row-major order."""
+    M, N, K = 48, 64, 96
+    of = oracle.E4M3 if fmt == "e4m3" else oracle.E5M2
+    w = nk_inputs.Workload("t", M, N, K, fmt, "f32", layout="row", epilogue="bias_relu", seed=13)
+    A, Bflat, bias = w.make()
+    assert bias.dtype == np.float32
+    Af, Bf = oracle.fp8_to_f32(A, of), oracle.fp8_to_f32(Bflat, of)
+    Y0, S0 = oracle.gemm(M, N, K, Af, Bf, bias, in_dtype=F32, epilogue=EPI_BIAS_RELU)
+    Y1, S1 = oracle.gemm_workload(w, A, Bflat, bias)
+    assert np.array_equal(Y0, Y1) and np.array_equal(S0, S1)
+    # blocked B: the bytes scattered by the INT8 rule (groups of four inside 32 x 32 blocks)
+    Bblk = oracle.to_blocked_s8(Bflat.reshape(K, N).view(np.int8)).view(np.uint8)
+    wb = nk_inputs.Workload("t", M, N, K, fmt, "f32", layout="b_blocked32", epilogue="bias_relu", seed=13)
+    Y2, S2 = oracle.gemm_workload(wb, A, Bblk, bias)
+    assert np.array_equal(Y0, Y2) and np.array_equal(S0, S2)
+    assert np.abs(Y0 - np.maximum(Af.astype(np.float64).reshape(M, K) @ Bf.astype(np.float64).reshape(K, N) + bias, 0)).max() < 1e-9
