@@ -64,9 +64,15 @@ typedef enum {
                   four"): B[N/32][K/32][8][32][4], packed[k/4][n][k%4] = flat[k][n] inside each 32 x 32 block.
                   The result is exact: INT32 accumulation of at most 2^17 - 1 products.  No epilogue, no beta,
                   no batch, no K split; N and K multiples of 32 */
-    NK_S32 = 4 /* signed 32-bit integers: the type of C for NK_S8 operands (and only for them).  NK_S8
+    NK_S32 = 4, /* signed 32-bit integers: the type of C for NK_S8 operands (and only for them).  NK_S8
                   operands may also have an NK_F32 C: the INT32 sum is converted (round to nearest even),
                   multiplied by desc.scale and given the epilogue (FP32 bias + ReLU) before the store */
+    NK_E4M3 = 5, /* 8-bit floating point, 4 exponent bits (bias 7), 3 fraction bits, no infinities, largest finite
+                    value 448 (the OCP FP8 E4M3 format) */
+    NK_E5M2 = 6  /* 8-bit floating point, 5 exponent bits (bias 15), 2 fraction bits, IEEE infinities and NaNs.
+                    Both: the 8-bit floating-point counterpart on this hardware of the packed types Section 5
+                    lists; A row-major, B NK_BLOCKED32 with four k per group like NK_S8, FP32 accumulation, FP32 C,
+                    FP32 bias; N and K multiples of 32; no batch */
 } nk_dtype_t;
 typedef enum { NK_ROW_MAJOR = 0, NK_BLOCKED32 = 1 } nk_layout_t;
 typedef enum { NK_EPI_NONE = 0, NK_EPI_BIAS_RELU = 1 } nk_epilogue_t;

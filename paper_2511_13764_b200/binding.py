@@ -10,7 +10,7 @@ import os
 
 from . import _build
 
-F32, BF16, F16, S8, S32 = 0, 1, 2, 3, 4
+F32, BF16, F16, S8, S32, E4M3, E5M2 = 0, 1, 2, 3, 4, 5, 6
 ROW_MAJOR, BLOCKED32 = 0, 1
 EPI_NONE, EPI_BIAS_RELU = 0, 1
 FLAG_KERNEL_NAIVE, FLAG_KERNEL_SIMT, FLAG_KERNEL_UMMA = 0x1, 0x2, 0x3
@@ -202,7 +202,7 @@ def plan_for(w, device=0, flags=0) -> Plan:
     layout ("row"/"blocked32") and epilogue ("none"/"bias_relu") attributes."""
     lay_a = BLOCKED32 if w.layout == "blocked32" else ROW_MAJOR
     lay_b = BLOCKED32 if w.layout in ("blocked32", "b_blocked32") else ROW_MAJOR
-    types = {"f32": F32, "bf16": BF16, "f16": F16, "s8": S8, "s32": S32}
+    types = {"f32": F32, "bf16": BF16, "f16": F16, "s8": S8, "s32": S32, "e4m3": E4M3, "e5m2": E5M2}
     return Plan(w.M, w.N, w.K, in_dtype=types[w.in_dtype], out_dtype=types[w.out_dtype],
                 layout_a=lay_a, layout_b=lay_b,
                 epilogue=EPI_BIAS_RELU if w.epilogue == "bias_relu" else EPI_NONE,

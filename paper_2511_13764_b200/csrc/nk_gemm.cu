@@ -106,16 +106,27 @@ struct DeviceGuard {
 
 static inline bool is16(int dt) { return dt == NK_BF16 || dt == NK_F16; }   // a 16-bit element type
 static inline bool is_s8(const nk_gemm_desc_t& d) { return d.in_dtype == NK_S8; }
+static inline bool is_f8(const nk_gemm_desc_t& d) { return d.in_dtype == NK_E4M3 || d.in_dtype == NK_E5M2; }
+static inline bool is_8bit(const nk_gemm_desc_t& d) { return is_s8(d) || is_f8(d); }
 // k elements in one stage row of the tensor-core kernels (128 bytes)
-static inline int kblock(const nk_gemm_desc_t& d) { return d.in_dtype == NK_S8 ? 2 * UMMA_BK : UMMA_BK; }
+static inline int kblock(const nk_gemm_desc_t& d) { return is_8bit(d) ? 2 * UMMA_BK : UMMA_BK; }
 static inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 static inline int ceil_div(int64_t a, int64_t b) { return static_cast<int>((a + b - 1) / b); }
 
 // tcgen05 instruction descriptor, kind::f16: D format FP32 (bit 4), A and B format at bits 7 and
 // 10 (0 = FP16, 1 = BF16), B major-ness (bit 16: 0 = K-major, 1 = N-major), N/8 at bit 17,
 // M/16 at bit 24.  A is always K-major.
-static uint32_t make_idesc(int m, int n, bool b_n_major, bool f16, bool s8 = false) {
+static uint32_t make_idesc(int m, int n, bool b_n_major, bool f16, bool s8 = false, int f8_format = -1) {
     uint32_t d = 0;
+    if (f8_format >= 0) {
+        // kind::f8f6f4: D format FP32 (1 at bit 4), A and B format at bits 7 and 10 (0 = E4M3, 1 = E5M2)
+        d |= 1u << 4;
+        d |= static_cast<uint32_t>(f8_format) << 7;
+        d |= static_cast<uint32_t>(f8_format) << 10;
+        d |= static_cast<uint32_t>(n >> 3) << 17;
+        d |= static_cast<uint32_t>(m >> 4) << 24;
+        return d;   // both operands K-major
+    }
     if (s8) {
         // kind::i8: D format INT32 (2 at bit 4), A and B format signed 8-bit (1 at bits 7 and 10)
         d |= 2u << 4;
@@ -163,6 +174,7 @@ static int max_clusters_for(bool pair, int bn, bool vnni, int splits);
 static bool cluster_reduce_fits(const nk_gemm_desc_t& d, int sms, bool pair, int bn, int eff_splits) {
     (void)sms;
     if (d.flags & NK_FLAG_SEPARATE_REDUCE) return false;
+    if (is_8bit(d)) return false;   // the cluster variants are built for the 16-bit kernels only
     if (eff_splits != 2 && eff_splits != 4 && !(eff_splits == 8 && !pair)) return false;
     const int64_t clusters = static_cast<int64_t>(desc_gemms(d)) * ceil_div(d.M, pair ? 2 * UMMA_BM : UMMA_BM) * ceil_div(d.N, bn);
     const bool vnni = d.layout_b == NK_BLOCKED32 && !(d.flags & NK_FLAG_REPACK_B);
@@ -346,9 +358,9 @@ static void choose_skinny(nk_gemm_s* p) {
 static nk_status_t encode_maps(nk_gemm_s* p, const void* A, const void* B) {
     if (p->cached_a == A && p->cached_b == B) return NK_OK;
     const nk_gemm_desc_t& d = p->d;
-    const CUtensorMapDataType half_type = d.in_dtype == NK_S8 ? CU_TENSOR_MAP_DATA_TYPE_UINT8
+    const CUtensorMapDataType half_type = is_8bit(d) ? CU_TENSOR_MAP_DATA_TYPE_UINT8
                                           : d.in_dtype == NK_F16 ? CU_TENSOR_MAP_DATA_TYPE_FLOAT16 : CU_TENSOR_MAP_DATA_TYPE_BFLOAT16;
-    const cuuint64_t esz = d.in_dtype == NK_S8 ? 1 : 2;   // bytes per operand element
+    const cuuint64_t esz = is_8bit(d) ? 1 : 2;   // bytes per operand element
     CUresult r;
     if (d.layout_a == NK_BLOCKED32) {
         // [M/32][K/32][32][32] as a 4-D tensor (k, m, k-block, m-block): a box of
@@ -458,20 +470,27 @@ static nk_status_t encode_c_map(nk_gemm_s* p, void* C) {
     return NK_OK;
 }
 
-template <int BN, int STAGES, bool VNNI, bool I8 = false>
+template <int BN, int STAGES, bool VNNI, int KIND = 0>
 static cudaError_t launch_umma_t(nk_gemm_s* p, const UmmaParams& up, int grid, cudaStream_t st) {
-    umma_bf16_kernel<BN, STAGES, VNNI, false, I8><<<grid, VNNI ? 320 : 192, umma_smem_bytes(BN, STAGES), st>>>(
+    umma_bf16_kernel<BN, STAGES, VNNI, false, KIND><<<grid, VNNI ? 320 : 192, umma_smem_bytes(BN, STAGES), st>>>(
         p->tmap_a, p->tmap_b, p->tmap_c, up);
     return cudaGetLastError();
 }
 
 static cudaError_t launch_umma(nk_gemm_s* p, const UmmaParams& up, int grid, cudaStream_t st) {
     const bool v = p->b_vnni_inkernel;
-    if (is_s8(p->d)) {   // INT8 operands: B is always blocked and re-laid in the kernel
+    if (is_s8(p->d)) {   // 8-bit operands: B is always blocked and re-laid in the kernel
         switch (p->bn) {
-            case 256: return launch_umma_t<256, 4, true, true>(p, up, grid, st);
-            case 128: return launch_umma_t<128, 6, true, true>(p, up, grid, st);
-            default:  return launch_umma_t<64, 8, true, true>(p, up, grid, st);
+            case 256: return launch_umma_t<256, 4, true, 1>(p, up, grid, st);
+            case 128: return launch_umma_t<128, 6, true, 1>(p, up, grid, st);
+            default:  return launch_umma_t<64, 8, true, 1>(p, up, grid, st);
+        }
+    }
+    if (is_f8(p->d)) {
+        switch (p->bn) {
+            case 256: return launch_umma_t<256, 4, true, 2>(p, up, grid, st);
+            case 128: return launch_umma_t<128, 6, true, 2>(p, up, grid, st);
+            default:  return launch_umma_t<64, 8, true, 2>(p, up, grid, st);
         }
     }
     switch (p->bn) {
@@ -550,7 +569,7 @@ static int max_clusters_for(bool pair, int bn, bool vnni, int splits) {
     return c > 0 ? c : 0;
 }
 
-template <int BN, int STAGES, bool VNNI, bool I8 = false>
+template <int BN, int STAGES, bool VNNI, int KIND = 0>
 static cudaError_t launch_pair_t(nk_gemm_s* p, const UmmaParams& up, int pairs, cudaStream_t st) {
     cudaLaunchConfig_t cfg;
     memset(&cfg, 0, sizeof(cfg));
@@ -565,12 +584,13 @@ static cudaError_t launch_pair_t(nk_gemm_s* p, const UmmaParams& up, int pairs, 
     attr.val.clusterDim.z = 1;
     cfg.attrs = &attr;
     cfg.numAttrs = 1;
-    return cudaLaunchKernelEx(&cfg, umma_bf16_pair_kernel<BN, STAGES, VNNI, false, I8>, p->tmap_a, p->tmap_b, p->tmap_c, up);
+    return cudaLaunchKernelEx(&cfg, umma_bf16_pair_kernel<BN, STAGES, VNNI, false, KIND>, p->tmap_a, p->tmap_b, p->tmap_c, up);
 }
 
 static cudaError_t launch_pair(nk_gemm_s* p, const UmmaParams& up, int pairs, cudaStream_t st) {
     const bool v = p->b_vnni_inkernel;
-    if (is_s8(p->d)) return p->bn == 256 ? launch_pair_t<256, 6, true, true>(p, up, pairs, st) : launch_pair_t<128, 8, true, true>(p, up, pairs, st);
+    if (is_s8(p->d)) return p->bn == 256 ? launch_pair_t<256, 6, true, 1>(p, up, pairs, st) : launch_pair_t<128, 8, true, 1>(p, up, pairs, st);
+    if (is_f8(p->d)) return p->bn == 256 ? launch_pair_t<256, 6, true, 2>(p, up, pairs, st) : launch_pair_t<128, 8, true, 2>(p, up, pairs, st);
     if (p->bn == 256) return v ? launch_pair_t<256, 6, true>(p, up, pairs, st) : launch_pair_t<256, 6, false>(p, up, pairs, st);
     return v ? launch_pair_t<128, 8, true>(p, up, pairs, st) : launch_pair_t<128, 8, false>(p, up, pairs, st);
 }
@@ -619,11 +639,16 @@ static cudaError_t prepare_umma_attrs() {
     if ((e = allow_smem(umma_bf16_pair_kernel<256, 6, true, true>, pair_smem_bytes(256, 6))) != cudaSuccess) return e;
     if ((e = allow_smem(umma_bf16_pair_kernel<128, 8, false, true>, pair_smem_bytes(128, 8))) != cudaSuccess) return e;
     if ((e = allow_smem(umma_bf16_pair_kernel<128, 8, true, true>, pair_smem_bytes(128, 8))) != cudaSuccess) return e;
-    if ((e = allow_smem(umma_bf16_kernel<256, 4, true, false, true>, umma_smem_bytes(256, 4))) != cudaSuccess) return e;
-    if ((e = allow_smem(umma_bf16_kernel<128, 6, true, false, true>, umma_smem_bytes(128, 6))) != cudaSuccess) return e;
-    if ((e = allow_smem(umma_bf16_kernel<64, 8, true, false, true>, umma_smem_bytes(64, 8))) != cudaSuccess) return e;
-    if ((e = allow_smem(umma_bf16_pair_kernel<256, 6, true, false, true>, pair_smem_bytes(256, 6))) != cudaSuccess) return e;
-    if ((e = allow_smem(umma_bf16_pair_kernel<128, 8, true, false, true>, pair_smem_bytes(128, 8))) != cudaSuccess) return e;
+    if ((e = allow_smem(umma_bf16_kernel<256, 4, true, false, 1>, umma_smem_bytes(256, 4))) != cudaSuccess) return e;
+    if ((e = allow_smem(umma_bf16_kernel<256, 4, true, false, 2>, umma_smem_bytes(256, 4))) != cudaSuccess) return e;
+    if ((e = allow_smem(umma_bf16_kernel<128, 6, true, false, 1>, umma_smem_bytes(128, 6))) != cudaSuccess) return e;
+    if ((e = allow_smem(umma_bf16_kernel<128, 6, true, false, 2>, umma_smem_bytes(128, 6))) != cudaSuccess) return e;
+    if ((e = allow_smem(umma_bf16_kernel<64, 8, true, false, 1>, umma_smem_bytes(64, 8))) != cudaSuccess) return e;
+    if ((e = allow_smem(umma_bf16_kernel<64, 8, true, false, 2>, umma_smem_bytes(64, 8))) != cudaSuccess) return e;
+    if ((e = allow_smem(umma_bf16_pair_kernel<256, 6, true, false, 1>, pair_smem_bytes(256, 6))) != cudaSuccess) return e;
+    if ((e = allow_smem(umma_bf16_pair_kernel<256, 6, true, false, 2>, pair_smem_bytes(256, 6))) != cudaSuccess) return e;
+    if ((e = allow_smem(umma_bf16_pair_kernel<128, 8, true, false, 1>, pair_smem_bytes(128, 8))) != cudaSuccess) return e;
+    if ((e = allow_smem(umma_bf16_pair_kernel<128, 8, true, false, 2>, pair_smem_bytes(128, 8))) != cudaSuccess) return e;
     return cudaSuccess;
 }
 
@@ -667,9 +692,18 @@ nk_status_t nk_gemm_create(const nk_gemm_desc_t* desc, nk_gemm_t* out) {
     if (d.M <= 0 || d.N <= 0 || d.K <= 0) return NK_ERR_INVALID_ARG;
     if (d.M > (1 << 24) || d.N > (1 << 24) || d.K > (1 << 24)) return NK_ERR_UNSUPPORTED;
     if (d.M * d.N >= (1ll << 31) || d.M * d.K >= (1ll << 33) || d.K * d.N >= (1ll << 33)) return NK_ERR_UNSUPPORTED;
-    if (d.in_dtype != NK_F32 && !is16(d.in_dtype) && d.in_dtype != NK_S8) return NK_ERR_INVALID_ARG;
+    if (d.in_dtype != NK_F32 && !is16(d.in_dtype) && !is_8bit(d)) return NK_ERR_INVALID_ARG;
     if (d.out_dtype != NK_F32 && !is16(d.out_dtype) && d.out_dtype != NK_S32) return NK_ERR_INVALID_ARG;
     if (d.out_dtype == NK_S32 && d.in_dtype != NK_S8) return NK_ERR_INVALID_ARG;   // an INT32 C belongs to INT8 operands
+    if (is_f8(d)) {
+        // 8-bit floating-point operands: A row-major, B packed in groups of four inside 32 x 32 blocks, FP32 C
+        if (d.out_dtype != NK_F32) return NK_ERR_INVALID_ARG;
+        if (d.layout_a != NK_ROW_MAJOR || d.layout_b != NK_BLOCKED32 || d.layout_c != NK_ROW_MAJOR) return NK_ERR_UNSUPPORTED;
+        if (d.batch > 1) return NK_ERR_UNSUPPORTED;
+        if (d.flags & NK_FLAG_REPACK_B) return NK_ERR_UNSUPPORTED;
+        const uint32_t fk = d.flags & NK_FLAG_KERNEL_MASK;
+        if (fk == NK_FLAG_KERNEL_NAIVE || fk == NK_FLAG_KERNEL_SIMT) return NK_ERR_UNSUPPORTED;
+    }
     if (d.in_dtype == NK_S8) {
         // the Int8 dot product: A row-major, B packed in groups of four inside 32 x 32 blocks; C is the exact
         // INT32 sum, or FP32 = scale * sum with the epilogue (quantised layer)
@@ -688,7 +722,7 @@ nk_status_t nk_gemm_create(const nk_gemm_desc_t* desc, nk_gemm_t* out) {
     if (d.epilogue != NK_EPI_NONE && d.epilogue != NK_EPI_BIAS_RELU) return NK_ERR_INVALID_ARG;
     if (is16(d.out_dtype) && d.in_dtype != d.out_dtype) return NK_ERR_INVALID_ARG;   // a 16-bit C has the operands' type
     const bool blocked = d.layout_a == NK_BLOCKED32 || d.layout_b == NK_BLOCKED32;
-    if (blocked && !is16(d.in_dtype) && d.in_dtype != NK_S8) return NK_ERR_UNSUPPORTED;
+    if (blocked && !is16(d.in_dtype) && !is_8bit(d)) return NK_ERR_UNSUPPORTED;
     if (d.layout_a == NK_BLOCKED32 && (d.M % 32 || d.K % 32)) return NK_ERR_MISALIGNED;
     if (d.layout_b == NK_BLOCKED32 && (d.N % 32 || d.K % 32)) return NK_ERR_MISALIGNED;
     if (d.beta != 0 && d.beta != 1) return NK_ERR_INVALID_ARG;
@@ -729,7 +763,7 @@ nk_status_t nk_gemm_create(const nk_gemm_desc_t* desc, nk_gemm_t* out) {
         if (is16(d.in_dtype) && (d.N % 8 || d.K % 8)) return NK_ERR_MISALIGNED;
         if (d.in_dtype == NK_F32 && (d.N % 4 || d.K % 4)) return NK_ERR_MISALIGNED;
         if (force == NK_FLAG_KERNEL_SIMT && d.in_dtype != NK_F32) return NK_ERR_UNSUPPORTED;
-        if (force == NK_FLAG_KERNEL_UMMA && !is16(d.in_dtype) && d.in_dtype != NK_S8) return NK_ERR_UNSUPPORTED;
+        if (force == NK_FLAG_KERNEL_UMMA && !is16(d.in_dtype) && !is_8bit(d)) return NK_ERR_UNSUPPORTED;
     }
 
     int ndev = 0;
@@ -902,6 +936,10 @@ nk_status_t nk_gemm_create(const nk_gemm_desc_t* desc, nk_gemm_t* out) {
         const size_t len = strlen(p->name);
         snprintf(p->name + len, sizeof(p->name) - len, "_f16");
     }
+    if (is_f8(d)) {
+        const size_t len = strlen(p->name);
+        snprintf(p->name + len, sizeof(p->name) - len, d.in_dtype == NK_E4M3 ? "_e4m3" : "_e5m2");
+    }
     if (d.in_dtype == NK_S8) {
         const size_t len = strlen(p->name);
         snprintf(p->name + len, sizeof(p->name) - len, d.out_dtype == NK_F32 ? "_s8_dequant" : "_s8");
@@ -1028,13 +1066,14 @@ nk_status_t nk_gemm_run(nk_gemm_t p, const void* A, const void* B, const void* b
         up.b_3d = p->b_3d ? 1 : 0;
         up.epilogue = d.epilogue;
         up.out_bf16 = is16(d.out_dtype);
-        up.idesc = make_idesc(p->pair ? 2 * UMMA_BM : UMMA_BM, p->bn, !p->b_vnni_inkernel, d.in_dtype == NK_F16, is_s8(d));
+        up.idesc = make_idesc(p->pair ? 2 * UMMA_BM : UMMA_BM, p->bn, !p->b_vnni_inkernel, d.in_dtype == NK_F16, is_s8(d),
+                              d.in_dtype == NK_E4M3 ? 0 : d.in_dtype == NK_E5M2 ? 1 : -1);
         up.f16 = d.in_dtype == NK_F16;
         up.bias = bias;
         up.C = C;
         up.partial = partial;
         up.status = p->status_dev;
-        up.bias_f32 = (p->bias_f32 || is_s8(d)) ? 1 : 0;
+        up.bias_f32 = (p->bias_f32 || is_8bit(d)) ? 1 : 0;
         up.dequant = (is_s8(d) && d.out_dtype == NK_F32) ? 1 : 0;
         up.scale = d.scale;
         up.item_remap = p->item_remap ? 1 : 0;
@@ -1059,7 +1098,7 @@ nk_status_t nk_gemm_run(nk_gemm_t p, const void* A, const void* B, const void* b
     if (p->variant == V_UMMA && p->tail_from >= 0) {
         const int tiles_m = ceil_div(d.M, 2 * UMMA_BM), tiles_n = ceil_div(d.N, p->bn);
         TailReduceParams tp = {static_cast<int>(d.M), static_cast<int>(d.N), 2 * UMMA_BM, p->bn, tiles_m, tiles_n, p->group_m,
-                               p->tail_from, p->tail_splits, d.epilogue, p->bias_f32 ? 0 : 1, is16(d.out_dtype), d.beta,
+                               p->tail_from, p->tail_splits, d.epilogue, (p->bias_f32 || is_8bit(d)) ? 0 : 1, is16(d.out_dtype), d.beta,
                                d.layout_c == NK_BLOCKED32, d.in_dtype == NK_F16, partial, bias, C};
         const int quads = 2 * UMMA_BM * p->bn / 4;
         dim3 grid(static_cast<unsigned>((quads + 255) / 256), static_cast<unsigned>(tiles_m * tiles_n - p->tail_from));
@@ -1085,7 +1124,7 @@ nk_status_t nk_gemm_run_host(nk_gemm_t p, const void* hA, const void* hB, const 
     if (!p || !hA || !hB || !hC || !dA || !dB || !dC) return NK_ERR_INVALID_ARG;
     const nk_gemm_desc_t& d = p->d;
     if (d.epilogue != NK_EPI_NONE && (!hbias || !dbias)) return NK_ERR_INVALID_ARG;
-    const size_t ein = d.in_dtype == NK_S8 ? 1 : is16(d.in_dtype) ? 2 : 4, eout = is16(d.out_dtype) ? 2 : 4;
+    const size_t ein = is_8bit(d) ? 1 : is16(d.in_dtype) ? 2 : 4, eout = is16(d.out_dtype) ? 2 : 4;
     cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
     DeviceGuard guard(d.device);
     if (guard.err != cudaSuccess) { set_err(p, "cudaSetDevice", guard.err); return NK_ERR_DEVICE; }
@@ -1130,18 +1169,19 @@ nk_status_t nk_gemm_run_host(nk_gemm_t p, const void* hA, const void* hB, const 
             }
         }
         if (p->chunk_plan) {
-            const size_t ein_b = d.in_dtype == NK_S8 ? 1 : is16(d.in_dtype) ? 2 : 4, eout_b = is16(d.out_dtype) ? 2 : 4;
+            const size_t ein_b = is_8bit(d) ? 1 : is16(d.in_dtype) ? 2 : 4, eout_b = is16(d.out_dtype) ? 2 : 4;
             const int panels = p->chunk_panels;
             const size_t rows = static_cast<size_t>(p->chunk_rows), cols = static_cast<size_t>(d.N) / panels;
             const size_t a_chunk = rows * d.K * ein_b;                         // also right for blocked A
             const size_t b_panel = static_cast<size_t>(d.K) * cols * ein_b;     // dense on the device
             const size_t c_block = rows * cols * eout_b;                       // dense on the device
             const bool has_bias = d.epilogue != NK_EPI_NONE;
+            const size_t ebias_b = is_8bit(d) ? 4 : ein_b;   // 8-bit operands come with an FP32 bias
             const bool b_rows_strided = d.layout_b == NK_ROW_MAJOR && panels > 1;   // a blocked B panel is contiguous
             bool ok = cudaEventRecord(p->ev_start, st) == cudaSuccess &&
                       cudaStreamWaitEvent(p->h2d_stream, p->ev_start, 0) == cudaSuccess &&
                       cudaStreamWaitEvent(p->d2h_stream, p->ev_start, 0) == cudaSuccess &&
-                      (!has_bias || cudaMemcpyAsync(dbias, hbias, static_cast<size_t>(d.N) * ein_b, cudaMemcpyHostToDevice, p->h2d_stream) == cudaSuccess);
+                      (!has_bias || cudaMemcpyAsync(dbias, hbias, static_cast<size_t>(d.N) * ebias_b, cudaMemcpyHostToDevice, p->h2d_stream) == cudaSuccess);
             int na = 0, nb = 0, nup = 0, ng = 0;     // row chunks and panels on the device; uploads and blocks so far
             while (ok && (na < kRowChunks || nb < panels)) {
                 // A0, B0, then B and A in turn until one runs out
@@ -1170,7 +1210,7 @@ nk_status_t nk_gemm_run_host(nk_gemm_t p, const void* hA, const void* hB, const 
                         char* dC_ij = static_cast<char*>(dC) + (static_cast<size_t>(i) * panels + j) * c_block;
                         nk_status_t rs = nk_gemm_run(p->chunk_plan, static_cast<char*>(dA) + i * a_chunk,
                                                      static_cast<char*>(dB) + j * b_panel,
-                                                     has_bias ? static_cast<char*>(dbias) + j * cols * ein_b : nullptr, dC_ij,
+                                                     has_bias ? static_cast<char*>(dbias) + j * cols * ebias_b : nullptr, dC_ij,
                                                      nullptr, 0, cuda_stream);
                         if (rs != NK_OK) {
                             snprintf(p->cuda_err, sizeof(p->cuda_err), "block %d,%d: %s", i, j, nk_gemm_last_cuda_error(p->chunk_plan));
@@ -1213,7 +1253,7 @@ nk_status_t nk_gemm_run_host(nk_gemm_t p, const void* hA, const void* hB, const 
         return NK_ERR_CUDA;
     }
     if (d.epilogue != NK_EPI_NONE &&
-        (e = cudaMemcpyAsync(dbias, hbias, ein * d.N, cudaMemcpyHostToDevice, st)) != cudaSuccess) {
+        (e = cudaMemcpyAsync(dbias, hbias, (is_8bit(d) ? 4 : ein) * d.N, cudaMemcpyHostToDevice, st)) != cudaSuccess) {
         set_err(p, "H2D copy", e);
         return NK_ERR_CUDA;
     }

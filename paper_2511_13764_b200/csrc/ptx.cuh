@@ -188,10 +188,25 @@ __device__ __forceinline__ void umma_i8_lohi(uint32_t d_tmem, uint32_t a_lo, uin
         "r"(a_lo), "r"(a_hi), "r"(b_lo), "r"(b_hi), "r"(idesc), "r"(accumulate)
         : "memory");
 }
-template <bool I8>
+// The 8-bit floating-point form (kind::f8f6f4 with E4M3 or E5M2 operands, 32 per k-step, FP32 accumulator).
+__device__ __forceinline__ void umma_f8_lohi(uint32_t d_tmem, uint32_t a_lo, uint32_t a_hi,
+                                             uint32_t b_lo, uint32_t b_hi, uint32_t idesc,
+                                             uint32_t accumulate) {
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t.reg .b64 da, db;\n\t"
+        "setp.ne.b32 p, %6, 0;\n\t"
+        "mov.b64 da, {%1, %2};\n\t"
+        "mov.b64 db, {%3, %4};\n\t"
+        "tcgen05.mma.cta_group::1.kind::f8f6f4 [%0], da, db, %5, p;\n\t}" ::"r"(d_tmem),
+        "r"(a_lo), "r"(a_hi), "r"(b_lo), "r"(b_hi), "r"(idesc), "r"(accumulate)
+        : "memory");
+}
+// KIND: 0 = 16-bit floating point, 1 = INT8, 2 = 8-bit floating point
+template <int KIND>
 __device__ __forceinline__ void umma_lohi(uint32_t d_tmem, uint32_t a_lo, uint32_t a_hi, uint32_t b_lo,
                                           uint32_t b_hi, uint32_t idesc, uint32_t accumulate) {
-    if (I8) umma_i8_lohi(d_tmem, a_lo, a_hi, b_lo, b_hi, idesc, accumulate);
+    if (KIND == 1) umma_i8_lohi(d_tmem, a_lo, a_hi, b_lo, b_hi, idesc, accumulate);
+    else if (KIND == 2) umma_f8_lohi(d_tmem, a_lo, a_hi, b_lo, b_hi, idesc, accumulate);
     else umma_f16_lohi(d_tmem, a_lo, a_hi, b_lo, b_hi, idesc, accumulate);
 }
 // Arrive on `bar` once every tcgen05.mma issued so far by this thread has completed.
@@ -341,10 +356,23 @@ __device__ __forceinline__ void umma_i8_pair_lohi(uint32_t d_tmem, uint32_t a_lo
         "r"(a_lo), "r"(a_hi), "r"(b_lo), "r"(b_hi), "r"(idesc), "r"(accumulate)
         : "memory");
 }
-template <bool I8>
+__device__ __forceinline__ void umma_f8_pair_lohi(uint32_t d_tmem, uint32_t a_lo, uint32_t a_hi,
+                                                  uint32_t b_lo, uint32_t b_hi, uint32_t idesc,
+                                                  uint32_t accumulate) {
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t.reg .b64 da, db;\n\t"
+        "setp.ne.b32 p, %6, 0;\n\t"
+        "mov.b64 da, {%1, %2};\n\t"
+        "mov.b64 db, {%3, %4};\n\t"
+        "tcgen05.mma.cta_group::2.kind::f8f6f4 [%0], da, db, %5, p;\n\t}" ::"r"(d_tmem),
+        "r"(a_lo), "r"(a_hi), "r"(b_lo), "r"(b_hi), "r"(idesc), "r"(accumulate)
+        : "memory");
+}
+template <int KIND>
 __device__ __forceinline__ void umma_pair_lohi(uint32_t d_tmem, uint32_t a_lo, uint32_t a_hi, uint32_t b_lo,
                                                uint32_t b_hi, uint32_t idesc, uint32_t accumulate) {
-    if (I8) umma_i8_pair_lohi(d_tmem, a_lo, a_hi, b_lo, b_hi, idesc, accumulate);
+    if (KIND == 1) umma_i8_pair_lohi(d_tmem, a_lo, a_hi, b_lo, b_hi, idesc, accumulate);
+    else if (KIND == 2) umma_f8_pair_lohi(d_tmem, a_lo, a_hi, b_lo, b_hi, idesc, accumulate);
     else umma_f16_pair_lohi(d_tmem, a_lo, a_hi, b_lo, b_hi, idesc, accumulate);
 }
 // Arrive, in every CTA of `cta_mask`, on the mbarrier at this shared offset once all MMAs

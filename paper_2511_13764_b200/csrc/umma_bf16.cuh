@@ -489,7 +489,7 @@ __device__ __forceinline__ void vnni_relayout_stage(uint32_t sb, int tw, int lan
     }
 }
 
-template <int BN, int STAGES, bool B_VNNI, bool CLUSTER_REDUCE = false, bool I8 = false>
+template <int BN, int STAGES, bool B_VNNI, bool CLUSTER_REDUCE = false, int KIND = 0>
 __global__ void __launch_bounds__(B_VNNI ? 320 : 192, 1)
 umma_bf16_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ CUtensorMap tmap_b,
                  const __grid_constant__ CUtensorMap tmap_c, const UmmaParams p) {
@@ -590,7 +590,7 @@ umma_bf16_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_consta
             int ia, ib;
             umma_item_pair(p, item, ia, ib);
             for (int kb = kb0; kb < kb1; ++kb) {
-                const int kx = kbl * (I8 ? 2 * UMMA_BK : UMMA_BK);   // a stage row is 128 bytes: 64 16-bit or 128 8-bit elements
+                const int kx = kbl * (KIND != 0 ? 2 * UMMA_BK : UMMA_BK);   // a stage row is 128 bytes: 64 16-bit or 128 8-bit elements
                 if (!mbar_wait(empty_bar(stage), phase ^ 1u, abort_flag)) {
                     if (lane == 0) give_up(0x100u + stage);
                     ok = false;
@@ -684,10 +684,10 @@ umma_bf16_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_consta
                 tc_fence_after_sync();
                 if (lane == 0) {
                     const uint32_t a_lo = a_lo0 + soff, b_lo = b_lo0 + soff;
-                    umma_lohi<I8>(d_tmem, a_lo, a_hi, b_lo, b_hi, idesc, accumulate);
-                    umma_lohi<I8>(d_tmem, a_lo + a_s1, a_hi, b_lo + b_s, b_hi, idesc, 1u);
-                    umma_lohi<I8>(d_tmem, a_lo + a_s2, a_hi, b_lo + 2 * b_s, b_hi, idesc, 1u);
-                    umma_lohi<I8>(d_tmem, a_lo + a_s3, a_hi, b_lo + 3 * b_s, b_hi, idesc, 1u);
+                    umma_lohi<KIND>(d_tmem, a_lo, a_hi, b_lo, b_hi, idesc, accumulate);
+                    umma_lohi<KIND>(d_tmem, a_lo + a_s1, a_hi, b_lo + b_s, b_hi, idesc, 1u);
+                    umma_lohi<KIND>(d_tmem, a_lo + a_s2, a_hi, b_lo + 2 * b_s, b_hi, idesc, 1u);
+                    umma_lohi<KIND>(d_tmem, a_lo + a_s3, a_hi, b_lo + 3 * b_s, b_hi, idesc, 1u);
                     umma_commit(empty_bar(stage));
                     if (kb == kb1 - 1) umma_commit(tfull_bar(acc));
                 }

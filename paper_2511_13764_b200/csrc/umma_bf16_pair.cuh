@@ -38,7 +38,7 @@ __host__ __device__ constexpr int pair_smem_bytes(int BN, int stages) {
 }
 
 // UmmaParams as for the single-CTA kernel, with tiles_m counted in 256-row tiles.
-template <int BN, int STAGES, bool B_VNNI, bool CLUSTER_REDUCE = false, bool I8 = false>
+template <int BN, int STAGES, bool B_VNNI, bool CLUSTER_REDUCE = false, int KIND = 0>
 __global__ void __launch_bounds__(B_VNNI ? 320 : 192, 1)
 umma_bf16_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ CUtensorMap tmap_b,
                       const __grid_constant__ CUtensorMap tmap_c, const UmmaParams p) {
@@ -152,7 +152,7 @@ umma_bf16_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_c
             int ia, ib;
             umma_item_pair(p, item, ia, ib);
             for (int kb = kb0; kb < kb1; ++kb) {
-                const int kx = kbl * (I8 ? 2 * UMMA_BK : UMMA_BK);   // 128 bytes of k per stage row
+                const int kx = kbl * (KIND != 0 ? 2 * UMMA_BK : UMMA_BK);   // 128 bytes of k per stage row
                 if (!mbar_wait(empty_bar(stage), phase ^ 1u, abort_flag)) {
                     if (lane == 0) give_up(0x100u + stage);
                     ok = false;
@@ -237,10 +237,10 @@ umma_bf16_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_c
                     tc_fence_after_sync();
                     if (lane == 0) {
                         const uint32_t a_lo = a_lo0 + soff, b_lo = b_lo0 + soff;
-                        umma_pair_lohi<I8>(d_tmem, a_lo, a_hi, b_lo, b_hi, idesc, accumulate);
-                        umma_pair_lohi<I8>(d_tmem, a_lo + a_s1, a_hi, b_lo + b_s, b_hi, idesc, 1u);
-                        umma_pair_lohi<I8>(d_tmem, a_lo + a_s2, a_hi, b_lo + 2 * b_s, b_hi, idesc, 1u);
-                        umma_pair_lohi<I8>(d_tmem, a_lo + a_s3, a_hi, b_lo + 3 * b_s, b_hi, idesc, 1u);
+                        umma_pair_lohi<KIND>(d_tmem, a_lo, a_hi, b_lo, b_hi, idesc, accumulate);
+                        umma_pair_lohi<KIND>(d_tmem, a_lo + a_s1, a_hi, b_lo + b_s, b_hi, idesc, 1u);
+                        umma_pair_lohi<KIND>(d_tmem, a_lo + a_s2, a_hi, b_lo + 2 * b_s, b_hi, idesc, 1u);
+                        umma_pair_lohi<KIND>(d_tmem, a_lo + a_s3, a_hi, b_lo + 3 * b_s, b_hi, idesc, 1u);
                         umma_commit_pair(empty_bar(stage), pair_mask);
                         if (kb == kb1 - 1) umma_commit_pair(tfull_bar(acc), pair_mask);
                     }

@@ -93,17 +93,23 @@ def time_workload(w, iters, flags=0, flush=None, graph_pairs=0, library=False):
     import torch
     import paper_2511_13764_b200 as nk
     dev = torch.device("cuda", 0)
-    tt = {"f32": torch.float32, "bf16": torch.bfloat16, "f16": torch.float16, "s8": torch.int8, "s32": torch.int32}
+    tt = {"f32": torch.float32, "bf16": torch.bfloat16, "f16": torch.float16, "s8": torch.int8, "s32": torch.int32,
+          "e4m3": torch.uint8, "e5m2": torch.uint8}
     ein, eout = tt[w.in_dtype], tt[w.out_dtype]
     g = torch.Generator(device=dev).manual_seed(w.seed)
     if w.in_dtype == "s8":
         A = torch.randint(-128, 128, (w.M * w.K,), device=dev, generator=g, dtype=torch.int8)
         B = torch.randint(-128, 128, (w.K * w.N,), device=dev, generator=g, dtype=torch.int8)
         library = False      # no library column for INT8
+    elif w.in_dtype in ("e4m3", "e5m2"):
+        f8 = torch.float8_e4m3fn if w.in_dtype == "e4m3" else torch.float8_e5m2
+        A = (torch.rand(w.M * w.K, device=dev, generator=g) * 2 - 1).to(f8)
+        B = (torch.rand(w.K * w.N, device=dev, generator=g) * 2 - 1).to(f8)
+        library = False      # nor for 8-bit floating point
     else:
         A = (torch.rand(w.M * w.K, device=dev, generator=g) * 2 - 1).to(ein)
         B = (torch.rand(w.K * w.N, device=dev, generator=g) * 2 - 1).to(ein)
-    bias = (torch.randn(w.N, device=dev, generator=g) * 0.02).to(ein) if w.epilogue != "none" else None
+    bias = (torch.randn(w.N, device=dev, generator=g) * 0.02).to(tt[w.bias_dtype]) if w.epilogue != "none" else None
     C = torch.empty(w.M * w.N, dtype=eout, device=dev)
     plan = nk.plan_for(w, flags=flags)
     wsb = plan.workspace_bytes
@@ -147,7 +153,7 @@ def main():
     fma_peak = prop.multi_processor_count * 128 * 2 * 1.965e9 / 1e12
     flush = None if args.no_flush else torch.empty(512 << 20, dtype=torch.uint8, device="cuda")
     works = ([nk_inputs.config(i) for i in (1, 2, 3, 4)] + nk_inputs.sweep() + nk_inputs.paper_mlp() + nk_inputs.f16_set()
-             + nk_inputs.s8_set())
+             + nk_inputs.s8_set() + nk_inputs.fp8_set())
     rows = []
     print(f"| workload | kernel | launches | median us | TFLOP/s | alg. GB/s | bound | frac ({src}) |"
           + (" cuBLAS us |" if args.library else ""))
@@ -166,8 +172,8 @@ def main():
                                                            library=args.library and not split)
         tf = w.flops / (med * 1e-3) / 1e12
         gbs = w.algorithmic_bytes / (med * 1e-3) / 1e9
-        # INT8 runs at twice the BF16 rate on the tensor cores (nominal ratio applied to the measured BF16 peak)
-        compute_peak = (tensor_peak / 6 if split else 2 * tensor_peak if w.in_dtype == "s8"
+        # 8-bit operands run at twice the BF16 rate on the tensor cores (nominal ratio applied to the measured BF16 peak)
+        compute_peak = (tensor_peak / 6 if split else 2 * tensor_peak if w.in_dtype in ("s8", "e4m3", "e5m2")
                         else tensor_peak if w.in_dtype != "f32" else fma_peak)
         t_compute = w.flops / (compute_peak * 1e12)
         t_hbm = w.algorithmic_bytes / (hbm_peak * 1e9)
