@@ -14,16 +14,20 @@
  * packed type Section 5 names next) widened exactly to FP32 with the products
  * accumulated in FP32.  C is FP32, or has the operands' 16-bit type, rounded to
  * nearest-even once, after the epilogue.  Wherever a rule below says BF16 it holds
- * for FP16 as well.
+ * for FP16 as well.  8-bit operands (NK_S8 with exact INT32 accumulation, the Int8 dot
+ * product Section 5 names among the next packed types; NK_E4M3 / NK_E5M2 with FP32
+ * accumulation) take A row-major and B blocked with four k per group; see nk_dtype_t.
  *
  * Operand layouts (Section 2.3, Figure 1 and Listing 1):
  *   NK_ROW_MAJOR   A[M][K], B[K][N]                      ("flat")
  *   NK_BLOCKED32   A[M/32][K/32][32][32]                 (m-block, k-block, m, k)
  *                  B[N/32][K/32][16][32][2]              (n-block, k-block, k/2, n, k%2):
  *                  every 32x32 block of B is VNNI-2 packed as in Figure 1,
- *                  packed[k/2][n][k%2] = flat[k][n]; 16-bit operands (BF16, FP16) only.
+ *                  packed[k/2][n][k%2] = flat[k][n] (16-bit operands);
+ *                  B[N/32][K/32][8][32][4], packed[k/4][n][k%4] = flat[k][n] (8-bit operands:
+ *                  Section 2, "INT8 elements in groups of four").
  * C is row-major [M][N] unless desc.layout_c asks for the blocked form; bias is [N] in the
- * operand type.
+ * operand type (FP32 for 8-bit operands).
  *
  * All data pointers are DEVICE pointers on the plan's device unless a function
  * says otherwise.  The library never allocates or frees device memory, never
@@ -139,8 +143,8 @@ typedef struct {
  * Build a plan (Section 3.1, register tiling; Section 5(a), tile-size selection:
  * here the choice of kernel, output tile and K split is made once, from the
  * shape).  Validates the descriptor, queries the device, and keeps only host
- * state.  Requirements: M, N, K > 0; blocked layouts need BF16 and the blocked
- * operand's two dimensions to be multiples of 32; row-major BF16 needs N and K
+ * state.  Requirements: M, N, K > 0; blocked layouts need 16-bit or 8-bit operands and the
+ * blocked operand's two dimensions to be multiples of 32; row-major BF16 needs N and K
  * to be multiples of 8, row-major FP32 needs N and K to be multiples of 4
  * (16-byte rows); BF16 output needs BF16 inputs.  batch > 1 (Section 2.1: the source tiles
  * of a batch-reduce GEMM need not be contiguous, the accumulation tile is C) needs
