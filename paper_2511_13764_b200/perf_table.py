@@ -39,7 +39,12 @@ def time_launch(launch, st, iters, flush, graph_pairs):
     graph of the flushes alone subtracted: CUDA-event stamps are a microsecond or two coarse on
     some boxes, the graph difference resolves a fraction of a microsecond, and the launches come
     without host gaps, as they would inside a captured pipeline."""
+    import time
     import torch
+    # a quarter of a second of idling first: a heavy row just before leaves the part power-throttled for
+    # a while, which a short FMA-bound row would otherwise inherit
+    torch.cuda.synchronize()
+    time.sleep(0.25)
     for _ in range(3):
         launch(st.cuda_stream)
     torch.cuda.synchronize()
