@@ -66,8 +66,9 @@ typedef enum {
     NK_S8 = 3, /* signed 8-bit integers: the Int8 dot product Section 5 names among the next packed types.  A is
                   row-major; B is NK_BLOCKED32 with four k per group (Section 2: "INT8 elements in groups of
                   four"): B[N/32][K/32][8][32][4], packed[k/4][n][k%4] = flat[k][n] inside each 32 x 32 block.
-                  The result is exact: INT32 accumulation of at most 2^17 - 1 products.  No epilogue, no beta,
-                  no batch, no K split; N and K multiples of 32 */
+                  The result is exact: INT32 accumulation of at most 2^17 - 1 products (K splits add their
+                  INT32 partial sums as integers).  No epilogue with an INT32 C, no beta, no batch; N and K
+                  multiples of 32 */
     NK_S32 = 4, /* signed 32-bit integers: the type of C for NK_S8 operands (and only for them).  NK_S8
                   operands may also have an NK_F32 C: the INT32 sum is converted (round to nearest even),
                   multiplied by desc.scale and given the epilogue (FP32 bias + ReLU) before the store */

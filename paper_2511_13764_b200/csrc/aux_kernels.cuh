@@ -84,7 +84,33 @@ struct ReduceParams {
     const void* bias;
     void* C;
     int f16;               // the 16-bit type (bias_bf16 / out_bf16) is IEEE binary16, not BF16
+    int int_partials;      // the partials are INT32 sums (INT8 operands): added as integers, exactly
+    int dequant;           // ... then converted to FP32 and multiplied by `scale` before the epilogue
+    float scale;
 };
+
+// Sum of the splits of four consecutive elements, in split order: FP32 adds, or exact INT32 adds (the
+// result then either keeps its integer bit pattern or becomes scale * sum in FP32).
+__device__ __forceinline__ float4 sum_partials(const float* first, size_t stride, int splits, int int_partials,
+                                               int dequant, float scale) {
+    if (!int_partials) {
+        float4 s = __ldcs(reinterpret_cast<const float4*>(first));
+        for (int sp = 1; sp < splits; ++sp) {
+            const float4 v = __ldcs(reinterpret_cast<const float4*>(first + sp * stride));
+            s.x += v.x; s.y += v.y; s.z += v.z; s.w += v.w;
+        }
+        return s;
+    }
+    int4 a = __ldcs(reinterpret_cast<const int4*>(first));
+    for (int sp = 1; sp < splits; ++sp) {
+        const int4 v = __ldcs(reinterpret_cast<const int4*>(first + sp * stride));
+        a.x += v.x; a.y += v.y; a.z += v.z; a.w += v.w;
+    }
+    if (dequant)
+        return make_float4(__int2float_rn(a.x) * scale, __int2float_rn(a.y) * scale, __int2float_rn(a.z) * scale,
+                           __int2float_rn(a.w) * scale);
+    return make_float4(__int_as_float(a.x), __int_as_float(a.y), __int_as_float(a.z), __int_as_float(a.w));
+}
 
 // C = epilogue(sum over splits, in split order): fixed order, so the result does
 // not depend on how CTAs were scheduled.  Four consecutive columns per thread.
@@ -100,11 +126,7 @@ __global__ void splitk_reduce_kernel(const ReduceParams p) {
         const size_t i = r / p.N, j = r - i * p.N;
         ce = g * per + ((i / 32 * (p.N / 32) + j / 32) * 32 + i % 32) * 32 + j % 32;
     }
-    float4 s = __ldcs(reinterpret_cast<const float4*>(p.partial + e));
-    for (int sp = 1; sp < p.splits; ++sp) {
-        const float4 v = __ldcs(reinterpret_cast<const float4*>(p.partial + sp * p.MN + e));
-        s.x += v.x; s.y += v.y; s.z += v.z; s.w += v.w;
-    }
+    float4 s = sum_partials(p.partial + e, p.MN, p.splits, p.int_partials, p.dequant, p.scale);
     if (p.beta) {
         if (p.out_bf16) {
             const uint2 w = *reinterpret_cast<const uint2*>(static_cast<const uint16_t*>(p.C) + ce);
@@ -148,6 +170,8 @@ struct TailReduceParams {
     const float* partial;       // [tail tile][split][tile_rows][tile_cols]
     const void* bias;
     void* C;
+    int int_partials, dequant;  // as in ReduceParams
+    float scale;
 };
 
 // Sums the K splits of the tail tiles (the last, partial wave of a large GEMM, see the pair
@@ -170,11 +194,7 @@ __global__ void tail_reduce_kernel(const TailReduceParams p) {
     if (i >= p.M || j >= p.N) return;
     const size_t slab = static_cast<size_t>(p.tile_rows) * p.tile_cols;
     const float* src = p.partial + static_cast<size_t>(blockIdx.y) * p.splits * slab + static_cast<size_t>(r) * p.tile_cols + c;
-    float4 s = __ldcs(reinterpret_cast<const float4*>(src));
-    for (int sp = 1; sp < p.splits; ++sp) {
-        const float4 v = __ldcs(reinterpret_cast<const float4*>(src + sp * slab));
-        s.x += v.x; s.y += v.y; s.z += v.z; s.w += v.w;
-    }
+    float4 s = sum_partials(src, slab, p.splits, p.int_partials, p.dequant, p.scale);
     const size_t ce = p.c_blocked ? ((static_cast<size_t>(i / 32) * (p.N / 32) + j / 32) * 32 + i % 32) * 32 + j % 32
                                   : static_cast<size_t>(i) * p.N + j;
     if (p.beta) {

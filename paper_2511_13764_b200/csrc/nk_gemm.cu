@@ -249,7 +249,6 @@ static void choose_umma(nk_gemm_s* p) {
                 int splits = forced_s > 0 ? forced_s : split_cands[si];
                 if (forced_s > 0 && si > 0) break;
                 if (splits > kb_total) splits = kb_total;
-                if (is_s8(d) && splits > 1) continue;   // INT32 partial sums have no reduce path: one unit per tile
                 if (forced_s == 0 && splits > 1) {
                     if (kb_total / splits < 4) continue;  // >= 4 k-blocks per split
                     if (static_cast<double>(splits) * desc_gemms(d) * d.M * d.N * 4.0 > 256.0 * 1024 * 1024) continue;
@@ -259,7 +258,7 @@ static void choose_umma(nk_gemm_s* p) {
             }
         }
     }
-    if (best.us >= 1e30) best = {false, 64, (forced_s > 0 && !is_s8(d)) ? forced_s : 1, 0.0};  // contradictory overrides
+    if (best.us >= 1e30) best = {false, 64, forced_s > 0 ? forced_s : 1, 0.0};  // contradictory overrides
     int splits = best.splits;
     if (splits > kb_total) splits = kb_total;
     if (splits < 1) splits = 1;
@@ -712,7 +711,7 @@ nk_status_t nk_gemm_create(const nk_gemm_desc_t* desc, nk_gemm_t* out) {
         if (d.beta != 0 || d.batch > 1) return NK_ERR_UNSUPPORTED;
         if (d.out_dtype == NK_S32 && d.epilogue != NK_EPI_NONE) return NK_ERR_UNSUPPORTED;
         if (d.out_dtype == NK_F32 && !(std::isfinite(d.scale) && d.scale != 0.0f)) return NK_ERR_INVALID_ARG;
-        if (d.flags & (NK_FLAG_REPACK_B | NK_FLAG_SEPARATE_REDUCE)) return NK_ERR_UNSUPPORTED;
+        if (d.flags & NK_FLAG_REPACK_B) return NK_ERR_UNSUPPORTED;
         const uint32_t fk = d.flags & NK_FLAG_KERNEL_MASK;
         if (fk == NK_FLAG_KERNEL_NAIVE || fk == NK_FLAG_KERNEL_SIMT) return NK_ERR_UNSUPPORTED;
         if (d.K >= (1ll << 17)) return NK_ERR_UNSUPPORTED;   // INT32 accumulation is exact below 2^17 terms
@@ -885,7 +884,7 @@ nk_status_t nk_gemm_create(const nk_gemm_desc_t* desc, nk_gemm_t* out) {
         // reduce kernel and the partials (FP32, written and read once).
         p->tail_from = -1;
         p->tail_splits = 0;
-        if (p->pair && p->splits == 1 && p->gemms == 1 && !(d.flags & NK_FLAG_NO_TAIL_SPLIT) && !is_s8(d)) {
+        if (p->pair && p->splits == 1 && p->gemms == 1 && !(d.flags & NK_FLAG_NO_TAIL_SPLIT)) {
             const int tiles = ceil_div(d.M, 2 * UMMA_BM) * ceil_div(d.N, p->bn);
             const int kb_total = p->batch * ceil_div(d.K, kblock(d));
             const int tail = tiles % p->max_pairs;
@@ -1099,7 +1098,8 @@ nk_status_t nk_gemm_run(nk_gemm_t p, const void* A, const void* B, const void* b
         const int tiles_m = ceil_div(d.M, 2 * UMMA_BM), tiles_n = ceil_div(d.N, p->bn);
         TailReduceParams tp = {static_cast<int>(d.M), static_cast<int>(d.N), 2 * UMMA_BM, p->bn, tiles_m, tiles_n, p->group_m,
                                p->tail_from, p->tail_splits, d.epilogue, (p->bias_f32 || is_8bit(d)) ? 0 : 1, is16(d.out_dtype), d.beta,
-                               d.layout_c == NK_BLOCKED32, d.in_dtype == NK_F16, partial, bias, C};
+                               d.layout_c == NK_BLOCKED32, d.in_dtype == NK_F16, partial, bias, C,
+                               is_s8(d) ? 1 : 0, (is_s8(d) && d.out_dtype == NK_F32) ? 1 : 0, d.scale};
         const int quads = 2 * UMMA_BM * p->bn / 4;
         dim3 grid(static_cast<unsigned>((quads + 255) / 256), static_cast<unsigned>(tiles_m * tiles_n - p->tail_from));
         tail_reduce_kernel<<<grid, 256, 0, st>>>(tp);
@@ -1109,7 +1109,8 @@ nk_status_t nk_gemm_run(nk_gemm_t p, const void* A, const void* B, const void* b
     if (p->splits > 1 && !p->cluster_reduce) {
         ReduceParams rp = {static_cast<size_t>(p->gemms) * d.M * d.N, static_cast<int>(d.N), p->splits, d.epilogue,
                            is16(d.in_dtype) && !p->bias_f32, is16(d.out_dtype), d.beta, d.layout_c == NK_BLOCKED32,
-                           static_cast<int>(d.M), partial, bias, C, d.in_dtype == NK_F16};
+                           static_cast<int>(d.M), partial, bias, C, d.in_dtype == NK_F16,
+                           is_s8(d) ? 1 : 0, (is_s8(d) && d.out_dtype == NK_F32) ? 1 : 0, d.scale};
         const size_t quads = rp.MN / 4;
         splitk_reduce_kernel<<<static_cast<unsigned>((quads + 255) / 256), 256, 0, st>>>(rp);
         e = cudaGetLastError();

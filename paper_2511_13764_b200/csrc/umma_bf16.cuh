@@ -154,7 +154,7 @@ __device__ __forceinline__ void umma_store_chunk(const UmmaParams& p, const CUte
 #pragma unroll
         for (int i = 0; i < 32; ++i) v[i] = 0u;
     }
-    if (p.dequant) {
+    if (p.dequant && !to_partial) {   // a K split's partial stays an INT32 sum; the reduce kernel converts
 #pragma unroll
         for (int i = 0; i < 32; ++i) v[i] = __float_as_uint(__int2float_rn(static_cast<int>(v[i])) * p.scale);
     }

@@ -27,8 +27,9 @@ def run_s8(M, N, K, flags=0, seed=1, A=None, B=None):
     Cbuf[:pad] = 7
     Cbuf[-pad:] = 7
     C = Cbuf[pad:pad + M * N]
-    assert plan.workspace_bytes == 0
-    plan.run(dA, dB, C, stream=torch.cuda.current_stream().cuda_stream)
+    wsb = plan.workspace_bytes            # K splits go through INT32 partials in the workspace
+    ws = torch.full((max(wsb, 16),), 0xFF, dtype=torch.uint8, device="cuda")
+    plan.run(dA, dB, C, workspace=ws if wsb else None, workspace_bytes=wsb, stream=torch.cuda.current_stream().cuda_stream)
     plan.check()
     torch.cuda.synchronize()
     assert torch.all(Cbuf[:pad] == 7) and torch.all(Cbuf[-pad:] == 7), "canary overwritten"
@@ -86,6 +87,51 @@ def test_s8_headline_shapes(i):
     lhs = got @ x
     rhs = A.reshape(w.M, w.K).astype(np.int64) @ bx
     assert np.array_equal(lhs, rhs)
+
+
+@pytest.mark.parametrize("mode", ["single", "pair"])
+@pytest.mark.parametrize("splits", [2, 3, 5])
+def test_s8_k_splits_add_integer_partials(splits, mode):
+    """K splits write INT32 partial sums to the workspace; the reduce kernel adds them as integers: still exact."""
+    M, N, K = 130, 160, 2080
+    A = nk_inputs.fill(7, nk_inputs.TENSOR_A, M * K, dtype="s8")
+    B = nk_inputs.fill(7, nk_inputs.TENSOR_B, K * N, dtype="s8")
+    plan = nk.Plan(M, N, K, in_dtype=nk.S8, out_dtype=nk.S32, layout_a=nk.ROW_MAJOR, layout_b=nk.BLOCKED32,
+                   flags=MODES[mode] | nk.flag_splitk(splits))
+    assert f"splitk{splits}" in plan.kernel_name and plan.workspace_bytes >= splits * M * N * 4 and plan.launches_per_run == 2
+    ws = torch.full((plan.workspace_bytes,), 0xFF, dtype=torch.uint8, device="cuda")
+    C = torch.full((M * N,), 12345, dtype=torch.int32, device="cuda")
+    plan.run(torch.from_numpy(A).cuda(), torch.from_numpy(B).cuda(), C, workspace=ws, workspace_bytes=plan.workspace_bytes,
+             stream=torch.cuda.current_stream().cuda_stream)
+    plan.check()
+    assert np.array_equal(C.cpu().numpy().astype(np.int64).reshape(M, N), oracle.gemm_s8(M, N, K, A, B, layout_b=oracle.BLOCKED32))
+
+
+@pytest.mark.parametrize("dequant", [False, True])
+def test_s8_tail_wave_split(dequant):
+    """More 256 x 256 tiles than CTA pairs: the last wave's tiles are cut along K, their INT32 partials summed
+    exactly by the tail reduce kernel (and scaled, biased and rectified there for an FP32 C)."""
+    M, N, K = 2304, 2304, 1024
+    A = nk_inputs.fill(8, nk_inputs.TENSOR_A, M * K, dtype="s8")
+    B = nk_inputs.fill(8, nk_inputs.TENSOR_B, K * N, dtype="s8")
+    bias = nk_inputs.fill(8, nk_inputs.TENSOR_BIAS, N, "normal", 50.0, "f32") if dequant else None
+    scale = 1e-4
+    plan = nk.Plan(M, N, K, in_dtype=nk.S8, out_dtype=nk.F32 if dequant else nk.S32, layout_a=nk.ROW_MAJOR,
+                   layout_b=nk.BLOCKED32, epilogue=nk.EPI_BIAS_RELU if dequant else nk.EPI_NONE, scale=scale,
+                   flags=nk.FLAG_CTA_PAIR | nk.flag_tile_n(4) | nk.flag_tail_split(2))
+    assert "_tail2" in plan.kernel_name
+    ws = torch.empty(plan.workspace_bytes, dtype=torch.uint8, device="cuda")
+    C = torch.empty(M * N, dtype=torch.float32 if dequant else torch.int32, device="cuda")
+    plan.run(torch.from_numpy(A).cuda(), torch.from_numpy(B).cuda(), C, bias=torch.from_numpy(bias).cuda() if dequant else None,
+             workspace=ws, workspace_bytes=plan.workspace_bytes, stream=torch.cuda.current_stream().cuda_stream)
+    plan.check()
+    rows = nk_inputs.stratified_rows(8, M, 96)
+    got = C.cpu().numpy().reshape(M, N)[rows]
+    if dequant:
+        want, S = oracle.gemm_s8_scaled(M, N, K, A, B, scale, bias=bias, layout_b=oracle.BLOCKED32, rows=rows, relu=True)
+        assert np.all(np.abs(got.astype(np.float64) - want) <= DEQ_TOL * S)
+    else:
+        assert np.array_equal(got.astype(np.int64), oracle.gemm_s8(M, N, K, A, B, layout_b=oracle.BLOCKED32, rows=rows))
 
 
 # ---------------------------------------------------------------- quantised layer: C = scale * (A.B) (+ FP32 bias, ReLU) in FP32
@@ -167,6 +213,3 @@ def test_s8_rejects_what_it_cannot_do():
         nk.Plan(64, 48, 64, **ok)          # N not a multiple of 32
     with pytest.raises(nk.NkError):
         nk.Plan(64, 64, 64, in_dtype=nk.BF16, out_dtype=nk.S32)   # INT32 C belongs to INT8 operands
-    # a forced K split is ignored: INT32 partial sums have no reduce path
-    p = nk.Plan(128, 64, 4096, flags=nk.flag_splitk(4), **ok)
-    assert "splitk1" in p.kernel_name and p.workspace_bytes == 0
