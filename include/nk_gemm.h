@@ -26,6 +26,7 @@
  *                  packed[k/2][n][k%2] = flat[k][n] (16-bit operands);
  *                  B[N/32][K/32][8][32][4], packed[k/4][n][k%4] = flat[k][n] (8-bit operands:
  *                  Section 2, "INT8 elements in groups of four").
+ *   NK_TRANSPOSED  (layout_b only) Bt[N][K]: B kept as its transpose, K contiguous.
  * C is row-major [M][N] unless desc.layout_c asks for the blocked form; bias is [N] in the
  * operand type (FP32 for 8-bit operands).
  *
@@ -79,7 +80,14 @@ typedef enum {
                     lists; A row-major, B NK_BLOCKED32 with four k per group like NK_S8, FP32 accumulation, FP32 C,
                     FP32 bias; N and K multiples of 32; no batch */
 } nk_dtype_t;
-typedef enum { NK_ROW_MAJOR = 0, NK_BLOCKED32 = 1 } nk_layout_t;
+typedef enum {
+    NK_ROW_MAJOR = 0,
+    NK_BLOCKED32 = 1,
+    NK_TRANSPOSED = 2 /* layout_b only: B is stored transposed, Bt[N][K] with K contiguous (the way a linear layer's
+                         weight [out][in] is usually kept).  16-bit and 8-bit operands; K a multiple of 16, N of 8;
+                         no batch.  Not one of the paper's layouts (flat [K][N] and VNNI-blocked): on this hardware
+                         it is the operand form the tensor core reads without any re-layout */
+} nk_layout_t;
 typedef enum { NK_EPI_NONE = 0, NK_EPI_BIAS_RELU = 1 } nk_epilogue_t;
 
 /* desc.flags: 0 lets the plan choose.  The rest are tuning/debug overrides. */

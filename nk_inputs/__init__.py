@@ -165,6 +165,7 @@ class Workload:
     in_dtype: str = "bf16"          # "f32" | "bf16" | "f16" | "s8"
     out_dtype: str = "f32"          # "f32" | "bf16" | "f16" (a 16-bit output has the input's type) | "s32" (INT8 operands)
     layout: str = "row"             # "row" | "blocked32" (A and B both) | "b_blocked32" (A row-major, B blocked)
+                                    # | "b_transposed" (A row-major, B kept as Bt[N][K])
     epilogue: str = "none"          # "none" | "bias_relu"
     dist_a: tuple = ("uniform", 1.0)
     dist_b: tuple = ("uniform", 1.0)
@@ -262,6 +263,17 @@ def fp8_set() -> list:
         Workload("x_e5m2_4096", 4096, 4096, 4096, "e5m2", "f32", layout="b_blocked32", seed=9018),
         Workload("x_e4m3_mlp_512x4096x4096", 512, 4096, 4096, "e4m3", "f32", layout="b_blocked32", epilogue="bias_relu",
                  dist_a=("normal", 1.0), dist_b=("normal", 0.02), seed=9019),
+    ]
+
+
+def bt_set() -> list:
+    """B kept as its transpose Bt[N][K] (the form a linear layer's weight usually has): the large square GEMM
+    in BF16, INT8 and E4M3."""
+    return [
+        Workload("xt_bf16_8192", 8192, 8192, 8192, "bf16", "f32", layout="b_transposed", seed=9517),
+        Workload("xt_s8_8192", 8192, 8192, 8192, "s8", "s32", layout="b_transposed", seed=9518),
+        Workload("xt_e4m3_8192", 8192, 8192, 8192, "e4m3", "f32", layout="b_transposed", seed=9519),
+        Workload("xt_s8_4096", 4096, 4096, 4096, "s8", "s32", layout="b_transposed", seed=9520),
     ]
 
 

@@ -19,7 +19,7 @@ _LIB = os.path.join(_HERE, "libnk_oracle.so")
 
 F32, BF16, F16 = 0, 1, 2
 E4M3, E5M2 = 5, 6
-ROW, BLOCKED32 = 0, 1
+ROW, BLOCKED32, TRANSPOSED = 0, 1, 2
 EPI_NONE, EPI_BIAS_RELU = 0, 1
 ACC_F64, ACC_F32_SEQ = 0, 1
 
@@ -248,7 +248,7 @@ def gemm_workload(w, A, B, bias, rows=None, cols=None, **kw):
     """Oracle on an ``nk_inputs.Workload``-shaped object (duck-typed: M, N, K,
     in_dtype, layout, epilogue attributes)."""
     lay_a = BLOCKED32 if w.layout == "blocked32" else ROW
-    lay_b = BLOCKED32 if w.layout in ("blocked32", "b_blocked32") else ROW
+    lay_b = BLOCKED32 if w.layout in ("blocked32", "b_blocked32") else TRANSPOSED if w.layout == "b_transposed" else ROW
     return gemm(w.M, w.N, w.K, A, B, bias,
                 in_dtype={"f32": F32, "bf16": BF16, "f16": F16, "e4m3": E4M3, "e5m2": E5M2}[w.in_dtype],
                 layout_a=lay_a, layout_b=lay_b,

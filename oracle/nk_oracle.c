@@ -18,7 +18,8 @@
  * exactly.  y is returned unrounded, as double; a BF16- or FP16-storing
  * implementation rounds once afterwards.
  *
- * Layouts: row-major A[M][K], B[K][N]; or 32x32-blocked with the VNNI-2
+ * Layouts: row-major A[M][K], B[K][N] (B may also be kept as its transpose Bt[N][K], an
+ * indexing variant of the same matrix); or 32x32-blocked with the VNNI-2
  * interleave of Figure 1 inside each B block:
  *     A_blk[M/32][K/32][32][32]         (m-block, k-block, m-in-block, k-in-block)
  *     B_blk[N/32][K/32][16][32][2]      (n-block, k-block, k-pair, n-in-block, k-parity)
@@ -42,7 +43,7 @@
 #include <string.h>
 
 enum { NKO_F32 = 0, NKO_BF16 = 1, NKO_F16 = 2, NKO_E4M3 = 5, NKO_E5M2 = 6 };
-enum { NKO_ROW = 0, NKO_BLOCKED32 = 1 };
+enum { NKO_ROW = 0, NKO_BLOCKED32 = 1, NKO_TRANSPOSED = 2 };   /* TRANSPOSED: layout_b only, Bt[N][K] */
 enum { NKO_EPI_NONE = 0, NKO_EPI_BIAS_RELU = 1 };
 enum { NKO_ACC_F64 = 0, NKO_ACC_F32_SEQ = 1 };
 
@@ -133,6 +134,7 @@ static int is_8bit(int32_t dtype) { return dtype == NKO_E4M3 || dtype == NKO_E5M
 
 static int64_t b_index(const nko_desc_t* d, int64_t k, int64_t j) {
     if (d->layout_b == NKO_ROW) return k * d->N + j;
+    if (d->layout_b == NKO_TRANSPOSED) return j * d->K + k;   /* B kept as its transpose, K contiguous */
     if (is_8bit(d->in_dtype))   /* 8-bit elements are packed in groups of four (Section 2) */
         return ((((j / 32) * (d->K / 32) + k / 32) * 8 + (k % 32) / 4) * 32 + j % 32) * 4 + k % 4;
     return ((((j / 32) * (d->K / 32) + k / 32) * 16 + (k % 32) / 2) * 32 + j % 32) * 2 + k % 2;
@@ -291,6 +293,7 @@ void nko_unpack_vnni4(const int8_t* packed, int64_t K, int64_t N, int8_t* flat) 
 /* Storage index of logical element (k,j) of an INT8 B operand. */
 int64_t nko_b_index_s8(int64_t K, int64_t N, int32_t layout_b, int64_t k, int64_t j) {
     if (layout_b == NKO_ROW) return k * N + j;
+    if (layout_b == NKO_TRANSPOSED) return j * K + k;
     return ((((j / 32) * (K / 32) + k / 32) * 8 + (k % 32) / 4) * 32 + j % 32) * 4 + k % 4;
 }
 
@@ -321,7 +324,7 @@ static void* worker_s8(void* arg) {
 int nko_gemm_s8(int64_t M, int64_t N, int64_t K, int32_t layout_b, const int8_t* A, const int8_t* B,
                 const int64_t* rows, int64_t nrows, int64_t* Y, int nthreads) {
     if (M <= 0 || N <= 0 || K <= 0 || !A || !B || !Y) return -1;
-    if (layout_b != NKO_ROW && (layout_b != NKO_BLOCKED32 || N % 32 || K % 32)) return -1;
+    if (layout_b != NKO_ROW && layout_b != NKO_TRANSPOSED && (layout_b != NKO_BLOCKED32 || N % 32 || K % 32)) return -1;
     const int64_t nr = rows ? nrows : M;
     if (rows)
         for (int64_t r = 0; r < nr; ++r)

@@ -11,7 +11,7 @@ import os
 from . import _build
 
 F32, BF16, F16, S8, S32, E4M3, E5M2 = 0, 1, 2, 3, 4, 5, 6
-ROW_MAJOR, BLOCKED32 = 0, 1
+ROW_MAJOR, BLOCKED32, TRANSPOSED = 0, 1, 2
 EPI_NONE, EPI_BIAS_RELU = 0, 1
 FLAG_KERNEL_NAIVE, FLAG_KERNEL_SIMT, FLAG_KERNEL_UMMA = 0x1, 0x2, 0x3
 FLAG_REPACK_B = 0x10
@@ -201,7 +201,7 @@ def plan_for(w, device=0, flags=0) -> Plan:
     """Plan for a workload record with M, N, K, in_dtype ("f32"/"bf16"/"f16"/"s8"), out_dtype,
     layout ("row"/"blocked32") and epilogue ("none"/"bias_relu") attributes."""
     lay_a = BLOCKED32 if w.layout == "blocked32" else ROW_MAJOR
-    lay_b = BLOCKED32 if w.layout in ("blocked32", "b_blocked32") else ROW_MAJOR
+    lay_b = BLOCKED32 if w.layout in ("blocked32", "b_blocked32") else TRANSPOSED if w.layout == "b_transposed" else ROW_MAJOR
     types = {"f32": F32, "bf16": BF16, "f16": F16, "s8": S8, "s32": S32, "e4m3": E4M3, "e5m2": E5M2}
     return Plan(w.M, w.N, w.K, in_dtype=types[w.in_dtype], out_dtype=types[w.out_dtype],
                 layout_a=lay_a, layout_b=lay_b,

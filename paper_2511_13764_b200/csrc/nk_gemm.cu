@@ -44,6 +44,7 @@ struct nk_gemm_s {
     bool b_vnni_inkernel;  // blocked B re-laid inside the GEMM kernel
     bool b_repack;         // blocked B unpacked to row-major scratch first
     bool b_3d;             // B tensor map is the 3-D slab view
+    bool b_kmajor;         // B is stored transposed, Bt[N][K]: K-major tiles by TMA, like A
     bool cluster_reduce;   // K splits of a tile = the CTAs of one cluster; partial sums meet in shared memory
     int tail_from, tail_splits;   // pair kernel: tiles >= tail_from (the last, partial wave) are cut into K splits; -1: off
     // SIMT
@@ -386,7 +387,23 @@ static nk_status_t encode_maps(nk_gemm_s* p, const void* A, const void* B) {
         snprintf(p->cuda_err, sizeof(p->cuda_err), "cuTensorMapEncodeTiled(A) failed: %d", (int)r);
         return NK_ERR_CUDA;
     }
-    if (!p->b_vnni_inkernel) {
+    if (p->b_kmajor) {
+        // B stored transposed, Bt[batch][N][K] (K contiguous): (k, n, item), one box of 128 bytes of k by
+        // the columns a CTA covers, K-major in shared memory exactly like A's tile
+        const int cols = p->pair ? p->bn / 2 : p->bn;
+        cuuint64_t dims[3] = {static_cast<cuuint64_t>(d.K), static_cast<cuuint64_t>(d.N),
+                              static_cast<cuuint64_t>(p->batch * p->gemms)};
+        cuuint64_t strides[2] = {static_cast<cuuint64_t>(d.K) * esz, static_cast<cuuint64_t>(p->stride_b) * esz};
+        cuuint32_t box[3] = {static_cast<cuuint32_t>(kblock(d)), static_cast<cuuint32_t>(cols), 1};
+        cuuint32_t es[3] = {1, 1, 1};
+        r = p->encode(&p->tmap_b, half_type, 3, const_cast<void*>(B), dims, strides,
+                      box, es, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+                      CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+        if (r != CUDA_SUCCESS) {
+            snprintf(p->cuda_err, sizeof(p->cuda_err), "cuTensorMapEncodeTiled(B transposed) failed: %d", (int)r);
+            return NK_ERR_CUDA;
+        }
+    } else if (!p->b_vnni_inkernel) {
         // B row-major [K][N], N contiguous.  When N is a multiple of 64 the map is the 3-D view
         // (n within a 64-column slab, k, slab): one box brings all the slabs of a stage, each
         // as 64 k-rows of 128 B.  Otherwise 64 (n) x 64 (k) boxes, one per slab.
@@ -478,18 +495,18 @@ static cudaError_t launch_umma_t(nk_gemm_s* p, const UmmaParams& up, int grid, c
 
 static cudaError_t launch_umma(nk_gemm_s* p, const UmmaParams& up, int grid, cudaStream_t st) {
     const bool v = p->b_vnni_inkernel;
-    if (is_s8(p->d)) {   // 8-bit operands: B is always blocked and re-laid in the kernel
+    if (is_s8(p->d)) {   // 8-bit operands: B blocked and re-laid in the kernel, or stored transposed
         switch (p->bn) {
-            case 256: return launch_umma_t<256, 4, true, 1>(p, up, grid, st);
-            case 128: return launch_umma_t<128, 6, true, 1>(p, up, grid, st);
-            default:  return launch_umma_t<64, 8, true, 1>(p, up, grid, st);
+            case 256: return v ? launch_umma_t<256, 4, true, 1>(p, up, grid, st) : launch_umma_t<256, 4, false, 1>(p, up, grid, st);
+            case 128: return v ? launch_umma_t<128, 6, true, 1>(p, up, grid, st) : launch_umma_t<128, 6, false, 1>(p, up, grid, st);
+            default:  return v ? launch_umma_t<64, 8, true, 1>(p, up, grid, st) : launch_umma_t<64, 8, false, 1>(p, up, grid, st);
         }
     }
     if (is_f8(p->d)) {
         switch (p->bn) {
-            case 256: return launch_umma_t<256, 4, true, 2>(p, up, grid, st);
-            case 128: return launch_umma_t<128, 6, true, 2>(p, up, grid, st);
-            default:  return launch_umma_t<64, 8, true, 2>(p, up, grid, st);
+            case 256: return v ? launch_umma_t<256, 4, true, 2>(p, up, grid, st) : launch_umma_t<256, 4, false, 2>(p, up, grid, st);
+            case 128: return v ? launch_umma_t<128, 6, true, 2>(p, up, grid, st) : launch_umma_t<128, 6, false, 2>(p, up, grid, st);
+            default:  return v ? launch_umma_t<64, 8, true, 2>(p, up, grid, st) : launch_umma_t<64, 8, false, 2>(p, up, grid, st);
         }
     }
     switch (p->bn) {
@@ -588,8 +605,14 @@ static cudaError_t launch_pair_t(nk_gemm_s* p, const UmmaParams& up, int pairs, 
 
 static cudaError_t launch_pair(nk_gemm_s* p, const UmmaParams& up, int pairs, cudaStream_t st) {
     const bool v = p->b_vnni_inkernel;
-    if (is_s8(p->d)) return p->bn == 256 ? launch_pair_t<256, 6, true, 1>(p, up, pairs, st) : launch_pair_t<128, 8, true, 1>(p, up, pairs, st);
-    if (is_f8(p->d)) return p->bn == 256 ? launch_pair_t<256, 6, true, 2>(p, up, pairs, st) : launch_pair_t<128, 8, true, 2>(p, up, pairs, st);
+    if (is_s8(p->d)) {
+        if (p->bn == 256) return v ? launch_pair_t<256, 6, true, 1>(p, up, pairs, st) : launch_pair_t<256, 6, false, 1>(p, up, pairs, st);
+        return v ? launch_pair_t<128, 8, true, 1>(p, up, pairs, st) : launch_pair_t<128, 8, false, 1>(p, up, pairs, st);
+    }
+    if (is_f8(p->d)) {
+        if (p->bn == 256) return v ? launch_pair_t<256, 6, true, 2>(p, up, pairs, st) : launch_pair_t<256, 6, false, 2>(p, up, pairs, st);
+        return v ? launch_pair_t<128, 8, true, 2>(p, up, pairs, st) : launch_pair_t<128, 8, false, 2>(p, up, pairs, st);
+    }
     if (p->bn == 256) return v ? launch_pair_t<256, 6, true>(p, up, pairs, st) : launch_pair_t<256, 6, false>(p, up, pairs, st);
     return v ? launch_pair_t<128, 8, true>(p, up, pairs, st) : launch_pair_t<128, 8, false>(p, up, pairs, st);
 }
@@ -639,15 +662,25 @@ static cudaError_t prepare_umma_attrs() {
     if ((e = allow_smem(umma_bf16_pair_kernel<128, 8, false, true>, pair_smem_bytes(128, 8))) != cudaSuccess) return e;
     if ((e = allow_smem(umma_bf16_pair_kernel<128, 8, true, true>, pair_smem_bytes(128, 8))) != cudaSuccess) return e;
     if ((e = allow_smem(umma_bf16_kernel<256, 4, true, false, 1>, umma_smem_bytes(256, 4))) != cudaSuccess) return e;
+    if ((e = allow_smem(umma_bf16_kernel<256, 4, false, false, 1>, umma_smem_bytes(256, 4))) != cudaSuccess) return e;
     if ((e = allow_smem(umma_bf16_kernel<256, 4, true, false, 2>, umma_smem_bytes(256, 4))) != cudaSuccess) return e;
+    if ((e = allow_smem(umma_bf16_kernel<256, 4, false, false, 2>, umma_smem_bytes(256, 4))) != cudaSuccess) return e;
     if ((e = allow_smem(umma_bf16_kernel<128, 6, true, false, 1>, umma_smem_bytes(128, 6))) != cudaSuccess) return e;
+    if ((e = allow_smem(umma_bf16_kernel<128, 6, false, false, 1>, umma_smem_bytes(128, 6))) != cudaSuccess) return e;
     if ((e = allow_smem(umma_bf16_kernel<128, 6, true, false, 2>, umma_smem_bytes(128, 6))) != cudaSuccess) return e;
+    if ((e = allow_smem(umma_bf16_kernel<128, 6, false, false, 2>, umma_smem_bytes(128, 6))) != cudaSuccess) return e;
     if ((e = allow_smem(umma_bf16_kernel<64, 8, true, false, 1>, umma_smem_bytes(64, 8))) != cudaSuccess) return e;
+    if ((e = allow_smem(umma_bf16_kernel<64, 8, false, false, 1>, umma_smem_bytes(64, 8))) != cudaSuccess) return e;
     if ((e = allow_smem(umma_bf16_kernel<64, 8, true, false, 2>, umma_smem_bytes(64, 8))) != cudaSuccess) return e;
+    if ((e = allow_smem(umma_bf16_kernel<64, 8, false, false, 2>, umma_smem_bytes(64, 8))) != cudaSuccess) return e;
     if ((e = allow_smem(umma_bf16_pair_kernel<256, 6, true, false, 1>, pair_smem_bytes(256, 6))) != cudaSuccess) return e;
+    if ((e = allow_smem(umma_bf16_pair_kernel<256, 6, false, false, 1>, pair_smem_bytes(256, 6))) != cudaSuccess) return e;
     if ((e = allow_smem(umma_bf16_pair_kernel<256, 6, true, false, 2>, pair_smem_bytes(256, 6))) != cudaSuccess) return e;
+    if ((e = allow_smem(umma_bf16_pair_kernel<256, 6, false, false, 2>, pair_smem_bytes(256, 6))) != cudaSuccess) return e;
     if ((e = allow_smem(umma_bf16_pair_kernel<128, 8, true, false, 1>, pair_smem_bytes(128, 8))) != cudaSuccess) return e;
+    if ((e = allow_smem(umma_bf16_pair_kernel<128, 8, false, false, 1>, pair_smem_bytes(128, 8))) != cudaSuccess) return e;
     if ((e = allow_smem(umma_bf16_pair_kernel<128, 8, true, false, 2>, pair_smem_bytes(128, 8))) != cudaSuccess) return e;
+    if ((e = allow_smem(umma_bf16_pair_kernel<128, 8, false, false, 2>, pair_smem_bytes(128, 8))) != cudaSuccess) return e;
     return cudaSuccess;
 }
 
@@ -697,7 +730,7 @@ nk_status_t nk_gemm_create(const nk_gemm_desc_t* desc, nk_gemm_t* out) {
     if (is_f8(d)) {
         // 8-bit floating-point operands: A row-major, B packed in groups of four inside 32 x 32 blocks, FP32 C
         if (d.out_dtype != NK_F32) return NK_ERR_INVALID_ARG;
-        if (d.layout_a != NK_ROW_MAJOR || d.layout_b != NK_BLOCKED32 || d.layout_c != NK_ROW_MAJOR) return NK_ERR_UNSUPPORTED;
+        if (d.layout_a != NK_ROW_MAJOR || d.layout_b == NK_ROW_MAJOR || d.layout_c != NK_ROW_MAJOR) return NK_ERR_UNSUPPORTED;
         if (d.batch > 1) return NK_ERR_UNSUPPORTED;
         if (d.flags & NK_FLAG_REPACK_B) return NK_ERR_UNSUPPORTED;
         const uint32_t fk = d.flags & NK_FLAG_KERNEL_MASK;
@@ -707,7 +740,7 @@ nk_status_t nk_gemm_create(const nk_gemm_desc_t* desc, nk_gemm_t* out) {
         // the Int8 dot product: A row-major, B packed in groups of four inside 32 x 32 blocks; C is the exact
         // INT32 sum, or FP32 = scale * sum with the epilogue (quantised layer)
         if (d.out_dtype != NK_S32 && d.out_dtype != NK_F32) return NK_ERR_INVALID_ARG;
-        if (d.layout_a != NK_ROW_MAJOR || d.layout_b != NK_BLOCKED32 || d.layout_c != NK_ROW_MAJOR) return NK_ERR_UNSUPPORTED;
+        if (d.layout_a != NK_ROW_MAJOR || d.layout_b == NK_ROW_MAJOR || d.layout_c != NK_ROW_MAJOR) return NK_ERR_UNSUPPORTED;
         if (d.beta != 0 || d.batch > 1) return NK_ERR_UNSUPPORTED;
         if (d.out_dtype == NK_S32 && d.epilogue != NK_EPI_NONE) return NK_ERR_UNSUPPORTED;
         if (d.out_dtype == NK_F32 && !(std::isfinite(d.scale) && d.scale != 0.0f)) return NK_ERR_INVALID_ARG;
@@ -717,7 +750,13 @@ nk_status_t nk_gemm_create(const nk_gemm_desc_t* desc, nk_gemm_t* out) {
         if (d.K >= (1ll << 17)) return NK_ERR_UNSUPPORTED;   // INT32 accumulation is exact below 2^17 terms
     }
     if (d.layout_a != NK_ROW_MAJOR && d.layout_a != NK_BLOCKED32) return NK_ERR_INVALID_ARG;
-    if (d.layout_b != NK_ROW_MAJOR && d.layout_b != NK_BLOCKED32) return NK_ERR_INVALID_ARG;
+    if (d.layout_b != NK_ROW_MAJOR && d.layout_b != NK_BLOCKED32 && d.layout_b != NK_TRANSPOSED) return NK_ERR_INVALID_ARG;
+    if (d.layout_b == NK_TRANSPOSED) {
+        // Bt[N][K]: 16-bit and 8-bit operands (the tensor-core kernels); rows of K elements must be 16-byte multiples
+        if (d.in_dtype == NK_F32) return NK_ERR_UNSUPPORTED;
+        if ((d.flags & NK_FLAG_KERNEL_MASK) == NK_FLAG_KERNEL_NAIVE || (d.flags & NK_FLAG_REPACK_B)) return NK_ERR_UNSUPPORTED;
+        if (d.K % 16 || d.N % 8) return NK_ERR_MISALIGNED;
+    }
     if (d.epilogue != NK_EPI_NONE && d.epilogue != NK_EPI_BIAS_RELU) return NK_ERR_INVALID_ARG;
     if (is16(d.out_dtype) && d.in_dtype != d.out_dtype) return NK_ERR_INVALID_ARG;   // a 16-bit C has the operands' type
     const bool blocked = d.layout_a == NK_BLOCKED32 || d.layout_b == NK_BLOCKED32;
@@ -730,7 +769,7 @@ nk_status_t nk_gemm_create(const nk_gemm_desc_t* desc, nk_gemm_t* out) {
     const int64_t str_a = d.stride_a > 0 ? d.stride_a : d.M * d.K;
     const int64_t str_b = d.stride_b > 0 ? d.stride_b : d.K * d.N;
     if (nbatch > 1) {
-        if (blocked) return NK_ERR_UNSUPPORTED;          // batch-reduce: row-major operands only
+        if (blocked || d.layout_b == NK_TRANSPOSED) return NK_ERR_UNSUPPORTED;          // batch-reduce: row-major operands only
         if (nbatch > 65535 || nbatch * d.K >= (1ll << 24)) return NK_ERR_UNSUPPORTED;
         const int64_t gran = is16(d.in_dtype) ? 8 : 4;
         if (str_a % gran || str_b % gran) return NK_ERR_MISALIGNED;
@@ -861,6 +900,7 @@ nk_status_t nk_gemm_create(const nk_gemm_desc_t* desc, nk_gemm_t* out) {
             p->b_repack = (d.flags & NK_FLAG_REPACK_B) != 0;
             p->b_vnni_inkernel = !p->b_repack;
         }
+        p->b_kmajor = d.layout_b == NK_TRANSPOSED;
         if (p->pair) {
             const bool v = p->b_vnni_inkernel;
             int n = 0;
@@ -916,7 +956,7 @@ nk_status_t nk_gemm_create(const nk_gemm_desc_t* desc, nk_gemm_t* out) {
         snprintf(p->name, sizeof(p->name), "umma_bf16_%s%dx%d_s%d_splitk%d%s%s%s",
                  p->pair ? "pair_256x" : "128x", p->bn, kblock(d), p->stages,
                  p->splits, p->cluster_reduce ? "_cluster" : "", d.layout_a == NK_BLOCKED32 ? "_ablk" : "",
-                 p->b_vnni_inkernel ? "_bvnni" : (p->b_repack ? "_brepack" : ""));
+                 p->b_vnni_inkernel ? "_bvnni" : p->b_repack ? "_brepack" : p->b_kmajor ? "_bt" : "");
     }
     if (p->batch > 1 || p->gemms > 1 || d.beta) {
         const size_t len = strlen(p->name);
@@ -1063,9 +1103,10 @@ nk_status_t nk_gemm_run(nk_gemm_t p, const void* A, const void* B, const void* b
         up.group_m = p->group_m;
         up.a_blocked = d.layout_a == NK_BLOCKED32;
         up.b_3d = p->b_3d ? 1 : 0;
+        up.b_kmajor = p->b_kmajor ? 1 : 0;
         up.epilogue = d.epilogue;
         up.out_bf16 = is16(d.out_dtype);
-        up.idesc = make_idesc(p->pair ? 2 * UMMA_BM : UMMA_BM, p->bn, !p->b_vnni_inkernel, d.in_dtype == NK_F16, is_s8(d),
+        up.idesc = make_idesc(p->pair ? 2 * UMMA_BM : UMMA_BM, p->bn, !p->b_vnni_inkernel && !p->b_kmajor, d.in_dtype == NK_F16, is_s8(d),
                               d.in_dtype == NK_E4M3 ? 0 : d.in_dtype == NK_E5M2 ? 1 : -1);
         up.f16 = d.in_dtype == NK_F16;
         up.bias = bias;

@@ -57,6 +57,7 @@ struct UmmaParams {
     int group_m;        // raster: this many M tiles sweep N together
     int a_blocked;      // A tensor map is the 4-D blocked view
     int b_3d;           // B tensor map is the 3-D (n-in-slab, k, slab) view: one box per stage
+    int b_kmajor;       // B is stored transposed, Bt[N][K]: its tiles are K-major like A's, one box per stage
     int epilogue;       // 0 none, 1 bias + ReLU
     int out_bf16;       // C is 16 bits wide (the operands' type), else FP32
     int f16;            // the 16-bit type of A, B, bias (and C) is IEEE binary16 instead of BF16
@@ -571,6 +572,7 @@ umma_bf16_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_consta
         // addresses advance by adds and the layout decisions are taken outside the loops.
         const bool a_blk = p.a_blocked != 0;
         const bool b3d = p.b_3d != 0;
+        const bool b_kmajor = p.b_kmajor != 0;
         int stage = 0;
         uint32_t phase = 0;
         uint32_t sa = smem_base, fb = full_bar(0);
@@ -610,6 +612,8 @@ umma_bf16_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_consta
                         // the stage's blocks as they are; warps 6-9 re-lay them in place
                         mbar_arrive_expect_tx(raw_bar(stage), B_STAGE);
                         tma_load_3d(sb, &tmap_b, raw_bar(stage), 0, kbl * (UMMA_BK / 2), col0 >> 5);
+                    } else if (b_kmajor) {
+                        tma_load_3d(sb, &tmap_b, fb, kx, col0, ib);   // BN rows (n) of 128 bytes of k
                     } else {
                         if (b3d) {
                             tma_load_4d(sb, &tmap_b, fb, 0, kx, col0 >> 6, ib);
@@ -645,15 +649,16 @@ umma_bf16_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_consta
         //   A blocked: two K-major slabs of 32 k (8192 B apart), 64-byte swizzle, 8-row groups
         //     512 B apart; k-steps at 0, 32 B, 8192 B, 8192 + 32 B.
         //   B row-major [K][N]: N-major, 64-column atoms 8192 B apart (leading), 8-k groups
-        //     1024 B apart (stride); k-steps 2048 B apart.  B re-laid from VNNI: K-major like A.
+        //     1024 B apart (stride); k-steps 2048 B apart.  B re-laid from VNNI, or stored transposed: K-major like A.
         const bool a_blk = p.a_blocked != 0;
         const uint64_t da0 = a_blk ? make_smem_desc(smem_base, 16, 512, 4) : make_smem_desc(smem_base, 16, 1024, 2);
-        const uint64_t db0 = B_VNNI ? make_smem_desc(smem_base + UMMA_A_STAGE_BYTES, 16, 1024, 2)
-                                    : make_smem_desc(smem_base + UMMA_A_STAGE_BYTES, 8192, 1024, 2);
+        const bool b_k = B_VNNI || p.b_kmajor != 0;
+        const uint64_t db0 = b_k ? make_smem_desc(smem_base + UMMA_A_STAGE_BYTES, 16, 1024, 2)
+                                 : make_smem_desc(smem_base + UMMA_A_STAGE_BYTES, 8192, 1024, 2);
         const uint32_t a_hi = static_cast<uint32_t>(da0 >> 32), b_hi = static_cast<uint32_t>(db0 >> 32);
         const uint32_t a_lo0 = static_cast<uint32_t>(da0), b_lo0 = static_cast<uint32_t>(db0);
         const uint32_t a_s1 = 2u, a_s2 = a_blk ? 512u : 4u, a_s3 = a_blk ? 514u : 6u;
-        constexpr uint32_t b_s = B_VNNI ? 2u : 128u;
+        const uint32_t b_s = b_k ? 2u : 128u, b_s2 = 2 * b_s, b_s3 = 3 * b_s;
         constexpr uint32_t STAGE16 = STAGE >> 4;
         const uint32_t idesc = p.idesc;
         int stage = 0;
@@ -686,8 +691,8 @@ umma_bf16_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_consta
                     const uint32_t a_lo = a_lo0 + soff, b_lo = b_lo0 + soff;
                     umma_lohi<KIND>(d_tmem, a_lo, a_hi, b_lo, b_hi, idesc, accumulate);
                     umma_lohi<KIND>(d_tmem, a_lo + a_s1, a_hi, b_lo + b_s, b_hi, idesc, 1u);
-                    umma_lohi<KIND>(d_tmem, a_lo + a_s2, a_hi, b_lo + 2 * b_s, b_hi, idesc, 1u);
-                    umma_lohi<KIND>(d_tmem, a_lo + a_s3, a_hi, b_lo + 3 * b_s, b_hi, idesc, 1u);
+                    umma_lohi<KIND>(d_tmem, a_lo + a_s2, a_hi, b_lo + b_s2, b_hi, idesc, 1u);
+                    umma_lohi<KIND>(d_tmem, a_lo + a_s3, a_hi, b_lo + b_s3, b_hi, idesc, 1u);
                     umma_commit(empty_bar(stage));
                     if (kb == kb1 - 1) umma_commit(tfull_bar(acc));
                 }

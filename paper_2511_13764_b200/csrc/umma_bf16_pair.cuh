@@ -134,6 +134,7 @@ umma_bf16_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_c
         // ------------------------------------------------ TMA producer (both CTAs)
         const bool a_blk = p.a_blocked != 0;
         const bool b3d = p.b_3d != 0;
+        const bool b_kmajor = p.b_kmajor != 0;
         const uint32_t lead_full0 = map_to_cta(full_bar(0), leader);  // leader's full[0], cluster address
         int stage = 0;
         uint32_t phase = 0;
@@ -172,6 +173,8 @@ umma_bf16_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_c
                         // this CTA's column blocks as they are, on its own barrier; its warps 6-9 re-lay them in place
                         mbar_arrive_expect_tx(raw_bar(stage), B_STAGE);
                         tma_load_3d(sb, &tmap_b, raw_bar(stage), 0, kbl * (UMMA_BK / 2), col0 >> 5);
+                    } else if (b_kmajor) {
+                        tma_load_3d_pair(sb, &tmap_b, lfb, kx, col0, ib);   // this CTA's HALF rows (n) of 128 bytes of k
                     } else {
                         if (b3d) {
                             tma_load_4d_pair(sb, &tmap_b, lfb, 0, kx, col0 >> 6, ib);
@@ -203,12 +206,13 @@ umma_bf16_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_c
         if (rank == 0) {
             const bool a_blk = p.a_blocked != 0;
             const uint64_t da0 = a_blk ? make_smem_desc(smem_base, 16, 512, 4) : make_smem_desc(smem_base, 16, 1024, 2);
-            const uint64_t db0 = B_VNNI ? make_smem_desc(smem_base + UMMA_A_STAGE_BYTES, 16, 1024, 2)
-                                        : make_smem_desc(smem_base + UMMA_A_STAGE_BYTES, 8192, 1024, 2);
+            const bool b_k = B_VNNI || p.b_kmajor != 0;
+            const uint64_t db0 = b_k ? make_smem_desc(smem_base + UMMA_A_STAGE_BYTES, 16, 1024, 2)
+                                     : make_smem_desc(smem_base + UMMA_A_STAGE_BYTES, 8192, 1024, 2);
             const uint32_t a_hi = static_cast<uint32_t>(da0 >> 32), b_hi = static_cast<uint32_t>(db0 >> 32);
             const uint32_t a_lo0 = static_cast<uint32_t>(da0), b_lo0 = static_cast<uint32_t>(db0);
             const uint32_t a_s1 = 2u, a_s2 = a_blk ? 512u : 4u, a_s3 = a_blk ? 514u : 6u;
-            constexpr uint32_t b_s = B_VNNI ? 2u : 128u;
+            const uint32_t b_s = b_k ? 2u : 128u, b_s2 = 2 * b_s, b_s3 = 3 * b_s;
             constexpr uint32_t STAGE16 = STAGE >> 4;
             const uint32_t idesc = p.idesc;
             int stage = 0;
@@ -239,8 +243,8 @@ umma_bf16_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_c
                         const uint32_t a_lo = a_lo0 + soff, b_lo = b_lo0 + soff;
                         umma_pair_lohi<KIND>(d_tmem, a_lo, a_hi, b_lo, b_hi, idesc, accumulate);
                         umma_pair_lohi<KIND>(d_tmem, a_lo + a_s1, a_hi, b_lo + b_s, b_hi, idesc, 1u);
-                        umma_pair_lohi<KIND>(d_tmem, a_lo + a_s2, a_hi, b_lo + 2 * b_s, b_hi, idesc, 1u);
-                        umma_pair_lohi<KIND>(d_tmem, a_lo + a_s3, a_hi, b_lo + 3 * b_s, b_hi, idesc, 1u);
+                        umma_pair_lohi<KIND>(d_tmem, a_lo + a_s2, a_hi, b_lo + b_s2, b_hi, idesc, 1u);
+                        umma_pair_lohi<KIND>(d_tmem, a_lo + a_s3, a_hi, b_lo + b_s3, b_hi, idesc, 1u);
                         umma_commit_pair(empty_bar(stage), pair_mask);
                         if (kb == kb1 - 1) umma_commit_pair(tfull_bar(acc), pair_mask);
                     }

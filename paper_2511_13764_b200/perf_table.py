@@ -158,7 +158,7 @@ def main():
     fma_peak = prop.multi_processor_count * 128 * 2 * 1.965e9 / 1e12
     flush = None if args.no_flush else torch.empty(512 << 20, dtype=torch.uint8, device="cuda")
     works = ([nk_inputs.config(i) for i in (1, 2, 3, 4)] + nk_inputs.sweep() + nk_inputs.paper_mlp() + nk_inputs.f16_set()
-             + nk_inputs.s8_set() + nk_inputs.fp8_set())
+             + nk_inputs.s8_set() + nk_inputs.fp8_set() + nk_inputs.bt_set())
     rows = []
     print(f"| workload | kernel | launches | median us | TFLOP/s | alg. GB/s | bound | frac ({src}) |"
           + (" cuBLAS us |" if args.library else ""))

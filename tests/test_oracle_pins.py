@@ -631,3 +631,22 @@ def test_fp8_gemm_equals_gemm_of_the_widened_operands(fmt):
     Y2, S2 = oracle.gemm_workload(wb, A, Bblk, bias)
     assert np.array_equal(Y0, Y2) and np.array_equal(S0, S2)
     assert np.abs(Y0 - np.maximum(Af.astype(np.float64).reshape(M, K) @ Bf.astype(np.float64).reshape(K, N) + bias, 0)).max() < 1e-9
+
+
+# ---------------------------------------------------------------- B kept as its transpose
+def test_transposed_b_is_the_same_matrix():
+    """layout_b = TRANSPOSED only changes where element (k, j) of B is stored: the oracle on Bt[N][K] equals,
+    bit for bit, the oracle on B[K][N]; and giving it B untransposed is caught."""
+    rng = np.random.default_rng(14)
+    M, N, K = 24, 40, 56
+    A = rng.standard_normal((M, K)).astype(np.float32)
+    B = rng.standard_normal((K, N)).astype(np.float32)
+    Y0, S0 = oracle.gemm(M, N, K, A, B)
+    Y1, S1 = oracle.gemm(M, N, K, A, np.ascontiguousarray(B.T), layout_b=oracle.TRANSPOSED)
+    assert np.array_equal(Y0, Y1) and np.array_equal(S0, S1)
+    Y2, _ = oracle.gemm(M, N, K, A, B, layout_b=oracle.TRANSPOSED)
+    assert not np.array_equal(Y0, Y2)
+    A8 = rng.integers(-128, 128, (M, K), dtype=np.int8)
+    B8 = rng.integers(-128, 128, (K, N), dtype=np.int8)
+    want = A8.astype(np.int64) @ B8.astype(np.int64)
+    assert np.array_equal(oracle.gemm_s8(M, N, K, A8, np.ascontiguousarray(B8.T), layout_b=oracle.TRANSPOSED), want)
