@@ -66,7 +66,8 @@ typedef enum {
                    kernels, layouts and rules as BF16, FP32 accumulation, one RNE rounding of a 16-bit C */
     NK_S8 = 3, /* signed 8-bit integers: the Int8 dot product Section 5 names among the next packed types.  A is
                   row-major; B is NK_BLOCKED32 with four k per group (Section 2: "INT8 elements in groups of
-                  four"): B[N/32][K/32][8][32][4], packed[k/4][n][k%4] = flat[k][n] inside each 32 x 32 block.
+                  four"): B[N/32][K/32][8][32][4], packed[k/4][n][k%4] = flat[k][n] inside each 32 x 32 block;
+                  or NK_TRANSPOSED (8-bit operands have no row-major [K][N] form here).
                   The result is exact: INT32 accumulation of at most 2^17 - 1 products (K splits add their
                   INT32 partial sums as integers).  No epilogue with an INT32 C, no beta, no batch; N and K
                   multiples of 32 */
@@ -77,7 +78,7 @@ typedef enum {
                     value 448 (the OCP FP8 E4M3 format) */
     NK_E5M2 = 6  /* 8-bit floating point, 5 exponent bits (bias 15), 2 fraction bits, IEEE infinities and NaNs.
                     Both: the 8-bit floating-point counterpart on this hardware of the packed types Section 5
-                    lists; A row-major, B NK_BLOCKED32 with four k per group like NK_S8, FP32 accumulation, FP32 C,
+                    lists; A row-major, B NK_BLOCKED32 with four k per group or NK_TRANSPOSED like NK_S8, FP32 accumulation, FP32 C,
                     FP32 bias; N and K multiples of 32; no batch */
 } nk_dtype_t;
 typedef enum {
