@@ -74,6 +74,44 @@ def test_bt_large_shape_sampled_rows():
     check_against_oracle(w, got, A, B, None, rows=nk_inputs.stratified_rows(w.seed, w.M, 64))
 
 
+@pytest.mark.parametrize("dt", ["s8", "e4m3"])
+def test_bt_host_buffers_pipelined(dt):
+    """nk_gemm_run_host on 8-bit operands large enough for the chunked pipeline (eight row chunks of A, four
+    panels of Bt's rows, blocks of C back as they are done): INT8 exactly, E4M3 with its FP32 bias under the
+    bound, on 64 stratified rows."""
+    M, N, K = 2048, 2048, 2560
+    rows = nk_inputs.stratified_rows(31, M, 64)
+    if dt == "s8":
+        A = nk_inputs.fill(31, nk_inputs.TENSOR_A, M * K, dtype="s8")
+        Bt = nk_inputs.fill(31, nk_inputs.TENSOR_B, K * N, dtype="s8")
+        bias = None
+        plan = nk.Plan(M, N, K, in_dtype=nk.S8, out_dtype=nk.S32, layout_b=nk.TRANSPOSED)
+        hC = torch.zeros(M * N, dtype=torch.int32).pin_memory()
+    else:
+        w = W("bt_host", "e4m3", M, N, K, epilogue="bias_relu", seed=31)
+        A, Bt, bias = w.make()
+        plan = nk.plan_for(w)
+        hC = torch.zeros(M * N, dtype=torch.float32).pin_memory()
+    hA, hB = torch.from_numpy(A).pin_memory(), torch.from_numpy(Bt).pin_memory()
+    hb = torch.from_numpy(bias).pin_memory() if bias is not None else None
+    dA, dB = torch.empty_like(hA, device="cuda"), torch.empty_like(hB, device="cuda")
+    db = torch.empty(N, dtype=torch.float32, device="cuda") if bias is not None else None
+    dC = torch.empty_like(hC, device="cuda")
+    wsb = plan.workspace_bytes
+    ws = torch.empty(max(wsb, 16), dtype=torch.uint8, device="cuda")
+    for call in range(2):
+        hC.fill_(0)
+        plan.run_host(hA, hB, hC, dA, dB, dC, hbias=hb, dbias=db, workspace=ws, workspace_bytes=wsb,
+                      stream=torch.cuda.current_stream().cuda_stream)
+        plan.check()
+        got = hC.numpy().reshape(M, N)
+        if dt == "s8":
+            assert np.array_equal(got[rows].astype(np.int64), oracle.gemm_s8(M, N, K, A, Bt, layout_b=oracle.TRANSPOSED, rows=rows))
+        else:
+            from nk_testlib import check_against_oracle
+            check_against_oracle(w, got.astype(np.float64), A, Bt, bias, rows=rows)
+
+
 def test_bt_rejects_what_it_cannot_do():
     with pytest.raises(nk.NkError):
         nk.Plan(64, 64, 64, in_dtype=nk.F32, out_dtype=nk.F32, layout_b=nk.TRANSPOSED)
