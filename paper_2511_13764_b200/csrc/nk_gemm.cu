@@ -175,7 +175,7 @@ static int max_clusters_for(bool pair, int bn, bool vnni, int splits);
 static bool cluster_reduce_fits(const nk_gemm_desc_t& d, int sms, bool pair, int bn, int eff_splits) {
     (void)sms;
     if (d.flags & NK_FLAG_SEPARATE_REDUCE) return false;
-    if (is_8bit(d)) return false;   // the cluster variants are built for the 16-bit kernels only
+    if (is_s8(d)) return false;   // INT32 partial sums: the cluster reduction adds FP32 pieces only
     if (eff_splits != 2 && eff_splits != 4 && !(eff_splits == 8 && !pair)) return false;
     const int64_t clusters = static_cast<int64_t>(desc_gemms(d)) * ceil_div(d.M, pair ? 2 * UMMA_BM : UMMA_BM) * ceil_div(d.N, bn);
     const bool vnni = d.layout_b == NK_BLOCKED32 && !(d.flags & NK_FLAG_REPACK_B);
@@ -539,27 +539,35 @@ static cudaError_t launch_clustered(Kernel kernel, nk_gemm_s* p, const UmmaParam
 }
 
 // `units` = tiles x splits; the single-CTA kernel runs one CTA per unit, the pair kernel two.
-static cudaError_t launch_cluster(nk_gemm_s* p, const UmmaParams& up, int units, int splits, cudaStream_t st,
-                                  int* max_clusters) {
+// KIND as in the kernels (0 = 16-bit floating point, 2 = 8-bit floating point; INT8 has no cluster form).
+template <int KIND>
+static cudaError_t launch_cluster_k(nk_gemm_s* p, const UmmaParams& up, int units, int splits, cudaStream_t st,
+                                    int* max_clusters) {
     const bool v = p->b_vnni_inkernel;
     const int th = v ? 320 : 192;
 #define NK_CL(K, ctas, cl, smem) launch_clustered(K, p, up, ctas, cl, th, smem, st, max_clusters)
     if (p->pair) {
         if (p->bn == 256)
-            return v ? NK_CL((umma_bf16_pair_kernel<256, 6, true, true>), 2 * units, 2 * splits, pair_smem_bytes(256, 6))
-                     : NK_CL((umma_bf16_pair_kernel<256, 6, false, true>), 2 * units, 2 * splits, pair_smem_bytes(256, 6));
-        return v ? NK_CL((umma_bf16_pair_kernel<128, 8, true, true>), 2 * units, 2 * splits, pair_smem_bytes(128, 8))
-                 : NK_CL((umma_bf16_pair_kernel<128, 8, false, true>), 2 * units, 2 * splits, pair_smem_bytes(128, 8));
+            return v ? NK_CL((umma_bf16_pair_kernel<256, 6, true, true, KIND>), 2 * units, 2 * splits, pair_smem_bytes(256, 6))
+                     : NK_CL((umma_bf16_pair_kernel<256, 6, false, true, KIND>), 2 * units, 2 * splits, pair_smem_bytes(256, 6));
+        return v ? NK_CL((umma_bf16_pair_kernel<128, 8, true, true, KIND>), 2 * units, 2 * splits, pair_smem_bytes(128, 8))
+                 : NK_CL((umma_bf16_pair_kernel<128, 8, false, true, KIND>), 2 * units, 2 * splits, pair_smem_bytes(128, 8));
     }
     if (p->bn == 256)
-        return v ? NK_CL((umma_bf16_kernel<256, 4, true, true>), units, splits, umma_smem_bytes(256, 4))
-                 : NK_CL((umma_bf16_kernel<256, 4, false, true>), units, splits, umma_smem_bytes(256, 4));
+        return v ? NK_CL((umma_bf16_kernel<256, 4, true, true, KIND>), units, splits, umma_smem_bytes(256, 4))
+                 : NK_CL((umma_bf16_kernel<256, 4, false, true, KIND>), units, splits, umma_smem_bytes(256, 4));
     if (p->bn == 128)
-        return v ? NK_CL((umma_bf16_kernel<128, 6, true, true>), units, splits, umma_smem_bytes(128, 6))
-                 : NK_CL((umma_bf16_kernel<128, 6, false, true>), units, splits, umma_smem_bytes(128, 6));
-    return v ? NK_CL((umma_bf16_kernel<64, 8, true, true>), units, splits, umma_smem_bytes(64, 8))
-             : NK_CL((umma_bf16_kernel<64, 8, false, true>), units, splits, umma_smem_bytes(64, 8));
+        return v ? NK_CL((umma_bf16_kernel<128, 6, true, true, KIND>), units, splits, umma_smem_bytes(128, 6))
+                 : NK_CL((umma_bf16_kernel<128, 6, false, true, KIND>), units, splits, umma_smem_bytes(128, 6));
+    return v ? NK_CL((umma_bf16_kernel<64, 8, true, true, KIND>), units, splits, umma_smem_bytes(64, 8))
+             : NK_CL((umma_bf16_kernel<64, 8, false, true, KIND>), units, splits, umma_smem_bytes(64, 8));
 #undef NK_CL
+}
+
+static cudaError_t launch_cluster(nk_gemm_s* p, const UmmaParams& up, int units, int splits, cudaStream_t st,
+                                  int* max_clusters) {
+    return is_f8(p->d) ? launch_cluster_k<2>(p, up, units, splits, st, max_clusters)
+                       : launch_cluster_k<0>(p, up, units, splits, st, max_clusters);
 }
 
 static int max_clusters_for(bool pair, int bn, bool vnni, int splits) {
@@ -681,6 +689,16 @@ static cudaError_t prepare_umma_attrs() {
     if ((e = allow_smem(umma_bf16_pair_kernel<128, 8, false, false, 1>, pair_smem_bytes(128, 8))) != cudaSuccess) return e;
     if ((e = allow_smem(umma_bf16_pair_kernel<128, 8, true, false, 2>, pair_smem_bytes(128, 8))) != cudaSuccess) return e;
     if ((e = allow_smem(umma_bf16_pair_kernel<128, 8, false, false, 2>, pair_smem_bytes(128, 8))) != cudaSuccess) return e;
+    if ((e = allow_smem(umma_bf16_kernel<256, 4, false, true, 2>, umma_smem_bytes(256, 4))) != cudaSuccess) return e;
+    if ((e = allow_smem(umma_bf16_kernel<256, 4, true, true, 2>, umma_smem_bytes(256, 4))) != cudaSuccess) return e;
+    if ((e = allow_smem(umma_bf16_kernel<128, 6, false, true, 2>, umma_smem_bytes(128, 6))) != cudaSuccess) return e;
+    if ((e = allow_smem(umma_bf16_kernel<128, 6, true, true, 2>, umma_smem_bytes(128, 6))) != cudaSuccess) return e;
+    if ((e = allow_smem(umma_bf16_kernel<64, 8, false, true, 2>, umma_smem_bytes(64, 8))) != cudaSuccess) return e;
+    if ((e = allow_smem(umma_bf16_kernel<64, 8, true, true, 2>, umma_smem_bytes(64, 8))) != cudaSuccess) return e;
+    if ((e = allow_smem(umma_bf16_pair_kernel<256, 6, false, true, 2>, pair_smem_bytes(256, 6))) != cudaSuccess) return e;
+    if ((e = allow_smem(umma_bf16_pair_kernel<256, 6, true, true, 2>, pair_smem_bytes(256, 6))) != cudaSuccess) return e;
+    if ((e = allow_smem(umma_bf16_pair_kernel<128, 8, false, true, 2>, pair_smem_bytes(128, 8))) != cudaSuccess) return e;
+    if ((e = allow_smem(umma_bf16_pair_kernel<128, 8, true, true, 2>, pair_smem_bytes(128, 8))) != cudaSuccess) return e;
     return cudaSuccess;
 }
 

@@ -56,13 +56,19 @@ def test_fp8_formats_differ_on_the_same_bits():
     check_against_oracle(w5, c5, A, B, None)
 
 
-@pytest.mark.parametrize("splits", [2, 3])
+@pytest.mark.parametrize("mode", ["single", "pair"])
+@pytest.mark.parametrize("splits,sep", [(2, False), (4, False), (3, False), (4, True)])
 @pytest.mark.parametrize("epi", ["none", "bias_relu"])
-def test_fp8_splitk_through_the_reduce_kernel(splits, epi):
-    f = nk.FLAG_SINGLE_CTA | nk.flag_splitk(splits)
+def test_fp8_splitk_cluster_and_reduce_kernel(splits, sep, epi, mode):
+    """K splits inside a thread-block cluster (FP32 pieces through shared memory), and through FP32 partials
+    and the reduce kernel; both with the FP32 bias."""
+    f = MODES[mode] | nk.flag_splitk(splits) | (nk.FLAG_SEPARATE_REDUCE if sep else 0)
     err, plan = run_and_check(W("fp8", "e4m3", 130, 160, 2080, epilogue=epi, integer=True), flags=f, exact=True)
-    assert f"splitk{splits}" in plan.kernel_name and "_cluster" not in plan.kernel_name and plan.workspace_bytes > 0
-    run_and_check(W("fp8", "e4m3", 130, 160, 2080, epilogue=epi, seed=9), flags=f)
+    assert f"splitk{splits}" in plan.kernel_name
+    assert ("_cluster" in plan.kernel_name) == (plan.workspace_bytes == 0)
+    if mode == "single":
+        assert ("_cluster" in plan.kernel_name) == (splits in (2, 4) and not sep)
+    run_and_check(W("fp8", "e5m2", 130, 160, 2080, epilogue=epi, seed=9), flags=f)
 
 
 def test_fp8_tail_wave_split():
