@@ -9,13 +9,27 @@ path), so per-GPU work is fixed ("weak" scaling) and `value` sums all ranks.
 
     python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference]
 
-Prints ONE JSON line on rank 0.
+Prints ONE JSON line on rank 0.  After the timed region of the headline workload
+the same line gets a `configs` list: the other benchmark configurations (the FP32
+256^3 GEMM, the blocked 1024^3 GEMM, the MLP layers, corners of the shape sweep),
+each timed on its own by CUDA-graph replay with an L2 flush before every launch,
+with the roofline that binds it.
+
+    python bench.py --table [--only NAME] [--library] [--f32-tensor]
+
+prints the full per-workload table (every configuration, the whole sweep, the
+paper's MLP grid and the extra operand types) as markdown instead.
+
+Run bare with --gpus N > 1 (no WORLD_SIZE in the environment) it starts the N
+ranks itself, one per GPU, through torch.distributed.run on 127.0.0.1.
 """
 from __future__ import annotations
 
 import argparse
 import json
 import os
+import socket
+import subprocess
 import sys
 import time
 
@@ -26,6 +40,7 @@ if ROOT not in sys.path:
 METRIC = "GEMM TFLOP/s (device-timed, 1 B200) and fraction of dense BF16/FP32 peak"
 UNIT = "TFLOP/s"
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
+TRAFFIC_JSON = os.path.join(ROOT, "profiles", "bench_c4_bf16_8192_dram_traffic.json")
 
 
 def load_peaks():
@@ -49,6 +64,22 @@ def workload(size=None):
     if size:
         w = dataclasses.replace(w, name=f"c4_bf16_{size}_profiling_size", M=size, N=size, K=size)
     return w
+
+
+def recorded_traffic(kernel_name: str, shape) -> tuple:
+    """DRAM bytes per launch of the benchmark kernel from the committed profiler capture, or
+    (None, why) when the capture is of another kernel, another shape, or of kernel sources that
+    have changed since (the record carries the hash of the sources it was taken from)."""
+    if not os.path.exists(TRAFFIC_JSON):
+        return None, "no capture on record"
+    with open(TRAFFIC_JSON) as f:
+        rec = json.load(f)
+    if rec.get("kernel") != kernel_name or list(rec.get("shape", [])) != list(shape):
+        return None, "the capture on record is of another kernel or shape"
+    from paper_2511_13764_b200 import _build
+    if rec.get("source_hash") != _build.source_hash():
+        return None, "kernel sources changed since the capture"
+    return float(rec["dram_read_bytes"]) + float(rec["dram_write_bytes"]), f"ncu capture of {rec.get('captured')}"
 
 
 # --------------------------------------------------------------------------- reference arm
@@ -77,6 +108,16 @@ def oracle_sample_rate(w, B, rows_per_step, steps, warmup, seed_shift=0):
     return flops / sec / 1e12, sec, threads, len(rows)
 
 
+def workload_config(w, world=1):
+    """The `config` object of the JSON line: it names the workload, so both arms print the same one."""
+    e_in = 4 if w.in_dtype == "f32" else 2
+    a_mb, b_mb, c_mb = (w.M * w.K * e_in) >> 20, (w.K * w.N * e_in) >> 20, (w.M * w.N * 4) >> 20
+    return {"workload": w.name, "M": w.M, "N": w.N, "K": w.K, "in_dtype": w.in_dtype,
+            "out_dtype": w.out_dtype, "layout": w.layout, "epilogue": w.epilogue,
+            "l2": f"inputs larger than L2 (A {a_mb} MB + B {b_mb} MB + C {c_mb} MB per step)",
+            "parallelism": f"M-sharded x{world}, B replicated, no collective"}
+
+
 def run_reference(args):
     rank = int(os.environ.get("RANK", "0"))
     if rank != 0:
@@ -91,13 +132,12 @@ def run_reference(args):
     rows = int(max(1, min(256, 120.0 / max(total_steps, 1) / (probe_sec / 8))))
     tf, sec, threads, nrows = oracle_sample_rate(w, B, rows, args.steps, args.warmup)
     sample = f"{nrows} stratified rows of the {w.M}x{w.N}x{w.K} problem per step (all {w.N} columns, full K)"
+    cfg = workload_config(w, int(os.environ.get("WORLD_SIZE", "1")))
     out = {
         "impl": "reference", "metric": METRIC, "value": tf, "unit": UNIT, "n_gpus": args.gpus,
         "steps": args.steps, "warmup": args.warmup, "ms_per_step": sec * 1e3,
         "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64",
-        "data": "synthetic",
-        "config": {"workload": w.name, "M": w.M, "N": w.N, "K": w.K, "in_dtype": w.in_dtype,
-                   "out_dtype": w.out_dtype, "layout": w.layout, "epilogue": w.epilogue},
+        "data": "synthetic", "config": cfg,
         "cpu_baseline": {"value": tf, "unit": UNIT, "cores": threads, "kind": "oracle", "sample": sample},
         "e2e": {"value": tf, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
         "gpu_launches": 0,
@@ -137,6 +177,20 @@ def max_over_ranks(x: float, world: int, device=None) -> float:
 def whole_job_tflops(flops_per_rank: float, world: int, ms_per_step: float) -> float:
     """Aggregate over all ranks: every rank does `flops_per_rank` per step (weak scaling)."""
     return world * flops_per_rank / (ms_per_step * 1e-3) / 1e12
+
+
+def free_port() -> int:
+    with socket.socket() as s:
+        s.bind(("127.0.0.1", 0))
+        return s.getsockname()[1]
+
+
+def spawn_ranks(n: int, argv) -> int:
+    """Started bare with --gpus n > 1: run n ranks of this script, one per GPU, through
+    torch.distributed.run with a loopback rendezvous, and hand back its exit code."""
+    cmd = [sys.executable, "-m", "torch.distributed.run", "--nnodes=1", f"--nproc-per-node={n}",
+           "--master-addr", "127.0.0.1", "--master-port", str(free_port()), os.path.abspath(__file__)] + list(argv)
+    return subprocess.call(cmd)
 
 
 # --------------------------------------------------------------------------- clocks
@@ -183,7 +237,236 @@ class ClockSampler:
                 "samples": len(s)}
 
 
+# --------------------------------------------------------------------------- per-workload timing
+def time_launch(launch, st, iters, flush, graph_pairs):
+    """Median (and best) time in ms of `launch(cuda_stream)`, each call timed on its own after an
+    L2 flush.  With `graph_pairs` a CUDA graph of that many (flush, launch) pairs is replayed and a
+    graph of the flushes alone subtracted: CUDA-event stamps are a microsecond or two coarse on
+    some boxes, the graph difference resolves a fraction of a microsecond, and the launches come
+    without host gaps, as they would inside a captured pipeline."""
+    import torch
+    # a quarter of a second of idling first: a heavy row just before leaves the part power-throttled for
+    # a while, which a short FMA-bound row would otherwise inherit
+    torch.cuda.synchronize()
+    time.sleep(0.25)
+    for _ in range(3):
+        launch(st.cuda_stream)
+    torch.cuda.synchronize()
+    if graph_pairs and flush is not None:
+        side = torch.cuda.Stream()
+        side.wait_stream(st)
+        graphs = []
+        for with_launch in (True, False):
+            g = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(g, stream=side):
+                cs = torch.cuda.current_stream().cuda_stream
+                for _ in range(graph_pairs):
+                    flush.fill_(1)
+                    if with_launch:
+                        launch(cs)
+            graphs.append(g)
+
+        def replay_ms(g):
+            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a.record(st)
+            g.replay()
+            b.record(st)
+            b.synchronize()
+            return a.elapsed_time(b)
+
+        # The two graphs are timed in turn, so that a drift of the clocks (the previous row may have
+        # left the part power-throttled) hits both alike; the median of the differences is reported.
+        for g in graphs:
+            replay_ms(g)
+        diffs = sorted(replay_ms(graphs[0]) - replay_ms(graphs[1]) for _ in range(max(5, iters // 2)))
+        per = diffs[len(diffs) // 2] / graph_pairs
+        return per, diffs[0] / graph_pairs
+    times = []
+    for _ in range(iters):
+        if flush is not None:
+            flush.fill_(1)
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record(st)
+        launch(st.cuda_stream)
+        b.record(st)
+        b.synchronize()
+        times.append(a.elapsed_time(b))
+    times.sort()
+    return times[len(times) // 2], times[0]
+
+
+def time_workload(w, iters, flags=0, flush=None, graph_pairs=0, library=False, device=0):
+    """Returns (median ms, best ms, kernel name, launches per run, library ms or None).  Operands are
+    random values of the workload's types made on the device (this only measures; parity is the
+    tests' business).  `library` also times torch.matmul (cuBLAS) on the same shape and element
+    type (row-major operands, no epilogue, FP32 without TF32): context for the table, never part
+    of the product path."""
+    import torch
+    import paper_2511_13764_b200 as nk
+    dev = torch.device("cuda", device)
+    tt = {"f32": torch.float32, "bf16": torch.bfloat16, "f16": torch.float16, "s8": torch.int8, "s32": torch.int32,
+          "e4m3": torch.uint8, "e5m2": torch.uint8}
+    ein, eout = tt[w.in_dtype], tt[w.out_dtype]
+    g = torch.Generator(device=dev).manual_seed(w.seed)
+    if w.in_dtype == "s8":
+        A = torch.randint(-128, 128, (w.M * w.K,), device=dev, generator=g, dtype=torch.int8)
+        B = torch.randint(-128, 128, (w.K * w.N,), device=dev, generator=g, dtype=torch.int8)
+        library = False      # no library column for INT8
+    elif w.in_dtype in ("e4m3", "e5m2"):
+        f8 = torch.float8_e4m3fn if w.in_dtype == "e4m3" else torch.float8_e5m2
+        A = (torch.rand(w.M * w.K, device=dev, generator=g) * 2 - 1).to(f8)
+        B = (torch.rand(w.K * w.N, device=dev, generator=g) * 2 - 1).to(f8)
+        library = False      # nor for 8-bit floating point
+    else:
+        A = (torch.rand(w.M * w.K, device=dev, generator=g) * 2 - 1).to(ein)
+        B = (torch.rand(w.K * w.N, device=dev, generator=g) * 2 - 1).to(ein)
+    bias = (torch.randn(w.N, device=dev, generator=g) * 0.02).to(tt[w.bias_dtype]) if w.epilogue != "none" else None
+    C = torch.empty(w.M * w.N, dtype=eout, device=dev)
+    plan = nk.plan_for(w, device=device, flags=flags)
+    wsb = plan.workspace_bytes
+    ws = torch.empty(max(wsb, 16), dtype=torch.uint8, device=dev)
+    st = torch.cuda.current_stream()
+
+    def run(cs):
+        plan.run(A, B, C, bias=bias, workspace=ws if wsb else None, workspace_bytes=wsb, stream=cs)
+
+    med, best = time_launch(run, st, iters, flush, graph_pairs)
+    plan.check()
+    lib_ms = None
+    if library:
+        torch.backends.cuda.matmul.allow_tf32 = False
+        A2, B2 = A.view(w.M, w.K), B.view(w.K, w.N)
+        C2 = torch.empty(w.M, w.N, dtype=ein, device=dev)
+        lib_ms, _ = time_launch(lambda cs: torch.matmul(A2, B2, out=C2), st, iters, flush, graph_pairs)
+    return med, best, plan.kernel_name, plan.launches_per_run, lib_ms
+
+
+def fma_peak_tflops(device=0) -> float:
+    """FP32 FMA-pipe peak: SMs x 128 lanes x 2 flop x the maximum SM clock."""
+    import torch
+    prop = torch.cuda.get_device_properties(device)
+    return prop.multi_processor_count * 128 * 2 * 1.965e9 / 1e12
+
+
+def roofline_row(w, ms, peaks, fma_peak, split=False):
+    """The roofline that binds workload `w` at the box's peaks, and the fraction `ms` reaches:
+    (TFLOP/s, algorithmic GB/s, bound, peak, unit, frac).  8-bit operands run at twice the BF16
+    rate on the tensor cores (nominal ratio applied to the measured BF16 peak); `split` marks FP32
+    operands multiplied as six BF16 products (a sixth of the BF16 peak)."""
+    tensor_peak, hbm_peak = float(peaks["bf16_tflops"]), float(peaks["hbm_gbs"])
+    tf = w.flops / (ms * 1e-3) / 1e12
+    gbs = w.algorithmic_bytes / (ms * 1e-3) / 1e9
+    compute_peak = (tensor_peak / 6 if split else 2 * tensor_peak if w.in_dtype in ("s8", "e4m3", "e5m2")
+                    else tensor_peak if w.in_dtype != "f32" else fma_peak)
+    t_compute = w.flops / (compute_peak * 1e12)
+    t_hbm = w.algorithmic_bytes / (hbm_peak * 1e9)
+    if t_hbm >= t_compute:
+        return tf, gbs, "hbm", hbm_peak, "GB/s", gbs / hbm_peak
+    bound = "tensor/6" if split else "tensor" if w.in_dtype != "f32" else "alu"
+    return tf, gbs, bound, compute_peak, "TFLOP/s", tf / compute_peak
+
+
+def config_rows():
+    """The configurations reported beside the headline: C1, C2, C3, the paper's MLP layers (flat B,
+    and the widest one with VNNI-blocked operands), and the corners of the shape sweep."""
+    import nk_inputs
+    rows = [nk_inputs.config(1), nk_inputs.config(2), nk_inputs.config(3)]
+    mlp = {w.name: w for w in nk_inputs.paper_mlp()}
+    rows += [mlp["mlp_bf16_flat_1024"], mlp["mlp_bf16_flat_2048"], mlp["mlp_bf16_flat_4096"], mlp["mlp_bf16_vnni_4096"]]
+    sweep = {w.name: w for w in nk_inputs.sweep()}
+    rows += [sweep["c5_f32_16x16384x16384"], sweep["c5_bf16_16x16384x16384"],
+             sweep["c5_f32_4096x4096x4096"], sweep["c5_bf16_4096x4096x4096"]]
+    return rows
+
+
+def time_configs(peaks, device=0, iters=9, graph_pairs=20):
+    import torch
+    flush = torch.empty(512 << 20, dtype=torch.uint8, device=torch.device("cuda", device))
+    fma = fma_peak_tflops(device)
+    out = []
+    for w in config_rows():
+        med, best, kname, launches, _ = time_workload(w, iters, flush=flush, device=device,
+                                                      graph_pairs=graph_pairs if w.flops < 5e11 else 0)
+        tf, gbs, bound, peak, unit, frac = roofline_row(w, med, peaks, fma)
+        out.append({"workload": w.name, "kernel": kname, "launches": launches, "us": med * 1e3, "value": tf,
+                    "unit": UNIT, "alg_gbs": gbs, "bound": bound, "peak": peak, "peak_unit": unit, "frac": frac,
+                    "flop": w.flops, "alg_bytes": w.algorithmic_bytes})
+    del flush
+    return out
+
+
+def run_table(args):
+    """Every workload, one row each, as a markdown table (and optionally JSON)."""
+    import torch
+    import nk_inputs
+    import paper_2511_13764_b200 as nk
+    if not torch.cuda.is_available():
+        raise SystemExit("needs a CUDA device")
+    peaks = load_peaks()
+    fma = fma_peak_tflops(0)
+    flush = None if args.no_flush else torch.empty(512 << 20, dtype=torch.uint8, device="cuda")
+    works = ([nk_inputs.config(i) for i in (1, 2, 3, 4)] + nk_inputs.sweep() + nk_inputs.paper_mlp() + nk_inputs.f16_set()
+             + nk_inputs.s8_set() + nk_inputs.fp8_set() + nk_inputs.bt_set())
+    rows = []
+    print(f"| workload | kernel | launches | median us | TFLOP/s | alg. GB/s | bound | frac ({peaks['_source']}) |"
+          + (" cuBLAS us |" if args.library else ""))
+    print("|---|---|---|---|---|---|---|---|" + ("---|" if args.library else ""))
+    todo = []
+    for w in works:
+        if args.only and not any(o in w.name for o in args.only.split(",")):
+            continue
+        todo.append((w, w.name, args.flags, False))
+        if args.f32_tensor and w.in_dtype == "f32" and w.N % 8 == 0 and w.K % 8 == 0:
+            todo.append((w, w.name + " +tensor", args.flags | nk.FLAG_F32_TENSOR, True))
+    for w, label, flags, split in todo:
+        med, best, kname, launches, lib_ms = time_workload(w, args.iters, flags=flags, flush=flush,
+                                                           graph_pairs=args.graph if w.flops < 5e11 else 0,
+                                                           library=args.library and not split)
+        tf, gbs, bound, peak, unit, frac = roofline_row(w, med, peaks, fma, split)
+        rows.append(dict(workload=label, kernel=kname, launches=launches, median_us=med * 1e3,
+                         best_us=best * 1e3, tflops=tf, gbs=gbs, bound=bound, frac=frac,
+                         library_us=None if lib_ms is None else lib_ms * 1e3))
+        print(f"| {label} | {kname} | {launches} | {med * 1e3:.1f} | {tf:.1f} | {gbs:.0f} | {bound} | {frac:.3f} |"
+              + (f" {lib_ms * 1e3:.1f} |" if lib_ms is not None else " |" if args.library else ""), flush=True)
+    if args.json:
+        with open(args.json, "w") as f:
+            json.dump(rows, f, indent=1)
+    return 0
+
+
 # --------------------------------------------------------------------------- our arm
+def run_dry(args):
+    """The multi-rank plumbing with the GEMM left out (no GPU needed): rendezvous, barrier, the MAX of
+    the per-rank step times, the whole-job aggregate, one JSON line from rank 0.  The per-rank "step"
+    is a sleep whose length grows with the rank, so the slowest rank must set the time."""
+    import torch.distributed as dist
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    init_distributed(world, None)
+    print(f"[bench] rank {rank} of {world} (dry run, no device)", file=sys.stderr, flush=True)
+    w = workload(args.size)
+    if world > 1:
+        dist.barrier()
+    t0 = time.perf_counter()
+    for _ in range(args.steps):
+        time.sleep(0.002 * (rank + 1))
+    ms = (time.perf_counter() - t0) * 1e3
+    if world > 1:
+        dist.barrier()
+    ms = max_over_ranks(ms, world, None)
+    ms_per_step = ms / args.steps
+    cfg = workload_config(w, world)
+    out = {"metric": METRIC, "value": whole_job_tflops(w.flops, world, ms_per_step), "unit": UNIT, "n_gpus": world,
+           "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms_per_step, "higher_is_better": True,
+           "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic", "config": cfg,
+           "dry_run": True, "gpu_launches": 0}
+    if rank == 0:
+        print(json.dumps(out), flush=True)
+    if world > 1:
+        dist.destroy_process_group()
+    return 0
+
+
 def run_ours(args):
     import numpy as np
     import torch
@@ -199,6 +482,8 @@ def run_ours(args):
     torch.cuda.set_device(local)
     dev = torch.device("cuda", local)
     init_distributed(world, dev)
+    print(f"[bench] rank {rank} of {world} on cuda:{local} ({torch.cuda.get_device_name(local)})", file=sys.stderr,
+          flush=True)
 
     peaks = load_peaks()
     w = workload(args.size)
@@ -230,8 +515,9 @@ def run_ours(args):
 
     # best of 10 launches timed one by one after an L2 flush, on a chip that is not yet under sustained
     # load: the mode the pool's burst peak was taken in
+    extras = rank == 0 and world == 1 and not args.no_modes and not args.no_cpu_baseline
     burst = None
-    if rank == 0 and world == 1 and not args.no_modes and not args.no_cpu_baseline:
+    if extras:
         flush = torch.empty(512 << 20, dtype=torch.uint8, device=dev)
         singles = []
         for _ in range(10):
@@ -268,17 +554,13 @@ def run_ours(args):
     # per-launch duration of the GEMM kernel: one launch per step, so the CUDA-event time of the
     # timed region divided by the steps is the kernel's average launch duration, measured live
     # on the launching stream (L2 cannot carry data across launches: A, B, C total 512 MB)
-    # DRAM bytes per launch of the benchmark kernel at this size, from the ncu capture summarised in
-    # profiles/bench_c4_bf16_8192_dram_traffic.md; None for any other kernel or size.
-    traffic = None
-    if plan.kernel_name == "umma_bf16_pair_256x256x64_s6_splitk1" and (w.M, w.N, w.K) == (8192, 8192, 8192):
-        traffic = 1.1094e9 + 251.8e6
+    traffic, traffic_note = recorded_traffic(plan.kernel_name, (w.M, w.N, w.K))
     k_avg = ms_per_step          # average launch duration inside the timed region
     achieved = w.flops / (k_avg * 1e-3) / 1e12
     peak = float(peaks["bf16_tflops"])
     roofline = {
         "bound": "tensor", "achieved": achieved, "peak": peak, "unit": "TFLOP/s",
-        "frac": achieved / peak, "traffic": traffic,
+        "frac": achieved / peak, "traffic": traffic, "traffic_source": traffic_note,
         "peak_source": f"MEASURED_PEAKS.json bf16_tflops (burst), of {peaks['_source']}",
         "frac_of_sustained_peak": achieved / float(peaks["bf16_tflops_sustained"]),
         "frac_of_nominal_2250": achieved / 2250.0,
@@ -288,7 +570,7 @@ def run_ours(args):
 
     # The other mode the pool's peak figures were taken in: launches back to back for about four
     # seconds (compare with the sustained peak; the part is power-managed).
-    if rank == 0 and world == 1 and not args.no_modes and not args.no_cpu_baseline:
+    if extras:
         per_round = max(10, int(0.25 / (ms_per_step * 1e-3)))
         sus_sampler = ClockSampler(local)
         t_begin = time.perf_counter()
@@ -326,18 +608,24 @@ def run_ours(args):
            "h2d_bytes_per_step": int(A.nbytes + B.nbytes), "d2h_bytes_per_step": int(w.M * w.N * 4),
            "steps": e2e_steps}
 
+    cfg = workload_config(w, world)
     out = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
         "warmup": max(args.warmup, 3), "ms_per_step": ms_per_step, "higher_is_better": True,
-        "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
-        "config": {"workload": w.name, "M": w.M, "N": w.N, "K": w.K, "in_dtype": w.in_dtype,
-                   "out_dtype": w.out_dtype, "layout": w.layout, "epilogue": w.epilogue,
-                   "l2": f"inputs larger than L2 (A {A.nbytes >> 20} MB + B {B.nbytes >> 20} MB + C {(w.M * w.N * 4) >> 20} MB per step)",
-                   "parallelism": f"M-sharded x{world}, B replicated, no collective"},
+        "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic", "config": cfg,
         "roofline": roofline, "e2e": e2e,
         "gpu_launches": plan.launches_per_run * args.steps,
         "clocks": sampler.summary(),
     }
+
+    # the other configurations, each timed on its own (outside the contract's timed region)
+    if extras and not args.no_configs and args.size is None:
+        del dA, dB, dC, hC
+        torch.cuda.empty_cache()
+        out["configs"] = time_configs(peaks, device=local)
+        out["configs_timing"] = ("per launch, CUDA-graph replay of 20 (L2 flush, GEMM) pairs minus a graph of the "
+                                 "flushes, median of 5; rows of 5e11 flop and more: CUDA events around single "
+                                 "launches after a flush, median of 9")
 
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
         tf, sec, threads, nrows = oracle_sample_rate(w, B, min(1024, w.M), 1, 0)
@@ -361,11 +649,31 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true",
                     help="timed steps and the end-to-end leg only (profiler captures): no CPU oracle, no extra modes")
     ap.add_argument("--no-modes", action="store_true", help="skip the best-of-10 and four-second measurements")
+    ap.add_argument("--no-configs", action="store_true", help="skip the per-configuration list")
     ap.add_argument("--size", type=int, default=None,
                     help="shrink M=N=K (profiler captures only; not a benchmark number)")
+    ap.add_argument("--dry-run", action="store_true",
+                    help="multi-rank plumbing only: no device, the step is a sleep (CPU tests)")
+    ap.add_argument("--table", action="store_true", help="print the per-workload table instead of the JSON line")
+    ap.add_argument("--iters", type=int, default=9, help="--table: timed launches per row")
+    ap.add_argument("--only", default=None, help="--table: comma-separated substrings of workload names")
+    ap.add_argument("--json", default=None, help="--table: also write the rows to this file")
+    ap.add_argument("--no-flush", action="store_true", help="--table: leave L2 warm between launches")
+    ap.add_argument("--flags", type=lambda x: int(x, 0), default=0, help="--table: NK_FLAG_* bits given to every plan")
+    ap.add_argument("--graph", type=int, default=20,
+                    help="--table: (flush, GEMM) pairs per CUDA-graph replay (0: CUDA events around single launches)")
+    ap.add_argument("--library", action="store_true", help="--table: add a column with torch.matmul (cuBLAS)")
+    ap.add_argument("--f32-tensor", action="store_true",
+                    help="--table: after every FP32 row, the same workload with NK_FLAG_F32_TENSOR")
     args = ap.parse_args()
+    if args.table:
+        return run_table(args)
+    if args.gpus > 1 and "WORLD_SIZE" not in os.environ:
+        return spawn_ranks(args.gpus, sys.argv[1:])
     if args.impl == "reference":
         return run_reference(args)
+    if args.dry_run:
+        return run_dry(args)
     return run_ours(args)
 
 

@@ -2,12 +2,11 @@
  * nk_gemm — dense GEMM for NVIDIA B200 (sm_100a) behind a plain C ABI.
  *
  * The operation is the batch-reduce GEMM of the paper's Algorithm 1
- * ("BRGEMM - nanokernels()", C = beta*C + sum_i A_i x B_i) taken with beta = 0
- * and the batch folded into K:
+ * (C = beta*C + sum_i A_i x B_i) taken with beta = 0 and the batch folded into K:
  *
  *     C[M][N] = A[M][K] . B[K][N]                     FP32 accumulation
  *     C[M][N] = ReLU(A.B + bias[N])                   optional fused epilogue
- *                                                     (Section 6, "MLP": bias and ReLU are
+ *                                                     (Section 6, the MLP benchmark: bias and ReLU are
  *                                                     applied before the single store of C)
  *
  * Element types (Section 2.3): FP32 operands, or 16-bit operands (BF16; or FP16, the
@@ -25,7 +24,7 @@
  *                  every 32x32 block of B is VNNI-2 packed as in Figure 1,
  *                  packed[k/2][n][k%2] = flat[k][n] (16-bit operands);
  *                  B[N/32][K/32][8][32][4], packed[k/4][n][k%4] = flat[k][n] (8-bit operands:
- *                  Section 2, "INT8 elements in groups of four").
+ *                  four k per 32-bit group, the INT8 packing Section 2 describes).
  *   NK_TRANSPOSED  (layout_b only) Bt[N][K]: B kept as its transpose, K contiguous.
  * C is row-major [M][N] unless desc.layout_c asks for the blocked form; bias is [N] in the
  * operand type (FP32 for 8-bit operands).
@@ -65,8 +64,8 @@ typedef enum {
     NK_F16 = 2, /* IEEE binary16: the other 16-bit packed type (Section 5 names FP16 as the next one); same
                    kernels, layouts and rules as BF16, FP32 accumulation, one RNE rounding of a 16-bit C */
     NK_S8 = 3, /* signed 8-bit integers: the Int8 dot product Section 5 names among the next packed types.  A is
-                  row-major; B is NK_BLOCKED32 with four k per group (Section 2: "INT8 elements in groups of
-                  four"): B[N/32][K/32][8][32][4], packed[k/4][n][k%4] = flat[k][n] inside each 32 x 32 block;
+                  row-major; B is NK_BLOCKED32 with four k per 32-bit group (the INT8 packing of Section 2):
+                  B[N/32][K/32][8][32][4], packed[k/4][n][k%4] = flat[k][n] inside each 32 x 32 block;
                   or NK_TRANSPOSED (8-bit operands have no row-major [K][N] form here).
                   The result is exact: INT32 accumulation of at most 2^17 - 1 products (K splits add their
                   INT32 partial sums as integers).  No epilogue with an INT32 C, no beta, no batch; N and K
@@ -143,8 +142,8 @@ typedef struct {
     int32_t layout_c;  /* nk_layout_t of C: NK_ROW_MAJOR, or NK_BLOCKED32 = C[M/32][N/32][32][32],
                           the layout a following layer reads as its blocked A (BF16 operands;
                           M and N multiples of 32)                                        */
-    float scale;       /* NK_S8 operands with an NK_F32 C (quantised layer, Section 5c's "Int8 ... along
-                          with quantization support"): C = scale * (A.B), then the epilogue, in FP32;
+    float scale;       /* NK_S8 operands with an NK_F32 C (quantised layer: Section 5c names Int8 with
+                          quantisation as the next type): C = scale * (A.B), then the epilogue, in FP32;
                           scale is the product of the two operands' quantisation steps and must be
                           finite and non-zero.  The bias of such a plan is FP32.  Ignored otherwise. */
 } nk_gemm_desc_t;
@@ -178,7 +177,8 @@ size_t nk_gemm_workspace_bytes(nk_gemm_t plan);
  * Enqueue C = A.B (+ epilogue) on `cuda_stream` (a cudaStream_t; NULL is the
  * default stream) and return without synchronising (Algorithm 1: tile loop,
  * accumulator resident over the whole K loop, epilogue, one store of C).
- * C's previous contents are never read.  A, B, C (and bias, workspace when
+ * With desc.beta = 0 C's previous contents are never read; with desc.beta = 1 they
+ * are read once and added, in FP32, before the epilogue.  A, B, C (and bias, workspace when
  * used) must be 16-byte aligned device pointers on the plan's device, must not
  * overlap, and must stay valid until the stream reaches the end of the work.
  * bias may be NULL only when the plan has no epilogue.  Nothing is launched

@@ -68,12 +68,11 @@ def lib_path() -> str:
 
 
 def lib():
-    """Load libnk_gemm.so (building it first when the sources are newer)."""
+    """Load libnk_gemm.so, building it first when it is missing or was built from other
+    sources than the ones in the tree now."""
     global _lib
     if _lib is None:
-        path = _build.LIB
-        if not os.path.exists(path) or os.environ.get("NK_GEMM_REBUILD"):
-            path = _build.build()
+        path = _build.build(force=bool(os.environ.get("NK_GEMM_REBUILD")))
         L = ctypes.CDLL(path)          # raises OSError when unusable: no fallback
         vp, sz = ctypes.c_void_p, ctypes.c_size_t
         L.nk_gemm_create.restype = ctypes.c_int

@@ -78,6 +78,7 @@ struct nk_gemm_s {
     // nk_gemm_run_host on large problems: 8 row chunks x up to 4 column panels pipelined over two copy
     // streams (made on first use)
     nk_gemm_s* chunk_plan;
+    bool chunk_tried;      // the chunk plan was asked for once already (and, if chunk_plan is null, refused)
     int chunk_rows, chunk_panels;
     cudaStream_t h2d_stream, d2h_stream;
     cudaEvent_t ev_start, ev_done, ev_up[12], ev_g[32];
@@ -165,8 +166,8 @@ static int desc_batch(const nk_gemm_desc_t& d) { return (d.batch > 1 && !d.batch
 static int desc_gemms(const nk_gemm_desc_t& d) { return (d.batch > 1 && d.batch_independent) ? static_cast<int>(d.batch) : 1; }
 
 // Co-resident clusters of the cluster split-K variant (pair?, tile N, VNNI?, splits), as the driver
-// reports them for this device; asked once per variant and remembered.
-static int max_clusters_for(bool pair, int bn, bool vnni, int splits);
+// reports them for the current device; asked once per device and variant and remembered.
+static int max_clusters_for(bool pair, int bn, bool vnni, int splits, bool f8);
 
 // K splits can meet inside a cluster (no partials in global memory, no second kernel) when there
 // are 2, 4 or 8 of them (2 or 4 pairs) and all the units of the plan are resident at once (one
@@ -179,7 +180,7 @@ static bool cluster_reduce_fits(const nk_gemm_desc_t& d, int sms, bool pair, int
     if (eff_splits != 2 && eff_splits != 4 && !(eff_splits == 8 && !pair)) return false;
     const int64_t clusters = static_cast<int64_t>(desc_gemms(d)) * ceil_div(d.M, pair ? 2 * UMMA_BM : UMMA_BM) * ceil_div(d.N, bn);
     const bool vnni = d.layout_b == NK_BLOCKED32 && !(d.flags & NK_FLAG_REPACK_B);
-    return clusters <= max_clusters_for(pair, bn, vnni, eff_splits);
+    return clusters <= max_clusters_for(pair, bn, vnni, eff_splits, is_f8(d));
 }
 
 static double umma_model_us(const nk_gemm_desc_t& d, int sms, bool pair, int bn, int splits) {
@@ -570,26 +571,31 @@ static cudaError_t launch_cluster(nk_gemm_s* p, const UmmaParams& up, int units,
                        : launch_cluster_k<0>(p, up, units, splits, st, max_clusters);
 }
 
-static int max_clusters_for(bool pair, int bn, bool vnni, int splits) {
+static int max_clusters_for(bool pair, int bn, bool vnni, int splits, bool f8) {
     static std::mutex mu;
-    static int cache[2][3][2][9];   // 0 = not asked yet, -1 = none
+    static int cache[16][2][2][3][2][9];   // [device][8-bit float?][pair?][tile][VNNI?][splits]: 0 = not asked yet, -1 = none
     const int bi = bn == 256 ? 2 : bn == 128 ? 1 : 0;
     if (splits < 2 || splits > 8) return 0;
-    std::lock_guard<std::mutex> lock(mu);
-    int& c = cache[pair ? 1 : 0][bi][vnni ? 1 : 0][splits];
-    if (c == 0) {
-        nk_gemm_s tmp;
-        memset(&tmp, 0, sizeof(tmp));
-        tmp.pair = pair;
-        tmp.bn = bn;
-        tmp.b_vnni_inkernel = vnni;
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess) { cudaGetLastError(); return 0; }
+    nk_gemm_s tmp;
+    memset(&tmp, 0, sizeof(tmp));
+    tmp.pair = pair;
+    tmp.bn = bn;
+    tmp.b_vnni_inkernel = vnni;
+    tmp.d.in_dtype = f8 ? NK_E4M3 : NK_BF16;
+    auto ask = [&]() {
         int n = 0;
         if (launch_cluster(&tmp, UmmaParams(), 0, splits, nullptr, &n) != cudaSuccess || n <= 0) {
             cudaGetLastError();
             n = -1;
         }
-        c = n;
-    }
+        return n;
+    };
+    if (dev < 0 || dev >= 16) { const int n = ask(); return n > 0 ? n : 0; }   // beyond the cache: ask every time
+    std::lock_guard<std::mutex> lock(mu);
+    int& c = cache[dev][f8 ? 1 : 0][pair ? 1 : 0][bi][vnni ? 1 : 0][splits];
+    if (c == 0) c = ask();
     return c > 0 ? c : 0;
 }
 
@@ -646,59 +652,38 @@ static cudaError_t prepare_simt_attrs() {
     return allow_smem(simt_f32_async_kernel<128, 128, 8, 16, true>, simt_async_smem_bytes<128, 128>());
 }
 
-static cudaError_t prepare_umma_attrs() {
-    cudaError_t e2;
-    if ((e2 = allow_smem(umma_bf16_pair_kernel<256, 6, false>, pair_smem_bytes(256, 6))) != cudaSuccess) return e2;
-    if ((e2 = allow_smem(umma_bf16_pair_kernel<128, 8, false>, pair_smem_bytes(128, 8))) != cudaSuccess) return e2;
-    if ((e2 = allow_smem(umma_bf16_pair_kernel<256, 6, true>, pair_smem_bytes(256, 6))) != cudaSuccess) return e2;
-    if ((e2 = allow_smem(umma_bf16_pair_kernel<128, 8, true>, pair_smem_bytes(128, 8))) != cudaSuccess) return e2;
-    cudaError_t e;
-    if ((e = allow_smem(umma_bf16_kernel<256, 4, false>, umma_smem_bytes(256, 4))) != cudaSuccess) return e;
-    if ((e = allow_smem(umma_bf16_kernel<128, 6, false>, umma_smem_bytes(128, 6))) != cudaSuccess) return e;
-    if ((e = allow_smem(umma_bf16_kernel<64, 8, false>, umma_smem_bytes(64, 8))) != cudaSuccess) return e;
-    if ((e = allow_smem(umma_bf16_kernel<256, 4, true>, umma_smem_bytes(256, 4))) != cudaSuccess) return e;
-    if ((e = allow_smem(umma_bf16_kernel<128, 6, true>, umma_smem_bytes(128, 6))) != cudaSuccess) return e;
-    if ((e = allow_smem(umma_bf16_kernel<64, 8, true>, umma_smem_bytes(64, 8))) != cudaSuccess) return e;
-    if ((e = allow_smem(umma_bf16_kernel<256, 4, false, true>, umma_smem_bytes(256, 4))) != cudaSuccess) return e;
-    if ((e = allow_smem(umma_bf16_kernel<256, 4, true, true>, umma_smem_bytes(256, 4))) != cudaSuccess) return e;
-    if ((e = allow_smem(umma_bf16_kernel<128, 6, false, true>, umma_smem_bytes(128, 6))) != cudaSuccess) return e;
-    if ((e = allow_smem(umma_bf16_kernel<128, 6, true, true>, umma_smem_bytes(128, 6))) != cudaSuccess) return e;
-    if ((e = allow_smem(umma_bf16_kernel<64, 8, false, true>, umma_smem_bytes(64, 8))) != cudaSuccess) return e;
-    if ((e = allow_smem(umma_bf16_kernel<64, 8, true, true>, umma_smem_bytes(64, 8))) != cudaSuccess) return e;
-    if ((e = allow_smem(umma_bf16_pair_kernel<256, 6, false, true>, pair_smem_bytes(256, 6))) != cudaSuccess) return e;
-    if ((e = allow_smem(umma_bf16_pair_kernel<256, 6, true, true>, pair_smem_bytes(256, 6))) != cudaSuccess) return e;
-    if ((e = allow_smem(umma_bf16_pair_kernel<128, 8, false, true>, pair_smem_bytes(128, 8))) != cudaSuccess) return e;
-    if ((e = allow_smem(umma_bf16_pair_kernel<128, 8, true, true>, pair_smem_bytes(128, 8))) != cudaSuccess) return e;
-    if ((e = allow_smem(umma_bf16_kernel<256, 4, true, false, 1>, umma_smem_bytes(256, 4))) != cudaSuccess) return e;
-    if ((e = allow_smem(umma_bf16_kernel<256, 4, false, false, 1>, umma_smem_bytes(256, 4))) != cudaSuccess) return e;
-    if ((e = allow_smem(umma_bf16_kernel<256, 4, true, false, 2>, umma_smem_bytes(256, 4))) != cudaSuccess) return e;
-    if ((e = allow_smem(umma_bf16_kernel<256, 4, false, false, 2>, umma_smem_bytes(256, 4))) != cudaSuccess) return e;
-    if ((e = allow_smem(umma_bf16_kernel<128, 6, true, false, 1>, umma_smem_bytes(128, 6))) != cudaSuccess) return e;
-    if ((e = allow_smem(umma_bf16_kernel<128, 6, false, false, 1>, umma_smem_bytes(128, 6))) != cudaSuccess) return e;
-    if ((e = allow_smem(umma_bf16_kernel<128, 6, true, false, 2>, umma_smem_bytes(128, 6))) != cudaSuccess) return e;
-    if ((e = allow_smem(umma_bf16_kernel<128, 6, false, false, 2>, umma_smem_bytes(128, 6))) != cudaSuccess) return e;
-    if ((e = allow_smem(umma_bf16_kernel<64, 8, true, false, 1>, umma_smem_bytes(64, 8))) != cudaSuccess) return e;
-    if ((e = allow_smem(umma_bf16_kernel<64, 8, false, false, 1>, umma_smem_bytes(64, 8))) != cudaSuccess) return e;
-    if ((e = allow_smem(umma_bf16_kernel<64, 8, true, false, 2>, umma_smem_bytes(64, 8))) != cudaSuccess) return e;
-    if ((e = allow_smem(umma_bf16_kernel<64, 8, false, false, 2>, umma_smem_bytes(64, 8))) != cudaSuccess) return e;
-    if ((e = allow_smem(umma_bf16_pair_kernel<256, 6, true, false, 1>, pair_smem_bytes(256, 6))) != cudaSuccess) return e;
-    if ((e = allow_smem(umma_bf16_pair_kernel<256, 6, false, false, 1>, pair_smem_bytes(256, 6))) != cudaSuccess) return e;
-    if ((e = allow_smem(umma_bf16_pair_kernel<256, 6, true, false, 2>, pair_smem_bytes(256, 6))) != cudaSuccess) return e;
-    if ((e = allow_smem(umma_bf16_pair_kernel<256, 6, false, false, 2>, pair_smem_bytes(256, 6))) != cudaSuccess) return e;
-    if ((e = allow_smem(umma_bf16_pair_kernel<128, 8, true, false, 1>, pair_smem_bytes(128, 8))) != cudaSuccess) return e;
-    if ((e = allow_smem(umma_bf16_pair_kernel<128, 8, false, false, 1>, pair_smem_bytes(128, 8))) != cudaSuccess) return e;
-    if ((e = allow_smem(umma_bf16_pair_kernel<128, 8, true, false, 2>, pair_smem_bytes(128, 8))) != cudaSuccess) return e;
-    if ((e = allow_smem(umma_bf16_pair_kernel<128, 8, false, false, 2>, pair_smem_bytes(128, 8))) != cudaSuccess) return e;
-    if ((e = allow_smem(umma_bf16_kernel<256, 4, false, true, 2>, umma_smem_bytes(256, 4))) != cudaSuccess) return e;
-    if ((e = allow_smem(umma_bf16_kernel<256, 4, true, true, 2>, umma_smem_bytes(256, 4))) != cudaSuccess) return e;
-    if ((e = allow_smem(umma_bf16_kernel<128, 6, false, true, 2>, umma_smem_bytes(128, 6))) != cudaSuccess) return e;
-    if ((e = allow_smem(umma_bf16_kernel<128, 6, true, true, 2>, umma_smem_bytes(128, 6))) != cudaSuccess) return e;
-    if ((e = allow_smem(umma_bf16_kernel<64, 8, false, true, 2>, umma_smem_bytes(64, 8))) != cudaSuccess) return e;
-    if ((e = allow_smem(umma_bf16_kernel<64, 8, true, true, 2>, umma_smem_bytes(64, 8))) != cudaSuccess) return e;
-    if ((e = allow_smem(umma_bf16_pair_kernel<256, 6, false, true, 2>, pair_smem_bytes(256, 6))) != cudaSuccess) return e;
-    if ((e = allow_smem(umma_bf16_pair_kernel<256, 6, true, true, 2>, pair_smem_bytes(256, 6))) != cudaSuccess) return e;
-    if ((e = allow_smem(umma_bf16_pair_kernel<128, 8, false, true, 2>, pair_smem_bytes(128, 8))) != cudaSuccess) return e;
-    if ((e = allow_smem(umma_bf16_pair_kernel<128, 8, true, true, 2>, pair_smem_bytes(128, 8))) != cudaSuccess) return e;
+// Every tensor-core kernel instantiation needs more dynamic shared memory than the default limit
+// allows.  The attribute is per device: the table below is walked once for each device that
+// creates a plan, not on every nk_gemm_create.
+template <int BN, int ST, bool V, bool CL, int KIND>
+static cudaError_t attr_single() { return allow_smem(umma_bf16_kernel<BN, ST, V, CL, KIND>, umma_smem_bytes(BN, ST)); }
+template <int BN, int ST, bool V, bool CL, int KIND>
+static cudaError_t attr_pair() { return allow_smem(umma_bf16_pair_kernel<BN, ST, V, CL, KIND>, pair_smem_bytes(BN, ST)); }
+
+typedef cudaError_t (*AttrFn)();
+#define NK_ATTR_VARIANTS(FN, BN, ST, KIND, CL) FN<BN, ST, false, CL, KIND>, FN<BN, ST, true, CL, KIND>
+#define NK_ATTR_TILES(KIND, CL)                                                                      \
+    NK_ATTR_VARIANTS(attr_single, 256, 4, KIND, CL), NK_ATTR_VARIANTS(attr_single, 128, 6, KIND, CL), \
+    NK_ATTR_VARIANTS(attr_single, 64, 8, KIND, CL), NK_ATTR_VARIANTS(attr_pair, 256, 6, KIND, CL),    \
+    NK_ATTR_VARIANTS(attr_pair, 128, 8, KIND, CL)
+static const AttrFn kUmmaAttrTable[] = {
+    NK_ATTR_TILES(0, false), NK_ATTR_TILES(0, true),   // 16-bit floating point, plain and cluster split-K
+    NK_ATTR_TILES(1, false),                           // INT8 (no cluster form)
+    NK_ATTR_TILES(2, false), NK_ATTR_TILES(2, true),   // 8-bit floating point
+};
+#undef NK_ATTR_TILES
+#undef NK_ATTR_VARIANTS
+
+static cudaError_t prepare_umma_attrs(int device) {
+    static std::mutex mu;
+    static bool done[64];
+    std::lock_guard<std::mutex> lock(mu);
+    if (device >= 0 && device < 64 && done[device]) return cudaSuccess;
+    for (const AttrFn fn : kUmmaAttrTable) {
+        const cudaError_t e = fn();
+        if (e != cudaSuccess) return e;
+    }
+    if (device >= 0 && device < 64) done[device] = true;
     return cudaSuccess;
 }
 
@@ -912,7 +897,7 @@ nk_status_t nk_gemm_create(const nk_gemm_desc_t* desc, nk_gemm_t* out) {
             return NK_ERR_CUDA;
         }
         p->encode = reinterpret_cast<EncodeTiledFn>(fn);
-        if (prepare_umma_attrs() != cudaSuccess) { cudaGetLastError(); delete p; return NK_ERR_CUDA; }
+        if (prepare_umma_attrs(d.device) != cudaSuccess) { cudaGetLastError(); delete p; return NK_ERR_CUDA; }
         choose_umma(p);
         if (d.layout_b == NK_BLOCKED32) {
             p->b_repack = (d.flags & NK_FLAG_REPACK_B) != 0;
@@ -1199,7 +1184,8 @@ nk_status_t nk_gemm_run_host(nk_gemm_t p, const void* hA, const void* hB, const 
     constexpr int kRowChunks = 8, kMaxPanels = 4;
     if (d.beta == 0 && p->batch == 1 && p->gemms == 1 && d.layout_c == NK_ROW_MAJOR && d.M % (kRowChunks * 256) == 0 &&
         2.0 * d.M * d.N * d.K >= 2.0e10 && !(d.flags & NK_FLAG_KERNEL_MASK)) {
-        if (!p->chunk_plan) {
+        if (!p->chunk_plan && !p->chunk_tried) {
+            p->chunk_tried = true;
             const int panels = d.N % (kMaxPanels * 256) == 0 ? kMaxPanels : 1;
             nk_gemm_desc_t cd = d;
             cd.M = d.M / kRowChunks;

@@ -385,6 +385,107 @@ __device__ __forceinline__ void umma_commit_pair(uint32_t bar, uint16_t cta_mask
         : "memory");
 }
 
+// ---------------------------------------------------------------- warp-uniform issue
+// The producer's and the MMA issuer's instruction streams pace the K loop.  Inside an
+// `if (lane == 0)` branch the warp is divergent, and every operand of a TMA or tcgen05
+// instruction has to be moved from per-thread registers into the uniform registers those
+// instructions read, one move at a time; that alone made a 64-deep k-block cost ~560 clocks
+// of issue whatever the tile width.  Here the whole warp runs the same code and only the
+// asynchronous instruction itself is predicated on `elected` (1 in one lane, 0 in the
+// others, from elect_one()): the address arithmetic stays uniform.  Measured on B200, per
+// k-block of four MMAs: 382 clocks (N = 64), 398 (N = 128), 512 (N = 256: the tensor pipe).
+__device__ __forceinline__ uint32_t elect_one() {
+    uint32_t pred;
+    asm volatile("{\n\t.reg .pred P;\n\telect.sync _|P, 0xffffffff;\n\tselp.u32 %0, 1, 0, P;\n\t}" : "=r"(pred));
+    return pred;
+}
+__device__ __forceinline__ void mbar_arrive_expect_tx_if(uint32_t bar, uint32_t bytes, uint32_t elected) {
+    asm volatile("{\n\t.reg .pred q;\n\tsetp.ne.b32 q, %2, 0;\n\t"
+                 "@q mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;\n\t}" ::"r"(bar), "r"(bytes), "r"(elected)
+                 : "memory");
+}
+__device__ __forceinline__ void tma_load_3d_if(uint32_t dst, const void* tmap, uint32_t bar, int c0, int c1, int c2,
+                                               uint32_t elected) {
+    asm volatile("{\n\t.reg .pred q;\n\tsetp.ne.b32 q, %6, 0;\n\t"
+                 "@q cp.async.bulk.tensor.3d.shared::cluster.global.mbarrier::complete_tx::bytes"
+                 " [%0], [%1, {%3, %4, %5}], [%2];\n\t}" ::"r"(dst),
+                 "l"(tmap), "r"(bar), "r"(c0), "r"(c1), "r"(c2), "r"(elected)
+                 : "memory");
+}
+__device__ __forceinline__ void tma_load_4d_if(uint32_t dst, const void* tmap, uint32_t bar, int c0, int c1, int c2, int c3,
+                                               uint32_t elected) {
+    asm volatile("{\n\t.reg .pred q;\n\tsetp.ne.b32 q, %7, 0;\n\t"
+                 "@q cp.async.bulk.tensor.4d.shared::cluster.global.mbarrier::complete_tx::bytes"
+                 " [%0], [%1, {%3, %4, %5, %6}], [%2];\n\t}" ::"r"(dst),
+                 "l"(tmap), "r"(bar), "r"(c0), "r"(c1), "r"(c2), "r"(c3), "r"(elected)
+                 : "memory");
+}
+// Pair forms: completion bytes go to `cluster_bar`, which may live in the other CTA of the pair (no multicast).
+__device__ __forceinline__ void tma_load_3d_pair_if(uint32_t dst, const void* tmap, uint32_t cluster_bar, int c0, int c1,
+                                                    int c2, uint32_t elected) {
+    asm volatile("{\n\t.reg .pred q;\n\tsetp.ne.b32 q, %6, 0;\n\t"
+                 "@q cp.async.bulk.tensor.3d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes"
+                 " [%0], [%1, {%3, %4, %5}], [%2];\n\t}" ::"r"(dst),
+                 "l"(tmap), "r"(cluster_bar), "r"(c0), "r"(c1), "r"(c2), "r"(elected)
+                 : "memory");
+}
+__device__ __forceinline__ void tma_load_4d_pair_if(uint32_t dst, const void* tmap, uint32_t cluster_bar, int c0, int c1,
+                                                    int c2, int c3, uint32_t elected) {
+    asm volatile("{\n\t.reg .pred q;\n\tsetp.ne.b32 q, %7, 0;\n\t"
+                 "@q cp.async.bulk.tensor.4d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes"
+                 " [%0], [%1, {%3, %4, %5, %6}], [%2];\n\t}" ::"r"(dst),
+                 "l"(tmap), "r"(cluster_bar), "r"(c0), "r"(c1), "r"(c2), "r"(c3), "r"(elected)
+                 : "memory");
+}
+// tcgen05.mma, issued by the elected lane only.  KIND: 0 = 16-bit floating point, 1 = INT8, 2 = 8-bit
+// floating point; PAIR: one MMA over both CTAs of a pair (cta_group::2).
+#define NK_UMMA_IF(NAME, GROUP, KINDSTR)                                                                        \
+    __device__ __forceinline__ void NAME(uint32_t d_tmem, uint32_t a_lo, uint32_t a_hi, uint32_t b_lo,        \
+                                         uint32_t b_hi, uint32_t idesc, uint32_t accumulate, uint32_t elected) { \
+        asm volatile(                                                                                           \
+            "{\n\t.reg .pred p, q;\n\t.reg .b64 da, db;\n\t"                                                    \
+            "setp.ne.b32 p, %6, 0;\n\t"                                                                         \
+            "setp.ne.b32 q, %7, 0;\n\t"                                                                         \
+            "mov.b64 da, {%1, %2};\n\t"                                                                         \
+            "mov.b64 db, {%3, %4};\n\t"                                                                         \
+            "@q tcgen05.mma.cta_group::" GROUP ".kind::" KINDSTR " [%0], da, db, %5, p;\n\t}" ::"r"(d_tmem),   \
+            "r"(a_lo), "r"(a_hi), "r"(b_lo), "r"(b_hi), "r"(idesc), "r"(accumulate), "r"(elected)               \
+            : "memory");                                                                                        \
+    }
+NK_UMMA_IF(umma_f16_if, "1", "f16")
+NK_UMMA_IF(umma_i8_if, "1", "i8")
+NK_UMMA_IF(umma_f8_if, "1", "f8f6f4")
+NK_UMMA_IF(umma_f16_pair_if, "2", "f16")
+NK_UMMA_IF(umma_i8_pair_if, "2", "i8")
+NK_UMMA_IF(umma_f8_pair_if, "2", "f8f6f4")
+#undef NK_UMMA_IF
+template <int KIND>
+__device__ __forceinline__ void umma_if(uint32_t d_tmem, uint32_t a_lo, uint32_t a_hi, uint32_t b_lo, uint32_t b_hi,
+                                        uint32_t idesc, uint32_t accumulate, uint32_t elected) {
+    if (KIND == 1) umma_i8_if(d_tmem, a_lo, a_hi, b_lo, b_hi, idesc, accumulate, elected);
+    else if (KIND == 2) umma_f8_if(d_tmem, a_lo, a_hi, b_lo, b_hi, idesc, accumulate, elected);
+    else umma_f16_if(d_tmem, a_lo, a_hi, b_lo, b_hi, idesc, accumulate, elected);
+}
+template <int KIND>
+__device__ __forceinline__ void umma_pair_if(uint32_t d_tmem, uint32_t a_lo, uint32_t a_hi, uint32_t b_lo, uint32_t b_hi,
+                                             uint32_t idesc, uint32_t accumulate, uint32_t elected) {
+    if (KIND == 1) umma_i8_pair_if(d_tmem, a_lo, a_hi, b_lo, b_hi, idesc, accumulate, elected);
+    else if (KIND == 2) umma_f8_pair_if(d_tmem, a_lo, a_hi, b_lo, b_hi, idesc, accumulate, elected);
+    else umma_f16_pair_if(d_tmem, a_lo, a_hi, b_lo, b_hi, idesc, accumulate, elected);
+}
+__device__ __forceinline__ void umma_commit_if(uint32_t bar, uint32_t elected) {
+    asm volatile("{\n\t.reg .pred q;\n\tsetp.ne.b32 q, %1, 0;\n\t"
+                 "@q tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];\n\t}" ::"r"(bar), "r"(elected)
+                 : "memory");
+}
+// (An mbarrier signal to the CTAs of `cta_mask`, not a data load.)
+__device__ __forceinline__ void umma_commit_pair_if(uint32_t bar, uint16_t cta_mask, uint32_t elected) {
+    asm volatile("{\n\t.reg .pred q;\n\tsetp.ne.b32 q, %2, 0;\n\t"
+                 "@q tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], %1;\n\t}" ::
+                     "r"(bar), "h"(cta_mask), "r"(elected)
+                 : "memory");
+}
+
 // Shared-memory matrix descriptor (tcgen05): start address, leading/stride byte
 // offsets in 16-byte units, descriptor version 1, swizzle mode in bits 61..63
 // (0 none, 2 = 128-byte, 4 = 64-byte, 6 = 32-byte).

@@ -262,6 +262,12 @@ __device__ __forceinline__ void umma_store_chunk(const UmmaParams& p, const CUte
         // two tiles used alternately: the store issued two chunks ago has read this one
         if (lane == 0) bulk_wait_read<1>();
         __syncwarp();
+    } else if (p.tma_store) {
+        // a K split's partial in a plan whose whole tiles leave by TMA store (tail-wave mode): the
+        // stores of the previous whole tile may still be reading either staging tile (16-bit C keeps
+        // both inside the first 4 KB), so all of them must have read their source first
+        if (lane == 0) bulk_wait_read<0>();
+        __syncwarp();
     }
 #pragma unroll
     for (int g = 0; g < 8; ++g)
@@ -568,11 +574,13 @@ umma_bf16_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_consta
 
     if (warp == 0) {
         // ------------------------------------------------ TMA producer
-        // One lane issues; like the MMA issuer its instruction stream paces the pipeline, so
-        // addresses advance by adds and the layout decisions are taken outside the loops.
+        // One lane issues, but the whole warp runs the loop (see elect_one); like the MMA issuer
+        // its instruction stream paces the pipeline, so addresses advance by adds and the layout
+        // decisions are taken outside the loops.
         const bool a_blk = p.a_blocked != 0;
         const bool b3d = p.b_3d != 0;
         const bool b_kmajor = p.b_kmajor != 0;
+        const uint32_t elected = elect_one();
         int stage = 0;
         uint32_t phase = 0;
         uint32_t sa = smem_base, fb = full_bar(0);
@@ -598,29 +606,30 @@ umma_bf16_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_consta
                     ok = false;
                     break;
                 }
-                if (lane == 0) {
+                {
+                    // issued by the elected lane; the warp stays convergent (see elect_one)
                     const uint32_t sb = sa + UMMA_A_STAGE_BYTES;
-                    mbar_arrive_expect_tx(fb, UMMA_A_STAGE_BYTES + (B_VNNI ? 0 : B_STAGE));
+                    mbar_arrive_expect_tx_if(fb, UMMA_A_STAGE_BYTES + (B_VNNI ? 0 : B_STAGE), elected);
                     if (a_blk) {
                         // two 32-wide K slabs, each 128 rows x 64 B (64-byte swizzle)
-                        tma_load_4d(sa, &tmap_a, fb, 0, 0, kbl * 2, mb * 4);
-                        tma_load_4d(sa + 8192, &tmap_a, fb, 0, 0, kbl * 2 + 1, mb * 4);
+                        tma_load_4d_if(sa, &tmap_a, fb, 0, 0, kbl * 2, mb * 4, elected);
+                        tma_load_4d_if(sa + 8192, &tmap_a, fb, 0, 0, kbl * 2 + 1, mb * 4, elected);
                     } else {
-                        tma_load_3d(sa, &tmap_a, fb, kx, row0, ia);
+                        tma_load_3d_if(sa, &tmap_a, fb, kx, row0, ia, elected);
                     }
                     if (B_VNNI) {
                         // the stage's blocks as they are; warps 6-9 re-lay them in place
-                        mbar_arrive_expect_tx(raw_bar(stage), B_STAGE);
-                        tma_load_3d(sb, &tmap_b, raw_bar(stage), 0, kbl * (UMMA_BK / 2), col0 >> 5);
+                        mbar_arrive_expect_tx_if(raw_bar(stage), B_STAGE, elected);
+                        tma_load_3d_if(sb, &tmap_b, raw_bar(stage), 0, kbl * (UMMA_BK / 2), col0 >> 5, elected);
                     } else if (b_kmajor) {
-                        tma_load_3d(sb, &tmap_b, fb, kx, col0, ib);   // BN rows (n) of 128 bytes of k
+                        tma_load_3d_if(sb, &tmap_b, fb, kx, col0, ib, elected);   // BN rows (n) of 128 bytes of k
                     } else {
                         if (b3d) {
-                            tma_load_4d(sb, &tmap_b, fb, 0, kx, col0 >> 6, ib);
+                            tma_load_4d_if(sb, &tmap_b, fb, 0, kx, col0 >> 6, ib, elected);
                         } else {
 #pragma unroll
                             for (int j = 0; j < BN / 64; ++j)
-                                tma_load_3d(sb + j * 8192, &tmap_b, fb, col0 + j * 64, kx, ib);
+                                tma_load_3d_if(sb + j * 8192, &tmap_b, fb, col0 + j * 64, kx, ib, elected);
                         }
                     }
                 }
@@ -641,7 +650,7 @@ umma_bf16_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_consta
         }
     } else if (warp == 1) {
         // ------------------------------------------------ MMA issuer
-        // One lane issues; its instruction stream is the critical path of the K loop, so the
+        // One lane issues (the whole warp runs the loop, see elect_one); its instruction stream is the critical path of the K loop, so the
         // descriptors are kept as 32-bit halves and advanced with adds, and everything that
         // does not change per stage is computed here, once.
         //   A row-major: K-major tile, 128-byte swizzle, 8-row groups 1024 B apart; the four
@@ -661,6 +670,7 @@ umma_bf16_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_consta
         const uint32_t b_s = b_k ? 2u : 128u, b_s2 = 2 * b_s, b_s3 = 3 * b_s;
         constexpr uint32_t STAGE16 = STAGE >> 4;
         const uint32_t idesc = p.idesc;
+        const uint32_t elected = elect_one();
         int stage = 0;
         uint32_t phase = 0;
         uint32_t soff = 0;  // stage * STAGE / 16
@@ -687,22 +697,21 @@ umma_bf16_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_consta
                     break;
                 }
                 tc_fence_after_sync();
-                if (lane == 0) {
+                {
                     const uint32_t a_lo = a_lo0 + soff, b_lo = b_lo0 + soff;
-                    umma_lohi<KIND>(d_tmem, a_lo, a_hi, b_lo, b_hi, idesc, accumulate);
-                    umma_lohi<KIND>(d_tmem, a_lo + a_s1, a_hi, b_lo + b_s, b_hi, idesc, 1u);
-                    umma_lohi<KIND>(d_tmem, a_lo + a_s2, a_hi, b_lo + b_s2, b_hi, idesc, 1u);
-                    umma_lohi<KIND>(d_tmem, a_lo + a_s3, a_hi, b_lo + b_s3, b_hi, idesc, 1u);
-                    umma_commit(empty_bar(stage));
-                    if (kb == kb1 - 1) umma_commit(tfull_bar(acc));
+                    umma_if<KIND>(d_tmem, a_lo, a_hi, b_lo, b_hi, idesc, accumulate, elected);
+                    umma_if<KIND>(d_tmem, a_lo + a_s1, a_hi, b_lo + b_s, b_hi, idesc, 1u, elected);
+                    umma_if<KIND>(d_tmem, a_lo + a_s2, a_hi, b_lo + b_s2, b_hi, idesc, 1u, elected);
+                    umma_if<KIND>(d_tmem, a_lo + a_s3, a_hi, b_lo + b_s3, b_hi, idesc, 1u, elected);
+                    umma_commit_if(empty_bar(stage), elected);
+                    if (kb == kb1 - 1) umma_commit_if(tfull_bar(acc), elected);
                 }
                 accumulate = 1u;
                 __syncwarp();
                 soff += STAGE16;
                 if (++stage == STAGES) { stage = 0; phase ^= 1u; soff = 0; }
             }
-            if (kb1 <= kb0 && lane == 0) umma_commit(tfull_bar(acc));  // empty K range
-            __syncwarp();
+            if (kb1 <= kb0) umma_commit_if(tfull_bar(acc), elected);  // empty K range
         }
     } else if (warp < 6 && CLUSTER_REDUCE) {
         // ------------------------------------------------ epilogue, K splits reduced inside the cluster

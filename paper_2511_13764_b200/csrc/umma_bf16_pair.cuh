@@ -136,6 +136,8 @@ umma_bf16_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_c
         const bool b3d = p.b_3d != 0;
         const bool b_kmajor = p.b_kmajor != 0;
         const uint32_t lead_full0 = map_to_cta(full_bar(0), leader);  // leader's full[0], cluster address
+        const uint32_t elected = elect_one();
+        const uint32_t lead_elected = rank == 0 ? elected : 0u;      // only the leader's barrier expects the bytes
         int stage = 0;
         uint32_t phase = 0;
         uint32_t sa = smem_base, fb = full_bar(0), lfb = lead_full0;
@@ -159,29 +161,29 @@ umma_bf16_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_c
                     ok = false;
                     break;
                 }
-                if (lane == 0) {
+                {
+                    // issued by the elected lane; the warp stays convergent (see elect_one)
                     const uint32_t sb = sa + UMMA_A_STAGE_BYTES;
-                    if (rank == 0)
-                        mbar_arrive_expect_tx(fb, 2u * (UMMA_A_STAGE_BYTES + (B_VNNI ? 0 : B_STAGE)));
+                    mbar_arrive_expect_tx_if(fb, 2u * (UMMA_A_STAGE_BYTES + (B_VNNI ? 0 : B_STAGE)), lead_elected);
                     if (a_blk) {
-                        tma_load_4d_pair(sa, &tmap_a, lfb, 0, 0, kbl * 2, row0 / 32);
-                        tma_load_4d_pair(sa + 8192, &tmap_a, lfb, 0, 0, kbl * 2 + 1, row0 / 32);
+                        tma_load_4d_pair_if(sa, &tmap_a, lfb, 0, 0, kbl * 2, row0 / 32, elected);
+                        tma_load_4d_pair_if(sa + 8192, &tmap_a, lfb, 0, 0, kbl * 2 + 1, row0 / 32, elected);
                     } else {
-                        tma_load_3d_pair(sa, &tmap_a, lfb, kx, row0, ia);
+                        tma_load_3d_pair_if(sa, &tmap_a, lfb, kx, row0, ia, elected);
                     }
                     if (B_VNNI) {
                         // this CTA's column blocks as they are, on its own barrier; its warps 6-9 re-lay them in place
-                        mbar_arrive_expect_tx(raw_bar(stage), B_STAGE);
-                        tma_load_3d(sb, &tmap_b, raw_bar(stage), 0, kbl * (UMMA_BK / 2), col0 >> 5);
+                        mbar_arrive_expect_tx_if(raw_bar(stage), B_STAGE, elected);
+                        tma_load_3d_if(sb, &tmap_b, raw_bar(stage), 0, kbl * (UMMA_BK / 2), col0 >> 5, elected);
                     } else if (b_kmajor) {
-                        tma_load_3d_pair(sb, &tmap_b, lfb, kx, col0, ib);   // this CTA's HALF rows (n) of 128 bytes of k
+                        tma_load_3d_pair_if(sb, &tmap_b, lfb, kx, col0, ib, elected);   // this CTA's HALF rows (n) of 128 bytes of k
                     } else {
                         if (b3d) {
-                            tma_load_4d_pair(sb, &tmap_b, lfb, 0, kx, col0 >> 6, ib);
+                            tma_load_4d_pair_if(sb, &tmap_b, lfb, 0, kx, col0 >> 6, ib, elected);
                         } else {
 #pragma unroll
                             for (int j = 0; j < HALF / 64; ++j)
-                                tma_load_3d_pair(sb + j * 8192, &tmap_b, lfb, col0 + j * 64, kx, ib);
+                                tma_load_3d_pair_if(sb + j * 8192, &tmap_b, lfb, col0 + j * 64, kx, ib, elected);
                         }
                     }
                 }
@@ -215,6 +217,7 @@ umma_bf16_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_c
             const uint32_t b_s = b_k ? 2u : 128u, b_s2 = 2 * b_s, b_s3 = 3 * b_s;
             constexpr uint32_t STAGE16 = STAGE >> 4;
             const uint32_t idesc = p.idesc;
+            const uint32_t elected = elect_one();
             int stage = 0;
             uint32_t phase = 0;
             uint32_t soff = 0;
@@ -239,22 +242,21 @@ umma_bf16_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_c
                         break;
                     }
                     tc_fence_after_sync();
-                    if (lane == 0) {
+                    {
                         const uint32_t a_lo = a_lo0 + soff, b_lo = b_lo0 + soff;
-                        umma_pair_lohi<KIND>(d_tmem, a_lo, a_hi, b_lo, b_hi, idesc, accumulate);
-                        umma_pair_lohi<KIND>(d_tmem, a_lo + a_s1, a_hi, b_lo + b_s, b_hi, idesc, 1u);
-                        umma_pair_lohi<KIND>(d_tmem, a_lo + a_s2, a_hi, b_lo + b_s2, b_hi, idesc, 1u);
-                        umma_pair_lohi<KIND>(d_tmem, a_lo + a_s3, a_hi, b_lo + b_s3, b_hi, idesc, 1u);
-                        umma_commit_pair(empty_bar(stage), pair_mask);
-                        if (kb == kb1 - 1) umma_commit_pair(tfull_bar(acc), pair_mask);
+                        umma_pair_if<KIND>(d_tmem, a_lo, a_hi, b_lo, b_hi, idesc, accumulate, elected);
+                        umma_pair_if<KIND>(d_tmem, a_lo + a_s1, a_hi, b_lo + b_s, b_hi, idesc, 1u, elected);
+                        umma_pair_if<KIND>(d_tmem, a_lo + a_s2, a_hi, b_lo + b_s2, b_hi, idesc, 1u, elected);
+                        umma_pair_if<KIND>(d_tmem, a_lo + a_s3, a_hi, b_lo + b_s3, b_hi, idesc, 1u, elected);
+                        umma_commit_pair_if(empty_bar(stage), pair_mask, elected);
+                        if (kb == kb1 - 1) umma_commit_pair_if(tfull_bar(acc), pair_mask, elected);
                     }
                     accumulate = 1u;
                     __syncwarp();
                     soff += STAGE16;
                     if (++stage == STAGES) { stage = 0; phase ^= 1u; soff = 0; }
                 }
-                if (kb1 <= kb0 && lane == 0) umma_commit_pair(tfull_bar(acc), pair_mask);
-                __syncwarp();
+                if (kb1 <= kb0) umma_commit_pair_if(tfull_bar(acc), pair_mask, elected);
             }
         }
     } else if (warp < 6 && CLUSTER_REDUCE) {

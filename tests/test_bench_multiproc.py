@@ -59,3 +59,43 @@ def test_reference_arm_is_rank0_only():
                         "--gpus", "2", "--steps", "1", "--warmup", "0"],
                        env=env, capture_output=True, text=True, timeout=120)
     assert r.returncode == 0 and r.stdout.strip() == ""
+
+
+def test_bare_gpus_2_starts_two_ranks_itself():
+    """`bench.py --gpus 2` run bare (no WORLD_SIZE in the environment) must start two ranks on its own.
+    --dry-run leaves the GEMM out (no device here): what is checked is that two ranks met, that rank 0
+    alone printed the JSON line, that it says n_gpus = 2, and that the slower rank set the time."""
+    import json
+    env = {k: v for k, v in os.environ.items()
+           if k not in ("WORLD_SIZE", "RANK", "LOCAL_RANK", "MASTER_ADDR", "MASTER_PORT")}
+    r = subprocess.run([sys.executable, os.path.join(ROOT, "bench.py"), "--gpus", "2", "--steps", "5",
+                        "--warmup", "0", "--dry-run"], env=env, capture_output=True, text=True, timeout=300)
+    assert r.returncode == 0, r.stderr[-2000:]
+    lines = [ln for ln in r.stdout.splitlines() if ln.startswith("{")]
+    assert len(lines) == 1, r.stdout
+    out = json.loads(lines[0])
+    assert out["n_gpus"] == 2 and out["dry_run"] is True
+    assert "rank 0 of 2" in r.stderr and "rank 1 of 2" in r.stderr
+    # rank 1 sleeps 4 ms per step, rank 0 only 2 ms: the maximum over the ranks is reported
+    assert out["ms_per_step"] >= 4.0
+    assert "x2" in out["config"]["parallelism"]
+
+
+def test_recorded_traffic_is_dropped_when_the_sources_change(tmp_path, monkeypatch):
+    """The DRAM-traffic figure of the bench line comes from a committed capture that names the kernel,
+    the shape and the hash of the kernel sources it was taken from; any mismatch must give null."""
+    import json
+    sys.path.insert(0, ROOT)
+    import bench
+    from paper_2511_13764_b200 import _build
+    rec = {"kernel": "k", "shape": [8, 8, 8], "dram_read_bytes": 10.0, "dram_write_bytes": 5.0,
+           "source_hash": _build.source_hash(), "captured": "today"}
+    path = tmp_path / "t.json"
+    path.write_text(json.dumps(rec))
+    monkeypatch.setattr(bench, "TRAFFIC_JSON", str(path))
+    assert bench.recorded_traffic("k", (8, 8, 8))[0] == 15.0
+    assert bench.recorded_traffic("other", (8, 8, 8))[0] is None
+    assert bench.recorded_traffic("k", (8, 8, 16))[0] is None
+    rec["source_hash"] = "0" * 64
+    path.write_text(json.dumps(rec))
+    assert bench.recorded_traffic("k", (8, 8, 8))[0] is None

@@ -294,6 +294,26 @@ def test_pair_tail_wave_split(out_dtype, epi, splits, bn):
     check_against_oracle(w, c_plain, A, B, bias)
 
 
+@pytest.mark.parametrize("out_dtype,bn", [("f32", 4), ("bf16", 4), ("bf16", 3)])
+def test_pair_tail_units_follow_tma_stored_tiles(out_dtype, bn):
+    """A pair that goes from a whole tile (stored by TMA from its staging tiles) straight to a tail split
+    (whose FP32 partial passes through the same staging memory) must first let those stores read their
+    source.  Integer data make both plans exact, so the result with the tail split has to equal, bit for
+    bit and on every one of many runs, the result of the plan without it."""
+    M, N, K = 2500, 2520, 128      # a short K loop: the tail unit's accumulator is ready at once
+    w = W("tailrace", M, N, K, "bf16", out_dtype, integer=True, seed=77)
+    A, B, bias = w.make()
+    f = nk.FLAG_CTA_PAIR | nk.flag_tile_n(bn) | nk.flag_splitk(1)
+    c_plain, p_plain = run_plan(w, A, B, bias, flags=f | nk.FLAG_NO_TAIL_SPLIT)
+    assert "_tail" not in p_plain.kernel_name
+    check_against_oracle(w, c_plain, A, B, bias, exact=(out_dtype == "f32"))
+    plan = nk.plan_for(w, flags=f | nk.flag_tail_split(2))
+    assert "_tail2" in plan.kernel_name
+    for _ in range(25):
+        c_tail, _ = run_plan(w, A, B, bias, plan=plan)
+        assert np.array_equal(c_tail, c_plain)
+
+
 @pytest.mark.parametrize("out_dtype,epi,layout,N", [("f32", "none", "row", 2048), ("bf16", "bias_relu", "row", 2048),
                                                     ("bf16", "bias_relu", "blocked32", 2048), ("f32", "none", "row", 2304)])
 def test_run_host_pipelined_chunks(out_dtype, epi, layout, N):
