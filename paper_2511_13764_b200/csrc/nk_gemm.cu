@@ -167,7 +167,7 @@ static int desc_gemms(const nk_gemm_desc_t& d) { return (d.batch > 1 && d.batch_
 
 // Co-resident clusters of the cluster split-K variant (pair?, tile N, VNNI?, splits), as the driver
 // reports them for the current device; asked once per device and variant and remembered.
-static int max_clusters_for(bool pair, int bn, bool vnni, int splits, bool f8);
+static int max_clusters_for(bool pair, int bn, bool vnni, int splits, int kind);
 
 // K splits can meet inside a cluster (no partials in global memory, no second kernel) when there
 // are 2, 4 or 8 of them (2 or 4 pairs) and all the units of the plan are resident at once (one
@@ -176,11 +176,10 @@ static int max_clusters_for(bool pair, int bn, bool vnni, int splits, bool f8);
 static bool cluster_reduce_fits(const nk_gemm_desc_t& d, int sms, bool pair, int bn, int eff_splits) {
     (void)sms;
     if (d.flags & NK_FLAG_SEPARATE_REDUCE) return false;
-    if (is_s8(d)) return false;   // INT32 partial sums: the cluster reduction adds FP32 pieces only
     if (eff_splits != 2 && eff_splits != 4 && !(eff_splits == 8 && !pair)) return false;
     const int64_t clusters = static_cast<int64_t>(desc_gemms(d)) * ceil_div(d.M, pair ? 2 * UMMA_BM : UMMA_BM) * ceil_div(d.N, bn);
     const bool vnni = d.layout_b == NK_BLOCKED32 && !(d.flags & NK_FLAG_REPACK_B);
-    return clusters <= max_clusters_for(pair, bn, vnni, eff_splits, is_f8(d));
+    return clusters <= max_clusters_for(pair, bn, vnni, eff_splits, is_f8(d) ? 2 : is_s8(d) ? 1 : 0);
 }
 
 static double umma_model_us(const nk_gemm_desc_t& d, int sms, bool pair, int bn, int splits) {
@@ -489,7 +488,7 @@ static nk_status_t encode_c_map(nk_gemm_s* p, void* C) {
 
 template <int BN, int STAGES, bool VNNI, int KIND = 0>
 static cudaError_t launch_umma_t(nk_gemm_s* p, const UmmaParams& up, int grid, cudaStream_t st) {
-    umma_bf16_kernel<BN, STAGES, VNNI, false, KIND><<<grid, VNNI ? 320 : 192, umma_smem_bytes(BN, STAGES), st>>>(
+    umma_bf16_kernel<BN, STAGES, VNNI, false, KIND><<<grid, UMMA_THREADS, umma_smem_bytes(BN, STAGES), st>>>(
         p->tmap_a, p->tmap_b, p->tmap_c, up);
     return cudaGetLastError();
 }
@@ -540,12 +539,12 @@ static cudaError_t launch_clustered(Kernel kernel, nk_gemm_s* p, const UmmaParam
 }
 
 // `units` = tiles x splits; the single-CTA kernel runs one CTA per unit, the pair kernel two.
-// KIND as in the kernels (0 = 16-bit floating point, 2 = 8-bit floating point; INT8 has no cluster form).
+// KIND as in the kernels (0 = 16-bit floating point, 1 = INT8, 2 = 8-bit floating point).
 template <int KIND>
 static cudaError_t launch_cluster_k(nk_gemm_s* p, const UmmaParams& up, int units, int splits, cudaStream_t st,
                                     int* max_clusters) {
     const bool v = p->b_vnni_inkernel;
-    const int th = v ? 320 : 192;
+    const int th = UMMA_THREADS;
 #define NK_CL(K, ctas, cl, smem) launch_clustered(K, p, up, ctas, cl, th, smem, st, max_clusters)
     if (p->pair) {
         if (p->bn == 256)
@@ -568,12 +567,13 @@ static cudaError_t launch_cluster_k(nk_gemm_s* p, const UmmaParams& up, int unit
 static cudaError_t launch_cluster(nk_gemm_s* p, const UmmaParams& up, int units, int splits, cudaStream_t st,
                                   int* max_clusters) {
     return is_f8(p->d) ? launch_cluster_k<2>(p, up, units, splits, st, max_clusters)
-                       : launch_cluster_k<0>(p, up, units, splits, st, max_clusters);
+           : is_s8(p->d) ? launch_cluster_k<1>(p, up, units, splits, st, max_clusters)
+                         : launch_cluster_k<0>(p, up, units, splits, st, max_clusters);
 }
 
-static int max_clusters_for(bool pair, int bn, bool vnni, int splits, bool f8) {
+static int max_clusters_for(bool pair, int bn, bool vnni, int splits, int kind) {
     static std::mutex mu;
-    static int cache[16][2][2][3][2][9];   // [device][8-bit float?][pair?][tile][VNNI?][splits]: 0 = not asked yet, -1 = none
+    static int cache[16][3][2][3][2][9];   // [device][kind][pair?][tile][VNNI?][splits]: 0 = not asked yet, -1 = none
     const int bi = bn == 256 ? 2 : bn == 128 ? 1 : 0;
     if (splits < 2 || splits > 8) return 0;
     int dev = 0;
@@ -583,7 +583,7 @@ static int max_clusters_for(bool pair, int bn, bool vnni, int splits, bool f8) {
     tmp.pair = pair;
     tmp.bn = bn;
     tmp.b_vnni_inkernel = vnni;
-    tmp.d.in_dtype = f8 ? NK_E4M3 : NK_BF16;
+    tmp.d.in_dtype = kind == 2 ? NK_E4M3 : kind == 1 ? NK_S8 : NK_BF16;
     auto ask = [&]() {
         int n = 0;
         if (launch_cluster(&tmp, UmmaParams(), 0, splits, nullptr, &n) != cudaSuccess || n <= 0) {
@@ -594,7 +594,7 @@ static int max_clusters_for(bool pair, int bn, bool vnni, int splits, bool f8) {
     };
     if (dev < 0 || dev >= 16) { const int n = ask(); return n > 0 ? n : 0; }   // beyond the cache: ask every time
     std::lock_guard<std::mutex> lock(mu);
-    int& c = cache[dev][f8 ? 1 : 0][pair ? 1 : 0][bi][vnni ? 1 : 0][splits];
+    int& c = cache[dev][kind][pair ? 1 : 0][bi][vnni ? 1 : 0][splits];
     if (c == 0) c = ask();
     return c > 0 ? c : 0;
 }
@@ -604,7 +604,7 @@ static cudaError_t launch_pair_t(nk_gemm_s* p, const UmmaParams& up, int pairs, 
     cudaLaunchConfig_t cfg;
     memset(&cfg, 0, sizeof(cfg));
     cfg.gridDim = dim3(static_cast<unsigned>(2 * pairs));
-    cfg.blockDim = dim3(VNNI ? 320 : 192);
+    cfg.blockDim = dim3(UMMA_THREADS);
     cfg.dynamicSmemBytes = pair_smem_bytes(BN, STAGES);
     cfg.stream = st;
     cudaLaunchAttribute attr;
@@ -636,7 +636,7 @@ static cudaError_t pair_occupancy(int* out) {
     cudaLaunchConfig_t cfg;
     memset(&cfg, 0, sizeof(cfg));
     cfg.gridDim = dim3(2);
-    cfg.blockDim = dim3(VNNI ? 320 : 192);
+    cfg.blockDim = dim3(UMMA_THREADS);
     cfg.dynamicSmemBytes = pair_smem_bytes(BN, STAGES);
     cudaLaunchAttribute attr;
     attr.id = cudaLaunchAttributeClusterDimension;
@@ -668,7 +668,7 @@ typedef cudaError_t (*AttrFn)();
     NK_ATTR_VARIANTS(attr_pair, 128, 8, KIND, CL)
 static const AttrFn kUmmaAttrTable[] = {
     NK_ATTR_TILES(0, false), NK_ATTR_TILES(0, true),   // 16-bit floating point, plain and cluster split-K
-    NK_ATTR_TILES(1, false),                           // INT8 (no cluster form)
+    NK_ATTR_TILES(1, false), NK_ATTR_TILES(1, true),   // INT8
     NK_ATTR_TILES(2, false), NK_ATTR_TILES(2, true),   // 8-bit floating point
 };
 #undef NK_ATTR_TILES
@@ -1119,6 +1119,7 @@ nk_status_t nk_gemm_run(nk_gemm_t p, const void* A, const void* B, const void* b
         up.bias_f32 = (p->bias_f32 || is_8bit(d)) ? 1 : 0;
         up.dequant = (is_s8(d) && d.out_dtype == NK_F32) ? 1 : 0;
         up.scale = d.scale;
+        up.acc_s32 = is_s8(d) ? 1 : 0;
         up.item_remap = p->item_remap ? 1 : 0;
         up.item_map_a = p->item_map_a;
         up.item_map_b = p->item_map_b;

@@ -8,16 +8,17 @@
 // pipelining of Algorithm 3, AMX branch), and bias + ReLU are applied to the
 // accumulator before the single store of C (Section 6, "MLP").
 //
-// Warp roles (192 threads, +128 when B is VNNI-blocked):
+// Warp roles (320 threads):
 //   warp 0      TMA producer: A tile 128 x 64 (K-major), B tile 64 x BN (N-major)
 //   warp 1      MMA issuer and TMEM owner: 4 x tcgen05.mma 128 x BN x 16 per stage
 //   warps 2-5   epilogue: tcgen05.ld -> (+bias, ReLU, cvt) -> global stores; two
 //               TMEM accumulators so tile t's epilogue overlaps tile t+1's K loop
-//   warps 6-9   (VNNI-blocked B only) re-layout: the producer's TMA box brings the
+//   warps 6-9   with VNNI-blocked B, re-layout: the producer's TMA box brings the
 //               [k/2][n][2] blocks of a stage as they are; these warps transpose them
 //               as 32-bit words, in place, into the K-major swizzled stage (the
 //               in-kernel counterpart of the paper's software-pipelined pack step,
-//               in the opposite direction)
+//               in the opposite direction).  In a CTA that delivers a single tile they
+//               are also the second half of the epilogue (half of the columns each)
 //
 // Every mbarrier wait is bounded; a role that gives up raises the CTA's abort
 // flag and the device status word, the other roles fall out of their loops, and
@@ -40,6 +41,7 @@ namespace nk {
 constexpr int UMMA_BM = 128;
 constexpr int UMMA_BK = 64;
 constexpr int UMMA_A_STAGE_BYTES = UMMA_BM * UMMA_BK * 2;  // 16 KB
+constexpr int UMMA_THREADS = 320;   // producer, MMA issuer, 4 epilogue warps, 4 re-layout / second-epilogue warps
 
 struct UmmaParams {
     int M, N, K;
@@ -70,6 +72,7 @@ struct UmmaParams {
     int bias_f32;       // the bias vector is FP32 although the operands are not (split-FP32 and quantised plans)
     int dequant;        // the accumulator holds INT32 sums: convert to FP32 and multiply by `scale` before the epilogue
     float scale;
+    int acc_s32;        // the accumulator holds INT32 sums (INT8 operands): K splits are added as integers
     int item_remap;     // batch item i multiplies A item (item_map_a >> 4i) & 15 by B item (item_map_b >> 4i) & 15
     uint32_t item_map_a, item_map_b;
     unsigned int* status;
@@ -98,25 +101,44 @@ __host__ __device__ constexpr int umma_smem_bytes(int BN, int stages) {
 // a CTA's 128 x BN accumulator are shared out over the splits, so a CTA's slots never exceed one
 // accumulator (BN * 512 bytes), which fits the stage ring of every variant
 
+// a / b for 0 <= a < 2^24, 0 < b < 2^24 without the integer-division routine (some forty dependent
+// instructions; the producer decodes its first unit before it can issue the first load, and on a
+// short problem that wait is visible): a single-precision estimate, then one exact correction step.
+__device__ __forceinline__ int div_small(int a, int b) {
+    int q = __float2int_rz(__fdividef(__int2float_rz(a), __int2float_rz(b)));
+    int r = a - q * b;             // the estimate is off by one at most (the loops run once or not at all)
+    while (r < 0) { --q; r += b; }
+    while (r >= b) { ++q; r -= b; }
+    return q;
+}
+
 // tile id -> (m block, n block): groups of `group_m` M tiles sweep across N so
 // that CTAs running at the same time share A rows and B columns in L2.
 __device__ __forceinline__ void umma_tile_coords(const UmmaParams& p, int tile, int& mb, int& nb) {
     const int per_group = p.group_m * p.tiles_n;
-    const int g = tile / per_group;
+    const int g = div_small(tile, per_group);
     const int within = tile - g * per_group;
     const int first_m = g * p.group_m;
     const int gm = min(p.group_m, p.tiles_m - first_m);
-    mb = first_m + within % gm;
-    nb = within / gm;
+    nb = div_small(within, gm);
+    mb = first_m + within - nb * gm;
 }
 
 // unit id -> (independent GEMM, tile, K split)
 __device__ __forceinline__ void umma_decode_unit(const UmmaParams& p, int unit, int& tile, int& split, int& gemm) {
-    const int per_gemm = p.tiles_m * p.tiles_n * p.splits;
-    gemm = unit / per_gemm;
-    const int u = unit - gemm * per_gemm;
-    tile = u / p.splits;
-    split = u - tile * p.splits;
+    gemm = 0;
+    int u = unit;
+    if (p.gemms > 1) {
+        const int per_gemm = p.tiles_m * p.tiles_n * p.splits;
+        gemm = div_small(unit, per_gemm);
+        u = unit - gemm * per_gemm;
+    }
+    tile = u;
+    split = 0;
+    if (p.splits > 1) {
+        tile = div_small(u, p.splits);
+        split = u - tile * p.splits;
+    }
 }
 
 // Where the FP32 partial of a chunk goes: base[(row0 + r) * ld + col0 + c], clipped to rows x cols.
@@ -124,6 +146,84 @@ struct PartialDst {
     float* base;
     int ld, row0, col0, rows, cols;
 };
+
+// Two FP32 adds in one instruction (add.rn.f32x2: the same IEEE results as two scalar adds).
+__device__ __forceinline__ void add2_f32(uint32_t& a0, uint32_t& a1, uint32_t b0, uint32_t b1) {
+    asm("{\n\t.reg .b64 x, y;\n\tmov.b64 x, {%0, %1};\n\tmov.b64 y, {%2, %3};\n\tadd.rn.f32x2 x, x, y;\n\tmov.b64 {%0, %1}, x;\n\t}"
+        : "+r"(a0), "+r"(a1)
+        : "r"(b0), "r"(b1));
+}
+
+// bias + ReLU (Section 6, the MLP layer) on one 32 x 32 chunk held as a row per lane.  `bias_sm`:
+// the chunk's 32 bias values as FP32 in shared memory (parked there by umma_park_bias while the K
+// loop was still running); without it the values come from global memory, 16-bit or FP32.
+__device__ __forceinline__ void umma_chunk_bias_relu(const UmmaParams& p, uint32_t (&v)[32], int col0,
+                                                     const float* bias_sm) {
+    if (!p.epilogue) return;
+    if (bias_sm) {
+#pragma unroll
+        for (int g = 0; g < 8; ++g) {
+            const uint4 b = reinterpret_cast<const uint4*>(bias_sm)[g];
+            add2_f32(v[4 * g], v[4 * g + 1], b.x, b.y);
+            add2_f32(v[4 * g + 2], v[4 * g + 3], b.z, b.w);
+        }
+#pragma unroll
+        for (int i = 0; i < 32; ++i) v[i] = __float_as_uint(fmaxf(__uint_as_float(v[i]), 0.0f));
+    } else if (p.bias_f32) {
+        const float4* bsrc = reinterpret_cast<const float4*>(static_cast<const float*>(p.bias) + col0);
+#pragma unroll
+        for (int g = 0; g < 8; ++g) {
+            if (col0 + 4 * g >= p.N) break;
+            const float4 b = __ldg(bsrc + g);
+            v[4 * g] = __float_as_uint(fmaxf(__uint_as_float(v[4 * g]) + b.x, 0.0f));
+            v[4 * g + 1] = __float_as_uint(fmaxf(__uint_as_float(v[4 * g + 1]) + b.y, 0.0f));
+            v[4 * g + 2] = __float_as_uint(fmaxf(__uint_as_float(v[4 * g + 2]) + b.z, 0.0f));
+            v[4 * g + 3] = __float_as_uint(fmaxf(__uint_as_float(v[4 * g + 3]) + b.w, 0.0f));
+        }
+    } else {
+        const uint4* bsrc = reinterpret_cast<const uint4*>(static_cast<const uint16_t*>(p.bias) + col0);
+#pragma unroll
+        for (int g = 0; g < 4; ++g) {
+            if (col0 + 8 * g >= p.N) break;
+            const uint4 b = __ldg(bsrc + g);
+            const uint32_t w[4] = {b.x, b.y, b.z, b.w};
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+                float x0 = __uint_as_float(v[8 * g + 2 * j]) + half_bits_to_f32(w[j] & 0xFFFFu, p.f16);
+                float x1 = __uint_as_float(v[8 * g + 2 * j + 1]) + half_bits_to_f32(w[j] >> 16, p.f16);
+                v[8 * g + 2 * j] = __float_as_uint(fmaxf(x0, 0.0f));
+                v[8 * g + 2 * j + 1] = __float_as_uint(fmaxf(x1, 0.0f));
+            }
+        }
+    }
+}
+
+// One 32 x 32 chunk in the layout a TMA store of a 32 x 32 box reads: FP32 rows of 128 bytes with the
+// 128-byte swizzle (16-byte group g of row t at group g ^ (t & 7)), 16-bit rows of 64 bytes with the
+// 64-byte swizzle (group g at g ^ ((t >> 1) & 3)); both conflict-free for a row per lane.
+template <bool F16>
+__device__ __forceinline__ void umma_write_tile16(const uint32_t (&v)[32], int lane, uint8_t* tile) {
+#pragma unroll
+    for (int g = 0; g < 4; ++g) {
+        uint4 o;
+        o.x = pack_half2(__uint_as_float(v[8 * g]), __uint_as_float(v[8 * g + 1]), F16);
+        o.y = pack_half2(__uint_as_float(v[8 * g + 2]), __uint_as_float(v[8 * g + 3]), F16);
+        o.z = pack_half2(__uint_as_float(v[8 * g + 4]), __uint_as_float(v[8 * g + 5]), F16);
+        o.w = pack_half2(__uint_as_float(v[8 * g + 6]), __uint_as_float(v[8 * g + 7]), F16);
+        *reinterpret_cast<uint4*>(tile + lane * 64 + ((g ^ ((lane >> 1) & 3)) << 4)) = o;
+    }
+}
+__device__ __forceinline__ void umma_write_store_tile(const UmmaParams& p, const uint32_t (&v)[32], int lane, uint8_t* tile) {
+    if (p.out_bf16) {
+        if (p.f16) umma_write_tile16<true>(v, lane, tile);
+        else umma_write_tile16<false>(v, lane, tile);
+    } else {
+#pragma unroll
+        for (int g = 0; g < 8; ++g)
+            *reinterpret_cast<uint4*>(tile + lane * 128 + ((g ^ (lane & 7)) << 4)) =
+                make_uint4(v[4 * g], v[4 * g + 1], v[4 * g + 2], v[4 * g + 3]);
+    }
+}
 
 // Epilogue for one 32 x 32 chunk of the accumulator: lane t holds row `row0 + t`, columns
 // col0 .. col0+31 as FP32 bit patterns.  Either the raw FP32 partial of a K split, or bias +
@@ -135,11 +235,11 @@ struct PartialDst {
 //
 // `staging` is the warp's 8 KB of shared memory: two 4 KB (FP32) or two 2 KB (BF16) tiles used
 // alternately (`parity`) as TMA-store sources; with BF16 output the bias slice of the tile
-// (`bias_smem`, one value per tile column, fetched while the K loop was still running) sits
+// (`bias_smem`, one FP32 value per tile column, fetched while the K loop was still running) sits
 // behind them.
 __device__ __forceinline__ void umma_store_chunk(const UmmaParams& p, const CUtensorMap* tmap_c, uint32_t (&v)[32],
                                                  int row0, int lane, int col0, int split, int gemm, bool empty_k,
-                                                 uint8_t* staging, int parity, const uint16_t* bias_smem,
+                                                 uint8_t* staging, int parity, const float* bias_smem,
                                                  const PartialDst* pd) {
     const bool to_partial = pd != nullptr;      // a K split's FP32 partial instead of the final C
     const bool tma_store = p.tma_store && !to_partial;
@@ -188,33 +288,7 @@ __device__ __forceinline__ void umma_store_chunk(const UmmaParams& p, const CUte
             }
         }
     }
-    if (!to_partial && p.epilogue && p.bias_f32) {
-        const float4* bsrc = reinterpret_cast<const float4*>(static_cast<const float*>(p.bias) + col0);
-#pragma unroll
-        for (int g = 0; g < 8; ++g) {
-            if (col0 + 4 * g >= p.N) break;
-            const float4 b = __ldg(bsrc + g);
-            v[4 * g] = __float_as_uint(fmaxf(__uint_as_float(v[4 * g]) + b.x, 0.0f));
-            v[4 * g + 1] = __float_as_uint(fmaxf(__uint_as_float(v[4 * g + 1]) + b.y, 0.0f));
-            v[4 * g + 2] = __float_as_uint(fmaxf(__uint_as_float(v[4 * g + 2]) + b.z, 0.0f));
-            v[4 * g + 3] = __float_as_uint(fmaxf(__uint_as_float(v[4 * g + 3]) + b.w, 0.0f));
-        }
-    } else if (!to_partial && p.epilogue) {
-        const uint4* bsrc = reinterpret_cast<const uint4*>(static_cast<const uint16_t*>(p.bias) + col0);
-#pragma unroll
-        for (int g = 0; g < 4; ++g) {
-            if (col0 + 8 * g >= p.N) break;
-            const uint4 b = bias_smem ? reinterpret_cast<const uint4*>(bias_smem)[g] : __ldg(bsrc + g);
-            const uint32_t w[4] = {b.x, b.y, b.z, b.w};
-#pragma unroll
-            for (int j = 0; j < 4; ++j) {
-                float x0 = __uint_as_float(v[8 * g + 2 * j]) + half_bits_to_f32(w[j] & 0xFFFFu, p.f16);
-                float x1 = __uint_as_float(v[8 * g + 2 * j + 1]) + half_bits_to_f32(w[j] >> 16, p.f16);
-                v[8 * g + 2 * j] = __float_as_uint(fmaxf(x0, 0.0f));
-                v[8 * g + 2 * j + 1] = __float_as_uint(fmaxf(x1, 0.0f));
-            }
-        }
-    }
+    if (!to_partial) umma_chunk_bias_relu(p, v, col0, bias_smem);
     if (!to_partial && p.out_bf16 && tma_store) {
         // BF16 rows (64 bytes) -> staging, 16-byte chunk g of row t at chunk g ^ ((t >> 1) & 3) (the
         // 64-byte swizzle: conflict-free stores) -> one TMA store of the 32 x 32 box
@@ -307,113 +381,165 @@ __device__ __forceinline__ void umma_store_chunk(const UmmaParams& p, const CUte
     __syncwarp();   // the buffer is reused by the next chunk
 }
 
-// With BF16 output the warp's staging tiles take 4 KB of its 8 KB: the bias slice of the tile
-// (BN values) is parked behind them before the wait for the accumulator, so that its global
-// latency is hidden behind the K loop instead of being paid in every chunk.
+// The bias slice of a tile (BN values from column col_tile0 on), widened to FP32 and parked at `dst`
+// in shared memory (BN * 4 bytes) before the wait for the accumulator, so that its global latency
+// hides behind the K loop and the chunks pay shared-memory reads only.  Null without an epilogue.
 template <int BN>
-__device__ __forceinline__ const uint16_t* umma_fetch_bias(const UmmaParams& p, uint8_t* staging, int col_tile0, int lane) {
-    if (!p.epilogue || !p.out_bf16 || p.splits > 1) return nullptr;   // (cluster plans park the slice in the ring)
-    uint4* dst = reinterpret_cast<uint4*>(staging + 4096);
+__device__ __forceinline__ const float* umma_park_bias(const UmmaParams& p, float* dst, int col_tile0, int lane) {
+    if (!p.epilogue) return nullptr;
     if (lane < BN / 8) {
-        const int col = col_tile0 + 8 * lane;
-        dst[lane] = col < p.N ? __ldg(reinterpret_cast<const uint4*>(static_cast<const uint16_t*>(p.bias) + col))
-                              : make_uint4(0u, 0u, 0u, 0u);
+        const int col = col_tile0 + 8 * lane;        // N is a multiple of 8: eight columns are in or out together
+        float4 lo = make_float4(0.f, 0.f, 0.f, 0.f), hi = lo;
+        if (col < p.N) {
+            if (p.bias_f32) {
+                lo = __ldg(reinterpret_cast<const float4*>(static_cast<const float*>(p.bias) + col));
+                hi = __ldg(reinterpret_cast<const float4*>(static_cast<const float*>(p.bias) + col) + 1);
+            } else {
+                const uint4 b = __ldg(reinterpret_cast<const uint4*>(static_cast<const uint16_t*>(p.bias) + col));
+                lo = make_float4(half_bits_to_f32(b.x & 0xFFFFu, p.f16), half_bits_to_f32(b.x >> 16, p.f16),
+                                 half_bits_to_f32(b.y & 0xFFFFu, p.f16), half_bits_to_f32(b.y >> 16, p.f16));
+                hi = make_float4(half_bits_to_f32(b.z & 0xFFFFu, p.f16), half_bits_to_f32(b.z >> 16, p.f16),
+                                 half_bits_to_f32(b.w & 0xFFFFu, p.f16), half_bits_to_f32(b.w >> 16, p.f16));
+            }
+        }
+        reinterpret_cast<float4*>(dst)[2 * lane] = lo;
+        reinterpret_cast<float4*>(dst)[2 * lane + 1] = hi;
     }
     __syncwarp();
-    return reinterpret_cast<const uint16_t*>(dst);
+    return dst;
 }
 
-// The lane's 16 bytes of the tile's bias slice (lanes 0 .. BN/8-1), for the cluster epilogue.
+// In the chunk-at-a-time epilogue the slice fits behind the staging tiles only with a 16-bit C
+// (two 2 KB tiles): parked at staging + 4096, else read from global memory chunk by chunk.
 template <int BN>
-__device__ __forceinline__ uint4 umma_load_bias_reg(const UmmaParams& p, int col_tile0, int lane, bool& have) {
-    have = p.epilogue && p.out_bf16;
-    uint4 r = make_uint4(0u, 0u, 0u, 0u);
-    const int col = col_tile0 + 8 * lane;
-    if (have && lane < BN / 8 && col < p.N)
-        r = __ldg(reinterpret_cast<const uint4*>(static_cast<const uint16_t*>(p.bias) + col));
-    return r;
+__device__ __forceinline__ const float* umma_fetch_bias(const UmmaParams& p, uint8_t* staging, int col_tile0, int lane) {
+    if (!p.out_bf16 || p.splits > 1) return nullptr;
+    return umma_park_bias<BN>(p, reinterpret_cast<float*>(staging + 4096), col_tile0, lane);
+}
+
+// Epilogue of a CTA that has a single tile to deliver (a problem of one wave or less), C row-major and
+// stored by TMA.  By the time the accumulator is complete every stage of the operand ring has been
+// consumed and nothing will be loaded again, so the ring serves as store staging: a warp converts
+// ALL its chunks first (a tile each, `tiles` = the warp's region of the ring, 1024-byte aligned), pays
+// one proxy fence and one warp barrier, and then issues its box stores back to back as one bulk
+// group.  The chunk-at-a-time scheme costs ~550 clocks per chunk in fence, barrier, issue and
+// buffer-reuse waits; this one ~150 per chunk plus ~300 once.  Two warps share each quarter of the
+// accumulator's rows (tensor-memory lanes are tied to warp % 4): this one takes chunks c0 .. c1-1.
+template <int BN>
+__device__ __forceinline__ void umma_epilogue_oneshot(const UmmaParams& p, const CUtensorMap* tmap_c, uint32_t taddr,
+                                                      uint8_t* tiles, int row0, int col_tile0, int gemm, int lane,
+                                                      bool empty_k, const float* bias_sm, int c0, int c1) {
+    const uint32_t tile_bytes = p.out_bf16 ? 2048u : 4096u;
+    if (row0 >= p.M) return;
+#pragma unroll 1
+    for (int c = c0; c < c1; c += 2) {
+        if (col_tile0 + c * 32 >= p.N) break;        // warp-uniform
+        const bool two = c + 1 < c1 && col_tile0 + c * 32 + 32 < p.N;
+        uint32_t v0[32], v1[32];
+        tmem_ld_32x32(taddr + c * 32, v0);
+        if (two) tmem_ld_32x32(taddr + c * 32 + 32, v1);
+        tmem_ld_wait();
+        if (empty_k) {
+#pragma unroll
+            for (int i = 0; i < 32; ++i) v0[i] = v1[i] = 0u;
+        }
+        if (p.dequant) {
+#pragma unroll
+            for (int i = 0; i < 32; ++i) {
+                v0[i] = __float_as_uint(__int2float_rn(static_cast<int>(v0[i])) * p.scale);
+                v1[i] = __float_as_uint(__int2float_rn(static_cast<int>(v1[i])) * p.scale);
+            }
+        }
+        umma_chunk_bias_relu(p, v0, col_tile0 + c * 32, bias_sm ? bias_sm + c * 32 : nullptr);
+        umma_write_store_tile(p, v0, lane, tiles + (c - c0) * tile_bytes);
+        if (two) {
+            umma_chunk_bias_relu(p, v1, col_tile0 + c * 32 + 32, bias_sm ? bias_sm + c * 32 + 32 : nullptr);
+            umma_write_store_tile(p, v1, lane, tiles + (c - c0 + 1) * tile_bytes);
+        }
+    }
+    fence_proxy_async_smem();
+    __syncwarp();
+    if (lane == 0) {
+#pragma unroll 1
+        for (int c = c0; c < c1; ++c)
+            if (col_tile0 + c * 32 < p.N) tma_store_3d(tmap_c, smem_u32(tiles + (c - c0) * tile_bytes), col_tile0 + c * 32, row0, gemm);
+        bulk_commit();
+    }
 }
 
 // Epilogue of a cluster split-K CTA.  Its accumulator (128 rows x BN columns, tensor-memory
 // columns 0..BN-1) is cut into 4 * BN / 32 pieces, piece u = quarter * (BN / 32) + chunk; the CTAs
 // that hold the S splits of the same rows have cluster ranks rank0 + s * rank_step.  Piece u
-// belongs to split u % S; the other splits send theirs into slot (u / S) * S + source split of
+// belongs to split u % S; the other splits write theirs into slot (u / S) * S + source split of
 // the owner's stage ring (idle by then), the owner's own contribution stays in tensor memory.
 //   barrier  every CTA of the cluster has finished its K loop: the rings may be overwritten
-//   send     tcgen05.ld -> the warp's staging tile (16-byte group g of row t at g * 512 +
-//            (t ^ g) * 16: conflict-free on both sides) -> one 4 KB bulk copy into the owner's
-//            slot, counted in on the owner's `recv` mbarrier (per-thread remote stores were
-//            several times slower)
-//   wait     the owner's mbarrier has seen all the bytes it expects (bounded wait)
-//   reduce   every owned piece is summed in split order (the result does not depend on timing)
-//            and leaves through the ordinary chunk epilogue: beta, bias + ReLU, conversion, store
-// Every thread of the cluster passes the barrier, also after a wait that gave up.
+//   send     tcgen05.ld -> remote shared-memory stores straight from the registers, a warp writing
+//            512 contiguous bytes per instruction (16-byte group g of row t at g * 512 + (t ^ g) * 16:
+//            conflict-free when the owner reads it back).  The SM-to-SM path moves 16-23 bytes per
+//            clock per CTA whatever the method (bulk copies, remote loads, remote stores; measured),
+//            so what counts is that all the pieces are in flight at once and nothing waits in between
+//   barrier  (release / acquire) every piece has landed everywhere
+//   reduce   every owned piece is summed in split order (the result does not depend on timing;
+//            INT32 sums are added as integers), gets the epilogue, and all the owned chunks leave
+//            as one batch of TMA stores staged behind the slots
+// Every thread of the cluster passes both barriers, also in a CTA where a wait gave up (`ok` false).
+// `bias_sm`: the tile's bias slice as FP32 in shared memory (umma_park_bias), or null.
 template <int BN>
-__host__ __device__ constexpr uint32_t umma_cluster_recv_bytes(uint32_t S) { return (4u * (BN / 32) / S) * (S - 1u) * 4096u; }
+__host__ __device__ constexpr uint32_t umma_cluster_slot_bytes() { return BN * 512u; }
 
+// Eight warps run this, two per quarter of the accumulator's rows (tensor-memory lanes are tied to
+// warp % 4); `half` (0 or 1) picks the warp's half of the BN / 32 chunks.  Plans that cannot store
+// by TMA (beta, blocked C) let the second set of warps send only: the first set then reduces and
+// stores all the owned chunks one at a time through its staging tiles.
 template <int BN>
 __device__ __forceinline__ bool umma_cluster_epilogue(const UmmaParams& p, const CUtensorMap* tmap_c, uint32_t tmem_base,
-                                                      uint32_t ring, const uint8_t* ring_gen, uint32_t recv_bar,
-                                                      volatile uint32_t* abort_flag, uint8_t* staging, uint8_t* bias_park,
-                                                      uint4 bias_reg, bool have_bias, int quarter, int lane, uint32_t S,
+                                                      uint32_t ring, uint8_t* ring_gen, uint8_t* staging,
+                                                      const float* bias_sm, int quarter, int half, int lane, uint32_t S,
                                                       uint32_t split, uint32_t rank0, uint32_t rank_step, int row_cta0,
                                                       int col_tile0, int gemm, bool ok) {
-    constexpr uint32_t NC = BN / 32;
+    constexpr uint32_t NC = BN / 32, HC = NC / 2;
     const uint32_t lane_tmem = static_cast<uint32_t>(quarter * 32) << 16;
+    const uint32_t c_lo = half * HC, c_hi = c_lo + HC;
     cluster_arrive();
     cluster_wait();
-    // The bias slice of the tile was loaded into a register per lane before the accumulator was
-    // ready; it is parked behind the receive slots of the ring now that the ring is free (the
-    // staging tiles, where the ordinary epilogue keeps it, are the send buffers here).
-    const uint16_t* bias_smem = nullptr;
-    if (have_bias) {
-        if (lane < BN / 8) reinterpret_cast<uint4*>(bias_park)[lane] = bias_reg;
-        __syncwarp();
-        bias_smem = reinterpret_cast<const uint16_t*>(bias_park);
-    }
     if (ok) {
-        uint32_t parity = 0;
 #pragma unroll 1
-        for (uint32_t c = 0; c < NC; ++c) {
-            const uint32_t u = quarter * NC + c, owner = u % S;
+        for (uint32_t c = c_lo; c < c_hi; ++c) {
+            const uint32_t u = quarter * NC + c, owner = u & (S - 1u);      // S is 2, 4 or 8
             if (owner == split) continue;                // mine: stays in tensor memory (warp-uniform)
             uint32_t v[32];
             tmem_ld_32x32(tmem_base + c * 32 + lane_tmem, v);
             tmem_ld_wait();
-            uint8_t* tile = staging + parity * 4096;
-            if (lane == 0) bulk_wait_read<1>();          // the copy issued two pieces ago has read this tile
-            __syncwarp();
+            const uint32_t dst = map_to_cta(ring + ((u & ~(S - 1u)) + split) * 4096u, rank0 + owner * rank_step);
 #pragma unroll
             for (int g = 0; g < 8; ++g)
-                *reinterpret_cast<uint4*>(tile + g * 512 + ((lane ^ g) << 4)) =
-                    make_uint4(v[4 * g], v[4 * g + 1], v[4 * g + 2], v[4 * g + 3]);
-            fence_proxy_async_smem();
-            __syncwarp();
-            if (lane == 0) {
-                const uint32_t peer = rank0 + owner * rank_step;
-                bulk_copy_to_cluster(map_to_cta(ring + ((u / S) * S + split) * 4096u, peer), smem_u32(tile), 4096u,
-                                     map_to_cta(recv_bar, peer));
-                bulk_commit();
-            }
-            parity ^= 1u;
+                st_cluster_v4(dst + g * 512 + ((lane ^ g) << 4), v[4 * g], v[4 * g + 1], v[4 * g + 2], v[4 * g + 3]);
         }
-        if (!mbar_wait(recv_bar, 0u, abort_flag)) ok = false;   // every piece sent to this CTA has landed
-    } else {
-        // this CTA gave up, but healthy peers may still be copying into it: let their copies land
-        mbar_wait(recv_bar, 0u, abort_flag, 1ll << 24);
     }
-    if (lane == 0) bulk_wait_read<0>();                  // the staging tiles are free again
-    __syncwarp();
+    cluster_arrive();
+    cluster_wait();
     if (!ok) return false;
+    const bool batched = p.tma_store != 0;
+    if (!batched && half != 0) return true;
+    const uint32_t r_lo = batched ? c_lo : 0u, r_hi = batched ? c_hi : NC;
+    // store tiles of the owned chunks: behind the receive slots, max(1, HC / S) per warp
+    constexpr uint32_t kSlots = umma_cluster_slot_bytes<BN>();
+    const uint32_t per_warp = HC / S > 0 ? HC / S : 1u;
+    const uint32_t tile_bytes = p.out_bf16 ? 2048u : 4096u;
+    uint8_t* tiles = ring_gen + kSlots + (quarter * 2 + half) * per_warp * 4096u;
+    const int row0 = row_cta0 + quarter * 32;
+    uint32_t ntiles = 0;
     int parity = 0;
 #pragma unroll 1
-    for (uint32_t c = 0; c < NC; ++c) {
+    for (uint32_t c = r_lo; c < r_hi; ++c) {
         const uint32_t u = quarter * NC + c;
-        if (u % S != split) continue;                    // warp-uniform
+        if ((u & (S - 1u)) != split) continue;           // warp-uniform
+        const int col0 = col_tile0 + static_cast<int>(c) * 32;
+        if (batched && (col0 >= p.N || row0 >= p.M)) continue;
         uint32_t own[32], v[32];
         tmem_ld_32x32(tmem_base + c * 32 + lane_tmem, own);
         tmem_ld_wait();
-        const uint8_t* slot0 = ring_gen + (u / S) * S * 4096u;
+        const uint8_t* slot0 = ring_gen + (u & ~(S - 1u)) * 4096u;
         // split order s = 0, 1, .., S-1, this CTA's own accumulator taking its place in the row
 #pragma unroll 1
         for (uint32_t sp = 0; sp < S; ++sp) {
@@ -421,30 +547,66 @@ __device__ __forceinline__ bool umma_cluster_epilogue(const UmmaParams& p, const
                 if (sp == 0) {
 #pragma unroll
                     for (int i = 0; i < 32; ++i) v[i] = own[i];
+                } else if (p.acc_s32) {
+#pragma unroll
+                    for (int i = 0; i < 32; ++i) v[i] += own[i];
                 } else {
 #pragma unroll
-                    for (int i = 0; i < 32; ++i) v[i] = __float_as_uint(__uint_as_float(v[i]) + __uint_as_float(own[i]));
+                    for (int i = 0; i < 32; i += 2) add2_f32(v[i], v[i + 1], own[i], own[i + 1]);
                 }
                 continue;
             }
             const uint8_t* slot = slot0 + sp * 4096u;
+            if (sp == 0) {
 #pragma unroll
-            for (int g = 0; g < 8; ++g) {
-                const uint4 t4 = *reinterpret_cast<const uint4*>(slot + g * 512 + ((lane ^ g) << 4));
-                if (sp == 0) {
+                for (int g = 0; g < 8; ++g) {
+                    const uint4 t4 = *reinterpret_cast<const uint4*>(slot + g * 512 + ((lane ^ g) << 4));
                     v[4 * g] = t4.x; v[4 * g + 1] = t4.y; v[4 * g + 2] = t4.z; v[4 * g + 3] = t4.w;
-                } else {
-                    v[4 * g] = __float_as_uint(__uint_as_float(v[4 * g]) + __uint_as_float(t4.x));
-                    v[4 * g + 1] = __float_as_uint(__uint_as_float(v[4 * g + 1]) + __uint_as_float(t4.y));
-                    v[4 * g + 2] = __float_as_uint(__uint_as_float(v[4 * g + 2]) + __uint_as_float(t4.z));
-                    v[4 * g + 3] = __float_as_uint(__uint_as_float(v[4 * g + 3]) + __uint_as_float(t4.w));
+                }
+            } else if (p.acc_s32) {
+#pragma unroll
+                for (int g = 0; g < 8; ++g) {
+                    const uint4 t4 = *reinterpret_cast<const uint4*>(slot + g * 512 + ((lane ^ g) << 4));
+                    v[4 * g] += t4.x; v[4 * g + 1] += t4.y; v[4 * g + 2] += t4.z; v[4 * g + 3] += t4.w;
+                }
+            } else {
+#pragma unroll
+                for (int g = 0; g < 8; ++g) {
+                    const uint4 t4 = *reinterpret_cast<const uint4*>(slot + g * 512 + ((lane ^ g) << 4));
+                    add2_f32(v[4 * g], v[4 * g + 1], t4.x, t4.y);
+                    add2_f32(v[4 * g + 2], v[4 * g + 3], t4.z, t4.w);
                 }
             }
         }
-        umma_store_chunk(p, tmap_c, v, row_cta0 + quarter * 32, lane, col_tile0 + static_cast<int>(c) * 32, 0, gemm,
-                         false, staging, parity, bias_smem ? bias_smem + c * 32 : nullptr, nullptr);
+        if (!batched) {
+            // beta, blocked C: the chunk-at-a-time path through the warp's staging tiles
+            umma_store_chunk(p, tmap_c, v, row0, lane, col0, 0, gemm, false, staging, parity, nullptr, nullptr);
+            __syncwarp();
+            parity ^= 1;
+            continue;
+        }
+        if (p.dequant) {
+#pragma unroll
+            for (int i = 0; i < 32; ++i) v[i] = __float_as_uint(__int2float_rn(static_cast<int>(v[i])) * p.scale);
+        }
+        umma_chunk_bias_relu(p, v, col0, bias_sm ? bias_sm + c * 32 : nullptr);
+        umma_write_store_tile(p, v, lane, tiles + ntiles * tile_bytes);
+        ++ntiles;
+    }
+    if (batched && ntiles > 0) {
+        fence_proxy_async_smem();
         __syncwarp();
-        parity ^= 1;
+        if (lane == 0) {
+            // the owned chunks of the range, in the order their tiles were filled
+            uint32_t k = 0;
+#pragma unroll 1
+            for (uint32_t c = r_lo; c < r_hi && k < ntiles; ++c) {
+                if (((quarter * NC + c) & (S - 1u)) != split) continue;
+                tma_store_3d(tmap_c, smem_u32(tiles + k * tile_bytes), col_tile0 + static_cast<int>(c) * 32, row0, gemm);
+                ++k;
+            }
+            bulk_commit();
+        }
     }
     if (lane == 0) bulk_wait_all();
     __syncwarp();
@@ -497,7 +659,7 @@ __device__ __forceinline__ void vnni_relayout_stage(uint32_t sb, int tw, int lan
 }
 
 template <int BN, int STAGES, bool B_VNNI, bool CLUSTER_REDUCE = false, int KIND = 0>
-__global__ void __launch_bounds__(B_VNNI ? 320 : 192, 1)
+__global__ void __launch_bounds__(UMMA_THREADS, 1)
 umma_bf16_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ CUtensorMap tmap_b,
                  const __grid_constant__ CUtensorMap tmap_c, const UmmaParams p) {
     static_assert(BN % 32 == 0 && BN >= 32 && BN <= 256, "tile N");
@@ -524,24 +686,17 @@ umma_bf16_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_consta
     const int warp = threadIdx.x >> 5;
     const int lane = threadIdx.x & 31;
 
-    if (threadIdx.x == 0) {
-        for (int s = 0; s < STAGES; ++s) {
-            mbar_init(full_bar(s), B_VNNI ? 1 + 4 : 1);
-            mbar_init(empty_bar(s), 1);
-            if (B_VNNI) mbar_init(raw_bar(s), 1);
-        }
-        for (int a = 0; a < 2; ++a) {
-            mbar_init(tfull_bar(a), 1);
-            mbar_init(tempty_bar(a), 128);
-        }
-        *abort_flag = 0;
-        if (CLUSTER_REDUCE) {
-            // the pieces other CTAs will send to this one are counted in on this barrier
-            mbar_init(bar_base + 192u, 1);
-        }
+    if (warp == 0) {
+        // one barrier per lane: full[STAGES], empty[STAGES], tmem_full[2], tmem_empty[2] (and raw[STAGES])
+        constexpr int NB = 2 * STAGES + 4;
+        static_assert(NB <= 32, "one barrier per lane");
+        if (lane < NB)
+            mbar_init(bar_base + 8u * lane, lane < STAGES ? (B_VNNI ? 1 + 4 : 1) : lane < 2 * STAGES + 2 ? 1 : 128);
+        if (B_VNNI && lane < STAGES) mbar_init(raw_bar(lane), 1);
+        if (lane == 0) *abort_flag = 0;
         fence_mbar_init();
-        if (CLUSTER_REDUCE)
-            mbar_arrive_expect_tx(bar_base + 192u, umma_cluster_recv_bytes<BN>(static_cast<uint32_t>(p.splits)));
+        __syncwarp();
+    } else if (warp == 2 && lane == 0) {
         tma_prefetch_desc(&tmap_a);
         tma_prefetch_desc(&tmap_b);
         if (p.tma_store) tma_prefetch_desc(&tmap_c);
@@ -550,7 +705,7 @@ umma_bf16_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_consta
         tmem_alloc(smem_u32(const_cast<uint32_t*>(tmem_slot)), TMEM_COLS);
         tmem_relinquish();
     }
-    // The producer warp needs nothing but the barriers its own lane 0 has just initialised: it
+    // The producer warp needs nothing but the barriers its own lanes have just initialised: it
     // signals the CTA barrier without waiting on it and starts fetching while tensor memory is
     // still being allocated (on a short problem this start-up is a visible part of the run).
     const uint32_t nthreads = blockDim.x;
@@ -566,6 +721,8 @@ umma_bf16_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_consta
     }
 
     const int total_units = p.gemms * p.tiles_m * p.tiles_n * p.splits;
+    // a CTA with a single tile to deliver, stored by TMA: its epilogue is batched through the idle ring
+    const bool one_shot = !CLUSTER_REDUCE && p.tma_store && p.splits == 1 && total_units <= static_cast<int>(gridDim.x);
 
     auto give_up = [&](unsigned int code) {
         *abort_flag = 1;
@@ -594,7 +751,7 @@ umma_bf16_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_consta
             const int kb1 = min(p.kb_total, kb0 + p.kb_per_split);
             const int row0 = mb * UMMA_BM, col0 = nb * BN;
             // k-block kb of the reduction = k-block (kb % kb_per_item) of batch item kb / kb_per_item
-            int item = kb0 / p.kb_per_item;
+            int item = kb0 == 0 ? 0 : div_small(kb0, p.kb_per_item);
             int kbl = kb0 - item * p.kb_per_item;
             item += gemm;   // independent batch: the unit's own (A, B) pair
             int ia, ib;
@@ -713,104 +870,142 @@ umma_bf16_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_consta
             }
             if (kb1 <= kb0) umma_commit_if(tfull_bar(acc), elected);  // empty K range
         }
-    } else if (warp < 6 && CLUSTER_REDUCE) {
-        // ------------------------------------------------ epilogue, K splits reduced inside the cluster
-        // One unit per CTA (grid = units); cluster rank = K split.
-        int tile, split, gemm;
-        umma_decode_unit(p, blockIdx.x, tile, split, gemm);
-        int mb, nb;
-        umma_tile_coords(p, tile, mb, nb);
-        bool ok = blockIdx.x < total_units;
-        uint8_t* staging = gen_base + STAGES * STAGE + (warp - 2) * 8192;
-        bool have_bias;
-        const uint4 bias_reg = umma_load_bias_reg<BN>(p, nb * BN, lane, have_bias);
-        if (ok && !mbar_wait(tfull_bar(0), 0u, abort_flag)) {
-            if (lane == 0) give_up(0x400u);
-            ok = false;
-        }
-        tc_fence_after_sync();
-        if (!umma_cluster_epilogue<BN>(p, &tmap_c, tmem_base, smem_base, gen_base, bar_base + 192u, abort_flag, staging,
-                                       gen_base + BN * 512 + (warp - 2) * 512, bias_reg, have_bias, warp & 3, lane, static_cast<uint32_t>(p.splits), cluster_ctarank(), 0u,
-                                       1u, mb * UMMA_BM, nb * BN, gemm, ok) && ok && lane == 0)
-            give_up(0x600u);
-    } else if (warp < 6) {
-        // ------------------------------------------------ epilogue
+    } else {
+        // ------------------------------------------------ warps 2..9
+        // Warps 2-5 are the epilogue.  Warps 6-9 first re-lay VNNI B (if that is the operand form),
+        // then join the epilogue of a CTA that delivers a single tile (one-shot, cluster split-K):
+        // tensor-memory lanes are tied to warp % 4, so each quarter of the rows has two warps,
+        // which take half of the columns each.
+        const int set = warp >= 6 ? 1 : 0;
         const int quarter = warp & 3;  // TMEM lanes 32*quarter .. +31 belong to this warp
-        int local = 0;
-        bool ok = true;
-        for (int unit = blockIdx.x; ok && unit < total_units; unit += gridDim.x, ++local) {
+        uint8_t* staging = gen_base + STAGES * STAGE + quarter * 8192;   // set 0: two store tiles; bias slices behind them
+        if (set == 1 && B_VNNI) {
+            // -------------------------------------------- VNNI re-layout
+            const int tw = warp - 6;
+            int stage = 0;
+            uint32_t phase = 0;
+            bool ok = true;
+            for (int unit = blockIdx.x; ok && unit < total_units; unit += gridDim.x) {
+                int tile, split, gemm;
+                umma_decode_unit(p, unit, tile, split, gemm);
+                const int kb0 = split * p.kb_per_split;
+                const int kb1 = min(p.kb_total, kb0 + p.kb_per_split);
+                for (int kb = kb0; kb < kb1; ++kb) {
+                    if (!mbar_wait(raw_bar(stage), phase, abort_flag)) {
+                        if (lane == 0) give_up(0x500u + stage);
+                        ok = false;
+                        break;
+                    }
+                    vnni_relayout_stage<BN>(smem_base + stage * STAGE + UMMA_A_STAGE_BYTES, tw, lane);
+                    fence_proxy_async_smem();
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(full_bar(stage));
+                    if (++stage == STAGES) { stage = 0; phase ^= 1u; }
+                }
+            }
+        }
+        if (CLUSTER_REDUCE) {
+            // -------------------------------------------- epilogue, K splits reduced inside the cluster
+            // One unit per CTA (grid = units); cluster rank = K split.
             int tile, split, gemm;
-            umma_decode_unit(p, unit, tile, split, gemm);
+            umma_decode_unit(p, blockIdx.x, tile, split, gemm);
             int mb, nb;
             umma_tile_coords(p, tile, mb, nb);
-            const int kb0 = split * p.kb_per_split;
-            const int kb1 = min(p.kb_total, kb0 + p.kb_per_split);
-            const int acc = local & 1;
-            uint8_t* staging = gen_base + STAGES * STAGE + (warp - 2) * 8192;
-            const uint16_t* bias_smem = umma_fetch_bias<BN>(p, staging, nb * BN, lane);
-            if (!mbar_wait(tfull_bar(acc), (local >> 1) & 1u, abort_flag)) {
-                if (lane == 0) give_up(0x400u + acc);
+            bool ok = blockIdx.x < total_units;
+            const float* bias_sm = p.tma_store ? umma_park_bias<BN>(p, reinterpret_cast<float*>(staging + set * 2048), nb * BN, lane)
+                                               : nullptr;
+            if (ok && !mbar_wait(tfull_bar(0), 0u, abort_flag)) {
+                if (lane == 0) give_up(0x400u);
                 ok = false;
-                break;
             }
             tc_fence_after_sync();
-            const int row0 = mb * UMMA_BM + quarter * 32;
-            const bool empty_k = kb1 <= kb0;
-            PartialDst pdst = {p.partial + (static_cast<size_t>(split) * p.gemms + gemm) * p.M * p.N, p.N, row0, 0, p.M, p.N};
-            const PartialDst* pd = p.splits > 1 ? &pdst : nullptr;
-            // two 32-column chunks per round: one wait for both tensor-memory loads
-#pragma unroll 1
-            for (int c0 = 0; c0 < BN; c0 += 64) {
-                uint32_t v0[32], v1[32];
-                const uint32_t taddr = tmem_base + acc * BN + c0 + (static_cast<uint32_t>(quarter * 32) << 16);
-                tmem_ld_32x32(taddr, v0);
-                tmem_ld_32x32(taddr + 32, v1);
-                tmem_ld_wait();
-                pdst.col0 = nb * BN + c0;
-                umma_store_chunk(p, &tmap_c, v0, row0, lane, nb * BN + c0, split, gemm, empty_k, staging, 0,
-                                 bias_smem ? bias_smem + c0 : nullptr, pd);
-                __syncwarp();
-                pdst.col0 = nb * BN + c0 + 32;
-                umma_store_chunk(p, &tmap_c, v1, row0, lane, nb * BN + c0 + 32, split, gemm, empty_k, staging, 1,
-                                 bias_smem ? bias_smem + c0 + 32 : nullptr, pd);
+            umma_cluster_epilogue<BN>(p, &tmap_c, tmem_base, smem_base, gen_base, staging, bias_sm, quarter, set, lane,
+                                      static_cast<uint32_t>(p.splits), cluster_ctarank(), 0u, 1u, mb * UMMA_BM, nb * BN, gemm, ok);
+        } else if (set == 1) {
+            // -------------------------------------------- second half of a one-shot epilogue
+            if (one_shot && static_cast<int>(blockIdx.x) < total_units) {
+                int tile, split, gemm;
+                umma_decode_unit(p, blockIdx.x, tile, split, gemm);
+                int mb, nb;
+                umma_tile_coords(p, tile, mb, nb);
+                const float* bias_sm = umma_park_bias<BN>(p, reinterpret_cast<float*>(staging + 6144), nb * BN, lane);
+                if (!mbar_wait(tfull_bar(0), 0u, abort_flag)) {
+                    if (lane == 0) give_up(0x480u);
+                } else {
+                    tc_fence_after_sync();
+                    umma_epilogue_oneshot<BN>(p, &tmap_c, tmem_base + (static_cast<uint32_t>(quarter * 32) << 16),
+                                              gen_base + (quarter * 2 + 1) * (BN * 64), mb * UMMA_BM + quarter * 32, nb * BN, gemm,
+                                              lane, p.kb_total <= 0, bias_sm, BN / 64, BN / 32);
+                }
+                if (lane == 0) bulk_wait_all();
                 __syncwarp();
             }
-            tc_fence_before_sync();
-            mbar_arrive(tempty_bar(acc));
-        }
-        // the TMA stores of this warp must have read their staging buffers (and, to be safe, be
-        // complete) before the CTA's shared memory goes away
-        if (lane == 0) bulk_wait_all();
-        __syncwarp();
-    } else if (B_VNNI) {
-        // ------------------------------------------------ VNNI re-layout warps (6..9)
-        const int tw = warp - 6;
-        int stage = 0;
-        uint32_t phase = 0;
-        bool ok = true;
-        for (int unit = blockIdx.x; ok && unit < total_units; unit += gridDim.x) {
-            int tile, split, gemm;
-            umma_decode_unit(p, unit, tile, split, gemm);
-            const int kb0 = split * p.kb_per_split;
-            const int kb1 = min(p.kb_total, kb0 + p.kb_per_split);
-            for (int kb = kb0; kb < kb1; ++kb) {
-                if (!mbar_wait(raw_bar(stage), phase, abort_flag)) {
-                    if (lane == 0) give_up(0x500u + stage);
+        } else {
+            // -------------------------------------------- epilogue
+            int local = 0;
+            bool ok = true;
+            for (int unit = blockIdx.x; ok && unit < total_units; unit += gridDim.x, ++local) {
+                int tile, split, gemm;
+                umma_decode_unit(p, unit, tile, split, gemm);
+                int mb, nb;
+                umma_tile_coords(p, tile, mb, nb);
+                const int kb0 = split * p.kb_per_split;
+                const int kb1 = min(p.kb_total, kb0 + p.kb_per_split);
+                const int acc = local & 1;
+                const float* bias_smem = one_shot ? umma_park_bias<BN>(p, reinterpret_cast<float*>(staging + 4096), nb * BN, lane)
+                                                  : umma_fetch_bias<BN>(p, staging, nb * BN, lane);
+                if (!mbar_wait(tfull_bar(acc), (local >> 1) & 1u, abort_flag)) {
+                    if (lane == 0) give_up(0x400u + acc);
                     ok = false;
                     break;
                 }
-                vnni_relayout_stage<BN>(smem_base + stage * STAGE + UMMA_A_STAGE_BYTES, tw, lane);
-                fence_proxy_async_smem();
-                __syncwarp();
-                if (lane == 0) mbar_arrive(full_bar(stage));
-                if (++stage == STAGES) { stage = 0; phase ^= 1u; }
+                tc_fence_after_sync();
+                const int row0 = mb * UMMA_BM + quarter * 32;
+                const bool empty_k = kb1 <= kb0;
+                if (one_shot) {
+                    // the only tile of this CTA: the ring is idle, batch the stores through it (first half
+                    // of the columns; warps 6-9 take the second)
+                    umma_epilogue_oneshot<BN>(p, &tmap_c, tmem_base + acc * BN + (static_cast<uint32_t>(quarter * 32) << 16),
+                                              gen_base + (quarter * 2) * (BN * 64), row0, nb * BN, gemm, lane, empty_k, bias_smem,
+                                              0, BN / 64);
+                    tc_fence_before_sync();
+                    mbar_arrive(tempty_bar(acc));
+                    continue;
+                }
+                PartialDst pdst = {p.partial + (static_cast<size_t>(split) * p.gemms + gemm) * p.M * p.N, p.N, row0, 0, p.M, p.N};
+                const PartialDst* pd = p.splits > 1 ? &pdst : nullptr;
+                // two 32-column chunks per round: one wait for both tensor-memory loads
+#pragma unroll 1
+                for (int c0 = 0; c0 < BN; c0 += 64) {
+                    uint32_t v0[32], v1[32];
+                    const uint32_t taddr = tmem_base + acc * BN + c0 + (static_cast<uint32_t>(quarter * 32) << 16);
+                    tmem_ld_32x32(taddr, v0);
+                    tmem_ld_32x32(taddr + 32, v1);
+                    tmem_ld_wait();
+                    pdst.col0 = nb * BN + c0;
+                    umma_store_chunk(p, &tmap_c, v0, row0, lane, nb * BN + c0, split, gemm, empty_k, staging, 0,
+                                     bias_smem ? bias_smem + c0 : nullptr, pd);
+                    __syncwarp();
+                    pdst.col0 = nb * BN + c0 + 32;
+                    umma_store_chunk(p, &tmap_c, v1, row0, lane, nb * BN + c0 + 32, split, gemm, empty_k, staging, 1,
+                                     bias_smem ? bias_smem + c0 + 32 : nullptr, pd);
+                    __syncwarp();
+                }
+                tc_fence_before_sync();
+                mbar_arrive(tempty_bar(acc));
             }
+            // the TMA stores of this warp must have read their staging buffers (and, to be safe, be
+            // complete) before the CTA's shared memory goes away
+            if (lane == 0) bulk_wait_all();
+            __syncwarp();
         }
     }
 
-    if (CLUSTER_REDUCE && !(warp >= 2 && warp < 6)) {
-        // the cluster barrier counts every thread: the other roles pass it here, once their part
-        // of the K loop is over (the producer has seen every stage consumed)
+    if (CLUSTER_REDUCE && warp < 2) {
+        // the cluster barriers count every thread: the other roles pass both of them here, once
+        // their part of the K loop is over (the producer has seen every stage consumed)
+        cluster_arrive();
+        cluster_wait();
         cluster_arrive();
         cluster_wait();
     }

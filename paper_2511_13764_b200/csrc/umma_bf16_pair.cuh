@@ -39,7 +39,7 @@ __host__ __device__ constexpr int pair_smem_bytes(int BN, int stages) {
 
 // UmmaParams as for the single-CTA kernel, with tiles_m counted in 256-row tiles.
 template <int BN, int STAGES, bool B_VNNI, bool CLUSTER_REDUCE = false, int KIND = 0>
-__global__ void __launch_bounds__(B_VNNI ? 320 : 192, 1)
+__global__ void __launch_bounds__(UMMA_THREADS, 1)
 umma_bf16_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ CUtensorMap tmap_b,
                       const __grid_constant__ CUtensorMap tmap_c, const UmmaParams p) {
     static_assert(BN == 128 || BN == 256, "pair tile N");
@@ -57,6 +57,7 @@ umma_bf16_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_c
     auto tfull_bar = [&](int a) { return bar_base + 8u * (2 * STAGES + a); };
     auto tempty_bar = [&](int a) { return bar_base + 8u * (2 * STAGES + 2 + a); };
     auto raw_bar = [&](int s) { return bar_base + UMMA_RAW_BAR_OFFSET + 8u * s; };   // VNNI B: this CTA's blocks of stage s have landed
+    const uint32_t peer_ready_bar = bar_base + 192u;   // leader: the peer CTA has allocated its tensor memory
     uint8_t* gen_base = smem_raw + (smem_base - smem_u32(smem_raw));
     volatile uint32_t* tmem_slot =
         reinterpret_cast<volatile uint32_t*>(gen_base + STAGES * STAGE + UMMA_EPI_STAGING + 8 * (2 * STAGES + 4));
@@ -71,34 +72,46 @@ umma_bf16_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_c
     const int pair_id = blockIdx.x >> 1;
     const int num_pairs = gridDim.x >> 1;
 
-    if (threadIdx.x == 0) {
-        for (int s = 0; s < STAGES; ++s) {
-            mbar_init(full_bar(s), B_VNNI ? 1 + 8 : 1);  // leader's producer (+ 4 re-layout warps per CTA)
-            mbar_init(empty_bar(s), 1);
-            if (B_VNNI) mbar_init(raw_bar(s), 1);
-        }
-        for (int a = 0; a < 2; ++a) {
-            mbar_init(tfull_bar(a), 1);
-            mbar_init(tempty_bar(a), 256);               // epilogue threads of both CTAs
-        }
-        *abort_flag = 0;
-        if (CLUSTER_REDUCE) mbar_init(bar_base + 192u, 1);   // counts in the pieces other CTAs send to this one
+    if (warp == 0) {
+        // one barrier per lane: full[STAGES], empty[STAGES], tmem_full[2], tmem_empty[2] (and raw[STAGES]).
+        // full[]: the leader's producer (+ 4 re-layout warps per CTA); tmem_empty[]: the epilogue threads of both CTAs
+        constexpr int NB = 2 * STAGES + 4;
+        static_assert(NB <= 32, "one barrier per lane");
+        if (lane < NB)
+            mbar_init(bar_base + 8u * lane, lane < STAGES ? (B_VNNI ? 1 + 8 : 1) : lane < 2 * STAGES + 2 ? 1 : 256);
+        if (B_VNNI && lane < STAGES) mbar_init(raw_bar(lane), 1);
+        if (lane == 31) mbar_init(peer_ready_bar, 1);
+        if (lane == 0) *abort_flag = 0;
         fence_mbar_init();
-        if (CLUSTER_REDUCE)
-            mbar_arrive_expect_tx(bar_base + 192u, umma_cluster_recv_bytes<BN>(static_cast<uint32_t>(p.splits)));
+        __syncwarp();
+    } else if (warp == 2 && lane == 0) {
         tma_prefetch_desc(&tmap_a);
         tma_prefetch_desc(&tmap_b);
         if (p.tma_store) tma_prefetch_desc(&tmap_c);
     }
+    // Start-up.  Every thread arrives on the cluster barrier at once (warp 0 after its barriers
+    // are initialised: the arrive releases them to the other CTAs) and waits on it before it first
+    // touches a barrier of the peer; the tensor-memory allocation runs meanwhile, and the producer
+    // starts fetching without waiting for it.  What the leader's MMA warp needs besides is the
+    // PEER's allocation: the peer's warp 1 reports it on the leader's `peer_ready` barrier.
+    cluster_arrive();
     if (warp == 1) {
         tmem_alloc_pair(smem_u32(const_cast<uint32_t*>(tmem_slot)), TMEM_COLS);
         tmem_relinquish_pair();
     }
-    tc_fence_before_sync();
-    __syncthreads();
-    cluster_sync_all();
-    tc_fence_after_sync();
-    const uint32_t tmem_base = *tmem_slot;
+    const uint32_t nthreads = blockDim.x;
+    uint32_t tmem_base = 0;
+    if (warp == 0) {
+        cluster_wait();
+        asm volatile("bar.arrive 0, %0;" ::"r"(nthreads) : "memory");
+    } else {
+        tc_fence_before_sync();
+        cluster_wait();
+        if (warp == 1 && rank == 1 && lane == 0) mbar_arrive_cluster_cta_release(map_to_cta(peer_ready_bar, leader));
+        asm volatile("bar.sync 0, %0;" ::"r"(nthreads) : "memory");
+        tc_fence_after_sync();
+        tmem_base = *tmem_slot;
+    }
 
     const bool tail_mode = p.tail_from >= 0;
     const int total_units = tail_mode ? p.tail_from + (p.tiles_m * p.tiles_n - p.tail_from) * p.tail_splits
@@ -125,6 +138,8 @@ umma_bf16_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_c
         kb0 = split * p.kb_per_split;
         kb1 = min(p.kb_total, kb0 + p.kb_per_split);
     };
+    // a pair with a single tile to deliver, stored by TMA: its epilogue is batched through the idle ring
+    const bool one_shot = !CLUSTER_REDUCE && p.tma_store && p.splits == 1 && !tail_mode && total_units <= num_pairs;
     auto give_up = [&](unsigned int code) {
         *abort_flag = 1;
         if (p.status) atomicCAS(p.status, 0u, code);
@@ -149,7 +164,7 @@ umma_bf16_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_c
             umma_tile_coords(p, tile, mb, nb);
             const int row0 = mb * BM2 + static_cast<int>(rank) * UMMA_BM;
             const int col0 = nb * BN + static_cast<int>(rank) * HALF;
-            int item = kb0 / p.kb_per_item;
+            int item = kb0 == 0 ? 0 : div_small(kb0, p.kb_per_item);
             int kbl = kb0 - item * p.kb_per_item;
             item += gemm;   // independent batch: the unit's own (A, B) pair
             int ia, ib;
@@ -223,6 +238,11 @@ umma_bf16_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_c
             uint32_t soff = 0;
             int local = 0;
             bool ok = true;
+            // the MMAs write the peer's half of the accumulator: its tensor memory must be allocated
+            if (!mbar_wait(peer_ready_bar, 0u, abort_flag)) {
+                if (lane == 0) give_up(0x700u);
+                ok = false;
+            }
             for (int unit = pair_id; ok && unit < total_units; unit += num_pairs, ++local) {
                 int tile, split, gemm, kb0, kb1, tail;
                 decode(unit, tile, split, gemm, kb0, kb1, tail);
@@ -259,105 +279,143 @@ umma_bf16_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_c
                 if (kb1 <= kb0) umma_commit_pair_if(tfull_bar(acc), pair_mask, elected);
             }
         }
-    } else if (warp < 6 && CLUSTER_REDUCE) {
-        // ------------------------------------------------ epilogue, K splits reduced inside the cluster
-        // One unit per pair (grid = 2 x units); this pair's split = its index in the cluster.  The
-        // other splits of this CTA's 128 rows are the CTAs with the same parity of cluster rank.
-        int tile, split, gemm;
-        umma_decode_unit(p, pair_id, tile, split, gemm);
-        int mb, nb;
-        umma_tile_coords(p, tile, mb, nb);
-        bool ok = pair_id < total_units;
-        uint8_t* staging = gen_base + STAGES * STAGE + (warp - 2) * 8192;
-        bool have_bias;
-        const uint4 bias_reg = umma_load_bias_reg<BN>(p, nb * BN, lane, have_bias);
-        if (ok && !mbar_wait(tfull_bar(0), 0u, abort_flag)) {
-            if (lane == 0) give_up(0x400u);
-            ok = false;
-        }
-        tc_fence_after_sync();
-        if (!umma_cluster_epilogue<BN>(p, &tmap_c, tmem_base, smem_base, gen_base, bar_base + 192u, abort_flag, staging,
-                                       gen_base + BN * 512 + (warp - 2) * 512, bias_reg, have_bias, warp & 3, lane, static_cast<uint32_t>(p.splits), crank >> 1, rank, 2u,
-                                       mb * BM2 + static_cast<int>(rank) * UMMA_BM, nb * BN, gemm, ok) && ok && lane == 0)
-            give_up(0x600u);
-    } else if (warp < 6) {
-        // ------------------------------------------------ epilogue (both CTAs, own 128 rows)
+    } else {
+        // ------------------------------------------------ warps 2..9 (both CTAs, own 128 rows)
+        // Warps 2-5: epilogue.  Warps 6-9: VNNI re-layout (if that is B's form), then the second half
+        // of the epilogue in a pair that delivers a single tile (see the single-CTA kernel).
+        const int set = warp >= 6 ? 1 : 0;
         const int quarter = warp & 3;
-        int local = 0;
-        bool ok = true;
-        for (int unit = pair_id; ok && unit < total_units; unit += num_pairs, ++local) {
-            int tile, split, gemm, kb0, kb1, tail;
-            decode(unit, tile, split, gemm, kb0, kb1, tail);
+        uint8_t* staging = gen_base + STAGES * STAGE + quarter * 8192;
+        if (set == 1 && B_VNNI) {
+            // -------------------------------------------- VNNI re-layout
+            // Each CTA re-lays its own HALF columns in place (see vnni_relayout_stage) and reports
+            // each finished stage to the leader's full[] barrier.
+            const int tw = warp - 6;
+            const uint32_t lead_full0 = map_to_cta(full_bar(0), leader);
+            int stage = 0;
+            uint32_t phase = 0;
+            bool ok = true;
+            for (int unit = pair_id; ok && unit < total_units; unit += num_pairs) {
+                int tile, split, gemm, kb0, kb1, tail;
+                decode(unit, tile, split, gemm, kb0, kb1, tail);
+                for (int kb = kb0; kb < kb1; ++kb) {
+                    if (!mbar_wait(raw_bar(stage), phase, abort_flag)) {
+                        if (lane == 0) give_up(0x500u + stage);
+                        ok = false;
+                        break;
+                    }
+                    vnni_relayout_stage<HALF>(smem_base + stage * STAGE + UMMA_A_STAGE_BYTES, tw, lane);
+                    fence_proxy_async_smem();
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive_cluster_cta_release(lead_full0 + 8u * stage);
+                    if (++stage == STAGES) { stage = 0; phase ^= 1u; }
+                }
+            }
+        }
+        if (CLUSTER_REDUCE) {
+            // -------------------------------------------- epilogue, K splits reduced inside the cluster
+            // One unit per pair (grid = 2 x units); this pair's split = its index in the cluster.  The
+            // other splits of this CTA's 128 rows are the CTAs with the same parity of cluster rank.
+            int tile, split, gemm;
+            umma_decode_unit(p, pair_id, tile, split, gemm);
             int mb, nb;
             umma_tile_coords(p, tile, mb, nb);
-            const int acc = local & 1;
-            uint8_t* staging = gen_base + STAGES * STAGE + (warp - 2) * 8192;
-            const uint16_t* bias_smem = umma_fetch_bias<BN>(p, staging, nb * BN, lane);
-            if (!mbar_wait(tfull_bar(acc), (local >> 1) & 1u, abort_flag)) {
-                if (lane == 0) give_up(0x400u + acc);
+            bool ok = pair_id < total_units;
+            const float* bias_sm = p.tma_store ? umma_park_bias<BN>(p, reinterpret_cast<float*>(staging + set * 2048), nb * BN, lane)
+                                               : nullptr;
+            if (ok && !mbar_wait(tfull_bar(0), 0u, abort_flag)) {
+                if (lane == 0) give_up(0x400u);
                 ok = false;
-                break;
             }
             tc_fence_after_sync();
-            const int row0 = mb * BM2 + static_cast<int>(rank) * UMMA_BM + quarter * 32;
-            const bool empty_k = kb1 <= kb0;
-            // FP32 partial of a K split: the [split][M][N] workspace, or this tail tile's own slab
-            PartialDst pdst = {p.partial + (static_cast<size_t>(split) * p.gemms + gemm) * p.M * p.N, p.N, row0, 0, p.M, p.N};
-            if (tail >= 0)
-                pdst = {p.partial + (static_cast<size_t>(tail) * p.tail_splits + split) * (BM2 * BN), BN,
-                        static_cast<int>(rank) * UMMA_BM + quarter * 32, 0, BM2, BN};
-            const PartialDst* pd = (p.splits > 1 || tail >= 0) ? &pdst : nullptr;
-            const int pcol0 = tail >= 0 ? 0 : nb * BN;
-#pragma unroll 1
-            for (int c0 = 0; c0 < BN; c0 += 64) {   // two 32-column chunks per round
-                uint32_t v0[32], v1[32];
-                const uint32_t taddr = tmem_base + acc * BN + c0 + (static_cast<uint32_t>(quarter * 32) << 16);
-                tmem_ld_32x32(taddr, v0);
-                tmem_ld_32x32(taddr + 32, v1);
-                tmem_ld_wait();
-                pdst.col0 = pcol0 + c0;
-                umma_store_chunk(p, &tmap_c, v0, row0, lane, nb * BN + c0, split, gemm, empty_k, staging, 0,
-                                 bias_smem ? bias_smem + c0 : nullptr, pd);
-                __syncwarp();
-                pdst.col0 = pcol0 + c0 + 32;
-                umma_store_chunk(p, &tmap_c, v1, row0, lane, nb * BN + c0 + 32, split, gemm, empty_k, staging, 1,
-                                 bias_smem ? bias_smem + c0 + 32 : nullptr, pd);
+            umma_cluster_epilogue<BN>(p, &tmap_c, tmem_base, smem_base, gen_base, staging, bias_sm, quarter, set, lane,
+                                      static_cast<uint32_t>(p.splits), crank >> 1, rank, 2u,
+                                      mb * BM2 + static_cast<int>(rank) * UMMA_BM, nb * BN, gemm, ok);
+        } else if (set == 1) {
+            // -------------------------------------------- second half of a one-shot epilogue
+            if (one_shot && pair_id < total_units) {
+                int tile, split, gemm, kb0, kb1, tail;
+                decode(pair_id, tile, split, gemm, kb0, kb1, tail);
+                int mb, nb;
+                umma_tile_coords(p, tile, mb, nb);
+                const float* bias_sm = umma_park_bias<BN>(p, reinterpret_cast<float*>(staging + 6144), nb * BN, lane);
+                if (!mbar_wait(tfull_bar(0), 0u, abort_flag)) {
+                    if (lane == 0) give_up(0x480u);
+                } else {
+                    tc_fence_after_sync();
+                    umma_epilogue_oneshot<BN>(p, &tmap_c, tmem_base + (static_cast<uint32_t>(quarter * 32) << 16),
+                                              gen_base + (quarter * 2 + 1) * (BN * 64),
+                                              mb * BM2 + static_cast<int>(rank) * UMMA_BM + quarter * 32, nb * BN, gemm, lane,
+                                              kb1 <= kb0, bias_sm, BN / 64, BN / 32);
+                }
+                if (lane == 0) bulk_wait_all();
                 __syncwarp();
             }
-            tc_fence_before_sync();
-            mbar_arrive_cluster_cta_release(map_to_cta(tempty_bar(acc), leader));
-        }
-        if (lane == 0) bulk_wait_all();   // this warp's TMA stores are done with the staging buffers
-        __syncwarp();
-    } else if (B_VNNI) {
-        // ------------------------------------------------ VNNI re-layout warps (both CTAs)
-        // Each CTA re-lays its own HALF columns in place (see vnni_relayout_stage) and reports
-        // each finished stage to the leader's full[] barrier.
-        const int tw = warp - 6;
-        const uint32_t lead_full0 = map_to_cta(full_bar(0), leader);
-        int stage = 0;
-        uint32_t phase = 0;
-        bool ok = true;
-        for (int unit = pair_id; ok && unit < total_units; unit += num_pairs) {
-            int tile, split, gemm, kb0, kb1, tail;
-            decode(unit, tile, split, gemm, kb0, kb1, tail);
-            for (int kb = kb0; kb < kb1; ++kb) {
-                if (!mbar_wait(raw_bar(stage), phase, abort_flag)) {
-                    if (lane == 0) give_up(0x500u + stage);
+        } else {
+            // -------------------------------------------- epilogue
+            int local = 0;
+            bool ok = true;
+            for (int unit = pair_id; ok && unit < total_units; unit += num_pairs, ++local) {
+                int tile, split, gemm, kb0, kb1, tail;
+                decode(unit, tile, split, gemm, kb0, kb1, tail);
+                int mb, nb;
+                umma_tile_coords(p, tile, mb, nb);
+                const int acc = local & 1;
+                const float* bias_smem = one_shot ? umma_park_bias<BN>(p, reinterpret_cast<float*>(staging + 4096), nb * BN, lane)
+                                                  : umma_fetch_bias<BN>(p, staging, nb * BN, lane);
+                if (!mbar_wait(tfull_bar(acc), (local >> 1) & 1u, abort_flag)) {
+                    if (lane == 0) give_up(0x400u + acc);
                     ok = false;
                     break;
                 }
-                vnni_relayout_stage<HALF>(smem_base + stage * STAGE + UMMA_A_STAGE_BYTES, tw, lane);
-                fence_proxy_async_smem();
-                __syncwarp();
-                if (lane == 0) mbar_arrive_cluster_cta_release(lead_full0 + 8u * stage);
-                if (++stage == STAGES) { stage = 0; phase ^= 1u; }
+                tc_fence_after_sync();
+                const int row0 = mb * BM2 + static_cast<int>(rank) * UMMA_BM + quarter * 32;
+                const bool empty_k = kb1 <= kb0;
+                if (one_shot) {
+                    // the only tile of this pair: the ring is idle, batch the stores through it (first half of
+                    // the columns; warps 6-9 take the second)
+                    umma_epilogue_oneshot<BN>(p, &tmap_c, tmem_base + acc * BN + (static_cast<uint32_t>(quarter * 32) << 16),
+                                              gen_base + (quarter * 2) * (BN * 64), row0, nb * BN, gemm, lane, empty_k, bias_smem,
+                                              0, BN / 64);
+                    tc_fence_before_sync();
+                    mbar_arrive_cluster_cta_release(map_to_cta(tempty_bar(acc), leader));
+                    continue;
+                }
+                // FP32 partial of a K split: the [split][M][N] workspace, or this tail tile's own slab
+                PartialDst pdst = {p.partial + (static_cast<size_t>(split) * p.gemms + gemm) * p.M * p.N, p.N, row0, 0, p.M, p.N};
+                if (tail >= 0)
+                    pdst = {p.partial + (static_cast<size_t>(tail) * p.tail_splits + split) * (BM2 * BN), BN,
+                            static_cast<int>(rank) * UMMA_BM + quarter * 32, 0, BM2, BN};
+                const PartialDst* pd = (p.splits > 1 || tail >= 0) ? &pdst : nullptr;
+                const int pcol0 = tail >= 0 ? 0 : nb * BN;
+#pragma unroll 1
+                for (int c0 = 0; c0 < BN; c0 += 64) {   // two 32-column chunks per round
+                    uint32_t v0[32], v1[32];
+                    const uint32_t taddr = tmem_base + acc * BN + c0 + (static_cast<uint32_t>(quarter * 32) << 16);
+                    tmem_ld_32x32(taddr, v0);
+                    tmem_ld_32x32(taddr + 32, v1);
+                    tmem_ld_wait();
+                    pdst.col0 = pcol0 + c0;
+                    umma_store_chunk(p, &tmap_c, v0, row0, lane, nb * BN + c0, split, gemm, empty_k, staging, 0,
+                                     bias_smem ? bias_smem + c0 : nullptr, pd);
+                    __syncwarp();
+                    pdst.col0 = pcol0 + c0 + 32;
+                    umma_store_chunk(p, &tmap_c, v1, row0, lane, nb * BN + c0 + 32, split, gemm, empty_k, staging, 1,
+                                     bias_smem ? bias_smem + c0 + 32 : nullptr, pd);
+                    __syncwarp();
+                }
+                tc_fence_before_sync();
+                mbar_arrive_cluster_cta_release(map_to_cta(tempty_bar(acc), leader));
             }
+            if (lane == 0) bulk_wait_all();   // this warp's TMA stores are done with the staging buffers
+            __syncwarp();
         }
     }
 
-    if (CLUSTER_REDUCE && !(warp >= 2 && warp < 6)) {
-        // the cluster barrier counts every thread: the other roles pass it here
+    if (CLUSTER_REDUCE && warp < 2) {
+        // the cluster barriers count every thread: the other roles pass both of them here
+        cluster_arrive();
+        cluster_wait();
         cluster_arrive();
         cluster_wait();
     }

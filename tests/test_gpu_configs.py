@@ -60,7 +60,12 @@ def freivalds(w, got, A, B):
         blk = _as_f64(A[m0 * w.K:(m0 + stepm) * w.K], w.in_dtype).reshape(-1, w.K)
         rhs[m0:m0 + blk.shape[0]] = blk @ bx
         bound[m0:m0 + blk.shape[0]] = np.abs(blk) @ absb      # >= any sum_k |a_ik b_kj|
-    tol = np.sqrt(w.N) * 1e-5 * bound.max() * 4
+    # Per element the kernel is within 1e-5 * Smax of the exact product (the acceptance bound; `bound` is an
+    # upper estimate of Smax).  The row sum over N elements with random signs of x grows like sqrt(N) if the
+    # errors are independent; the factor 4 is four standard deviations of that sum, so a correct kernel
+    # passes, while one wrong 128-row or 128-column tile (errors of the size of Smax itself) fails by
+    # orders of magnitude.
+    tol = 4 * np.sqrt(w.N) * 1e-5 * bound.max()
     err = np.abs(lhs - rhs).max()
     assert err <= tol, f"Freivalds check failed: {err} > {tol}"
 

@@ -97,7 +97,7 @@ def test_s8_k_splits_add_integer_partials(splits, mode):
     A = nk_inputs.fill(7, nk_inputs.TENSOR_A, M * K, dtype="s8")
     B = nk_inputs.fill(7, nk_inputs.TENSOR_B, K * N, dtype="s8")
     plan = nk.Plan(M, N, K, in_dtype=nk.S8, out_dtype=nk.S32, layout_a=nk.ROW_MAJOR, layout_b=nk.BLOCKED32,
-                   flags=MODES[mode] | nk.flag_splitk(splits))
+                   flags=MODES[mode] | nk.flag_splitk(splits) | nk.FLAG_SEPARATE_REDUCE)
     assert f"splitk{splits}" in plan.kernel_name and plan.workspace_bytes >= splits * M * N * 4 and plan.launches_per_run == 2
     ws = torch.full((plan.workspace_bytes,), 0xFF, dtype=torch.uint8, device="cuda")
     C = torch.full((M * N,), 12345, dtype=torch.int32, device="cuda")
@@ -105,6 +105,40 @@ def test_s8_k_splits_add_integer_partials(splits, mode):
              stream=torch.cuda.current_stream().cuda_stream)
     plan.check()
     assert np.array_equal(C.cpu().numpy().astype(np.int64).reshape(M, N), oracle.gemm_s8(M, N, K, A, B, layout_b=oracle.BLOCKED32))
+
+
+@pytest.mark.parametrize("mode,tile", [("single", 2), ("single", 3), ("single", 4), ("pair", 3), ("pair", 4)])
+@pytest.mark.parametrize("splits", [2, 4])
+@pytest.mark.parametrize("dequant", [False, True])
+def test_s8_k_splits_meet_inside_a_cluster(splits, mode, tile, dequant):
+    """K splits as the CTAs (or pairs) of one cluster: the INT32 pieces cross shared memory and are added as
+    integers: one launch, no workspace, the exact result; with the dequantising epilogue the FP32 result has
+    the bits of the two-kernel path (same integer sum, same FP32 operations after it)."""
+    M, N, K = 250, 544, 2080
+    A = nk_inputs.fill(17, nk_inputs.TENSOR_A, M * K, dtype="s8")
+    B = nk_inputs.fill(17, nk_inputs.TENSOR_B, K * N, dtype="s8")
+    bias = nk_inputs.fill(17, nk_inputs.TENSOR_BIAS, N, "normal", 50.0, "f32") if dequant else None
+    scale = 1e-4
+    sp = torch.cuda.current_stream().cuda_stream
+    outs = []
+    for extra in (0, nk.FLAG_SEPARATE_REDUCE):
+        plan = nk.Plan(M, N, K, in_dtype=nk.S8, out_dtype=nk.F32 if dequant else nk.S32, layout_a=nk.ROW_MAJOR,
+                       layout_b=nk.BLOCKED32, epilogue=nk.EPI_BIAS_RELU if dequant else nk.EPI_NONE, scale=scale,
+                       flags=MODES[mode] | nk.flag_tile_n(tile) | nk.flag_splitk(splits) | extra)
+        assert ("_cluster" in plan.kernel_name) == (extra == 0), plan.kernel_name
+        assert (plan.workspace_bytes == 0) == (extra == 0) and plan.launches_per_run == (1 if extra == 0 else 2)
+        ws = torch.full((max(plan.workspace_bytes, 16),), 0xFF, dtype=torch.uint8, device="cuda")
+        C = torch.full((M * N,), 12345, dtype=torch.float32 if dequant else torch.int32, device="cuda")
+        plan.run(torch.from_numpy(A).cuda(), torch.from_numpy(B).cuda(), C, bias=torch.from_numpy(bias).cuda() if dequant else None,
+                 workspace=ws if plan.workspace_bytes else None, workspace_bytes=plan.workspace_bytes, stream=sp)
+        plan.check()
+        outs.append(C.cpu().numpy().reshape(M, N))
+    assert np.array_equal(outs[0], outs[1])
+    if dequant:
+        want, S = oracle.gemm_s8_scaled(M, N, K, A, B, scale, bias=bias, layout_b=oracle.BLOCKED32, relu=True)
+        assert np.all(np.abs(outs[0].astype(np.float64) - want) <= DEQ_TOL * S)
+    else:
+        assert np.array_equal(outs[0].astype(np.int64), oracle.gemm_s8(M, N, K, A, B, layout_b=oracle.BLOCKED32))
 
 
 @pytest.mark.parametrize("dequant", [False, True])

@@ -143,10 +143,26 @@ def test_umma_bf16_splitk(splits, out_dtype, epi, mode):
     run_and_check(W("umma", 130, 200, 1096, "bf16", out_dtype, epilogue=epi, seed=9), flags=f)
 
 
-@pytest.mark.parametrize("mode,tile", [("single", 2), ("single", 3), ("single", 4), ("pair", 3), ("pair", 4)])
+def _cluster_cases():
+    """(shape, splits, mode, tile) combinations whose plan forms a cluster: the K splits that survive (no empty
+    split) number 2, 4 or 8 (8: single CTAs only), and all the CTAs of the plan are resident at once."""
+    out = []
+    shapes = [((130, 200, 1096), 2), ((520, 776, 2048), 4), ((256, 1024, 1024), 4), ((16, 1024, 1024), 8),
+              ((100, 72, 128), 2), ((300, 520, 512), 2)]
+    for (M, N, K), splits in shapes:
+        for mode, tile in [("single", 2), ("single", 3), ("single", 4), ("pair", 3), ("pair", 4)]:
+            kb = -(-K // 64)
+            nsplit = -(-kb // -(-kb // splits))
+            bn = 32 << (tile - 1)
+            ctas = nsplit * -(-M // (256 if mode == "pair" else 128)) * -(-N // bn) * (2 if mode == "pair" else 1)
+            if nsplit in (2, 4) or (nsplit == 8 and mode == "single"):
+                if ctas <= 100:
+                    out.append(pytest.param((M, N, K), splits, mode, tile, id=f"{M}x{N}x{K}-s{splits}-{mode}-bn{bn}"))
+    return out
+
+
 @pytest.mark.parametrize("out_dtype,epi", [("f32", "none"), ("bf16", "bias_relu")])
-@pytest.mark.parametrize("shape,splits", [((130, 200, 1096), 2), ((520, 776, 2048), 4), ((256, 4096, 1024), 4),
-                                          ((16, 1024, 1024), 8), ((100, 72, 64), 2), ((300, 520, 512), 2)])
+@pytest.mark.parametrize("shape,splits,mode,tile", _cluster_cases())
 def test_umma_splitk_cluster_reduce_equals_reduce_kernel(shape, splits, out_dtype, epi, mode, tile):
     """K splits as the CTAs (or CTA pairs) of one cluster: the partial sums meet in shared memory and
     are added in split order, exactly as the separate reduce kernel adds them: same bits, one
@@ -156,12 +172,7 @@ def test_umma_splitk_cluster_reduce_equals_reduce_kernel(shape, splits, out_dtyp
     A, B, bias = w.make()
     f = MODES[mode] | nk.flag_splitk(splits) | nk.flag_tile_n(tile)
     c_one, p_one = run_plan(w, A, B, bias, flags=f)
-    if "_cluster" not in p_one.kernel_name:
-        # not a cluster size (the plan drops empty splits), or the clusters are not all resident at once
-        nsplit = int(p_one.kernel_name.split("splitk")[1].split("_")[0])
-        ctas = nsplit * -(-M // 128) * -(-N // (32 << (tile - 1)))
-        assert nsplit not in (2, 4, 8) or ctas > 100 or (mode == "pair" and nsplit == 8), p_one.kernel_name
-        pytest.skip("no cluster for this plan")
+    assert "_cluster" in p_one.kernel_name, p_one.kernel_name
     c_two, p_two = run_plan(w, A, B, bias, flags=f | nk.FLAG_SEPARATE_REDUCE)
     assert p_two.launches_per_run == 2 and p_one.launches_per_run == 1
     assert "_cluster" not in p_two.kernel_name and ("pair" in p_one.kernel_name) == (mode == "pair")

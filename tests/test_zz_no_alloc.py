@@ -5,10 +5,11 @@ on the allocator, a plug-in that is handed buffers and owns no allocator) still
 needs split-K plans to work.  The entry point takes the split-K scratch from a
 16 MiB array built into the library.  This test runs it through the C ABI twice
 in a row, on different inputs, and compares each result with what nk_gemm_run
-produces for the same plan with caller-provided scratch; the two share the
-kernels and the summation order, so the results must agree bit for bit (which
-is inside the tolerance the other tests use).  It is collected last so that a
-failure here cannot hide one elsewhere.
+produces for the same plan with caller-provided scratch (the two share the
+kernels and the summation order, so the results must agree bit for bit, which
+is inside the tolerance the other tests use) and with the CPU oracle under the
+acceptance bound of the parity tests.  It is collected last so that a failure
+here cannot hide one elsewhere.
 """
 import numpy as np
 import pytest
@@ -16,7 +17,7 @@ import torch
 
 import nk_inputs
 import paper_2511_13764_b200 as nk
-from nk_testlib import to_device, c_to_f64, TOL_REL_SMAX
+from nk_testlib import to_device, c_to_f64, check_against_oracle, TOL_REL_SMAX
 
 pytestmark = pytest.mark.gpu
 
@@ -40,6 +41,8 @@ def _run_both(plan, w, seed):
     # nothing was allocated on the device: neither through torch's allocator nor behind its back
     assert torch.cuda.memory_stats().get("allocation.all.allocated", 0) == allocs_before
     assert torch.cuda.mem_get_info()[0] >= free_before
+    # the static-scratch result against the oracle, element by element, under the acceptance bound
+    check_against_oracle(w, c_to_f64(got).reshape(w.M, w.N), A, B, bias)
     return c_to_f64(got), c_to_f64(ref)
 
 
