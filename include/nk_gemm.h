@@ -117,7 +117,12 @@ typedef enum { NK_EPI_NONE = 0, NK_EPI_BIAS_RELU = 1 } nk_epilogue_t;
                                        path is FMA arithmetic (Algorithm 1); this flag is an opt-in departure
                                        for compute-bound shapes.  Needs N and K multiples of 8.  A value beyond
                                        the largest BF16 (3.39e38) counts as infinite.                        */
-#define NK_FLAG_TAIL_SPLIT_SHIFT 24 /* bits 24..27: force this many K splits (2..8) for the last wave's tiles */
+#define NK_FLAG_TAIL_SPLIT_SHIFT 24 /* bits 24..27: cut every tile of the last, partial wave into this many equal K
+                                      splits (2..8) instead of sharing its k-blocks out evenly over the pairs; 15: share
+                                      them out evenly even where the plan's cost model would not */
+#define NK_FLAG_RASTER_SHIFT 28 /* bits 28..30: M tiles that sweep N together in the tile raster of the tensor-core
+                                   kernels: 0 = 8 (default), 1 = 4, 2 = 6, 3 = 12, 4 = 16, 5 = 24, 6 = 2, 7 = 32;
+                                   bit 31: switch off the serpentine sweep (every other group sweeps N backwards) */
 #define NK_FLAG_SPLITK_SHIFT 8    /* bits 8..15: force this many K splits (0 = auto)          */
 #define NK_FLAG_TILE_N_SHIFT 16   /* bits 16..19: force tile N: 1=32 2=64 3=128 4=256 (0 = auto) */
 

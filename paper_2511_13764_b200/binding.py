@@ -39,6 +39,11 @@ def flag_tail_split(n: int) -> int:
     return (n & 0xF) << 24
 
 
+def flag_raster(group_code: int, serpentine: bool = True) -> int:
+    """Tile raster of the tensor-core kernels: group_code 0..7 = 8, 4, 6, 12, 16, 24, 2, 32 M tiles per group."""
+    return ((group_code & 7) << 28) | (0 if serpentine else (1 << 31))
+
+
 def flag_tile_n(code: int) -> int:
     """1=32, 2=64, 3=128, 4=256."""
     return (code & 0xF) << 16

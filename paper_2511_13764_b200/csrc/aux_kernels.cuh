@@ -165,18 +165,22 @@ struct TailReduceParams {
     int M, N;
     int tile_rows, tile_cols;   // 256 x BN
     int tiles_m, tiles_n, group_m, first_tile;   // raster of the GEMM kernel; first_tile = id of tail tile 0
-    int splits;
+    int serpentine;             // raster: odd groups of M tiles sweep N backwards
+    int kb_total, sk_share;     // k-blocks of a tile; k-blocks of the tail each pair took (segment boundaries)
+    int max_segs;               // slabs reserved per tail tile
     int epilogue, bias_bf16, out_bf16, beta, c_blocked, f16;
-    const float* partial;       // [tail tile][split][tile_rows][tile_cols]
+    const float* partial;       // [tail tile][segment][tile_rows][tile_cols]
     const void* bias;
     void* C;
     int int_partials, dequant;  // as in ReduceParams
     float scale;
 };
 
-// Sums the K splits of the tail tiles (the last, partial wave of a large GEMM, see the pair
-// kernel) in split order and applies the epilogue: blockIdx.y = tail tile, four consecutive
-// columns per thread.
+// Sums the segments of the tail tiles (the last, partial wave of a large GEMM, shared out by
+// k-blocks over all the CTA pairs: see the pair kernel) in segment order, which is k order, and
+// applies the epilogue: blockIdx.y = tail tile, four consecutive columns per thread.  Pair i took
+// the k-blocks [i * sk_share, (i + 1) * sk_share) of the tail tiles laid end to end, so tile t was
+// cut by the pairs t * kb_total / sk_share .. ((t + 1) * kb_total - 1) / sk_share.
 __global__ void tail_reduce_kernel(const TailReduceParams p) {
     const int q = blockIdx.x * blockDim.x + threadIdx.x;
     const int per_row = p.tile_cols / 4;
@@ -189,12 +193,16 @@ __global__ void tail_reduce_kernel(const TailReduceParams p) {
     const int within = tile - g * per_group;
     const int first_m = g * p.group_m;
     const int gm = min(p.group_m, p.tiles_m - first_m);
-    const int mb = first_m + within % gm, nb = within / gm;
+    const int mb = first_m + within % gm;
+    int nb = within / gm;
+    if (p.serpentine && (g & 1)) nb = p.tiles_n - 1 - nb;
     const int i = mb * p.tile_rows + r, j = nb * p.tile_cols + c;
     if (i >= p.M || j >= p.N) return;
+    const int t = blockIdx.y;
+    const int segs = ((t + 1) * p.kb_total - 1) / p.sk_share - (t * p.kb_total) / p.sk_share + 1;
     const size_t slab = static_cast<size_t>(p.tile_rows) * p.tile_cols;
-    const float* src = p.partial + static_cast<size_t>(blockIdx.y) * p.splits * slab + static_cast<size_t>(r) * p.tile_cols + c;
-    float4 s = sum_partials(src, slab, p.splits, p.int_partials, p.dequant, p.scale);
+    const float* src = p.partial + static_cast<size_t>(t) * p.max_segs * slab + static_cast<size_t>(r) * p.tile_cols + c;
+    float4 s = sum_partials(src, slab, segs, p.int_partials, p.dequant, p.scale);
     const size_t ce = p.c_blocked ? ((static_cast<size_t>(i / 32) * (p.N / 32) + j / 32) * 32 + i % 32) * 32 + j % 32
                                   : static_cast<size_t>(i) * p.N + j;
     if (p.beta) {

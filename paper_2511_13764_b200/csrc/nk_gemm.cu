@@ -39,6 +39,7 @@ struct nk_gemm_s {
     int sm_count;
     // UMMA
     int bn, stages, splits, group_m;
+    bool serpentine;       // raster: odd groups of M tiles sweep N backwards
     bool pair;             // CTA pairs: 256-row tiles, cta_group::2
     int max_pairs;         // co-resident clusters of 2 for the chosen pair kernel
     bool b_vnni_inkernel;  // blocked B re-laid inside the GEMM kernel
@@ -46,7 +47,8 @@ struct nk_gemm_s {
     bool b_3d;             // B tensor map is the 3-D slab view
     bool b_kmajor;         // B is stored transposed, Bt[N][K]: K-major tiles by TMA, like A
     bool cluster_reduce;   // K splits of a tile = the CTAs of one cluster; partial sums meet in shared memory
-    int tail_from, tail_splits;   // pair kernel: tiles >= tail_from (the last, partial wave) are cut into K splits; -1: off
+    int tail_from, tail_splits;   // pair kernel: tiles >= tail_from (the last, partial wave) are shared out by k-blocks; -1: off.  tail_splits: the forced cut, else 0
+    int sk_share, sk_max_segs;    // k-blocks of the tail per pair; partial slabs reserved per tail tile
     // SIMT
     int simt_tile;  // 128, 64 or 32
     int kt_per_split;
@@ -270,6 +272,13 @@ static void choose_umma(nk_gemm_s* p) {
     p->stages = best.pair ? (best.bn == 256 ? 6 : 8) : umma_stages_for(best.bn);
     p->splits = splits;
     p->group_m = 8;
+    p->serpentine = false;
+    {
+        // tuning override of the raster: bits 28-30 pick the group size, bit 31 switches the serpentine sweep off
+        static const int kGroups[8] = {8, 4, 6, 12, 16, 24, 2, 32};
+        p->group_m = kGroups[(d.flags >> NK_FLAG_RASTER_SHIFT) & 7u];
+        p->serpentine = ((d.flags >> (NK_FLAG_RASTER_SHIFT + 3)) & 1u) == 0;
+    }
     p->cluster_reduce = splits > 1 && cluster_reduce_fits(d, sms, best.pair, best.bn, splits);
 }
 
@@ -922,28 +931,37 @@ nk_status_t nk_gemm_create(const nk_gemm_desc_t* desc, nk_gemm_t* out) {
                 p->cluster_reduce = false;
             }
         }
-        // Tail wave: when the tiles do not fill the last wave of pairs, cutting those tiles along K lets
-        // them use all the pairs for 1/s of a wave; worth it when the K loop saved outweighs the small
-        // reduce kernel and the partials (FP32, written and read once).
+        // Ragged last wave (stream-K): when the tiles left after the last full wave do not fill the
+        // pairs, their k-blocks are shared out evenly over all the pairs, so that the wave takes a
+        // fraction of a K loop; worth it when the K loop saved outweighs the small reduce kernel and
+        // the partials (FP32, written and read once).  NK_FLAG_TAIL_SPLIT forces equal cuts instead.
         p->tail_from = -1;
         p->tail_splits = 0;
+        p->sk_share = p->sk_max_segs = 0;
         if (p->pair && p->splits == 1 && p->gemms == 1 && !(d.flags & NK_FLAG_NO_TAIL_SPLIT)) {
             const int tiles = ceil_div(d.M, 2 * UMMA_BM) * ceil_div(d.N, p->bn);
             const int kb_total = p->batch * ceil_div(d.K, kblock(d));
-            const int tail = tiles % p->max_pairs;
-            if (tiles > p->max_pairs && tail > 0 && (2 * tail <= p->max_pairs || ((d.flags >> NK_FLAG_TAIL_SPLIT_SHIFT) & 0xF) >= 2)) {
-                int sp = p->max_pairs / tail;
-                if (sp > 4) sp = 4;
-                while (sp > 1 && kb_total / sp < 8) --sp;
+            const int P = p->max_pairs;
+            const int tail = tiles % P;
+            int forced_tail = (d.flags >> NK_FLAG_TAIL_SPLIT_SHIFT) & 0xF;
+            bool forced_even = forced_tail == 15;            // the even share, whatever the cost model says
+            if (forced_tail >= 2 && forced_tail <= 8 && tail * forced_tail > P) forced_even = true;   // equal cuts would need more pairs than there are
+            if (forced_tail < 2 || forced_tail > 8 || forced_tail > kb_total || tail * forced_tail > P) forced_tail = 0;
+            if (tiles > P && tail > 0 && kb_total >= 2) {
+                int share = forced_tail ? ceil_div(kb_total, forced_tail) : ceil_div(static_cast<int64_t>(tail) * kb_total, P);
+                if (!forced_tail && !forced_even && share < 4) share = kb_total < 4 ? kb_total : 4;   // shorter ranges are all overhead
+                const int segments = tail + ceil_div(static_cast<int64_t>(tail) * kb_total, share);   // at most: every pair, every tile boundary
                 const double t_kb = p->bn == 256 ? 0.385 : 0.35;
-                const double slab_bytes = static_cast<double>(tail) * sp * 2 * UMMA_BM * p->bn * 4;
-                const double saved_us = kb_total * t_kb * (1.0 - 1.0 / sp);
-                const double cost_us = 5.5 + 2.0 * slab_bytes / 7.0e6;   // measured: ~10 us for 18 MB of partials (they stay in L2)
-                const int forced_tail = (d.flags >> NK_FLAG_TAIL_SPLIT_SHIFT) & 0xF;
-                if (forced_tail >= 2 && forced_tail <= 8 && forced_tail <= kb_total) sp = forced_tail;
-                if (sp > 1 && (saved_us > cost_us || forced_tail >= 2)) {
+                const double slab_bytes = static_cast<double>(segments) * 2 * UMMA_BM * p->bn * 4;
+                const double saved_us = (kb_total - share) * t_kb;
+                // measured: ~10 us for 18 MB of partials (they stay in L2); a pair whose range straddles two tiles
+                // drains two accumulators
+                const double cost_us = 5.5 + 2.0 * slab_bytes / 7.0e6 + p->bn / 32 * 0.5;
+                if (share < kb_total && (saved_us > cost_us || forced_tail || forced_even)) {
                     p->tail_from = tiles - tail;
-                    p->tail_splits = sp;
+                    p->tail_splits = forced_tail;
+                    p->sk_share = share;
+                    p->sk_max_segs = (kb_total + share - 2) / share + 1;
                 }
             }
         }
@@ -953,7 +971,7 @@ nk_status_t nk_gemm_create(const nk_gemm_desc_t* desc, nk_gemm_t* out) {
         p->ws_partial_bytes = (p->splits > 1 && !p->cluster_reduce) ? static_cast<size_t>(p->splits) * p->gemms * d.M * d.N * 4 : 0;
         if (p->tail_from >= 0) {
             const int tiles = ceil_div(d.M, 2 * UMMA_BM) * ceil_div(d.N, p->bn);
-            p->ws_partial_bytes = static_cast<size_t>(tiles - p->tail_from) * p->tail_splits * 2 * UMMA_BM * p->bn * 4;
+            p->ws_partial_bytes = static_cast<size_t>(tiles - p->tail_from) * p->sk_max_segs * 2 * UMMA_BM * p->bn * 4;
         }
         p->launches = 1 + ((p->splits > 1 && !p->cluster_reduce) || p->tail_from >= 0 ? 1 : 0) + (p->b_repack ? 1 : 0);
         snprintf(p->name, sizeof(p->name), "umma_bf16_%s%dx%d_s%d_splitk%d%s%s%s",
@@ -972,7 +990,8 @@ nk_status_t nk_gemm_create(const nk_gemm_desc_t* desc, nk_gemm_t* out) {
     }
     if (p->variant == V_UMMA && p->tail_from >= 0) {
         const size_t len = strlen(p->name);
-        snprintf(p->name + len, sizeof(p->name) - len, "_tail%d", p->tail_splits);
+        if (p->tail_splits) snprintf(p->name + len, sizeof(p->name) - len, "_tail%d", p->tail_splits);
+        else snprintf(p->name + len, sizeof(p->name) - len, "_streamk%d", p->sk_share);
     }
     if (d.in_dtype == NK_F16) {
         const size_t len = strlen(p->name);
@@ -1104,6 +1123,7 @@ nk_status_t nk_gemm_run(nk_gemm_t p, const void* A, const void* B, const void* b
         up.cluster_reduce = p->cluster_reduce ? 1 : 0;
         up.kb_per_split = ceil_div(up.kb_total, p->splits);
         up.group_m = p->group_m;
+        up.serpentine = p->serpentine ? 1 : 0;
         up.a_blocked = d.layout_a == NK_BLOCKED32;
         up.b_3d = p->b_3d ? 1 : 0;
         up.b_kmajor = p->b_kmajor ? 1 : 0;
@@ -1124,9 +1144,10 @@ nk_status_t nk_gemm_run(nk_gemm_t p, const void* A, const void* B, const void* b
         up.item_map_a = p->item_map_a;
         up.item_map_b = p->item_map_b;
         up.tail_from = p->tail_from;
-        up.tail_splits = p->tail_splits;
-        const int units = p->tail_from >= 0 ? p->tail_from + (up.tiles_m * up.tiles_n - p->tail_from) * p->tail_splits
-                                            : up.gemms * up.tiles_m * up.tiles_n * up.splits;
+        up.sk_share = p->sk_share;
+        up.sk_max_segs = p->sk_max_segs;
+        // (tail mode: more tiles than pairs, so every pair is launched; each adds up to two tail segments to its whole tiles)
+        const int units = p->tail_from >= 0 ? p->tail_from + 2 * p->max_pairs : up.gemms * up.tiles_m * up.tiles_n * up.splits;
         if (p->cluster_reduce) {
             e = launch_cluster(p, up, units, p->splits, st, nullptr);
         } else if (p->pair) {
@@ -1142,7 +1163,8 @@ nk_status_t nk_gemm_run(nk_gemm_t p, const void* A, const void* B, const void* b
     if (p->variant == V_UMMA && p->tail_from >= 0) {
         const int tiles_m = ceil_div(d.M, 2 * UMMA_BM), tiles_n = ceil_div(d.N, p->bn);
         TailReduceParams tp = {static_cast<int>(d.M), static_cast<int>(d.N), 2 * UMMA_BM, p->bn, tiles_m, tiles_n, p->group_m,
-                               p->tail_from, p->tail_splits, d.epilogue, (p->bias_f32 || is_8bit(d)) ? 0 : 1, is16(d.out_dtype), d.beta,
+                               p->tail_from, p->serpentine ? 1 : 0, p->batch * ceil_div(d.K, kblock(d)), p->sk_share, p->sk_max_segs,
+                               d.epilogue, (p->bias_f32 || is_8bit(d)) ? 0 : 1, is16(d.out_dtype), d.beta,
                                d.layout_c == NK_BLOCKED32, d.in_dtype == NK_F16, partial, bias, C,
                                is_s8(d) ? 1 : 0, (is_s8(d) && d.out_dtype == NK_F32) ? 1 : 0, d.scale};
         const int quads = 2 * UMMA_BM * p->bn / 4;

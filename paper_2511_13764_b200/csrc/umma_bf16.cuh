@@ -57,6 +57,7 @@ struct UmmaParams {
     int cluster_reduce; // the K splits of a tile are the CTAs of one cluster and meet in shared memory
     int kb_per_split;   // ceil(kb_total / splits)
     int group_m;        // raster: this many M tiles sweep N together
+    int serpentine;     // raster: every other group of M tiles sweeps N in the opposite direction
     int a_blocked;      // A tensor map is the 4-D blocked view
     int b_3d;           // B tensor map is the 3-D (n-in-slab, k, slab) view: one box per stage
     int b_kmajor;       // B is stored transposed, Bt[N][K]: its tiles are K-major like A's, one box per stage
@@ -66,9 +67,10 @@ struct UmmaParams {
     uint32_t idesc;     // tcgen05 instruction descriptor
     const void* bias;   // BF16 [N] or null
     void* C;            // [M][N] FP32 or BF16
-    float* partial;     // [splits][M][N] when splits > 1; [tail tile][tail split][tile rows][BN] in tail mode
-    int tail_from;      // tail mode (pair kernel): units >= tail_from are K splits of the last, partial wave's tiles; else -1
-    int tail_splits;    // K splits of each tail tile
+    float* partial;     // [splits][M][N] when splits > 1; [tail tile][segment][tile rows][BN] in tail mode
+    int tail_from;      // stream-K tail (pair kernel): tiles >= tail_from, the last, partial wave, are shared out by k-blocks; else -1
+    int sk_share;       // k-blocks of the tail each pair takes: pair i has [i * sk_share, (i + 1) * sk_share) of the tail tiles' k-blocks laid end to end
+    int sk_max_segs;    // partial slabs reserved per tail tile (a tile is cut into at most this many segments)
     int bias_f32;       // the bias vector is FP32 although the operands are not (split-FP32 and quantised plans)
     int dequant;        // the accumulator holds INT32 sums: convert to FP32 and multiply by `scale` before the epilogue
     float scale;
@@ -122,6 +124,8 @@ __device__ __forceinline__ void umma_tile_coords(const UmmaParams& p, int tile, 
     const int gm = min(p.group_m, p.tiles_m - first_m);
     nb = div_small(within, gm);
     mb = first_m + within - nb * gm;
+    // odd groups sweep N backwards: the B columns a group ends on are the ones the next group starts with
+    if (p.serpentine && (g & 1)) nb = p.tiles_n - 1 - nb;
 }
 
 // unit id -> (independent GEMM, tile, K split)

@@ -18,10 +18,13 @@
 //   - cluster-wide barriers fence the start (barriers initialised) and the end (nobody
 //     leaves while its peer may still touch its shared memory or barriers).
 //
-// Tail mode (p.tail_from >= 0): the tiles of the last, partial wave are each cut into
-// p.tail_splits K splits so that they occupy all the pairs for a fraction of a wave instead
-// of a fraction of the pairs for a whole one; their FP32 partials go to the workspace and a
-// small kernel sums them (tail_reduce_kernel).  Units 0 .. tail_from-1 are whole tiles.
+// Tail mode (p.tail_from >= 0), the stream-K treatment of a ragged last wave: the tiles that are
+// left after the last full wave would occupy a fraction of the pairs for a whole K loop.  Their
+// k-blocks, laid end to end, are instead shared out evenly over ALL the pairs (p.sk_share each),
+// so the wave takes a fraction of a K loop.  A pair's range covers part of one tile or the end
+// of one and the start of the next; for each part it writes an FP32 (INT32 for INT8) partial
+// slab, and a small kernel (tail_reduce_kernel) adds the slabs of a tile in segment order, which
+// is k order: deterministic, no atomics.  Units 0 .. tail_from-1 are whole tiles.
 //
 // With CLUSTER_REDUCE the cluster holds S pairs, one per K split of the same 256-row tile
 // (ranks 2s and 2s + 1 are the pair of split s; a pair's leader is its even rank); the
@@ -114,29 +117,45 @@ umma_bf16_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_c
     }
 
     const bool tail_mode = p.tail_from >= 0;
-    const int total_units = tail_mode ? p.tail_from + (p.tiles_m * p.tiles_n - p.tail_from) * p.tail_splits
-                                      : p.gemms * p.tiles_m * p.tiles_n * p.splits;
-    // unit -> tile, K split, GEMM of the batch, k-block range; tail >= 0: index of the tail tile
-    auto decode = [&](int unit, int& tile, int& split, int& gemm, int& kb0, int& kb1, int& tail) {
+    // tail mode: every pair has its whole tiles (units below tail_from, a multiple of the number of
+    // pairs) and then up to two segments of the tail (its k-block range may straddle two tiles)
+    const int total_units = tail_mode ? p.tail_from + 2 * num_pairs : p.gemms * p.tiles_m * p.tiles_n * p.splits;
+    // unit -> tile, K split (segment number inside a tail tile), GEMM of the batch, k-block range;
+    // tail >= 0: index of the tail tile.  False: nothing to do (an empty segment; only a pair's last
+    // units can be empty, so the accumulator and barrier phases of the roles stay in step).
+    auto decode = [&](int unit, int& tile, int& split, int& gemm, int& kb0, int& kb1, int& tail) -> bool {
         tail = -1;
         if (tail_mode) {
             gemm = 0;
             if (unit < p.tail_from) {
                 tile = unit; split = 0; kb0 = 0; kb1 = p.kb_total;
-            } else {
-                const int u = unit - p.tail_from;
-                tail = u / p.tail_splits;
-                split = u - tail * p.tail_splits;
-                tile = p.tail_from + tail;
-                const int per = (p.kb_total + p.tail_splits - 1) / p.tail_splits;
-                kb0 = split * per;
-                kb1 = min(p.kb_total, kb0 + per);
+                return true;
             }
-            return;
+            const int u = unit - p.tail_from;
+            const int second = u >= num_pairs ? 1 : 0;
+            const int j = u - second * num_pairs;                       // this pair
+            const int total = (p.tiles_m * p.tiles_n - p.tail_from) * p.kb_total;
+            const int start = j * p.sk_share, end = min(start + p.sk_share, total);
+            if (start >= end) return false;
+            const int first_tile = div_small(start, p.kb_total);
+            if (!second) {
+                tail = first_tile;
+                kb0 = start - first_tile * p.kb_total;
+                kb1 = min(p.kb_total, end - first_tile * p.kb_total);
+            } else {
+                tail = first_tile + 1;
+                kb0 = 0;
+                kb1 = end - tail * p.kb_total;
+                if (kb1 <= 0) return false;
+            }
+            tile = p.tail_from + tail;
+            split = j - div_small(tail * p.kb_total, p.sk_share);       // segments of a tile are numbered by pair
+            return true;
         }
         umma_decode_unit(p, unit, tile, split, gemm);
         kb0 = split * p.kb_per_split;
         kb1 = min(p.kb_total, kb0 + p.kb_per_split);
+        return true;
     };
     // a pair with a single tile to deliver, stored by TMA: its epilogue is batched through the idle ring
     const bool one_shot = !CLUSTER_REDUCE && p.tma_store && p.splits == 1 && !tail_mode && total_units <= num_pairs;
@@ -159,7 +178,7 @@ umma_bf16_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_c
         bool ok = true;
         for (int unit = pair_id; ok && unit < total_units; unit += num_pairs) {
             int tile, split, gemm, kb0, kb1, tail;
-            decode(unit, tile, split, gemm, kb0, kb1, tail);
+            if (!decode(unit, tile, split, gemm, kb0, kb1, tail)) continue;
             int mb, nb;
             umma_tile_coords(p, tile, mb, nb);
             const int row0 = mb * BM2 + static_cast<int>(rank) * UMMA_BM;
@@ -245,7 +264,7 @@ umma_bf16_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_c
             }
             for (int unit = pair_id; ok && unit < total_units; unit += num_pairs, ++local) {
                 int tile, split, gemm, kb0, kb1, tail;
-                decode(unit, tile, split, gemm, kb0, kb1, tail);
+                if (!decode(unit, tile, split, gemm, kb0, kb1, tail)) continue;
                 const int acc = local & 1;
                 if (!mbar_wait(tempty_bar(acc), ((local >> 1) & 1u) ^ 1u, abort_flag)) {
                     if (lane == 0) give_up(0x200u + acc);
@@ -297,7 +316,7 @@ umma_bf16_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_c
             bool ok = true;
             for (int unit = pair_id; ok && unit < total_units; unit += num_pairs) {
                 int tile, split, gemm, kb0, kb1, tail;
-                decode(unit, tile, split, gemm, kb0, kb1, tail);
+                if (!decode(unit, tile, split, gemm, kb0, kb1, tail)) continue;
                 for (int kb = kb0; kb < kb1; ++kb) {
                     if (!mbar_wait(raw_bar(stage), phase, abort_flag)) {
                         if (lane == 0) give_up(0x500u + stage);
@@ -335,7 +354,7 @@ umma_bf16_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_c
             // -------------------------------------------- second half of a one-shot epilogue
             if (one_shot && pair_id < total_units) {
                 int tile, split, gemm, kb0, kb1, tail;
-                decode(pair_id, tile, split, gemm, kb0, kb1, tail);
+                if (!decode(pair_id, tile, split, gemm, kb0, kb1, tail)) tile = 0;
                 int mb, nb;
                 umma_tile_coords(p, tile, mb, nb);
                 const float* bias_sm = umma_park_bias<BN>(p, reinterpret_cast<float*>(staging + 6144), nb * BN, lane);
@@ -357,7 +376,7 @@ umma_bf16_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_c
             bool ok = true;
             for (int unit = pair_id; ok && unit < total_units; unit += num_pairs, ++local) {
                 int tile, split, gemm, kb0, kb1, tail;
-                decode(unit, tile, split, gemm, kb0, kb1, tail);
+                if (!decode(unit, tile, split, gemm, kb0, kb1, tail)) continue;
                 int mb, nb;
                 umma_tile_coords(p, tile, mb, nb);
                 const int acc = local & 1;
@@ -384,7 +403,7 @@ umma_bf16_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_c
                 // FP32 partial of a K split: the [split][M][N] workspace, or this tail tile's own slab
                 PartialDst pdst = {p.partial + (static_cast<size_t>(split) * p.gemms + gemm) * p.M * p.N, p.N, row0, 0, p.M, p.N};
                 if (tail >= 0)
-                    pdst = {p.partial + (static_cast<size_t>(tail) * p.tail_splits + split) * (BM2 * BN), BN,
+                    pdst = {p.partial + (static_cast<size_t>(tail) * p.sk_max_segs + split) * (BM2 * BN), BN,
                             static_cast<int>(rank) * UMMA_BM + quarter * 32, 0, BM2, BN};
                 const PartialDst* pd = (p.splits > 1 || tail >= 0) ? &pdst : nullptr;
                 const int pcol0 = tail >= 0 ? 0 : nb * BN;

@@ -141,6 +141,30 @@ def test_s8_k_splits_meet_inside_a_cluster(splits, mode, tile, dequant):
         assert np.array_equal(outs[0].astype(np.int64), oracle.gemm_s8(M, N, K, A, B, layout_b=oracle.BLOCKED32))
 
 
+@pytest.mark.parametrize("shape", [(4096, 4096, 1408), (3072, 2048, 2176)], ids=["3.46waves", "1.3waves"])
+def test_s8_stream_k_is_exact(shape):
+    """INT8 operands, a ragged last wave shared out by k-blocks over all the pairs: INT32 partial slabs, added as
+    integers by the tail kernel: the exact result on sampled rows, and the same bits as the plan without it."""
+    M, N, K = shape
+    A = nk_inputs.fill(18, nk_inputs.TENSOR_A, M * K, dtype="s8")
+    B = nk_inputs.fill(18, nk_inputs.TENSOR_B, K * N, dtype="s8")
+    sp = torch.cuda.current_stream().cuda_stream
+    outs = []
+    for extra in (nk.flag_tail_split(15), nk.FLAG_NO_TAIL_SPLIT):
+        plan = nk.Plan(M, N, K, in_dtype=nk.S8, out_dtype=nk.S32, layout_a=nk.ROW_MAJOR, layout_b=nk.BLOCKED32,
+                       flags=nk.FLAG_CTA_PAIR | nk.flag_tile_n(4) | nk.flag_splitk(1) | extra)
+        assert ("_streamk" in plan.kernel_name) == (extra != nk.FLAG_NO_TAIL_SPLIT), plan.kernel_name
+        ws = torch.full((max(plan.workspace_bytes, 16),), 0xFF, dtype=torch.uint8, device="cuda")
+        C = torch.full((M * N,), 12345, dtype=torch.int32, device="cuda")
+        plan.run(torch.from_numpy(A).cuda(), torch.from_numpy(B).cuda(), C, workspace=ws if plan.workspace_bytes else None,
+                 workspace_bytes=plan.workspace_bytes, stream=sp)
+        plan.check()
+        outs.append(C.cpu().numpy().reshape(M, N))
+    assert np.array_equal(outs[0], outs[1])
+    rows = nk_inputs.stratified_rows(18, M, 48)
+    assert np.array_equal(outs[0][rows].astype(np.int64), oracle.gemm_s8(M, N, K, A, B, layout_b=oracle.BLOCKED32, rows=rows))
+
+
 @pytest.mark.parametrize("dequant", [False, True])
 def test_s8_tail_wave_split(dequant):
     """More 256 x 256 tiles than CTA pairs: the last wave's tiles are cut along K, their INT32 partials summed

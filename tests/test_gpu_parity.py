@@ -295,14 +295,40 @@ def test_pair_tail_wave_split(out_dtype, epi, splits, bn):
     f = nk.FLAG_CTA_PAIR | nk.flag_tile_n(bn) | nk.flag_splitk(1) | nk.flag_tail_split(splits)
     w = W("tail", M, N, K, "bf16", out_dtype, epilogue=epi, integer=True)
     err, plan = run_and_check(w, flags=f, exact=(out_dtype == "f32"))
-    assert f"_tail{splits}" in plan.kernel_name and plan.launches_per_run == 2 and plan.workspace_bytes > 0
+    # (equal cuts where the tail tiles times the cuts fit the pairs; else the even share of the k-blocks)
+    assert (f"_tail{splits}" in plan.kernel_name or "_streamk" in plan.kernel_name), plan.kernel_name
+    assert plan.launches_per_run == 2 and plan.workspace_bytes > 0
     w = W("tail", M, N, K, "bf16", out_dtype, epilogue=epi, seed=31)
     A, B, bias = w.make()
     c_tail, _ = run_plan(w, A, B, bias, flags=f)
     check_against_oracle(w, c_tail, A, B, bias)
     c_plain, p_plain = run_plan(w, A, B, bias, flags=f & ~nk.flag_tail_split(15) | nk.FLAG_NO_TAIL_SPLIT)
-    assert "_tail" not in p_plain.kernel_name
+    assert "_tail" not in p_plain.kernel_name and "_streamk" not in p_plain.kernel_name
     check_against_oracle(w, c_plain, A, B, bias)
+
+
+@pytest.mark.parametrize("shape", [(4096, 4096, 704), (3072, 2048, 1088), (2500, 2520, 320)], ids=["3.46waves", "1.3waves", "ragged"])
+@pytest.mark.parametrize("out_dtype,epi", [("f32", "none"), ("bf16", "bias_relu")])
+def test_pair_stream_k_shares_the_last_wave(shape, out_dtype, epi):
+    """More 256 x 256 tiles than CTA pairs and a ragged last wave: the k-blocks of the tiles left over are shared
+    out evenly over all the pairs (a pair's range may straddle two tiles), the partial slabs of a tile are
+    summed in k order by the tail kernel.  Exact on integer data (bit for bit against the oracle and against
+    the plan without the tail treatment), then random data under the acceptance bound."""
+    M, N, K = shape
+    f = nk.FLAG_CTA_PAIR | nk.flag_tile_n(4) | nk.flag_splitk(1)
+    rows = nk_inputs.stratified_rows(5, M, 48)
+    w = W("streamk", M, N, K, "bf16", out_dtype, epilogue=epi, integer=True)
+    A, B, bias = w.make()
+    c_sk, plan = run_plan(w, A, B, bias, flags=f | nk.flag_tail_split(15))
+    assert "_streamk" in plan.kernel_name and plan.launches_per_run == 2 and plan.workspace_bytes > 0, plan.kernel_name
+    check_against_oracle(w, c_sk, A, B, bias, rows=rows, exact=(out_dtype == "f32"))
+    c_plain, p_plain = run_plan(w, A, B, bias, flags=f | nk.FLAG_NO_TAIL_SPLIT)
+    assert "_streamk" not in p_plain.kernel_name and "_tail" not in p_plain.kernel_name
+    assert np.array_equal(c_sk, c_plain)
+    w = W("streamk", M, N, K, "bf16", out_dtype, epilogue=epi, seed=33)
+    A, B, bias = w.make()
+    c_sk, _ = run_plan(w, A, B, bias, plan=plan)
+    check_against_oracle(w, c_sk, A, B, bias, rows=rows)
 
 
 @pytest.mark.parametrize("out_dtype,bn", [("f32", 4), ("bf16", 4), ("bf16", 3)])
@@ -311,7 +337,7 @@ def test_pair_tail_units_follow_tma_stored_tiles(out_dtype, bn):
     (whose FP32 partial passes through the same staging memory) must first let those stores read their
     source.  Integer data make both plans exact, so the result with the tail split has to equal, bit for
     bit and on every one of many runs, the result of the plan without it."""
-    M, N, K = 2500, 2520, 128      # a short K loop: the tail unit's accumulator is ready at once
+    M, N, K = 2500, 2520, 256      # a short K loop: the tail unit's accumulator is ready at once
     w = W("tailrace", M, N, K, "bf16", out_dtype, integer=True, seed=77)
     A, B, bias = w.make()
     f = nk.FLAG_CTA_PAIR | nk.flag_tile_n(bn) | nk.flag_splitk(1)
@@ -319,7 +345,7 @@ def test_pair_tail_units_follow_tma_stored_tiles(out_dtype, bn):
     assert "_tail" not in p_plain.kernel_name
     check_against_oracle(w, c_plain, A, B, bias, exact=(out_dtype == "f32"))
     plan = nk.plan_for(w, flags=f | nk.flag_tail_split(2))
-    assert "_tail2" in plan.kernel_name
+    assert "_tail2" in plan.kernel_name or "_streamk" in plan.kernel_name, plan.kernel_name
     for _ in range(25):
         c_tail, _ = run_plan(w, A, B, bias, plan=plan)
         assert np.array_equal(c_tail, c_plain)
