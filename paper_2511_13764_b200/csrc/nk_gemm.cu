@@ -24,7 +24,7 @@ namespace nk {
 // loads the library).  Kernels receive its device address as a parameter.
 __device__ unsigned int g_status_word[4];
 
-enum Variant { V_NAIVE = 0, V_SIMT = 1, V_UMMA = 2, V_SKINNY = 3, V_SPLIT3 = 4 };
+enum Variant { V_NAIVE = 0, V_SIMT = 1, V_UMMA = 2, V_SKINNY = 3, V_SPLIT3 = 4, V_SMALL = 5 };
 
 typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*,
                                   const cuuint64_t*, const cuuint64_t*, const cuuint32_t*,
@@ -887,6 +887,16 @@ nk_status_t nk_gemm_create(const nk_gemm_desc_t* desc, nk_gemm_t* out) {
         p->launches = p->splits > 1 ? 2 : 1;
         snprintf(p->name, sizeof(p->name), "simt_f32_skinny_%dx512_kc%d_splitk%d", d.M <= 16 ? 16 : 32,
                  p->skinny_kc, p->splits);
+    } else if (d.in_dtype == NK_F32 && force == NK_FLAG_KERNEL_AUTO && nbatch == 1 && d.K <= SMALL_KMAX &&
+               !(d.flags & (0xFu << NK_FLAG_TILE_N_SHIFT)) && !(d.flags & (0xFFu << NK_FLAG_SPLITK_SHIFT)) &&
+               static_cast<int64_t>(ceil_div(d.M, SMALL_BM)) * ceil_div(d.N, SMALL_BN) <= 2 * p->sm_count &&
+               ceil_div(d.M, SMALL_BM) <= 65535) {
+        // a small problem: whole K in shared memory, one launch (see simt_f32_small_kernel)
+        p->variant = V_SMALL;
+        if (allow_smem(simt_f32_small_kernel, simt_small_smem_bytes(SMALL_KMAX)) != cudaSuccess) { cudaGetLastError(); delete p; return NK_ERR_CUDA; }
+        p->splits = 1;
+        p->launches = 1;
+        snprintf(p->name, sizeof(p->name), "simt_f32_small_32x32_k%d", static_cast<int>(d.K));
     } else if (d.in_dtype == NK_F32) {
         p->variant = V_SIMT;
         if (prepare_simt_attrs() != cudaSuccess) { cudaGetLastError(); delete p; return NK_ERR_CUDA; }
@@ -1076,7 +1086,15 @@ nk_status_t nk_gemm_run(nk_gemm_t p, const void* A, const void* B, const void* b
     uint8_t* ws = static_cast<uint8_t*>(workspace);
     float* partial = p->ws_partial_bytes ? reinterpret_cast<float*>(ws + p->ws_repack_bytes) : nullptr;
 
-    if (p->variant == V_SKINNY) {
+    if (p->variant == V_SMALL) {
+        SmallParams mp = {static_cast<int>(d.M), static_cast<int>(d.N), static_cast<int>(d.K), d.beta, d.epilogue,
+                          static_cast<const float*>(A), static_cast<const float*>(B), static_cast<const float*>(bias),
+                          static_cast<float*>(C)};
+        dim3 grid(ceil_div(d.N, SMALL_BN), ceil_div(d.M, SMALL_BM));
+        simt_f32_small_kernel<<<grid, SMALL_THREADS, simt_small_smem_bytes(static_cast<int>(d.K)), st>>>(mp);
+        e = cudaGetLastError();
+        if (e != cudaSuccess) { set_err(p, "small launch", e); return NK_ERR_CUDA; }
+    } else if (p->variant == V_SKINNY) {
         SkinnyParams kp = {static_cast<int>(d.M), static_cast<int>(d.N), static_cast<int>(d.K), p->skinny_kc,
                            p->splits, d.epilogue, static_cast<const float*>(A), static_cast<const float*>(B),
                            static_cast<const float*>(bias), static_cast<float*>(C), partial};

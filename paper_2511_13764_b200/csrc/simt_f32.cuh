@@ -470,3 +470,121 @@ simt_f32_async_kernel(const SimtParams p) {
 }
 
 }  // namespace nk
+
+namespace nk {
+
+// Small FP32 GEMM: a problem whose whole K fits shared memory next to a 32 x 32 tile of C and
+// whose tiles number a CTA or two per SM.  Such a problem is all latency: a pipelined K loop
+// would pay a global-load round trip per k-tile, and K splits a second kernel.  Here a CTA issues
+// every copy of its A and B slabs at once (one round trip), then its 256 threads multiply: four
+// groups of 64 threads take a quarter of K each, a thread keeps 4 x 4 of C in registers
+// (Algorithm 1's resident accumulator), and the four partial tiles meet in shared memory and are
+// added in group order (k order: deterministic) by the first group, which applies beta, bias +
+// ReLU and stores.  One launch, no workspace.
+constexpr int SMALL_BM = 32, SMALL_BN = 32, SMALL_THREADS = 256, SMALL_KMAX = 512;
+constexpr int SMALL_AP = SMALL_BM + 4;    // padded row of the transposed A slab As[k][m]
+// the two slabs, or the three partial tiles that later take their place, whichever is larger
+__host__ __device__ constexpr int simt_small_smem_bytes(int K) {
+    return K * (SMALL_AP + SMALL_BN) * 4 > 3 * 64 * 16 * 4 ? K * (SMALL_AP + SMALL_BN) * 4 : 3 * 64 * 16 * 4;
+}
+
+struct SmallParams {
+    int M, N, K;
+    int beta, epilogue;
+    const float* A;    // [M][K]
+    const float* B;    // [K][N]
+    const float* bias; // [N] or null
+    float* C;          // [M][N]
+};
+
+__global__ void __launch_bounds__(SMALL_THREADS, 2) simt_f32_small_kernel(const SmallParams p) {
+    extern __shared__ __align__(16) float small_smem[];
+    float* As = small_smem;                       // [K][AP]
+    float* Bs = small_smem + p.K * SMALL_AP;      // [K][BN]
+    const uint32_t as_u32 = smem_u32(As), bs_u32 = smem_u32(Bs);
+    const int t = threadIdx.x, lane = t & 31, warp = t >> 5;
+    const int m0 = blockIdx.y * SMALL_BM, n0 = blockIdx.x * SMALL_BN;
+
+    // A: 4-byte copies that transpose on the way.  A warp copies 8 consecutive k of 4 consecutive
+    // rows per instruction (whole 32-byte sectors of global memory; the 32 shared-memory words
+    // k * 36 + row fall into 32 different banks).  Warp w takes rows 4 w .. 4 w + 3, one k octet per step.
+    {
+        const int kq = lane & 7, r4 = lane >> 3;
+        const int octets = (p.K + 7) >> 3;
+        for (int idx = warp; idx < 8 * octets; idx += SMALL_THREADS / 32) {   // idx = row group (0..7) + 8 * k octet
+            const int row = (idx & 7) * 4 + r4, k = (idx >> 3) * 8 + kq;
+            const bool ok = m0 + row < p.M && k < p.K;
+            if (k < p.K)
+                cp_async_4(as_u32 + (k * SMALL_AP + row) * 4, ok ? p.A + static_cast<size_t>(m0 + row) * p.K + k : p.A, ok ? 4u : 0u);
+        }
+        // B: 16-byte copies, a row of the slab (32 columns) per 8 lanes
+        const int nq = (t & 7) * 4;
+        const bool col_ok = n0 + nq < p.N;          // N is a multiple of 4
+        for (int k = t >> 3; k < p.K; k += SMALL_THREADS / 8)
+            cp_async_16(bs_u32 + (k * SMALL_BN + nq) * 4, col_ok ? p.B + static_cast<size_t>(k) * p.N + n0 + nq : p.B, col_ok ? 16u : 0u);
+        cp_async_commit();
+        cp_async_wait_group<0>();
+    }
+    __syncthreads();
+
+    const int g = t >> 6, tt = t & 63, ty = tt >> 3, tx = tt & 7;
+    const int kper = (p.K + 3) >> 2;
+    const int k0 = g * kper, k1 = min(p.K, k0 + kper);
+    float acc[4][4];
+#pragma unroll
+    for (int i = 0; i < 4; ++i)
+#pragma unroll
+        for (int j = 0; j < 4; ++j) acc[i][j] = 0.0f;
+#pragma unroll 4
+    for (int k = k0; k < k1; ++k) {
+        const float4 a = *reinterpret_cast<const float4*>(As + k * SMALL_AP + ty * 4);
+        const float4 b = *reinterpret_cast<const float4*>(Bs + k * SMALL_BN + tx * 4);
+        const float av[4] = {a.x, a.y, a.z, a.w}, bv[4] = {b.x, b.y, b.z, b.w};
+#pragma unroll
+        for (int i = 0; i < 4; ++i)
+#pragma unroll
+            for (int j = 0; j < 4; ++j) acc[i][j] = fmaf(av[i], bv[j], acc[i][j]);
+    }
+    __syncthreads();                                // the slabs are consumed: the partial tiles take their place
+    float* red = small_smem;                        // [3][64][16]
+    if (g > 0) {
+        float4* dst = reinterpret_cast<float4*>(red + ((g - 1) * 64 + tt) * 16);
+#pragma unroll
+        for (int i = 0; i < 4; ++i) dst[i] = make_float4(acc[i][0], acc[i][1], acc[i][2], acc[i][3]);
+    }
+    __syncthreads();
+    if (g > 0) return;
+#pragma unroll
+    for (int s = 0; s < 3; ++s) {
+        const float4* src = reinterpret_cast<const float4*>(red + (s * 64 + tt) * 16);
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            const float4 v = src[i];
+            acc[i][0] += v.x; acc[i][1] += v.y; acc[i][2] += v.z; acc[i][3] += v.w;
+        }
+    }
+    const int gn = n0 + tx * 4;
+    if (gn >= p.N) return;
+    float4 bias4 = make_float4(0.f, 0.f, 0.f, 0.f);
+    if (p.epilogue) bias4 = __ldg(reinterpret_cast<const float4*>(p.bias + gn));
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        const int gm = m0 + ty * 4 + i;
+        if (gm >= p.M) break;
+        float4 v = make_float4(acc[i][0], acc[i][1], acc[i][2], acc[i][3]);
+        float* dst = p.C + static_cast<size_t>(gm) * p.N + gn;
+        if (p.beta) {       // beta = 1: the accumulation tile starts from the stored C
+            const float4 cv = *reinterpret_cast<const float4*>(dst);
+            v.x += cv.x; v.y += cv.y; v.z += cv.z; v.w += cv.w;
+        }
+        if (p.epilogue) {
+            v.x = fmaxf(v.x + bias4.x, 0.f);
+            v.y = fmaxf(v.y + bias4.y, 0.f);
+            v.z = fmaxf(v.z + bias4.z, 0.f);
+            v.w = fmaxf(v.w + bias4.w, 0.f);
+        }
+        *reinterpret_cast<float4*>(dst) = v;
+    }
+}
+
+}  // namespace nk

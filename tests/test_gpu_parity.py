@@ -52,6 +52,22 @@ def test_simt_f32_exact_integer(shape, tile):
     run_and_check(w, flags=nk.FLAG_KERNEL_SIMT | nk.flag_tile_n(tile), exact=True, expect_kernel="simt_f32")
 
 
+SMALL_SHAPES = [(256, 256, 256), (33, 132, 68), (130, 260, 100), (300, 520, 40), (512, 384, 512), (40, 4, 4),
+                (64, 64, 8), (900, 320, 36)]
+
+
+@pytest.mark.parametrize("shape", SMALL_SHAPES)
+@pytest.mark.parametrize("epi", ["none", "bias_relu"])
+def test_simt_f32_small_kernel(shape, epi):
+    """Small FP32 problems (K <= 512, a CTA or two per SM): whole-K slabs in shared memory, four k groups per
+    CTA summed in order, one launch, no workspace.  Exact on integer data, then random data; ragged M, N, K."""
+    M, N, K = shape
+    err, plan = run_and_check(W("small", M, N, K, "f32", epilogue=epi, integer=True), exact=True,
+                              expect_kernel="simt_f32_small")
+    assert plan.launches_per_run == 1 and plan.workspace_bytes == 0
+    run_and_check(W("small", M, N, K, "f32", epilogue=epi, seed=12), expect_kernel="simt_f32_small")
+
+
 @pytest.mark.parametrize("shape", SIMT_SHAPES)
 def test_simt_f32_random_auto(shape):
     M, N, K = shape
