@@ -71,6 +71,10 @@ def lib():
         L.nko_brgemm.argtypes = [ctypes.c_int64] * 6 + [ctypes.c_int32, ctypes.c_int32, ctypes.c_double,
                                  ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p,
                                  ctypes.c_void_p, ctypes.c_void_p]
+        L.nko_brgemm_layout.restype = ctypes.c_int
+        L.nko_brgemm_layout.argtypes = [ctypes.c_int64] * 6 + [ctypes.c_int32] * 4 + [ctypes.c_double,
+                                        ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p,
+                                        ctypes.c_void_p, ctypes.c_void_p]
         for f in (L.nko_pack_vnni4, L.nko_unpack_vnni4):
             f.restype = None
             f.argtypes = [ctypes.c_void_p, ctypes.c_int64, ctypes.c_int64, ctypes.c_void_p]
@@ -257,10 +261,11 @@ def gemm_workload(w, A, B, bias, rows=None, cols=None, **kw):
 
 
 def brgemm(M, N, K, batch, A, B, bias=None, C0=None, *, in_dtype=F32, epilogue=EPI_NONE, beta=0.0,
-           stride_a=None, stride_b=None):
-    """Batch-reduce GEMM (Algorithm 1's output line): beta*C0 + sum_b A_b.B_b, row-major.
+           stride_a=None, stride_b=None, layout_a=ROW, layout_b=ROW):
+    """Batch-reduce GEMM (Algorithm 1's output line): beta*C0 + sum_b A_b.B_b.
     A and B are storage buffers holding all batch items (item b of A starts at b*stride_a
-    elements; default M*K and K*N).  C0: float64 [M][N] (the stored C widened) when beta = 1.
+    elements; default M*K and K*N), every item row-major or 32x32-blocked / VNNI-packed
+    (Listing 1's items).  C0: float64 [M][N] (the stored C widened) when beta = 1.
     Returns (Y, S) float64 [M][N]."""
     dt = _np_dtype(in_dtype)
     A = np.ascontiguousarray(A, dtype=dt)
@@ -279,8 +284,12 @@ def brgemm(M, N, K, batch, A, B, bias=None, C0=None, *, in_dtype=F32, epilogue=E
         cp = C0.ctypes.data
     Y = np.empty((M, N), dtype=np.float64)
     S = np.empty((M, N), dtype=np.float64)
-    rc = lib().nko_brgemm(M, N, K, batch, stride_a, stride_b, in_dtype, epilogue, float(beta),
-                          A.ctypes.data, B.ctypes.data, bp, cp, Y.ctypes.data, S.ctypes.data)
+    if layout_a == ROW and layout_b == ROW:
+        rc = lib().nko_brgemm(M, N, K, batch, stride_a, stride_b, in_dtype, epilogue, float(beta),
+                              A.ctypes.data, B.ctypes.data, bp, cp, Y.ctypes.data, S.ctypes.data)
+    else:
+        rc = lib().nko_brgemm_layout(M, N, K, batch, stride_a, stride_b, in_dtype, layout_a, layout_b, epilogue,
+                                     float(beta), A.ctypes.data, B.ctypes.data, bp, cp, Y.ctypes.data, S.ctypes.data)
     if rc != 0:
         raise ValueError("oracle rejected the arguments")
     return Y, S

@@ -243,21 +243,26 @@ int nko_gemm(const nko_desc_t* d, const void* A, const void* B, const void* bias
  * epilogue as nko_gemm.  S receives sum |a.b| + |beta.C0| (+ |bias|).  Plain loops, one
  * thread: this is the definition, used on test sizes only.
  */
-int nko_brgemm(int64_t M, int64_t N, int64_t K, int64_t batch, int64_t stride_a, int64_t stride_b,
-               int32_t in_dtype, int32_t epilogue, double beta, const void* A, const void* B,
-               const void* bias, const double* C0, double* Y, double* S) {
+int nko_brgemm_layout(int64_t M, int64_t N, int64_t K, int64_t batch, int64_t stride_a, int64_t stride_b,
+                      int32_t in_dtype, int32_t layout_a, int32_t layout_b, int32_t epilogue, double beta,
+                      const void* A, const void* B, const void* bias, const double* C0, double* Y, double* S) {
     if (!A || !B || !Y || M <= 0 || N <= 0 || K <= 0 || batch <= 0) return -1;
     if (beta != 0.0 && beta != 1.0) return -1;
     if (beta != 0.0 && !C0) return -1;
     if (epilogue == NKO_EPI_BIAS_RELU && !bias) return -1;
+    if (layout_a == NKO_BLOCKED32 && (M % 32 || K % 32)) return -1;
+    if (layout_b == NKO_BLOCKED32 && (N % 32 || K % 32)) return -1;
+    /* every batch item is one operand in the given layout (Listing 1: VNNI-packed items), item b
+     * starting b * stride elements into the buffer; inside an item the index formulas of nko_gemm */
+    nko_desc_t d = {M, N, K, in_dtype, layout_a, layout_b, epilogue, NKO_ACC_F64};
     for (int64_t i = 0; i < M; ++i) {
         for (int64_t j = 0; j < N; ++j) {
             double acc = beta != 0.0 ? beta * C0[i * N + j] : 0.0;
             double s = fabs(acc);
             for (int64_t b = 0; b < batch; ++b) {
                 for (int64_t k = 0; k < K; ++k) {
-                    double p = load(A, in_dtype, b * stride_a + i * K + k) *
-                               load(B, in_dtype, b * stride_b + k * N + j);
+                    double p = load(A, in_dtype, b * stride_a + a_index(&d, i, k)) *
+                               load(B, in_dtype, b * stride_b + b_index(&d, k, j));
                     acc += p;
                     s += fabs(p);
                 }
@@ -273,6 +278,14 @@ int nko_brgemm(int64_t M, int64_t N, int64_t K, int64_t batch, int64_t stride_a,
         }
     }
     return 0;
+}
+
+/* The row-major form (the first interface): the same loops with row-major index formulas. */
+int nko_brgemm(int64_t M, int64_t N, int64_t K, int64_t batch, int64_t stride_a, int64_t stride_b,
+               int32_t in_dtype, int32_t epilogue, double beta, const void* A, const void* B,
+               const void* bias, const double* C0, double* Y, double* S) {
+    return nko_brgemm_layout(M, N, K, batch, stride_a, stride_b, in_dtype, NKO_ROW, NKO_ROW, epilogue, beta,
+                             A, B, bias, C0, Y, S);
 }
 
 /* ------------------------------------------------------------------ INT8

@@ -391,6 +391,58 @@ def test_brgemm_beta_and_strides():
         oracle.brgemm(M, N, K, batch, A, B, C0=C0, beta=0.5, stride_a=sa, stride_b=sb)
 
 
+def _pack_items_figure1(As, Bs):
+    """Blocked storage of batch items written with numpy reshapes from the layout's definition (not with the
+    oracle's index functions): A[M/32][K/32][32][32]; B[N/32][K/32][16][32][2] with Figure 1's rule
+    packed[k/2][n][k%2] = flat[k][n] inside every 32 x 32 block."""
+    out_a, out_b = [], []
+    for A, B in zip(As, Bs):
+        M, K = A.shape
+        N = B.shape[1]
+        out_a.append(A.reshape(M // 32, 32, K // 32, 32).transpose(0, 2, 1, 3).reshape(-1))
+        blk = B.reshape(K // 32, 32, N // 32, 32).transpose(2, 0, 1, 3)          # [n-block][k-block][k][n]
+        out_b.append(blk.reshape(N // 32, K // 32, 16, 2, 32).transpose(0, 1, 2, 4, 3).reshape(-1))
+    return out_a, out_b
+
+
+@pytest.mark.parametrize("M,N,K,batch", [(32, 192, 32, 4), (64, 64, 64, 2), (96, 32, 160, 3)])
+def test_brgemm_over_blocked_items_is_the_flat_brgemm(M, N, K, batch):
+    """Listing 1's kernel is a batch-reduce over VNNI-packed items.  Items packed from the layout's definition
+    (numpy reshapes, Figure 1's pair rule) give, through the blocked interface, bit for bit what the flat
+    interface gives on the flat items (same products, same k order), also with gaps between the items and
+    with beta = 1; a swapped pair order or a transposed block is caught."""
+    As = [_rand_int((M, K), 700 + i) for i in range(batch)]
+    Bs = [_rand_int((K, N), 800 + i) for i in range(batch)]
+    Yf, Sf = oracle.brgemm(M, N, K, batch, _bits(np.stack(As).reshape(-1)), _bits(np.stack(Bs).reshape(-1)), in_dtype=BF16)
+    pa, pb = _pack_items_figure1(As, Bs)
+    gap_a, gap_b = 64, 32
+    A = np.zeros((batch - 1) * (M * K + gap_a) + M * K, dtype=np.float32)
+    B = np.zeros((batch - 1) * (K * N + gap_b) + K * N, dtype=np.float32)
+    for b in range(batch):
+        A[b * (M * K + gap_a):b * (M * K + gap_a) + M * K] = pa[b]
+        B[b * (K * N + gap_b):b * (K * N + gap_b) + K * N] = pb[b]
+    kw = dict(in_dtype=BF16, layout_a=BLOCKED32, layout_b=BLOCKED32, stride_a=M * K + gap_a, stride_b=K * N + gap_b)
+    Yb, Sb = oracle.brgemm(M, N, K, batch, _bits(A), _bits(B), **kw)
+    assert np.array_equal(Yb, Yf) and np.array_equal(Sb, Sf)
+    C0 = _rand_int((M, N), 900).astype(np.float64)
+    Y1, _ = oracle.brgemm(M, N, K, batch, _bits(A), _bits(B), C0=C0, beta=1.0, **kw)
+    assert np.array_equal(Y1, Yf + C0)
+    # planted mistakes: the odd/even pair swapped inside B's words; B's block read as its transpose
+    Bsw = B.copy()
+    for b in range(batch):
+        seg = Bsw[b * (K * N + gap_b):b * (K * N + gap_b) + K * N].reshape(-1, 2)
+        seg[:] = seg[:, ::-1]
+    Yw, _ = oracle.brgemm(M, N, K, batch, _bits(A), _bits(Bsw), **kw)
+    assert not np.array_equal(Yw, Yf)
+    # mixed forms: blocked A with flat B, flat A with blocked B
+    Ym, _ = oracle.brgemm(M, N, K, batch, _bits(A), _bits(np.stack(Bs).reshape(-1)), in_dtype=BF16, layout_a=BLOCKED32,
+                          stride_a=M * K + gap_a)
+    assert np.array_equal(Ym, Yf)
+    Yn, _ = oracle.brgemm(M, N, K, batch, _bits(np.stack(As).reshape(-1)), _bits(B), in_dtype=BF16, layout_b=BLOCKED32,
+                          stride_b=K * N + gap_b)
+    assert np.array_equal(Yn, Yf)
+
+
 def test_brgemm_batch_one_is_gemm():
     M, N, K = 9, 12, 20
     A = nk_inputs.fill(60, 0, M * K)
