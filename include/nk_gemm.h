@@ -84,8 +84,8 @@ typedef enum {
     NK_ROW_MAJOR = 0,
     NK_BLOCKED32 = 1,
     NK_TRANSPOSED = 2 /* layout_b only: B is stored transposed, Bt[N][K] with K contiguous (the way a linear layer's
-                         weight [out][in] is usually kept).  16-bit and 8-bit operands; K a multiple of 16, N of 8;
-                         no batch.  Not one of the paper's layouts (flat [K][N] and VNNI-blocked): on this hardware
+                         weight [out][in] is usually kept).  16-bit and 8-bit operands; K a multiple of 16, N of 8.
+                         Not one of the paper's layouts (flat [K][N] and VNNI-blocked): on this hardware
                          it is the operand form the tensor core reads without any re-layout */
 } nk_layout_t;
 typedef enum { NK_EPI_NONE = 0, NK_EPI_BIAS_RELU = 1 } nk_epilogue_t;
@@ -161,8 +161,10 @@ typedef struct {
  * blocked operand's two dimensions to be multiples of 32; row-major BF16 needs N and K
  * to be multiples of 8, row-major FP32 needs N and K to be multiples of 4
  * (16-byte rows); BF16 output needs BF16 inputs.  batch > 1 (Section 2.1: the source tiles
- * of a batch-reduce GEMM need not be contiguous, the accumulation tile is C) needs
- * row-major operands and strides that are multiples of 8 (BF16) or 4 (FP32) elements; with
+ * of a batch-reduce GEMM need not be contiguous, the accumulation tile is C) takes every
+ * item in the operand's layout (row-major, blocked / VNNI-packed as in Listing 1, or B
+ * transposed; 16-bit and FP32 operands) and needs strides that are multiples of 8 (16-bit)
+ * or 4 (FP32) elements; with
  * beta = 1, y = epilogue(C_old + sum_b A_b.B_b), C_old read in C's own layout.  A blocked C
  * needs BF16 operands and M, N multiples of 32.  On failure *out is NULL.
  */

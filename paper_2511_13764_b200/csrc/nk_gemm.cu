@@ -374,11 +374,14 @@ static nk_status_t encode_maps(nk_gemm_s* p, const void* A, const void* B) {
     if (d.layout_a == NK_BLOCKED32) {
         // [M/32][K/32][32][32] as a 4-D tensor (k, m, k-block, m-block): a box of
         // 32 x 32 x 1 x 4 lands in shared memory as 128 rows of 32 consecutive k (64 B).
-        cuuint64_t dims[4] = {32, 32, static_cast<cuuint64_t>(d.K / 32), static_cast<cuuint64_t>(d.M / 32)};
-        cuuint64_t strides[3] = {32 * 2, 1024 * 2, static_cast<cuuint64_t>(d.K / 32) * 1024 * 2};
-        cuuint32_t box[4] = {32, 32, 1, 4};
-        cuuint32_t es[4] = {1, 1, 1, 1};
-        r = p->encode(&p->tmap_a, half_type, 4, const_cast<void*>(A), dims, strides,
+        // Batch items (stride_a elements apart) are the fifth dimension.
+        cuuint64_t dims[5] = {32, 32, static_cast<cuuint64_t>(d.K / 32), static_cast<cuuint64_t>(d.M / 32),
+                              static_cast<cuuint64_t>(p->batch * p->gemms)};
+        cuuint64_t strides[4] = {32 * 2, 1024 * 2, static_cast<cuuint64_t>(d.K / 32) * 1024 * 2,
+                                 static_cast<cuuint64_t>(p->stride_a) * 2};
+        cuuint32_t box[5] = {32, 32, 1, 4, 1};
+        cuuint32_t es[5] = {1, 1, 1, 1, 1};
+        r = p->encode(&p->tmap_a, half_type, 5, const_cast<void*>(A), dims, strides,
                       box, es, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_64B,
                       CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
     } else {
@@ -454,11 +457,13 @@ static nk_status_t encode_maps(nk_gemm_s* p, const void* A, const void* B) {
         // INT8: the same bytes with four k per group: [N/32][K/32][8][32][4] is (128 elements, K/4, N/32).
         const int cols = p->pair ? p->bn / 2 : p->bn;
         const cuuint64_t group = 4 / esz;   // k per 32-bit word: 2 (16-bit) or 4 (8-bit)
-        cuuint64_t dims[3] = {128 / esz, static_cast<cuuint64_t>(d.K) / group, static_cast<cuuint64_t>(d.N / 32)};
-        cuuint64_t strides[2] = {128, static_cast<cuuint64_t>(d.K) * 32 * esz};
-        cuuint32_t box[3] = {static_cast<cuuint32_t>(128 / esz), UMMA_BK / 2, static_cast<cuuint32_t>(cols / 32)};
-        cuuint32_t es[3] = {1, 1, 1};
-        r = p->encode(&p->tmap_b, half_type, 3, const_cast<void*>(B), dims, strides,
+        // Batch items (stride_b elements apart) are the fourth dimension.
+        cuuint64_t dims[4] = {128 / esz, static_cast<cuuint64_t>(d.K) / group, static_cast<cuuint64_t>(d.N / 32),
+                              static_cast<cuuint64_t>(p->batch * p->gemms)};
+        cuuint64_t strides[3] = {128, static_cast<cuuint64_t>(d.K) * 32 * esz, static_cast<cuuint64_t>(p->stride_b) * esz};
+        cuuint32_t box[4] = {static_cast<cuuint32_t>(128 / esz), UMMA_BK / 2, static_cast<cuuint32_t>(cols / 32), 1};
+        cuuint32_t es[4] = {1, 1, 1, 1};
+        r = p->encode(&p->tmap_b, half_type, 4, const_cast<void*>(B), dims, strides,
                       box, es, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
                       CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
         if (r != CUDA_SUCCESS) {
@@ -781,7 +786,6 @@ nk_status_t nk_gemm_create(const nk_gemm_desc_t* desc, nk_gemm_t* out) {
     const int64_t str_a = d.stride_a > 0 ? d.stride_a : d.M * d.K;
     const int64_t str_b = d.stride_b > 0 ? d.stride_b : d.K * d.N;
     if (nbatch > 1) {
-        if (blocked || d.layout_b == NK_TRANSPOSED) return NK_ERR_UNSUPPORTED;          // batch-reduce: row-major operands only
         if (nbatch > 65535 || nbatch * d.K >= (1ll << 24)) return NK_ERR_UNSUPPORTED;
         const int64_t gran = is16(d.in_dtype) ? 8 : 4;
         if (str_a % gran || str_b % gran) return NK_ERR_MISALIGNED;

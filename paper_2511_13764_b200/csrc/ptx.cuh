@@ -420,6 +420,14 @@ __device__ __forceinline__ void tma_load_4d_if(uint32_t dst, const void* tmap, u
                  "l"(tmap), "r"(bar), "r"(c0), "r"(c1), "r"(c2), "r"(c3), "r"(elected)
                  : "memory");
 }
+__device__ __forceinline__ void tma_load_5d_if(uint32_t dst, const void* tmap, uint32_t bar, int c0, int c1, int c2, int c3,
+                                               int c4, uint32_t elected) {
+    asm volatile("{\n\t.reg .pred q;\n\tsetp.ne.b32 q, %8, 0;\n\t"
+                 "@q cp.async.bulk.tensor.5d.shared::cluster.global.mbarrier::complete_tx::bytes"
+                 " [%0], [%1, {%3, %4, %5, %6, %7}], [%2];\n\t}" ::"r"(dst),
+                 "l"(tmap), "r"(bar), "r"(c0), "r"(c1), "r"(c2), "r"(c3), "r"(c4), "r"(elected)
+                 : "memory");
+}
 // Pair forms: completion bytes go to `cluster_bar`, which may live in the other CTA of the pair (no multicast).
 __device__ __forceinline__ void tma_load_3d_pair_if(uint32_t dst, const void* tmap, uint32_t cluster_bar, int c0, int c1,
                                                     int c2, uint32_t elected) {
@@ -435,6 +443,14 @@ __device__ __forceinline__ void tma_load_4d_pair_if(uint32_t dst, const void* tm
                  "@q cp.async.bulk.tensor.4d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes"
                  " [%0], [%1, {%3, %4, %5, %6}], [%2];\n\t}" ::"r"(dst),
                  "l"(tmap), "r"(cluster_bar), "r"(c0), "r"(c1), "r"(c2), "r"(c3), "r"(elected)
+                 : "memory");
+}
+__device__ __forceinline__ void tma_load_5d_pair_if(uint32_t dst, const void* tmap, uint32_t cluster_bar, int c0, int c1,
+                                                    int c2, int c3, int c4, uint32_t elected) {
+    asm volatile("{\n\t.reg .pred q;\n\tsetp.ne.b32 q, %8, 0;\n\t"
+                 "@q cp.async.bulk.tensor.5d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes"
+                 " [%0], [%1, {%3, %4, %5, %6, %7}], [%2];\n\t}" ::"r"(dst),
+                 "l"(tmap), "r"(cluster_bar), "r"(c0), "r"(c1), "r"(c2), "r"(c3), "r"(c4), "r"(elected)
                  : "memory");
 }
 // tcgen05.mma, issued by the elected lane only.  KIND: 0 = 16-bit floating point, 1 = INT8, 2 = 8-bit

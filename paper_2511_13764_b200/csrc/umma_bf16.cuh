@@ -773,15 +773,15 @@ umma_bf16_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_consta
                     mbar_arrive_expect_tx_if(fb, UMMA_A_STAGE_BYTES + (B_VNNI ? 0 : B_STAGE), elected);
                     if (a_blk) {
                         // two 32-wide K slabs, each 128 rows x 64 B (64-byte swizzle)
-                        tma_load_4d_if(sa, &tmap_a, fb, 0, 0, kbl * 2, mb * 4, elected);
-                        tma_load_4d_if(sa + 8192, &tmap_a, fb, 0, 0, kbl * 2 + 1, mb * 4, elected);
+                        tma_load_5d_if(sa, &tmap_a, fb, 0, 0, kbl * 2, mb * 4, ia, elected);
+                        tma_load_5d_if(sa + 8192, &tmap_a, fb, 0, 0, kbl * 2 + 1, mb * 4, ia, elected);
                     } else {
                         tma_load_3d_if(sa, &tmap_a, fb, kx, row0, ia, elected);
                     }
                     if (B_VNNI) {
                         // the stage's blocks as they are; warps 6-9 re-lay them in place
                         mbar_arrive_expect_tx_if(raw_bar(stage), B_STAGE, elected);
-                        tma_load_3d_if(sb, &tmap_b, raw_bar(stage), 0, kbl * (UMMA_BK / 2), col0 >> 5, elected);
+                        tma_load_4d_if(sb, &tmap_b, raw_bar(stage), 0, kbl * (UMMA_BK / 2), col0 >> 5, ib, elected);
                     } else if (b_kmajor) {
                         tma_load_3d_if(sb, &tmap_b, fb, kx, col0, ib, elected);   // BN rows (n) of 128 bytes of k
                     } else {

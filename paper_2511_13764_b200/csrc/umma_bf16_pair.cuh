@@ -200,15 +200,15 @@ umma_bf16_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_c
                     const uint32_t sb = sa + UMMA_A_STAGE_BYTES;
                     mbar_arrive_expect_tx_if(fb, 2u * (UMMA_A_STAGE_BYTES + (B_VNNI ? 0 : B_STAGE)), lead_elected);
                     if (a_blk) {
-                        tma_load_4d_pair_if(sa, &tmap_a, lfb, 0, 0, kbl * 2, row0 / 32, elected);
-                        tma_load_4d_pair_if(sa + 8192, &tmap_a, lfb, 0, 0, kbl * 2 + 1, row0 / 32, elected);
+                        tma_load_5d_pair_if(sa, &tmap_a, lfb, 0, 0, kbl * 2, row0 / 32, ia, elected);
+                        tma_load_5d_pair_if(sa + 8192, &tmap_a, lfb, 0, 0, kbl * 2 + 1, row0 / 32, ia, elected);
                     } else {
                         tma_load_3d_pair_if(sa, &tmap_a, lfb, kx, row0, ia, elected);
                     }
                     if (B_VNNI) {
                         // this CTA's column blocks as they are, on its own barrier; its warps 6-9 re-lay them in place
                         mbar_arrive_expect_tx_if(raw_bar(stage), B_STAGE, elected);
-                        tma_load_3d_if(sb, &tmap_b, raw_bar(stage), 0, kbl * (UMMA_BK / 2), col0 >> 5, elected);
+                        tma_load_4d_if(sb, &tmap_b, raw_bar(stage), 0, kbl * (UMMA_BK / 2), col0 >> 5, ib, elected);
                     } else if (b_kmajor) {
                         tma_load_3d_pair_if(sb, &tmap_b, lfb, kx, col0, ib, elected);   // this CTA's HALF rows (n) of 128 bytes of k
                     } else {

@@ -56,8 +56,8 @@ def test_status_strings():
     (dict(M=32, N=32, K=48, in_dtype=1, layout_b=1), 3),
     (dict(M=8, N=12, K=8, in_dtype=1), 3),                       # BF16 rows must be 16-byte multiples
     (dict(M=8, N=8, K=6, in_dtype=0), 3),
-    (dict(M=32, N=32, K=32, in_dtype=1, layout_a=1, batch=2), 2),       # batch-reduce needs row-major
-    (dict(M=32, N=32, K=32, in_dtype=1, layout_b=1, batch=2), 2),
+    (dict(M=32, N=32, K=32, in_dtype=1, layout_a=1, batch=2, stride_a=1028), 3),   # blocked items: strides in 8-element steps too
+    (dict(M=32, N=32, K=32, in_dtype=3, out_dtype=4, layout_b=1, batch=2), 2),     # no batch with 8-bit operands
     (dict(M=8, N=8, K=8, in_dtype=1, batch=2, stride_a=68), 3),           # stride not a multiple of 8
     (dict(M=8, N=8, K=8, in_dtype=0, batch=2, stride_b=32), 1),           # items overlap
     (dict(M=8, N=8, K=8, in_dtype=0, beta=2), 1),

@@ -138,3 +138,60 @@ def test_batched_matmul_auto_and_naive():
     _run_bmm(256, 256, 256, 16, "bf16", "f32", False, 0, integer=False)
     _run_bmm(24, 40, 16, 3, "f32", "f32", True, 1, pad_c=4, flags=nk.FLAG_KERNEL_NAIVE)
     _run_bmm(16, 64, 64, 4, "f32", "f32", False, 0)      # small M, batched: tiled kernel, not the streaming one
+
+
+# ---------------------------------------------------------------- batch items in the blocked / VNNI-packed layout
+def _run_layout(M, N, K, batch, out_dt, epi, beta, layout, pad_a=0, pad_b=0, flags=0, integer=True, seed=1,
+                independent=False):
+    """Batch items stored blocked (A[M/32][K/32][32][32], B VNNI-packed [N/32][K/32][16][32][2]) or with B kept
+    as its transpose; entries are i.i.d., so a buffer of the right length filled by index is a valid operand
+    in any layout.  Compared with the oracle's layout-aware batch-reduce."""
+    sa, sb = M * K + pad_a, K * N + pad_b
+    dist = "int" if integer else "uniform"
+    A = nk_inputs.fill(seed, nk_inputs.TENSOR_A, (batch - 1) * sa + M * K, dist, dtype="bf16")
+    B = nk_inputs.fill(seed, nk_inputs.TENSOR_B, (batch - 1) * sb + K * N, dist, dtype="bf16")
+    bias = nk_inputs.fill(seed, nk_inputs.TENSOR_BIAS, N, dist, dtype="bf16") if epi else None
+    C0 = nk_inputs.fill(seed, 5, M * N, dist, dtype=out_dt)
+    lay_a = nk.BLOCKED32 if layout == "blocked" else nk.ROW_MAJOR
+    lay_b = nk.BLOCKED32 if layout == "blocked" else nk.TRANSPOSED
+    plan = nk.Plan(M, N, K, nk.BF16, nk.BF16 if out_dt == "bf16" else nk.F32, layout_a=lay_a, layout_b=lay_b,
+                   epilogue=nk.EPI_BIAS_RELU if epi else nk.EPI_NONE, flags=flags, beta=beta, batch=batch,
+                   stride_a=sa if pad_a else 0, stride_b=sb if pad_b else 0)
+    dC = to_device(C0).clone()
+    ws = torch.empty(max(plan.workspace_bytes, 16), dtype=torch.uint8, device="cuda")
+    plan.run(to_device(A), to_device(B), dC, bias=to_device(bias) if epi else None,
+             workspace=ws if plan.workspace_bytes else None, workspace_bytes=plan.workspace_bytes,
+             stream=torch.cuda.current_stream().cuda_stream)
+    plan.check()
+    got = c_to_f64(dC).reshape(M, N)
+    c0 = (C0.astype(np.uint32) << 16).view(np.float32) if out_dt == "bf16" else C0
+    Y, S = oracle.brgemm(M, N, K, batch, A, B, bias, C0=c0.astype(np.float64).reshape(M, N) if beta else None,
+                         in_dtype=oracle.BF16, epilogue=oracle.EPI_BIAS_RELU if epi else oracle.EPI_NONE, beta=float(beta),
+                         stride_a=sa, stride_b=sb,
+                         layout_a=oracle.BLOCKED32 if layout == "blocked" else oracle.ROW,
+                         layout_b=oracle.BLOCKED32 if layout == "blocked" else oracle.TRANSPOSED)
+    if integer and out_dt == "f32":
+        assert np.array_equal(got, Y), plan.kernel_name
+    else:
+        tol = TOL_REL_SMAX * S.max() + (TOL_BF16_REL * np.abs(Y) if out_dt == "bf16" else 0.0)
+        assert np.all(np.abs(got - Y) <= tol), plan.kernel_name
+    return plan
+
+
+@pytest.mark.parametrize("beta", [0, 1])
+def test_listing1_vnni_packed_brgemm_runs_as_printed(beta):
+    """The paper's running example (Listing 1): a batch of four 32x32 A tiles and four VNNI-packed 32x192 B tiles
+    reduced into one 32x192 C, consumed in the packed layout with no unpacking pass."""
+    plan = _run_layout(32, 192, 32, 4, "f32", False, beta, "blocked")
+    assert "_br4" in plan.kernel_name and "_bvnni" in plan.kernel_name and "_ablk" in plan.kernel_name
+    _run_layout(64, 64, 64, 2, "f32", False, beta, "blocked")          # the appendix BF16 kernel's shape
+
+
+@pytest.mark.parametrize("mode", ["single", "pair"])
+@pytest.mark.parametrize("layout", ["blocked", "transposed"])
+@pytest.mark.parametrize("out_dt,epi,beta", [("f32", False, 0), ("f32", True, 1), ("bf16", True, 0)])
+def test_brgemm_over_packed_operands(mode, layout, out_dt, epi, beta):
+    f = nk.FLAG_SINGLE_CTA if mode == "single" else nk.FLAG_CTA_PAIR
+    _run_layout(224, 320, 160, 5, out_dt, epi, beta, layout, pad_a=64, pad_b=32, flags=f)      # gaps between the items
+    _run_layout(288, 256, 96, 3, out_dt, epi, beta, layout, flags=f | nk.flag_splitk(2), integer=False, seed=3)
+    _run_layout(512, 512, 256, 4, out_dt, epi, beta, layout, integer=False, seed=4)            # plan on auto

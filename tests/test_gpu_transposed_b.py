@@ -118,6 +118,6 @@ def test_bt_rejects_what_it_cannot_do():
     with pytest.raises(nk.NkError):
         nk.Plan(64, 64, 72, in_dtype=nk.BF16, out_dtype=nk.F32, layout_b=nk.TRANSPOSED)     # K not a multiple of 16
     with pytest.raises(nk.NkError):
-        nk.Plan(64, 64, 64, in_dtype=nk.BF16, out_dtype=nk.F32, layout_b=nk.TRANSPOSED, batch=2)
+        nk.Plan(64, 64, 64, in_dtype=nk.S8, out_dtype=nk.S32, layout_b=nk.TRANSPOSED, batch=2)    # no batch with 8-bit operands
     with pytest.raises(nk.NkError):
         nk.Plan(64, 64, 64, in_dtype=nk.BF16, out_dtype=nk.F32, layout_a=nk.TRANSPOSED)
