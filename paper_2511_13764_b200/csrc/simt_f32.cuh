@@ -195,7 +195,7 @@ namespace nk {
 // A CTA of 128 threads owns 512 consecutive columns and a chunk of K: it parks its slice of A
 // in shared memory once (transposed, so the MR values of one k are read with broadcast
 // 128-bit loads), then streams B with no barrier in the loop: every thread keeps 8 independent
-// 16-byte loads in flight (row segments of 512 B per warp) and holds an MR x 4 block of C in
+// 16-byte loads in flight (row segments of 512 B per warp; a rolling window) and holds an MR x 4 block of C in
 // registers (Algorithm 1's resident accumulator), as MR / 2 x 4 register pairs along M that are
 // updated with packed FMAs (fma.rn.f32x2: the pair of A values comes straight from shared
 // memory, the B value is copied into both halves), which halves the issue slots the 16 FMAs
@@ -217,7 +217,7 @@ struct SkinnyParams {
 };
 
 template <int MR>
-__global__ void __launch_bounds__(SKINNY_THREADS, MR == 16 ? 3 : 2) simt_f32_skinny_kernel(const SkinnyParams p) {
+__global__ void __launch_bounds__(SKINNY_THREADS, MR == 16 ? 4 : 2) simt_f32_skinny_kernel(const SkinnyParams p) {
     __shared__ __align__(16) float As[SKINNY_A_FLOATS];   // As[kk][MR]
     const int t = threadIdx.x;
     const int n = blockIdx.x * SKINNY_COLS + t * 4;
@@ -244,25 +244,24 @@ __global__ void __launch_bounds__(SKINNY_THREADS, MR == 16 ? 3 : 2) simt_f32_ski
 
     const bool col_ok = n < p.N;
     const float* bptr = p.B + static_cast<size_t>(k0) * p.N + (col_ok ? n : 0);
-    float4 bnext[8];
-    auto load_group = [&](int kk) {
-#pragma unroll
-        for (int i = 0; i < 8; ++i)
-            bnext[i] = (col_ok && kk + i < klen)
-                           ? __ldcs(reinterpret_cast<const float4*>(bptr + static_cast<size_t>(kk + i) * p.N))
-                           : make_float4(0.f, 0.f, 0.f, 0.f);
+    // a rolling window of 8 rows of B per thread: row kk + 8 + i is requested as soon as row kk + i has
+    // been taken out of its register, so eight 16-byte loads stay in flight with one set of registers
+    // (a second, "next group" set cost 32 registers and a CTA per SM)
+    float4 b[8];
+    auto load_row = [&](int k) {
+        return (col_ok && k < klen) ? __ldcs(reinterpret_cast<const float4*>(bptr + static_cast<size_t>(k) * p.N))
+                                    : make_float4(0.f, 0.f, 0.f, 0.f);
     };
-    load_group(0);
-    for (int kk = 0; kk < klen; kk += 8) {
-        float4 b[8];
 #pragma unroll
-        for (int i = 0; i < 8; ++i) b[i] = bnext[i];
-        if (kk + 8 < klen) load_group(kk + 8);
+    for (int i = 0; i < 8; ++i) b[i] = load_row(i);
+    for (int kk = 0; kk < klen; kk += 8) {
 #pragma unroll
         for (int i = 0; i < 8; ++i) {
+            const float4 cur = b[i];
+            b[i] = load_row(kk + 8 + i);
             const float* arow = &As[(kk + i) * MR];
-            const float2 bx = make_float2(b[i].x, b[i].x), by = make_float2(b[i].y, b[i].y);
-            const float2 bz = make_float2(b[i].z, b[i].z), bw = make_float2(b[i].w, b[i].w);
+            const float2 bx = make_float2(cur.x, cur.x), by = make_float2(cur.y, cur.y);
+            const float2 bz = make_float2(cur.z, cur.z), bw = make_float2(cur.w, cur.w);
 #pragma unroll
             for (int mq = 0; mq < MR; mq += 4) {
                 const float4 a = *reinterpret_cast<const float4*>(arow + mq);

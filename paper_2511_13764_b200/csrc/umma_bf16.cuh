@@ -612,7 +612,7 @@ __device__ __forceinline__ bool umma_cluster_epilogue(const UmmaParams& p, const
             bulk_commit();
         }
     }
-    if (lane == 0) bulk_wait_all();
+    if (lane == 0) bulk_wait_read<0>();
     __syncwarp();
     return true;
 }
@@ -941,7 +941,7 @@ umma_bf16_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_consta
                                               gen_base + (quarter * 2 + 1) * (BN * 64), mb * UMMA_BM + quarter * 32, nb * BN, gemm,
                                               lane, p.kb_total <= 0, bias_sm, BN / 64, BN / 32);
                 }
-                if (lane == 0) bulk_wait_all();
+                if (lane == 0) bulk_wait_read<0>();
                 __syncwarp();
             }
         } else {
@@ -998,9 +998,9 @@ umma_bf16_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_consta
                 tc_fence_before_sync();
                 mbar_arrive(tempty_bar(acc));
             }
-            // the TMA stores of this warp must have read their staging buffers (and, to be safe, be
-            // complete) before the CTA's shared memory goes away
-            if (lane == 0) bulk_wait_all();
+            // the TMA stores of this warp must have read their staging buffers before the CTA's shared
+            // memory goes away; their global writes are part of the grid's work and complete with it
+            if (lane == 0) bulk_wait_read<0>();
             __syncwarp();
         }
     }

@@ -367,7 +367,7 @@ umma_bf16_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_c
                                               mb * BM2 + static_cast<int>(rank) * UMMA_BM + quarter * 32, nb * BN, gemm, lane,
                                               kb1 <= kb0, bias_sm, BN / 64, BN / 32);
                 }
-                if (lane == 0) bulk_wait_all();
+                if (lane == 0) bulk_wait_read<0>();
                 __syncwarp();
             }
         } else {
@@ -426,7 +426,7 @@ umma_bf16_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_c
                 tc_fence_before_sync();
                 mbar_arrive_cluster_cta_release(map_to_cta(tempty_bar(acc), leader));
             }
-            if (lane == 0) bulk_wait_all();   // this warp's TMA stores are done with the staging buffers
+            if (lane == 0) bulk_wait_read<0>();   // this warp's TMA stores are done with the staging buffers
             __syncwarp();
         }
     }
