@@ -17,6 +17,7 @@
 #include "simt_f32.cuh"
 #include "umma_bf16.cuh"
 #include "umma_bf16_pair.cuh"
+#include "umma_swap.cuh"
 
 namespace nk {
 
@@ -24,7 +25,7 @@ namespace nk {
 // loads the library).  Kernels receive its device address as a parameter.
 __device__ unsigned int g_status_word[4];
 
-enum Variant { V_NAIVE = 0, V_SIMT = 1, V_UMMA = 2, V_SKINNY = 3, V_SPLIT3 = 4, V_SMALL = 5 };
+enum Variant { V_NAIVE = 0, V_SIMT = 1, V_UMMA = 2, V_SKINNY = 3, V_SPLIT3 = 4, V_SMALL = 5, V_SWAP = 6 };
 
 typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*,
                                   const cuuint64_t*, const cuuint64_t*, const cuuint32_t*,
@@ -39,6 +40,7 @@ struct nk_gemm_s {
     int sm_count;
     // UMMA
     int bn, stages, splits, group_m;
+    int swap_mp;           // swap-AB skinny kernel: M rounded up to 16, 32 or 64
     bool serpentine;       // raster: odd groups of M tiles sweep N backwards
     bool pair;             // CTA pairs: 256-row tiles, cta_group::2
     int max_pairs;         // co-resident clusters of 2 for the chosen pair kernel
@@ -146,6 +148,20 @@ static uint32_t make_idesc(int m, int n, bool b_n_major, bool f16, bool s8 = fal
     d |= (b_n_major ? 1u : 0u) << 16;
     d |= static_cast<uint32_t>(n >> 3) << 17;
     d |= static_cast<uint32_t>(m >> 4) << 24;
+    return d;
+}
+
+// The same for the swapped-operand skinny kernel: the MMA's A operand is the GEMM's B tile (MN-major
+// when B is row-major [K][N], bit 15; K-major when B is stored transposed), its B operand the GEMM's
+// A tile (K-major), M = 128, N = the padded row count of the GEMM's A.
+static uint32_t make_idesc_swap(int n, bool a_mn_major, bool f16) {
+    uint32_t d = 0;
+    d |= 1u << 4;
+    d |= (f16 ? 0u : 1u) << 7;
+    d |= (f16 ? 0u : 1u) << 10;
+    d |= (a_mn_major ? 1u : 0u) << 15;
+    d |= static_cast<uint32_t>(n >> 3) << 17;
+    d |= static_cast<uint32_t>(UMMA_BM >> 4) << 24;
     return d;
 }
 
@@ -389,7 +405,7 @@ static nk_status_t encode_maps(nk_gemm_s* p, const void* A, const void* B) {
         cuuint64_t dims[3] = {static_cast<cuuint64_t>(d.K), static_cast<cuuint64_t>(d.M),
                               static_cast<cuuint64_t>(p->batch * p->gemms)};
         cuuint64_t strides[2] = {static_cast<cuuint64_t>(d.K) * esz, static_cast<cuuint64_t>(p->stride_a) * esz};
-        cuuint32_t box[3] = {static_cast<cuuint32_t>(kblock(d)), UMMA_BM, 1};   // 128 bytes of k per row
+        cuuint32_t box[3] = {static_cast<cuuint32_t>(kblock(d)), static_cast<cuuint32_t>(p->variant == V_SWAP ? p->swap_mp : UMMA_BM), 1};   // 128 bytes of k per row
         cuuint32_t es[3] = {1, 1, 1};
         r = p->encode(&p->tmap_a, half_type, 3, const_cast<void*>(A), dims, strides,
                       box, es, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
@@ -402,7 +418,7 @@ static nk_status_t encode_maps(nk_gemm_s* p, const void* A, const void* B) {
     if (p->b_kmajor) {
         // B stored transposed, Bt[batch][N][K] (K contiguous): (k, n, item), one box of 128 bytes of k by
         // the columns a CTA covers, K-major in shared memory exactly like A's tile
-        const int cols = p->pair ? p->bn / 2 : p->bn;
+        const int cols = p->variant == V_SWAP ? 128 : p->pair ? p->bn / 2 : p->bn;
         cuuint64_t dims[3] = {static_cast<cuuint64_t>(d.K), static_cast<cuuint64_t>(d.N),
                               static_cast<cuuint64_t>(p->batch * p->gemms)};
         cuuint64_t strides[2] = {static_cast<cuuint64_t>(d.K) * esz, static_cast<cuuint64_t>(p->stride_b) * esz};
@@ -420,7 +436,7 @@ static nk_status_t encode_maps(nk_gemm_s* p, const void* A, const void* B) {
         // (n within a 64-column slab, k, slab): one box brings all the slabs of a stage, each
         // as 64 k-rows of 128 B.  Otherwise 64 (n) x 64 (k) boxes, one per slab.
         p->b_3d = d.N % 64 == 0;
-        const int slabs = (p->pair ? p->bn / 2 : p->bn) / 64;
+        const int slabs = p->variant == V_SWAP ? 2 : (p->pair ? p->bn / 2 : p->bn) / 64;
         if (p->b_3d) {
             // (n within slab, k, slab, item)
             cuuint64_t dims[4] = {64, static_cast<cuuint64_t>(d.K), static_cast<cuuint64_t>(d.N / 64),
@@ -910,6 +926,48 @@ nk_status_t nk_gemm_create(const nk_gemm_desc_t* desc, nk_gemm_t* out) {
         snprintf(p->name, sizeof(p->name), "simt_f32%s_%dx%dx16_splitk%d",
                  (p->simt_tile == 128 && !(d.flags & NK_FLAG_SCALAR_FMA)) ? "x2" : "", p->simt_tile, p->simt_tile,
                  p->splits);
+    } else if (is16(d.in_dtype) && d.M <= 64 && force == NK_FLAG_KERNEL_AUTO && nbatch == 1 && d.layout_a == NK_ROW_MAJOR &&
+               (d.layout_b == NK_ROW_MAJOR || d.layout_b == NK_TRANSPOSED) && d.layout_c == NK_ROW_MAJOR &&
+               !(d.flags & (NK_FLAG_SINGLE_CTA | NK_FLAG_CTA_PAIR | (0xFu << NK_FLAG_TILE_N_SHIFT)))) {
+        // few rows of A: the operands swap roles, B's columns become the rows of the MMA (see umma_swap_kernel)
+        p->variant = V_SWAP;
+        void* fn = nullptr;
+        cudaDriverEntryPointQueryResult q;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &q) != cudaSuccess ||
+            q != cudaDriverEntryPointSuccess || !fn) {
+            delete p;
+            return NK_ERR_CUDA;
+        }
+        p->encode = reinterpret_cast<EncodeTiledFn>(fn);
+        p->swap_mp = d.M <= 16 ? 16 : d.M <= 32 ? 32 : 64;
+        if (allow_smem(umma_swap_kernel<16, false>, swap_smem_bytes(16, swap_stages(16))) != cudaSuccess ||
+            allow_smem(umma_swap_kernel<16, true>, swap_smem_bytes(16, swap_stages(16))) != cudaSuccess ||
+            allow_smem(umma_swap_kernel<32, false>, swap_smem_bytes(32, swap_stages(32))) != cudaSuccess ||
+            allow_smem(umma_swap_kernel<32, true>, swap_smem_bytes(32, swap_stages(32))) != cudaSuccess ||
+            allow_smem(umma_swap_kernel<64, false>, swap_smem_bytes(64, swap_stages(64))) != cudaSuccess ||
+            allow_smem(umma_swap_kernel<64, true>, swap_smem_bytes(64, swap_stages(64))) != cudaSuccess) {
+            cudaGetLastError();
+            delete p;
+            return NK_ERR_CUDA;
+        }
+        p->b_kmajor = d.layout_b == NK_TRANSPOSED;
+        // K splits: enough CTAs to pull B from every SM; they meet in one CTA of a cluster (at most 8
+        // CTAs; 4 with 64 rows, whose accumulators must fit the stage ring of the receiving CTA)
+        const int tiles_n = ceil_div(d.N, 128);
+        const int kb_total = ceil_div(d.K, UMMA_BK);
+        const int forced_s = (d.flags >> NK_FLAG_SPLITK_SHIFT) & 0xFF;
+        const int max_s = p->swap_mp == 64 ? 4 : 8;
+        int splits = forced_s > 0 ? forced_s : p->sm_count / tiles_n;
+        if (splits > max_s && !(forced_s > 0 && (d.flags & NK_FLAG_SEPARATE_REDUCE))) splits = max_s;
+        if (splits > kb_total) splits = kb_total;
+        if (splits < 1) splits = 1;
+        const int per = ceil_div(kb_total, splits);
+        p->splits = ceil_div(kb_total, per);
+        p->cluster_reduce = p->splits > 1 && p->splits <= max_s && !(d.flags & NK_FLAG_SEPARATE_REDUCE);
+        p->ws_partial_bytes = (p->splits > 1 && !p->cluster_reduce) ? static_cast<size_t>(p->splits) * d.M * d.N * 4 : 0;
+        p->launches = (p->splits > 1 && !p->cluster_reduce) ? 2 : 1;
+        snprintf(p->name, sizeof(p->name), "umma_swap_128x%dx64_s%d_splitk%d%s%s", p->swap_mp, swap_stages(p->swap_mp), p->splits,
+                 p->cluster_reduce ? "_cluster" : "", p->b_kmajor ? "_bt" : "");
     } else {
         p->variant = V_UMMA;
         void* fn = nullptr;
@@ -1115,6 +1173,50 @@ nk_status_t nk_gemm_run(nk_gemm_t p, const void* A, const void* B, const void* b
                          static_cast<float*>(C), partial};
         e = launch_simt(p, sp, st);
         if (e != cudaSuccess) { set_err(p, "simt launch", e); return NK_ERR_CUDA; }
+    } else if (p->variant == V_SWAP) {
+        nk_status_t s = encode_maps(p, A, B);
+        if (s != NK_OK) return s;
+        SwapParams sp;
+        memset(&sp, 0, sizeof(sp));
+        sp.M = static_cast<int>(d.M); sp.N = static_cast<int>(d.N); sp.K = static_cast<int>(d.K);
+        sp.tiles_n = ceil_div(d.N, 128);
+        sp.splits = p->splits;
+        sp.kb_total = ceil_div(d.K, UMMA_BK);
+        sp.kb_per_split = ceil_div(sp.kb_total, p->splits);
+        sp.cluster = p->cluster_reduce ? 1 : 0;
+        sp.b_3d = p->b_3d ? 1 : 0;
+        sp.b_kmajor = p->b_kmajor ? 1 : 0;
+        sp.epilogue = d.epilogue;
+        sp.out_bf16 = is16(d.out_dtype);
+        sp.f16 = d.in_dtype == NK_F16;
+        sp.bias_f32 = 0;
+        sp.beta = d.beta;
+        sp.idesc = make_idesc_swap(p->swap_mp, !p->b_kmajor, d.in_dtype == NK_F16);
+        sp.bias = bias;
+        sp.C = C;
+        sp.partial = partial;
+        sp.status = p->status_dev;
+        cudaLaunchConfig_t cfg;
+        memset(&cfg, 0, sizeof(cfg));
+        cfg.gridDim = dim3(static_cast<unsigned>(sp.tiles_n * p->splits));
+        cfg.blockDim = dim3(192);
+        cfg.dynamicSmemBytes = static_cast<size_t>(swap_smem_bytes(p->swap_mp, swap_stages(p->swap_mp)));
+        cfg.stream = st;
+        cudaLaunchAttribute attr;
+        attr.id = cudaLaunchAttributeClusterDimension;
+        attr.val.clusterDim.x = static_cast<unsigned>(p->cluster_reduce ? p->splits : 1);
+        attr.val.clusterDim.y = 1;
+        attr.val.clusterDim.z = 1;
+        cfg.attrs = &attr;
+        cfg.numAttrs = 1;
+        const bool cl = p->cluster_reduce;
+        if (p->swap_mp == 16) e = cl ? cudaLaunchKernelEx(&cfg, umma_swap_kernel<16, true>, p->tmap_a, p->tmap_b, sp)
+                                     : cudaLaunchKernelEx(&cfg, umma_swap_kernel<16, false>, p->tmap_a, p->tmap_b, sp);
+        else if (p->swap_mp == 32) e = cl ? cudaLaunchKernelEx(&cfg, umma_swap_kernel<32, true>, p->tmap_a, p->tmap_b, sp)
+                                          : cudaLaunchKernelEx(&cfg, umma_swap_kernel<32, false>, p->tmap_a, p->tmap_b, sp);
+        else e = cl ? cudaLaunchKernelEx(&cfg, umma_swap_kernel<64, true>, p->tmap_a, p->tmap_b, sp)
+                    : cudaLaunchKernelEx(&cfg, umma_swap_kernel<64, false>, p->tmap_a, p->tmap_b, sp);
+        if (e != cudaSuccess) { set_err(p, "swap launch", e); return NK_ERR_CUDA; }
     } else {
         const void* Buse = B;
         if (p->b_repack) {

@@ -398,3 +398,49 @@ def test_run_host_pipelined_chunks(out_dtype, epi, layout, N):
         else:
             got = (hC.numpy().view(np.uint16).astype(np.uint32) << 16).view(np.float32).astype(np.float64)
         check_against_oracle(w, got.reshape(M, N), A, B, bias, rows=rows)
+
+
+# ---------------------------------------------------------------- swap-AB skinny kernel (M <= 64, 16-bit operands)
+SWAP_SHAPES = [(16, 1024, 1024), (1, 128, 64), (17, 200, 136), (33, 4096, 512), (64, 328, 1096), (5, 72, 2048),
+               (48, 1032, 264)]
+
+
+@pytest.mark.parametrize("shape", SWAP_SHAPES)
+@pytest.mark.parametrize("out_dtype,epi", [("f32", "none"), ("f32", "bias_relu"), ("bf16", "bias_relu")])
+def test_swap_ab_skinny_kernel(shape, out_dtype, epi):
+    """Few rows of A: B's columns become the rows of the MMA, C leaves transposed back.  Plan on auto (K splits
+    inside a cluster where there are several); exact on integer data, then random data; ragged M, N, K."""
+    M, N, K = shape
+    err, plan = run_and_check(W("swap", M, N, K, "bf16", out_dtype, epilogue=epi, integer=True), exact=(out_dtype == "f32"),
+                              expect_kernel="umma_swap")
+    assert plan.launches_per_run == 1 and plan.workspace_bytes == 0
+    run_and_check(W("swap", M, N, K, "bf16", out_dtype, epilogue=epi, seed=14), expect_kernel="umma_swap")
+
+
+@pytest.mark.parametrize("splits", [1, 2, 3, 4, 8])
+@pytest.mark.parametrize("M", [16, 40, 64])
+def test_swap_ab_splits_cluster_equals_reduce_kernel(splits, M):
+    """K splits of the skinny kernel: summed in split order inside one CTA of the cluster, or through FP32
+    partials and the reduce kernel: the same bits, and both within the bound of the oracle."""
+    N, K = 520, 2112
+    w = W("swapsplit", M, N, K, "bf16", "f32", epilogue="bias_relu", seed=15)
+    A, B, bias = w.make()
+    c_one, p_one = run_plan(w, A, B, bias, flags=nk.flag_splitk(splits))
+    assert "umma_swap" in p_one.kernel_name and p_one.launches_per_run == 1
+    check_against_oracle(w, c_one, A, B, bias)
+    if splits > 1 and f"splitk{splits}" in p_one.kernel_name:
+        assert "_cluster" in p_one.kernel_name
+        c_two, p_two = run_plan(w, A, B, bias, flags=nk.flag_splitk(splits) | nk.FLAG_SEPARATE_REDUCE)
+        assert "_cluster" not in p_two.kernel_name and p_two.launches_per_run == 2 and p_two.workspace_bytes > 0
+        assert np.array_equal(c_one, c_two)
+
+
+@pytest.mark.parametrize("dt", ["bf16", "f16"])
+@pytest.mark.parametrize("layout", ["row", "b_transposed"])
+def test_swap_ab_types_and_transposed_b(dt, layout):
+    w = nk_inputs.Workload("swapt", 24, 392 if layout == "row" else 400, 1040, dt, dt, layout, "bias_relu", seed=16,
+                           dist_a=("normal", 1.0), dist_b=("uniform", 1.0))
+    err, plan = run_and_check(w, expect_kernel="umma_swap")
+    assert ("_bt" in plan.kernel_name) == (layout == "b_transposed")
+    wi = nk_inputs.Workload("swapt", 24, 384, 1024, dt, "f32", layout, "none", seed=17, dist_a=INT, dist_b=INT)
+    run_and_check(wi, exact=True, expect_kernel="umma_swap")
