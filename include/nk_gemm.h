@@ -121,7 +121,11 @@ typedef enum { NK_EPI_NONE = 0, NK_EPI_BIAS_RELU = 1 } nk_epilogue_t;
                                       splits (2..8) instead of sharing its k-blocks out evenly over the pairs; 15: share
                                       them out evenly even where the plan's cost model would not */
 #define NK_FLAG_RASTER_SHIFT 28 /* bits 28..30: M tiles that sweep N together in the tile raster of the tensor-core
-                                   kernels: 0 = 8 (default), 1 = 4, 2 = 6, 3 = 12, 4 = 16, 5 = 24, 6 = 2, 7 = 32;
+                                   kernels: 0 = 8 (default), 1 = 4, 2 = 6, 3 = 12, 4 = 16, 5 = 24, 6 = 2; 7 = 8 with
+                                   every tile's K walked upwards (by default a CTA pair walks K downwards on every
+                                   other of its whole tiles, so that a wave of tiles starts on the part of the shared
+                                   operand strips that the wave before it read last and finds it in L2; FP32 sums
+                                   then differ in their last bits from the upward order, integer sums do not);
                                    bit 31: switch off the serpentine sweep (every other group sweeps N backwards) */
 #define NK_FLAG_SPLITK_SHIFT 8    /* bits 8..15: force this many K splits (0 = auto)          */
 #define NK_FLAG_TILE_N_SHIFT 16   /* bits 16..19: force tile N: 1=32 2=64 3=128 4=256 (0 = auto) */

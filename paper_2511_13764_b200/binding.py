@@ -40,7 +40,8 @@ def flag_tail_split(n: int) -> int:
 
 
 def flag_raster(group_code: int, serpentine: bool = True) -> int:
-    """Tile raster of the tensor-core kernels: group_code 0..7 = 8, 4, 6, 12, 16, 24, 2, 32 M tiles per group."""
+    """Tile raster of the tensor-core kernels: group_code 0..6 = 8, 4, 6, 12, 16, 24, 2 M tiles per group;
+    7 = 8 with K walked upwards on every tile (no K serpentine)."""
     return ((group_code & 7) << 28) | (0 if serpentine else (1 << 31))
 
 

@@ -42,6 +42,7 @@ struct nk_gemm_s {
     int bn, stages, splits, group_m;
     int swap_mp;           // swap-AB skinny kernel: M rounded up to 16, 32 or 64
     bool serpentine;       // raster: odd groups of M tiles sweep N backwards
+    bool k_serpentine;     // pair kernel: a pair's odd whole tiles walk K downwards
     bool pair;             // CTA pairs: 256-row tiles, cta_group::2
     int max_pairs;         // co-resident clusters of 2 for the chosen pair kernel
     bool b_vnni_inkernel;  // blocked B re-laid inside the GEMM kernel
@@ -290,9 +291,10 @@ static void choose_umma(nk_gemm_s* p) {
     p->group_m = 8;
     p->serpentine = false;
     {
-        // tuning override of the raster: bits 28-30 pick the group size, bit 31 switches the serpentine sweep off
-        static const int kGroups[8] = {8, 4, 6, 12, 16, 24, 2, 32};
+        // tuning override of the raster: bits 28-30 pick the group size (7: no K serpentine), bit 31 switches the serpentine sweep off
+        static const int kGroups[8] = {8, 4, 6, 12, 16, 24, 2, 8};
         p->group_m = kGroups[(d.flags >> NK_FLAG_RASTER_SHIFT) & 7u];
+        p->k_serpentine = ((d.flags >> NK_FLAG_RASTER_SHIFT) & 7u) != 7u;   // code 7: K always upwards
         p->serpentine = ((d.flags >> (NK_FLAG_RASTER_SHIFT + 3)) & 1u) == 0;
     }
     p->cluster_reduce = splits > 1 && cluster_reduce_fits(d, sms, best.pair, best.bn, splits);
@@ -1248,6 +1250,7 @@ nk_status_t nk_gemm_run(nk_gemm_t p, const void* A, const void* B, const void* b
         up.kb_per_split = ceil_div(up.kb_total, p->splits);
         up.group_m = p->group_m;
         up.serpentine = p->serpentine ? 1 : 0;
+        up.k_serpentine = (p->k_serpentine && p->pair && p->splits == 1 && p->batch == 1) ? 1 : 0;
         up.a_blocked = d.layout_a == NK_BLOCKED32;
         up.b_3d = p->b_3d ? 1 : 0;
         up.b_kmajor = p->b_kmajor ? 1 : 0;

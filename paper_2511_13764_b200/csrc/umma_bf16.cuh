@@ -58,6 +58,8 @@ struct UmmaParams {
     int kb_per_split;   // ceil(kb_total / splits)
     int group_m;        // raster: this many M tiles sweep N together
     int serpentine;     // raster: every other group of M tiles sweeps N in the opposite direction
+    int k_serpentine;   // pair kernel, no batch: every other whole tile of a pair walks K downwards, so that a
+                        // wave begins with the part of the shared strips that the wave before it read last
     int a_blocked;      // A tensor map is the 4-D blocked view
     int b_3d;           // B tensor map is the 3-D (n-in-slab, k, slab) view: one box per stage
     int b_kmajor;       // B is stored transposed, Bt[N][K]: its tiles are K-major like A's, one box per stage

@@ -176,11 +176,14 @@ umma_bf16_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_c
         uint32_t phase = 0;
         uint32_t sa = smem_base, fb = full_bar(0), lfb = lead_full0;
         bool ok = true;
-        for (int unit = pair_id; ok && unit < total_units; unit += num_pairs) {
+        int local = 0;
+        for (int unit = pair_id; ok && unit < total_units; unit += num_pairs, ++local) {
             int tile, split, gemm, kb0, kb1, tail;
             if (!decode(unit, tile, split, gemm, kb0, kb1, tail)) continue;
             int mb, nb;
             umma_tile_coords(p, tile, mb, nb);
+            // K order of a whole tile: downwards on a pair's odd tiles when the plan asks for it
+            const bool k_down = p.k_serpentine && (local & 1) && kb0 == 0 && kb1 == p.kb_total;
             const int row0 = mb * BM2 + static_cast<int>(rank) * UMMA_BM;
             const int col0 = nb * BN + static_cast<int>(rank) * HALF;
             int item = kb0 == 0 ? 0 : div_small(kb0, p.kb_per_item);
@@ -188,6 +191,8 @@ umma_bf16_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_c
             item += gemm;   // independent batch: the unit's own (A, B) pair
             int ia, ib;
             umma_item_pair(p, item, ia, ib);
+            if (k_down) kbl = kb1 - 1;
+            const int kstep = k_down ? -1 : 1;
             for (int kb = kb0; kb < kb1; ++kb) {
                 const int kx = kbl * (KIND != 0 ? 2 * UMMA_BK : UMMA_BK);   // 128 bytes of k per stage row
                 if (!mbar_wait(empty_bar(stage), phase ^ 1u, abort_flag)) {
@@ -221,7 +226,8 @@ umma_bf16_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_c
                         }
                     }
                 }
-                if (++kbl == p.kb_per_item) { kbl = 0; ++item; umma_item_pair(p, item, ia, ib); }
+                kbl += kstep;
+                if (kbl == p.kb_per_item) { kbl = 0; ++item; umma_item_pair(p, item, ia, ib); }
                 __syncwarp();
                 sa += STAGE;
                 fb += 8;

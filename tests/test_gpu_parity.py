@@ -347,6 +347,29 @@ def test_pair_stream_k_shares_the_last_wave(shape, out_dtype, epi):
     check_against_oracle(w, c_sk, A, B, bias, rows=rows)
 
 
+@pytest.mark.parametrize("layout,K", [("row", 680), ("blocked32", 672)])
+def test_pair_k_serpentine_order(layout, K):
+    """Three and a half tiles per CTA pair: every other whole tile of a pair is reduced with K walked downwards
+    (operand strips shared with the wave before are met where that wave left them in L2).  The order of the sum
+    is all that changes: integer data give the oracle's result bit for bit and the same bits as the plan that
+    walks K upwards everywhere; random data stay under the acceptance bound, ragged K tail included."""
+    M, N = 4096, 4096
+    f = nk.FLAG_CTA_PAIR | nk.flag_tile_n(4) | nk.flag_splitk(1) | nk.FLAG_NO_TAIL_SPLIT
+    rows = nk_inputs.stratified_rows(9, M, 48)
+    w = W("kserp", M, N, K, "bf16", "f32", layout, integer=True, seed=5)
+    A, B, bias = w.make()
+    c_down, plan = run_plan(w, A, B, bias, flags=f)
+    check_against_oracle(w, c_down, A, B, bias, rows=rows, exact=True)
+    c_up, _ = run_plan(w, A, B, bias, flags=f | nk.flag_raster(7))
+    assert np.array_equal(c_down, c_up)
+    w = W("kserp", M, N, K, "bf16", "f32", layout, seed=6)
+    A, B, bias = w.make()
+    c_down, _ = run_plan(w, A, B, bias, plan=plan)
+    check_against_oracle(w, c_down, A, B, bias, rows=rows)
+    c_up, _ = run_plan(w, A, B, bias, flags=f | nk.flag_raster(7))
+    assert not np.array_equal(c_down, c_up)     # the two orders round differently somewhere: both orders really ran
+
+
 @pytest.mark.parametrize("out_dtype,bn", [("f32", 4), ("bf16", 4), ("bf16", 3)])
 def test_pair_tail_units_follow_tma_stored_tiles(out_dtype, bn):
     """A pair that goes from a whole tile (stored by TMA from its staging tiles) straight to a tail split
