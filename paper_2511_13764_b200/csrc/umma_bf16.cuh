@@ -96,10 +96,11 @@ __host__ __device__ constexpr int umma_b_stage_bytes(int BN) { return BN * UMMA_
 __host__ __device__ constexpr int umma_stage_bytes(int BN) {
     return UMMA_A_STAGE_BYTES + umma_b_stage_bytes(BN);
 }
+constexpr uint32_t UMMA_RECV_BAR_OFFSET = 264;    // in the barrier block, after the raw-block barriers: one per epilogue warp of a cluster split-K CTA
 constexpr uint32_t UMMA_RAW_BAR_OFFSET = 200;     // in the barrier block: after full/empty/tmem barriers (<= 168 B) and the cluster barrier (192)
 constexpr int UMMA_EPI_STAGING = 4 * 2 * 4096;   // two 32 x 32 FP32 chunks per epilogue warp (1024-byte aligned: TMA store source)
 __host__ __device__ constexpr int umma_smem_bytes(int BN, int stages) {
-    return stages * umma_stage_bytes(BN) + 1024 /*alignment slack*/ + UMMA_EPI_STAGING + 320 /*barriers*/;
+    return stages * umma_stage_bytes(BN) + 1024 /*alignment slack*/ + UMMA_EPI_STAGING + 384 /*barriers*/;
 }
 // cluster split-K: one 4 KB slot per (32 x 32 piece this CTA owns, split it comes from); the pieces of
 // a CTA's 128 x BN accumulator are shared out over the splits, so a CTA's slots never exceed one
@@ -479,16 +480,20 @@ __device__ __forceinline__ void umma_epilogue_oneshot(const UmmaParams& p, const
 // belongs to split u % S; the other splits write theirs into slot (u / S) * S + source split of
 // the owner's stage ring (idle by then), the owner's own contribution stays in tensor memory.
 //   barrier  every CTA of the cluster has finished its K loop: the rings may be overwritten
-//   send     tcgen05.ld -> remote shared-memory stores straight from the registers, a warp writing
-//            512 contiguous bytes per instruction (16-byte group g of row t at g * 512 + (t ^ g) * 16:
-//            conflict-free when the owner reads it back).  The SM-to-SM path moves 16-23 bytes per
+//   send     tcgen05.ld -> asynchronous remote shared-memory stores straight from the registers, a
+//            warp writing 512 contiguous bytes per instruction (16-byte group g of row t at
+//            g * 512 + (t ^ g) * 16: conflict-free when the owner reads it back), every store counted
+//            in on the receiving warp's mbarrier `recv_bar`.  The SM-to-SM path moves 16-23 bytes per
 //            clock per CTA whatever the method (bulk copies, remote loads, remote stores; measured),
 //            so what counts is that all the pieces are in flight at once and nothing waits in between
-//   barrier  (release / acquire) every piece has landed everywhere
+//   wait     each warp waits on its own mbarrier for the pieces it owns (armed with their byte
+//            count before the first barrier); no second barrier of the whole cluster
 //   reduce   every owned piece is summed in split order (the result does not depend on timing;
 //            INT32 sums are added as integers), gets the epilogue, and all the owned chunks leave
 //            as one batch of TMA stores staged behind the slots
-// Every thread of the cluster passes both barriers, also in a CTA where a wait gave up (`ok` false).
+// Every thread of the cluster passes the barrier, also in a CTA where a wait gave up (`ok` false);
+// the warps that then wait for its pieces give up after their bounded wait.  A CTA leaves only
+// after all its warps have what they wait for, so nothing is written into an exited CTA.
 // `bias_sm`: the tile's bias slice as FP32 in shared memory (umma_park_bias), or null.
 template <int BN>
 __host__ __device__ constexpr uint32_t umma_cluster_slot_bytes() { return BN * 512u; }
@@ -502,10 +507,17 @@ __device__ __forceinline__ bool umma_cluster_epilogue(const UmmaParams& p, const
                                                       uint32_t ring, uint8_t* ring_gen, uint8_t* staging,
                                                       const float* bias_sm, int quarter, int half, int lane, uint32_t S,
                                                       uint32_t split, uint32_t rank0, uint32_t rank_step, int row_cta0,
-                                                      int col_tile0, int gemm, bool ok) {
+                                                      int col_tile0, int gemm, bool ok, uint32_t recv_bar0,
+                                                      volatile uint32_t* abort_flag) {
     constexpr uint32_t NC = BN / 32, HC = NC / 2;
     const uint32_t lane_tmem = static_cast<uint32_t>(quarter * 32) << 16;
     const uint32_t c_lo = half * HC, c_hi = c_lo + HC;
+    const uint32_t my_bar = recv_bar0 + 8u * (quarter * 2 + half);
+    // pieces of this warp's chunk range that this CTA owns: each brings 4 KB from every other split
+    uint32_t owned = 0;
+#pragma unroll
+    for (uint32_t c = 0; c < HC; ++c) owned += ((quarter * NC + c_lo + c) & (S - 1u)) == split ? 1u : 0u;
+    if (lane == 0) mbar_arrive_expect_tx(my_bar, owned * (S - 1u) * 4096u);
     cluster_arrive();
     cluster_wait();
     if (ok) {
@@ -516,16 +528,20 @@ __device__ __forceinline__ bool umma_cluster_epilogue(const UmmaParams& p, const
             uint32_t v[32];
             tmem_ld_32x32(tmem_base + c * 32 + lane_tmem, v);
             tmem_ld_wait();
-            const uint32_t dst = map_to_cta(ring + ((u & ~(S - 1u)) + split) * 4096u, rank0 + owner * rank_step);
+            const uint32_t orank = rank0 + owner * rank_step;
+            const uint32_t dst = map_to_cta(ring + ((u & ~(S - 1u)) + split) * 4096u, orank);
+            const uint32_t obar = map_to_cta(my_bar, orank);     // the same (quarter, half) warp of the owner
 #pragma unroll
             for (int g = 0; g < 8; ++g)
-                st_cluster_v4(dst + g * 512 + ((lane ^ g) << 4), v[4 * g], v[4 * g + 1], v[4 * g + 2], v[4 * g + 3]);
+                st_async_cluster_v4(dst + g * 512 + ((lane ^ g) << 4), v[4 * g], v[4 * g + 1], v[4 * g + 2], v[4 * g + 3], obar);
         }
     }
-    cluster_arrive();
-    cluster_wait();
     if (!ok) return false;
     const bool batched = p.tma_store != 0;
+    // the pieces this warp will reduce have landed: its own range, and without batched stores (set 0
+    // reduces every chunk of its rows) the other half's range as well
+    if (!mbar_wait_cluster(my_bar, 0u, abort_flag)) return false;
+    if (!batched && !mbar_wait_cluster(recv_bar0 + 8u * (quarter * 2 + (half ^ 1)), 0u, abort_flag)) return false;
     if (!batched && half != 0) return true;
     const uint32_t r_lo = batched ? c_lo : 0u, r_hi = batched ? c_hi : NC;
     // store tiles of the owned chunks: behind the receive slots, max(1, HC / S) per warp
@@ -536,8 +552,65 @@ __device__ __forceinline__ bool umma_cluster_epilogue(const UmmaParams& p, const
     const int row0 = row_cta0 + quarter * 32;
     uint32_t ntiles = 0;
     int parity = 0;
+    bool reduced = false;
+    if constexpr (HC >= 4) {
+        if (batched && S == 2u) {
+            // Two splits, two owned chunks per warp (c_lo + split and the next but one; quarter * NC and
+            // c_lo are even): both are reduced side by side, so that the loads of one hide behind the
+            // arithmetic of the other.  With two terms the order of the sum does not matter (a + b is
+            // b + a bit for bit), so the result is the one the general loop below gives.
+            reduced = true;
+            const uint32_t ca = c_lo + split, cb = ca + 2u;
+            const int cola = col_tile0 + static_cast<int>(ca) * 32, colb = cola + 64;
+            if (row0 < p.M && cola < p.N) {
+                const bool two = colb < p.N;
+                uint32_t v0[32], v1[32];
+                tmem_ld_32x32(tmem_base + ca * 32 + lane_tmem, v0);
+                if (two) tmem_ld_32x32(tmem_base + cb * 32 + lane_tmem, v1);
+                tmem_ld_wait();
+                const uint8_t* sa = ring_gen + (((quarter * NC + ca) & ~1u) + (split ^ 1u)) * 4096u;   // the other split's piece
+                const uint8_t* sb = sa + 2u * 4096u;
+#pragma unroll
+                for (int g = 0; g < 8; ++g) {
+                    const uint32_t off = g * 512 + ((lane ^ g) << 4);
+                    const uint4 ta = *reinterpret_cast<const uint4*>(sa + off);
+                    if (p.acc_s32) {
+                        v0[4 * g] += ta.x; v0[4 * g + 1] += ta.y; v0[4 * g + 2] += ta.z; v0[4 * g + 3] += ta.w;
+                    } else {
+                        add2_f32(v0[4 * g], v0[4 * g + 1], ta.x, ta.y);
+                        add2_f32(v0[4 * g + 2], v0[4 * g + 3], ta.z, ta.w);
+                    }
+                    if (two) {
+                        const uint4 tb = *reinterpret_cast<const uint4*>(sb + off);
+                        if (p.acc_s32) {
+                            v1[4 * g] += tb.x; v1[4 * g + 1] += tb.y; v1[4 * g + 2] += tb.z; v1[4 * g + 3] += tb.w;
+                        } else {
+                            add2_f32(v1[4 * g], v1[4 * g + 1], tb.x, tb.y);
+                            add2_f32(v1[4 * g + 2], v1[4 * g + 3], tb.z, tb.w);
+                        }
+                    }
+                }
+                if (p.dequant) {
+#pragma unroll
+                    for (int i = 0; i < 32; ++i) v0[i] = __float_as_uint(__int2float_rn(static_cast<int>(v0[i])) * p.scale);
+                }
+                umma_chunk_bias_relu(p, v0, cola, bias_sm ? bias_sm + ca * 32 : nullptr);
+                umma_write_store_tile(p, v0, lane, tiles);
+                ntiles = 1;
+                if (two) {
+                    if (p.dequant) {
+#pragma unroll
+                        for (int i = 0; i < 32; ++i) v1[i] = __float_as_uint(__int2float_rn(static_cast<int>(v1[i])) * p.scale);
+                    }
+                    umma_chunk_bias_relu(p, v1, colb, bias_sm ? bias_sm + cb * 32 : nullptr);
+                    umma_write_store_tile(p, v1, lane, tiles + tile_bytes);
+                    ntiles = 2;
+                }
+            }
+        }
+    }
 #pragma unroll 1
-    for (uint32_t c = r_lo; c < r_hi; ++c) {
+    for (uint32_t c = r_lo; c < r_hi && !reduced; ++c) {
         const uint32_t u = quarter * NC + c;
         if ((u & (S - 1u)) != split) continue;           // warp-uniform
         const int col0 = col_tile0 + static_cast<int>(c) * 32;
@@ -684,6 +757,7 @@ umma_bf16_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_consta
     auto tfull_bar = [&](int a) { return bar_base + 8u * (2 * STAGES + a); };
     auto tempty_bar = [&](int a) { return bar_base + 8u * (2 * STAGES + 2 + a); };
     auto raw_bar = [&](int s) { return bar_base + UMMA_RAW_BAR_OFFSET + 8u * s; };   // VNNI B: blocks of stage s have landed
+    const uint32_t recv_bar0 = bar_base + UMMA_RECV_BAR_OFFSET;   // cluster split-K: pieces for epilogue warp w have landed
     uint8_t* gen_base = smem_raw + (smem_base - smem_u32(smem_raw));
     volatile uint32_t* tmem_slot =
         reinterpret_cast<volatile uint32_t*>(gen_base + STAGES * STAGE + UMMA_EPI_STAGING + 8 * (2 * STAGES + 4));
@@ -699,6 +773,7 @@ umma_bf16_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_consta
         if (lane < NB)
             mbar_init(bar_base + 8u * lane, lane < STAGES ? (B_VNNI ? 1 + 4 : 1) : lane < 2 * STAGES + 2 ? 1 : 128);
         if (B_VNNI && lane < STAGES) mbar_init(raw_bar(lane), 1);
+        if (CLUSTER_REDUCE && lane >= 24) mbar_init(recv_bar0 + 8u * (lane - 24), 1);   // one per epilogue warp
         if (lane == 0) *abort_flag = 0;
         fence_mbar_init();
         __syncwarp();
@@ -926,7 +1001,8 @@ umma_bf16_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_consta
             }
             tc_fence_after_sync();
             umma_cluster_epilogue<BN>(p, &tmap_c, tmem_base, smem_base, gen_base, staging, bias_sm, quarter, set, lane,
-                                      static_cast<uint32_t>(p.splits), cluster_ctarank(), 0u, 1u, mb * UMMA_BM, nb * BN, gemm, ok);
+                                      static_cast<uint32_t>(p.splits), cluster_ctarank(), 0u, 1u, mb * UMMA_BM, nb * BN, gemm, ok,
+                                      recv_bar0, abort_flag);
         } else if (set == 1) {
             // -------------------------------------------- second half of a one-shot epilogue
             if (one_shot && static_cast<int>(blockIdx.x) < total_units) {
@@ -1008,10 +1084,8 @@ umma_bf16_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_consta
     }
 
     if (CLUSTER_REDUCE && warp < 2) {
-        // the cluster barriers count every thread: the other roles pass both of them here, once
-        // their part of the K loop is over (the producer has seen every stage consumed)
-        cluster_arrive();
-        cluster_wait();
+        // the cluster barrier counts every thread: the other roles pass it here, once their part
+        // of the K loop is over (the producer has seen every stage consumed)
         cluster_arrive();
         cluster_wait();
     }

@@ -37,7 +37,7 @@ namespace nk {
 
 __host__ __device__ constexpr int pair_stage_bytes(int BN) { return UMMA_A_STAGE_BYTES + (BN / 2) * UMMA_BK * 2; }
 __host__ __device__ constexpr int pair_smem_bytes(int BN, int stages) {
-    return stages * pair_stage_bytes(BN) + 1024 + UMMA_EPI_STAGING + 320;
+    return stages * pair_stage_bytes(BN) + 1024 + UMMA_EPI_STAGING + 384;
 }
 
 // UmmaParams as for the single-CTA kernel, with tiles_m counted in 256-row tiles.
@@ -61,6 +61,7 @@ umma_bf16_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_c
     auto tempty_bar = [&](int a) { return bar_base + 8u * (2 * STAGES + 2 + a); };
     auto raw_bar = [&](int s) { return bar_base + UMMA_RAW_BAR_OFFSET + 8u * s; };   // VNNI B: this CTA's blocks of stage s have landed
     const uint32_t peer_ready_bar = bar_base + 192u;   // leader: the peer CTA has allocated its tensor memory
+    const uint32_t recv_bar0 = bar_base + UMMA_RECV_BAR_OFFSET;   // cluster split-K: pieces for epilogue warp w have landed
     uint8_t* gen_base = smem_raw + (smem_base - smem_u32(smem_raw));
     volatile uint32_t* tmem_slot =
         reinterpret_cast<volatile uint32_t*>(gen_base + STAGES * STAGE + UMMA_EPI_STAGING + 8 * (2 * STAGES + 4));
@@ -84,6 +85,7 @@ umma_bf16_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_c
             mbar_init(bar_base + 8u * lane, lane < STAGES ? (B_VNNI ? 1 + 8 : 1) : lane < 2 * STAGES + 2 ? 1 : 256);
         if (B_VNNI && lane < STAGES) mbar_init(raw_bar(lane), 1);
         if (lane == 31) mbar_init(peer_ready_bar, 1);
+        if (CLUSTER_REDUCE && lane >= 20 && lane < 28) mbar_init(recv_bar0 + 8u * (lane - 20), 1);   // one per epilogue warp
         if (lane == 0) *abort_flag = 0;
         fence_mbar_init();
         __syncwarp();
@@ -355,7 +357,7 @@ umma_bf16_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_c
             tc_fence_after_sync();
             umma_cluster_epilogue<BN>(p, &tmap_c, tmem_base, smem_base, gen_base, staging, bias_sm, quarter, set, lane,
                                       static_cast<uint32_t>(p.splits), crank >> 1, rank, 2u,
-                                      mb * BM2 + static_cast<int>(rank) * UMMA_BM, nb * BN, gemm, ok);
+                                      mb * BM2 + static_cast<int>(rank) * UMMA_BM, nb * BN, gemm, ok, recv_bar0, abort_flag);
         } else if (set == 1) {
             // -------------------------------------------- second half of a one-shot epilogue
             if (one_shot && pair_id < total_units) {
@@ -438,9 +440,7 @@ umma_bf16_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_c
     }
 
     if (CLUSTER_REDUCE && warp < 2) {
-        // the cluster barriers count every thread: the other roles pass both of them here
-        cluster_arrive();
-        cluster_wait();
+        // the cluster barrier counts every thread: the other roles pass it here
         cluster_arrive();
         cluster_wait();
     }
