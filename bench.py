@@ -428,6 +428,30 @@ def run_table(args):
                          library_us=None if lib_ms is None else lib_ms * 1e3))
         print(f"| {label} | {kname} | {launches} | {med * 1e3:.1f} | {tf:.1f} | {gbs:.0f} | {bound} | {frac:.3f} |"
               + (f" {lib_ms * 1e3:.1f} |" if lib_ms is not None else " |" if args.library else ""), flush=True)
+    if not args.only or any(o in "x_quantize_s8_8192x8192" for o in args.only.split(",")):
+        # the quantisation kernel of the INT8 path: an HBM stream of 4 bytes in and 1 byte out per element
+        n = 8192 * 8192
+        x = torch.rand(n, device="cuda") * 2 - 1
+        q = torch.empty(n, dtype=torch.int8, device="cuda")
+        st = torch.cuda.current_stream().cuda_stream
+        times = []
+        for i in range(args.iters + 3):
+            if flush is not None:
+                flush.fill_(1)
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record()
+            nk.quantize_s8(x, q, n, 127.0, stream=st)
+            e1.record()
+            torch.cuda.synchronize()
+            if i >= 3:
+                times.append(e0.elapsed_time(e1))
+        med = sorted(times)[len(times) // 2]
+        gbs = 5.0 * n / (med * 1e-3) / 1e9
+        frac = gbs / float(peaks["hbm_gbs"])
+        rows.append(dict(workload="x_quantize_s8_8192x8192", kernel="quantize_s8", launches=1, median_us=med * 1e3,
+                         best_us=min(times) * 1e3, tflops=0.0, gbs=gbs, bound="hbm", frac=frac, library_us=None))
+        print(f"| x_quantize_s8_8192x8192 | quantize_s8 | 1 | {med * 1e3:.1f} | 0.0 | {gbs:.0f} | hbm | {frac:.3f} |"
+              + (" |" if args.library else ""), flush=True)
     if args.json:
         with open(args.json, "w") as f:
             json.dump(rows, f, indent=1)
