@@ -17,8 +17,9 @@
 //               [k/2][n][2] blocks of a stage as they are; these warps transpose them
 //               as 32-bit words, in place, into the K-major swizzled stage (the
 //               in-kernel counterpart of the paper's software-pipelined pack step,
-//               in the opposite direction).  In a CTA that delivers a single tile they
-//               are also the second half of the epilogue (half of the columns each)
+//               in the opposite direction); warps 6-7 take the even stages, 8-9 the odd
+//               ones.  In a CTA that delivers a single tile they are also the second
+//               half of the epilogue (half of the columns each)
 //
 // Every mbarrier wait is bounded; a role that gives up raises the CTA's abort
 // flag and the device status word, the other roles fall out of their loops, and
@@ -27,8 +28,8 @@
 // Split-K inside a thread-block cluster (CLUSTER_REDUCE): the K splits of one tile are the CTAs
 // of one cluster, one unit per CTA.  After its K loop every CTA sends the 32 x 32 pieces of its
 // accumulator that other CTAs own straight into their shared memory (distributed shared memory;
-// they land in the stage ring, which is idle by then); after a cluster barrier every CTA adds
-// the pieces it owns in split order, applies the epilogue and stores them.  No partial ever
+// they land in the stage ring, which is idle by then) and counts them in on the receiving warp's
+// mbarrier; every CTA adds the pieces it owns in split order, applies the epilogue and stores them.  No partial ever
 // goes to global memory and there is no second kernel.
 #pragma once
 #include <cuda.h>
@@ -709,22 +710,41 @@ __device__ __forceinline__ bool umma_cluster_epilogue(const UmmaParams& p, const
 // eight different 16-byte bank groups in the loads and in the stores, so neither side has
 // bank conflicts.  This is the paper's software-pipelined pack (Algorithm 3, AMX branch) in the
 // opposite direction: the copies of later stages are in flight while a stage is re-laid.
-template <int COLS>
-__device__ __forceinline__ void vnni_relayout_stage(uint32_t sb, int tw, int lane) {
+// Who does what: with ALT the four warps take turns by stage (warps 6-7 the even stages, 8-9 the
+// odd ones; STAGES is even), two warps sharing the regions of a stage, so that a warp has two stage
+// times for its fixed costs (barrier wait, warp barriers, proxy fence, arrive); without it all four
+// warps work on every stage.  Measured: ALT wins where a stage has two regions (64 columns per CTA:
+// the other scheme leaves two warps idle) and in the pair kernel (+4.5 % on 8-bit 8192^3), and
+// loses on single CTAs with four or more regions per stage (8-bit 512 x 4096 x 4096: 19.0 against
+// 17.5 us), where the short stage time makes the longer per-stage latency count.
+template <int COLS, bool PAIR>
+__host__ __device__ constexpr bool vnni_alt() { return COLS / 32 == 2 || PAIR; }
+
+template <int COLS, int WARPS>
+__device__ __forceinline__ void vnni_relayout_stage(uint32_t sb, int first, int lane) {
+    // This warp's regions of the stage: first, first + WARPS, ...  Regions go two at a time: all
+    // loads of both, one warp barrier, all stores.
     // block (q, nq): pair rows 16h + 4q .. + 3 (h = 0, 1), columns 4nq .. 4nq + 3
+    constexpr int REGIONS = COLS / 32;
+    constexpr int MINE = (REGIONS + WARPS - 1) / WARPS;
+    if (first >= REGIONS) return;           // 64 columns shared by four warps: two have nothing to move
     const uint32_t l0 = lane & 1, l1 = (lane >> 1) & 1, l2 = (lane >> 2) & 1, l3 = (lane >> 3) & 1, l4 = lane >> 4;
     const uint32_t q = l2 * 2 + l1;
     const uint32_t nq = l3 * 4 + (l2 ^ l4) * 2 + l0;
 #pragma unroll
-    for (int j = tw; j < COLS / 32; j += 4) {
-        const uint32_t rb = sb + j * 4096;
-        uint32_t w[2][4][4];
+    for (int b = 0; b < MINE; b += 2) {
+        const bool two = b + 1 < MINE;      // compile-time after unrolling
+        const uint32_t rb0 = sb + (first + WARPS * b) * 4096;
+        const uint32_t rb1 = rb0 + WARPS * 4096;
+        uint32_t w0[2][4][4], w1[2][4][4];
 #pragma unroll
         for (int h = 0; h < 2; ++h)
 #pragma unroll
             for (int r = 0; r < 4; ++r) {
                 const uint32_t R = 16 * h + 4 * q + r;
-                ld_shared_v4(rb + R * 128 + ((nq ^ (R & 7)) << 4), w[h][r]);
+                const uint32_t off = R * 128 + ((nq ^ (R & 7)) << 4);
+                ld_shared_v4(rb0 + off, w0[h][r]);
+                if (two) ld_shared_v4(rb1 + off, w1[h][r]);
             }
         __syncwarp();
 #pragma unroll
@@ -732,7 +752,9 @@ __device__ __forceinline__ void vnni_relayout_stage(uint32_t sb, int tw, int lan
 #pragma unroll
             for (int c = 0; c < 4; ++c) {
                 const uint32_t n = 4 * nq + c;
-                st_shared_v4(rb + n * 128 + (((4 * h + q) ^ (n & 7)) << 4), w[h][0][c], w[h][1][c], w[h][2][c], w[h][3][c]);
+                const uint32_t off = n * 128 + (((4 * h + q) ^ (n & 7)) << 4);
+                st_shared_v4(rb0 + off, w0[h][0][c], w0[h][1][c], w0[h][2][c], w0[h][3][c]);
+                if (two) st_shared_v4(rb1 + off, w1[h][0][c], w1[h][1][c], w1[h][2][c], w1[h][3][c]);
             }
     }
 }
@@ -770,8 +792,10 @@ umma_bf16_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_consta
         // one barrier per lane: full[STAGES], empty[STAGES], tmem_full[2], tmem_empty[2] (and raw[STAGES])
         constexpr int NB = 2 * STAGES + 4;
         static_assert(NB <= 32, "one barrier per lane");
+        static_assert(!B_VNNI || STAGES % 2 == 0, "the re-layout warps take alternate stages");
         if (lane < NB)
-            mbar_init(bar_base + 8u * lane, lane < STAGES ? (B_VNNI ? 1 + 4 : 1) : lane < 2 * STAGES + 2 ? 1 : 128);
+            mbar_init(bar_base + 8u * lane, lane < STAGES ? (B_VNNI ? 1 + (vnni_alt<BN, false>() ? 2 : 4) : 1)
+                                                          : lane < 2 * STAGES + 2 ? 1 : 128);
         if (B_VNNI && lane < STAGES) mbar_init(raw_bar(lane), 1);
         if (CLUSTER_REDUCE && lane >= 24) mbar_init(recv_bar0 + 8u * (lane - 24), 1);   // one per epilogue warp
         if (lane == 0) *abort_flag = 0;
@@ -963,6 +987,7 @@ umma_bf16_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_consta
         if (set == 1 && B_VNNI) {
             // -------------------------------------------- VNNI re-layout
             const int tw = warp - 6;
+            constexpr bool ALT = vnni_alt<BN, false>();
             int stage = 0;
             uint32_t phase = 0;
             bool ok = true;
@@ -972,15 +997,17 @@ umma_bf16_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_consta
                 const int kb0 = split * p.kb_per_split;
                 const int kb1 = min(p.kb_total, kb0 + p.kb_per_split);
                 for (int kb = kb0; kb < kb1; ++kb) {
-                    if (!mbar_wait(raw_bar(stage), phase, abort_flag)) {
-                        if (lane == 0) give_up(0x500u + stage);
-                        ok = false;
-                        break;
+                    if (!ALT || (stage & 1) == (tw >> 1)) {
+                        if (!mbar_wait(raw_bar(stage), phase, abort_flag)) {
+                            if (lane == 0) give_up(0x500u + stage);
+                            ok = false;
+                            break;
+                        }
+                        vnni_relayout_stage<BN, ALT ? 2 : 4>(smem_base + stage * STAGE + UMMA_A_STAGE_BYTES, ALT ? (tw & 1) : tw, lane);
+                        fence_proxy_async_smem();
+                        __syncwarp();
+                        if (lane == 0) mbar_arrive(full_bar(stage));
                     }
-                    vnni_relayout_stage<BN>(smem_base + stage * STAGE + UMMA_A_STAGE_BYTES, tw, lane);
-                    fence_proxy_async_smem();
-                    __syncwarp();
-                    if (lane == 0) mbar_arrive(full_bar(stage));
                     if (++stage == STAGES) { stage = 0; phase ^= 1u; }
                 }
             }

@@ -78,11 +78,12 @@ umma_bf16_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_c
 
     if (warp == 0) {
         // one barrier per lane: full[STAGES], empty[STAGES], tmem_full[2], tmem_empty[2] (and raw[STAGES]).
-        // full[]: the leader's producer (+ 4 re-layout warps per CTA); tmem_empty[]: the epilogue threads of both CTAs
+        // full[]: the leader's producer (+ the 2 re-layout warps per CTA whose turn the stage is); tmem_empty[]: the epilogue threads of both CTAs
         constexpr int NB = 2 * STAGES + 4;
         static_assert(NB <= 32, "one barrier per lane");
+        static_assert(!B_VNNI || STAGES % 2 == 0, "the re-layout warps take alternate stages");
         if (lane < NB)
-            mbar_init(bar_base + 8u * lane, lane < STAGES ? (B_VNNI ? 1 + 8 : 1) : lane < 2 * STAGES + 2 ? 1 : 256);
+            mbar_init(bar_base + 8u * lane, lane < STAGES ? (B_VNNI ? 1 + 4 : 1) : lane < 2 * STAGES + 2 ? 1 : 256);
         if (B_VNNI && lane < STAGES) mbar_init(raw_bar(lane), 1);
         if (lane == 31) mbar_init(peer_ready_bar, 1);
         if (CLUSTER_REDUCE && lane >= 20 && lane < 28) mbar_init(recv_bar0 + 8u * (lane - 20), 1);   // one per epilogue warp
@@ -326,15 +327,18 @@ umma_bf16_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_c
                 int tile, split, gemm, kb0, kb1, tail;
                 if (!decode(unit, tile, split, gemm, kb0, kb1, tail)) continue;
                 for (int kb = kb0; kb < kb1; ++kb) {
-                    if (!mbar_wait(raw_bar(stage), phase, abort_flag)) {
-                        if (lane == 0) give_up(0x500u + stage);
-                        ok = false;
-                        break;
+                    // even stages: warps 6 and 7, odd stages: warps 8 and 9 (STAGES is even)
+                    if ((stage & 1) == (tw >> 1)) {
+                        if (!mbar_wait(raw_bar(stage), phase, abort_flag)) {
+                            if (lane == 0) give_up(0x500u + stage);
+                            ok = false;
+                            break;
+                        }
+                        vnni_relayout_stage<HALF, 2>(smem_base + stage * STAGE + UMMA_A_STAGE_BYTES, tw & 1, lane);
+                        fence_proxy_async_smem();
+                        __syncwarp();
+                        if (lane == 0) mbar_arrive_cluster_cta_release(lead_full0 + 8u * stage);
                     }
-                    vnni_relayout_stage<HALF>(smem_base + stage * STAGE + UMMA_A_STAGE_BYTES, tw, lane);
-                    fence_proxy_async_smem();
-                    __syncwarp();
-                    if (lane == 0) mbar_arrive_cluster_cta_release(lead_full0 + 8u * stage);
                     if (++stage == STAGES) { stage = 0; phase ^= 1u; }
                 }
             }
