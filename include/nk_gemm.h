@@ -219,13 +219,15 @@ nk_status_t nk_gemm_run_host(nk_gemm_t plan, const void* hA, const void* hB, con
                              size_t workspace_bytes, void* cuda_stream);
 
 /*
- * Synchronise the plan's device and read the library's device status word.
+ * Synchronise the plan's device and read the plan's device status word.
  * Every wait inside the kernels (on a TMA or MMA completion barrier) is
  * bounded; a wait that runs out records itself in that word, the kernel drains
  * and exits, and this call returns NK_ERR_TIMEOUT once (the word is cleared;
  * results of the affected run are undefined).  NK_OK otherwise.  The word is a
- * small static device variable of the library, one per device, shared by all
- * plans on that device.
+ * slot of a static device table of the library (1024 slots per device, taken
+ * round robin at nk_gemm_create and cleared there; nothing is allocated): a
+ * plan reports the waits of its own kernels, unless more than 1024 plans were
+ * created on the device since it was.
  */
 nk_status_t nk_gemm_check(nk_gemm_t plan);
 

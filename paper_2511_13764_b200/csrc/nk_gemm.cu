@@ -18,12 +18,18 @@
 #include "umma_bf16.cuh"
 #include "umma_bf16_pair.cuh"
 #include "umma_swap.cuh"
+#include <atomic>
 
 namespace nk {
 
-// One status word per device (the module is instantiated on every device that
-// loads the library).  Kernels receive its device address as a parameter.
-__device__ unsigned int g_status_word[4];
+// Status words, a static table per device (the module is instantiated on every device that
+// loads the library).  A plan takes the next slot of the table when it is created (round robin:
+// two plans share a word only when more than NK_STATUS_SLOTS plans were created in between), so a
+// wait that ran out is reported by the plan whose kernel it was.  Kernels receive the slot's
+// device address as a parameter; nothing is allocated.
+constexpr unsigned NK_STATUS_SLOTS = 1024;
+__device__ unsigned int g_status_word[NK_STATUS_SLOTS];
+static std::atomic<unsigned> g_next_status_slot{0};
 
 enum Variant { V_NAIVE = 0, V_SIMT = 1, V_UMMA = 2, V_SKINNY = 3, V_SPLIT3 = 4, V_SMALL = 5, V_SWAP = 6 };
 
@@ -866,7 +872,12 @@ nk_status_t nk_gemm_create(const nk_gemm_desc_t* desc, nk_gemm_t* out) {
     if (guard.err != cudaSuccess) { delete p; return NK_ERR_DEVICE; }
     void* sym = nullptr;
     if (cudaGetSymbolAddress(&sym, g_status_word) != cudaSuccess) { delete p; return NK_ERR_CUDA; }
-    p->status_dev = static_cast<unsigned int*>(sym);
+    p->status_dev = static_cast<unsigned int*>(sym) + (g_next_status_slot.fetch_add(1) % NK_STATUS_SLOTS);
+    {
+        // the slot may carry the word of a plan that was destroyed without a check
+        const unsigned int z = 0;
+        if (cudaMemcpy(p->status_dev, &z, sizeof(z), cudaMemcpyHostToDevice) != cudaSuccess) { delete p; return NK_ERR_CUDA; }
+    }
 
     if (d.in_dtype == NK_F32 && (d.flags & NK_FLAG_F32_TENSOR) && force != NK_FLAG_KERNEL_NAIVE) {
         // x = hi + mid + lo in BF16 (to 2^-27 of x); A.B = sum of the nine cross terms, of which the six
@@ -884,6 +895,7 @@ nk_status_t nk_gemm_create(const nk_gemm_desc_t* desc, nk_gemm_t* out) {
         nk_gemm_t inner = nullptr;
         const nk_status_t is = nk_gemm_create(&id, &inner);
         if (is != NK_OK) { delete p; return is; }
+        inner->status_dev = p->status_dev;   // the plan that the caller holds reports for its inner plan
         inner->bias_f32 = true;
         inner->item_remap = true;
         inner->item_map_a = 0x001102u;   // items 0..5: planes 2 0 1 1 0 0 (0 = hi)
@@ -1343,6 +1355,7 @@ nk_status_t nk_gemm_run_host(nk_gemm_t p, const void* hA, const void* hB, const 
             cd.flags = (d.flags & ~(0xFFu << NK_FLAG_SPLITK_SHIFT)) | (1u << NK_FLAG_SPLITK_SHIFT) | NK_FLAG_NO_TAIL_SPLIT;
             nk_gemm_t cp = nullptr;
             nk_status_t cs = nk_gemm_create(&cd, &cp);
+            if (cs == NK_OK) cp->status_dev = p->status_dev;   // the caller's plan reports for its chunk plan
             if (cs == NK_OK && nk_gemm_workspace_bytes(cp) == 0) {
                 bool ok = cudaStreamCreateWithFlags(&p->h2d_stream, cudaStreamNonBlocking) == cudaSuccess &&
                           cudaStreamCreateWithFlags(&p->d2h_stream, cudaStreamNonBlocking) == cudaSuccess &&

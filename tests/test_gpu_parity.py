@@ -300,6 +300,20 @@ def test_bounded_wait_reports_timeout_and_context_survives():
     check_against_oracle(w, got, A, B, bias, exact=True)
 
 
+def test_a_timeout_is_reported_by_the_plan_it_happened_in():
+    """Every plan has a status word of its own: a wait that ran out in one plan's kernel leaves the
+    check of another plan (created before or after it) clean."""
+    w = W("whose_timeout", 128, 128, 128, "bf16", integer=True)
+    before, plan, after = nk.plan_for(w), nk.plan_for(w), nk.plan_for(w)
+    plan.selftest_timeout(stream=torch.cuda.current_stream().cuda_stream)
+    before.check()
+    after.check()
+    with pytest.raises(nk.NkError) as e:
+        plan.check()
+    assert e.value.status == 7
+    plan.check()
+
+
 @pytest.mark.parametrize("bn", [3, 4])
 @pytest.mark.parametrize("out_dtype,epi,splits", [("f32", "none", 2), ("bf16", "bias_relu", 3), ("f32", "bias_relu", 4)])
 def test_pair_tail_wave_split(out_dtype, epi, splits, bn):
