@@ -559,8 +559,7 @@ static cudaError_t launch_umma(nk_gemm_s* p, const UmmaParams& up, int grid, cud
 template <typename Kernel>
 static cudaError_t launch_clustered(Kernel kernel, nk_gemm_s* p, const UmmaParams& up, int ctas, int cluster, int threads,
                                     int smem, cudaStream_t st, int* max_clusters) {
-    cudaLaunchConfig_t cfg;
-    memset(&cfg, 0, sizeof(cfg));
+    cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3(static_cast<unsigned>(max_clusters ? cluster : ctas));
     cfg.blockDim = dim3(static_cast<unsigned>(threads));
     cfg.dynamicSmemBytes = static_cast<size_t>(smem);
@@ -639,8 +638,7 @@ static int max_clusters_for(bool pair, int bn, bool vnni, int splits, int kind) 
 
 template <int BN, int STAGES, bool VNNI, int KIND = 0>
 static cudaError_t launch_pair_t(nk_gemm_s* p, const UmmaParams& up, int pairs, cudaStream_t st) {
-    cudaLaunchConfig_t cfg;
-    memset(&cfg, 0, sizeof(cfg));
+    cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3(static_cast<unsigned>(2 * pairs));
     cfg.blockDim = dim3(UMMA_THREADS);
     cfg.dynamicSmemBytes = pair_smem_bytes(BN, STAGES);
@@ -671,8 +669,7 @@ static cudaError_t launch_pair(nk_gemm_s* p, const UmmaParams& up, int pairs, cu
 
 template <int BN, int STAGES, bool VNNI>
 static cudaError_t pair_occupancy(int* out) {
-    cudaLaunchConfig_t cfg;
-    memset(&cfg, 0, sizeof(cfg));
+    cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3(2);
     cfg.blockDim = dim3(UMMA_THREADS);
     cfg.dynamicSmemBytes = pair_smem_bytes(BN, STAGES);
@@ -1210,8 +1207,7 @@ nk_status_t nk_gemm_run(nk_gemm_t p, const void* A, const void* B, const void* b
         sp.C = C;
         sp.partial = partial;
         sp.status = p->status_dev;
-        cudaLaunchConfig_t cfg;
-        memset(&cfg, 0, sizeof(cfg));
+        cudaLaunchConfig_t cfg = {};
         cfg.gridDim = dim3(static_cast<unsigned>(sp.tiles_n * p->splits));
         cfg.blockDim = dim3(192);
         cfg.dynamicSmemBytes = static_cast<size_t>(swap_smem_bytes(p->swap_mp, swap_stages(p->swap_mp)));
