@@ -199,6 +199,24 @@ def test_umma_splitk_cluster_reduce_equals_reduce_kernel(shape, splits, out_dtyp
     check_against_oracle(w, c_one, A, B, bias)
 
 
+@pytest.mark.parametrize("shape,epi,out_dtype", [((256, 4096, 4096), "bias_relu", "bf16"), ((512, 4096, 4096), "bias_relu", "bf16"),
+                                                 ((128, 4096, 4096), "none", "f32"), ((512, 1024, 1024), "bias_relu", "bf16")],
+                         ids=["c3", "mlp4096", "128rows", "mlp1024"])
+def test_cluster_exchange_gives_the_same_bits_every_time(shape, epi, out_dtype):
+    """The pieces of a cluster split-K travel as asynchronous remote stores and every receiving warp waits
+    on a barrier of its own: whatever order they land in, a full-GPU launch (every SM in some cluster) must
+    give the same bits on every one of many back-to-back runs, and those bits are within the bound."""
+    M, N, K = shape
+    w = W("exchange", M, N, K, "bf16", out_dtype, epilogue=epi, seed=29)
+    A, B, bias = w.make()
+    first, plan = run_plan(w, A, B, bias)
+    assert "_cluster" in plan.kernel_name and plan.launches_per_run == 1, plan.kernel_name
+    check_against_oracle(w, first, A, B, bias, rows=nk_inputs.stratified_rows(3, M, 32))
+    for _ in range(60):
+        again, _ = run_plan(w, A, B, bias, plan=plan)
+        assert np.array_equal(again, first)
+
+
 @pytest.mark.parametrize("mode", ["single", "pair"])
 @pytest.mark.parametrize("splits", [2, 4])
 def test_umma_splitk_cluster_blocked_operands(splits, mode):
